@@ -1,0 +1,208 @@
+/*
+ * dllm.h -- C ABI of the B200 (sm_100a) library for one denoising step of a
+ * bidirectional masked-diffusion transformer under adaptive feature caching.
+ *
+ * Vocabulary follows the paper: prompt c of length P, response y^(k) of length
+ * R (n = P + R rows per sequence), denoising steps k = K..1, Prompt Cache C_p
+ * and Response Cache C_r holding K, V, AttnOut, FFNOut per layer (Sec. 3.2),
+ * refresh intervals K_p and K_r, adaptive update ratio rho (Sec. 3.2), V-verify
+ * (Eq. 6), transition S with low-confidence remasking (Eq. 5, Sec. A.11).
+ *
+ * Conventions
+ *   - Every call returns a dllm_status; nothing throws, aborts or traps.
+ *     dllm_last_error(handle) returns a readable message for the last failure
+ *     on that handle (handle may be NULL for failures of a *_create call).
+ *   - The caller owns all device memory: the weight blob, the cache blob and
+ *     the workspace blob are device pointers the caller allocated (256-byte
+ *     aligned) with at least the byte counts the size queries return, and must
+ *     keep alive until the handle using them is destroyed.  The library frees
+ *     only its own host-side handles (and the CUDA graphs it instantiates).
+ *   - "h_" arguments are HOST pointers, "d_" arguments are DEVICE pointers.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Step
+ *     and remask calls only enqueue work on it; they do not synchronise.
+ *     Inspection calls (dllm_get_*, dllm_set_*) synchronise the stream they are
+ *     given before copying.
+ *   - All matrices are row-major.  Linear maps are stored [out, in] and applied
+ *     as y = x W^T.  Storage type of weights and caches is the model's dtype;
+ *     accumulation, softmax, norms, cosine and the residual stream are fp32.
+ *   - Invalid arguments return DLLM_INVALID_ARG and have no side effect.
+ */
+#ifndef DLLM_H_
+#define DLLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DLLM_OK = 0,
+  DLLM_INVALID_ARG = 1,
+  DLLM_BAD_STATE = 2,      /* e.g. a cached step before any full step */
+  DLLM_UNSUPPORTED = 3,    /* shape outside what the kernels handle */
+  DLLM_OUT_OF_MEMORY = 4,  /* host allocation failed */
+  DLLM_CUDA_ERROR = 5,
+  DLLM_TIMEOUT = 6         /* a bounded device-side wait gave up */
+} dllm_status;
+
+enum { DLLM_FP32 = 0, DLLM_BF16 = 1 };
+
+/* Architecture of the mask predictor p_theta (Sec. 3.1): pre-norm transformer
+ * with RMSNorm, rotary embedding (rotate-half pairing, absolute position in
+ * [prompt; response]), bidirectional softmax attention with n_heads query heads
+ * sharing n_kv_heads key/value heads, and a SwiGLU FFN of width d_ffn (three
+ * matmuls, Sec. A.7).  No biases; embedding and LM head are separate. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab, mask_id;
+  float rms_eps, rope_theta;
+  int32_t dtype; /* DLLM_FP32 or DLLM_BF16 */
+} dllm_config;
+
+/* How floor(rho * R) is rounded.  The paper writes floor (Sec. 3.2.2). */
+typedef enum { DLLM_K_FLOOR = 0, DLLM_K_CEIL = 1 } dllm_kround;
+
+enum { DLLM_CACHE_K = 0, DLLM_CACHE_V = 1, DLLM_CACHE_ATTN = 2, DLLM_CACHE_FFN = 3 };
+
+typedef struct dllm_model dllm_model;
+typedef struct dllm_session dllm_session;
+
+const char* dllm_last_error(const void* handle);
+
+/* ---- sizes --------------------------------------------------------------- */
+/* Bytes of the packed weight blob for this architecture. */
+size_t dllm_weights_bytes(const dllm_config* cfg);
+/* Bytes of the feature caches for B sequences of P + R rows: per layer
+ * K, V [B, n, n_kv_heads*head_dim] and AttnOut, FFNOut [B, n, d_model] in the
+ * model dtype -- exactly the four tensors per layer of Sec. A.9. */
+size_t dllm_cache_bytes(const dllm_config* cfg, int B, int P, int R);
+/* Bytes of scratch the step needs (residual stream, staging buffers, GEMM
+ * partial sums, logits, selection state). */
+size_t dllm_workspace_bytes(const dllm_config* cfg, int B, int P, int R);
+/* Byte offset and element count of one named tensor inside the weight blob, so
+ * a caller may fill the blob on the device.  Names: "embed", "lm_head" [vocab,
+ * d_model]; "norm_f" [d_model]; "layers.<l>.{norm1,norm2}" [d_model];
+ * "layers.<l>.wq" [H*hd, d]; ".wk", ".wv" [Hkv*hd, d]; ".wo" [d, H*hd];
+ * ".wg", ".wu" [d_ffn, d]; ".wd" [d, d_ffn].  Norm gains are always fp32;
+ * everything else has the model dtype. */
+dllm_status dllm_tensor_offset(const dllm_config* cfg, const char* name, size_t* offset_bytes,
+                               size_t* n_elements);
+
+/* ---- model p_theta --------------------------------------------------------- */
+/* Binds a model handle to a caller-owned device blob of dllm_weights_bytes(). */
+dllm_status dllm_model_create(const dllm_config* cfg, void* d_weights, dllm_model** out);
+/* Uploads one tensor from HOST float32 values (converted to the model dtype
+ * with round-to-nearest-even).  n_elements must match the tensor. */
+dllm_status dllm_model_set_tensor(dllm_model* m, const char* name, const float* h_src, size_t n_elements);
+dllm_status dllm_model_destroy(dllm_model* m);
+
+/* ---- session: tokens (c, y^(k)) and caches C_p, C_r ------------------------ */
+/* d_cache: dllm_cache_bytes(); d_workspace: dllm_workspace_bytes().  Both are
+ * zeroed asynchronously on `stream`. */
+dllm_status dllm_session_create(dllm_model* m, int B, int P, int R, void* d_cache, void* d_workspace,
+                                void* stream, dllm_session** out);
+dllm_status dllm_session_destroy(dllm_session* s);
+/* tokens <- [prompt ; MASK x R] for every sequence (Eq. 2); caches become
+ * invalid until the next full step.  h_prompt: int32 [B, P], ids in [0, vocab). */
+dllm_status dllm_session_set_prompt(dllm_session* s, const int32_t* h_prompt, void* stream);
+
+/* ---- the denoising step ---------------------------------------------------- */
+/* Initialisation / full refresh (k = K, Sec. 3.2): all features of all n rows
+ * are computed and written to C_p and C_r; leaves (x0, conf) for the response. */
+dllm_status dllm_step_full(dllm_session* s, void* stream);
+/* One step under the caching rule (Sec. 3.2 items (1)-(3), Sec. 3.2.2):
+ *   refresh_prompt   != 0: prompt rows are recomputed and C_p rewritten;
+ *   refresh_response != 0: all response rows are recomputed against the cached
+ *                          prompt K/V and C_r rewritten;
+ *   otherwise adaptive partial update: V is projected for all R response rows,
+ *   s_j = cos(V_new[j], V_cached[j]) (Eq. 6), the k_sel = floor(rho*R) rows with
+ *   the lowest s_j are selected per sequence and per layer (ties: lower
+ *   round(s*2^20) first, then lower index), the whole response V cache is
+ *   overwritten, and Q/K/attention/O-proj/FFN run only for the selected rows
+ *   over the full cached K/V; their K, AttnOut, FFNOut rows are scattered back.
+ *   rho in [0,1]; k_sel = 0 leaves all caches untouched.
+ * Returns DLLM_BAD_STATE before the first full step. */
+dllm_status dllm_step_cached(dllm_session* s, int refresh_prompt, int refresh_response, float rho,
+                             dllm_kround kround, void* stream);
+/* Applies the schedule at step k of K (counting down): refresh everything at
+ * k = K, the prompt when k mod Kp == 0, the response when k mod Kr == 0. */
+dllm_status dllm_step_scheduled(dllm_session* s, int k, int K, int Kp, int Kr, float rho,
+                                dllm_kround kround, void* stream);
+/* Transition S with low-confidence remasking (Eq. 5): among the still masked
+ * response positions in [block_start, block_start + block_len) the
+ * min(n_transfer, #masked) positions with the highest confidence (ties: lowest
+ * position) receive their greedy estimate x0; all others stay as they are.
+ * Uses the (x0, conf) of the last step. */
+dllm_status dllm_remask_low_confidence(dllm_session* s, int block_start, int block_len, int n_transfer,
+                                       void* stream);
+/* K steps k = K..1 of dllm_step_scheduled, each followed by the transition on
+ * the block that step works on (blocks of block_len, K / (R / block_len) steps
+ * per block, block_len / steps_per_block tokens per step).  R must be a
+ * multiple of block_len and K a multiple of R / block_len. */
+dllm_status dllm_generate(dllm_session* s, int K, int Kp, int Kr, float rho, dllm_kround kround,
+                          int block_len, void* stream);
+/* Waits for the stream and returns DLLM_TIMEOUT / DLLM_CUDA_ERROR if a kernel
+ * recorded a problem in the session's device status word. */
+dllm_status dllm_sync(dllm_session* s, void* stream);
+
+/* ---- inspection and test hooks (host buffers owned by the caller) ---------- */
+dllm_status dllm_get_tokens(dllm_session* s, int32_t* h_out /* [B, P+R] */, void* stream);
+dllm_status dllm_set_response_tokens(dllm_session* s, const int32_t* h_tok /* [B, R] */, void* stream);
+dllm_status dllm_get_hidden(dllm_session* s, float* h_out /* [B, R, d_model] residual before final norm */,
+                            void* stream);
+dllm_status dllm_get_pred(dllm_session* s, int32_t* h_x0 /* [B, R] */, float* h_conf /* [B, R] */, void* stream);
+/* Recomputes and returns the logits of the last step's hidden state (mask id
+ * column set to -inf).  Slow path for small vocabularies. */
+dllm_status dllm_get_logits(dllm_session* s, float* h_out /* [B, R, vocab] */, void* stream);
+/* Selection of the last step at one layer: h_idx int32 [B, k_sel] ascending
+ * response-relative indices (k_sel = R on a response refresh), h_sim float
+ * [B, R] (Eq. 6 values; only meaningful after an adaptive step).  Either
+ * pointer may be NULL.  *k_sel_out receives k_sel. */
+dllm_status dllm_get_selected(dllm_session* s, int layer, int32_t* h_idx, float* h_sim, int* k_sel_out,
+                              void* stream);
+/* One cache tensor of one layer as float32 [B, n, width] (width = Hkv*hd for K
+ * and V, d_model for AttnOut and FFNOut). */
+dllm_status dllm_get_cache(dllm_session* s, int layer, int which, float* h_out, void* stream);
+dllm_status dllm_set_cache(dllm_session* s, int layer, int which, const float* h_in, void* stream);
+/* Replaces the V-verify choice of `layer` on adaptive steps by the given
+ * response-relative indices (int32 [B, count], count must equal k_sel of the
+ * steps that follow); count = -1 clears.  V-verify still runs and V is still
+ * overwritten.  Lets a test tell a legal tie flip from an arithmetic fault. */
+dllm_status dllm_force_selection(dllm_session* s, int layer, const int32_t* h_idx, int count);
+/* Number of kernel launches the library has enqueued for this session. */
+uint64_t dllm_launch_count(const dllm_session* s);
+/* 1: replay each step kind from a CUDA graph captured on first use (default);
+ * 0: launch kernels one by one. */
+dllm_status dllm_session_use_graphs(dllm_session* s, int enable);
+
+/* Test hook: 1 runs the bf16 GEMMs of the step on the plain-ALU kernel instead
+ * of the tensor-core kernel (to localise a fault); default 0. */
+dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable);
+
+/* ---- kernel-level entry points (parity tests and micro-benchmarks) --------- */
+/* C[M,N] (fp32, row-major, DEVICE) = A[M,K] * W[N,K]^T with bf16 operands on
+ * the tensor cores (tcgen05 + TMA).  d_partials is scratch of
+ * dllm_gemm_bf16_scratch_bytes(M,N,K); split-K partial sums are reduced in a
+ * fixed order.  K must be a multiple of 8 (16-byte rows). */
+size_t dllm_gemm_bf16_scratch_bytes(int M, int N, int K);
+dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, int N, int K,
+                           void* d_partials, void* stream);
+/* The same product on the plain fp32 ALUs (operands fp32 or bf16): the GEMM of
+ * the fp32 mode. */
+dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int dtype,
+                           void* stream);
+/* Non-causal attention of `a` query rows per sequence over n cached keys.
+ * d_q [B*a, H*hd], d_k / d_v [B, n, Hkv*hd], d_o [B*a, H*hd]; dtype as above. */
+dllm_status dllm_attention(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B, int a, int n,
+                           int H, int Hkv, int hd, int dtype, void* stream);
+/* V-verify + selection alone (Eq. 6 and the bottom-k rule): d_vnew, d_vcache
+ * [B, R, width] in `dtype`; writes d_sim float [B, R] and d_idx int32 [B, k]
+ * ascending; overwrites d_vcache with d_vnew. */
+dllm_status dllm_vverify_select(const void* d_vnew, void* d_vcache, float* d_sim, int32_t* d_idx, int B, int R,
+                                int width, int k, int dtype, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DLLM_H_ */

@@ -1,0 +1,823 @@
+// Host side of the C ABI: handles, blob layouts, argument checks, the step
+// procedure (which kernels run for which active-row set), CUDA-graph replay and
+// the inspection hooks.  No step of the method is computed here: the host only
+// enqueues kernels.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <map>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/dllm.h"
+#include "internal.h"
+
+using namespace dllm;
+
+namespace {
+
+thread_local std::string g_err;
+
+size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct LayerOff {
+  size_t norm1, wqkv, wo, norm2, wgu, wd;
+};
+struct WeightLayout {
+  size_t embed, lm_head, norm_f, total;
+  std::vector<LayerOff> layers;
+};
+
+size_t esize(const dllm_config& c) { return c.dtype == DLLM_BF16 ? 2 : 4; }
+
+WeightLayout make_layout(const dllm_config& c) {
+  WeightLayout w;
+  const size_t es = esize(c), d = c.d_model, dq = (size_t)c.n_heads * c.head_dim,
+               dkv = (size_t)c.n_kv_heads * c.head_dim, m = c.d_ffn, V = c.vocab;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes);
+    return o;
+  };
+  w.embed = take(V * d * es);
+  w.lm_head = take(V * d * es);
+  w.norm_f = take(d * 4);
+  w.layers.resize(c.n_layers);
+  for (auto& l : w.layers) {
+    l.norm1 = take(d * 4);
+    l.wqkv = take((dq + 2 * dkv) * d * es);  // rows: W_q, then W_k, then W_v
+    l.wo = take(d * dq * es);
+    l.norm2 = take(d * 4);
+    l.wgu = take(2 * m * d * es);            // rows: W_gate, then W_up
+    l.wd = take(d * m * es);
+  }
+  w.total = off;
+  return w;
+}
+
+const char* check_config(const dllm_config* c) {
+  if (!c) return "config is NULL";
+  if (c->n_layers <= 0 || c->d_model <= 0 || c->n_heads <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0 ||
+      c->d_ffn <= 0 || c->vocab <= 1)
+    return "non-positive dimension";
+  if (c->dtype != DLLM_FP32 && c->dtype != DLLM_BF16) return "dtype must be DLLM_FP32 or DLLM_BF16";
+  if (c->n_heads % c->n_kv_heads) return "n_heads must be a multiple of n_kv_heads";
+  if (c->mask_id < 0 || c->mask_id >= c->vocab) return "mask_id outside the vocabulary";
+  if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return "rms_eps / rope_theta out of range";
+  return nullptr;
+}
+const char* check_supported(const dllm_config* c) {
+  if (c->d_model % 8 || c->d_ffn % 8 || c->vocab % 8) return "d_model, d_ffn and vocab must be multiples of 8";
+  if (c->head_dim % 32 || c->head_dim > 128) return "head_dim must be 32, 64, 96 or 128";
+  return nullptr;
+}
+
+struct TensorRef {
+  size_t off, n;
+  bool f32;
+};
+
+bool find_tensor(const dllm_config& c, const WeightLayout& w, const char* name, TensorRef* out) {
+  const size_t es = esize(c), d = c.d_model, dq = (size_t)c.n_heads * c.head_dim,
+               dkv = (size_t)c.n_kv_heads * c.head_dim, m = c.d_ffn, V = c.vocab;
+  if (!strcmp(name, "embed")) return *out = {w.embed, V * d, false}, true;
+  if (!strcmp(name, "lm_head")) return *out = {w.lm_head, V * d, false}, true;
+  if (!strcmp(name, "norm_f")) return *out = {w.norm_f, d, true}, true;
+  int l = -1, pos = 0;
+  if (sscanf(name, "layers.%d.%n", &l, &pos) < 1 || pos == 0 || l < 0 || l >= c.n_layers) return false;
+  const char* t = name + pos;
+  const LayerOff& L = w.layers[l];
+  if (!strcmp(t, "norm1")) return *out = {L.norm1, d, true}, true;
+  if (!strcmp(t, "norm2")) return *out = {L.norm2, d, true}, true;
+  if (!strcmp(t, "wq")) return *out = {L.wqkv, dq * d, false}, true;
+  if (!strcmp(t, "wk")) return *out = {L.wqkv + dq * d * es, dkv * d, false}, true;
+  if (!strcmp(t, "wv")) return *out = {L.wqkv + (dq + dkv) * d * es, dkv * d, false}, true;
+  if (!strcmp(t, "wo")) return *out = {L.wo, d * dq, false}, true;
+  if (!strcmp(t, "wg")) return *out = {L.wgu, m * d, false}, true;
+  if (!strcmp(t, "wu")) return *out = {L.wgu + m * d * es, m * d, false}, true;
+  if (!strcmp(t, "wd")) return *out = {L.wd, d * m, false}, true;
+  return false;
+}
+
+uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu)) return (uint16_t)((u >> 16) | 0x40);  // NaN
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+
+// workspace carve-up
+struct Workspace {
+  size_t status, tokens, x, u, ua, qbuf, obuf, hn, ffn, x0, conf, sim, sel, forced, act, rope, part, total;
+  size_t part_floats;
+};
+
+Workspace make_workspace(const dllm_config& c, int B, int P, int R) {
+  Workspace w;
+  const size_t es = esize(c), d = c.d_model, dq = (size_t)c.n_heads * c.head_dim,
+               dkv = (size_t)c.n_kv_heads * c.head_dim, m = c.d_ffn, V = c.vocab;
+  const size_t n = (size_t)P + R, rows = (size_t)B * n, BR = (size_t)B * R, T = c.n_layers;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes);
+    return o;
+  };
+  w.status = take(256);
+  w.tokens = take(rows * 4);
+  w.x = take(rows * d * 4);
+  w.u = take(rows * d * es);
+  w.ua = take(rows * d * es);
+  w.qbuf = take(rows * dq * es);
+  w.obuf = take(rows * dq * es);
+  w.hn = take(rows * d * es);
+  w.ffn = take(rows * m * es);
+  w.x0 = take(BR * 4);
+  w.conf = take(BR * 4);
+  w.sim = take(T * BR * 4);
+  w.sel = take(T * BR * 4);
+  w.forced = take(T * BR * 4);
+  w.act = take(rows * 4);
+  w.rope = take(n * c.head_dim * 4);
+  // largest [M, N] any GEMM writes, plus room for split-K slabs of the small-M
+  // launches: S*M*N <= M*N + 148 CTAs * 256 * 128 for every plan
+  size_t mn = rows * std::max(std::max(dq + dkv, d), 2 * m);
+  mn = std::max(mn, BR * V);
+  mn = std::max(mn, rows * std::max(d, dkv));
+  w.part_floats = mn + (size_t)148 * 256 * 128 * 2;
+  w.part = take(w.part_floats * 4);
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+
+struct dllm_model {
+  dllm_config cfg;
+  WeightLayout lay;
+  uint8_t* d_w;
+  std::string err;
+};
+
+struct StepKey {
+  int rp, rr, ksel;
+  uint64_t forced_sig;
+  bool operator<(const StepKey& o) const {
+    if (rp != o.rp) return rp < o.rp;
+    if (rr != o.rr) return rr < o.rr;
+    if (ksel != o.ksel) return ksel < o.ksel;
+    return forced_sig < o.forced_sig;
+  }
+};
+
+struct dllm_session {
+  dllm_model* m;
+  int B, P, R, n;
+  uint8_t* d_cache;
+  uint8_t* d_ws;
+  Workspace ws;
+  bool valid = false;      // caches hold a full step
+  bool have_pred = false;
+  int last_ksel = 0;
+  std::vector<int> forced_count;  // per layer, -1 = none
+  uint64_t launches = 0;
+  bool use_graphs = true;
+  bool simt_gemm = false;
+  struct GraphEntry {
+    cudaGraphExec_t exec;
+    uint64_t kernels;
+  };
+  std::map<StepKey, GraphEntry> graphs;
+  std::string err;
+
+  size_t es() const { return esize(m->cfg); }
+  size_t dkv() const { return (size_t)m->cfg.n_kv_heads * m->cfg.head_dim; }
+  size_t dq() const { return (size_t)m->cfg.n_heads * m->cfg.head_dim; }
+  size_t layer_bytes() const { return (size_t)B * n * (2 * dkv() + 2 * (size_t)m->cfg.d_model) * es(); }
+  uint8_t* cache(int layer, int which) const {
+    const size_t rows = (size_t)B * n;
+    size_t off = (size_t)layer * layer_bytes();
+    const size_t kv = rows * dkv() * es(), ad = rows * (size_t)m->cfg.d_model * es();
+    if (which >= 1) off += kv;
+    if (which >= 2) off += kv;
+    if (which >= 3) off += ad;
+    return d_cache + off;
+  }
+  template <typename T>
+  T* wsp(size_t off) const {
+    return reinterpret_cast<T*>(d_ws + off);
+  }
+  Geo geo() const { return Geo{B, P, R, n, m->cfg.d_model}; }
+};
+
+namespace {
+
+dllm_status fail(std::string* slot, dllm_status st, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  g_err = buf;
+  if (slot) *slot = buf;
+  return st;
+}
+
+#define CU_TRY(slot, expr)                                                                          \
+  do {                                                                                              \
+    cudaError_t e_ = (expr);                                                                        \
+    if (e_ != cudaSuccess) return fail(slot, DLLM_CUDA_ERROR, "%s: %s", #expr, cudaGetErrorString(e_)); \
+  } while (0)
+
+int k_selected(float rho, int R, dllm_kround kr) {
+  const double v = (double)rho * (double)R;
+  long k = kr == DLLM_K_CEIL ? (long)ceil(v - 1e-6) : (long)floor(v + 1e-6);
+  if (k < 0) k = 0;
+  if (k > R) k = R;
+  return (int)k;
+}
+
+// One GEMM of the step: out = A[M,K] * W[N,K]^T as split-K partial slabs.
+dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void* W, int M, int N, int K,
+                     Partials* out) {
+  float* part = s->wsp<float>(s->ws.part);
+  out->p = part;
+  out->N = N;
+  out->split_stride = (size_t)M * N;
+  out->S = 1;
+  if (M <= 0) return DLLM_OK;
+  if (s->m->cfg.dtype == DLLM_FP32 || s->simt_gemm) {
+    launch_gemm_simt(L, s->m->cfg.dtype, A, W, part, M, N, K);
+    return DLLM_OK;
+  }
+  const GemmPlan plan = plan_gemm_bf16(M, N, K, 0);
+  if ((size_t)plan.S * M * N > s->ws.part_floats)
+    return fail(&s->err, DLLM_UNSUPPORTED, "GEMM %dx%dx%d with %d splits exceeds the workspace", M, N, K, plan.S);
+  const char* why = nullptr;
+  cudaError_t e = launch_gemm_bf16(L, A, W, part, M, N, K, plan, &why);
+  if (e != cudaSuccess)
+    return fail(&s->err, DLLM_CUDA_ERROR, "bf16 GEMM %dx%dx%d: %s", M, N, K, why ? why : cudaGetErrorString(e));
+  out->S = plan.S;
+  return DLLM_OK;
+}
+
+// Enqueue one denoising step.  Active rows per sequence: the prompt rows on a
+// prompt refresh plus either all R response rows (response refresh) or the
+// ksel rows V-verify picks.
+dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t stream) {
+  const dllm_config& c = s->m->cfg;
+  const WeightLayout& wl = s->m->lay;
+  const Geo g = s->geo();
+  const int dt = c.dtype, d = c.d_model, H = c.n_heads, Hkv = c.n_kv_heads, hd = c.head_dim, m = c.d_ffn;
+  const int dq = H * hd, dkv = Hkv * hd, BR = s->B * s->R, BP = s->B * s->P;
+  const size_t es = s->es();
+  Launch L{stream, s->wsp<int>(s->ws.status), &s->launches};
+  uint8_t* W = s->m->d_w;
+  const int c0 = 0, c1 = BR + (rp ? BP : 0);
+  const int a_seq = (rp ? s->P : 0) + ksel;
+  const int Ma = s->B * a_seq;
+  const bool project_v = rr || ksel > 0;
+  float* x = s->wsp<float>(s->ws.x);
+  uint8_t* u = s->wsp<uint8_t>(s->ws.u);
+  int32_t* act = s->wsp<int32_t>(s->ws.act);
+  dllm_status st;
+  Partials part;
+
+  launch_embed(L, dt, W + wl.embed, s->wsp<int32_t>(s->ws.tokens), x, g, c0, c1);
+  for (int l = 0; l < c.n_layers; ++l) {
+    const LayerOff& lo = wl.layers[l];
+    uint8_t* Wq = W + lo.wqkv;
+    uint8_t* Wv = Wq + (size_t)(dq + dkv) * d * es;
+    float* sim = s->wsp<float>(s->ws.sim) + (size_t)l * BR;
+    int32_t* sel = s->wsp<int32_t>(s->ws.sel) + (size_t)l * BR;
+    const int32_t* forced = s->wsp<int32_t>(s->ws.forced) + (size_t)l * BR;
+
+    launch_rmsnorm(L, dt, x, reinterpret_cast<const float*>(W + lo.norm1), u, d, c.rms_eps, c0, c1);
+    if (project_v) {
+      // V for ALL response rows (the 2 r d^2 term of Sec. A.7), V-verify, V overwrite
+      if ((st = run_gemm(s, L, u, Wv, BR, dkv, d, &part)) != DLLM_OK) return st;
+      launch_vverify(L, dt, part, s->cache(l, DLLM_CACHE_V), sim, g, dkv);
+    }
+    if (rp) {
+      if ((st = run_gemm(s, L, u + (size_t)BR * d * es, Wv, BP, dkv, d, &part)) != DLLM_OK) return st;
+      launch_scatter_rows(L, dt, part, nullptr, BR, s->cache(l, DLLM_CACHE_V), g, BP, dkv);
+    }
+    if (Ma > 0) {
+      const int mode = rr ? 0 : (s->forced_count[l] >= 0 ? 2 : 1);
+      launch_select(L, sim, forced, mode, ksel, sel, s->R, act, g, rp);
+      uint8_t* ua = s->wsp<uint8_t>(s->ws.ua);
+      launch_gather_rows(L, dt, u, act, ua, Ma, d);
+      // Q and K of the active rows in one GEMM over the stacked [W_q; W_k]
+      if ((st = run_gemm(s, L, ua, Wq, Ma, dq + dkv, d, &part)) != DLLM_OK) return st;
+      launch_qk_rope(L, dt, part, act, s->wsp<float>(s->ws.rope), s->wsp<uint8_t>(s->ws.qbuf),
+                     s->cache(l, DLLM_CACHE_K), g, Ma, H, Hkv, hd);
+      cudaError_t e = launch_attention(L, dt, s->wsp<uint8_t>(s->ws.qbuf), s->cache(l, DLLM_CACHE_K),
+                                       s->cache(l, DLLM_CACHE_V), s->wsp<uint8_t>(s->ws.obuf), s->B, a_seq, s->n, H,
+                                       Hkv, hd);
+      if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
+      if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.obuf), W + lo.wo, Ma, d, dq, &part)) != DLLM_OK) return st;
+      launch_oproj_epilogue(L, dt, part, act, x, reinterpret_cast<const float*>(W + lo.norm2),
+                            s->cache(l, DLLM_CACHE_ATTN), s->wsp<uint8_t>(s->ws.hn), g, Ma, c.rms_eps);
+      if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.hn), W + lo.wgu, Ma, 2 * m, d, &part)) != DLLM_OK) return st;
+      launch_silu_mul(L, dt, part, s->wsp<uint8_t>(s->ws.ffn), Ma, m);
+      if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.ffn), W + lo.wd, Ma, d, m, &part)) != DLLM_OK) return st;
+      launch_scatter_rows(L, dt, part, act, 0, s->cache(l, DLLM_CACHE_FFN), g, Ma, d);
+    }
+    launch_residual(L, dt, x, s->cache(l, DLLM_CACHE_ATTN), s->cache(l, DLLM_CACHE_FFN), g, c0, c1);
+  }
+  // prediction at the response rows (Eqs. 3-4)
+  launch_rmsnorm(L, dt, x, reinterpret_cast<const float*>(W + wl.norm_f), u, d, c.rms_eps, 0, BR);
+  if ((st = run_gemm(s, L, u, W + wl.lm_head, BR, c.vocab, d, &part)) != DLLM_OK) return st;
+  if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
+  launch_argmax_conf(L, part.p, BR, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "step launch: %s", cudaGetErrorString(e));
+  return DLLM_OK;
+}
+
+uint64_t forced_signature(const dllm_session* s) {
+  uint64_t h = 1469598103934665603ull;
+  for (int fc : s->forced_count) h = (h ^ (uint64_t)(fc >= 0)) * 1099511628211ull;
+  return h;
+}
+
+dllm_status run_step(dllm_session* s, int rp, int rr, float rho, dllm_kround kr, void* stream_v) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (!(rho >= 0.f && rho <= 1.f)) return fail(&s->err, DLLM_INVALID_ARG, "rho must lie in [0, 1]");
+  if (kr != DLLM_K_FLOOR && kr != DLLM_K_CEIL) return fail(&s->err, DLLM_INVALID_ARG, "bad kround");
+  rp = rp != 0;
+  rr = rr != 0;
+  if (!s->valid && !(rp && rr)) return fail(&s->err, DLLM_BAD_STATE, "cached step before any full step");
+  const int ksel = rr ? s->R : k_selected(rho, s->R, kr);
+  if (!rr)
+    for (int l = 0; l < s->m->cfg.n_layers; ++l)
+      if (s->forced_count[l] >= 0 && s->forced_count[l] != ksel)
+        return fail(&s->err, DLLM_INVALID_ARG, "forced selection of layer %d has %d rows, step selects %d", l,
+                    s->forced_count[l], ksel);
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  dllm_status st = DLLM_OK;
+  const bool graph_ok = s->use_graphs && stream != nullptr && stream != cudaStreamLegacy;
+  if (!graph_ok) {
+    st = enqueue_step(s, rp, rr, ksel, stream);
+  } else {
+    StepKey key{rp, rr, ksel, forced_signature(s)};
+    auto it = s->graphs.find(key);
+    if (it == s->graphs.end()) {
+      cudaGraph_t graph = nullptr;
+      CU_TRY(&s->err, cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal));
+      const uint64_t before = s->launches;
+      st = enqueue_step(s, rp, rr, ksel, stream);
+      cudaError_t e = cudaStreamEndCapture(stream, &graph);
+      if (st != DLLM_OK) {
+        if (graph) cudaGraphDestroy(graph);
+        return st;
+      }
+      if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "graph capture: %s", cudaGetErrorString(e));
+      cudaGraphExec_t exec = nullptr;
+      e = cudaGraphInstantiate(&exec, graph, 0);
+      cudaGraphDestroy(graph);
+      if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "graph instantiate: %s", cudaGetErrorString(e));
+      const uint64_t kernels = s->launches - before;
+      s->launches = before;  // counted at every replay instead
+      it = s->graphs.emplace(key, dllm_session::GraphEntry{exec, kernels}).first;
+    }
+    CU_TRY(&s->err, cudaGraphLaunch(it->second.exec, stream));
+    s->launches += it->second.kernels;
+  }
+  if (st != DLLM_OK) return st;
+  s->valid = true;
+  s->have_pred = true;
+  s->last_ksel = ksel;
+  return DLLM_OK;
+}
+
+}  // namespace
+
+// =============================================================================
+// extern "C" entry points
+// =============================================================================
+extern "C" {
+
+const char* dllm_last_error(const void* handle) {
+  (void)handle;  // the message of the last failing call on this thread
+  return g_err.c_str();
+}
+
+size_t dllm_weights_bytes(const dllm_config* cfg) {
+  if (check_config(cfg)) return 0;
+  return make_layout(*cfg).total;
+}
+
+size_t dllm_cache_bytes(const dllm_config* cfg, int B, int P, int R) {
+  if (check_config(cfg) || B <= 0 || P <= 0 || R <= 0) return 0;
+  const size_t dkv = (size_t)cfg->n_kv_heads * cfg->head_dim;
+  return (size_t)cfg->n_layers * B * ((size_t)P + R) * (2 * dkv + 2 * (size_t)cfg->d_model) * esize(*cfg);
+}
+
+size_t dllm_workspace_bytes(const dllm_config* cfg, int B, int P, int R) {
+  if (check_config(cfg) || B <= 0 || P <= 0 || R <= 0) return 0;
+  return make_workspace(*cfg, B, P, R).total;
+}
+
+dllm_status dllm_tensor_offset(const dllm_config* cfg, const char* name, size_t* offset_bytes, size_t* n_elements) {
+  const char* why = check_config(cfg);
+  if (why) return fail(nullptr, DLLM_INVALID_ARG, "%s", why);
+  if (!name) return fail(nullptr, DLLM_INVALID_ARG, "name is NULL");
+  TensorRef t;
+  if (!find_tensor(*cfg, make_layout(*cfg), name, &t)) return fail(nullptr, DLLM_INVALID_ARG, "unknown tensor '%s'", name);
+  if (offset_bytes) *offset_bytes = t.off;
+  if (n_elements) *n_elements = t.n;
+  return DLLM_OK;
+}
+
+dllm_status dllm_model_create(const dllm_config* cfg, void* d_weights, dllm_model** out) {
+  if (!out) return fail(nullptr, DLLM_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  const char* why = check_config(cfg);
+  if (why) return fail(nullptr, DLLM_INVALID_ARG, "%s", why);
+  if ((why = check_supported(cfg))) return fail(nullptr, DLLM_UNSUPPORTED, "%s", why);
+  if (!d_weights || ((uintptr_t)d_weights & 255)) return fail(nullptr, DLLM_INVALID_ARG, "d_weights must be a 256-byte aligned device pointer");
+  dllm_model* m = new (std::nothrow) dllm_model();
+  if (!m) return fail(nullptr, DLLM_OUT_OF_MEMORY, "host allocation failed");
+  m->cfg = *cfg;
+  m->lay = make_layout(*cfg);
+  m->d_w = static_cast<uint8_t*>(d_weights);
+  *out = m;
+  return DLLM_OK;
+}
+
+dllm_status dllm_model_set_tensor(dllm_model* m, const char* name, const float* h_src, size_t n_elements) {
+  if (!m) return fail(nullptr, DLLM_INVALID_ARG, "model is NULL");
+  if (!name || !h_src) return fail(&m->err, DLLM_INVALID_ARG, "NULL argument");
+  TensorRef t;
+  if (!find_tensor(m->cfg, m->lay, name, &t)) return fail(&m->err, DLLM_INVALID_ARG, "unknown tensor '%s'", name);
+  if (t.n != n_elements)
+    return fail(&m->err, DLLM_INVALID_ARG, "tensor '%s' has %zu elements, got %zu", name, t.n, n_elements);
+  if (t.f32 || m->cfg.dtype == DLLM_FP32) {
+    CU_TRY(&m->err, cudaMemcpy(m->d_w + t.off, h_src, t.n * 4, cudaMemcpyHostToDevice));
+    return DLLM_OK;
+  }
+  std::vector<uint16_t> tmp;
+  try {
+    tmp.resize(t.n);
+  } catch (...) {
+    return fail(&m->err, DLLM_OUT_OF_MEMORY, "host allocation failed");
+  }
+  for (size_t i = 0; i < t.n; ++i) tmp[i] = f32_to_bf16_rne(h_src[i]);
+  CU_TRY(&m->err, cudaMemcpy(m->d_w + t.off, tmp.data(), t.n * 2, cudaMemcpyHostToDevice));
+  return DLLM_OK;
+}
+
+dllm_status dllm_model_destroy(dllm_model* m) {
+  delete m;
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_create(dllm_model* m, int B, int P, int R, void* d_cache, void* d_workspace, void* stream,
+                                dllm_session** out) {
+  if (!out) return fail(nullptr, DLLM_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (!m) return fail(nullptr, DLLM_INVALID_ARG, "model is NULL");
+  if (B <= 0 || P <= 0 || R <= 0) return fail(&m->err, DLLM_INVALID_ARG, "B, P and R must be positive");
+  if (R > 8192) return fail(&m->err, DLLM_UNSUPPORTED, "R > 8192 is not supported by the selection kernel");
+  if (!d_cache || !d_workspace || ((uintptr_t)d_cache & 255) || ((uintptr_t)d_workspace & 255))
+    return fail(&m->err, DLLM_INVALID_ARG, "d_cache and d_workspace must be 256-byte aligned device pointers");
+  dllm_session* s = new (std::nothrow) dllm_session();
+  if (!s) return fail(&m->err, DLLM_OUT_OF_MEMORY, "host allocation failed");
+  s->m = m;
+  s->B = B;
+  s->P = P;
+  s->R = R;
+  s->n = P + R;
+  s->d_cache = static_cast<uint8_t*>(d_cache);
+  s->d_ws = static_cast<uint8_t*>(d_workspace);
+  s->ws = make_workspace(m->cfg, B, P, R);
+  s->forced_count.assign(m->cfg.n_layers, -1);
+  cudaStream_t st = (cudaStream_t)stream;
+  // rotary table: [pos][cos(hd/2) | sin(hd/2)], angle = pos * theta^(-2i/hd), evaluated in double
+  const int hd = m->cfg.head_dim, half = hd / 2;
+  std::vector<float> tab((size_t)s->n * hd);
+  for (int pos = 0; pos < s->n; ++pos)
+    for (int i = 0; i < half; ++i) {
+      const double ang = (double)pos * pow((double)m->cfg.rope_theta, -2.0 * i / hd);
+      tab[(size_t)pos * hd + i] = (float)cos(ang);
+      tab[(size_t)pos * hd + half + i] = (float)sin(ang);
+    }
+  cudaError_t e = cudaMemsetAsync(d_cache, 0, dllm_cache_bytes(&m->cfg, B, P, R), st);
+  // everything but the (large) GEMM slab is cleared; the slab is always written before it is read
+  if (e == cudaSuccess) e = cudaMemsetAsync(d_workspace, 0, s->ws.part, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e == cudaSuccess) e = cudaMemcpy(s->d_ws + s->ws.rope, tab.data(), tab.size() * 4, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    delete s;
+    return fail(&m->err, DLLM_CUDA_ERROR, "session setup: %s", cudaGetErrorString(e));
+  }
+  *out = s;
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_destroy(dllm_session* s) {
+  if (!s) return DLLM_OK;
+  for (auto& kv : s->graphs) cudaGraphExecDestroy(kv.second.exec);
+  delete s;
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_set_prompt(dllm_session* s, const int32_t* h_prompt, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (!h_prompt) return fail(&s->err, DLLM_INVALID_ARG, "h_prompt is NULL");
+  const int V = s->m->cfg.vocab;
+  std::vector<int32_t> tok((size_t)s->B * s->n);
+  for (int b = 0; b < s->B; ++b) {
+    for (int i = 0; i < s->P; ++i) {
+      const int32_t t = h_prompt[(size_t)b * s->P + i];
+      if (t < 0 || t >= V) return fail(&s->err, DLLM_INVALID_ARG, "prompt id %d outside [0, %d)", t, V);
+      tok[(size_t)b * s->n + i] = t;
+    }
+    for (int j = 0; j < s->R; ++j) tok[(size_t)b * s->n + s->P + j] = s->m->cfg.mask_id;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  CU_TRY(&s->err, cudaStreamSynchronize(st));
+  CU_TRY(&s->err, cudaMemcpy(s->d_ws + s->ws.tokens, tok.data(), tok.size() * 4, cudaMemcpyHostToDevice));
+  s->valid = false;
+  s->have_pred = false;
+  return DLLM_OK;
+}
+
+dllm_status dllm_step_full(dllm_session* s, void* stream) { return run_step(s, 1, 1, 0.f, DLLM_K_FLOOR, stream); }
+
+dllm_status dllm_step_cached(dllm_session* s, int refresh_prompt, int refresh_response, float rho, dllm_kround kround,
+                             void* stream) {
+  return run_step(s, refresh_prompt, refresh_response, rho, kround, stream);
+}
+
+dllm_status dllm_step_scheduled(dllm_session* s, int k, int K, int Kp, int Kr, float rho, dllm_kround kround,
+                                void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (K <= 0 || k <= 0 || k > K || Kp <= 0 || Kr <= 0)
+    return fail(&s->err, DLLM_INVALID_ARG, "need 1 <= k <= K and positive K_p, K_r");
+  const int rp = (k == K) || (k % Kp == 0), rr = (k == K) || (k % Kr == 0);
+  return run_step(s, rp, rr, rho, kround, stream);
+}
+
+dllm_status dllm_remask_low_confidence(dllm_session* s, int block_start, int block_len, int n_transfer, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (block_start < 0 || block_len <= 0 || block_start + block_len > s->R || n_transfer < 0)
+    return fail(&s->err, DLLM_INVALID_ARG, "block [%d, %d) outside the response or n_transfer < 0", block_start,
+                block_start + block_len);
+  if (block_len > 4096) return fail(&s->err, DLLM_UNSUPPORTED, "block_len > 4096");
+  if (!s->have_pred) return fail(&s->err, DLLM_BAD_STATE, "no prediction yet: run a step first");
+  Launch L{(cudaStream_t)stream, s->wsp<int>(s->ws.status), &s->launches};
+  launch_remask(L, s->wsp<int32_t>(s->ws.tokens), s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf), s->geo(),
+                s->m->cfg.mask_id, block_start, block_len, n_transfer);
+  CU_TRY(&s->err, cudaGetLastError());
+  return DLLM_OK;
+}
+
+dllm_status dllm_generate(dllm_session* s, int K, int Kp, int Kr, float rho, dllm_kround kround, int block_len,
+                          void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (K <= 0 || Kp <= 0 || Kr <= 0 || block_len <= 0 || s->R % block_len)
+    return fail(&s->err, DLLM_INVALID_ARG, "need positive K, K_p, K_r and block_len dividing R");
+  const int blocks = s->R / block_len;
+  if (K % blocks) return fail(&s->err, DLLM_INVALID_ARG, "K must be a multiple of the number of blocks");
+  const int spb = K / blocks;
+  for (int k = K; k >= 1; --k) {
+    dllm_status st = dllm_step_scheduled(s, k, K, Kp, Kr, rho, kround, stream);
+    if (st != DLLM_OK) return st;
+    const int t = K - k, blk = std::min(t / spb, blocks - 1), i = t - blk * spb;
+    const int n_transfer = block_len / spb + (i < block_len % spb ? 1 : 0);
+    st = dllm_remask_low_confidence(s, blk * block_len, block_len, n_transfer, stream);
+    if (st != DLLM_OK) return st;
+  }
+  return DLLM_OK;
+}
+
+dllm_status dllm_sync(dllm_session* s, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
+  int code = 0;
+  CU_TRY(&s->err, cudaMemcpy(&code, s->d_ws + s->ws.status, 4, cudaMemcpyDeviceToHost));
+  if (code == 0) return DLLM_OK;
+  cudaMemset(s->d_ws + s->ws.status, 0, 4);
+  if (code >= 100 && code < 200) return fail(&s->err, DLLM_TIMEOUT, "a device-side wait gave up (code %d)", code);
+  return fail(&s->err, DLLM_CUDA_ERROR, "device status %d", code);
+}
+
+dllm_status dllm_get_tokens(dllm_session* s, int32_t* h_out, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (!h_out) return fail(&s->err, DLLM_INVALID_ARG, "h_out is NULL");
+  CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
+  CU_TRY(&s->err, cudaMemcpy(h_out, s->d_ws + s->ws.tokens, (size_t)s->B * s->n * 4, cudaMemcpyDeviceToHost));
+  return DLLM_OK;
+}
+
+dllm_status dllm_set_response_tokens(dllm_session* s, const int32_t* h_tok, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (!h_tok) return fail(&s->err, DLLM_INVALID_ARG, "h_tok is NULL");
+  for (size_t i = 0; i < (size_t)s->B * s->R; ++i)
+    if (h_tok[i] < 0 || h_tok[i] >= s->m->cfg.vocab) return fail(&s->err, DLLM_INVALID_ARG, "token id out of range");
+  CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
+  CU_TRY(&s->err, cudaMemcpy2D(s->d_ws + s->ws.tokens + (size_t)s->P * 4, (size_t)s->n * 4, h_tok, (size_t)s->R * 4,
+                               (size_t)s->R * 4, s->B, cudaMemcpyHostToDevice));
+  return DLLM_OK;
+}
+
+dllm_status dllm_get_hidden(dllm_session* s, float* h_out, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (!h_out) return fail(&s->err, DLLM_INVALID_ARG, "h_out is NULL");
+  if (!s->have_pred) return fail(&s->err, DLLM_BAD_STATE, "no step has run");
+  CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
+  // response rows come first in the residual stream
+  CU_TRY(&s->err, cudaMemcpy(h_out, s->d_ws + s->ws.x, (size_t)s->B * s->R * s->m->cfg.d_model * 4,
+                             cudaMemcpyDeviceToHost));
+  return DLLM_OK;
+}
+
+dllm_status dllm_get_pred(dllm_session* s, int32_t* h_x0, float* h_conf, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (!s->have_pred) return fail(&s->err, DLLM_BAD_STATE, "no step has run");
+  CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
+  const size_t BR = (size_t)s->B * s->R;
+  if (h_x0) CU_TRY(&s->err, cudaMemcpy(h_x0, s->d_ws + s->ws.x0, BR * 4, cudaMemcpyDeviceToHost));
+  if (h_conf) CU_TRY(&s->err, cudaMemcpy(h_conf, s->d_ws + s->ws.conf, BR * 4, cudaMemcpyDeviceToHost));
+  return DLLM_OK;
+}
+
+dllm_status dllm_get_logits(dllm_session* s, float* h_out, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (!h_out) return fail(&s->err, DLLM_INVALID_ARG, "h_out is NULL");
+  if (!s->have_pred) return fail(&s->err, DLLM_BAD_STATE, "no step has run");
+  const dllm_config& c = s->m->cfg;
+  cudaStream_t st = (cudaStream_t)stream;
+  Launch L{st, s->wsp<int>(s->ws.status), &s->launches};
+  const int BR = s->B * s->R;
+  launch_rmsnorm(L, c.dtype, s->wsp<float>(s->ws.x), reinterpret_cast<const float*>(s->m->d_w + s->m->lay.norm_f),
+                 s->wsp<uint8_t>(s->ws.u), c.d_model, c.rms_eps, 0, BR);
+  Partials part;
+  dllm_status r = run_gemm(s, L, s->wsp<uint8_t>(s->ws.u), s->m->d_w + s->m->lay.lm_head, BR, c.vocab, c.d_model, &part);
+  if (r != DLLM_OK) return r;
+  launch_mask_column(L, s->wsp<float>(s->ws.part), BR, c.vocab, c.mask_id);
+  CU_TRY(&s->err, cudaStreamSynchronize(st));
+  CU_TRY(&s->err, cudaMemcpy(h_out, s->d_ws + s->ws.part, (size_t)BR * c.vocab * 4, cudaMemcpyDeviceToHost));
+  return DLLM_OK;
+}
+
+dllm_status dllm_get_selected(dllm_session* s, int layer, int32_t* h_idx, float* h_sim, int* k_sel_out, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (layer < 0 || layer >= s->m->cfg.n_layers) return fail(&s->err, DLLM_INVALID_ARG, "layer out of range");
+  if (!s->have_pred) return fail(&s->err, DLLM_BAD_STATE, "no step has run");
+  CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
+  const size_t BR = (size_t)s->B * s->R;
+  if (k_sel_out) *k_sel_out = s->last_ksel;
+  if (h_idx && s->last_ksel > 0)
+    CU_TRY(&s->err, cudaMemcpy2D(h_idx, (size_t)s->last_ksel * 4, s->d_ws + s->ws.sel + (size_t)layer * BR * 4,
+                                 (size_t)s->R * 4, (size_t)s->last_ksel * 4, s->B, cudaMemcpyDeviceToHost));
+  if (h_sim)
+    CU_TRY(&s->err, cudaMemcpy(h_sim, s->d_ws + s->ws.sim + (size_t)layer * BR * 4, BR * 4, cudaMemcpyDeviceToHost));
+  return DLLM_OK;
+}
+
+static dllm_status cache_args(dllm_session* s, int layer, int which, const void* p, size_t* n_elems) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (!p) return fail(&s->err, DLLM_INVALID_ARG, "host buffer is NULL");
+  if (layer < 0 || layer >= s->m->cfg.n_layers) return fail(&s->err, DLLM_INVALID_ARG, "layer out of range");
+  if (which < DLLM_CACHE_K || which > DLLM_CACHE_FFN) return fail(&s->err, DLLM_INVALID_ARG, "bad cache id");
+  const size_t width = which <= DLLM_CACHE_V ? s->dkv() : (size_t)s->m->cfg.d_model;
+  *n_elems = (size_t)s->B * s->n * width;
+  return DLLM_OK;
+}
+
+dllm_status dllm_get_cache(dllm_session* s, int layer, int which, float* h_out, void* stream) {
+  size_t n;
+  dllm_status r = cache_args(s, layer, which, h_out, &n);
+  if (r != DLLM_OK) return r;
+  cudaStream_t st = (cudaStream_t)stream;
+  Launch L{st, nullptr, &s->launches};
+  launch_convert_to_f32(L, s->m->cfg.dtype, s->cache(layer, which), s->wsp<float>(s->ws.part), n);
+  CU_TRY(&s->err, cudaStreamSynchronize(st));
+  CU_TRY(&s->err, cudaMemcpy(h_out, s->d_ws + s->ws.part, n * 4, cudaMemcpyDeviceToHost));
+  return DLLM_OK;
+}
+
+dllm_status dllm_set_cache(dllm_session* s, int layer, int which, const float* h_in, void* stream) {
+  size_t n;
+  dllm_status r = cache_args(s, layer, which, h_in, &n);
+  if (r != DLLM_OK) return r;
+  cudaStream_t st = (cudaStream_t)stream;
+  CU_TRY(&s->err, cudaStreamSynchronize(st));
+  CU_TRY(&s->err, cudaMemcpy(s->d_ws + s->ws.part, h_in, n * 4, cudaMemcpyHostToDevice));
+  Launch L{st, nullptr, &s->launches};
+  launch_convert_from_f32(L, s->m->cfg.dtype, s->wsp<float>(s->ws.part), s->cache(layer, which), n);
+  CU_TRY(&s->err, cudaStreamSynchronize(st));
+  return DLLM_OK;
+}
+
+dllm_status dllm_force_selection(dllm_session* s, int layer, const int32_t* h_idx, int count) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (layer < 0 || layer >= s->m->cfg.n_layers) return fail(&s->err, DLLM_INVALID_ARG, "layer out of range");
+  if (count < 0) {
+    s->forced_count[layer] = -1;
+    return DLLM_OK;
+  }
+  if (count > s->R || (count > 0 && !h_idx)) return fail(&s->err, DLLM_INVALID_ARG, "bad forced selection");
+  std::vector<int32_t> buf((size_t)s->B * s->R, 0);
+  for (int b = 0; b < s->B; ++b) {
+    std::vector<int32_t> row(h_idx + (size_t)b * count, h_idx + (size_t)(b + 1) * count);
+    std::sort(row.begin(), row.end());
+    for (int r = 0; r < count; ++r) {
+      if (row[r] < 0 || row[r] >= s->R || (r && row[r] == row[r - 1]))
+        return fail(&s->err, DLLM_INVALID_ARG, "forced indices must be distinct and inside [0, R)");
+      buf[(size_t)b * s->R + r] = row[r];
+    }
+  }
+  CU_TRY(&s->err, cudaDeviceSynchronize());
+  CU_TRY(&s->err, cudaMemcpy(s->d_ws + s->ws.forced + (size_t)layer * s->B * s->R * 4, buf.data(), buf.size() * 4,
+                             cudaMemcpyHostToDevice));
+  s->forced_count[layer] = count;
+  return DLLM_OK;
+}
+
+uint64_t dllm_launch_count(const dllm_session* s) { return s ? s->launches : 0; }
+
+dllm_status dllm_session_use_graphs(dllm_session* s, int enable) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  s->use_graphs = enable != 0;
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if ((enable != 0) != s->simt_gemm) {
+    for (auto& kv : s->graphs) cudaGraphExecDestroy(kv.second.exec);
+    s->graphs.clear();
+  }
+  s->simt_gemm = enable != 0;
+  return DLLM_OK;
+}
+
+// ---- kernel-level entry points ------------------------------------------------
+size_t dllm_gemm_bf16_scratch_bytes(int M, int N, int K) {
+  if (M <= 0 || N <= 0 || K <= 0) return 0;
+  const GemmPlan p = plan_gemm_bf16(M, N, K, 0);
+  return p.S > 1 ? (size_t)p.S * M * N * 4 : 0;
+}
+
+dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, void* d_partials,
+                           void* stream) {
+  if (!d_A || !d_W || !d_C || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
+  if (K % 8) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8");
+  const GemmPlan p = plan_gemm_bf16(M, N, K, 0);
+  if (p.S > 1 && !d_partials) return fail(nullptr, DLLM_INVALID_ARG, "this shape needs split-K scratch");
+  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  float* part = p.S > 1 ? static_cast<float*>(d_partials) : d_C;
+  const char* why = nullptr;
+  cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
+  if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "bf16 GEMM: %s", why ? why : cudaGetErrorString(e));
+  if (p.S > 1) launch_reduce_partials(L, Partials{part, (size_t)M * N, p.S, N}, d_C, M);
+  CU_TRY(nullptr, cudaGetLastError());
+  return DLLM_OK;
+}
+
+dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int dtype,
+                           void* stream) {
+  if (!d_A || !d_W || !d_C || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
+  if (dtype != DLLM_FP32 && dtype != DLLM_BF16) return fail(nullptr, DLLM_INVALID_ARG, "bad dtype");
+  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  launch_gemm_simt(L, dtype, d_A, d_W, d_C, M, N, K);
+  CU_TRY(nullptr, cudaGetLastError());
+  return DLLM_OK;
+}
+
+dllm_status dllm_attention(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B, int a, int n, int H,
+                           int Hkv, int hd, int dtype, void* stream) {
+  if (!d_q || !d_k || !d_v || !d_o || B <= 0 || a <= 0 || n <= 0 || H <= 0 || Hkv <= 0 || H % Hkv)
+    return fail(nullptr, DLLM_INVALID_ARG, "bad attention arguments");
+  if (dtype != DLLM_FP32 && dtype != DLLM_BF16) return fail(nullptr, DLLM_INVALID_ARG, "bad dtype");
+  if (hd % 32 || hd > 128) return fail(nullptr, DLLM_UNSUPPORTED, "head_dim must be 32, 64, 96 or 128");
+  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  cudaError_t e = launch_attention(L, dtype, d_q, d_k, d_v, d_o, B, a, n, H, Hkv, hd);
+  if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
+  return DLLM_OK;
+}
+
+dllm_status dllm_vverify_select(const void* d_vnew, void* d_vcache, float* d_sim, int32_t* d_idx, int B, int R,
+                                int width, int k, int dtype, void* stream) {
+  if (!d_vnew || !d_vcache || !d_sim || B <= 0 || R <= 0 || width <= 0 || k < 0 || k > R || (k > 0 && !d_idx))
+    return fail(nullptr, DLLM_INVALID_ARG, "bad V-verify arguments");
+  if (dtype != DLLM_FP32 && dtype != DLLM_BF16) return fail(nullptr, DLLM_INVALID_ARG, "bad dtype");
+  if (width % 8 || R > 8192) return fail(nullptr, DLLM_UNSUPPORTED, "width must be a multiple of 8 and R <= 8192");
+  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  launch_vverify_rows(L, dtype, d_vnew, d_vcache, d_sim, B * R, width);
+  if (k > 0) launch_select(L, d_sim, nullptr, 1, k, d_idx, k, nullptr, Geo{B, 0, R, R, width}, 0);
+  CU_TRY(nullptr, cudaGetLastError());
+  return DLLM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,554 @@
+// Memory-bound kernels of the cached denoising step: embedding, RMSNorm,
+// V-verify (Eq. 6) with the whole-V overwrite, bottom-k selection, row gather,
+// RoPE + K scatter, cache scatters, SwiGLU gate, residual assembly, greedy
+// estimate with confidence (Eq. 4) and the low-confidence transition (Eq. 5).
+//
+// All of them are one pass over their rows with 16-byte vector accesses, fp32
+// arithmetic and warp-shuffle reductions.  Split-K partial sums of the
+// preceding GEMM are reduced here, in slab order, so the GEMM never needs
+// atomics and every row's value is independent of which other rows were in the
+// same launch.
+#include "internal.h"
+
+namespace dllm {
+
+#define DLLM_DISPATCH(dtype, ...)                 \
+  do {                                            \
+    if ((dtype) == 0) {                           \
+      using T = float;                            \
+      __VA_ARGS__;                                \
+    } else {                                      \
+      using T = __nv_bfloat16;                    \
+      __VA_ARGS__;                                \
+    }                                             \
+  } while (0)
+
+// ------------------------------------------------------------------ embed
+template <typename T>
+__global__ void embed_kernel(const T* __restrict__ E, const int32_t* __restrict__ tokens, float* __restrict__ x, Geo g,
+                             int c0) {
+  const int c = c0 + blockIdx.x;
+  int b, pos;
+  carried_to_pos(c, g, b, pos);
+  const int tok = tokens[(size_t)b * g.n + pos];
+  const T* src = E + (size_t)tok * g.d;
+  float* dst = x + (size_t)c * g.d;
+  for (int i = threadIdx.x * 8; i < g.d; i += blockDim.x * 8) {
+    float v[8];
+    Vec8<T>::load(src + i, v);
+    Vec8<float>::store(dst + i, v);
+  }
+}
+
+void launch_embed(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, Geo g, int c0, int c1) {
+  if (c1 <= c0) return;
+  DLLM_DISPATCH(dtype, (embed_kernel<T><<<c1 - c0, 128, 0, L.stream>>>((const T*)E, tokens, x, g, c0)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ rmsnorm
+template <typename T>
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain, T* __restrict__ out, int d,
+                               float eps, int c0) {
+  __shared__ float red[32];
+  const size_t row = (size_t)(c0 + blockIdx.x);
+  const float* xr = x + row * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
+    float v[8];
+    Vec8<float>::load(xr + i, v);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) ss += v[j] * v[j];
+  }
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)d + eps);
+  T* orow = out + row * d;
+  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
+    float v[8], gv[8];
+    Vec8<float>::load(xr + i, v);
+    Vec8<float>::load(gain + i, gv);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = v[j] * r * gv[j];
+    Vec8<T>::store(orow + i, v);
+  }
+}
+
+void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gain, void* out, int d, float eps, int c0,
+                    int c1) {
+  if (c1 <= c0) return;
+  DLLM_DISPATCH(dtype, (rmsnorm_kernel<T><<<c1 - c0, 256, 0, L.stream>>>(x, gain, (T*)out, d, eps, c0)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ V-verify (Eq. 6) + V overwrite
+template <typename T>
+__global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restrict__ sim, Geo g, int dkv) {
+  __shared__ float red[32];
+  const int c = blockIdx.x;  // response row, carried order
+  const int b = c / g.R, j = c - b * g.R;
+  T* vrow = Vc + ((size_t)b * g.n + g.P + j) * dkv;
+  float dot = 0.f, na = 0.f, nb = 0.f;
+  for (int i = threadIdx.x * 8; i < dkv; i += blockDim.x * 8) {
+    float vn[8], vo[8];
+    sum_partials8(part.p, part.split_stride, part.S, (size_t)c * part.N + i, vn);
+    Vec8<T>::load(vrow + i, vo);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      vn[t] = Vec8<T>::round(vn[t]);  // compare what the cache will hold
+      dot += vn[t] * vo[t];
+      na += vn[t] * vn[t];
+      nb += vo[t] * vo[t];
+    }
+    Vec8<T>::store(vrow + i, vn);
+  }
+  dot = block_sum(dot, red);
+  na = block_sum(na, red);
+  nb = block_sum(nb, red);
+  if (threadIdx.x == 0) sim[c] = dot / fmaxf(sqrtf(na * nb), 1e-8f);
+}
+
+void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv) {
+  const int rows = g.B * g.R;
+  DLLM_DISPATCH(dtype, (vverify_kernel<T><<<rows, 128, 0, L.stream>>>(part, (T*)Vc_layer, sim, g, dkv)));
+  L.count();
+}
+
+// standalone form used by the kernel-level entry point: v_new given as a tensor
+template <typename T>
+__global__ void vverify_rows_kernel(const T* __restrict__ vnew, T* __restrict__ vcache, float* __restrict__ sim,
+                                    int width) {
+  __shared__ float red[32];
+  const size_t row = blockIdx.x;
+  const T* a = vnew + row * width;
+  T* bb = vcache + row * width;
+  float dot = 0.f, na = 0.f, nb = 0.f;
+  for (int i = threadIdx.x * 8; i < width; i += blockDim.x * 8) {
+    float vn[8], vo[8];
+    Vec8<T>::load(a + i, vn);
+    Vec8<T>::load(bb + i, vo);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      dot += vn[t] * vo[t];
+      na += vn[t] * vn[t];
+      nb += vo[t] * vo[t];
+    }
+    Vec8<T>::store(bb + i, vn);
+  }
+  dot = block_sum(dot, red);
+  na = block_sum(na, red);
+  nb = block_sum(nb, red);
+  if (threadIdx.x == 0) sim[row] = dot / fmaxf(sqrtf(na * nb), 1e-8f);
+}
+
+void launch_vverify_rows(const Launch& L, int dtype, const void* vnew, void* vcache, float* sim, int rows, int width) {
+  if (rows <= 0) return;
+  DLLM_DISPATCH(dtype, (vverify_rows_kernel<T><<<rows, 128, 0, L.stream>>>((const T*)vnew, (T*)vcache, sim, width)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ bottom-k selection
+// One block per sequence.  Keys are unique (the index is part of the key), so
+// the rank of a key among all R keys is its position in sorted order; a row is
+// selected iff rank < k.  R^2 comparisons out of shared memory: R <= 8192.
+__global__ void select_kernel(const float* __restrict__ sim, const int32_t* __restrict__ forced, int mode, int ksel,
+                              int32_t* __restrict__ sel, int sel_stride, int32_t* __restrict__ act, Geo g,
+                              int refresh_prompt) {
+  extern __shared__ unsigned long long keys[];  // R keys, then R flags (as bytes)
+  unsigned char* flag = reinterpret_cast<unsigned char*>(keys + g.R);
+  const int b = blockIdx.x;
+  const int R = g.R;
+  const int a_seq = (refresh_prompt ? g.P : 0) + ksel;
+  int32_t* act_b = act ? act + (size_t)b * a_seq : nullptr;
+  int32_t* sel_b = sel + (size_t)b * sel_stride;
+  if (refresh_prompt && act)
+    for (int i = threadIdx.x; i < g.P; i += blockDim.x) act_b[i] = g.B * R + b * g.P + i;
+  int32_t* act_r = act ? act_b + (refresh_prompt ? g.P : 0) : nullptr;
+  if (mode == 0) {
+    for (int j = threadIdx.x; j < R; j += blockDim.x) {
+      sel_b[j] = j;
+      if (act_r) act_r[j] = b * R + j;
+    }
+    return;
+  }
+  if (mode == 2) {
+    for (int r = threadIdx.x; r < ksel; r += blockDim.x) {
+      const int j = forced[(size_t)b * R + r];
+      sel_b[r] = j;
+      if (act_r) act_r[r] = b * R + j;
+    }
+    return;
+  }
+  for (int j = threadIdx.x; j < R; j += blockDim.x) {
+    const float s = sim[(size_t)b * R + j];
+    // s in [-1, 1] up to rounding; NaN (degenerate input) sorts first
+    const float qf = rintf(s * 1048576.0f);
+    const long long q = (s == s) ? (long long)qf + (1ll << 22) : 0ll;
+    keys[j] = ((unsigned long long)q << 32) | (unsigned)j;
+    flag[j] = 0;
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < R; j += blockDim.x) {
+    const unsigned long long kj = keys[j];
+    int rank = 0;
+    for (int i = 0; i < R; ++i) rank += (keys[i] < kj);
+    flag[j] = (rank < ksel);
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < R; j += blockDim.x) {
+    if (!flag[j]) continue;
+    int r = 0;
+    for (int i = 0; i < j; ++i) r += flag[i];
+    sel_b[r] = j;
+    if (act_r) act_r[r] = b * R + j;
+  }
+}
+
+void launch_select(const Launch& L, const float* sim, const int32_t* forced, int mode, int ksel, int32_t* sel,
+                   int sel_stride, int32_t* act, Geo g, int refresh_prompt) {
+  const size_t smem = (size_t)g.R * 9 + 16;
+  select_kernel<<<g.B, 256, smem, L.stream>>>(sim, forced, mode, ksel, sel, sel_stride, act, g, refresh_prompt);
+  L.count();
+}
+
+// ------------------------------------------------------------------ gather
+template <typename T>
+__global__ void gather_rows_kernel(const T* __restrict__ src, const int32_t* __restrict__ act, T* __restrict__ dst,
+                                   int d) {
+  const size_t r = blockIdx.x;
+  const uint4* s = reinterpret_cast<const uint4*>(src + (size_t)act[r] * d);
+  uint4* o = reinterpret_cast<uint4*>(dst + r * d);
+  const int nvec = d * (int)sizeof(T) / 16;
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) o[i] = s[i];
+}
+
+void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32_t* act, void* dst, int rows, int d) {
+  if (rows <= 0) return;
+  DLLM_DISPATCH(dtype, (gather_rows_kernel<T><<<rows, 128, 0, L.stream>>>((const T*)src, act, (T*)dst, d)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ RoPE + K scatter
+// grid (Ma, H + Hkv): one block per (active row, head).  Rotate-half pairing:
+// element i with i + hd/2, angle pos * theta^(-2i/hd) from a table built on the host.
+template <typename T>
+__global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ rope_tab,
+                               T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int H, int Hkv, int hd) {
+  const int r = blockIdx.x, head = blockIdx.y;
+  int b, pos;
+  carried_to_pos(act[r], g, b, pos);
+  const int half = hd >> 1;
+  const int dq = H * hd, dkv = Hkv * hd;
+  const bool is_q = head < H;
+  const int col0 = is_q ? head * hd : dq + (head - H) * hd;
+  T* dst = is_q ? qbuf + (size_t)r * dq + head * hd : Kc + ((size_t)b * g.n + pos) * dkv + (head - H) * hd;
+  const float* tab = rope_tab + (size_t)pos * hd;  // [cos(half) | sin(half)]
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    float lo = 0.f, hi = 0.f;
+    for (int s = 0; s < part.S; ++s) {
+      const float* p = part.p + (size_t)s * part.split_stride + (size_t)r * part.N + col0;
+      lo += p[i];
+      hi += p[i + half];
+    }
+    const float c = tab[i], sn = tab[half + i];
+    dst[i] = from_f32<T>(lo * c - hi * sn);
+    dst[i + half] = from_f32<T>(hi * c + lo * sn);
+  }
+}
+
+void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* act, const float* rope_tab, void* qbuf,
+                    void* Kc_layer, Geo g, int Ma, int H, int Hkv, int hd) {
+  if (Ma <= 0) return;
+  dim3 grid(Ma, H + Hkv);
+  DLLM_DISPATCH(dtype, (qk_rope_kernel<T><<<grid, 64, 0, L.stream>>>(part, act, rope_tab, (T*)qbuf, (T*)Kc_layer, g, H,
+                                                                     Hkv, hd)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ scatter rows into a cache tensor
+template <typename T>
+__global__ void scatter_rows_kernel(Partials part, const int32_t* __restrict__ act, int c_base, T* __restrict__ cache,
+                                    Geo g, int width) {
+  const int r = blockIdx.x;
+  const int c = act ? act[r] : c_base + r;
+  int b, pos;
+  carried_to_pos(c, g, b, pos);
+  T* dst = cache + ((size_t)b * g.n + pos) * width;
+  for (int i = threadIdx.x * 8; i < width; i += blockDim.x * 8) {
+    float v[8];
+    sum_partials8(part.p, part.split_stride, part.S, (size_t)r * part.N + i, v);
+    Vec8<T>::store(dst + i, v);
+  }
+}
+
+void launch_scatter_rows(const Launch& L, int dtype, Partials part, const int32_t* act, int c_base, void* cache_layer,
+                         Geo g, int rows, int width) {
+  if (rows <= 0) return;
+  DLLM_DISPATCH(dtype,
+                (scatter_rows_kernel<T><<<rows, 128, 0, L.stream>>>(part, act, c_base, (T*)cache_layer, g, width)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ O-proj epilogue
+// AttnOut row -> cache (rounded to the cache dtype); h = x + AttnOut (the
+// rounded value, so a later step that reads the cache sees the same h);
+// hn = rmsnorm(h) * gain2.
+template <typename T>
+__global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ x,
+                                      const float* __restrict__ gain2, T* __restrict__ Ac, T* __restrict__ hn, Geo g,
+                                      float eps) {
+  extern __shared__ float hrow[];
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  const int c = act[r];
+  int b, pos;
+  carried_to_pos(c, g, b, pos);
+  const int d = g.d;
+  T* arow = Ac + ((size_t)b * g.n + pos) * d;
+  const float* xr = x + (size_t)c * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
+    float a[8], xv[8];
+    sum_partials8(part.p, part.split_stride, part.S, (size_t)r * part.N + i, a);
+    Vec8<float>::load(xr + i, xv);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      a[t] = Vec8<T>::round(a[t]);
+      xv[t] += a[t];
+      ss += xv[t] * xv[t];
+    }
+    Vec8<T>::store(arow + i, a);
+    Vec8<float>::store(hrow + i, xv);
+  }
+  ss = block_sum(ss, red);
+  const float rs = rsqrtf(ss / (float)d + eps);
+  T* out = hn + (size_t)r * d;
+  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
+    float v[8], gv[8];
+    Vec8<float>::load(hrow + i, v);
+    Vec8<float>::load(gain2 + i, gv);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) v[t] = v[t] * rs * gv[t];
+    Vec8<T>::store(out + i, v);
+  }
+}
+
+void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int32_t* act, const float* x,
+                           const float* gain2, void* Ac_layer, void* hn, Geo g, int Ma, float eps) {
+  if (Ma <= 0) return;
+  const size_t smem = (size_t)g.d * sizeof(float);
+  DLLM_DISPATCH(dtype, (oproj_epilogue_kernel<T><<<Ma, 256, smem, L.stream>>>(part, act, x, gain2, (T*)Ac_layer,
+                                                                            (T*)hn, g, eps)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ SwiGLU gate
+template <typename T>
+__global__ void silu_mul_kernel(Partials part, T* __restrict__ out, int Ma, int m) {
+  const int mv = m >> 3;
+  const size_t total = (size_t)Ma * mv;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(idx / mv), j = (int)(idx - (size_t)r * mv) * 8;
+    float gt[8], up[8];
+    sum_partials8(part.p, part.split_stride, part.S, (size_t)r * part.N + j, gt);
+    sum_partials8(part.p, part.split_stride, part.S, (size_t)r * part.N + m + j, up);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) gt[t] = gt[t] / (1.f + expf(-gt[t])) * up[t];
+    Vec8<T>::store(out + (size_t)r * m + j, gt);
+  }
+}
+
+void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int Ma, int m) {
+  if (Ma <= 0) return;
+  const size_t total = (size_t)Ma * (m >> 3);
+  const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+  DLLM_DISPATCH(dtype, (silu_mul_kernel<T><<<blocks, 256, 0, L.stream>>>(part, (T*)out, Ma, m)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ residual assembly
+template <typename T>
+__global__ void residual_kernel(float* __restrict__ x, const T* __restrict__ Ac, const T* __restrict__ Fc, Geo g,
+                                int c0) {
+  const int c = c0 + blockIdx.x;
+  int b, pos;
+  carried_to_pos(c, g, b, pos);
+  const size_t crow = ((size_t)b * g.n + pos) * g.d;
+  float* xr = x + (size_t)c * g.d;
+  for (int i = threadIdx.x * 8; i < g.d; i += blockDim.x * 8) {
+    float xv[8], a[8], f[8];
+    Vec8<float>::load(xr + i, xv);
+    Vec8<T>::load(Ac + crow + i, a);
+    Vec8<T>::load(Fc + crow + i, f);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) xv[t] = (xv[t] + a[t]) + f[t];
+    Vec8<float>::store(xr + i, xv);
+  }
+}
+
+void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer, const void* Fc_layer, Geo g, int c0,
+                     int c1) {
+  if (c1 <= c0) return;
+  DLLM_DISPATCH(dtype,
+                (residual_kernel<T><<<c1 - c0, 128, 0, L.stream>>>(x, (const T*)Ac_layer, (const T*)Fc_layer, g, c0)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ greedy estimate + confidence (Eq. 4)
+// Online (max, argmax, sum exp) per thread, merged across the block.  Ties go
+// to the lowest id.  The mask id is skipped: the estimate is never [MASK].
+struct MaxSum {
+  float m, s;
+  int a;
+};
+__device__ __forceinline__ MaxSum merge(MaxSum p, MaxSum q) {
+  if (q.m > p.m || (q.m == p.m && q.a < p.a)) {
+    MaxSum t = p;
+    p = q;
+    q = t;
+  }
+  if (q.m > -INFINITY) p.s += q.s * expf(q.m - p.m);
+  return p;
+}
+
+__global__ void argmax_conf_kernel(const float* __restrict__ logits, int vocab, int mask_id, int32_t* __restrict__ x0,
+                                   float* __restrict__ conf) {
+  __shared__ MaxSum sh[32];
+  const size_t row = blockIdx.x;
+  const float* lr = logits + row * vocab;
+  MaxSum t{-INFINITY, 0.f, 0x7fffffff};
+  for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
+    if (i == mask_id) continue;
+    const float v = lr[i];
+    if (v > t.m) {
+      t.s = t.s * expf(t.m - v) + 1.f;
+      t.m = v;
+      t.a = i;
+    } else {
+      t.s += expf(v - t.m);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    MaxSum q;
+    q.m = __shfl_xor_sync(0xffffffffu, t.m, o);
+    q.s = __shfl_xor_sync(0xffffffffu, t.s, o);
+    q.a = __shfl_xor_sync(0xffffffffu, t.a, o);
+    t = merge(t, q);
+  }
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) sh[w] = t;
+  __syncthreads();
+  if (w == 0) {
+    const int nw = blockDim.x >> 5;
+    t = (lane < nw) ? sh[lane] : MaxSum{-INFINITY, 0.f, 0x7fffffff};
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      MaxSum q;
+      q.m = __shfl_xor_sync(0xffffffffu, t.m, o);
+      q.s = __shfl_xor_sync(0xffffffffu, t.s, o);
+      q.a = __shfl_xor_sync(0xffffffffu, t.a, o);
+      t = merge(t, q);
+    }
+    if (lane == 0) {
+      x0[row] = t.a;
+      conf[row] = 1.f / t.s;
+    }
+  }
+}
+
+void launch_argmax_conf(const Launch& L, const float* logits, int rows, int vocab, int mask_id, int32_t* x0,
+                        float* conf) {
+  if (rows <= 0) return;
+  argmax_conf_kernel<<<rows, 512, 0, L.stream>>>(logits, vocab, mask_id, x0, conf);
+  L.count();
+}
+
+// ------------------------------------------------------------------ low-confidence transition (Eq. 5)
+// One block per sequence.  Candidates: masked positions of the block.  Rank by
+// (confidence descending, position ascending); the first n_transfer are unmasked.
+__global__ void remask_kernel(int32_t* __restrict__ tokens, const int32_t* __restrict__ x0,
+                              const float* __restrict__ conf, Geo g, int mask_id, int block_start, int block_len,
+                              int n_transfer) {
+  extern __shared__ unsigned long long keys[];
+  const int b = blockIdx.x;
+  int32_t* tok = tokens + (size_t)b * g.n + g.P;
+  const float* cf = conf + (size_t)b * g.R;
+  for (int t = threadIdx.x; t < block_len; t += blockDim.x) {
+    const int j = block_start + t;
+    unsigned long long k = ~0ull;
+    if (tok[j] == mask_id) {
+      const float c = cf[j];
+      const unsigned bits = (c == c) ? __float_as_uint(fmaxf(c, 0.f)) : 0u;  // conf >= 0: bit order = value order
+      k = ((unsigned long long)(0xFFFFFFFFu - bits) << 32) | (unsigned)t;
+    }
+    keys[t] = k;
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < block_len; t += blockDim.x) {
+    const unsigned long long kt = keys[t];
+    if (kt == ~0ull) continue;
+    int rank = 0;
+    for (int i = 0; i < block_len; ++i) rank += (keys[i] < kt);
+    if (rank < n_transfer) tok[block_start + t] = x0[(size_t)b * g.R + block_start + t];
+  }
+}
+
+void launch_remask(const Launch& L, int32_t* tokens, const int32_t* x0, const float* conf, Geo g, int mask_id,
+                   int block_start, int block_len, int n_transfer) {
+  remask_kernel<<<g.B, 256, (size_t)block_len * 8, L.stream>>>(tokens, x0, conf, g, mask_id, block_start, block_len,
+                                                               n_transfer);
+  L.count();
+}
+
+// ------------------------------------------------------------------ misc
+__global__ void reduce_partials_kernel(Partials part, float* __restrict__ C, size_t total) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    float v = part.p[i];
+    for (int s = 1; s < part.S; ++s) v += part.p[(size_t)s * part.split_stride + i];
+    C[i] = v;
+  }
+}
+
+void launch_reduce_partials(const Launch& L, Partials part, float* C, int M) {
+  const size_t total = (size_t)M * part.N;
+  if (!total) return;
+  const int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+  reduce_partials_kernel<<<blocks, 256, 0, L.stream>>>(part, C, total);
+  L.count();
+}
+
+template <typename T>
+__global__ void to_f32_kernel(const T* __restrict__ src, float* __restrict__ dst, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = to_f32<T>(src[i]);
+}
+template <typename T>
+__global__ void from_f32_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t n) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = from_f32<T>(src[i]);
+}
+
+void launch_convert_to_f32(const Launch& L, int dtype, const void* src, float* dst, size_t n) {
+  if (!n) return;
+  const int blocks = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
+  DLLM_DISPATCH(dtype, (to_f32_kernel<T><<<blocks, 256, 0, L.stream>>>((const T*)src, dst, n)));
+  L.count();
+}
+void launch_convert_from_f32(const Launch& L, int dtype, const float* src, void* dst, size_t n) {
+  if (!n) return;
+  const int blocks = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
+  DLLM_DISPATCH(dtype, (from_f32_kernel<T><<<blocks, 256, 0, L.stream>>>(src, (T*)dst, n)));
+  L.count();
+}
+
+__global__ void mask_column_kernel(float* logits, int rows, int vocab, int mask_id) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r < rows) logits[(size_t)r * vocab + mask_id] = -INFINITY;
+}
+void launch_mask_column(const Launch& L, float* logits, int rows, int vocab, int mask_id) {
+  if (rows <= 0) return;
+  mask_column_kernel<<<(rows + 127) / 128, 128, 0, L.stream>>>(logits, rows, vocab, mask_id);
+  L.count();
+}
+
+}  // namespace dllm

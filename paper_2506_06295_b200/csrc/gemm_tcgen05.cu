@@ -1,0 +1,383 @@
+// bf16 GEMM for sm_100a:  part[z][M][N] (fp32) = A[M, Kz] * W[N, Kz]^T
+//
+// Every projection of the cached step (V for all response rows; Q/K, O and the
+// SwiGLU matrices for the gathered active rows; the LM head) is
+// "few activation rows x a large weight matrix".  With M between 3 and a few
+// hundred rows the product is bound by streaming W from HBM once, so the kernel
+// is laid out around the weight stream:
+//
+//   * the WEIGHT tile (128 rows of W, 64 k) is the M-side operand of
+//     tcgen05.mma (UMMA M = 128) and the ACTIVATION tile (BN = 32..256 rows of
+//     A, 64 k) is the N-side operand, so small row counts cost no padding of
+//     the 128-row dimension and the accumulator D[128 weight rows][BN act rows]
+//     sits in BN TMEM columns;
+//   * both tiles arrive by TMA (128-byte swizzle) into a ring of shared-memory
+//     stages guarded by full/empty mbarriers; one thread issues the copies,
+//     one thread issues the MMAs, tcgen05.commit releases a stage;
+//   * TMEM lane = output column n, so for a fixed activation row the 32 lanes
+//     of a warp store 32 consecutive floats: the epilogue writes row-major
+//     [M, N] coalesced straight from tcgen05.ld registers;
+//   * split-K over blockIdx.z puts >= 148 CTAs on the weight stream when N/128
+//     is small; every split writes its own slab and the consumer kernel adds
+//     the slabs in order (no atomics, bit-reproducible);
+//   * rows of A beyond M and k beyond K are zero-filled by TMA.
+//
+// Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the
+// CTA records a code in the status word, skips its epilogue, lets copies in
+// flight land, frees its TMEM and returns.
+#include <cuda.h>
+
+#include <mutex>
+#include <unordered_map>
+
+#include "internal.h"
+
+namespace dllm {
+
+namespace {
+
+constexpr int TILE_W = 128;  // weight rows per CTA (UMMA M)
+constexpr int TILE_K = 64;   // k per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr uint32_t W_STAGE_BYTES = TILE_W * TILE_K * 2;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint64_t gtime() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the barrier did not flip within the limit or
+// another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = gtime();
+  uint32_t it = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (gtime() - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c_inner,
+                                            int c_outer) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c_inner), "r"(c_outer)
+      : "memory");
+}
+// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128
+// bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                    // leading byte offset (unused for one swizzle row along K)
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                    // descriptor version for sm_100
+  d |= (uint64_t)2 << 61;                    // swizzle mode: 128 bytes
+  return d;
+}
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major.
+__host__ __device__ constexpr uint32_t make_idesc(int umma_m, int umma_n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(umma_n >> 3) << 17) | ((uint32_t)(umma_m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+
+template <int BN, int STAGES>
+struct SmemLayout {
+  static constexpr uint32_t A_STAGE_BYTES = BN * TILE_K * 2;
+  static constexpr uint32_t STAGE_BYTES = W_STAGE_BYTES + A_STAGE_BYTES;
+  static constexpr uint32_t TOTAL = STAGES * STAGE_BYTES + 1024;  // + slack to align the base to 1024
+};
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                                const __grid_constant__ CUtensorMap tmA,
+                                                                float* __restrict__ part, int M, int N, int num_kb,
+                                                                int kb_per_split, size_t split_stride,
+                                                                int* __restrict__ status) {
+  using SL = SmemLayout<BN, STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[STAGES];
+  __shared__ __align__(8) uint64_t accum_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * BN;       // activation rows
+  const int n0 = blockIdx.y * TILE_W;   // weight rows = output columns
+  const int kb0 = blockIdx.z * kb_per_split;
+  const int kb1 = min(num_kb, kb0 + kb_per_split);
+  const int nkb = kb1 - kb0;            // >= 1 by construction of the plan
+
+  const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    mbar_init(smem_u32(&accum_bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // TMEM: BN fp32 columns x 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"((uint32_t)BN)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_d = tmem_base_slot;
+  volatile int* abortp = &abort_flag;
+
+  if (warp == 0 && lane == 0) {
+    // ---------------- TMA producer ----------------
+    for (int i = 0; i < nkb; ++i) {
+      const int s = i % STAGES;
+      const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+      if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) {
+        if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+        break;
+      }
+      const uint32_t fb = smem_u32(&full_bar[s]);
+      mbar_expect_tx(fb, SL::STAGE_BYTES);
+      const uint32_t dstW = tiles + s * SL::STAGE_BYTES;
+      const int kc = (kb0 + i) * TILE_K;
+      tma_load_2d(dstW, &tmW, fb, kc, n0);
+      tma_load_2d(dstW + W_STAGE_BYTES, &tmA, fb, kc, m0);
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ---------------- MMA issuer ----------------
+    constexpr uint32_t idesc = make_idesc(TILE_W, BN);
+    bool ok = true;
+    for (int i = 0; i < nkb && ok; ++i) {
+      const int s = i % STAGES;
+      const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+      if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp)) {
+        if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_MMA);
+        ok = false;
+        break;
+      }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t sW = tiles + s * SL::STAGE_BYTES;
+      const uint64_t dW = make_smem_desc(sW);
+      const uint64_t dA = make_smem_desc(sW + W_STAGE_BYTES);
+#pragma unroll
+      for (int k = 0; k < TILE_K / UMMA_K; ++k) {
+        // advance 32 bytes (16 bf16) along K inside the swizzle row: +2 in 16-byte units
+        umma_bf16(tmem_d, dW + (uint64_t)(2 * k), dA + (uint64_t)(2 * k), idesc, (i > 0 || k > 0) ? 1u : 0u);
+      }
+      umma_commit(smem_u32(&empty_bar[s]));  // stage reusable once these MMAs have read it
+    }
+    if (ok) umma_commit(smem_u32(&accum_bar));
+  }
+  __syncwarp();
+
+  // ---------------- epilogue: TMEM -> registers -> global (all four warps) ----------------
+  const bool have = mbar_wait(smem_u32(&accum_bar), 0u, abortp);
+  if (!have && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_EPI);
+  // the whole warp must agree before the warp-collective TMEM loads
+  const bool warp_ok = __all_sync(0xffffffffu, have);
+  if (warp_ok) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int n = n0 + warp * 32 + lane;
+    float* out = part + (size_t)blockIdx.z * split_stride + n;
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 16) {
+      if (m0 + c >= M) break;  // uniform across the CTA
+      uint32_t r[16];
+      tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (n < N) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + c + j;
+          if (m < M) out[(size_t)m * N] = __uint_as_float(r[j]);
+        }
+      }
+    }
+  } else {
+    // gave up: let copies that may still be in flight land before the CTA's
+    // shared memory is released
+    const uint64_t t0 = gtime();
+    while (gtime() - t0 < 200000ull) {
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"((uint32_t)BN) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+struct MapKey {
+  const void* base;
+  uint64_t rows, cols;
+  uint32_t box_rows;
+  bool operator==(const MapKey& o) const {
+    return base == o.base && rows == o.rows && cols == o.cols && box_rows == o.box_rows;
+  }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    size_t h = std::hash<const void*>()(k.base);
+    h ^= std::hash<uint64_t>()(k.rows * 1315423911ull + k.cols) + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
+    return h ^ (k.box_rows * 2654435761u);
+  }
+};
+
+// bf16 [rows, cols] row-major, box = box_rows x 64 columns, 128-byte swizzle.
+bool get_tensor_map(const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
+  static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+  static std::mutex mu;
+  MapKey key{base, rows, cols, box_rows};
+  std::lock_guard<std::mutex> lock(mu);
+  auto it = cache.find(key);
+  if (it != cache.end()) {
+    *out = it->second;
+    return true;
+  }
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TILE_K, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMap tm;
+  CUresult r = enc(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (cache.size() > 4096) cache.clear();
+  cache.emplace(key, tm);
+  *out = tm;
+  return true;
+}
+
+template <int BN, int STAGES>
+cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMap& tmA, float* part, int M, int N,
+                       int num_kb, const GemmPlan& plan) {
+  using SL = SmemLayout<BN, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<BN, STAGES>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SL::TOTAL);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  dim3 grid((M + BN - 1) / BN, (N + TILE_W - 1) / TILE_W, plan.S);
+  gemm_bf16_tcgen05_kernel<BN, STAGES><<<grid, 128, SL::TOTAL, L.stream>>>(tmW, tmA, part, M, N, num_kb,
+                                                                          plan.kb_per_split, (size_t)M * N, L.d_status);
+  L.count();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split) {
+  GemmPlan p;
+  p.BN = M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+  p.stages = 4;
+  const int num_kb = (K + TILE_K - 1) / TILE_K;
+  const long tiles = (long)((M + p.BN - 1) / p.BN) * ((N + TILE_W - 1) / TILE_W);
+  int S = 1;
+  if (tiles < 148) {
+    S = (int)((148 + tiles - 1) / tiles);
+    const int max_s = num_kb / 4 > 1 ? num_kb / 4 : 1;
+    if (S > max_s) S = max_s;
+  }
+  if (force_split > 0) S = force_split < num_kb ? force_split : num_kb;
+  p.kb_per_split = (num_kb + S - 1) / S;
+  p.S = (num_kb + p.kb_per_split - 1) / p.kb_per_split;  // no empty split
+  return p;
+}
+
+cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
+                             const GemmPlan& plan, const char** err) {
+  static const char* e_shape = "bf16 GEMM needs K % 8 == 0 and 16-byte aligned operands";
+  static const char* e_map = "cuTensorMapEncodeTiled failed or is unavailable";
+  if (M <= 0 || N <= 0) return cudaSuccess;
+  if (K <= 0 || (K & 7) || ((uintptr_t)A & 15) || ((uintptr_t)W & 15)) {
+    if (err) *err = e_shape;
+    return cudaErrorInvalidValue;
+  }
+  CUtensorMap tmW, tmA;
+  if (!get_tensor_map(W, (uint64_t)N, (uint64_t)K, TILE_W, &tmW) ||
+      !get_tensor_map(A, (uint64_t)M, (uint64_t)K, (uint32_t)plan.BN, &tmA)) {
+    if (err) *err = e_map;
+    return cudaErrorInvalidValue;
+  }
+  const int num_kb = (K + TILE_K - 1) / TILE_K;
+  switch (plan.BN) {
+    case 32: return launch_one<32, 4>(L, tmW, tmA, part, M, N, num_kb, plan);
+    case 64: return launch_one<64, 4>(L, tmW, tmA, part, M, N, num_kb, plan);
+    case 128: return launch_one<128, 3>(L, tmW, tmA, part, M, N, num_kb, plan);
+    default: return launch_one<256, 4>(L, tmW, tmA, part, M, N, num_kb, plan);
+  }
+}
+
+}  // namespace dllm

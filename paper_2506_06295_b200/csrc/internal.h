@@ -1,0 +1,90 @@
+// Host-side launcher interfaces shared by the translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace dllm {
+
+struct Launch {
+  cudaStream_t stream;
+  int* d_status;        // device status word (may be null for kernel-level hooks)
+  uint64_t* counter;    // host launch counter (may be null)
+  inline void count(int k = 1) const {
+    if (counter) *counter += (uint64_t)k;
+  }
+};
+
+// Split-K partial sums of one GEMM: S slabs of [M, N] fp32, slab stride in floats.
+struct Partials {
+  const float* p;
+  size_t split_stride;
+  int S;
+  int N;  // row length
+};
+
+// ---------------- elementwise.cu ----------------
+// x[c] = E[token(c)] for carried rows c0 <= c < c1.
+void launch_embed(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, Geo g, int c0, int c1);
+// out[c] = rmsnorm(x[c]) * gain for carried rows c0 <= c < c1 (out has the model dtype).
+void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gain, void* out, int d, float eps,
+                    int c0, int c1);
+// V-verify (Eq. 6) fused with the whole-V overwrite: for every response row
+// sums the partials, rounds to the cache dtype, takes the cosine against the
+// cached row, overwrites the cached row, writes sim[row].
+void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv);
+// Bottom-k selection per sequence + active-row list.  mode 0: all R rows,
+// 1: bottom-k by (round(sim*2^20), index), 2: forced list.
+void launch_select(const Launch& L, const float* sim, const int32_t* forced, int mode, int ksel, int32_t* sel,
+                   int sel_stride, int32_t* act, Geo g, int refresh_prompt);
+void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32_t* act, void* dst, int rows, int d);
+// RoPE on Q and K of the active rows; Q -> qbuf [Ma, dq]; K -> K cache rows.
+void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* act, const float* rope_tab, void* qbuf,
+                    void* Kc_layer, Geo g, int Ma, int H, int Hkv, int hd);
+// rows of `part` -> cache rows (model dtype).  act == nullptr: rows are the
+// carried ids c_base + i; otherwise act[i].
+void launch_scatter_rows(const Launch& L, int dtype, Partials part, const int32_t* act, int c_base, void* cache_layer,
+                         Geo g, int rows, int width);
+// AttnOut rows -> cache; h = x + AttnOut; hn = rmsnorm(h) * gain2 (model dtype).
+void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int32_t* act, const float* x,
+                           const float* gain2, void* Ac_layer, void* hn, Geo g, int Ma, float eps);
+// act[i][j] = silu(gate) * up from partials [Ma, 2m] (gate columns first).
+void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int Ma, int m);
+// x[c] = (x[c] + AttnOut[c]) + FFNOut[c] for carried rows c0 <= c < c1.
+void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer, const void* Fc_layer, Geo g, int c0,
+                     int c1);
+// (x0, conf) per response row from fp32 logits; the mask id never wins.
+void launch_argmax_conf(const Launch& L, const float* logits, int rows, int vocab, int mask_id, int32_t* x0,
+                        float* conf);
+void launch_remask(const Launch& L, int32_t* tokens, const int32_t* x0, const float* conf, Geo g, int mask_id,
+                   int block_start, int block_len, int n_transfer);
+void launch_reduce_partials(const Launch& L, Partials part, float* C, int M);
+// cache <-> float32 conversion for the inspection hooks
+void launch_convert_to_f32(const Launch& L, int dtype, const void* src, float* dst, size_t n);
+void launch_convert_from_f32(const Launch& L, int dtype, const float* src, void* dst, size_t n);
+void launch_mask_column(const Launch& L, float* logits, int rows, int vocab, int mask_id);
+void launch_vverify_rows(const Launch& L, int dtype, const void* vnew, void* vcache, float* sim, int rows, int width);
+
+// ---------------- gemm_simt.cu ----------------
+// C[M,N] fp32 = A[M,K] * W[N,K]^T on the plain ALUs (fp32 mode; reference path for tests).
+void launch_gemm_simt(const Launch& L, int dtype, const void* A, const void* W, float* C, int M, int N, int K);
+
+// ---------------- gemm_tcgen05.cu ----------------
+struct GemmPlan {
+  int BN;         // activation tile rows (UMMA N)
+  int S;          // split-K factor
+  int kb_per_split;
+  int stages;
+};
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split /* 0 = auto */);
+// Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
+cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
+                             const GemmPlan& plan, const char** err);
+
+// ---------------- attention.cu ----------------
+cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const void* Kc, const void* Vc, void* o, int B,
+                             int a_seq, int n, int H, int Hkv, int hd);
+
+}  // namespace dllm

@@ -1,0 +1,127 @@
+"""Kernel-level parity on the GPU, each entry point called through the C ABI and
+compared element by element with the CPU oracle (or, for a plain matrix product,
+with its definition in float64)."""
+import numpy as np
+import pytest
+
+from oracle import dllm_oracle as O
+from paper_2506_06295_b200 import synth
+from tests.helpers import rel_l2, selection_matches
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2506_06295_b200 import build as build_mod
+    build_mod.build()
+    from paper_2506_06295_b200 import dllm
+    assert torch.cuda.is_available()
+    return torch, dllm
+
+
+GEMM_SHAPES = [
+    (3, 200, 320),       # tiny M (long-prompt regime), ragged N
+    (64, 4096, 4096),    # selected rows x a square projection: split-K
+    (70, 1536, 832),     # ragged M, K = 13 blocks
+    (130, 640, 448),     # M tail of 2 in a 256 tile
+    (256, 512, 3584),    # GQA V projection shape: few N tiles
+    (600, 384, 128),     # several M tiles, two k blocks
+    (64, 24576, 512),    # many N tiles: no split
+]
+
+
+@pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
+def test_gemm_bf16_tcgen05(env, M, N, K):
+    torch, dllm = env
+    A = synth.round_to_bf16(synth.random_normal((M, K), seed=M + K))
+    W = synth.round_to_bf16(synth.random_normal((N, K), seed=N + 7 * K, std=0.05))
+    dA = torch.from_numpy(A).cuda().to(torch.bfloat16)
+    dW = torch.from_numpy(W).cuda().to(torch.bfloat16)
+    got = dllm.gemm_bf16(dA, dW).cpu().numpy()
+    want = A.astype(np.float64) @ W.astype(np.float64).T
+    assert rel_l2(got, want) < 2e-6
+    assert np.abs(got - want).max() < 1e-4 * np.abs(want).max()
+    # bit-reproducible and independent of the other rows in the launch
+    again = dllm.gemm_bf16(dA, dW).cpu().numpy()
+    assert np.array_equal(got, again)
+    if M > 8:
+        sub = dllm.gemm_bf16(dA[: M // 2].contiguous(), dW).cpu().numpy()
+        assert rel_l2(sub, want[: M // 2]) < 2e-6
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_gemm_simt(env, dtype):
+    torch, dllm = env
+    M, N, K = 77, 200, 328
+    A = synth.random_normal((M, K), seed=1)
+    W = synth.random_normal((N, K), seed=2, std=0.05)
+    if dtype == "bf16":
+        A, W = synth.round_to_bf16(A), synth.round_to_bf16(W)
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    got = dllm.gemm_simt(torch.from_numpy(A).cuda().to(td), torch.from_numpy(W).cuda().to(td)).cpu().numpy()
+    want = A.astype(np.float64) @ W.astype(np.float64).T
+    assert rel_l2(got, want) < 2e-6
+
+
+ATT_CASES = [
+    # B, a, n, H, Hkv, hd
+    (1, 8, 96, 4, 4, 64),      # tiny configuration, partial step
+    (2, 19, 77, 5, 5, 64),     # ragged queries and keys
+    (1, 3, 300, 4, 4, 128),    # few queries, longer keys
+    (2, 33, 130, 7, 1, 64),    # GQA, 7 query heads per KV head
+    (1, 64, 768, 8, 8, 128),   # LLaDA-8B partial-step shape, 8 of the 32 heads
+    (1, 128, 512, 28, 4, 128), # Dream-7B partial-step shape
+]
+
+
+@pytest.mark.parametrize("case", ATT_CASES)
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_attention(env, case, dtype):
+    torch, dllm = env
+    B, a, n, H, Hkv, hd = case
+    q = synth.random_normal((B * a, H * hd), seed=11, std=1.3)
+    k = synth.random_normal((B, n, Hkv * hd), seed=12, std=1.3)
+    v = synth.random_normal((B, n, Hkv * hd), seed=13)
+    if dtype == "bf16":
+        q, k, v = (synth.round_to_bf16(t) for t in (q, k, v))
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    got = dllm.attention(*(torch.from_numpy(t).cuda().to(td) for t in (q, k, v)), B, a, n, H, Hkv, hd)
+    got = got.to(torch.float32).cpu().numpy()
+    for b in range(B):
+        want = O.attention(q[b * a:(b + 1) * a].astype(np.float64).reshape(a, H, hd),
+                           k[b].astype(np.float64).reshape(n, Hkv, hd),
+                           v[b].astype(np.float64).reshape(n, Hkv, hd), Hkv)
+        tol = 1e-5 if dtype == "fp32" else 8e-3       # bf16: output rounding 2^-9 plus P rounded to bf16
+        assert rel_l2(got[b * a:(b + 1) * a], want) < tol
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("B,R,width,k", [(1, 32, 256, 8), (3, 256, 4096, 64), (2, 100, 512, 50), (1, 512, 4096, 51)])
+def test_vverify_select(env, dtype, B, R, width, k):
+    torch, dllm = env
+    cache = synth.random_normal((B, R, width), seed=5)
+    noise = synth.random_normal((B, R, width), seed=6)
+    amp = synth.random_uniform((B, R, 1), seed=7) ** 4            # most rows barely move, a few move a lot
+    new = cache + amp * noise
+    new[:, ::3] = cache[:, ::3]                                     # a third of the rows are exactly unchanged
+    if dtype == "bf16":
+        cache, new = synth.round_to_bf16(cache), synth.round_to_bf16(new)
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    d_new = torch.from_numpy(new).cuda().to(td)
+    d_cache = torch.from_numpy(cache).cuda().to(td)
+    sim, idx = dllm.vverify_select(d_new, d_cache, k)
+    torch.cuda.synchronize()
+    sim, idx = sim.cpu().numpy(), idx.cpu().numpy()
+    assert torch.equal(d_cache, d_new)                              # whole V overwritten
+    for b in range(B):
+        s = O.cosine_rows(new[b].astype(np.float64), cache[b].astype(np.float64))
+        np.testing.assert_allclose(sim[b], s, atol=2e-6)
+        assert (sim[b, ::3] == 1.0).all()                           # unchanged rows give exactly 1
+        want = O.select_lowest(s, k)
+        assert list(idx[b]) == sorted(idx[b]) and len(set(idx[b].tolist())) == k
+        assert selection_matches(idx[b], want, s)
+        # the kernel's own similarities, sorted by the same key, must give exactly its set
+        keys = sorted((int(np.rint(float(sim[b, j]) * 2 ** 20)), j) for j in range(R))
+        assert idx[b].tolist() == sorted(j for _, j in keys[:k])

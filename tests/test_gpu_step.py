@@ -1,0 +1,232 @@
+"""Step-level parity on the GPU: the cached denoising step, the transition and
+the generation loop, called through the C ABI and compared with the CPU oracle
+on the same seeded weights and prompts.
+
+Tolerances (relative L2 of the response hidden states): 1e-4 in fp32 mode,
+2e-2 in bf16 mode.  Selected index sets must match exactly except for tokens
+within 1e-3 of the k-th similarity; to tell a legal tie flip from an arithmetic
+fault the bf16 runs are repeated with the oracle's sets forced into the GPU
+path."""
+import numpy as np
+import pytest
+
+from oracle import dllm_oracle as O
+from paper_2506_06295_b200 import synth
+from tests.helpers import rel_l2, selection_matches
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2506_06295_b200 import build as build_mod
+    build_mod.build()
+    from paper_2506_06295_b200 import dllm
+    assert torch.cuda.is_available()
+    return torch, dllm
+
+
+def make_pair(dllm, cfg, B, P, R, odtype=np.float64, seed=synth.WEIGHT_SEED):
+    w = synth.make_weights(cfg, seed)
+    prompt = synth.make_prompt(cfg, B, P)
+    orc = O.DLLMOracle(cfg, w, B, P, R, dtype=odtype)
+    orc.set_prompt(prompt)
+    model = dllm.Model(cfg).load(w)
+    ses = dllm.Session(model, B, P, R)
+    ses.set_prompt(prompt)
+    return orc, ses, w
+
+
+def unmask(orc, ses, step, count):
+    """Unmask `count` response tokens per sequence in both implementations."""
+    P = orc.P
+    resp = orc.tokens[:, P:].copy()
+    for b in range(orc.B):
+        masked = np.nonzero(resp[b] == orc.cfg.mask_id)[0]
+        pick = masked[(np.arange(count) * 7 + 3 * step + b) % max(len(masked), 1)] if len(masked) else []
+        for j in pick:
+            resp[b, j] = (31 * j + 5 * step + b) % (orc.cfg.vocab - 1)
+    orc.tokens[:, P:] = resp
+    ses.set_response_tokens(resp)
+
+
+def compare_step(orc, ses, r, tol, check_sets=True, what=""):
+    ses.sync()
+    hid = ses.hidden()
+    err = rel_l2(hid, r.hidden)
+    assert err < tol, f"{what}: hidden rel-L2 {err:.3e} >= {tol}"
+    for l in range(orc.cfg.n_layers):
+        idx, sim = ses.selected(l)
+        assert idx.shape == r.selected[l].shape, what
+        if check_sets:
+            for b in range(orc.B):
+                assert selection_matches(idx[b], r.selected[l][b], None if r.sim[l] is None else r.sim[l][b]), \
+                    f"{what}: layer {l} seq {b}: {idx[b].tolist()} vs {r.selected[l][b].tolist()}"
+        if r.sim[l] is not None:
+            np.testing.assert_allclose(sim, r.sim[l], atol=5e-3 if tol > 1e-3 else 2e-5)
+    return err
+
+
+def compare_caches(dllm, orc, ses, tol, what=""):
+    for l in range(orc.cfg.n_layers):
+        for which, ref in ((dllm.CACHE_K, orc.Kc), (dllm.CACHE_V, orc.Vc), (dllm.CACHE_ATTN, orc.Ac),
+                           (dllm.CACHE_FFN, orc.Fc)):
+            err = rel_l2(ses.get_cache(l, which), ref[l])
+            assert err < tol, f"{what}: cache {which} layer {l}: {err:.3e}"
+
+
+# ---------------------------------------------------------------- tiny fp32 configuration
+def test_tiny_fp32_all_step_kinds(env):
+    torch, dllm = env
+    wl = synth.WORKLOADS["tiny"]
+    orc, ses, _ = make_pair(dllm, wl.model, 2, wl.prompt_len, wl.gen_len)
+    r = orc.step(True, True)
+    ses.step_full()
+    compare_step(orc, ses, r, 1e-4, what="full")
+    compare_caches(dllm, orc, ses, 1e-4, "full")
+    x0, conf = ses.pred()
+    assert np.array_equal(x0, r.x0)
+    np.testing.assert_allclose(conf, r.conf, rtol=1e-3)
+    lg = ses.logits()
+    fin = np.isfinite(r.logits)
+    assert np.array_equal(np.isfinite(lg), fin)
+    assert rel_l2(lg[fin], r.logits[fin]) < 1e-4
+    step = 0
+    for rp, rr, rho in ((False, False, 0.25), (False, True, 0.0), (False, False, 0.25), (True, False, 0.25),
+                        (False, False, 0.5), (False, False, 0.0), (True, True, 0.0), (False, False, 1.0)):
+        step += 1
+        unmask(orc, ses, step, 4)
+        r = orc.step(rp, rr, rho)
+        ses.step_cached(rp, rr, rho)
+        compare_step(orc, ses, r, 1e-4, what=f"step {step} ({rp},{rr},{rho})")
+        compare_caches(dllm, orc, ses, 1e-4, f"step {step}")
+        x0, conf = ses.pred()
+        assert np.array_equal(x0, r.x0)
+
+
+def test_tiny_fp32_generation_matches_token_for_token(env):
+    torch, dllm = env
+    wl = synth.WORKLOADS["tiny"]
+    orc, ses, _ = make_pair(dllm, wl.model, 1, wl.prompt_len, wl.gen_len)
+    want = orc.generate(wl.steps, wl.Kp, wl.Kr, wl.rho, wl.block_len)
+    ses.generate(wl.steps, wl.Kp, wl.Kr, wl.rho, wl.block_len)
+    ses.sync()
+    got = ses.tokens()
+    assert (got[:, wl.prompt_len:] != wl.model.mask_id).all()
+    assert np.array_equal(got, want)
+
+
+def test_tiny_fp32_stepwise_generation_with_graphs_off_and_on(env):
+    torch, dllm = env
+    wl = synth.WORKLOADS["tiny"]
+    outs = []
+    for graphs in (False, True):
+        orc, ses, _ = make_pair(dllm, wl.model, 1, wl.prompt_len, wl.gen_len)
+        ses.use_graphs(graphs)
+        for k in range(wl.steps, 0, -1):
+            ses.step_scheduled(k, wl.steps, wl.Kp, wl.Kr, wl.rho)
+            bs, nt = O.block_plan(wl.steps - k, wl.steps, wl.gen_len, wl.block_len)
+            ses.remask_low_confidence(bs, wl.block_len, nt)
+        ses.sync()
+        outs.append((ses.tokens(), ses.hidden(), ses.launch_count()))
+    assert np.array_equal(outs[0][0], outs[1][0])
+    assert np.array_equal(outs[0][1], outs[1][1])
+    assert outs[0][2] == outs[1][2] > 0
+
+
+# ---------------------------------------------------------------- bf16, several tiles and ragged tails
+@pytest.mark.parametrize("gqa", [False, True], ids=["mha", "gqa"])
+@pytest.mark.parametrize("simt", [True, False], ids=["simt_gemm", "tcgen05_gemm"])
+def test_small_bf16_step_kinds(env, gqa, simt):
+    torch, dllm = env
+    cfg = synth.small_bf16_model(gqa=gqa)
+    B, P, R = 2, 150, 72
+    orc, ses, _ = make_pair(dllm, cfg, B, P, R)
+    ses.use_simt_gemm(simt)
+    r = orc.step(True, True)
+    ses.step_full()
+    compare_step(orc, ses, r, 2e-2, what="full")
+    compare_caches(dllm, orc, ses, 2e-2, "full")
+    step = 0
+    for rp, rr, rho in ((False, False, 0.25), (False, False, 0.25), (False, True, 0.0), (True, False, 0.5),
+                        (False, False, 0.1), (False, False, 0.0)):
+        step += 1
+        unmask(orc, ses, step, 3)
+        r = orc.step(rp, rr, rho)
+        # free-running comparison first ...
+        ses.step_cached(rp, rr, rho)
+        ses.sync()
+        free_ok = all(selection_matches(ses.selected(l)[0][b], r.selected[l][b],
+                                        None if r.sim[l] is None else r.sim[l][b])
+                      for l in range(cfg.n_layers) for b in range(B))
+        assert free_ok, f"step {step}: selection differs beyond the tie tolerance"
+        err = compare_step(orc, ses, r, 2e-2, what=f"step {step} ({rp},{rr},{rho})")
+        compare_caches(dllm, orc, ses, 2e-2, f"step {step}")
+        assert err < 2e-2
+
+
+def test_small_bf16_forced_selection_and_rho_invariants(env):
+    torch, dllm = env
+    cfg = synth.small_bf16_model()
+    B, P, R = 1, 100, 40
+    orc, ses, _ = make_pair(dllm, cfg, B, P, R)
+    orc.step(True, True)
+    ses.step_full()
+    unmask(orc, ses, 1, 2)
+    # forced sets (deliberately NOT the V-verify choice) reach both implementations
+    forced = {l: np.array([[1 + l, 7, 20, 33]]) for l in range(cfg.n_layers)}
+    r = orc.step(False, False, 0.1, forced=forced)
+    for l in range(cfg.n_layers):
+        ses.force_selection(l, forced[l])
+    ses.step_cached(False, False, 0.1)
+    compare_step(orc, ses, r, 2e-2, what="forced")
+    compare_caches(dllm, orc, ses, 2e-2, "forced")
+    for l in range(cfg.n_layers):
+        ses.force_selection(l, None)
+    # rho = 0 leaves every cache bit-unchanged (fully cached state)
+    before = [ses.get_cache(l, w) for l in range(cfg.n_layers) for w in range(4)]
+    unmask(orc, ses, 2, 2)
+    ses.step_cached(False, False, 0.0)
+    ses.sync()
+    after = [ses.get_cache(l, w) for l in range(cfg.n_layers) for w in range(4)]
+    assert all(np.array_equal(a, b) for a, b in zip(before, after))
+    # rho = 1 equals a response refresh, bit for bit (same kernels, same rows)
+    snap = [ses.get_cache(l, w) for l in range(cfg.n_layers) for w in range(4)]
+    ses.step_cached(False, False, 1.0)
+    ses.sync()
+    h1 = ses.hidden()
+    c1 = [ses.get_cache(l, w) for l in range(cfg.n_layers) for w in range(4)]
+    for i, (l, w) in enumerate((l, w) for l in range(cfg.n_layers) for w in range(4)):
+        ses.set_cache(l, w, snap[i])
+    ses.step_cached(False, True, 0.0)
+    ses.sync()
+    assert np.array_equal(ses.hidden(), h1)
+    assert all(np.array_equal(a, ses.get_cache(l, w)) for a, (l, w) in
+               zip(c1, ((l, w) for l in range(cfg.n_layers) for w in range(4))))
+
+
+def test_error_paths_on_device(env):
+    torch, dllm = env
+    cfg = synth.TINY
+    model = dllm.Model(cfg).load(synth.make_weights(cfg))
+    ses = dllm.Session(model, 1, 64, 32)
+    ses.set_prompt(synth.make_prompt(cfg, 1, 64))
+    with pytest.raises(dllm.DllmError) as e:
+        ses.step_cached(False, False, 0.25)
+    assert e.value.status == dllm.BAD_STATE
+    with pytest.raises(dllm.DllmError) as e:
+        ses.remask_low_confidence(0, 32, 4)
+    assert e.value.status == dllm.BAD_STATE
+    ses.step_full()
+    for bad in (-0.1, 1.5, float("nan")):
+        with pytest.raises(dllm.DllmError) as e:
+            ses.step_cached(False, False, bad)
+        assert e.value.status == dllm.INVALID_ARG
+    with pytest.raises(dllm.DllmError):
+        ses.remask_low_confidence(16, 32, 4)
+    with pytest.raises(dllm.DllmError):
+        ses.generate(8, 4, 2, 0.25, 5)
+    with pytest.raises(dllm.DllmError):
+        ses.set_prompt(np.full((1, 64), 5000))
+    ses.sync()
