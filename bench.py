@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the cached denoising step on one B200 (replicas on N GPUs).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llada8b] [--impl reference]
+
+A "step" is one pass of the whole hot path over one batch: one denoising step
+under the dLLM-Cache schedule (full / response-refresh / mixed / adaptive
+partial, as the step index decides) followed by the low-confidence transition.
+The default workload is the LLaDA-8B-shaped configuration: batch 1, prompt 512,
+generation 256 in blocks of 32, 256 steps, K_p = 100, K_r = 6, rho = 0.25,
+random-init bf16 weights, uniform random prompt ids (synthetic stand-in for the
+paper's benchmark prompts).  `--steps K` times the first K steps of that
+schedule (it wraps into a new generation after 256).
+
+Prints ONE JSON line.  value = generated tokens/s with everything resident in
+HBM; e2e = the same loop driven through host buffers (token state copied
+host->device before and device->host after every step).  --impl reference
+times the CPU oracle instead (host cores, bounded sample).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2506_06295_b200 import synth  # noqa: E402
+
+METRIC = "generated tokens/s, cached denoising steps (dLLM-Cache schedule)"
+
+
+def schedule_kind(k, K, Kp, Kr):
+    rp = (k == K) or (k % Kp == 0)
+    rr = (k == K) or (k % Kr == 0)
+    return rp, rr, ("full" if rp and rr else "refresh" if rr else "mixed" if rp else "partial")
+
+
+def block_plan(t, K, R, block_len):
+    blocks = R // block_len
+    spb = K // blocks
+    blk = min(t // spb, blocks - 1)
+    i = t - blk * spb
+    return blk * block_len, block_len // spb + (1 if i < block_len % spb else 0)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs (read-only query)."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [r.split(",") for r in open(self.path).read().strip().splitlines() if r.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm, reasons = [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1]))
+                out["sm_max_mhz"] = float(r[2])
+            except ValueError:
+                continue
+            for nm, v in zip(names, r[5:9]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(nm)
+        if sm:
+            out["sm_mhz"] = float(np.median(sm))
+        out["reasons"] = sorted(reasons)
+        out["samples"] = len(sm)
+        return out
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ----------------------------------------------------------------------------------------------
+def time_oracle(wl, budget_s: float, steps: int | None = None):
+    """Times the oracle, as it stands, on the host cores on a bounded sample of
+    the workload: the same widths, sequence lengths and schedule, but a
+    2-layer model, float32 numpy; per-kind step times are extrapolated to the
+    full depth as (t_kind - t_head) * T/2 + t_head, the LM head timed by
+    calling the oracle's own projection on the same rows."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import dllm_oracle as O
+    cores = len(os.sched_getaffinity(0))
+    Tsample = 2
+    cfg = wl.model.with_layers(Tsample)
+    names = synth.tensor_names(cfg)
+    with ThreadPoolExecutor(max_workers=min(8, cores)) as ex:
+        w = dict(zip([n for n, _ in names], ex.map(lambda ns: synth.make_tensor(cfg, ns[0], ns[1]), names)))
+    orc = O.DLLMOracle(cfg, w, wl.batch, wl.prompt_len, wl.gen_len, dtype=np.float32)
+    orc.set_prompt(synth.make_prompt(cfg, wl.batch, wl.prompt_len))
+    times = {}
+    t_start = time.perf_counter()
+    K = wl.steps
+    order = []
+    for k in range(K, 0, -1):          # first occurrence of each kind, in schedule order
+        kind = schedule_kind(k, K, wl.Kp, wl.Kr)[2]
+        if kind not in [o[1] for o in order]:
+            order.append((k, kind))
+    done_steps = 0
+    for k, kind in order:
+        rp, rr, _ = schedule_kind(k, K, wl.Kp, wl.Kr)
+        t0 = time.perf_counter()
+        r = orc.step(rp, rr, wl.rho)
+        bs, nt = block_plan(K - k, K, wl.gen_len, wl.block_len)
+        orc.remask(bs, wl.block_len, nt)
+        times[kind] = time.perf_counter() - t0
+        done_steps += 1
+        if time.perf_counter() - t_start > budget_s and "partial" in times:
+            break
+    # LM head alone (the oracle's own projection + greedy estimate), to extrapolate depth correctly
+    z = O.rmsnorm(r.hidden[0].astype(np.float32), w["norm_f"], cfg.rms_eps)
+    t0 = time.perf_counter()
+    for _ in range(wl.batch):
+        lg = orc._lin(z, "lm_head", "lm_head")
+        lg.argmax(-1)
+        np.exp(lg - lg.max(-1, keepdims=True)).sum(-1)
+    t_head = time.perf_counter() - t0
+    T = wl.model.n_layers
+    full_depth = {kind: max(t - t_head, 0.0) * (T / Tsample) + t_head for kind, t in times.items()}
+    counts = {}
+    n_steps = steps if steps is not None else K
+    for i in range(n_steps):
+        kind = schedule_kind(K - (i % K), K, wl.Kp, wl.Kr)[2]
+        counts[kind] = counts.get(kind, 0) + 1
+    fallback = full_depth.get("full", max(full_depth.values()))
+    total = sum(c * full_depth.get(kind, fallback) for kind, c in counts.items())
+    tokens = n_steps * wl.batch * wl.gen_len / K
+    return {"tokens_per_s": tokens / total, "cores": cores, "ms_per_step": 1e3 * total / n_steps,
+            "per_kind_s_full_depth": {k: round(v, 3) for k, v in full_depth.items()},
+            "sample": (f"{Tsample}-layer model at full width ({cfg.d_model}/{cfg.d_ffn}/{cfg.vocab}), B={wl.batch} "
+                       f"P={wl.prompt_len} R={wl.gen_len}, float32 numpy, one step of each kind "
+                       f"({', '.join(times)}) + LM head timed separately, extrapolated to {T} layers over "
+                       f"{n_steps} scheduled steps"),
+            "cpu_seconds": round(time.perf_counter() - t_start, 1)}
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    t = time_oracle(wl, budget_s=90.0, steps=args.steps)
+    line = {"impl": "reference", "metric": METRIC, "value": t["tokens_per_s"], "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": t["ms_per_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(wl, args),
+            "cpu_baseline": {"value": t["tokens_per_s"], "unit": "tokens/s", "cores": t["cores"], "kind": "oracle",
+                             "sample": t["sample"]},
+            "e2e": {"value": t["tokens_per_s"], "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "per_kind_s": t["per_kind_s_full_depth"]}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl, args):
+    c = wl.model
+    return {"workload": f"{wl.name}: {c.n_layers} layers, d={c.d_model}, {c.n_heads}x{c.head_dim} heads "
+                        f"({c.n_kv_heads} KV), FFN {c.d_ffn}, vocab {c.vocab}; batch {wl.batch}, prompt "
+                        f"{wl.prompt_len}, generation {wl.gen_len} in blocks of {wl.block_len}, {wl.steps} steps",
+            "Kp": wl.Kp, "Kr": wl.Kr, "rho": wl.rho, "k_round": "floor",
+            "l2": "inputs larger than L2: every step streams all layer weights (>= 14 GB) through the 126 MB L2",
+            "replicas": args.gpus}
+
+
+# ----------------------------------------------------------------------------------------------
+# the CUDA arm
+# ----------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llada8b", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--full-steps", type=int, default=6, help="timed full-recompute steps for the speedup figure")
+    args = ap.parse_args()
+    wl = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2506_06295_b200 import build as build_mod
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank == 0:
+        build_mod.build()
+    if world > 1:
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    from paper_2506_06295_b200 import dllm
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    cfg = wl.model
+    K, W = args.steps, max(args.warmup, 3)
+
+    model = dllm.Model(cfg, device=dev).random_init_on_device(synth.WEIGHT_SEED + rank)
+    ses = dllm.Session(model, wl.batch, wl.prompt_len, wl.gen_len)
+    prompt = synth.make_prompt(cfg, wl.batch, wl.prompt_len, seed=1 + 1000 * rank)
+    ses.set_prompt(prompt)
+    stream = ses.stream
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def run_steps(n, per_step=None):
+        for i in range(n):
+            k = wl.steps - (i % wl.steps)
+            if i and k == wl.steps:
+                ses.set_prompt(prompt)          # a new generation starts
+            ses.step_scheduled(k, wl.steps, wl.Kp, wl.Kr, wl.rho)
+            bs, nt = block_plan(wl.steps - k, wl.steps, wl.gen_len, wl.block_len)
+            ses.remask_low_confidence(bs, wl.block_len, nt)
+            if per_step:
+                per_step(i)
+
+    # warm-up: every step kind W times (also instantiates the CUDA graphs)
+    ses.step_full()
+    for _ in range(W):
+        for rp, rr in ((True, True), (True, False), (False, True), (False, False)):
+            ses.step_cached(rp, rr, wl.rho)
+    ses.sync()
+    ses.set_prompt(prompt)
+
+    # ---- timed region: K steps, everything resident ------------------------------------------
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = ses.launch_count()
+    ev0.record(stream)
+    run_steps(K)
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = ses.launch_count() - l0
+    ses.sync()
+    final_tokens = ses.tokens()
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- per-kind step times and the full-recompute baseline of the same library -------------
+    def time_kind(rp, rr, reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(dev)
+        a.record(stream)
+        for _ in range(reps):
+            ses.step_cached(rp, rr, wl.rho)
+        b.record(stream)
+        torch.cuda.synchronize(dev)
+        return a.elapsed_time(b) / reps
+    per_kind = {"full": time_kind(True, True, args.full_steps), "refresh": time_kind(False, True, 6),
+                "mixed": time_kind(True, False, 6), "partial": time_kind(False, False, 12)}
+
+    # ---- end to end through host buffers ---------------------------------------------------------
+    ses.set_prompt(prompt)
+    host_tok = torch.empty((wl.batch, wl.gen_len), dtype=torch.int32).pin_memory()
+    host_tok.fill_(cfg.mask_id)
+    host_np = host_tok.numpy()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+
+    def roundtrip(i):
+        out = ses.tokens()                                  # device -> host: the step's result
+        host_np[...] = out[:, wl.prompt_len:]
+    for i in range(K):
+        k = wl.steps - (i % wl.steps)
+        if i and k == wl.steps:
+            ses.set_prompt(prompt)
+            host_np[...] = cfg.mask_id
+        ses.set_response_tokens(host_np)                    # host -> device: this step's token state
+        ses.step_scheduled(k, wl.steps, wl.Kp, wl.Kr, wl.rho)
+        bs, nt = block_plan(wl.steps - k, wl.steps, wl.gen_len, wl.block_len)
+        ses.remask_low_confidence(bs, wl.block_len, nt)
+        roundtrip(i)
+    e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+
+    # ---- per-kernel times: same K steps, launched kernel by kernel with event pairs --------------
+    ses.set_prompt(prompt)
+    ses.profile(True)
+    run_steps(K)
+    ses.sync()
+    g = ses.profile_read(0)
+    at = ses.profile_read(1)
+    ses.profile(False)
+
+    # max over ranks
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    tokens = K * wl.batch * wl.gen_len / wl.steps * world       # one token per sequence per step on this schedule
+    value = tokens / (ms / 1e3)
+    gemm_gbs = g["bytes"] / (g["ms"] / 1e3) / 1e9 if g["ms"] > 0 else 0.0
+    counts = {}
+    for i in range(K):
+        kind = schedule_kind(wl.steps - (i % wl.steps), wl.steps, wl.Kp, wl.Kr)[2]
+        counts[kind] = counts.get(kind, 0) + 1
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": workload_config(wl, args),
+        "steps_per_s": K * world / (ms / 1e3),
+        "step_kinds": counts,
+        "ms_per_kind": {k: round(v, 4) for k, v in per_kind.items()},
+        "speedup_vs_full_recompute": per_kind["full"] / (ms / K),
+        "full_recompute_tokens_per_s": wl.batch * wl.gen_len / wl.steps * world / (per_kind["full"] / 1e3),
+        "e2e": {"value": tokens / (ms_e2e / 1e3), "unit": "tokens/s",
+                "h2d_bytes_per_step": wl.batch * wl.gen_len * 4, "d2h_bytes_per_step": wl.batch * (wl.prompt_len + wl.gen_len) * 4},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"kernel": "gemm_bf16_tcgen05_kernel", "bound": "hbm", "achieved": gemm_gbs,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"],
+                     "peak_source": peaks["source"], "traffic": TRAFFIC_PER_LAUNCH.get(args.workload),
+                     "launches": g["launches"], "avg_launch_us": 1e3 * g["ms"] / max(g["launches"], 1),
+                     "algorithmic_bytes_per_launch": g["bytes"] / max(g["launches"], 1),
+                     "gemm_share_of_step": g["ms"] / max(ms, 1e-9),
+                     "attention": {"ms_total": at["ms"], "launches": at["launches"],
+                                   "gbs": at["bytes"] / (at["ms"] / 1e3) / 1e9 if at["ms"] > 0 else 0.0,
+                                   "tflops": at["flops"] / (at["ms"] / 1e3) / 1e12 if at["ms"] > 0 else 0.0},
+                     "how": "CUDA-event pairs around every GEMM launch in a kernel-by-kernel replay of the same K steps"},
+        "unmasked_tokens": int((final_tokens[:, wl.prompt_len:] != cfg.mask_id).sum()),
+    }
+    if not args.no_cpu_baseline:
+        t = time_oracle(wl, budget_s=25.0, steps=K)
+        line["cpu_baseline"] = {"value": t["tokens_per_s"], "unit": "tokens/s", "cores": t["cores"], "kind": "oracle",
+                                "sample": t["sample"]}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch from the ncu capture summarised under
+# profiles/ (average over the captured launches, scaled where stated there); None until captured.
+TRAFFIC_PER_LAUNCH = {}
+
+if __name__ == "__main__":
+    main()

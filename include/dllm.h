@@ -176,6 +176,16 @@ uint64_t dllm_launch_count(const dllm_session* s);
  * 0: launch kernels one by one. */
 dllm_status dllm_session_use_graphs(dllm_session* s, int enable);
 
+/* Per-kernel timing.  While enabled, steps are launched kernel by kernel (no
+ * graph replay) and every projection GEMM (class 0) and attention launch
+ * (class 1) is bracketed by CUDA events on the caller's stream.  _profile_read
+ * synchronises the device and returns, for one class, the summed event time,
+ * the number of launches, and the algorithmic bytes and FLOPs of those launches
+ * (GEMM: W and A once in, one fp32 result out; attention: K, V, Q in, O out).
+ * Enabling or disabling discards earlier records. */
+dllm_status dllm_session_profile(dllm_session* s, int enable);
+dllm_status dllm_session_profile_read(dllm_session* s, int cls, double* total_ms, uint64_t* launches,
+                                      double* algorithmic_bytes, double* flops);
 /* Test hook: 1 runs the bf16 GEMMs of the step on the plain-ALU kernel instead
  * of the tensor-core kernel (to localise a fault); default 0. */
 dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable);

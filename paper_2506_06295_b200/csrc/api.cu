@@ -195,6 +195,35 @@ struct dllm_session {
   };
   std::map<StepKey, GraphEntry> graphs;
   std::string err;
+  // profiling: event pairs around GEMM (class 0) and attention (class 1) launches
+  struct ProfRec {
+    int cls;
+    cudaEvent_t a, b;
+    double bytes, flops;
+  };
+  bool profiling = false;
+  std::vector<ProfRec> prof;
+  std::vector<cudaEvent_t> event_pool;
+  cudaEvent_t take_event() {
+    if (!event_pool.empty()) {
+      cudaEvent_t e = event_pool.back();
+      event_pool.pop_back();
+      return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+  }
+  void prof_begin(int cls, double bytes, double flops, cudaStream_t st) {
+    if (!profiling) return;
+    ProfRec r{cls, take_event(), take_event(), bytes, flops};
+    cudaEventRecord(r.a, st);
+    prof.push_back(r);
+  }
+  void prof_end(cudaStream_t st) {
+    if (!profiling) return;
+    cudaEventRecord(prof.back().b, st);
+  }
 
   size_t es() const { return esize(m->cfg); }
   size_t dkv() const { return (size_t)m->cfg.n_kv_heads * m->cfg.head_dim; }
@@ -252,6 +281,15 @@ dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void
   out->split_stride = (size_t)M * N;
   out->S = 1;
   if (M <= 0) return DLLM_OK;
+  // algorithmic traffic of one projection: the weight matrix and the activation
+  // rows once in, one fp32 result out (split-K slabs are overhead, not counted)
+  const double es = (double)s->es();
+  s->prof_begin(0, ((double)N * K + (double)M * K) * es + (double)M * N * 4.0, 2.0 * M * N * K, L.stream);
+  struct End {
+    dllm_session* s;
+    cudaStream_t st;
+    ~End() { s->prof_end(st); }
+  } end_guard{s, L.stream};
   if (s->m->cfg.dtype == DLLM_FP32 || s->simt_gemm) {
     launch_gemm_simt(L, s->m->cfg.dtype, A, W, part, M, N, K);
     return DLLM_OK;
@@ -317,9 +355,12 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
       if ((st = run_gemm(s, L, ua, Wq, Ma, dq + dkv, d, &part)) != DLLM_OK) return st;
       launch_qk_rope(L, dt, part, act, s->wsp<float>(s->ws.rope), s->wsp<uint8_t>(s->ws.qbuf),
                      s->cache(l, DLLM_CACHE_K), g, Ma, H, Hkv, hd);
+      // algorithmic traffic: K and V of every sequence once, Q in, O out
+      s->prof_begin(1, (2.0 * s->B * s->n * dkv + 2.0 * Ma * dq) * (double)es, 4.0 * Ma * (double)s->n * dq, stream);
       cudaError_t e = launch_attention(L, dt, s->wsp<uint8_t>(s->ws.qbuf), s->cache(l, DLLM_CACHE_K),
                                        s->cache(l, DLLM_CACHE_V), s->wsp<uint8_t>(s->ws.obuf), s->B, a_seq, s->n, H,
                                        Hkv, hd);
+      s->prof_end(stream);
       if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.obuf), W + lo.wo, Ma, d, dq, &part)) != DLLM_OK) return st;
       launch_oproj_epilogue(L, dt, part, act, x, reinterpret_cast<const float*>(W + lo.norm2),
@@ -362,7 +403,7 @@ dllm_status run_step(dllm_session* s, int rp, int rr, float rho, dllm_kround kr,
                     s->forced_count[l], ksel);
   cudaStream_t stream = (cudaStream_t)stream_v;
   dllm_status st = DLLM_OK;
-  const bool graph_ok = s->use_graphs && stream != nullptr && stream != cudaStreamLegacy;
+  const bool graph_ok = s->use_graphs && !s->profiling && stream != nullptr && stream != cudaStreamLegacy;
   if (!graph_ok) {
     st = enqueue_step(s, rp, rr, ksel, stream);
   } else {
@@ -525,6 +566,11 @@ dllm_status dllm_session_create(dllm_model* m, int B, int P, int R, void* d_cach
 dllm_status dllm_session_destroy(dllm_session* s) {
   if (!s) return DLLM_OK;
   for (auto& kv : s->graphs) cudaGraphExecDestroy(kv.second.exec);
+  for (auto& r : s->prof) {
+    cudaEventDestroy(r.a);
+    cudaEventDestroy(r.b);
+  }
+  for (auto e : s->event_pool) cudaEventDestroy(e);
   delete s;
   return DLLM_OK;
 }
@@ -759,6 +805,41 @@ dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable) {
     s->graphs.clear();
   }
   s->simt_gemm = enable != 0;
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_profile(dllm_session* s, int enable) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  CU_TRY(&s->err, cudaDeviceSynchronize());
+  for (auto& r : s->prof) {
+    s->event_pool.push_back(r.a);
+    s->event_pool.push_back(r.b);
+  }
+  s->prof.clear();
+  s->profiling = enable != 0;
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_profile_read(dllm_session* s, int cls, double* total_ms, uint64_t* launches,
+                                      double* algorithmic_bytes, double* flops) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (cls < 0 || cls > 1) return fail(&s->err, DLLM_INVALID_ARG, "class must be 0 (GEMM) or 1 (attention)");
+  CU_TRY(&s->err, cudaDeviceSynchronize());
+  double ms = 0, by = 0, fl = 0;
+  uint64_t cnt = 0;
+  for (auto& r : s->prof) {
+    if (r.cls != cls) continue;
+    float t = 0.f;
+    CU_TRY(&s->err, cudaEventElapsedTime(&t, r.a, r.b));
+    ms += t;
+    by += r.bytes;
+    fl += r.flops;
+    ++cnt;
+  }
+  if (total_ms) *total_ms = ms;
+  if (launches) *launches = cnt;
+  if (algorithmic_bytes) *algorithmic_bytes = by;
+  if (flops) *flops = fl;
   return DLLM_OK;
 }
 

@@ -66,6 +66,9 @@ SIGNATURES = {
     "dllm_launch_count": (C.c_uint64, [_P]),
     "dllm_session_use_graphs": (_I, [_P, _I]),
     "dllm_session_use_simt_gemm": (_I, [_P, _I]),
+    "dllm_session_profile": (_I, [_P, _I]),
+    "dllm_session_profile_read": (_I, [_P, _I, C.POINTER(C.c_double), C.POINTER(C.c_uint64),
+                                       C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "dllm_gemm_bf16_scratch_bytes": (_SZ, [_I, _I, _I]),
     "dllm_gemm_bf16": (_I, [_P, _P, _P, _I, _I, _I, _P, _P]),
     "dllm_gemm_simt": (_I, [_P, _P, _P, _I, _I, _I, _I, _P]),
@@ -293,6 +296,14 @@ class Session:
 
     def use_simt_gemm(self, enable: bool) -> None:
         _check(lib.dllm_session_use_simt_gemm(self.handle, int(enable)))
+
+    def profile(self, enable: bool) -> None:
+        _check(lib.dllm_session_profile(self.handle, int(enable)))
+
+    def profile_read(self, cls: int) -> dict:
+        ms, by, fl, cnt = C.c_double(), C.c_double(), C.c_double(), C.c_uint64()
+        _check(lib.dllm_session_profile_read(self.handle, cls, C.byref(ms), C.byref(cnt), C.byref(by), C.byref(fl)))
+        return {"ms": ms.value, "launches": cnt.value, "bytes": by.value, "flops": fl.value}
 
     def close(self):
         if getattr(self, "handle", None):
