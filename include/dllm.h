@@ -186,8 +186,8 @@ dllm_status dllm_session_use_graphs(dllm_session* s, int enable);
 dllm_status dllm_session_profile(dllm_session* s, int enable);
 dllm_status dllm_session_profile_read(dllm_session* s, int cls, double* total_ms, uint64_t* launches,
                                       double* algorithmic_bytes, double* flops);
-/* Test hook: 1 runs the bf16 GEMMs of the step on the plain-ALU kernel instead
- * of the tensor-core kernel (to localise a fault); default 0. */
+/* Test hook: 1 runs the bf16 GEMMs and attention of the step on the plain-ALU
+ * kernels instead of the tensor-core kernels (to localise a fault); default 0. */
 dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable);
 
 /* ---- kernel-level entry points (parity tests and micro-benchmarks) --------- */
@@ -202,10 +202,15 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
  * the fp32 mode. */
 dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int dtype,
                            void* stream);
-/* Non-causal attention of `a` query rows per sequence over n cached keys.
- * d_q [B*a, H*hd], d_k / d_v [B, n, Hkv*hd], d_o [B*a, H*hd]; dtype as above. */
+/* Non-causal attention of `a` query rows per sequence over n cached keys
+ * (Sec. A.7, the 4 r n d term).  d_q [B*a, H*hd], d_k / d_v [B, n, Hkv*hd], d_o
+ * [B*a, H*hd]; dtype as above.  bf16 with head_dim 64 or 128 runs on the tensor
+ * cores and, when few rows are active, splits the key range over CTAs; the
+ * partial results of the splits go to d_scratch (device,
+ * dllm_attention_scratch_bytes(); with less the key range is not split). */
+size_t dllm_attention_scratch_bytes(int B, int a, int n, int H, int Hkv, int hd, int dtype);
 dllm_status dllm_attention(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B, int a, int n,
-                           int H, int Hkv, int hd, int dtype, void* stream);
+                           int H, int Hkv, int hd, int dtype, void* d_scratch, size_t scratch_bytes, void* stream);
 /* V-verify + selection alone (Eq. 6 and the bottom-k rule): d_vnew, d_vcache
  * [B, R, width] in `dtype`; writes d_sim float [B, R] and d_idx int32 [B, k]
  * ascending; overwrites d_vcache with d_vnew. */

@@ -114,8 +114,8 @@ uint16_t f32_to_bf16_rne(float f) {
 
 // workspace carve-up
 struct Workspace {
-  size_t status, tokens, x, u, ua, qbuf, obuf, hn, ffn, x0, conf, sim, sel, forced, act, rope, part, total;
-  size_t part_floats;
+  size_t status, tokens, x, u, ua, qbuf, obuf, hn, ffn, x0, conf, sim, sel, forced, act, rope, attn, part, total;
+  size_t part_floats, attn_floats;
 };
 
 Workspace make_workspace(const dllm_config& c, int B, int P, int R) {
@@ -145,6 +145,10 @@ Workspace make_workspace(const dllm_config& c, int B, int P, int R) {
   w.forced = take(T * BR * 4);
   w.act = take(rows * 4);
   w.rope = take(n * c.head_dim * 4);
+  // partial outputs of split key ranges: splits happen only while fewer than
+  // 148 CTAs of 64 (row, head) pairs exist, so S * pairs < 2 * 148 * 64
+  w.attn_floats = (size_t)2 * 148 * 64 * (128 + 2);
+  w.attn = take(w.attn_floats * 4);
   // largest [M, N] any GEMM writes, plus room for split-K slabs of the small-M
   // launches: S*M*N <= M*N + 148 CTAs * 256 * 128 for every plan
   size_t mn = rows * std::max(std::max(dq + dkv, d), 2 * m);
@@ -264,6 +268,16 @@ dllm_status fail(std::string* slot, dllm_status st, const char* fmt, ...) {
     if (e_ != cudaSuccess) return fail(slot, DLLM_CUDA_ERROR, "%s: %s", #expr, cudaGetErrorString(e_)); \
   } while (0)
 
+// Host -> device copy ordered on the caller's stream and complete on return.
+// (A plain cudaMemcpy from pageable memory may return before its DMA has
+// finished and is ordered only against the legacy stream, so kernels enqueued
+// on a non-blocking stream afterwards could read stale data.)
+cudaError_t h2d(void* dst, const void* src, size_t bytes, cudaStream_t st) {
+  cudaError_t e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return e;
+  return cudaStreamSynchronize(st);
+}
+
 int k_selected(float rho, int R, dllm_kround kr) {
   const double v = (double)rho * (double)R;
   long k = kr == DLLM_K_CEIL ? (long)ceil(v - 1e-6) : (long)floor(v + 1e-6);
@@ -359,7 +373,7 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
       s->prof_begin(1, (2.0 * s->B * s->n * dkv + 2.0 * Ma * dq) * (double)es, 4.0 * Ma * (double)s->n * dq, stream);
       cudaError_t e = launch_attention(L, dt, s->wsp<uint8_t>(s->ws.qbuf), s->cache(l, DLLM_CACHE_K),
                                        s->cache(l, DLLM_CACHE_V), s->wsp<uint8_t>(s->ws.obuf), s->B, a_seq, s->n, H,
-                                       Hkv, hd);
+                                       Hkv, hd, s->wsp<float>(s->ws.attn), s->ws.attn_floats, s->simt_gemm);
       s->prof_end(stream);
       if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.obuf), W + lo.wo, Ma, d, dq, &part)) != DLLM_OK) return st;
@@ -502,6 +516,7 @@ dllm_status dllm_model_set_tensor(dllm_model* m, const char* name, const float* 
     return fail(&m->err, DLLM_INVALID_ARG, "tensor '%s' has %zu elements, got %zu", name, t.n, n_elements);
   if (t.f32 || m->cfg.dtype == DLLM_FP32) {
     CU_TRY(&m->err, cudaMemcpy(m->d_w + t.off, h_src, t.n * 4, cudaMemcpyHostToDevice));
+    CU_TRY(&m->err, cudaDeviceSynchronize());  // DMA from pageable memory has landed on return
     return DLLM_OK;
   }
   std::vector<uint16_t> tmp;
@@ -512,6 +527,7 @@ dllm_status dllm_model_set_tensor(dllm_model* m, const char* name, const float* 
   }
   for (size_t i = 0; i < t.n; ++i) tmp[i] = f32_to_bf16_rne(h_src[i]);
   CU_TRY(&m->err, cudaMemcpy(m->d_w + t.off, tmp.data(), t.n * 2, cudaMemcpyHostToDevice));
+  CU_TRY(&m->err, cudaDeviceSynchronize());
   return DLLM_OK;
 }
 
@@ -554,7 +570,7 @@ dllm_status dllm_session_create(dllm_model* m, int B, int P, int R, void* d_cach
   // everything but the (large) GEMM slab is cleared; the slab is always written before it is read
   if (e == cudaSuccess) e = cudaMemsetAsync(d_workspace, 0, s->ws.part, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-  if (e == cudaSuccess) e = cudaMemcpy(s->d_ws + s->ws.rope, tab.data(), tab.size() * 4, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = h2d(s->d_ws + s->ws.rope, tab.data(), tab.size() * 4, st);
   if (e != cudaSuccess) {
     delete s;
     return fail(&m->err, DLLM_CUDA_ERROR, "session setup: %s", cudaGetErrorString(e));
@@ -590,7 +606,7 @@ dllm_status dllm_session_set_prompt(dllm_session* s, const int32_t* h_prompt, vo
   }
   cudaStream_t st = (cudaStream_t)stream;
   CU_TRY(&s->err, cudaStreamSynchronize(st));
-  CU_TRY(&s->err, cudaMemcpy(s->d_ws + s->ws.tokens, tok.data(), tok.size() * 4, cudaMemcpyHostToDevice));
+  CU_TRY(&s->err, h2d(s->d_ws + s->ws.tokens, tok.data(), tok.size() * 4, st));
   s->valid = false;
   s->have_pred = false;
   return DLLM_OK;
@@ -651,7 +667,8 @@ dllm_status dllm_sync(dllm_session* s, void* stream) {
   int code = 0;
   CU_TRY(&s->err, cudaMemcpy(&code, s->d_ws + s->ws.status, 4, cudaMemcpyDeviceToHost));
   if (code == 0) return DLLM_OK;
-  cudaMemset(s->d_ws + s->ws.status, 0, 4);
+  cudaMemsetAsync(s->d_ws + s->ws.status, 0, 4, (cudaStream_t)stream);
+  cudaStreamSynchronize((cudaStream_t)stream);
   if (code >= 100 && code < 200) return fail(&s->err, DLLM_TIMEOUT, "a device-side wait gave up (code %d)", code);
   return fail(&s->err, DLLM_CUDA_ERROR, "device status %d", code);
 }
@@ -670,8 +687,10 @@ dllm_status dllm_set_response_tokens(dllm_session* s, const int32_t* h_tok, void
   for (size_t i = 0; i < (size_t)s->B * s->R; ++i)
     if (h_tok[i] < 0 || h_tok[i] >= s->m->cfg.vocab) return fail(&s->err, DLLM_INVALID_ARG, "token id out of range");
   CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
-  CU_TRY(&s->err, cudaMemcpy2D(s->d_ws + s->ws.tokens + (size_t)s->P * 4, (size_t)s->n * 4, h_tok, (size_t)s->R * 4,
-                               (size_t)s->R * 4, s->B, cudaMemcpyHostToDevice));
+  CU_TRY(&s->err, cudaMemcpy2DAsync(s->d_ws + s->ws.tokens + (size_t)s->P * 4, (size_t)s->n * 4, h_tok,
+                                    (size_t)s->R * 4, (size_t)s->R * 4, s->B, cudaMemcpyHostToDevice,
+                                    (cudaStream_t)stream));
+  CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
   return DLLM_OK;
 }
 
@@ -758,7 +777,7 @@ dllm_status dllm_set_cache(dllm_session* s, int layer, int which, const float* h
   if (r != DLLM_OK) return r;
   cudaStream_t st = (cudaStream_t)stream;
   CU_TRY(&s->err, cudaStreamSynchronize(st));
-  CU_TRY(&s->err, cudaMemcpy(s->d_ws + s->ws.part, h_in, n * 4, cudaMemcpyHostToDevice));
+  CU_TRY(&s->err, h2d(s->d_ws + s->ws.part, h_in, n * 4, st));
   Launch L{st, nullptr, &s->launches};
   launch_convert_from_f32(L, s->m->cfg.dtype, s->wsp<float>(s->ws.part), s->cache(layer, which), n);
   CU_TRY(&s->err, cudaStreamSynchronize(st));
@@ -786,6 +805,7 @@ dllm_status dllm_force_selection(dllm_session* s, int layer, const int32_t* h_id
   CU_TRY(&s->err, cudaDeviceSynchronize());
   CU_TRY(&s->err, cudaMemcpy(s->d_ws + s->ws.forced + (size_t)layer * s->B * s->R * 4, buf.data(), buf.size() * 4,
                              cudaMemcpyHostToDevice));
+  CU_TRY(&s->err, cudaDeviceSynchronize());  // the copy's DMA has landed before any stream may read it
   s->forced_count[layer] = count;
   return DLLM_OK;
 }
@@ -876,14 +896,21 @@ dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, 
   return DLLM_OK;
 }
 
+size_t dllm_attention_scratch_bytes(int B, int a, int n, int H, int Hkv, int hd, int dtype) {
+  if (B <= 0 || a <= 0 || n <= 0 || H <= 0 || Hkv <= 0 || H % Hkv || dtype != DLLM_BF16 || (hd != 64 && hd != 128))
+    return 0;
+  return plan_attention(B, a, n, H, Hkv).scratch_floats * 4;
+}
+
 dllm_status dllm_attention(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B, int a, int n, int H,
-                           int Hkv, int hd, int dtype, void* stream) {
+                           int Hkv, int hd, int dtype, void* d_scratch, size_t scratch_bytes, void* stream) {
   if (!d_q || !d_k || !d_v || !d_o || B <= 0 || a <= 0 || n <= 0 || H <= 0 || Hkv <= 0 || H % Hkv)
     return fail(nullptr, DLLM_INVALID_ARG, "bad attention arguments");
   if (dtype != DLLM_FP32 && dtype != DLLM_BF16) return fail(nullptr, DLLM_INVALID_ARG, "bad dtype");
   if (hd % 32 || hd > 128) return fail(nullptr, DLLM_UNSUPPORTED, "head_dim must be 32, 64, 96 or 128");
   Launch L{(cudaStream_t)stream, nullptr, nullptr};
-  cudaError_t e = launch_attention(L, dtype, d_q, d_k, d_v, d_o, B, a, n, H, Hkv, hd);
+  cudaError_t e = launch_attention(L, dtype, d_q, d_k, d_v, d_o, B, a, n, H, Hkv, hd, static_cast<float*>(d_scratch),
+                                   scratch_bytes / 4, false);
   if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
   return DLLM_OK;
 }

@@ -25,12 +25,11 @@
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the
 // CTA records a code in the status word, skips its epilogue, lets copies in
 // flight land, frees its TMEM and returns.
-#include <cuda.h>
-
 #include <mutex>
 #include <unordered_map>
 
 #include "internal.h"
+#include "tma.cuh"
 
 namespace dllm {
 
@@ -40,55 +39,7 @@ constexpr int TILE_W = 128;  // weight rows per CTA (UMMA M)
 constexpr int TILE_K = 64;   // k per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr uint32_t W_STAGE_BYTES = TILE_W * TILE_K * 2;
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint64_t gtime() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false if the barrier did not flip within the limit or
-// another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = gtime();
-  uint32_t it = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++it & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (gtime() - t0 > WAIT_LIMIT_NS) {
-        *abort_flag = 1;
-        return false;
-      }
-    }
-  }
-  return true;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c_inner,
-                                            int c_outer) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c_inner), "r"(c_outer)
-      : "memory");
-}
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128
 // bytes, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
@@ -162,7 +113,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
     mbar_init(smem_u32(&accum_bar), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_fence_init();
   }
   if (warp == 1) {  // TMEM: BN fp32 columns x 128 lanes
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
@@ -243,11 +194,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
       }
     }
   } else {
-    // gave up: let copies that may still be in flight land before the CTA's
-    // shared memory is released
-    const uint64_t t0 = gtime();
-    while (gtime() - t0 < 200000ull) {
-    }
+    drain_delay();  // gave up: let copies in flight land before shared memory is released
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -276,25 +223,24 @@ EncodeTiledFn get_encode_fn() {
 
 struct MapKey {
   const void* base;
-  uint64_t rows, cols;
+  uint64_t batch, rows, cols;
   uint32_t box_rows;
   bool operator==(const MapKey& o) const {
-    return base == o.base && rows == o.rows && cols == o.cols && box_rows == o.box_rows;
+    return base == o.base && batch == o.batch && rows == o.rows && cols == o.cols && box_rows == o.box_rows;
   }
 };
 struct MapKeyHash {
   size_t operator()(const MapKey& k) const {
     size_t h = std::hash<const void*>()(k.base);
-    h ^= std::hash<uint64_t>()(k.rows * 1315423911ull + k.cols) + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2);
+    h ^= std::hash<uint64_t>()(k.rows * 1315423911ull + k.cols + k.batch * 2654435761ull) + 0x9e3779b97f4a7c15ull +
+         (h << 6) + (h >> 2);
     return h ^ (k.box_rows * 2654435761u);
   }
 };
 
-// bf16 [rows, cols] row-major, box = box_rows x 64 columns, 128-byte swizzle.
-bool get_tensor_map(const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
+bool get_map(const MapKey& key, CUtensorMap* out) {
   static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
   static std::mutex mu;
-  MapKey key{base, rows, cols, box_rows};
   std::lock_guard<std::mutex> lock(mu);
   auto it = cache.find(key);
   if (it != cache.end()) {
@@ -303,16 +249,17 @@ bool get_tensor_map(const void* base, uint64_t rows, uint64_t cols, uint32_t box
   }
   EncodeTiledFn enc = get_encode_fn();
   if (!enc) return false;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {(cuuint32_t)TILE_K, box_rows};
-  cuuint32_t estr[2] = {1, 1};
+  const bool three = key.batch > 0;
+  cuuint64_t dims[3] = {key.cols, key.rows, three ? key.batch : 1};
+  cuuint64_t strides[2] = {key.cols * 2, key.rows * key.cols * 2};
+  cuuint32_t box[3] = {(cuuint32_t)TILE_K, key.box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
   CUtensorMap tm;
-  CUresult r = enc(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = enc(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, three ? 3 : 2, const_cast<void*>(key.base), dims, strides,
+                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
-  if (cache.size() > 4096) cache.clear();
+  if (cache.size() > 8192) cache.clear();
   cache.emplace(key, tm);
   *out = tm;
   return true;
@@ -337,6 +284,14 @@ cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMa
 }
 
 }  // namespace
+
+bool get_tensor_map_2d(const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
+  return get_map(MapKey{base, 0, rows, cols, box_rows}, out);
+}
+bool get_tensor_map_3d(const void* base, uint64_t batch, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                       CUtensorMap* out) {
+  return get_map(MapKey{base, batch, rows, cols, box_rows}, out);
+}
 
 GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split) {
   GemmPlan p;
@@ -366,8 +321,8 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
     return cudaErrorInvalidValue;
   }
   CUtensorMap tmW, tmA;
-  if (!get_tensor_map(W, (uint64_t)N, (uint64_t)K, TILE_W, &tmW) ||
-      !get_tensor_map(A, (uint64_t)M, (uint64_t)K, (uint32_t)plan.BN, &tmA)) {
+  if (!get_tensor_map_2d(W, (uint64_t)N, (uint64_t)K, TILE_W, &tmW) ||
+      !get_tensor_map_2d(A, (uint64_t)M, (uint64_t)K, (uint32_t)plan.BN, &tmA)) {
     if (err) *err = e_map;
     return cudaErrorInvalidValue;
   }

@@ -84,7 +84,17 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
                              const GemmPlan& plan, const char** err);
 
 // ---------------- attention.cu ----------------
+struct AttnPlan {
+  int S;               // key-range splits
+  int keys_per_split;  // multiple of 64
+  size_t scratch_floats;
+};
+AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv);
+// bf16 with head_dim 64 / 128 runs on the tensor cores (scratch holds the
+// partials of split key ranges; without it one split is used); everything else
+// on the plain-ALU kernel.
 cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const void* Kc, const void* Vc, void* o, int B,
-                             int a_seq, int n, int H, int Hkv, int hd);
+                             int a_seq, int n, int H, int Hkv, int hd, float* scratch, size_t scratch_floats,
+                             bool force_simt);
 
 }  // namespace dllm

@@ -72,7 +72,8 @@ SIGNATURES = {
     "dllm_gemm_bf16_scratch_bytes": (_SZ, [_I, _I, _I]),
     "dllm_gemm_bf16": (_I, [_P, _P, _P, _I, _I, _I, _P, _P]),
     "dllm_gemm_simt": (_I, [_P, _P, _P, _I, _I, _I, _I, _P]),
-    "dllm_attention": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P]),
+    "dllm_attention_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I, _I, _I]),
+    "dllm_attention": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
     "dllm_vverify_select": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _P]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
@@ -344,14 +345,18 @@ def gemm_simt(A, W, stream=None):
     return Cm
 
 
-def attention(q, k, v, B, a, n, H, Hkv, hd, stream=None):
-    """q [B*a, H*hd], k/v [B, n, Hkv*hd] torch CUDA tensors (fp32 or bf16); returns o like q."""
+def attention(q, k, v, B, a, n, H, Hkv, hd, stream=None, split=True):
+    """q [B*a, H*hd], k/v [B, n, Hkv*hd] torch CUDA tensors (fp32 or bf16); returns o like q.
+    split=False withholds the scratch buffer, so the key range is processed by one CTA per row tile."""
     import torch
     o = torch.empty_like(q)
     sp = _stream_ptr(stream if stream is not None else torch.cuda.current_stream(q.device))
     dt = BF16 if q.dtype == torch.bfloat16 else FP32
+    sb = lib.dllm_attention_scratch_bytes(B, a, n, H, Hkv, hd, dt) if split else 0
+    scratch = torch.empty(max(sb, 16), dtype=torch.uint8, device=q.device)
     _check(lib.dllm_attention(C.c_void_p(q.data_ptr()), C.c_void_p(k.data_ptr()), C.c_void_p(v.data_ptr()),
-                              C.c_void_p(o.data_ptr()), B, a, n, H, Hkv, hd, dt, C.c_void_p(sp)))
+                              C.c_void_p(o.data_ptr()), B, a, n, H, Hkv, hd, dt, C.c_void_p(scratch.data_ptr()), sb,
+                              C.c_void_p(sp)))
     return o
 
 

@@ -73,21 +73,25 @@ ATT_CASES = [
     (2, 33, 130, 7, 1, 64),    # GQA, 7 query heads per KV head
     (1, 64, 768, 8, 8, 128),   # LLaDA-8B partial-step shape, 8 of the 32 heads
     (1, 128, 512, 28, 4, 128), # Dream-7B partial-step shape
+    (1, 3, 4128, 2, 2, 128),   # long-prompt regime: 3 queries, 65 key tiles, ragged last tile
+    (2, 200, 333, 4, 2, 64),   # several row tiles, G = 2, ragged keys
 ]
 
 
 @pytest.mark.parametrize("case", ATT_CASES)
-@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("dtype", ["fp32", "bf16", "bf16_nosplit"])
 def test_attention(env, case, dtype):
     torch, dllm = env
     B, a, n, H, Hkv, hd = case
     q = synth.random_normal((B * a, H * hd), seed=11, std=1.3)
     k = synth.random_normal((B, n, Hkv * hd), seed=12, std=1.3)
     v = synth.random_normal((B, n, Hkv * hd), seed=13)
+    split = dtype != "bf16_nosplit"
+    dtype = dtype[:4]
     if dtype == "bf16":
         q, k, v = (synth.round_to_bf16(t) for t in (q, k, v))
     td = torch.bfloat16 if dtype == "bf16" else torch.float32
-    got = dllm.attention(*(torch.from_numpy(t).cuda().to(td) for t in (q, k, v)), B, a, n, H, Hkv, hd)
+    got = dllm.attention(*(torch.from_numpy(t).cuda().to(td) for t in (q, k, v)), B, a, n, H, Hkv, hd, split=split)
     got = got.to(torch.float32).cpu().numpy()
     for b in range(B):
         want = O.attention(q[b * a:(b + 1) * a].astype(np.float64).reshape(a, H, hd),
