@@ -218,6 +218,9 @@ def main():
     ap.add_argument("--workload", default="llada8b", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--full-steps", type=int, default=6, help="timed full-recompute steps for the speedup figure")
+    ap.add_argument("--ncu-kinds", default="", help="comma list of step kinds (full,refresh,mixed,partial): after "
+                    "warm-up run one step of each between cudaProfilerStart/Stop and exit (for "
+                    "`ncu --profile-from-start off`); prints no bench line")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -272,6 +275,20 @@ def main():
             ses.step_cached(rp, rr, wl.rho)
     ses.sync()
     ses.set_prompt(prompt)
+
+    if args.ncu_kinds:
+        flags = {"full": (True, True), "refresh": (False, True), "mixed": (True, False), "partial": (False, False)}
+        ses.step_full()
+        ses.sync()
+        torch.cuda.profiler.start()
+        for kind in args.ncu_kinds.split(","):
+            rp, rr = flags[kind]
+            ses.step_cached(rp, rr, wl.rho)
+            ses.remask_low_confidence(0, wl.block_len, 1)
+        ses.sync()
+        torch.cuda.profiler.stop()
+        print(json.dumps({"ncu_window": args.ncu_kinds.split(","), "launches": ses.launch_count()}))
+        return
 
     # ---- timed region: K steps, everything resident ------------------------------------------
     sampler = ClockSampler(local_rank)
