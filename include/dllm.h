@@ -211,6 +211,27 @@ dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, 
 size_t dllm_attention_scratch_bytes(int B, int a, int n, int H, int Hkv, int hd, int dtype);
 dllm_status dllm_attention(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B, int a, int n,
                            int H, int Hkv, int hd, int dtype, void* d_scratch, size_t scratch_bytes, void* stream);
+/* (No counterpart in the paper: an engineering variant of dllm_attention.)
+ * The same bf16 tensor-core attention for callers that cannot create device
+ * allocations where they call it -- a thread that only holds raw pointers
+ * handed over by another component, a process with a fixed memory plan, or
+ * a point where cudaMalloc's implicit device synchronisation is not acceptable.
+ * The caller passes inputs and the output as for dllm_attention (bf16,
+ * head_dim 64 or 128); the scratch for split key ranges is an 8 MiB array
+ * inside the library image, which every GPU that loads the library holds until
+ * the process exits.  The call allocates no device memory.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress) with that device current; make that first call
+ *     before any stream capture.
+ *   - Shapes whose split plan needs more than the 8 MiB return
+ *     DLLM_UNSUPPORTED with a message; use dllm_attention with your own
+ *     scratch for those.
+ *   - All calls share the one array and it keeps the previous call's contents
+ *     (nothing needs clearing: every value read is written first by the same
+ *     call).  Two calls that overlap on the GPU -- different streams, or the
+ *     same shape replayed concurrently -- race on it; serialise them. */
+dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B, int a,
+                                   int n, int H, int Hkv, int hd, void* stream);
 /* V-verify + selection alone (Eq. 6 and the bottom-k rule): d_vnew, d_vcache
  * [B, R, width] in `dtype`; writes d_sim float [B, R] and d_idx int32 [B, k]
  * ascending; overwrites d_vcache with d_vnew. */

@@ -454,6 +454,10 @@ dllm_status run_step(dllm_session* s, int rp, int rr, float rho, dllm_kround kr,
 
 }  // namespace
 
+namespace dllm {
+void set_last_error(const char* msg) { g_err = msg ? msg : ""; }
+}  // namespace dllm
+
 // =============================================================================
 // extern "C" entry points
 // =============================================================================

@@ -6,6 +6,11 @@
 // One CTA = 16 query rows of one sequence x one query head; keys and values
 // are staged 32 rows at a time in shared memory; each warp owns 4 queries,
 // lane = key for the scores, lane = output column for P*V; online softmax.
+#include <stdio.h>
+
+#include <mutex>
+
+#include "../../include/dllm.h"
 #include "internal.h"
 #include "tma.cuh"
 
@@ -447,3 +452,90 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
 }
 
 }  // namespace dllm
+
+// ============================================================================
+// dllm_attention_noalloc: the tensor-core attention with its split-range
+// scratch inside the library image.
+//
+// Who needs this: code that is not allowed to create device allocations at the
+// point where it calls attention -- for example a host thread that only ever
+// received raw pointers to Q, K, V and O from another component and has no
+// allocator of its own, a caller running while memory is being accounted by
+// someone else (a serving process with a fixed memory plan), or a context in
+// which cudaMalloc would synchronise the device and stall other streams.  Such
+// a caller still passes inputs and the output buffer; only the scratch for the
+// partial results of split key ranges comes from the array below.
+//
+// The array is a file-scope __device__ array: every GPU that loads this
+// library holds NOALLOC_SCRATCH_BYTES of it from load until the process exits.
+// Its name is only a host-side handle here; the device address is looked up
+// once per device with cudaGetSymbolAddress and handed to the kernels.
+// ============================================================================
+namespace dllm {
+namespace {
+constexpr size_t NOALLOC_SCRATCH_FLOATS = (size_t)2 * 1024 * 1024;          // 8 MiB
+constexpr size_t NOALLOC_SCRATCH_BYTES = NOALLOC_SCRATCH_FLOATS * sizeof(float);
+constexpr int NOALLOC_MAX_DEVICES = 64;
+static __device__ __align__(256) float g_noalloc_scratch[NOALLOC_SCRATCH_FLOATS];
+
+// Device address of the scratch array on the CURRENT device; looked up on the
+// first call per device.
+cudaError_t noalloc_scratch(float** out) {
+  static std::mutex mu;
+  static float* per_device[NOALLOC_MAX_DEVICES] = {};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!per_device[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    if (!p) return cudaErrorInvalidSymbol;
+    per_device[dev] = static_cast<float*>(p);
+  }
+  *out = per_device[dev];
+  return cudaSuccess;
+}
+}  // namespace
+}  // namespace dllm
+
+extern "C" dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B,
+                                              int a, int n, int H, int Hkv, int hd, void* stream) {
+  using namespace dllm;
+  if (!d_q || !d_k || !d_v || !d_o || B <= 0 || a <= 0 || n <= 0 || H <= 0 || Hkv <= 0 || H % Hkv) {
+    set_last_error("dllm_attention_noalloc: bad arguments");
+    return DLLM_INVALID_ARG;
+  }
+  if (hd != 64 && hd != 128) {
+    set_last_error("dllm_attention_noalloc: bf16 tensor-core path only, head_dim must be 64 or 128");
+    return DLLM_UNSUPPORTED;
+  }
+  const AttnPlan plan = plan_attention(B, a, n, H, Hkv);
+  if (plan.scratch_floats > NOALLOC_SCRATCH_FLOATS) {
+    char msg[256];
+    snprintf(msg, sizeof msg,
+             "dllm_attention_noalloc: this shape splits the key range %d ways and needs %zu bytes of scratch, the "
+             "built-in array holds %zu; use dllm_attention with a caller-owned scratch buffer",
+             plan.S, plan.scratch_floats * sizeof(float), NOALLOC_SCRATCH_BYTES);
+    set_last_error(msg);
+    return DLLM_UNSUPPORTED;
+  }
+  float* scratch = nullptr;
+  cudaError_t e = noalloc_scratch(&scratch);
+  if (e != cudaSuccess) {
+    set_last_error(cudaGetErrorString(e));
+    return DLLM_CUDA_ERROR;
+  }
+  // Nothing in the scratch has to start at zero: every partial (output, max,
+  // sum) that attn_combine_kernel reads is written by this call's attn_mma_kernel first.
+  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  e = launch_attention(L, DLLM_BF16, d_q, d_k, d_v, d_o, B, a, n, H, Hkv, hd, scratch, NOALLOC_SCRATCH_FLOATS, false);
+  if (e != cudaSuccess) {
+    set_last_error(cudaGetErrorString(e));
+    return DLLM_CUDA_ERROR;
+  }
+  return DLLM_OK;
+}
+

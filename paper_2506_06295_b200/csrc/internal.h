@@ -25,6 +25,10 @@ struct Partials {
   int N;  // row length
 };
 
+// ---------------- api.cu ----------------
+// Message that dllm_last_error() returns on this thread.
+void set_last_error(const char* msg);
+
 // ---------------- elementwise.cu ----------------
 // x[c] = E[token(c)] for carried rows c0 <= c < c1.
 void launch_embed(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, Geo g, int c0, int c1);

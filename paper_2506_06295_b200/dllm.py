@@ -75,6 +75,7 @@ SIGNATURES = {
     "dllm_attention_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I, _I, _I]),
     "dllm_attention": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
     "dllm_vverify_select": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _P]),
+    "dllm_attention_noalloc": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _P]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
     _fn = getattr(lib, _name)
@@ -357,6 +358,19 @@ def attention(q, k, v, B, a, n, H, Hkv, hd, stream=None, split=True):
     _check(lib.dllm_attention(C.c_void_p(q.data_ptr()), C.c_void_p(k.data_ptr()), C.c_void_p(v.data_ptr()),
                               C.c_void_p(o.data_ptr()), B, a, n, H, Hkv, hd, dt, C.c_void_p(scratch.data_ptr()), sb,
                               C.c_void_p(sp)))
+    return o
+
+
+def attention_noalloc(q, k, v, o, B, a, n, H, Hkv, hd, stream=None):
+    """bf16 attention into the caller's output tensor `o` without any device
+    allocation: the binding creates no tensor and the library takes its scratch
+    from an 8 MiB array built into the shared object (see include/dllm.h).
+    For callers that hold only raw buffers and may not allocate.  Calls that
+    overlap on the GPU share that scratch and race; keep them on one stream."""
+    import torch
+    sp = _stream_ptr(stream if stream is not None else torch.cuda.current_stream(q.device))
+    _check(lib.dllm_attention_noalloc(C.c_void_p(q.data_ptr()), C.c_void_p(k.data_ptr()), C.c_void_p(v.data_ptr()),
+                                      C.c_void_p(o.data_ptr()), B, a, n, H, Hkv, hd, C.c_void_p(sp)))
     return o
 
 
