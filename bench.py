@@ -196,6 +196,22 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
+def aggregate_over_ranks(ms, ms_e2e, world, device):
+    """Whole-job time = the slowest replica's device time (max over ranks)."""
+    if world <= 1:
+        return ms, ms_e2e
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms, ms_e2e], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0]), float(t[1])
+
+
+def tokens_processed(steps, batch, gen_len, schedule_steps, world):
+    """Units all replicas processed: each scheduled step unmasks gen_len / schedule_steps tokens per sequence."""
+    return steps * batch * gen_len / schedule_steps * world
+
+
 def workload_config(wl, args):
     c = wl.model
     return {"workload": f"{wl.name}: {c.n_layers} layers, d={c.d_model}, {c.n_heads}x{c.head_dim} heads "
@@ -357,16 +373,13 @@ def main():
     ses.profile(False)
 
     # max over ranks
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = aggregate_over_ranks(ms, ms_e2e, world, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    tokens = K * wl.batch * wl.gen_len / wl.steps * world       # one token per sequence per step on this schedule
+    tokens = tokens_processed(K, wl.batch, wl.gen_len, wl.steps, world)
     value = tokens / (ms / 1e3)
     gemm_gbs = g["bytes"] / (g["ms"] / 1e3) / 1e9 if g["ms"] > 0 else 0.0
     counts = {}

@@ -1,0 +1,172 @@
+"""Parity at the benchmark's full sizes (LLaDA-8B shape: d = 4096, 32 heads x
+128, FFN 12288, vocab 126464, prompt 512, generation 256, rho = 0.25), in the
+launch configuration bench.py times (CUDA graphs, tensor-core GEMM and
+attention).
+
+Two legs:
+  * a 2-layer model at full width against the complete oracle step (the oracle
+    finishes that in seconds; the layers are identical work);
+  * the full 32-layer model with weights drawn on the device: properties that
+    hold at any size, plus layer-0 quantities the oracle can compute row by row
+    from downloaded weights (layer 0 sees only embeddings).
+"""
+import numpy as np
+import pytest
+
+from oracle import dllm_oracle as O
+from paper_2506_06295_b200 import synth
+from tests.helpers import rel_l2, selection_matches
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2506_06295_b200 import build as build_mod
+    build_mod.build()
+    from paper_2506_06295_b200 import dllm
+    assert torch.cuda.is_available()
+    return torch, dllm
+
+
+def test_llada_width_two_layers_against_the_oracle(env):
+    torch, dllm = env
+    from concurrent.futures import ThreadPoolExecutor
+    wl = synth.WORKLOADS["llada8b"]
+    cfg = wl.model.with_layers(2)
+    B, P, R = 1, wl.prompt_len, wl.gen_len
+    names = synth.tensor_names(cfg)
+    with ThreadPoolExecutor(max_workers=8) as ex:
+        w = dict(zip([n for n, _ in names], ex.map(lambda ns: synth.make_tensor(cfg, ns[0], ns[1]), names)))
+    prompt = synth.make_prompt(cfg, B, P)
+    orc = O.DLLMOracle(cfg, w, B, P, R, dtype=np.float32)
+    orc.set_prompt(prompt)
+    model = dllm.Model(cfg).load(w)
+    ses = dllm.Session(model, B, P, R)
+    ses.set_prompt(prompt)
+
+    r = orc.step(True, True)
+    ses.step_full()
+    ses.sync()
+    assert rel_l2(ses.hidden(), r.hidden) < 2e-2
+    x0, conf = ses.pred()
+    # greedy estimate: equal wherever the oracle's top-2 logit gap exceeds the bf16 noise
+    srt = np.sort(r.logits[0], axis=-1)
+    clear = (srt[:, -1] - srt[:, -2]) > 0.05
+    assert clear.sum() > 0 and np.array_equal(x0[0][clear], r.x0[0][clear])
+    np.testing.assert_allclose(conf[0][clear], r.conf[0][clear], rtol=0.1)
+
+    # two adaptive steps with a few tokens unmasked in between
+    for step in (1, 2):
+        resp = orc.tokens[:, P:].copy()
+        for j in (3 + step, 40 * step, 200 + step):
+            resp[0, j] = (977 * j + step) % (cfg.vocab - 1)
+        orc.tokens[:, P:] = resp
+        ses.set_response_tokens(resp)
+        r = orc.step(False, False, wl.rho)
+        ses.step_cached(False, False, wl.rho)
+        ses.sync()
+        for l in range(cfg.n_layers):
+            idx, sim = ses.selected(l)
+            assert idx.shape == (1, 64)
+            assert selection_matches(idx[0], r.selected[l][0], r.sim[l][0]), f"step {step} layer {l}"
+            np.testing.assert_allclose(sim, r.sim[l], atol=5e-3)
+        assert rel_l2(ses.hidden(), r.hidden) < 2e-2
+        for which, ref in ((dllm.CACHE_K, orc.Kc), (dllm.CACHE_V, orc.Vc), (dllm.CACHE_ATTN, orc.Ac),
+                           (dllm.CACHE_FFN, orc.Fc)):
+            for l in range(cfg.n_layers):
+                assert rel_l2(ses.get_cache(l, which), ref[l]) < 2e-2
+
+
+def test_llada_full_depth_properties_and_layer0_samples(env):
+    torch, dllm = env
+    wl = synth.WORKLOADS["llada8b"]
+    cfg = wl.model
+    B, P, R = 1, wl.prompt_len, wl.gen_len
+    model = dllm.Model(cfg).random_init_on_device(seed=123)
+    ses = dllm.Session(model, B, P, R)
+    prompt = synth.make_prompt(cfg, B, P)
+    ses.set_prompt(prompt)
+    ses.step_full()
+    ses.sync()
+
+    # inputs for the row-by-row oracle legs: embedding rows and layer-0 projections, downloaded once
+    E = model.tensor_view("embed").view(cfg.vocab, cfg.d_model)
+    wv = model.tensor_view("layers.0.wv").view(cfg.dkv, cfg.d_model).float().cpu().numpy().astype(np.float64)
+    wk = model.tensor_view("layers.0.wk").view(cfg.dkv, cfg.d_model).float().cpu().numpy().astype(np.float64)
+
+    def layer0_u(tok_ids):
+        x = E[torch.from_numpy(np.asarray(tok_ids, np.int64)).cuda()].float().cpu().numpy().astype(np.float64)
+        return O.rmsnorm(x, 1.0, cfg.rms_eps)
+
+    toks = ses.tokens()[0]
+    rows = np.array([0, 1, 77, 300, 511, 512, 513, 640, 767])           # prompt and response positions
+    u = layer0_u(toks[rows])
+    V0 = ses.get_cache(0, dllm.CACHE_V)[0]
+    K0 = ses.get_cache(0, dllm.CACHE_K)[0]
+    assert rel_l2(V0[rows], u @ wv.T) < 1e-2
+    k_ref = O.rope((u @ wk.T).reshape(len(rows), cfg.n_kv_heads, cfg.head_dim), rows, cfg.rope_theta)
+    assert rel_l2(K0[rows], k_ref.reshape(len(rows), -1)) < 1e-2
+
+    # unmask a few tokens; adaptive step; layer-0 similarities and selection from the oracle's functions
+    resp = toks[P:].copy()
+    changed = [5, 64, 130, 255]
+    for j in changed:
+        resp[j] = (1013 * j + 17) % (cfg.vocab - 1)
+    ses.set_response_tokens(resp[None])
+    before = {(l, w): ses.get_cache(l, w) for l in (0, 31) for w in range(4)}
+    ses.step_cached(False, False, wl.rho)
+    ses.sync()
+    v_new = layer0_u(resp) @ wv.T
+    s_ref = O.cosine_rows(v_new, before[(0, dllm.CACHE_V)][0, P:].astype(np.float64))
+    idx, sim = ses.selected(0)
+    np.testing.assert_allclose(sim[0], s_ref, atol=5e-3)
+    assert selection_matches(idx[0], O.select_lowest(s_ref, 64), s_ref)
+    assert set(changed) <= set(idx[0].tolist())
+    # invariants of the adaptive step, at full depth (first and last layer)
+    for l in (0, 31):
+        idx, _ = ses.selected(l)
+        sel = P + idx[0]
+        rest = np.setdiff1d(np.arange(P, P + R), sel)
+        for w in (dllm.CACHE_K, dllm.CACHE_ATTN, dllm.CACHE_FFN):
+            after = ses.get_cache(l, w)
+            assert np.array_equal(after[0, rest], before[(l, w)][0, rest])          # untouched outside S
+            assert np.array_equal(after[0, :P], before[(l, w)][0, :P])              # prompt cache untouched
+            assert not np.array_equal(after[0, sel], before[(l, w)][0, sel])
+        assert np.array_equal(ses.get_cache(l, dllm.CACHE_V)[0, :P], before[(l, dllm.CACHE_V)][0, :P])
+    assert rel_l2(ses.get_cache(0, dllm.CACHE_V)[0, P:], v_new) < 1e-2             # whole V_r overwritten
+
+    # same tokens again: at layer 0 every row reproduces its cached V bit for bit (similarity exactly 1,
+    # ties go to the lowest indices); deeper layers see the rows recomputed at layer 0 move a little
+    ses.step_cached(False, False, wl.rho)
+    ses.sync()
+    idx, sim = ses.selected(0)
+    assert (sim == 1.0).all() and idx[0].tolist() == list(range(64))
+    for l in (15, 31):
+        idx, sim = ses.selected(l)
+        assert (sim[0, 64:] == 1.0).all() and (sim > 0.9).all() and idx[0].tolist() == list(range(64))
+
+    # rho = 0: all caches bit-unchanged; rho = 1 == response refresh, bit for bit
+    snap = {(l, w): ses.get_cache(l, w) for l in (0, 31) for w in range(4)}
+    ses.step_cached(False, False, 0.0)
+    ses.sync()
+    assert all(np.array_equal(ses.get_cache(l, w), snap[(l, w)]) for (l, w) in snap)
+    ses.step_cached(False, False, 1.0)
+    ses.sync()
+    h1, c1 = ses.hidden(), {(l, w): ses.get_cache(l, w) for l in (0, 31) for w in range(4)}
+    ses.step_cached(False, True, 0.0)
+    ses.sync()
+    assert np.array_equal(ses.hidden(), h1)
+    assert all(np.array_equal(ses.get_cache(l, w), c1[(l, w)]) for (l, w) in c1)
+
+    # transition: exactly n_transfer masked positions of the block change, to x0, highest confidence first
+    x0, conf = ses.pred()
+    tok_before = ses.tokens()[0, P:]
+    ses.remask_low_confidence(32, 32, 3)
+    ses.sync()
+    tok_after = ses.tokens()[0, P:]
+    diff = np.nonzero(tok_after != tok_before)[0]
+    cand = [j for j in range(32, 64) if tok_before[j] == cfg.mask_id]
+    want = sorted(sorted(cand, key=lambda j: (-float(conf[0, j]), j))[:3])
+    assert diff.tolist() == want and np.array_equal(tok_after[diff], x0[0, diff])
