@@ -234,11 +234,16 @@ def main():
     ap.add_argument("--workload", default="llada8b", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--full-steps", type=int, default=6, help="timed full-recompute steps for the speedup figure")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (small case for ncu "
+                    "captures: same widths, a few GB of weights); the bench line then names the reduced depth")
     ap.add_argument("--ncu-kinds", default="", help="comma list of step kinds (full,refresh,mixed,partial): after "
                     "warm-up run one step of each between cudaProfilerStart/Stop and exit (for "
                     "`ncu --profile-from-start off`); prints no bench line")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
+    if args.layers > 0:
+        from dataclasses import replace
+        wl = replace(wl, name=f"{wl.name}-{args.layers}layers", model=wl.model.with_layers(args.layers))
     if args.impl == "reference":
         run_reference(args, wl)
         return
@@ -314,10 +319,12 @@ def main():
     barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     l0 = ses.launch_count()
+    torch.cuda.profiler.start()       # no-op unless a profiler waits for it (`ncu --profile-from-start off`)
     ev0.record(stream)
     run_steps(K)
     ev1.record(stream)
     barrier()
+    torch.cuda.profiler.stop()
     ms = ev0.elapsed_time(ev1)
     launches = ses.launch_count() - l0
     ses.sync()
