@@ -198,6 +198,14 @@ dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable);
 size_t dllm_gemm_bf16_scratch_bytes(int M, int N, int K);
 dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, int N, int K,
                            void* d_partials, void* stream);
+/* The same product with an explicit launch plan, for tuning: act_tile = rows of
+ * A per CTA (32, 64, 128 or 256), splits = split-K factor, stages = depth of the
+ * TMA ring (clamped to what fits shared memory); 0 picks the default of each.
+ * d_partials (device, partials_bytes) must hold splits*M*N floats when splits > 1;
+ * with splits > 1 and d_C NULL the slabs are left unreduced in d_partials (what
+ * the step's fused consumers read). */
+dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
+                                   int splits, int stages, void* d_partials, size_t partials_bytes, void* stream);
 /* The same product on the plain fp32 ALUs (operands fp32 or bf16): the GEMM of
  * the fp32 mode. */
 dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int dtype,

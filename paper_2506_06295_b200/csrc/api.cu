@@ -308,7 +308,7 @@ dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void
     launch_gemm_simt(L, s->m->cfg.dtype, A, W, part, M, N, K);
     return DLLM_OK;
   }
-  const GemmPlan plan = plan_gemm_bf16(M, N, K, 0);
+  const GemmPlan plan = plan_gemm_bf16(M, N, K);
   if ((size_t)plan.S * M * N > s->ws.part_floats)
     return fail(&s->err, DLLM_UNSUPPORTED, "GEMM %dx%dx%d with %d splits exceeds the workspace", M, N, K, plan.S);
   const char* why = nullptr;
@@ -870,7 +870,7 @@ dllm_status dllm_session_profile_read(dllm_session* s, int cls, double* total_ms
 // ---- kernel-level entry points ------------------------------------------------
 size_t dllm_gemm_bf16_scratch_bytes(int M, int N, int K) {
   if (M <= 0 || N <= 0 || K <= 0) return 0;
-  const GemmPlan p = plan_gemm_bf16(M, N, K, 0);
+  const GemmPlan p = plan_gemm_bf16(M, N, K);
   return p.S > 1 ? (size_t)p.S * M * N * 4 : 0;
 }
 
@@ -878,7 +878,7 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
                            void* stream) {
   if (!d_A || !d_W || !d_C || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
   if (K % 8) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8");
-  const GemmPlan p = plan_gemm_bf16(M, N, K, 0);
+  const GemmPlan p = plan_gemm_bf16(M, N, K);
   if (p.S > 1 && !d_partials) return fail(nullptr, DLLM_INVALID_ARG, "this shape needs split-K scratch");
   Launch L{(cudaStream_t)stream, nullptr, nullptr};
   float* part = p.S > 1 ? static_cast<float*>(d_partials) : d_C;
@@ -886,6 +886,27 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
   cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
   if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "bf16 GEMM: %s", why ? why : cudaGetErrorString(e));
   if (p.S > 1) launch_reduce_partials(L, Partials{part, (size_t)M * N, p.S, N}, d_C, M);
+  CU_TRY(nullptr, cudaGetLastError());
+  return DLLM_OK;
+}
+
+dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
+                                   int splits, int stages, void* d_partials, size_t partials_bytes, void* stream) {
+  if (!d_A || !d_W || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
+  if (K % 8) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8");
+  if (act_tile < 0 || splits < 0 || stages < 0) return fail(nullptr, DLLM_INVALID_ARG, "negative plan parameter");
+  if (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 256)
+    return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128 or 256");
+  const GemmPlan p = plan_gemm_bf16(M, N, K, splits, stages, act_tile);
+  if (p.S > 1 && (!d_partials || partials_bytes < (size_t)p.S * M * N * 4))
+    return fail(nullptr, DLLM_INVALID_ARG, "this plan needs %zu bytes of split-K scratch", (size_t)p.S * M * N * 4);
+  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  if (!d_C && (p.S == 1 || !d_partials)) return fail(nullptr, DLLM_INVALID_ARG, "d_C is NULL");
+  float* part = p.S > 1 ? static_cast<float*>(d_partials) : d_C;
+  const char* why = nullptr;
+  cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
+  if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "bf16 GEMM: %s", why ? why : cudaGetErrorString(e));
+  if (p.S > 1 && d_C) launch_reduce_partials(L, Partials{part, (size_t)M * N, p.S, N}, d_C, M);
   CU_TRY(nullptr, cudaGetLastError());
   return DLLM_OK;
 }

@@ -76,23 +76,25 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "memory");
 }
 
-template <int BN, int STAGES>
+constexpr int MAX_STAGES = 12;
+
+template <int BN>
 struct SmemLayout {
   static constexpr uint32_t A_STAGE_BYTES = BN * TILE_K * 2;
   static constexpr uint32_t STAGE_BYTES = W_STAGE_BYTES + A_STAGE_BYTES;
-  static constexpr uint32_t TOTAL = STAGES * STAGE_BYTES + 1024;  // + slack to align the base to 1024
+  static constexpr uint32_t total(int stages) { return (uint32_t)stages * STAGE_BYTES + 1024; }  // + slack to align the base to 1024
 };
 
-template <int BN, int STAGES>
+template <int BN>
 __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                 const __grid_constant__ CUtensorMap tmA,
                                                                 float* __restrict__ part, int M, int N, int num_kb,
-                                                                int kb_per_split, size_t split_stride,
+                                                                int kb_per_split, size_t split_stride, int STAGES,
                                                                 int* __restrict__ status) {
-  using SL = SmemLayout<BN, STAGES>;
+  using SL = SmemLayout<BN>;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[STAGES];
-  __shared__ __align__(8) uint64_t empty_bar[STAGES];
+  __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t accum_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
@@ -129,9 +131,11 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
 
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer ----------------
+    prefetch_tensormap(&tmW);
+    prefetch_tensormap(&tmA);
+    int s = 0;
+    uint32_t ph = 0;
     for (int i = 0; i < nkb; ++i) {
-      const int s = i % STAGES;
-      const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
       if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) {
         if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
         break;
@@ -142,14 +146,18 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
       const int kc = (kb0 + i) * TILE_K;
       tma_load_2d(dstW, &tmW, fb, kc, n0);
       tma_load_2d(dstW + W_STAGE_BYTES, &tmA, fb, kc, m0);
+      if (++s == STAGES) {
+        s = 0;
+        ph ^= 1u;
+      }
     }
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer ----------------
     constexpr uint32_t idesc = make_idesc(TILE_W, BN);
     bool ok = true;
+    int s = 0;
+    uint32_t ph = 0;
     for (int i = 0; i < nkb && ok; ++i) {
-      const int s = i % STAGES;
-      const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
       if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp)) {
         if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_MMA);
         ok = false;
@@ -165,6 +173,10 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
         umma_bf16(tmem_d, dW + (uint64_t)(2 * k), dA + (uint64_t)(2 * k), idesc, (i > 0 || k > 0) ? 1u : 0u);
       }
       umma_commit(smem_u32(&empty_bar[s]));  // stage reusable once these MMAs have read it
+      if (++s == STAGES) {
+        s = 0;
+        ph ^= 1u;
+      }
     }
     if (ok) umma_commit(smem_u32(&accum_bar));
   }
@@ -265,20 +277,27 @@ bool get_map(const MapKey& key, CUtensorMap* out) {
   return true;
 }
 
-template <int BN, int STAGES>
+// Most stages whose ring fits the 227 KB of shared memory one CTA may use.
+constexpr int max_stages(int bn) {
+  const int fit = (227 * 1024 - 1024 - 256) / (int)(W_STAGE_BYTES + bn * TILE_K * 2);
+  return fit < MAX_STAGES ? fit : MAX_STAGES;
+}
+
+template <int BN>
 cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMap& tmA, float* part, int M, int N,
                        int num_kb, const GemmPlan& plan) {
-  using SL = SmemLayout<BN, STAGES>;
+  using SL = SmemLayout<BN>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<BN, STAGES>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SL::TOTAL);
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)SL::total(max_stages(BN)));
     if (e != cudaSuccess) return e;
     configured = true;
   }
+  const int stages = plan.stages < 2 ? 2 : plan.stages > max_stages(BN) ? max_stages(BN) : plan.stages;
   dim3 grid((M + BN - 1) / BN, (N + TILE_W - 1) / TILE_W, plan.S);
-  gemm_bf16_tcgen05_kernel<BN, STAGES><<<grid, 128, SL::TOTAL, L.stream>>>(tmW, tmA, part, M, N, num_kb,
-                                                                          plan.kb_per_split, (size_t)M * N, L.d_status);
+  gemm_bf16_tcgen05_kernel<BN><<<grid, 128, SL::total(stages), L.stream>>>(
+      tmW, tmA, part, M, N, num_kb, plan.kb_per_split, (size_t)M * N, stages, L.d_status);
   L.count();
   return cudaGetLastError();
 }
@@ -293,9 +312,10 @@ bool get_tensor_map_3d(const void* base, uint64_t batch, uint64_t rows, uint64_t
   return get_map(MapKey{base, batch, rows, cols, box_rows}, out);
 }
 
-GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split) {
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, int force_bn) {
   GemmPlan p;
   p.BN = M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+  if (force_bn == 32 || force_bn == 64 || force_bn == 128 || force_bn == 256) p.BN = force_bn;
   p.stages = 4;
   const int num_kb = (K + TILE_K - 1) / TILE_K;
   const long tiles = (long)((M + p.BN - 1) / p.BN) * ((N + TILE_W - 1) / TILE_W);
@@ -306,6 +326,7 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split) {
     if (S > max_s) S = max_s;
   }
   if (force_split > 0) S = force_split < num_kb ? force_split : num_kb;
+  if (force_stages > 0) p.stages = force_stages;
   p.kb_per_split = (num_kb + S - 1) / S;
   p.S = (num_kb + p.kb_per_split - 1) / p.kb_per_split;  // no empty split
   return p;
@@ -328,10 +349,10 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
   }
   const int num_kb = (K + TILE_K - 1) / TILE_K;
   switch (plan.BN) {
-    case 32: return launch_one<32, 4>(L, tmW, tmA, part, M, N, num_kb, plan);
-    case 64: return launch_one<64, 4>(L, tmW, tmA, part, M, N, num_kb, plan);
-    case 128: return launch_one<128, 3>(L, tmW, tmA, part, M, N, num_kb, plan);
-    default: return launch_one<256, 4>(L, tmW, tmA, part, M, N, num_kb, plan);
+    case 32: return launch_one<32>(L, tmW, tmA, part, M, N, num_kb, plan);
+    case 64: return launch_one<64>(L, tmW, tmA, part, M, N, num_kb, plan);
+    case 128: return launch_one<128>(L, tmW, tmA, part, M, N, num_kb, plan);
+    default: return launch_one<256>(L, tmW, tmA, part, M, N, num_kb, plan);
   }
 }
 

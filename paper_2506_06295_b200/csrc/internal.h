@@ -82,7 +82,7 @@ struct GemmPlan {
   int kb_per_split;
   int stages;
 };
-GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split /* 0 = auto */);
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split = 0, int force_stages = 0, int force_bn = 0);  // 0 = auto
 // Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
                              const GemmPlan& plan, const char** err);

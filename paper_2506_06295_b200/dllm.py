@@ -71,6 +71,7 @@ SIGNATURES = {
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "dllm_gemm_bf16_scratch_bytes": (_SZ, [_I, _I, _I]),
     "dllm_gemm_bf16": (_I, [_P, _P, _P, _I, _I, _I, _P, _P]),
+    "dllm_gemm_bf16_planned": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
     "dllm_gemm_simt": (_I, [_P, _P, _P, _I, _I, _I, _I, _P]),
     "dllm_attention_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I, _I, _I]),
     "dllm_attention": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
@@ -331,6 +332,23 @@ def gemm_bf16(A, W, stream=None):
     sp = _stream_ptr(stream if stream is not None else torch.cuda.current_stream(A.device))
     _check(lib.dllm_gemm_bf16(C.c_void_p(A.data_ptr()), C.c_void_p(W.data_ptr()), C.c_void_p(Cm.data_ptr()), M, N, K,
                               C.c_void_p(scratch.data_ptr()), C.c_void_p(sp)))
+    return Cm
+
+
+def gemm_bf16_planned(A, W, act_tile=0, splits=0, stages=0, out=None, scratch=None, stream=None, reduce=True):
+    """gemm_bf16 with an explicit launch plan (tuning hook); `out` / `scratch` may be preallocated.
+    reduce=False with splits > 1 leaves the split-K slabs unreduced in `scratch`."""
+    import torch
+    M, K = A.shape
+    N = W.shape[0]
+    Cm = out if out is not None else torch.empty((M, N), dtype=torch.float32, device=A.device)
+    if scratch is None:
+        scratch = torch.empty(max(splits, 1) * M * N * 4 + 16, dtype=torch.uint8, device=A.device)
+    sp = _stream_ptr(stream if stream is not None else torch.cuda.current_stream(A.device))
+    cptr = Cm.data_ptr() if (reduce or splits <= 1) else None
+    _check(lib.dllm_gemm_bf16_planned(C.c_void_p(A.data_ptr()), C.c_void_p(W.data_ptr()), C.c_void_p(cptr),
+                                      M, N, K, act_tile, splits, stages, C.c_void_p(scratch.data_ptr()),
+                                      scratch.numel(), C.c_void_p(sp)))
     return Cm
 
 
