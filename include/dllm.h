@@ -176,6 +176,11 @@ uint64_t dllm_launch_count(const dllm_session* s);
  * 0: launch kernels one by one. */
 dllm_status dllm_session_use_graphs(dllm_session* s, int enable);
 
+/* 1 (default): the kernels of a step are launched with programmatic stream
+ * serialization, so each kernel's set-up (and the weight prefetch of the
+ * projections) overlaps the tail of the kernel before it; 0: plain launches. */
+dllm_status dllm_session_use_pdl(dllm_session* s, int enable);
+
 /* Per-kernel timing.  While enabled, steps are launched kernel by kernel (no
  * graph replay) and every projection GEMM (class 0) and attention launch
  * (class 1) is bracketed by CUDA events on the caller's stream.  _profile_read

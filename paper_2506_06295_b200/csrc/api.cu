@@ -193,6 +193,7 @@ struct dllm_session {
   uint64_t launches = 0;
   bool use_graphs = true;
   bool simt_gemm = false;
+  bool use_pdl = true;
   struct GraphEntry {
     cudaGraphExec_t exec;
     uint64_t kernels;
@@ -329,7 +330,7 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
   const int dt = c.dtype, d = c.d_model, H = c.n_heads, Hkv = c.n_kv_heads, hd = c.head_dim, m = c.d_ffn;
   const int dq = H * hd, dkv = Hkv * hd, BR = s->B * s->R, BP = s->B * s->P;
   const size_t es = s->es();
-  Launch L{stream, s->wsp<int>(s->ws.status), &s->launches};
+  Launch L{stream, s->wsp<int>(s->ws.status), &s->launches, s->use_pdl && !s->profiling};
   uint8_t* W = s->m->d_w;
   const int c0 = 0, c1 = BR + (rp ? BP : 0);
   const int a_seq = (rp ? s->P : 0) + ksel;
@@ -819,6 +820,16 @@ uint64_t dllm_launch_count(const dllm_session* s) { return s ? s->launches : 0; 
 dllm_status dllm_session_use_graphs(dllm_session* s, int enable) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
   s->use_graphs = enable != 0;
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_use_pdl(dllm_session* s, int enable) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if ((enable != 0) != s->use_pdl) {
+    for (auto& kv : s->graphs) cudaGraphExecDestroy(kv.second.exec);
+    s->graphs.clear();
+  }
+  s->use_pdl = enable != 0;
   return DLLM_OK;
 }
 

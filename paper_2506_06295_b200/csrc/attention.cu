@@ -35,6 +35,8 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(const T* __restrict__ q,
   const int kh = h / (H / Hkv);
   const int dq = H * hd, dkv = Hkv * hd;
   const int nd = hd >> 5;  // output columns per lane
+  pdl_wait();
+  pdl_trigger();
 
   for (int e = threadIdx.x; e < TQ * hd; e += blockDim.x) {
     const int r = e / hd, c = e - r * hd;
@@ -202,6 +204,8 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ C
       tma_load_3d(dst + TILE_BYTES + p * (AT_KEYS * 128), &tmV, fb, kh * HD + p * 64, key0, b);
     }
   };
+  pdl_wait();  // K, V and Q come from the preceding kernels
+  pdl_trigger();
   if (threadIdx.x == 0) {
     issue(0);
     if (n_tiles > 1) issue(1);
@@ -356,6 +360,8 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ C
 // Merges the key-range splits: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
 __global__ void attn_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ ml_part,
                                     __nv_bfloat16* __restrict__ o, size_t total, int S, int hd) {
+  pdl_wait();
+  pdl_trigger();
   const size_t rh = blockIdx.x;
   float M = -INFINITY;
   for (int s = 0; s < S; ++s) M = fmaxf(M, ml_part[((size_t)s * total + rh) * 2]);
@@ -389,12 +395,12 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
   float* ml_part = scratch ? scratch + (size_t)S * total * HD : nullptr;
   dim3 grid((a_seq * G + AT_ROWS - 1) / AT_ROWS, Hkv, B * S);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
-  attn_mma_kernel<HD><<<grid, 128, SMEM, L.stream>>>(tmK, tmV, (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part,
+  launch_k(L, attn_mma_kernel<HD>, dim3(grid), dim3(128), SMEM, tmK, tmV, (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part,
                                                      ml_part, a_seq, n, H, Hkv, S, keys_per_split, scale_log2,
                                                      L.d_status);
   L.count();
   if (S > 1) {
-    attn_combine_kernel<<<(unsigned)total, HD / 2, 0, L.stream>>>(o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
+    launch_k(L, attn_combine_kernel, dim3((unsigned)total), dim3(HD / 2), 0, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
     L.count();
   }
   return cudaGetLastError();
@@ -441,10 +447,10 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
   const float scale = 1.0f / sqrtf((float)hd);
   dim3 grid((a_seq + TQ - 1) / TQ, H, B);
   if (dtype == 0)
-    attn_simt_kernel<float><<<grid, 128, 0, L.stream>>>((const float*)q, (const float*)Kc, (const float*)Vc,
+    launch_k(L, attn_simt_kernel<float>, dim3(grid), dim3(128), 0, (const float*)q, (const float*)Kc, (const float*)Vc,
                                                         (float*)o, a_seq, n, H, Hkv, hd, scale);
   else
-    attn_simt_kernel<__nv_bfloat16><<<grid, 128, 0, L.stream>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)Kc,
+    launch_k(L, attn_simt_kernel<__nv_bfloat16>, dim3(grid), dim3(128), 0, (const __nv_bfloat16*)q, (const __nv_bfloat16*)Kc,
                                                                 (const __nv_bfloat16*)Vc, (__nv_bfloat16*)o, a_seq, n,
                                                                 H, Hkv, hd, scale);
   L.count();

@@ -29,6 +29,13 @@ __host__ __device__ inline void carried_to_pos(int c, const Geo& g, int& b, int&
 // device status word codes
 enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103, ST_RANGE = 201 };
 
+// Programmatic dependent launch.  pdl_wait(): blocks until the preceding grid
+// in the stream has completed and its writes are visible (returns at once for
+// a launch without the attribute).  pdl_trigger(): lets the next grid become
+// resident once every CTA of this grid has called it.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 template <typename T>
 struct Vec8;  // eight consecutive elements, 16-byte (bf16) or 32-byte (fp32) aligned
 

@@ -27,6 +27,8 @@ namespace dllm {
 template <typename T>
 __global__ void embed_kernel(const T* __restrict__ E, const int32_t* __restrict__ tokens, float* __restrict__ x, Geo g,
                              int c0) {
+  pdl_wait();
+  pdl_trigger();
   const int c = c0 + blockIdx.x;
   int b, pos;
   carried_to_pos(c, g, b, pos);
@@ -42,7 +44,7 @@ __global__ void embed_kernel(const T* __restrict__ E, const int32_t* __restrict_
 
 void launch_embed(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, Geo g, int c0, int c1) {
   if (c1 <= c0) return;
-  DLLM_DISPATCH(dtype, (embed_kernel<T><<<c1 - c0, 128, 0, L.stream>>>((const T*)E, tokens, x, g, c0)));
+  DLLM_DISPATCH(dtype, (launch_k(L, embed_kernel<T>, dim3(c1 - c0), dim3(128), 0, (const T*)E, tokens, x, g, c0)));
   L.count();
 }
 
@@ -50,6 +52,8 @@ void launch_embed(const Launch& L, int dtype, const void* E, const int32_t* toke
 template <typename T>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain, T* __restrict__ out, int d,
                                float eps, int c0) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ float red[32];
   const size_t row = (size_t)(c0 + blockIdx.x);
   const float* xr = x + row * d;
@@ -76,13 +80,15 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
 void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gain, void* out, int d, float eps, int c0,
                     int c1) {
   if (c1 <= c0) return;
-  DLLM_DISPATCH(dtype, (rmsnorm_kernel<T><<<c1 - c0, 256, 0, L.stream>>>(x, gain, (T*)out, d, eps, c0)));
+  DLLM_DISPATCH(dtype, (launch_k(L, rmsnorm_kernel<T>, dim3(c1 - c0), dim3(256), 0, x, gain, (T*)out, d, eps, c0)));
   L.count();
 }
 
 // ------------------------------------------------------------------ V-verify (Eq. 6) + V overwrite
 template <typename T>
 __global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restrict__ sim, Geo g, int dkv) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ float red[32];
   const int c = blockIdx.x;  // response row, carried order
   const int b = c / g.R, j = c - b * g.R;
@@ -109,7 +115,7 @@ __global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restr
 
 void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv) {
   const int rows = g.B * g.R;
-  DLLM_DISPATCH(dtype, (vverify_kernel<T><<<rows, 128, 0, L.stream>>>(part, (T*)Vc_layer, sim, g, dkv)));
+  DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(128), 0, part, (T*)Vc_layer, sim, g, dkv)));
   L.count();
 }
 
@@ -117,6 +123,8 @@ void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, f
 template <typename T>
 __global__ void vverify_rows_kernel(const T* __restrict__ vnew, T* __restrict__ vcache, float* __restrict__ sim,
                                     int width) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ float red[32];
   const size_t row = blockIdx.x;
   const T* a = vnew + row * width;
@@ -142,7 +150,7 @@ __global__ void vverify_rows_kernel(const T* __restrict__ vnew, T* __restrict__ 
 
 void launch_vverify_rows(const Launch& L, int dtype, const void* vnew, void* vcache, float* sim, int rows, int width) {
   if (rows <= 0) return;
-  DLLM_DISPATCH(dtype, (vverify_rows_kernel<T><<<rows, 128, 0, L.stream>>>((const T*)vnew, (T*)vcache, sim, width)));
+  DLLM_DISPATCH(dtype, (launch_k(L, vverify_rows_kernel<T>, dim3(rows), dim3(128), 0, (const T*)vnew, (T*)vcache, sim, width)));
   L.count();
 }
 
@@ -153,6 +161,8 @@ void launch_vverify_rows(const Launch& L, int dtype, const void* vnew, void* vca
 __global__ void select_kernel(const float* __restrict__ sim, const int32_t* __restrict__ forced, int mode, int ksel,
                               int32_t* __restrict__ sel, int sel_stride, int32_t* __restrict__ act, Geo g,
                               int refresh_prompt) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ unsigned long long keys[];  // R keys, then R flags (as bytes)
   unsigned char* flag = reinterpret_cast<unsigned char*>(keys + g.R);
   const int b = blockIdx.x;
@@ -206,7 +216,7 @@ __global__ void select_kernel(const float* __restrict__ sim, const int32_t* __re
 void launch_select(const Launch& L, const float* sim, const int32_t* forced, int mode, int ksel, int32_t* sel,
                    int sel_stride, int32_t* act, Geo g, int refresh_prompt) {
   const size_t smem = (size_t)g.R * 9 + 16;
-  select_kernel<<<g.B, 256, smem, L.stream>>>(sim, forced, mode, ksel, sel, sel_stride, act, g, refresh_prompt);
+  launch_k(L, select_kernel, dim3(g.B), dim3(256), smem, sim, forced, mode, ksel, sel, sel_stride, act, g, refresh_prompt);
   L.count();
 }
 
@@ -214,6 +224,8 @@ void launch_select(const Launch& L, const float* sim, const int32_t* forced, int
 template <typename T>
 __global__ void gather_rows_kernel(const T* __restrict__ src, const int32_t* __restrict__ act, T* __restrict__ dst,
                                    int d) {
+  pdl_wait();
+  pdl_trigger();
   const size_t r = blockIdx.x;
   const uint4* s = reinterpret_cast<const uint4*>(src + (size_t)act[r] * d);
   uint4* o = reinterpret_cast<uint4*>(dst + r * d);
@@ -223,7 +235,7 @@ __global__ void gather_rows_kernel(const T* __restrict__ src, const int32_t* __r
 
 void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32_t* act, void* dst, int rows, int d) {
   if (rows <= 0) return;
-  DLLM_DISPATCH(dtype, (gather_rows_kernel<T><<<rows, 128, 0, L.stream>>>((const T*)src, act, (T*)dst, d)));
+  DLLM_DISPATCH(dtype, (launch_k(L, gather_rows_kernel<T>, dim3(rows), dim3(128), 0, (const T*)src, act, (T*)dst, d)));
   L.count();
 }
 
@@ -233,6 +245,8 @@ void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32
 template <typename T>
 __global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ rope_tab,
                                T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int H, int Hkv, int hd) {
+  pdl_wait();
+  pdl_trigger();
   const int r = blockIdx.x, head = blockIdx.y;
   int b, pos;
   carried_to_pos(act[r], g, b, pos);
@@ -259,7 +273,7 @@ void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* ac
                     void* Kc_layer, Geo g, int Ma, int H, int Hkv, int hd) {
   if (Ma <= 0) return;
   dim3 grid(Ma, H + Hkv);
-  DLLM_DISPATCH(dtype, (qk_rope_kernel<T><<<grid, 64, 0, L.stream>>>(part, act, rope_tab, (T*)qbuf, (T*)Kc_layer, g, H,
+  DLLM_DISPATCH(dtype, (launch_k(L, qk_rope_kernel<T>, dim3(grid), dim3(64), 0, part, act, rope_tab, (T*)qbuf, (T*)Kc_layer, g, H,
                                                                      Hkv, hd)));
   L.count();
 }
@@ -268,6 +282,8 @@ void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* ac
 template <typename T>
 __global__ void scatter_rows_kernel(Partials part, const int32_t* __restrict__ act, int c_base, T* __restrict__ cache,
                                     Geo g, int width) {
+  pdl_wait();
+  pdl_trigger();
   const int r = blockIdx.x;
   const int c = act ? act[r] : c_base + r;
   int b, pos;
@@ -284,7 +300,7 @@ void launch_scatter_rows(const Launch& L, int dtype, Partials part, const int32_
                          Geo g, int rows, int width) {
   if (rows <= 0) return;
   DLLM_DISPATCH(dtype,
-                (scatter_rows_kernel<T><<<rows, 128, 0, L.stream>>>(part, act, c_base, (T*)cache_layer, g, width)));
+                (launch_k(L, scatter_rows_kernel<T>, dim3(rows), dim3(128), 0, part, act, c_base, (T*)cache_layer, g, width)));
   L.count();
 }
 
@@ -296,6 +312,8 @@ template <typename T>
 __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ x,
                                       const float* __restrict__ gain2, T* __restrict__ Ac, T* __restrict__ hn, Geo g,
                                       float eps) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ float hrow[];
   __shared__ float red[32];
   const int r = blockIdx.x;
@@ -336,7 +354,7 @@ void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int3
                            const float* gain2, void* Ac_layer, void* hn, Geo g, int Ma, float eps) {
   if (Ma <= 0) return;
   const size_t smem = (size_t)g.d * sizeof(float);
-  DLLM_DISPATCH(dtype, (oproj_epilogue_kernel<T><<<Ma, 256, smem, L.stream>>>(part, act, x, gain2, (T*)Ac_layer,
+  DLLM_DISPATCH(dtype, (launch_k(L, oproj_epilogue_kernel<T>, dim3(Ma), dim3(256), smem, part, act, x, gain2, (T*)Ac_layer,
                                                                             (T*)hn, g, eps)));
   L.count();
 }
@@ -344,6 +362,8 @@ void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int3
 // ------------------------------------------------------------------ SwiGLU gate
 template <typename T>
 __global__ void silu_mul_kernel(Partials part, T* __restrict__ out, int Ma, int m) {
+  pdl_wait();
+  pdl_trigger();
   const int mv = m >> 3;
   const size_t total = (size_t)Ma * mv;
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
@@ -361,7 +381,7 @@ void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int M
   if (Ma <= 0) return;
   const size_t total = (size_t)Ma * (m >> 3);
   const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
-  DLLM_DISPATCH(dtype, (silu_mul_kernel<T><<<blocks, 256, 0, L.stream>>>(part, (T*)out, Ma, m)));
+  DLLM_DISPATCH(dtype, (launch_k(L, silu_mul_kernel<T>, dim3(blocks), dim3(256), 0, part, (T*)out, Ma, m)));
   L.count();
 }
 
@@ -369,6 +389,8 @@ void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int M
 template <typename T>
 __global__ void residual_kernel(float* __restrict__ x, const T* __restrict__ Ac, const T* __restrict__ Fc, Geo g,
                                 int c0) {
+  pdl_wait();
+  pdl_trigger();
   const int c = c0 + blockIdx.x;
   int b, pos;
   carried_to_pos(c, g, b, pos);
@@ -389,7 +411,7 @@ void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer,
                      int c1) {
   if (c1 <= c0) return;
   DLLM_DISPATCH(dtype,
-                (residual_kernel<T><<<c1 - c0, 128, 0, L.stream>>>(x, (const T*)Ac_layer, (const T*)Fc_layer, g, c0)));
+                (launch_k(L, residual_kernel<T>, dim3(c1 - c0), dim3(128), 0, x, (const T*)Ac_layer, (const T*)Fc_layer, g, c0)));
   L.count();
 }
 
@@ -412,6 +434,8 @@ __device__ __forceinline__ MaxSum merge(MaxSum p, MaxSum q) {
 
 __global__ void argmax_conf_kernel(const float* __restrict__ logits, int vocab, int mask_id, int32_t* __restrict__ x0,
                                    float* __restrict__ conf) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ MaxSum sh[32];
   const size_t row = blockIdx.x;
   const float* lr = logits + row * vocab;
@@ -459,7 +483,7 @@ __global__ void argmax_conf_kernel(const float* __restrict__ logits, int vocab, 
 void launch_argmax_conf(const Launch& L, const float* logits, int rows, int vocab, int mask_id, int32_t* x0,
                         float* conf) {
   if (rows <= 0) return;
-  argmax_conf_kernel<<<rows, 512, 0, L.stream>>>(logits, vocab, mask_id, x0, conf);
+  launch_k(L, argmax_conf_kernel, dim3(rows), dim3(512), 0, logits, vocab, mask_id, x0, conf);
   L.count();
 }
 
@@ -469,6 +493,8 @@ void launch_argmax_conf(const Launch& L, const float* logits, int rows, int voca
 __global__ void remask_kernel(int32_t* __restrict__ tokens, const int32_t* __restrict__ x0,
                               const float* __restrict__ conf, Geo g, int mask_id, int block_start, int block_len,
                               int n_transfer) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ unsigned long long keys[];
   const int b = blockIdx.x;
   int32_t* tok = tokens + (size_t)b * g.n + g.P;
@@ -495,13 +521,15 @@ __global__ void remask_kernel(int32_t* __restrict__ tokens, const int32_t* __res
 
 void launch_remask(const Launch& L, int32_t* tokens, const int32_t* x0, const float* conf, Geo g, int mask_id,
                    int block_start, int block_len, int n_transfer) {
-  remask_kernel<<<g.B, 256, (size_t)block_len * 8, L.stream>>>(tokens, x0, conf, g, mask_id, block_start, block_len,
+  launch_k(L, remask_kernel, dim3(g.B), dim3(256), (size_t)block_len * 8, tokens, x0, conf, g, mask_id, block_start, block_len,
                                                                n_transfer);
   L.count();
 }
 
 // ------------------------------------------------------------------ misc
 __global__ void reduce_partials_kernel(Partials part, float* __restrict__ C, size_t total) {
+  pdl_wait();
+  pdl_trigger();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     float v = part.p[i];
     for (int s = 1; s < part.S; ++s) v += part.p[(size_t)s * part.split_stride + i];
@@ -513,17 +541,21 @@ void launch_reduce_partials(const Launch& L, Partials part, float* C, int M) {
   const size_t total = (size_t)M * part.N;
   if (!total) return;
   const int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
-  reduce_partials_kernel<<<blocks, 256, 0, L.stream>>>(part, C, total);
+  launch_k(L, reduce_partials_kernel, dim3(blocks), dim3(256), 0, part, C, total);
   L.count();
 }
 
 template <typename T>
 __global__ void to_f32_kernel(const T* __restrict__ src, float* __restrict__ dst, size_t n) {
+  pdl_wait();
+  pdl_trigger();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     dst[i] = to_f32<T>(src[i]);
 }
 template <typename T>
 __global__ void from_f32_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t n) {
+  pdl_wait();
+  pdl_trigger();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     dst[i] = from_f32<T>(src[i]);
 }
@@ -531,23 +563,25 @@ __global__ void from_f32_kernel(const float* __restrict__ src, T* __restrict__ d
 void launch_convert_to_f32(const Launch& L, int dtype, const void* src, float* dst, size_t n) {
   if (!n) return;
   const int blocks = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
-  DLLM_DISPATCH(dtype, (to_f32_kernel<T><<<blocks, 256, 0, L.stream>>>((const T*)src, dst, n)));
+  DLLM_DISPATCH(dtype, (launch_k(L, to_f32_kernel<T>, dim3(blocks), dim3(256), 0, (const T*)src, dst, n)));
   L.count();
 }
 void launch_convert_from_f32(const Launch& L, int dtype, const float* src, void* dst, size_t n) {
   if (!n) return;
   const int blocks = (int)((n + 255) / 256 < 148 * 16 ? (n + 255) / 256 : 148 * 16);
-  DLLM_DISPATCH(dtype, (from_f32_kernel<T><<<blocks, 256, 0, L.stream>>>(src, (T*)dst, n)));
+  DLLM_DISPATCH(dtype, (launch_k(L, from_f32_kernel<T>, dim3(blocks), dim3(256), 0, src, (T*)dst, n)));
   L.count();
 }
 
 __global__ void mask_column_kernel(float* logits, int rows, int vocab, int mask_id) {
+  pdl_wait();
+  pdl_trigger();
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r < rows) logits[(size_t)r * vocab + mask_id] = -INFINITY;
 }
 void launch_mask_column(const Launch& L, float* logits, int rows, int vocab, int mask_id) {
   if (rows <= 0) return;
-  mask_column_kernel<<<(rows + 127) / 128, 128, 0, L.stream>>>(logits, rows, vocab, mask_id);
+  launch_k(L, mask_column_kernel, dim3((rows + 127) / 128), dim3(128), 0, logits, rows, vocab, mask_id);
   L.count();
 }
 

@@ -11,6 +11,8 @@ namespace dllm {
 template <typename T>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A, const T* __restrict__ W,
                                                         float* __restrict__ C, int M, int N, int K) {
+  pdl_wait();
+  pdl_trigger();
   constexpr int BM = 64, BN = 64, BK = 16;
   __shared__ float As[BK][BM + 4];
   __shared__ float Ws[BK][BN + 4];
@@ -56,10 +58,9 @@ void launch_gemm_simt(const Launch& L, int dtype, const void* A, const void* W, 
   if (M <= 0 || N <= 0) return;
   dim3 grid((N + 63) / 64, (M + 63) / 64);
   if (dtype == 0)
-    gemm_simt_kernel<float><<<grid, 256, 0, L.stream>>>((const float*)A, (const float*)W, C, M, N, K);
+    launch_k(L, gemm_simt_kernel<float>, dim3(grid), dim3(256), 0, (const float*)A, (const float*)W, C, M, N, K);
   else
-    gemm_simt_kernel<__nv_bfloat16>
-        <<<grid, 256, 0, L.stream>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)W, C, M, N, K);
+    launch_k(L, gemm_simt_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, (const __nv_bfloat16*)A, (const __nv_bfloat16*)W, C, M, N, K);
   L.count();
 }
 

@@ -128,6 +128,8 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_d = tmem_base_slot;
   volatile int* abortp = &abort_flag;
+  pdl_wait();     // the activation rows come from the preceding kernel
+  pdl_trigger();
 
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer ----------------
@@ -296,7 +298,7 @@ cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMa
   }
   const int stages = plan.stages < 2 ? 2 : plan.stages > max_stages(BN) ? max_stages(BN) : plan.stages;
   dim3 grid((M + BN - 1) / BN, (N + TILE_W - 1) / TILE_W, plan.S);
-  gemm_bf16_tcgen05_kernel<BN><<<grid, 128, SL::total(stages), L.stream>>>(
+  launch_k(L, gemm_bf16_tcgen05_kernel<BN>, dim3(grid), dim3(128), SL::total(stages), 
       tmW, tmA, part, M, N, num_kb, plan.kb_per_split, (size_t)M * N, stages, L.d_status);
   L.count();
   return cudaGetLastError();

@@ -12,10 +12,33 @@ struct Launch {
   cudaStream_t stream;
   int* d_status;        // device status word (may be null for kernel-level hooks)
   uint64_t* counter;    // host launch counter (may be null)
+  bool pdl = false;     // launch with programmatic stream serialization (see launch_k)
   inline void count(int k = 1) const {
     if (counter) *counter += (uint64_t)k;
   }
 };
+
+// Launches `kernel`.  With L.pdl the launch carries the programmatic stream
+// serialization attribute: the grid may become resident while its predecessor
+// in the stream is still running, and everything it does before pdl_wait()
+// (set-up, prefetch of weights, which no kernel writes) overlaps the
+// predecessor's tail.  Every kernel of the library calls pdl_wait() before it
+// touches memory another kernel writes or reads.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(const Launch& L, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                            Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = L.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = L.pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // Split-K partial sums of one GEMM: S slabs of [M, N] fp32, slab stride in floats.
 struct Partials {

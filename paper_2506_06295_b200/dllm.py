@@ -66,6 +66,7 @@ SIGNATURES = {
     "dllm_launch_count": (C.c_uint64, [_P]),
     "dllm_session_use_graphs": (_I, [_P, _I]),
     "dllm_session_use_simt_gemm": (_I, [_P, _I]),
+    "dllm_session_use_pdl": (_I, [_P, _I]),
     "dllm_session_profile": (_I, [_P, _I]),
     "dllm_session_profile_read": (_I, [_P, _I, C.POINTER(C.c_double), C.POINTER(C.c_uint64),
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]),
@@ -296,6 +297,9 @@ class Session:
 
     def use_graphs(self, enable: bool) -> None:
         _check(lib.dllm_session_use_graphs(self.handle, int(enable)))
+
+    def use_pdl(self, enable: bool) -> None:
+        _check(lib.dllm_session_use_pdl(self.handle, int(enable)))
 
     def use_simt_gemm(self, enable: bool) -> None:
         _check(lib.dllm_session_use_simt_gemm(self.handle, int(enable)))
