@@ -149,12 +149,14 @@ Workspace make_workspace(const dllm_config& c, int B, int P, int R) {
   // 148 CTAs of 64 (row, head) pairs exist, so S * pairs < 2 * 148 * 64
   w.attn_floats = (size_t)2 * 148 * 64 * (128 + 2);
   w.attn = take(w.attn_floats * 4);
-  // largest [M, N] any GEMM writes, plus room for split-K slabs of the small-M
-  // launches: S*M*N <= M*N + 148 CTAs * 256 * 128 for every plan
+  // largest [M, N] any GEMM writes, or the slabs of a GEMM whose tiles are
+  // split: splitting happens only below 8 tiles per SM (M*N <= 8 G tiles of
+  // 256 x 128) and a tile has at most G/tiles + 2 slabs, so slabs * M * N <=
+  // (1 + 2 * 8) * G * 256 * 128 floats with G = 160 >= the SM count
   size_t mn = rows * std::max(std::max(dq + dkv, d), 2 * m);
   mn = std::max(mn, BR * V);
   mn = std::max(mn, rows * std::max(d, dkv));
-  w.part_floats = mn + (size_t)148 * 256 * 128 * 2;
+  w.part_floats = std::max(mn, (size_t)17 * 160 * 256 * 128) + 4096;
   w.part = take(w.part_floats * 4);
   w.total = off;
   return w;
@@ -289,12 +291,9 @@ int k_selected(float rho, int R, dllm_kround kr) {
 
 // One GEMM of the step: out = A[M,K] * W[N,K]^T as split-K partial slabs.
 dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void* W, int M, int N, int K,
-                     Partials* out) {
+                     Partials* out, bool whole_tiles = false) {
   float* part = s->wsp<float>(s->ws.part);
-  out->p = part;
-  out->N = N;
-  out->split_stride = (size_t)M * N;
-  out->S = 1;
+  *out = Partials{part, (size_t)M * N, 1, N};
   if (M <= 0) return DLLM_OK;
   // algorithmic traffic of one projection: the weight matrix and the activation
   // rows once in, one fp32 result out (split-K slabs are overhead, not counted)
@@ -309,14 +308,14 @@ dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void
     launch_gemm_simt(L, s->m->cfg.dtype, A, W, part, M, N, K);
     return DLLM_OK;
   }
-  const GemmPlan plan = plan_gemm_bf16(M, N, K);
-  if ((size_t)plan.S * M * N > s->ws.part_floats)
-    return fail(&s->err, DLLM_UNSUPPORTED, "GEMM %dx%dx%d with %d splits exceeds the workspace", M, N, K, plan.S);
+  const GemmPlan plan = plan_gemm_bf16(M, N, K, 0, 0, 0, whole_tiles);
+  if ((size_t)plan.S_max * M * N > s->ws.part_floats)
+    return fail(&s->err, DLLM_UNSUPPORTED, "GEMM %dx%dx%d with %d slabs exceeds the workspace", M, N, K, plan.S_max);
   const char* why = nullptr;
   cudaError_t e = launch_gemm_bf16(L, A, W, part, M, N, K, plan, &why);
   if (e != cudaSuccess)
     return fail(&s->err, DLLM_CUDA_ERROR, "bf16 GEMM %dx%dx%d: %s", M, N, K, why ? why : cudaGetErrorString(e));
-  out->S = plan.S;
+  *out = make_partials(part, M, N, plan);
   return DLLM_OK;
 }
 
@@ -389,7 +388,8 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
   }
   // prediction at the response rows (Eqs. 3-4)
   launch_rmsnorm(L, dt, x, reinterpret_cast<const float*>(W + wl.norm_f), u, d, c.rms_eps, 0, BR);
-  if ((st = run_gemm(s, L, u, W + wl.lm_head, BR, c.vocab, d, &part)) != DLLM_OK) return st;
+  // whole tiles per CTA: the greedy estimate reads the logits as one slab
+  if ((st = run_gemm(s, L, u, W + wl.lm_head, BR, c.vocab, d, &part, true)) != DLLM_OK) return st;
   if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
   launch_argmax_conf(L, part.p, BR, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf));
   cudaError_t e = cudaGetLastError();
@@ -731,7 +731,8 @@ dllm_status dllm_get_logits(dllm_session* s, float* h_out, void* stream) {
   launch_rmsnorm(L, c.dtype, s->wsp<float>(s->ws.x), reinterpret_cast<const float*>(s->m->d_w + s->m->lay.norm_f),
                  s->wsp<uint8_t>(s->ws.u), c.d_model, c.rms_eps, 0, BR);
   Partials part;
-  dllm_status r = run_gemm(s, L, s->wsp<uint8_t>(s->ws.u), s->m->d_w + s->m->lay.lm_head, BR, c.vocab, c.d_model, &part);
+  dllm_status r = run_gemm(s, L, s->wsp<uint8_t>(s->ws.u), s->m->d_w + s->m->lay.lm_head, BR, c.vocab, c.d_model, &part,
+                           true);
   if (r != DLLM_OK) return r;
   launch_mask_column(L, s->wsp<float>(s->ws.part), BR, c.vocab, c.mask_id);
   CU_TRY(&s->err, cudaStreamSynchronize(st));
@@ -882,7 +883,7 @@ dllm_status dllm_session_profile_read(dllm_session* s, int cls, double* total_ms
 size_t dllm_gemm_bf16_scratch_bytes(int M, int N, int K) {
   if (M <= 0 || N <= 0 || K <= 0) return 0;
   const GemmPlan p = plan_gemm_bf16(M, N, K);
-  return p.S > 1 ? (size_t)p.S * M * N * 4 : 0;
+  return p.S_max > 1 ? (size_t)p.S_max * M * N * 4 : 0;
 }
 
 dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, void* d_partials,
@@ -890,34 +891,42 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
   if (!d_A || !d_W || !d_C || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
   if (K % 8) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8");
   const GemmPlan p = plan_gemm_bf16(M, N, K);
-  if (p.S > 1 && !d_partials) return fail(nullptr, DLLM_INVALID_ARG, "this shape needs split-K scratch");
+  if (p.S_max > 1 && !d_partials) return fail(nullptr, DLLM_INVALID_ARG, "this shape needs slab scratch");
   Launch L{(cudaStream_t)stream, nullptr, nullptr};
-  float* part = p.S > 1 ? static_cast<float*>(d_partials) : d_C;
+  float* part = p.S_max > 1 ? static_cast<float*>(d_partials) : d_C;
   const char* why = nullptr;
   cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
   if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "bf16 GEMM: %s", why ? why : cudaGetErrorString(e));
-  if (p.S > 1) launch_reduce_partials(L, Partials{part, (size_t)M * N, p.S, N}, d_C, M);
+  if (p.S_max > 1) launch_reduce_partials(L, make_partials(part, M, N, p), d_C, M);
   CU_TRY(nullptr, cudaGetLastError());
   return DLLM_OK;
 }
 
+size_t dllm_gemm_bf16_planned_scratch_bytes(int M, int N, int K, int act_tile, int w_sub, int ctas) {
+  if (M <= 0 || N <= 0 || K <= 0 || act_tile < 0 || ctas < 0 || w_sub < 0) return 0;
+  const GemmPlan p = plan_gemm_bf16(M, N, K, ctas, 0, act_tile, false, w_sub);
+  return p.S_max > 1 ? (size_t)p.S_max * M * N * 4 : 0;
+}
+
 dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
-                                   int splits, int stages, void* d_partials, size_t partials_bytes, void* stream) {
+                                   int w_sub, int ctas, int stages, int w_tiled, void* d_partials, size_t partials_bytes,
+                                   void* stream) {
   if (!d_A || !d_W || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
   if (K % 8) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8");
-  if (act_tile < 0 || splits < 0 || stages < 0) return fail(nullptr, DLLM_INVALID_ARG, "negative plan parameter");
+  if (act_tile < 0 || ctas < 0 || stages < 0 || w_sub < 0) return fail(nullptr, DLLM_INVALID_ARG, "negative plan parameter");
   if (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 256)
     return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128 or 256");
-  const GemmPlan p = plan_gemm_bf16(M, N, K, splits, stages, act_tile);
-  if (p.S > 1 && (!d_partials || partials_bytes < (size_t)p.S * M * N * 4))
-    return fail(nullptr, DLLM_INVALID_ARG, "this plan needs %zu bytes of split-K scratch", (size_t)p.S * M * N * 4);
+  GemmPlan p = plan_gemm_bf16(M, N, K, ctas, stages, act_tile, false, w_sub);
+  p.w_tiled = w_tiled != 0;
+  if (p.S_max > 1 && (!d_partials || partials_bytes < (size_t)p.S_max * M * N * 4))
+    return fail(nullptr, DLLM_INVALID_ARG, "this plan needs %zu bytes of slab scratch", (size_t)p.S_max * M * N * 4);
   Launch L{(cudaStream_t)stream, nullptr, nullptr};
-  if (!d_C && (p.S == 1 || !d_partials)) return fail(nullptr, DLLM_INVALID_ARG, "d_C is NULL");
-  float* part = p.S > 1 ? static_cast<float*>(d_partials) : d_C;
+  if (!d_C && (p.S_max == 1 || !d_partials)) return fail(nullptr, DLLM_INVALID_ARG, "d_C is NULL");
+  float* part = p.S_max > 1 ? static_cast<float*>(d_partials) : d_C;
   const char* why = nullptr;
   cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
   if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "bf16 GEMM: %s", why ? why : cudaGetErrorString(e));
-  if (p.S > 1 && d_C) launch_reduce_partials(L, Partials{part, (size_t)M * N, p.S, N}, d_C, M);
+  if (p.S_max > 1 && d_C) launch_reduce_partials(L, make_partials(part, M, N, p), d_C, M);
   CU_TRY(nullptr, cudaGetLastError());
   return DLLM_OK;
 }

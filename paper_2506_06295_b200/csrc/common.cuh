@@ -113,11 +113,11 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return warp_sum(t);
 }
 
-// Sum of `S` split-K partial results for eight consecutive columns.
-__device__ __forceinline__ void sum_partials8(const float* part, size_t split_stride, int S, size_t off,
+// Sum of n_slabs partial results for eight consecutive columns, slab 0 first.
+__device__ __forceinline__ void sum_partials8(const float* part, size_t split_stride, int n_slabs, size_t off,
                                               float (&v)[8]) {
   Vec8<float>::load(part + off, v);
-  for (int s = 1; s < S; ++s) {
+  for (int s = 1; s < n_slabs; ++s) {
     float t[8];
     Vec8<float>::load(part + (size_t)s * split_stride + off, t);
 #pragma unroll

@@ -96,7 +96,7 @@ __global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restr
   float dot = 0.f, na = 0.f, nb = 0.f;
   for (int i = threadIdx.x * 8; i < dkv; i += blockDim.x * 8) {
     float vn[8], vo[8];
-    sum_partials8(part.p, part.split_stride, part.S, (size_t)c * part.N + i, vn);
+    sum_partials8(part.p, part.split_stride, part.count(c, i), (size_t)c * part.N + i, vn);
     Vec8<T>::load(vrow + i, vo);
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
@@ -258,11 +258,10 @@ __global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, c
   const float* tab = rope_tab + (size_t)pos * hd;  // [cos(half) | sin(half)]
   for (int i = threadIdx.x; i < half; i += blockDim.x) {
     float lo = 0.f, hi = 0.f;
-    for (int s = 0; s < part.S; ++s) {
-      const float* p = part.p + (size_t)s * part.split_stride + (size_t)r * part.N + col0;
-      lo += p[i];
-      hi += p[i + half];
-    }
+    const int n_lo = part.count(r, col0 + i), n_hi = part.count(r, col0 + i + half);
+    const float* p = part.p + (size_t)r * part.N + col0;
+    for (int s = 0; s < n_lo; ++s) lo += p[(size_t)s * part.split_stride + i];
+    for (int s = 0; s < n_hi; ++s) hi += p[(size_t)s * part.split_stride + i + half];
     const float c = tab[i], sn = tab[half + i];
     dst[i] = from_f32<T>(lo * c - hi * sn);
     dst[i + half] = from_f32<T>(hi * c + lo * sn);
@@ -291,7 +290,7 @@ __global__ void scatter_rows_kernel(Partials part, const int32_t* __restrict__ a
   T* dst = cache + ((size_t)b * g.n + pos) * width;
   for (int i = threadIdx.x * 8; i < width; i += blockDim.x * 8) {
     float v[8];
-    sum_partials8(part.p, part.split_stride, part.S, (size_t)r * part.N + i, v);
+    sum_partials8(part.p, part.split_stride, part.count(r, i), (size_t)r * part.N + i, v);
     Vec8<T>::store(dst + i, v);
   }
 }
@@ -326,7 +325,7 @@ __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__
   float ss = 0.f;
   for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
     float a[8], xv[8];
-    sum_partials8(part.p, part.split_stride, part.S, (size_t)r * part.N + i, a);
+    sum_partials8(part.p, part.split_stride, part.count(r, i), (size_t)r * part.N + i, a);
     Vec8<float>::load(xr + i, xv);
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
@@ -369,8 +368,8 @@ __global__ void silu_mul_kernel(Partials part, T* __restrict__ out, int Ma, int 
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
     const int r = (int)(idx / mv), j = (int)(idx - (size_t)r * mv) * 8;
     float gt[8], up[8];
-    sum_partials8(part.p, part.split_stride, part.S, (size_t)r * part.N + j, gt);
-    sum_partials8(part.p, part.split_stride, part.S, (size_t)r * part.N + m + j, up);
+    sum_partials8(part.p, part.split_stride, part.count(r, j), (size_t)r * part.N + j, gt);
+    sum_partials8(part.p, part.split_stride, part.count(r, m + j), (size_t)r * part.N + m + j, up);
 #pragma unroll
     for (int t = 0; t < 8; ++t) gt[t] = gt[t] / (1.f + expf(-gt[t])) * up[t];
     Vec8<T>::store(out + (size_t)r * m + j, gt);
@@ -532,7 +531,8 @@ __global__ void reduce_partials_kernel(Partials part, float* __restrict__ C, siz
   pdl_trigger();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     float v = part.p[i];
-    for (int s = 1; s < part.S; ++s) v += part.p[(size_t)s * part.split_stride + i];
+    const int n_slabs = part.count((int)(i / part.N), (int)(i % part.N));
+    for (int s = 1; s < n_slabs; ++s) v += part.p[(size_t)s * part.split_stride + i];
     C[i] = v;
   }
 }

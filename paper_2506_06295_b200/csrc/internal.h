@@ -40,12 +40,22 @@ inline cudaError_t launch_k(const Launch& L, void (*kernel)(KArgs...), dim3 grid
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Split-K partial sums of one GEMM: S slabs of [M, N] fp32, slab stride in floats.
+// Partial sums of one GEMM: slabs of [M, N] fp32, slab stride in floats.  With
+// upc == 0 every element has S slabs; otherwise the tile that holds (row, col)
+// has as many slabs as CTAs of the persistent GEMM touched it (see
+// gemm_tcgen05.cu): units of a tile are [tile*num_kb, (tile+1)*num_kb) and CTA
+// i owns units [i*upc, (i+1)*upc).
 struct Partials {
   const float* p;
   size_t split_stride;
   int S;
   int N;  // row length
+  int upc = 0, num_kb = 0, m_tiles = 1, BN = 256, TW = 128;
+  __host__ __device__ inline int count(int row, int col) const {
+    if (upc == 0) return S;
+    const int tile = (col / TW) * m_tiles + row / BN;
+    return ((tile + 1) * num_kb - 1) / upc - (tile * num_kb) / upc + 1;
+  }
 };
 
 // ---------------- api.cu ----------------
@@ -100,12 +110,21 @@ void launch_gemm_simt(const Launch& L, int dtype, const void* A, const void* W, 
 
 // ---------------- gemm_tcgen05.cu ----------------
 struct GemmPlan {
-  int BN;         // activation tile rows (UMMA N)
-  int S;          // split-K factor
-  int kb_per_split;
-  int stages;
+  int BN;           // activation tile rows (UMMA N)
+  int stages;       // depth of the TMA ring
+  int num_kb;       // k-blocks of 64 per tile
+  int m_tiles;      // activation tiles
+  int total_units;  // tiles * num_kb
+  int upc;          // units per CTA
+  int ctas;         // grid size
+  int S_max;        // most slabs any tile is spread over
+  int WM = 1;       // weight sub-tiles of 128 rows per tile
+  int w_tiled = 0;  // W is stored as contiguous 128 x 64 tiles, [N/128][K/64][128][64]
 };
-GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split = 0, int force_stages = 0, int force_bn = 0);  // 0 = auto
+// 0 = auto; whole_tiles: never split a tile's k range (one slab, no reduction needed)
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_ctas = 0, int force_stages = 0, int force_bn = 0,
+                        bool whole_tiles = false, int force_wm = 0);
+Partials make_partials(const float* p, int M, int N, const GemmPlan& plan);
 // Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
                              const GemmPlan& plan, const char** err);
