@@ -181,6 +181,11 @@ dllm_status dllm_session_use_graphs(dllm_session* s, int enable);
  * projections) overlaps the tail of the kernel before it; 0: plain launches. */
 dllm_status dllm_session_use_pdl(dllm_session* s, int enable);
 
+/* 1 (default): steps without prompt refresh (response refresh, adaptive partial)
+ * in bf16 run all layers in one persistent cooperative kernel; 0: kernel by
+ * kernel like the other step kinds. */
+dllm_status dllm_session_use_layer_kernel(dllm_session* s, int enable);
+
 /* Per-kernel timing.  While enabled, steps are launched kernel by kernel (no
  * graph replay) and every projection GEMM (class 0) and attention launch
  * (class 1) is bracketed by CUDA events on the caller's stream.  _profile_read

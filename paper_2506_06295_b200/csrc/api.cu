@@ -15,6 +15,7 @@
 
 #include "../../include/dllm.h"
 #include "internal.h"
+#include "tma.cuh"
 
 using namespace dllm;
 
@@ -114,7 +115,8 @@ uint16_t f32_to_bf16_rne(float f) {
 
 // workspace carve-up
 struct Workspace {
-  size_t status, tokens, x, u, ua, qbuf, obuf, hn, ffn, x0, conf, sim, sel, forced, act, rope, attn, part, total;
+  size_t status, tokens, x, u, ua, qbuf, obuf, hn, ffn, x0, conf, sim, sel, forced, act, inv, mkbar, mkmaps, rope, attn, part,
+      total;
   size_t part_floats, attn_floats;
 };
 
@@ -144,6 +146,9 @@ Workspace make_workspace(const dllm_config& c, int B, int P, int R) {
   w.sel = take(T * BR * 4);
   w.forced = take(T * BR * 4);
   w.act = take(rows * 4);
+  w.inv = take(BR * 4);
+  w.mkbar = take((1 + 13 * T) * 4);  // one grid-barrier counter per phase of the persistent layer kernel
+  w.mkmaps = take((size_t)7 * T * sizeof(CUtensorMap));
   w.rope = take(n * c.head_dim * 4);
   // partial outputs of split key ranges: splits happen only while fewer than
   // 148 CTAs of 64 (row, head) pairs exist, so S * pairs < 2 * 148 * 64
@@ -196,6 +201,8 @@ struct dllm_session {
   bool use_graphs = true;
   bool simt_gemm = false;
   bool use_pdl = true;
+  bool use_mk = true;          // persistent layer kernel for the step kinds it covers
+  bool mk_maps_ready = false;  // weight / cache tensor maps uploaded to the workspace
   struct GraphEntry {
     cudaGraphExec_t exec;
     uint64_t kernels;
@@ -319,6 +326,105 @@ dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void
   return DLLM_OK;
 }
 
+// The layers of a step without prompt refresh as one persistent kernel, then
+// the LM head and the greedy estimate.
+dllm_status enqueue_step_mk(dllm_session* s, int rr, int ksel, cudaStream_t stream) {
+  const dllm_config& c = s->m->cfg;
+  const WeightLayout& wl = s->m->lay;
+  const int d = c.d_model, H = c.n_heads, Hkv = c.n_kv_heads, hd = c.head_dim, m = c.d_ffn;
+  const int dq = H * hd, dkv = Hkv * hd, BR = s->B * s->R;
+  const size_t es = 2, rows = (size_t)s->B * s->n;
+  Launch L{stream, s->wsp<int>(s->ws.status), &s->launches, s->use_pdl};
+  uint8_t* W = s->m->d_w;
+  MkParams p;
+  memset(&p, 0, sizeof p);
+  p.B = s->B; p.P = s->P; p.R = s->R; p.n = s->n; p.d = d; p.H = H; p.Hkv = Hkv; p.hd = hd; p.dq = dq; p.dkv = dkv;
+  p.m = m; p.T = c.n_layers; p.eps = c.rms_eps;
+  p.rr = rr; p.ksel = ksel; p.a_seq = ksel; p.Ma = s->B * ksel; p.BR = BR;
+  for (int l = 0; l < c.n_layers; ++l)
+    if (!rr && s->forced_count[l] >= 0) p.forced_mask |= 1ull << l;
+  p.W = W;
+  const LayerOff& l0 = wl.layers[0];
+  p.o_embed = wl.embed; p.o_norm1 = l0.norm1; p.o_wqkv = l0.wqkv; p.o_wo = l0.wo; p.o_norm2 = l0.norm2;
+  p.o_wgu = l0.wgu; p.o_wd = l0.wd; p.o_norm_f = wl.norm_f;
+  p.layer_stride = c.n_layers > 1 ? wl.layers[1].norm1 - l0.norm1 : 0;
+  p.cache = s->d_cache;
+  p.cache_layer_bytes = s->layer_bytes();
+  p.c_v = rows * dkv * es;
+  p.c_a = 2 * p.c_v;
+  p.c_f = p.c_a + rows * d * es;
+  p.tokens = s->wsp<int32_t>(s->ws.tokens);
+  p.x = s->wsp<float>(s->ws.x);
+  p.u = s->wsp<uint8_t>(s->ws.u);
+  p.ua = rr ? p.u : (void*)s->wsp<uint8_t>(s->ws.ua);  // response refresh: the active rows are all rows, in place
+  p.qbuf = s->wsp<uint8_t>(s->ws.qbuf);
+  p.obuf = s->wsp<uint8_t>(s->ws.obuf);
+  p.hn = s->wsp<uint8_t>(s->ws.hn);
+  p.ffn = s->wsp<uint8_t>(s->ws.ffn);
+  p.sim = s->wsp<float>(s->ws.sim);
+  p.sel = s->wsp<int32_t>(s->ws.sel);
+  p.forced = s->wsp<int32_t>(s->ws.forced);
+  p.act = s->wsp<int32_t>(s->ws.act);
+  p.inv = s->wsp<int32_t>(s->ws.inv);
+  p.rope = s->wsp<float>(s->ws.rope);
+  p.attn_scratch = s->wsp<float>(s->ws.attn);
+  p.part = s->wsp<float>(s->ws.part);
+  p.status = s->wsp<int>(s->ws.status);
+  p.bar = s->wsp<unsigned int>(s->ws.mkbar);
+  p.maps_fixed = s->wsp<CUtensorMap>(s->ws.mkmaps);
+  mk_plan(p);
+  if (p.attn_S > 1 && plan_attention(p.B, p.a_seq, p.n, H, Hkv).scratch_floats > s->ws.attn_floats) {
+    p.attn_S = 1;  // no room for the partials of split key ranges
+    p.attn_kps = (p.n + 63) / 64 * 64;
+    p.has_comb = 0;
+  }
+  if (mk_part_floats(p) > s->ws.part_floats)
+    return fail(&s->err, DLLM_UNSUPPORTED, "the slabs of the persistent layer kernel exceed the workspace");
+  if (!s->mk_maps_ready) {
+    std::vector<CUtensorMap> maps((size_t)7 * c.n_layers);
+    bool ok = true;
+    for (int l = 0; l < c.n_layers && ok; ++l) {
+      const LayerOff& lo = wl.layers[l];
+      uint8_t* Wq = W + lo.wqkv;
+      ok = ok && get_tensor_map_2d(Wq + (size_t)(dq + dkv) * d * es, dkv, d, 128, &maps[l * 5 + MK_V]);
+      ok = ok && get_tensor_map_2d(Wq, dq + dkv, d, 128, &maps[l * 5 + MK_QK]);
+      ok = ok && get_tensor_map_2d(W + lo.wo, d, dq, 128, &maps[l * 5 + MK_O]);
+      ok = ok && get_tensor_map_2d(W + lo.wgu, 2 * (uint64_t)m, d, 128, &maps[l * 5 + MK_GU]);
+      ok = ok && get_tensor_map_2d(W + lo.wd, d, m, 128, &maps[l * 5 + MK_D]);
+      ok = ok && get_tensor_map_3d(s->cache(l, DLLM_CACHE_K), s->B, s->n, dkv, 64, &maps[5 * c.n_layers + 2 * l]);
+      ok = ok && get_tensor_map_3d(s->cache(l, DLLM_CACHE_V), s->B, s->n, dkv, 64, &maps[5 * c.n_layers + 2 * l + 1]);
+    }
+    if (!ok) return fail(&s->err, DLLM_CUDA_ERROR, "cuTensorMapEncodeTiled failed or is unavailable");
+    CU_TRY(&s->err, cudaStreamSynchronize(stream));
+    CU_TRY(&s->err, h2d(s->d_ws + s->ws.mkmaps, maps.data(), maps.size() * sizeof(CUtensorMap), stream));
+    s->mk_maps_ready = true;
+  }
+  const void* a_ptr[5] = {p.u, p.ua, p.obuf, p.hn, p.ffn};
+  const int a_cols[5] = {d, d, dq, d, m};
+  for (int g = 0; g < 5; ++g)
+    if (!get_tensor_map_2d(a_ptr[g], (uint64_t)p.g[g].M, (uint64_t)a_cols[g], (uint32_t)p.g[g].BN, &p.amap[g]))
+      return fail(&s->err, DLLM_CUDA_ERROR, "cuTensorMapEncodeTiled failed or is unavailable");
+  CU_TRY(&s->err, cudaMemsetAsync(p.bar, 0, (size_t)(1 + 13 * c.n_layers) * 4, stream));
+  cudaError_t e = launch_layer_megakernel(L, p);
+  if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "persistent layer kernel: %s", cudaGetErrorString(e));
+  // prediction at the response rows (Eqs. 3-4); u already holds the final norm
+  Partials part;
+  dllm_status st = run_gemm(s, L, p.u, W + wl.lm_head, BR, c.vocab, d, &part, true);
+  if (st != DLLM_OK) return st;
+  if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
+  launch_argmax_conf(L, part.p, BR, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf));
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "step launch: %s", cudaGetErrorString(e));
+  return DLLM_OK;
+}
+
+bool step_uses_mk(const dllm_session* s, int rp, int ksel) {
+  const dllm_config& c = s->m->cfg;
+  return s->use_mk && !s->profiling && !s->simt_gemm &&
+         mk_supported(c.dtype, s->B, s->P, s->R, c.d_model, c.n_heads, c.n_kv_heads, c.head_dim, c.d_ffn, c.n_layers, rp,
+                      ksel);
+}
+
 // Enqueue one denoising step.  Active rows per sequence: the prompt rows on a
 // prompt refresh plus either all R response rows (response refresh) or the
 // ksel rows V-verify picks.
@@ -419,7 +525,9 @@ dllm_status run_step(dllm_session* s, int rp, int rr, float rho, dllm_kround kr,
   cudaStream_t stream = (cudaStream_t)stream_v;
   dllm_status st = DLLM_OK;
   const bool graph_ok = s->use_graphs && !s->profiling && stream != nullptr && stream != cudaStreamLegacy;
-  if (!graph_ok) {
+  if (step_uses_mk(s, rp, ksel)) {
+    st = enqueue_step_mk(s, rr, ksel, stream);  // a handful of launches: no graph needed
+  } else if (!graph_ok) {
     st = enqueue_step(s, rp, rr, ksel, stream);
   } else {
     StepKey key{rp, rr, ksel, forced_signature(s)};
@@ -831,6 +939,12 @@ dllm_status dllm_session_use_pdl(dllm_session* s, int enable) {
     s->graphs.clear();
   }
   s->use_pdl = enable != 0;
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_use_layer_kernel(dllm_session* s, int enable) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  s->use_mk = enable != 0;
   return DLLM_OK;
 }
 

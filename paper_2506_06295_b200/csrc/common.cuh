@@ -27,7 +27,7 @@ __host__ __device__ inline void carried_to_pos(int c, const Geo& g, int& b, int&
 }
 
 // device status word codes
-enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103, ST_RANGE = 201 };
+enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103, ST_TIMEOUT_GRID = 104, ST_RANGE = 201 };
 
 // Programmatic dependent launch.  pdl_wait(): blocks until the preceding grid
 // in the stream has completed and its writes are visible (returns at once for
@@ -47,6 +47,13 @@ struct Vec8<float> {
     v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
     v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
   }
+  // the same through L2 only (data another CTA of the running grid may have written)
+  static __device__ __forceinline__ void load_cg(const float* p, float (&v)[8]) {
+    const float4 a = __ldcg(reinterpret_cast<const float4*>(p));
+    const float4 b = __ldcg(reinterpret_cast<const float4*>(p + 4));
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
   static __device__ __forceinline__ void store(float* p, const float (&v)[8]) {
     *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
     *reinterpret_cast<float4*>(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
@@ -58,6 +65,15 @@ template <>
 struct Vec8<__nv_bfloat16> {
   static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8]) {
     const uint4 u = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+  static __device__ __forceinline__ void load_cg(const __nv_bfloat16* p, float (&v)[8]) {
+    const uint4 u = __ldcg(reinterpret_cast<const uint4*>(p));
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -116,10 +132,10 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 // Sum of n_slabs partial results for eight consecutive columns, slab 0 first.
 __device__ __forceinline__ void sum_partials8(const float* part, size_t split_stride, int n_slabs, size_t off,
                                               float (&v)[8]) {
-  Vec8<float>::load(part + off, v);
+  Vec8<float>::load_cg(part + off, v);
   for (int s = 1; s < n_slabs; ++s) {
     float t[8];
-    Vec8<float>::load(part + (size_t)s * split_stride + off, t);
+    Vec8<float>::load_cg(part + (size_t)s * split_stride + off, t);
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] += t[i];
   }

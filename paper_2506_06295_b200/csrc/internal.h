@@ -1,5 +1,6 @@
 // Host-side launcher interfaces shared by the translation units of the library.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -128,6 +129,51 @@ Partials make_partials(const float* p, int M, int N, const GemmPlan& plan);
 // Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
                              const GemmPlan& plan, const char** err);
+
+// ---------------- megakernel.cu ----------------
+// One projection inside the persistent layer kernel: units (tile, k-block) in
+// tile-major order, tile = nt * m_tiles + mt, CTA i owns units [i*upc, (i+1)*upc).
+struct MkGemm {
+  int M, N, K, BN, m_tiles, num_kb, total, upc;
+};
+enum { MK_V = 0, MK_QK = 1, MK_O = 2, MK_GU = 3, MK_D = 4 };
+struct alignas(64) MkParams {
+  CUtensorMap amap[5];           // activation operands of V, QK, O, GU, D (rows = the operand's row count)
+  int B, P, R, n, d, H, Hkv, hd, dq, dkv, m, T;
+  float eps;
+  int rr, ksel, a_seq, Ma, BR;
+  int attn_S, attn_kps;          // key-range splits of the attention phase, keys per split
+  int has_comb;                  // attention partials are merged in a phase of their own
+  unsigned long long forced_mask;  // bit l: layer l takes its selection from the forced list
+  const uint8_t* W;              // weight blob
+  size_t o_embed, o_norm1, o_wqkv, o_wo, o_norm2, o_wgu, o_wd, o_norm_f, layer_stride;
+  uint8_t* cache;                // cache blob: per layer K, V, AttnOut, FFNOut
+  size_t cache_layer_bytes, c_v, c_a, c_f;
+  const int32_t* tokens;
+  float* x;
+  void *u, *ua, *qbuf, *obuf, *hn, *ffn;
+  float* sim;                    // [T][BR]
+  int32_t* sel;                  // [T][BR]
+  const int32_t* forced;         // [T][BR]
+  int32_t* act;                  // [Ma]
+  int32_t* inv;                  // [BR]: position in the active list or -1
+  const float* rope;
+  float* attn_scratch;
+  float* part;
+  int* status;
+  unsigned int* bar;             // grid barrier counters, one per phase (1 + 13 T), zero at launch
+  const CUtensorMap* maps_fixed; // device: [T][5] weights (V, QK, O, GU, D), then [T][2] K and V caches
+  MkGemm g[5];
+};
+// True if the persistent layer kernel covers this step shape (bf16, no prompt
+// refresh, at least one active row, bounded sizes).
+bool mk_supported(int dtype, int B, int P, int R, int d, int H, int Hkv, int hd, int m, int T, int rp, int ksel);
+// Fills p.g[], attn_S, attn_kps, has_comb from the shapes already in p.
+void mk_plan(MkParams& p);
+size_t mk_part_floats(const MkParams& p);
+// Activation tile rows the kernel uses for an M-row operand.
+int mk_act_tile(int M);
+cudaError_t launch_layer_megakernel(const Launch& L, const MkParams& p);
 
 // ---------------- attention.cu ----------------
 struct AttnPlan {

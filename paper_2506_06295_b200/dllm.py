@@ -67,6 +67,7 @@ SIGNATURES = {
     "dllm_session_use_graphs": (_I, [_P, _I]),
     "dllm_session_use_simt_gemm": (_I, [_P, _I]),
     "dllm_session_use_pdl": (_I, [_P, _I]),
+    "dllm_session_use_layer_kernel": (_I, [_P, _I]),
     "dllm_session_profile": (_I, [_P, _I]),
     "dllm_session_profile_read": (_I, [_P, _I, C.POINTER(C.c_double), C.POINTER(C.c_uint64),
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]),
@@ -301,6 +302,9 @@ class Session:
 
     def use_pdl(self, enable: bool) -> None:
         _check(lib.dllm_session_use_pdl(self.handle, int(enable)))
+
+    def use_layer_kernel(self, enable: bool) -> None:
+        _check(lib.dllm_session_use_layer_kernel(self.handle, int(enable)))
 
     def use_simt_gemm(self, enable: bool) -> None:
         _check(lib.dllm_session_use_simt_gemm(self.handle, int(enable)))
