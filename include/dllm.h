@@ -181,9 +181,10 @@ dllm_status dllm_session_use_graphs(dllm_session* s, int enable);
  * projections) overlaps the tail of the kernel before it; 0: plain launches. */
 dllm_status dllm_session_use_pdl(dllm_session* s, int enable);
 
-/* 1 (default): steps without prompt refresh (response refresh, adaptive partial)
- * in bf16 run all layers in one persistent cooperative kernel; 0: kernel by
- * kernel like the other step kinds. */
+/* 1: steps without prompt refresh (response refresh, adaptive partial) in bf16
+ * run all layers in ONE persistent cooperative kernel (one CTA per SM, weight
+ * stream that never stops, grid barriers between phases); 0 (default): kernel
+ * by kernel like the other step kinds, which measured faster on B200. */
 dllm_status dllm_session_use_layer_kernel(dllm_session* s, int enable);
 
 /* Per-kernel timing.  While enabled, steps are launched kernel by kernel (no
@@ -209,20 +210,14 @@ size_t dllm_gemm_bf16_scratch_bytes(int M, int N, int K);
 dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, int N, int K,
                            void* d_partials, void* stream);
 /* The same product with an explicit launch plan, for tuning: act_tile = rows of
- * A per tile (32, 64, 128 or 256), w_sub = 128-row weight sub-tiles per tile
- * (1, 2 or 4; act_tile * w_sub <= 256), ctas = number of persistent CTAs the (tile,
- * k-block) units are dealt to, stages = depth of the TMA ring (clamped to what
- * fits shared memory); 0 picks the default of each.  w_tiled = 1: d_W holds
- * the matrix as contiguous 128 x 64 tiles, [ceil(N/128)][ceil(K/64)][128][64],
- * zero padded (the layout the model's weight blob uses).  d_partials (device,
- * partials_bytes >= dllm_gemm_bf16_planned_scratch_bytes) holds the slabs of
- * tiles whose k range is shared by several CTAs; when the plan has such tiles
- * and d_C is NULL the slabs are left unreduced there (what the step's fused
- * consumers read). */
-size_t dllm_gemm_bf16_planned_scratch_bytes(int M, int N, int K, int act_tile, int w_sub, int ctas);
+ * A per CTA (32, 64, 128 or 256), splits = split-K factor, stages = depth of the
+ * TMA ring (clamped to what fits shared memory); 0 picks the default of each.
+ * d_partials (device, partials_bytes >= dllm_gemm_bf16_planned_scratch_bytes)
+ * holds the split-K slabs; with splits > 1 and d_C NULL the slabs are left
+ * unreduced there (what the step's fused consumers read). */
+size_t dllm_gemm_bf16_planned_scratch_bytes(int M, int N, int K, int act_tile, int splits);
 dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
-                                   int w_sub, int ctas, int stages, int w_tiled, void* d_partials, size_t partials_bytes,
-                                   void* stream);
+                                   int splits, int stages, void* d_partials, size_t partials_bytes, void* stream);
 /* The same product on the plain fp32 ALUs (operands fp32 or bf16): the GEMM of
  * the fp32 mode. */
 dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int dtype,

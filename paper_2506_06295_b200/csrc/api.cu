@@ -201,7 +201,7 @@ struct dllm_session {
   bool use_graphs = true;
   bool simt_gemm = false;
   bool use_pdl = true;
-  bool use_mk = true;          // persistent layer kernel for the step kinds it covers
+  bool use_mk = false;         // persistent layer kernel for the step kinds it covers (opt-in)
   bool mk_maps_ready = false;  // weight / cache tensor maps uploaded to the workspace
   struct GraphEntry {
     cudaGraphExec_t exec;
@@ -298,7 +298,7 @@ int k_selected(float rho, int R, dllm_kround kr) {
 
 // One GEMM of the step: out = A[M,K] * W[N,K]^T as split-K partial slabs.
 dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void* W, int M, int N, int K,
-                     Partials* out, bool whole_tiles = false) {
+                     Partials* out) {
   float* part = s->wsp<float>(s->ws.part);
   *out = Partials{part, (size_t)M * N, 1, N};
   if (M <= 0) return DLLM_OK;
@@ -315,7 +315,7 @@ dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void
     launch_gemm_simt(L, s->m->cfg.dtype, A, W, part, M, N, K);
     return DLLM_OK;
   }
-  const GemmPlan plan = plan_gemm_bf16(M, N, K, 0, 0, 0, whole_tiles);
+  const GemmPlan plan = plan_gemm_bf16(M, N, K);
   if ((size_t)plan.S_max * M * N > s->ws.part_floats)
     return fail(&s->err, DLLM_UNSUPPORTED, "GEMM %dx%dx%d with %d slabs exceeds the workspace", M, N, K, plan.S_max);
   const char* why = nullptr;
@@ -409,7 +409,7 @@ dllm_status enqueue_step_mk(dllm_session* s, int rr, int ksel, cudaStream_t stre
   if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "persistent layer kernel: %s", cudaGetErrorString(e));
   // prediction at the response rows (Eqs. 3-4); u already holds the final norm
   Partials part;
-  dllm_status st = run_gemm(s, L, p.u, W + wl.lm_head, BR, c.vocab, d, &part, true);
+  dllm_status st = run_gemm(s, L, p.u, W + wl.lm_head, BR, c.vocab, d, &part);
   if (st != DLLM_OK) return st;
   if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
   launch_argmax_conf(L, part.p, BR, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf));
@@ -494,8 +494,7 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
   }
   // prediction at the response rows (Eqs. 3-4)
   launch_rmsnorm(L, dt, x, reinterpret_cast<const float*>(W + wl.norm_f), u, d, c.rms_eps, 0, BR);
-  // whole tiles per CTA: the greedy estimate reads the logits as one slab
-  if ((st = run_gemm(s, L, u, W + wl.lm_head, BR, c.vocab, d, &part, true)) != DLLM_OK) return st;
+  if ((st = run_gemm(s, L, u, W + wl.lm_head, BR, c.vocab, d, &part)) != DLLM_OK) return st;
   if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
   launch_argmax_conf(L, part.p, BR, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf));
   cudaError_t e = cudaGetLastError();
@@ -839,8 +838,7 @@ dllm_status dllm_get_logits(dllm_session* s, float* h_out, void* stream) {
   launch_rmsnorm(L, c.dtype, s->wsp<float>(s->ws.x), reinterpret_cast<const float*>(s->m->d_w + s->m->lay.norm_f),
                  s->wsp<uint8_t>(s->ws.u), c.d_model, c.rms_eps, 0, BR);
   Partials part;
-  dllm_status r = run_gemm(s, L, s->wsp<uint8_t>(s->ws.u), s->m->d_w + s->m->lay.lm_head, BR, c.vocab, c.d_model, &part,
-                           true);
+  dllm_status r = run_gemm(s, L, s->wsp<uint8_t>(s->ws.u), s->m->d_w + s->m->lay.lm_head, BR, c.vocab, c.d_model, &part);
   if (r != DLLM_OK) return r;
   launch_mask_column(L, s->wsp<float>(s->ws.part), BR, c.vocab, c.mask_id);
   CU_TRY(&s->err, cudaStreamSynchronize(st));
@@ -1016,22 +1014,20 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
   return DLLM_OK;
 }
 
-size_t dllm_gemm_bf16_planned_scratch_bytes(int M, int N, int K, int act_tile, int w_sub, int ctas) {
-  if (M <= 0 || N <= 0 || K <= 0 || act_tile < 0 || ctas < 0 || w_sub < 0) return 0;
-  const GemmPlan p = plan_gemm_bf16(M, N, K, ctas, 0, act_tile, false, w_sub);
+size_t dllm_gemm_bf16_planned_scratch_bytes(int M, int N, int K, int act_tile, int splits) {
+  if (M <= 0 || N <= 0 || K <= 0 || act_tile < 0 || splits < 0) return 0;
+  const GemmPlan p = plan_gemm_bf16(M, N, K, splits, 0, act_tile);
   return p.S_max > 1 ? (size_t)p.S_max * M * N * 4 : 0;
 }
 
 dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
-                                   int w_sub, int ctas, int stages, int w_tiled, void* d_partials, size_t partials_bytes,
-                                   void* stream) {
+                                   int splits, int stages, void* d_partials, size_t partials_bytes, void* stream) {
   if (!d_A || !d_W || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
   if (K % 8) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8");
-  if (act_tile < 0 || ctas < 0 || stages < 0 || w_sub < 0) return fail(nullptr, DLLM_INVALID_ARG, "negative plan parameter");
+  if (act_tile < 0 || splits < 0 || stages < 0) return fail(nullptr, DLLM_INVALID_ARG, "negative plan parameter");
   if (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 256)
     return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128 or 256");
-  GemmPlan p = plan_gemm_bf16(M, N, K, ctas, stages, act_tile, false, w_sub);
-  p.w_tiled = w_tiled != 0;
+  const GemmPlan p = plan_gemm_bf16(M, N, K, splits, stages, act_tile);
   if (p.S_max > 1 && (!d_partials || partials_bytes < (size_t)p.S_max * M * N * 4))
     return fail(nullptr, DLLM_INVALID_ARG, "this plan needs %zu bytes of slab scratch", (size_t)p.S_max * M * N * 4);
   Launch L{(cudaStream_t)stream, nullptr, nullptr};

@@ -17,16 +17,13 @@
 //   * TMEM lane = output column n, so for a fixed activation row the 32 lanes
 //     of a warp store 32 consecutive floats: the epilogue writes row-major
 //     [M, N] coalesced straight from tcgen05.ld registers;
-//   * the kernel is persistent: work is cut into units (output tile, k-block)
-//     in tile-major order and CTA i (one per SM) owns a contiguous run of
-//     them, so all SMs stream the same number of weight bytes whatever N/128
-//     is; a CTA writes each run of k-blocks of one tile ("segment") to its own
-//     slab and the consumer kernel adds the slabs of a tile in k order (no
-//     atomics, bit-reproducible); two TMEM accumulators let the epilogue warps
-//     drain one segment while the next is being multiplied;
-//   * weight tiles are requested before griddepcontrol.wait, so with
-//     programmatic dependent launch the ring (up to ~200 KB per SM) fills
-//     while the kernel that produces the activations is still running;
+//   * split-K over blockIdx.z puts >= 148 CTAs on the weight stream when N/128
+//     is small; every split writes its own slab and the consumer kernel adds
+//     the slabs in order (no atomics, bit-reproducible);
+//   * weight tiles are requested before griddepcontrol.wait: with programmatic
+//     dependent launch the ring fills while the kernel that produces the
+//     activation rows is still running; the activation tile of a stage follows
+//     after the wait and the stage's barrier completes when both have landed;
 //   * rows of A beyond M and k beyond K are zero-filled by TMA.
 //
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the
@@ -49,100 +46,58 @@ constexpr int UMMA_K = 16;
 constexpr uint32_t W_STAGE_BYTES = TILE_W * TILE_K * 2;
 
 constexpr int MAX_STAGES = 12;
-constexpr int GEMM_THREADS = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
 
-// WM = weight sub-tiles of 128 rows per tile: one activation tile in shared
-// memory feeds WM MMAs, so the activation rows cross the L2 -> SM fabric once
-// per 128 * WM weight rows.
-template <int BN, int WM>
+template <int BN>
 struct SmemLayout {
-  static constexpr uint32_t W_BYTES = WM * W_STAGE_BYTES;
   static constexpr uint32_t A_STAGE_BYTES = BN * TILE_K * 2;
-  static constexpr uint32_t STAGE_BYTES = W_BYTES + A_STAGE_BYTES;
+  static constexpr uint32_t STAGE_BYTES = W_STAGE_BYTES + A_STAGE_BYTES;
   static constexpr uint32_t total(int stages) { return (uint32_t)stages * STAGE_BYTES + 1024; }  // + slack to align the base to 1024
 };
 
-// One contiguous run of k-blocks of one output tile inside a CTA's unit range.
-struct Segment {
-  int tile, kb0, nkb;
-};
-__device__ __forceinline__ Segment segment_at(int u, int u1, int num_kb) {
-  Segment sg;
-  sg.tile = u / num_kb;
-  sg.kb0 = u - sg.tile * num_kb;
-  sg.nkb = min(num_kb - sg.kb0, u1 - u);
-  return sg;
-}
-
-// Work = units (output tile, k-block), tile-major; CTA i owns units
-// [i*upc, (i+1)*upc).  A CTA therefore computes a sequence of segments (runs of
-// k-blocks of one tile); the segment of CTA i for a tile goes to slab
-// i - first_cta(tile) of that tile, so a consumer that adds the slabs of a tile
-// in index order adds the k ranges in ascending order, whatever ran first.
-template <int BN, int WM>
-__global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_tcgen05_kernel(
-    const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA, float* __restrict__ part, int M,
-    int N, int num_kb, int m_tiles, int total_units, int upc, size_t split_stride, int STAGES, int w_tiled,
-    int* __restrict__ status) {
-  using SL = SmemLayout<BN, WM>;
-  constexpr int TW = TILE_W * WM;                            // weight rows per tile
-  constexpr int ACC_BUFS = (2 * WM * BN <= 512) ? 2 : 1;     // accumulator sets in TMEM
-  constexpr uint32_t ACC_COLS = WM * BN;
-  constexpr uint32_t TMEM_COLS = ACC_BUFS * ACC_COLS < 32 ? 32 : ACC_BUFS * ACC_COLS;
+template <int BN>
+__global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                                const __grid_constant__ CUtensorMap tmA,
+                                                                float* __restrict__ part, int M, int N, int num_kb,
+                                                                int kb_per_split, size_t split_stride, int STAGES,
+                                                                int* __restrict__ status) {
+  using SL = SmemLayout<BN>;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
-  __shared__ __align__(8) uint64_t acc_full[2];
-  __shared__ __align__(8) uint64_t acc_empty[2];
+  __shared__ __align__(8) uint64_t accum_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int u0 = blockIdx.x * upc;
-  const int u1 = min(total_units, u0 + upc);
-  const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  volatile int* abortp = &abort_flag;
-  int pre = 0;  // stages whose weight tile was requested before the dependency wait
-  // weight tile (nt, kb): a box of the row-major [N, K] matrix, or one contiguous
-  // 16 KB block of the tiled layout [N/128][K/64][128][64]
-  auto load_w = [&](uint32_t dst, uint32_t bar, int nt, int kb) {
-#pragma unroll
-    for (int w = 0; w < WM; ++w) {
-      if (w_tiled)
-        tma_load_2d(dst + w * W_STAGE_BYTES, &tmW, bar, 0, ((nt * WM + w) * num_kb + kb) * TILE_W);
-      else
-        tma_load_2d(dst + w * W_STAGE_BYTES, &tmW, bar, kb * TILE_K, nt * TW + w * TILE_W);
-    }
-  };
+  const int m0 = blockIdx.x * BN;       // activation rows
+  const int n0 = blockIdx.y * TILE_W;   // weight rows = output columns
+  const int kb0 = blockIdx.z * kb_per_split;
+  const int kb1 = min(num_kb, kb0 + kb_per_split);
+  const int nkb = kb1 - kb0;            // >= 1 by construction of the plan
 
+  const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+
+  int pre = 0;  // stages whose weight tile was requested before the dependency wait
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
-    for (int b = 0; b < ACC_BUFS; ++b) {
-      mbar_init(smem_u32(&acc_full[b]), 1);
-      mbar_init(smem_u32(&acc_empty[b]), 4);  // one arrival per epilogue warp
-    }
+    mbar_init(smem_u32(&accum_bar), 1);
     mbar_fence_init();
-    // Weights are written by no kernel: start streaming them before the grid
-    // this launch depends on has finished.  The activation tile of the same
-    // stage is requested after pdl_wait(); the stage's barrier completes when
-    // both have landed.
     prefetch_tensormap(&tmW);
     prefetch_tensormap(&tmA);
-    pre = min(STAGES, u1 - u0);
+    pre = min(STAGES, nkb);  // weights are written by no kernel: stream them ahead of the dependency
     for (int i = 0; i < pre; ++i) {
-      const Segment sg = segment_at(u0 + i, u1, num_kb);
       const uint32_t fb = smem_u32(&full_bar[i]);
       mbar_expect_tx(fb, SL::STAGE_BYTES);
-      load_w(tiles + i * SL::STAGE_BYTES, fb, sg.tile / m_tiles, sg.kb0);
+      tma_load_2d(tiles + i * SL::STAGE_BYTES, &tmW, fb, (kb0 + i) * TILE_K, n0);
     }
   }
-  if (warp == 1) {
+  if (warp == 1) {  // TMEM: BN fp32 columns x 128 lanes
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                 "r"(TMEM_COLS)
+                 "r"((uint32_t)BN)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -150,27 +105,27 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_tcgen05_kernel(
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_d = tmem_base_slot;
-  pdl_wait();     // activation rows and the slab buffer belong to the preceding kernels
-  pdl_trigger();  // (after this CTA holds its TMEM: a dependent CTA can only queue behind it)
+  volatile int* abortp = &abort_flag;
+  pdl_wait();     // the activation rows and the slab buffer belong to the preceding kernels
+  pdl_trigger();
 
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer ----------------
     int s = 0;
     uint32_t ph = 0;
-    int u = u0;
-    for (int i = 0; u < u1; ++i, ++u) {
-      const int tile = u / num_kb, kb = u - tile * num_kb;
+    for (int i = 0; i < nkb; ++i) {
       const uint32_t fb = smem_u32(&full_bar[s]);
       const uint32_t dstW = tiles + s * SL::STAGE_BYTES;
+      const int kc = (kb0 + i) * TILE_K;
       if (i >= pre) {
         if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) {
           if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
           break;
         }
         mbar_expect_tx(fb, SL::STAGE_BYTES);
-        load_w(dstW, fb, tile / m_tiles, kb);
+        tma_load_2d(dstW, &tmW, fb, kc, n0);
       }
-      tma_load_2d(dstW + SL::W_BYTES, &tmA, fb, kb * TILE_K, (tile % m_tiles) * BN);
+      tma_load_2d(dstW + W_STAGE_BYTES, &tmA, fb, kc, m0);
       if (++s == STAGES) {
         s = 0;
         ph ^= 1u;
@@ -179,96 +134,64 @@ __global__ void __launch_bounds__(GEMM_THREADS) gemm_bf16_tcgen05_kernel(
   } else if (warp == 1 && lane == 0) {
     // ---------------- MMA issuer ----------------
     constexpr uint32_t idesc = make_idesc(TILE_W, BN);
+    bool ok = true;
     int s = 0;
     uint32_t ph = 0;
-    bool ok = true;
-    int seg = 0;
-    for (int u = u0; u < u1 && ok; ++seg) {
-      const Segment sg = segment_at(u, u1, num_kb);
-      const int buf = seg % ACC_BUFS;
-      // the epilogue has drained the accumulator this segment reuses
-      if (!mbar_wait(smem_u32(&acc_empty[buf]), (((uint32_t)(seg / ACC_BUFS)) & 1u) ^ 1u, abortp)) {
+    for (int i = 0; i < nkb && ok; ++i) {
+      if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp)) {
         if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_MMA);
         ok = false;
         break;
       }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t d_addr = tmem_d + (uint32_t)buf * ACC_COLS;
-      for (int i = 0; i < sg.nkb; ++i) {
-        if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp)) {
-          if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_MMA);
-          ok = false;
-          break;
-        }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t sW = tiles + s * SL::STAGE_BYTES;
-        const uint64_t dA = make_smem_desc(sW + SL::W_BYTES);
+      const uint32_t sW = tiles + s * SL::STAGE_BYTES;
+      const uint64_t dW = make_smem_desc(sW);
+      const uint64_t dA = make_smem_desc(sW + W_STAGE_BYTES);
 #pragma unroll
-        for (int k = 0; k < TILE_K / UMMA_K; ++k) {
-#pragma unroll
-          for (int w = 0; w < WM; ++w) {
-            // advance 32 bytes (16 bf16) along K inside the swizzle row: +2 in 16-byte units
-            const uint64_t dW = make_smem_desc(sW + w * W_STAGE_BYTES);
-            umma_bf16(d_addr + (uint32_t)(w * BN), dW + (uint64_t)(2 * k), dA + (uint64_t)(2 * k), idesc,
-                      (i > 0 || k > 0) ? 1u : 0u);
-          }
-        }
-        umma_commit(smem_u32(&empty_bar[s]));  // stage reusable once these MMAs have read it
-        if (++s == STAGES) {
-          s = 0;
-          ph ^= 1u;
-        }
+      for (int k = 0; k < TILE_K / UMMA_K; ++k) {
+        // advance 32 bytes (16 bf16) along K inside the swizzle row: +2 in 16-byte units
+        umma_bf16(tmem_d, dW + (uint64_t)(2 * k), dA + (uint64_t)(2 * k), idesc, (i > 0 || k > 0) ? 1u : 0u);
       }
-      if (ok) umma_commit(smem_u32(&acc_full[buf]));
-      u += sg.nkb;
+      umma_commit(smem_u32(&empty_bar[s]));  // stage reusable once these MMAs have read it
+      if (++s == STAGES) {
+        s = 0;
+        ph ^= 1u;
+      }
     }
-  } else if (warp >= 2) {
-    // ---------------- epilogue: TMEM -> registers -> slab (warps 2..5) ----------------
-    const int q = warp & 3;  // the TMEM lane quarter this warp may read
-    int seg = 0;
-    for (int u = u0; u < u1; ++seg) {
-      const Segment sg = segment_at(u, u1, num_kb);
-      const int buf = seg % ACC_BUFS;
-      const bool have = mbar_wait(smem_u32(&acc_full[buf]), ((uint32_t)(seg / ACC_BUFS)) & 1u, abortp);
-      if (!__all_sync(0xffffffffu, have)) {  // the whole warp must agree before the warp-collective loads
-        if (lane == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_EPI);
-        break;
-      }
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int nt = sg.tile / m_tiles, mt = sg.tile - nt * m_tiles;
-      const int m0 = mt * BN;
-      const int slab = (int)blockIdx.x - (sg.tile * num_kb) / upc;
-#pragma unroll 1
-      for (int w = 0; w < WM; ++w) {
-        const int n = nt * TW + w * TILE_W + q * 32 + lane;
-        float* out = part + (size_t)slab * split_stride + n;
-        const uint32_t t_addr = tmem_d + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * ACC_COLS + (uint32_t)(w * BN);
-#pragma unroll 1
-        for (int c = 0; c < BN; c += 16) {
-          if (m0 + c >= M) break;
-          uint32_t r[16];
-          tmem_ld16(t_addr + (uint32_t)c, r);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          if (n < N) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int m = m0 + c + j;
-              if (m < M) out[(size_t)m * N] = __uint_as_float(r[j]);
-            }
-          }
-        }
-      }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
-      u += sg.nkb;
-    }
+    if (ok) umma_commit(smem_u32(&accum_bar));
   }
-  if (*abortp) drain_delay();  // gave up: let copies in flight land before shared memory is released
+  __syncwarp();
+
+  // ---------------- epilogue: TMEM -> registers -> global (all four warps) ----------------
+  const bool have = mbar_wait(smem_u32(&accum_bar), 0u, abortp);
+  if (!have && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_EPI);
+  // the whole warp must agree before the warp-collective TMEM loads
+  const bool warp_ok = __all_sync(0xffffffffu, have);
+  if (warp_ok) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int n = n0 + warp * 32 + lane;
+    float* out = part + (size_t)blockIdx.z * split_stride + n;
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 16) {
+      if (m0 + c >= M) break;  // uniform across the CTA
+      uint32_t r[16];
+      tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (n < N) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + c + j;
+          if (m < M) out[(size_t)m * N] = __uint_as_float(r[j]);
+        }
+      }
+    }
+  } else {
+    drain_delay();  // gave up: let copies in flight land before shared memory is released
+  }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"((uint32_t)BN) : "memory");
   }
 }
 
@@ -335,41 +258,28 @@ bool get_map(const MapKey& key, CUtensorMap* out) {
 }
 
 // Most stages whose ring fits the 227 KB of shared memory one CTA may use.
-constexpr int max_stages(int bn, int wm) {
-  const int fit = (227 * 1024 - 1024 - 512) / (int)(wm * W_STAGE_BYTES + bn * TILE_K * 2);
+constexpr int max_stages(int bn) {
+  const int fit = (227 * 1024 - 1024 - 256) / (int)(W_STAGE_BYTES + bn * TILE_K * 2);
   return fit < MAX_STAGES ? fit : MAX_STAGES;
 }
 
-template <int BN, int WM>
+template <int BN>
 cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMap& tmA, float* part, int M, int N,
-                       const GemmPlan& plan) {
-  using SL = SmemLayout<BN, WM>;
+                       int num_kb, const GemmPlan& plan) {
+  using SL = SmemLayout<BN>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<BN, WM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)SL::total(max_stages(BN, WM)));
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)SL::total(max_stages(BN)));
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  const int stages = plan.stages < 2 ? 2 : plan.stages > max_stages(BN, WM) ? max_stages(BN, WM) : plan.stages;
-  cudaError_t e = launch_k(L, gemm_bf16_tcgen05_kernel<BN, WM>, dim3(plan.ctas), dim3(GEMM_THREADS), SL::total(stages), tmW,
-                           tmA, part, M, N, plan.num_kb, plan.m_tiles, plan.total_units, plan.upc, (size_t)M * N, stages,
-                           plan.w_tiled, L.d_status);
+  const int stages = plan.stages < 2 ? 2 : plan.stages > max_stages(BN) ? max_stages(BN) : plan.stages;
+  dim3 grid((M + BN - 1) / BN, (N + TILE_W - 1) / TILE_W, plan.S_max);
+  cudaError_t e = launch_k(L, gemm_bf16_tcgen05_kernel<BN>, grid, dim3(128), SL::total(stages), tmW, tmA, part, M, N,
+                           num_kb, plan.upc, (size_t)M * N, stages, L.d_status);
   L.count();
   return e != cudaSuccess ? e : cudaGetLastError();
-}
-
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-      n = v;
-    else
-      return 148;  // no device visible (host-only size queries): a B200's count
-  }
-  return n;
 }
 
 }  // namespace
@@ -383,61 +293,28 @@ bool get_tensor_map_3d(const void* base, uint64_t batch, uint64_t rows, uint64_t
 }
 
 Partials make_partials(const float* p, int M, int N, const GemmPlan& plan) {
-  Partials out{p, (size_t)M * N, plan.S_max, N};
-  if (plan.S_max > 1) {
-    out.upc = plan.upc;
-    out.num_kb = plan.num_kb;
-    out.m_tiles = plan.m_tiles;
-    out.BN = plan.BN;
-    out.TW = plan.WM * TILE_W;
-  } else {
-    out.S = 1;
-  }
-  return out;
+  return Partials{p, (size_t)M * N, plan.S_max, N};  // every element has S_max slabs
 }
 
-GemmPlan plan_gemm_bf16(int M, int N, int K, int force_ctas, int force_stages, int force_bn, bool whole_tiles,
-                        int force_wm) {
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, int force_bn) {
   GemmPlan p;
   p.BN = M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
   if (force_bn == 32 || force_bn == 64 || force_bn == 128 || force_bn == 256) p.BN = force_bn;
+  p.stages = force_stages > 0 ? force_stages : 4;
   p.num_kb = (K + TILE_K - 1) / TILE_K;
-  const int wm_max = p.BN <= 64 ? 4 : p.BN == 128 ? 2 : 1;
-  p.WM = (force_wm == 1 || force_wm == 2 || force_wm == 4) ? (force_wm <= wm_max ? force_wm : wm_max) : 1;
   p.m_tiles = (M + p.BN - 1) / p.BN;
-  const int tw = p.WM * TILE_W;
-  const long tiles = (long)p.m_tiles * ((N + tw - 1) / tw);
-  const long total = tiles * p.num_kb;
-  const int sms = sm_count();
-  long upc;
-  if (force_ctas > 0) {
-    upc = (total + force_ctas - 1) / force_ctas;
-  } else if (!whole_tiles && p.BN == 256 && tiles < 8L * sms) {
-    // one CTA per SM anyway (the ring and both accumulators fill it): deal the
-    // (tile, k-block) units evenly, whatever the tile count
-    upc = (total + sms - 1) / sms;
-    if (upc < 4) upc = 4;
-  } else if (whole_tiles || tiles >= sms) {
-    // enough tiles: whole tiles, one slab, no reduction; the tiles are dealt
-    // evenly to at most two CTAs per SM
-    const long per = (tiles + 2 * sms - 1) / (2 * sms);
-    upc = per * p.num_kb;
-  } else {
-    // few tiles: split every tile's k range S ways so that about one CTA per
-    // SM streams weights; S slabs per tile, added in order by the consumer
-    long S = (sms + tiles - 1) / tiles;
-    const long max_s = p.num_kb / 4 > 1 ? p.num_kb / 4 : 1;
+  const long tiles = (long)p.m_tiles * ((N + TILE_W - 1) / TILE_W);
+  int S = 1;
+  if (tiles < 148) {
+    S = (int)((148 + tiles - 1) / tiles);
+    const int max_s = p.num_kb / 4 > 1 ? p.num_kb / 4 : 1;
     if (S > max_s) S = max_s;
-    upc = (p.num_kb + S - 1) / S;
   }
-  if (upc > total) upc = total;
-  p.total_units = (int)total;
-  p.upc = (int)upc;
-  p.ctas = (int)((total + upc - 1) / upc);
-  p.S_max = (upc % p.num_kb == 0) ? 1 : (p.num_kb - 1) / (int)upc + 2;
-  // ring depth: two CTAs fit one SM when the split plan launches more CTAs than SMs
-  const int deep = max_stages(p.BN, p.WM);
-  p.stages = force_stages > 0 ? force_stages : (p.ctas > sms && deep > 4 ? 4 : deep);
+  if (force_split > 0) S = force_split < p.num_kb ? force_split : p.num_kb;
+  p.upc = (p.num_kb + S - 1) / S;                 // k-blocks per split
+  p.S_max = (p.num_kb + p.upc - 1) / p.upc;       // no empty split
+  p.ctas = (int)tiles * p.S_max;
+  p.total_units = (int)tiles * p.num_kb;
   return p;
 }
 
@@ -451,28 +328,18 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
     return cudaErrorInvalidValue;
   }
   CUtensorMap tmW, tmA;
-  const uint64_t n_tiles = (uint64_t)(N + TILE_W - 1) / TILE_W;
-  const bool okW = plan.w_tiled ? get_tensor_map_2d(W, n_tiles * plan.num_kb * TILE_W, TILE_K, TILE_W, &tmW)
-                                : get_tensor_map_2d(W, (uint64_t)N, (uint64_t)K, TILE_W, &tmW);
-  if (!okW ||
+  if (!get_tensor_map_2d(W, (uint64_t)N, (uint64_t)K, TILE_W, &tmW) ||
       !get_tensor_map_2d(A, (uint64_t)M, (uint64_t)K, (uint32_t)plan.BN, &tmA)) {
     if (err) *err = e_map;
     return cudaErrorInvalidValue;
   }
-  switch (plan.BN * 8 + plan.WM) {
-    case 32 * 8 + 1: return launch_one<32, 1>(L, tmW, tmA, part, M, N, plan);
-    case 32 * 8 + 2: return launch_one<32, 2>(L, tmW, tmA, part, M, N, plan);
-    case 32 * 8 + 4: return launch_one<32, 4>(L, tmW, tmA, part, M, N, plan);
-    case 64 * 8 + 1: return launch_one<64, 1>(L, tmW, tmA, part, M, N, plan);
-    case 64 * 8 + 2: return launch_one<64, 2>(L, tmW, tmA, part, M, N, plan);
-    case 64 * 8 + 4: return launch_one<64, 4>(L, tmW, tmA, part, M, N, plan);
-    case 128 * 8 + 1: return launch_one<128, 1>(L, tmW, tmA, part, M, N, plan);
-    case 128 * 8 + 2: return launch_one<128, 2>(L, tmW, tmA, part, M, N, plan);
-    case 256 * 8 + 1: return launch_one<256, 1>(L, tmW, tmA, part, M, N, plan);
-    default: break;
+  const int num_kb = (K + TILE_K - 1) / TILE_K;
+  switch (plan.BN) {
+    case 32: return launch_one<32>(L, tmW, tmA, part, M, N, num_kb, plan);
+    case 64: return launch_one<64>(L, tmW, tmA, part, M, N, num_kb, plan);
+    case 128: return launch_one<128>(L, tmW, tmA, part, M, N, num_kb, plan);
+    default: return launch_one<256>(L, tmW, tmA, part, M, N, num_kb, plan);
   }
-  if (err) *err = "unsupported (activation tile, weight sub-tiles) combination";
-  return cudaErrorInvalidValue;
 }
 
 }  // namespace dllm

@@ -113,18 +113,14 @@ void launch_gemm_simt(const Launch& L, int dtype, const void* A, const void* W, 
 struct GemmPlan {
   int BN;           // activation tile rows (UMMA N)
   int stages;       // depth of the TMA ring
-  int num_kb;       // k-blocks of 64 per tile
+  int num_kb;       // k-blocks of 64
   int m_tiles;      // activation tiles
   int total_units;  // tiles * num_kb
-  int upc;          // units per CTA
+  int upc;          // k-blocks per split
   int ctas;         // grid size
-  int S_max;        // most slabs any tile is spread over
-  int WM = 1;       // weight sub-tiles of 128 rows per tile
-  int w_tiled = 0;  // W is stored as contiguous 128 x 64 tiles, [N/128][K/64][128][64]
+  int S_max;        // split-K factor: slabs per output element
 };
-// 0 = auto; whole_tiles: never split a tile's k range (one slab, no reduction needed)
-GemmPlan plan_gemm_bf16(int M, int N, int K, int force_ctas = 0, int force_stages = 0, int force_bn = 0,
-                        bool whole_tiles = false, int force_wm = 0);
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split = 0, int force_stages = 0, int force_bn = 0);  // 0 = auto
 Partials make_partials(const float* p, int M, int N, const GemmPlan& plan);
 // Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,

@@ -73,8 +73,8 @@ SIGNATURES = {
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "dllm_gemm_bf16_scratch_bytes": (_SZ, [_I, _I, _I]),
     "dllm_gemm_bf16": (_I, [_P, _P, _P, _I, _I, _I, _P, _P]),
-    "dllm_gemm_bf16_planned_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I, _I]),
-    "dllm_gemm_bf16_planned": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
+    "dllm_gemm_bf16_planned_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I]),
+    "dllm_gemm_bf16_planned": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
     "dllm_gemm_simt": (_I, [_P, _P, _P, _I, _I, _I, _I, _P]),
     "dllm_attention_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I, _I, _I]),
     "dllm_attention": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
@@ -344,34 +344,20 @@ def gemm_bf16(A, W, stream=None):
     return Cm
 
 
-def tile_weight(W):
-    """[N, K] torch tensor -> the tiled layout [ceil(N/128)][ceil(K/64)][128][64], zero padded."""
-    import torch
-    N, K = W.shape
-    Np, Kp = (N + 127) // 128 * 128, (K + 63) // 64 * 64
-    Wp = torch.zeros((Np, Kp), dtype=W.dtype, device=W.device)
-    Wp[:N, :K] = W
-    return Wp.view(Np // 128, 128, Kp // 64, 64).permute(0, 2, 1, 3).contiguous()
-
-
-def gemm_bf16_planned(A, W, act_tile=0, ctas=0, stages=0, out=None, scratch=None, stream=None, reduce=True,
-                      w_tiled=None, N=None, w_sub=0):
+def gemm_bf16_planned(A, W, act_tile=0, splits=0, stages=0, out=None, scratch=None, stream=None, reduce=True):
     """gemm_bf16 with an explicit launch plan (tuning hook); `out` / `scratch` may be preallocated.
-    reduce=False leaves the slabs of shared tiles unreduced in `scratch` when the plan has any."""
+    reduce=False with a split plan leaves the split-K slabs unreduced in `scratch`."""
     import torch
     M, K = A.shape
-    if w_tiled is None:
-        w_tiled = W.dim() == 4
-    if N is None:
-        N = W.shape[0] * 128 if w_tiled else W.shape[0]
+    N = W.shape[0]
     Cm = out if out is not None else torch.empty((M, N), dtype=torch.float32, device=A.device)
-    sb = lib.dllm_gemm_bf16_planned_scratch_bytes(M, N, K, act_tile, w_sub, ctas)
+    sb = lib.dllm_gemm_bf16_planned_scratch_bytes(M, N, K, act_tile, splits)
     if scratch is None:
         scratch = torch.empty(max(sb, 16), dtype=torch.uint8, device=A.device)
     sp = _stream_ptr(stream if stream is not None else torch.cuda.current_stream(A.device))
     cptr = Cm.data_ptr() if (reduce or sb == 0) else None
     _check(lib.dllm_gemm_bf16_planned(C.c_void_p(A.data_ptr()), C.c_void_p(W.data_ptr()), C.c_void_p(cptr),
-                                      M, N, K, act_tile, w_sub, ctas, stages, int(bool(w_tiled)), C.c_void_p(scratch.data_ptr()),
+                                      M, N, K, act_tile, splits, stages, C.c_void_p(scratch.data_ptr()),
                                       scratch.numel(), C.c_void_p(sp)))
     return Cm
 

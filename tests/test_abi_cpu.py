@@ -99,7 +99,7 @@ def test_invalid_arguments_are_rejected_without_a_gpu(dllm):
         assert getattr(dllm.lib, fn)(*args) == dllm.INVALID_ARG
     assert dllm.lib.dllm_gemm_bf16(None, None, None, 1, 1, 8, None, None) == dllm.INVALID_ARG
     assert dllm.lib.dllm_gemm_bf16_scratch_bytes(64, 4096, 4096) > 0
-    assert dllm.lib.dllm_gemm_bf16_scratch_bytes(2048, 126464, 4096) == 0     # many tiles per SM: whole tiles, no slabs
+    assert dllm.lib.dllm_gemm_bf16_scratch_bytes(256, 126464, 4096) == 0      # enough tiles: no split
 
 
 def test_binding_has_no_fallback():

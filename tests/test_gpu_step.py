@@ -137,13 +137,17 @@ def test_tiny_fp32_stepwise_generation_with_graphs_off_and_on(env):
 
 # ---------------------------------------------------------------- bf16, several tiles and ragged tails
 @pytest.mark.parametrize("gqa", [False, True], ids=["mha", "gqa"])
-@pytest.mark.parametrize("simt", [True, False], ids=["simt_gemm", "tcgen05_gemm"])
-def test_small_bf16_step_kinds(env, gqa, simt):
+@pytest.mark.parametrize("path", ["simt_gemm", "tcgen05_gemm", "layer_kernel"])
+def test_small_bf16_step_kinds(env, gqa, path):
+    """Every step kind against the oracle, on the plain-ALU kernels, on the
+    tensor-core kernels launched one by one, and with the persistent layer
+    kernel (which takes the steps without prompt refresh)."""
     torch, dllm = env
     cfg = synth.small_bf16_model(gqa=gqa)
     B, P, R = 2, 150, 72
     orc, ses, _ = make_pair(dllm, cfg, B, P, R)
-    ses.use_simt_gemm(simt)
+    ses.use_simt_gemm(path == "simt_gemm")
+    ses.use_layer_kernel(path == "layer_kernel")
     r = orc.step(True, True)
     ses.step_full()
     compare_step(orc, ses, r, 2e-2, what="full")
