@@ -130,14 +130,32 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 // Sum of n_slabs partial results for eight consecutive columns, slab 0 first.
+// The loads of up to four slabs are issued together so that their latencies
+// overlap; the adds keep the slab order.
 __device__ __forceinline__ void sum_partials8(const float* part, size_t split_stride, int n_slabs, size_t off,
                                               float (&v)[8]) {
   Vec8<float>::load_cg(part + off, v);
-  for (int s = 1; s < n_slabs; ++s) {
-    float t[8];
-    Vec8<float>::load_cg(part + (size_t)s * split_stride + off, t);
+  int s = 1;
+  for (; s + 4 <= n_slabs; s += 4) {
+    float t[4][8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] += t[i];
+    for (int q = 0; q < 4; ++q) Vec8<float>::load_cg(part + (size_t)(s + q) * split_stride + off, t[q]);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] += t[q][i];
+  }
+  if (s < n_slabs) {  // up to three left: loaded together (index clamped, the surplus is not added)
+    float t[3][8];
+#pragma unroll
+    for (int q = 0; q < 3; ++q)
+      Vec8<float>::load_cg(part + (size_t)min(s + q, n_slabs - 1) * split_stride + off, t[q]);
+#pragma unroll
+    for (int q = 0; q < 3; ++q)
+      if (s + q < n_slabs) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] += t[q][i];
+      }
   }
 }
 

@@ -292,24 +292,41 @@ bool get_tensor_map_3d(const void* base, uint64_t batch, uint64_t rows, uint64_t
   return get_map(MapKey{base, batch, rows, cols, box_rows}, out);
 }
 
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      n = v;
+    else
+      return 148;  // no device visible (host-only size queries): a B200's count
+  }
+  return n;
+}
+
 Partials make_partials(const float* p, int M, int N, const GemmPlan& plan) {
   return Partials{p, (size_t)M * N, plan.S_max, N};  // every element has S_max slabs
 }
 
+// Tile shape, ring depth and split-K factor, from sweeps on B200: up to 256
+// activation rows the product is bound by streaming W, so k ranges are split
+// until at least one CTA per SM (two with 128-row tiles) streams weights.
 GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, int force_bn) {
   GemmPlan p;
-  p.BN = M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+  p.BN = M <= 32 ? 32 : M <= 64 ? 64 : M <= 256 ? 128 : 256;
   if (force_bn == 32 || force_bn == 64 || force_bn == 128 || force_bn == 256) p.BN = force_bn;
-  p.stages = force_stages > 0 ? force_stages : 4;
+  p.stages = force_stages > 0 ? force_stages : (p.BN == 128 ? 3 : 4);
   p.num_kb = (K + TILE_K - 1) / TILE_K;
   p.m_tiles = (M + p.BN - 1) / p.BN;
   const long tiles = (long)p.m_tiles * ((N + TILE_W - 1) / TILE_W);
-  int S = 1;
-  if (tiles < 148) {
-    S = (int)((148 + tiles - 1) / tiles);
-    const int max_s = p.num_kb / 4 > 1 ? p.num_kb / 4 : 1;
-    if (S > max_s) S = max_s;
-  }
+  const int sms = sm_count();
+  // every split adds a slab the consumer has to read: with few activation rows
+  // one wave of CTAs is enough, with 128-row tiles two CTAs per SM pay off
+  int S = p.BN == 128 ? (int)((2L * sms + tiles / 2) / tiles) : (int)((sms + tiles - 1) / tiles);
+  const int max_s = p.num_kb / 4 > 1 ? p.num_kb / 4 : 1;
+  if (S > max_s) S = max_s;
+  if (S < 1) S = 1;
   if (force_split > 0) S = force_split < p.num_kb ? force_split : p.num_kb;
   p.upc = (p.num_kb + S - 1) / S;                 // k-blocks per split
   p.S_max = (p.num_kb + p.upc - 1) / p.upc;       // no empty split
