@@ -146,7 +146,7 @@ Workspace make_workspace(const dllm_config& c, int B, int P, int R) {
   w.sel = take(T * BR * 4);
   w.forced = take(T * BR * 4);
   w.act = take(rows * 4);
-  w.inv = take(BR * 4);
+  w.inv = take(rows * 4);
   w.mkbar = take((1 + 13 * T) * 4);  // one grid-barrier counter per phase of the persistent layer kernel
   w.mkmaps = take((size_t)7 * T * sizeof(CUtensorMap));
   w.rope = take(n * c.head_dim * 4);
@@ -408,7 +408,7 @@ dllm_status enqueue_step_mk(dllm_session* s, int rr, int ksel, cudaStream_t stre
   cudaError_t e = launch_layer_megakernel(L, p);
   if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "persistent layer kernel: %s", cudaGetErrorString(e));
   // prediction at the response rows (Eqs. 3-4); u already holds the final norm
-  Partials part;
+  Partials part{nullptr, 0, 1, 0};
   dllm_status st = run_gemm(s, L, p.u, W + wl.lm_head, BR, c.vocab, d, &part);
   if (st != DLLM_OK) return st;
   if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
@@ -445,9 +445,11 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
   uint8_t* u = s->wsp<uint8_t>(s->ws.u);
   int32_t* act = s->wsp<int32_t>(s->ws.act);
   dllm_status st;
-  Partials part;
+  Partials part{nullptr, 0, 1, 0};
 
-  launch_embed(L, dt, W + wl.embed, s->wsp<int32_t>(s->ws.tokens), x, g, c0, c1);
+  int32_t* inv = s->wsp<int32_t>(s->ws.inv);
+  launch_embed_norm(L, dt, W + wl.embed, s->wsp<int32_t>(s->ws.tokens), x,
+                    reinterpret_cast<const float*>(W + wl.layers[0].norm1), u, g, c0, c1, c.rms_eps);
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerOff& lo = wl.layers[l];
     uint8_t* Wq = W + lo.wqkv;
@@ -456,7 +458,6 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
     int32_t* sel = s->wsp<int32_t>(s->ws.sel) + (size_t)l * BR;
     const int32_t* forced = s->wsp<int32_t>(s->ws.forced) + (size_t)l * BR;
 
-    launch_rmsnorm(L, dt, x, reinterpret_cast<const float*>(W + lo.norm1), u, d, c.rms_eps, c0, c1);
     if (project_v) {
       // V for ALL response rows (the 2 r d^2 term of Sec. A.7), V-verify, V overwrite
       if ((st = run_gemm(s, L, u, Wv, BR, dkv, d, &part)) != DLLM_OK) return st;
@@ -468,9 +469,13 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
     }
     if (Ma > 0) {
       const int mode = rr ? 0 : (s->forced_count[l] >= 0 ? 2 : 1);
-      launch_select(L, sim, forced, mode, ksel, sel, s->R, act, g, rp);
       uint8_t* ua = s->wsp<uint8_t>(s->ws.ua);
-      launch_gather_rows(L, dt, u, act, ua, Ma, d);
+      if (s->R <= 1024) {
+        launch_select_gather(L, dt, sim, forced, mode, ksel, sel, act, inv, u, ua, g, rp);
+      } else {
+        launch_select(L, sim, forced, mode, ksel, sel, s->R, act, inv, g, rp);
+        launch_gather_rows(L, dt, u, act, ua, Ma, d);
+      }
       // Q and K of the active rows in one GEMM over the stacked [W_q; W_k]
       if ((st = run_gemm(s, L, ua, Wq, Ma, dq + dkv, d, &part)) != DLLM_OK) return st;
       launch_qk_rope(L, dt, part, act, s->wsp<float>(s->ws.rope), s->wsp<uint8_t>(s->ws.qbuf),
@@ -488,12 +493,13 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.hn), W + lo.wgu, Ma, 2 * m, d, &part)) != DLLM_OK) return st;
       launch_silu_mul(L, dt, part, s->wsp<uint8_t>(s->ws.ffn), Ma, m);
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.ffn), W + lo.wd, Ma, d, m, &part)) != DLLM_OK) return st;
-      launch_scatter_rows(L, dt, part, act, 0, s->cache(l, DLLM_CACHE_FFN), g, Ma, d);
     }
-    launch_residual(L, dt, x, s->cache(l, DLLM_CACHE_ATTN), s->cache(l, DLLM_CACHE_FFN), g, c0, c1);
+    // FFNOut rows -> cache, residual assembly for all carried rows, next norm
+    const float* gain_next = reinterpret_cast<const float*>(l + 1 < c.n_layers ? W + wl.layers[l + 1].norm1 : W + wl.norm_f);
+    launch_tail(L, dt, part, Ma > 0 ? inv : nullptr, x, s->cache(l, DLLM_CACHE_ATTN), s->cache(l, DLLM_CACHE_FFN),
+                gain_next, u, g, c0, c1, c.rms_eps);
   }
-  // prediction at the response rows (Eqs. 3-4)
-  launch_rmsnorm(L, dt, x, reinterpret_cast<const float*>(W + wl.norm_f), u, d, c.rms_eps, 0, BR);
+  // prediction at the response rows (Eqs. 3-4); u holds the final norm
   if ((st = run_gemm(s, L, u, W + wl.lm_head, BR, c.vocab, d, &part)) != DLLM_OK) return st;
   if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
   launch_argmax_conf(L, part.p, BR, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf));
@@ -837,7 +843,7 @@ dllm_status dllm_get_logits(dllm_session* s, float* h_out, void* stream) {
   const int BR = s->B * s->R;
   launch_rmsnorm(L, c.dtype, s->wsp<float>(s->ws.x), reinterpret_cast<const float*>(s->m->d_w + s->m->lay.norm_f),
                  s->wsp<uint8_t>(s->ws.u), c.d_model, c.rms_eps, 0, BR);
-  Partials part;
+  Partials part{nullptr, 0, 1, 0};
   dllm_status r = run_gemm(s, L, s->wsp<uint8_t>(s->ws.u), s->m->d_w + s->m->lay.lm_head, BR, c.vocab, c.d_model, &part);
   if (r != DLLM_OK) return r;
   launch_mask_column(L, s->wsp<float>(s->ws.part), BR, c.vocab, c.mask_id);
@@ -1078,7 +1084,7 @@ dllm_status dllm_vverify_select(const void* d_vnew, void* d_vcache, float* d_sim
   if (width % 8 || R > 8192) return fail(nullptr, DLLM_UNSUPPORTED, "width must be a multiple of 8 and R <= 8192");
   Launch L{(cudaStream_t)stream, nullptr, nullptr};
   launch_vverify_rows(L, dtype, d_vnew, d_vcache, d_sim, B * R, width);
-  if (k > 0) launch_select(L, d_sim, nullptr, 1, k, d_idx, k, nullptr, Geo{B, 0, R, R, width}, 0);
+  if (k > 0) launch_select(L, d_sim, nullptr, 1, k, d_idx, k, nullptr, nullptr, Geo{B, 0, R, R, width}, 0);
   CU_TRY(nullptr, cudaGetLastError());
   return DLLM_OK;
 }

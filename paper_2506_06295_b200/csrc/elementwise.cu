@@ -115,7 +115,7 @@ __global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restr
 
 void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv) {
   const int rows = g.B * g.R;
-  DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(128), 0, part, (T*)Vc_layer, sim, g, dkv)));
+  DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(256), 0, part, (T*)Vc_layer, sim, g, dkv)));
   L.count();
 }
 
@@ -159,8 +159,8 @@ void launch_vverify_rows(const Launch& L, int dtype, const void* vnew, void* vca
 // the rank of a key among all R keys is its position in sorted order; a row is
 // selected iff rank < k.  R^2 comparisons out of shared memory: R <= 8192.
 __global__ void select_kernel(const float* __restrict__ sim, const int32_t* __restrict__ forced, int mode, int ksel,
-                              int32_t* __restrict__ sel, int sel_stride, int32_t* __restrict__ act, Geo g,
-                              int refresh_prompt) {
+                              int32_t* __restrict__ sel, int sel_stride, int32_t* __restrict__ act,
+                              int32_t* __restrict__ inv, Geo g, int refresh_prompt) {
   pdl_wait();
   pdl_trigger();
   extern __shared__ unsigned long long keys[];  // R keys, then R flags (as bytes)
@@ -170,21 +170,31 @@ __global__ void select_kernel(const float* __restrict__ sim, const int32_t* __re
   const int a_seq = (refresh_prompt ? g.P : 0) + ksel;
   int32_t* act_b = act ? act + (size_t)b * a_seq : nullptr;
   int32_t* sel_b = sel + (size_t)b * sel_stride;
+  const int np = refresh_prompt ? g.P : 0;
   if (refresh_prompt && act)
-    for (int i = threadIdx.x; i < g.P; i += blockDim.x) act_b[i] = g.B * R + b * g.P + i;
-  int32_t* act_r = act ? act_b + (refresh_prompt ? g.P : 0) : nullptr;
+    for (int i = threadIdx.x; i < g.P; i += blockDim.x) {
+      act_b[i] = g.B * R + b * g.P + i;
+      if (inv) inv[(size_t)g.B * R + (size_t)b * g.P + i] = b * a_seq + i;
+    }
+  int32_t* act_r = act ? act_b + np : nullptr;
   if (mode == 0) {
     for (int j = threadIdx.x; j < R; j += blockDim.x) {
       sel_b[j] = j;
       if (act_r) act_r[j] = b * R + j;
+      if (inv) inv[(size_t)b * R + j] = b * a_seq + np + j;
     }
     return;
   }
   if (mode == 2) {
+    if (inv) {
+      for (int j = threadIdx.x; j < R; j += blockDim.x) inv[(size_t)b * R + j] = -1;
+      __syncthreads();
+    }
     for (int r = threadIdx.x; r < ksel; r += blockDim.x) {
       const int j = forced[(size_t)b * R + r];
       sel_b[r] = j;
       if (act_r) act_r[r] = b * R + j;
+      if (inv) inv[(size_t)b * R + j] = b * a_seq + np + r;
     }
     return;
   }
@@ -205,18 +215,23 @@ __global__ void select_kernel(const float* __restrict__ sim, const int32_t* __re
   }
   __syncthreads();
   for (int j = threadIdx.x; j < R; j += blockDim.x) {
-    if (!flag[j]) continue;
+    if (!flag[j]) {
+      if (inv) inv[(size_t)b * R + j] = -1;
+      continue;
+    }
     int r = 0;
     for (int i = 0; i < j; ++i) r += flag[i];
     sel_b[r] = j;
     if (act_r) act_r[r] = b * R + j;
+    if (inv) inv[(size_t)b * R + j] = b * a_seq + np + r;
   }
 }
 
 void launch_select(const Launch& L, const float* sim, const int32_t* forced, int mode, int ksel, int32_t* sel,
-                   int sel_stride, int32_t* act, Geo g, int refresh_prompt) {
+                   int sel_stride, int32_t* act, int32_t* inv, Geo g, int refresh_prompt) {
   const size_t smem = (size_t)g.R * 9 + 16;
-  launch_k(L, select_kernel, dim3(g.B), dim3(256), smem, sim, forced, mode, ksel, sel, sel_stride, act, g, refresh_prompt);
+  launch_k(L, select_kernel, dim3(g.B), dim3(256), smem, sim, forced, mode, ksel, sel, sel_stride, act, inv, g,
+           refresh_prompt);
   L.count();
 }
 
@@ -411,6 +426,206 @@ void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer,
   if (c1 <= c0) return;
   DLLM_DISPATCH(dtype,
                 (launch_k(L, residual_kernel<T>, dim3(c1 - c0), dim3(128), 0, x, (const T*)Ac_layer, (const T*)Fc_layer, g, c0)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ embedding + first RMSNorm
+// x[c] = E[token(c)], u[c] = rmsnorm(x[c]) * gain for carried rows c0 <= c < c1.
+template <typename T>
+__global__ void embed_norm_kernel(const T* __restrict__ E, const int32_t* __restrict__ tokens, float* __restrict__ x,
+                                  const float* __restrict__ gain, T* __restrict__ u, Geo g, int c0, float eps) {
+  pdl_wait();
+  pdl_trigger();
+  __shared__ float red[32];
+  const int c = c0 + blockIdx.x;
+  int b, pos;
+  carried_to_pos(c, g, b, pos);
+  const int tok = tokens[(size_t)b * g.n + pos];
+  const T* src = E + (size_t)tok * g.d;
+  float* xr = x + (size_t)c * g.d;
+  float ss = 0.f;
+  for (int i = threadIdx.x * 8; i < g.d; i += blockDim.x * 8) {
+    float v[8];
+    Vec8<T>::load(src + i, v);
+    Vec8<float>::store(xr + i, v);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) ss += v[j] * v[j];
+  }
+  ss = block_sum(ss, red);
+  const float r = rsqrtf(ss / (float)g.d + eps);
+  T* orow = u + (size_t)c * g.d;
+  for (int i = threadIdx.x * 8; i < g.d; i += blockDim.x * 8) {
+    float v[8], gv[8];
+    Vec8<T>::load(src + i, v);
+    Vec8<float>::load(gain + i, gv);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = v[j] * r * gv[j];
+    Vec8<T>::store(orow + i, v);
+  }
+}
+
+void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, const float* gain,
+                       void* u, Geo g, int c0, int c1, float eps) {
+  if (c1 <= c0) return;
+  DLLM_DISPATCH(dtype, (launch_k(L, embed_norm_kernel<T>, dim3(c1 - c0), dim3(256), 0, (const T*)E, tokens, x, gain,
+                                 (T*)u, g, c0, eps)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ layer tail
+// For every carried row: the FFNOut row of an active row (inv[c] >= 0: its
+// position in the active list, whose slabs `part` holds) goes to the cache,
+// rounded to the cache dtype; x <- (x + AttnOut) + FFNOut from the caches
+// (Sec. 3.2 item (3)); u = rmsnorm(x) * gain, the next layer's first norm (the
+// final norm after the last layer).  inv == nullptr: no row is active.
+template <typename T>
+__global__ void tail_kernel(Partials part, const int32_t* __restrict__ inv, float* __restrict__ x,
+                            const T* __restrict__ Ac, T* __restrict__ Fc, const float* __restrict__ gain,
+                            T* __restrict__ u, Geo g, int c0, float eps) {
+  pdl_wait();
+  pdl_trigger();
+  extern __shared__ float hrow[];
+  __shared__ float red[32];
+  const int c = c0 + blockIdx.x;
+  int b, pos;
+  carried_to_pos(c, g, b, pos);
+  const int d = g.d;
+  const size_t crow = ((size_t)b * g.n + pos) * d;
+  const int r = inv ? inv[c] : -1;
+  float* xr = x + (size_t)c * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
+    float xv[8], a[8], f[8];
+    Vec8<float>::load(xr + i, xv);
+    Vec8<T>::load(Ac + crow + i, a);
+    if (r >= 0) {
+      sum_partials8(part.p, part.split_stride, part.count(r, i), (size_t)r * part.N + i, f);
+      Vec8<T>::store(Fc + crow + i, f);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) f[t] = Vec8<T>::round(f[t]);
+    } else {
+      Vec8<T>::load(Fc + crow + i, f);
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      xv[t] = (xv[t] + a[t]) + f[t];
+      ss += xv[t] * xv[t];
+    }
+    Vec8<float>::store(xr + i, xv);
+    Vec8<float>::store(hrow + i, xv);
+  }
+  ss = block_sum(ss, red);
+  const float rs = rsqrtf(ss / (float)d + eps);
+  T* orow = u + (size_t)c * d;
+  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
+    float v[8], gv[8];
+    Vec8<float>::load(hrow + i, v);
+    Vec8<float>::load(gain + i, gv);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) v[t] = v[t] * rs * gv[t];
+    Vec8<T>::store(orow + i, v);
+  }
+}
+
+void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, const void* Ac_layer,
+                 void* Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps) {
+  if (c1 <= c0) return;
+  const size_t smem = (size_t)g.d * sizeof(float);
+  DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T>, dim3(c1 - c0), dim3(256), smem, part, inv, x, (const T*)Ac_layer,
+                                 (T*)Fc_layer, gain, (T*)u, g, c0, eps)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ selection + gather in one launch
+// grid (a_seq, B): CTA (i, b) produces row i of sequence b's active list and
+// copies that row of u into ua.  Rows below the prompt length (on a prompt
+// refresh) are the prompt rows; the others are the selected response rows, for
+// which every CTA repeats the bottom-k selection of its sequence (R <= 1024,
+// R^2 comparisons out of shared memory) instead of waiting for another launch.
+// CTA (0, b) writes the index list, the active list and its inverse.
+template <typename T>
+__global__ void select_gather_kernel(const float* __restrict__ sim, const int32_t* __restrict__ forced, int mode,
+                                     int ksel, int32_t* __restrict__ sel, int32_t* __restrict__ act,
+                                     int32_t* __restrict__ inv, const T* __restrict__ u, T* __restrict__ ua, Geo g,
+                                     int refresh_prompt) {
+  pdl_wait();
+  pdl_trigger();
+  extern __shared__ unsigned long long keys[];  // R keys, R slots (int), R flags (bytes)
+  const int R = g.R, b = blockIdx.y, ridx = blockIdx.x;
+  int32_t* slot = reinterpret_cast<int32_t*>(keys + R);
+  unsigned char* flag = reinterpret_cast<unsigned char*>(slot + R);
+  __shared__ int my_j;
+  const int np = refresh_prompt ? g.P : 0;
+  const int a_seq = np + ksel;
+  const bool leader = ridx == 0;
+  if (ridx >= np || leader) {
+    if (mode == 0) {
+      for (int j = threadIdx.x; j < R; j += blockDim.x) slot[j] = j;
+    } else if (mode == 2) {
+      for (int j = threadIdx.x; j < R; j += blockDim.x) slot[j] = -1;
+      __syncthreads();
+      for (int r = threadIdx.x; r < ksel; r += blockDim.x) slot[forced[(size_t)b * R + r]] = r;
+    } else {
+      for (int j = threadIdx.x; j < R; j += blockDim.x) {
+        const float s = sim[(size_t)b * R + j];
+        // s in [-1, 1] up to rounding; NaN (degenerate input) sorts first
+        const float qf = rintf(s * 1048576.0f);
+        const long long q = (s == s) ? (long long)qf + (1ll << 22) : 0ll;
+        keys[j] = ((unsigned long long)q << 32) | (unsigned)j;
+      }
+      __syncthreads();
+      for (int j = threadIdx.x; j < R; j += blockDim.x) {
+        const unsigned long long kj = keys[j];
+        int rank = 0;
+        for (int i = 0; i < R; ++i) rank += (keys[i] < kj);
+        flag[j] = (rank < ksel);
+      }
+      __syncthreads();
+      for (int j = threadIdx.x; j < R; j += blockDim.x) {
+        int r = -1;
+        if (flag[j]) {
+          r = 0;
+          for (int i = 0; i < j; ++i) r += flag[i];
+        }
+        slot[j] = r;
+      }
+    }
+    __syncthreads();
+    // slot[j]: position of response row j among the selected rows, or -1
+    if (ridx >= np)
+      for (int j = threadIdx.x; j < R; j += blockDim.x)
+        if (slot[j] == ridx - np) my_j = j;
+    if (leader) {
+      for (int j = threadIdx.x; j < R; j += blockDim.x) {
+        const int r = slot[j];
+        inv[(size_t)b * R + j] = r >= 0 ? b * a_seq + np + r : -1;
+        if (r >= 0) {
+          sel[(size_t)b * R + r] = j;
+          act[(size_t)b * a_seq + np + r] = b * R + j;
+        }
+      }
+      for (int i = threadIdx.x; i < np; i += blockDim.x) {
+        act[(size_t)b * a_seq + i] = g.B * R + b * g.P + i;
+        inv[(size_t)g.B * R + (size_t)b * g.P + i] = b * a_seq + i;
+      }
+    }
+    __syncthreads();
+  }
+  const int c = ridx < np ? g.B * R + b * g.P + ridx : b * R + my_j;
+  const uint4* s4 = reinterpret_cast<const uint4*>(u + (size_t)c * g.d);
+  uint4* o4 = reinterpret_cast<uint4*>(ua + ((size_t)b * a_seq + ridx) * g.d);
+  const int nvec = g.d * (int)sizeof(T) / 16;
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) o4[i] = s4[i];
+}
+
+void launch_select_gather(const Launch& L, int dtype, const float* sim, const int32_t* forced, int mode, int ksel,
+                          int32_t* sel, int32_t* act, int32_t* inv, const void* u, void* ua, Geo g,
+                          int refresh_prompt) {
+  const int a_seq = (refresh_prompt ? g.P : 0) + ksel;
+  if (a_seq <= 0) return;
+  const size_t smem = (size_t)g.R * 13 + 16;
+  DLLM_DISPATCH(dtype, (launch_k(L, select_gather_kernel<T>, dim3(a_seq, g.B), dim3(256), smem, sim, forced, mode, ksel,
+                                 sel, act, inv, (const T*)u, (T*)ua, g, refresh_prompt)));
   L.count();
 }
 

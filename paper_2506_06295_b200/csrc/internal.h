@@ -75,8 +75,22 @@ void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gai
 void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv);
 // Bottom-k selection per sequence + active-row list.  mode 0: all R rows,
 // 1: bottom-k by (round(sim*2^20), index), 2: forced list.
+// inv (may be null): for every carried row its position in the active list, or -1.
 void launch_select(const Launch& L, const float* sim, const int32_t* forced, int mode, int ksel, int32_t* sel,
-                   int sel_stride, int32_t* act, Geo g, int refresh_prompt);
+                   int sel_stride, int32_t* act, int32_t* inv, Geo g, int refresh_prompt);
+// Selection, active list, inverse list and the gather of the active rows of u
+// into ua in one launch (R <= 1024; sel rows have stride R).
+void launch_select_gather(const Launch& L, int dtype, const float* sim, const int32_t* forced, int mode, int ksel,
+                          int32_t* sel, int32_t* act, int32_t* inv, const void* u, void* ua, Geo g,
+                          int refresh_prompt);
+// x[c] = E[token(c)], u[c] = rmsnorm(x[c]) * gain for carried rows c0 <= c < c1.
+void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, const float* gain,
+                       void* u, Geo g, int c0, int c1, float eps);
+// End of a layer for carried rows c0 <= c < c1: FFNOut rows of the active set
+// (slabs in `part`, row = inv[c]) -> cache; x <- (x + AttnOut) + FFNOut from the
+// caches; u = rmsnorm(x) * gain.  inv == nullptr: no active row.
+void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, const void* Ac_layer,
+                 void* Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps);
 void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32_t* act, void* dst, int rows, int d);
 // RoPE on Q and K of the active rows; Q -> qbuf [Ma, dq]; K -> K cache rows.
 void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* act, const float* rope_tab, void* qbuf,
