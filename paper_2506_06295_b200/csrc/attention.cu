@@ -147,21 +147,59 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ C
   if (!ok && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
 }
 
-// Merges the key-range splits: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.
-__global__ void attn_combine_kernel(const float* __restrict__ o_part, const float* __restrict__ ml_part,
-                                    __nv_bfloat16* __restrict__ o, size_t total, int S, int hd) {
+// Merges the key-range splits: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s,
+// splits in index order.  One warp per (row, head); the (max, sum) pairs of all
+// splits are fetched together, then the partial outputs.
+template <int MAXS>
+__device__ __forceinline__ void combine_row(const float* __restrict__ o_part, const float* __restrict__ ml_part,
+                                            __nv_bfloat16* __restrict__ o, size_t total, size_t rh, int S, int hd,
+                                            int lane) {
+  float2 ml[MAXS];
+  float wgt[MAXS];
+#pragma unroll
+  for (int s = 0; s < MAXS; ++s)
+    ml[s] = *reinterpret_cast<const float2*>(ml_part + ((size_t)min(s, S - 1) * total + rh) * 2);
+  float M = -INFINITY, L = 0.f;
+#pragma unroll
+  for (int s = 0; s < MAXS; ++s)
+    if (s < S) M = fmaxf(M, ml[s].x);
+#pragma unroll
+  for (int s = 0; s < MAXS; ++s) {
+    wgt[s] = s < S ? exp2f(ml[s].x - M) : 0.f;
+    if (s < S) L += wgt[s] * ml[s].y;
+  }
+  const float inv = 1.f / L;
+  for (int d = lane; d < hd; d += 32) {
+    float v[MAXS];
+#pragma unroll
+    for (int s = 0; s < MAXS; ++s) v[s] = o_part[((size_t)min(s, S - 1) * total + rh) * hd + d];
+    float acc = 0.f;
+#pragma unroll
+    for (int s = 0; s < MAXS; ++s)
+      if (s < S) acc += wgt[s] * v[s];
+    o[rh * hd + d] = __float2bfloat16_rn(acc * inv);
+  }
+}
+
+__global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restrict__ o_part,
+                                                           const float* __restrict__ ml_part,
+                                                           __nv_bfloat16* __restrict__ o, size_t total, int S, int hd) {
   pdl_wait();
   pdl_trigger();
-  const size_t rh = blockIdx.x;
-  float M = -INFINITY;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const size_t rh = (size_t)blockIdx.x * 8 + warp;
+  if (rh >= total) return;
+  if (S <= 4) return combine_row<4>(o_part, ml_part, o, total, rh, S, hd, lane);
+  if (S <= 8) return combine_row<8>(o_part, ml_part, o, total, rh, S, hd, lane);
+  if (S <= 16) return combine_row<16>(o_part, ml_part, o, total, rh, S, hd, lane);
+  float M = -INFINITY, L = 0.f;
   for (int s = 0; s < S; ++s) M = fmaxf(M, ml_part[((size_t)s * total + rh) * 2]);
-  float L = 0.f;
   for (int s = 0; s < S; ++s) {
     const float* ml = ml_part + ((size_t)s * total + rh) * 2;
     L += exp2f(ml[0] - M) * ml[1];
   }
   const float inv = 1.f / L;
-  for (int d = threadIdx.x; d < hd; d += blockDim.x) {
+  for (int d = lane; d < hd; d += 32) {
     float acc = 0.f;
     for (int s = 0; s < S; ++s)
       acc += exp2f(ml_part[((size_t)s * total + rh) * 2] - M) * o_part[((size_t)s * total + rh) * hd + d];
@@ -190,7 +228,7 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
                                                      L.d_status);
   L.count();
   if (S > 1) {
-    launch_k(L, attn_combine_kernel, dim3((unsigned)total), dim3(HD / 2), 0, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
+    launch_k(L, attn_combine_kernel, dim3((unsigned)((total + 7) / 8)), dim3(256), 0, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
     L.count();
   }
   return cudaGetLastError();

@@ -255,40 +255,78 @@ void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32
 }
 
 // ------------------------------------------------------------------ RoPE + K scatter
-// grid (Ma, H + Hkv): one block per (active row, head).  Rotate-half pairing:
+// One thread per (active row, head, four rotation pairs).  Rotate-half pairing:
 // element i with i + hd/2, angle pos * theta^(-2i/hd) from a table built on the host.
 template <typename T>
+__device__ __forceinline__ void store4(T* p, const float (&v)[4]);
+template <>
+__device__ __forceinline__ void store4<float>(float* p, const float (&v)[4]) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+template <>
+__device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, const float (&v)[4]) {
+  const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+}
+// Sum of the slabs of four consecutive columns, slab 0 first; up to four loads in flight.
+__device__ __forceinline__ void sum_partials4(const Partials& part, int row, int col, float (&v)[4]) {
+  const int n = part.count(row, col);
+  const float* base = part.p + (size_t)row * part.N + col;
+  v[0] = v[1] = v[2] = v[3] = 0.f;
+  for (int s = 0; s < n; s += 4) {
+    float4 t[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      t[q] = __ldcg(reinterpret_cast<const float4*>(base + (size_t)min(s + q, n - 1) * part.split_stride));
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (s + q < n) {
+        v[0] += t[q].x; v[1] += t[q].y; v[2] += t[q].z; v[3] += t[q].w;
+      }
+  }
+}
+
+template <typename T>
 __global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ rope_tab,
-                               T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int H, int Hkv, int hd) {
+                               T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int Ma, int H, int Hkv, int hd) {
   pdl_wait();
   pdl_trigger();
-  const int r = blockIdx.x, head = blockIdx.y;
+  const int half = hd >> 1, q4 = half >> 2;
+  const int groups = (H + Hkv) * q4;
+  const long w = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (w >= (long)Ma * groups) return;
+  const int r = (int)(w / groups), gidx = (int)(w - (long)r * groups);
+  const int head = gidx / q4, i0 = (gidx - head * q4) * 4;
   int b, pos;
   carried_to_pos(act[r], g, b, pos);
-  const int half = hd >> 1;
   const int dq = H * hd, dkv = Hkv * hd;
   const bool is_q = head < H;
   const int col0 = is_q ? head * hd : dq + (head - H) * hd;
   T* dst = is_q ? qbuf + (size_t)r * dq + head * hd : Kc + ((size_t)b * g.n + pos) * dkv + (head - H) * hd;
   const float* tab = rope_tab + (size_t)pos * hd;  // [cos(half) | sin(half)]
-  for (int i = threadIdx.x; i < half; i += blockDim.x) {
-    float lo = 0.f, hi = 0.f;
-    const int n_lo = part.count(r, col0 + i), n_hi = part.count(r, col0 + i + half);
-    const float* p = part.p + (size_t)r * part.N + col0;
-    for (int s = 0; s < n_lo; ++s) lo += p[(size_t)s * part.split_stride + i];
-    for (int s = 0; s < n_hi; ++s) hi += p[(size_t)s * part.split_stride + i + half];
-    const float c = tab[i], sn = tab[half + i];
-    dst[i] = from_f32<T>(lo * c - hi * sn);
-    dst[i + half] = from_f32<T>(hi * c + lo * sn);
+  float lo[4], hi[4];
+  sum_partials4(part, r, col0 + i0, lo);
+  sum_partials4(part, r, col0 + i0 + half, hi);
+  const float4 cs = *reinterpret_cast<const float4*>(tab + i0);
+  const float4 sn = *reinterpret_cast<const float4*>(tab + half + i0);
+  const float cc[4] = {cs.x, cs.y, cs.z, cs.w}, ss[4] = {sn.x, sn.y, sn.z, sn.w};
+  float o_lo[4], o_hi[4];
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    o_lo[t] = lo[t] * cc[t] - hi[t] * ss[t];
+    o_hi[t] = hi[t] * cc[t] + lo[t] * ss[t];
   }
+  store4<T>(dst + i0, o_lo);
+  store4<T>(dst + i0 + half, o_hi);
 }
 
 void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* act, const float* rope_tab, void* qbuf,
                     void* Kc_layer, Geo g, int Ma, int H, int Hkv, int hd) {
   if (Ma <= 0) return;
-  dim3 grid(Ma, H + Hkv);
-  DLLM_DISPATCH(dtype, (launch_k(L, qk_rope_kernel<T>, dim3(grid), dim3(64), 0, part, act, rope_tab, (T*)qbuf, (T*)Kc_layer, g, H,
-                                                                     Hkv, hd)));
+  const long total = (long)Ma * (H + Hkv) * (hd >> 3);
+  const unsigned blocks = (unsigned)((total + 255) / 256);
+  DLLM_DISPATCH(dtype, (launch_k(L, qk_rope_kernel<T>, dim3(blocks), dim3(256), 0, part, act, rope_tab, (T*)qbuf,
+                                 (T*)Kc_layer, g, Ma, H, Hkv, hd)));
   L.count();
 }
 
@@ -646,6 +684,16 @@ __device__ __forceinline__ MaxSum merge(MaxSum p, MaxSum q) {
   return p;
 }
 
+__device__ __forceinline__ void online_add(MaxSum& t, float v, int i) {
+  if (v > t.m) {
+    t.s = t.s * expf(t.m - v) + 1.f;
+    t.m = v;
+    t.a = i;
+  } else {
+    t.s += expf(v - t.m);
+  }
+}
+
 __global__ void argmax_conf_kernel(const float* __restrict__ logits, int vocab, int mask_id, int32_t* __restrict__ x0,
                                    float* __restrict__ conf) {
   pdl_wait();
@@ -654,17 +702,27 @@ __global__ void argmax_conf_kernel(const float* __restrict__ logits, int vocab, 
   const size_t row = blockIdx.x;
   const float* lr = logits + row * vocab;
   MaxSum t{-INFINITY, 0.f, 0x7fffffff};
-  for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
-    if (i == mask_id) continue;
-    const float v = lr[i];
-    if (v > t.m) {
-      t.s = t.s * expf(t.m - v) + 1.f;
-      t.m = v;
-      t.a = i;
-    } else {
-      t.s += expf(v - t.m);
+  // 16 floats per thread and trip (four 16-byte loads in flight); rows are 16-byte aligned when vocab % 4 == 0
+  const int v16 = ((vocab & 3) == 0) ? vocab / 16 * 16 : 0;
+  for (int i0 = threadIdx.x * 4; i0 < v16; i0 += blockDim.x * 16) {
+    float4 q[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = i0 + k * blockDim.x * 4;
+      q[k] = i < v16 ? *reinterpret_cast<const float4*>(lr + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int i = i0 + k * blockDim.x * 4;
+      if (i >= v16) continue;
+      const float e[4] = {q[k].x, q[k].y, q[k].z, q[k].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (i + j != mask_id) online_add(t, e[j], i + j);
     }
   }
+  for (int i = v16 + threadIdx.x; i < vocab; i += blockDim.x)
+    if (i != mask_id) online_add(t, lr[i], i);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     MaxSum q;
