@@ -323,7 +323,7 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
   const int sms = sm_count();
   // every split adds a slab the consumer has to read: with few activation rows
   // one wave of CTAs is enough, with 128-row tiles two CTAs per SM pay off
-  int S = p.BN == 128 ? (int)((2L * sms + tiles / 2) / tiles) : (int)((sms + tiles - 1) / tiles);
+  int S = p.BN == 128 ? (int)(2L * sms / tiles) : (int)((sms + tiles - 1) / tiles);  // all CTAs resident at once
   const int max_s = p.num_kb / 4 > 1 ? p.num_kb / 4 : 1;
   if (S > max_s) S = max_s;
   if (S < 1) S = 1;
