@@ -440,7 +440,8 @@ def main():
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch from the ncu capture summarised under
-# profiles/ (average over the captured launches, scaled where stated there); None until captured.
+# profiles/ncu_gemm_bf16_tcgen05_partial_step_2layers.md: 451 MB per layer of an adaptive partial step over 5
+# launches, plus the LM head's 1,036 MB once per step scaled in by its bytes (32 layers: 15.47 GB / 161 launches).
 TRAFFIC_PER_LAUNCH = {"llada8b": 96.1e6}
 
 if __name__ == "__main__":
