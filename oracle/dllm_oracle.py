@@ -98,6 +98,14 @@ def cosine_rows(a: np.ndarray, b: np.ndarray) -> np.ndarray:
     return (dot / np.maximum(den, COS_EPS)).astype(np.float32)
 
 
+def l2_score_rows(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    """The alternative metric of Sec. A.6: Euclidean distance between the new and
+    the cached vector of a token.  Returned NEGATED (as float32) so that, as with
+    the cosine, the least similar tokens have the lowest score."""
+    diff = a - b
+    return (-np.sqrt(np.sum(diff * diff, axis=-1))).astype(np.float32)
+
+
 def k_selected(rho: float, R: int, kround: str = "floor") -> int:
     """Number of response tokens updated in an adaptive step: floor(rho * L)
     (Sec. 3.2.2).  'ceil' is the alternative wording of the benchmark statement."""
@@ -211,11 +219,26 @@ class DLLMOracle:
 
     # -- one denoising step --------------------------------------------------
     def step(self, refresh_prompt: bool, refresh_response: bool, rho: float = 0.0,
-             kround: str = "floor", forced: dict | None = None) -> StepResult:
+             kround: str = "floor", forced: dict | None = None, strategy: str = "v_verify",
+             metric: str = "cosine", v_update: str = "all", scores=None) -> StepResult:
         """One forward pass under the caching rule.  (True, True) is the
         initialisation / full refresh.  `forced[(layer)] = int array [B, k]`
         replaces the V-verify choice of that layer (used to separate legal tie
-        flips from arithmetic differences in parity tests)."""
+        flips from arithmetic differences in parity tests).
+
+        The paper's ablations of the adaptive step (Sec. 4.3, Sec. A.5, Sec. A.6):
+          strategy  "v_verify" (default, Eq. 6 on V), "k_verify" (the same test on
+                    the post-RoPE K; read symmetrically: K of ALL response rows is
+                    projected and overwritten, V only at the selected rows), or
+                    "random" (no projection over all rows: the lowest of the given
+                    `scores` [T, B, R] are taken, V only at the selected rows);
+          metric    "cosine" (default) or "l2" (Sec. A.6);
+          v_update  "all" (default: whole V_r overwritten) or "selected" (Sec. A.5:
+                    only the selected tokens' V)."""
+        if strategy not in ("v_verify", "k_verify", "random") or metric not in ("cosine", "l2") \
+                or v_update not in ("all", "selected"):
+            raise ValueError("unknown selection variant")
+        score_rows = cosine_rows if metric == "cosine" else l2_score_rows
         c, B, P, R, n = self.cfg, self.B, self.P, self.R, self.n
         if not self.valid and not (refresh_prompt and refresh_response):
             raise RuntimeError("cached step before any full step")
@@ -241,19 +264,32 @@ class DLLMOracle:
                 u[carried] = rmsnorm(x[carried], self.w[p + "norm1"].astype(self.dt), c.rms_eps)
                 # b-d. which response rows are recomputed
                 have_v = np.zeros(n, bool)
-                v_rows = np.zeros((n, Vc.shape[1]), self.dt)
                 if refresh_response:
                     S = np.arange(R)
                 elif ksel == 0:
                     S = np.zeros(0, np.int64)            # fully cached: nothing projected
-                else:
+                elif strategy == "v_verify":
                     v_new = self._lin(u[P:], p + "wv", "proj")          # all R rows
-                    s = cosine_rows(v_new, Vc[P:])                         # Eq. 6
+                    s = score_rows(v_new, Vc[P:])                          # Eq. 6 (or Sec. A.6)
                     res.sim[l][b] = s
                     S = select_lowest(s, ksel)
-                    Vc[P:] = v_new                                          # whole V_r overwritten
-                    v_rows[P:] = v_new
-                    have_v[P:] = True
+                    if v_update == "all":
+                        Vc[P:] = v_new                                      # whole V_r overwritten
+                        have_v[P:] = True
+                    else:                                                   # Sec. A.5 variant
+                        Vc[P + S] = v_new[S]
+                        have_v[P + S] = True
+                elif strategy == "k_verify":
+                    k_new = self._lin(u[P:], p + "wk", "proj").reshape(-1, Hkv, hd)
+                    k_new = rope(k_new, np.arange(P, n), c.rope_theta).reshape(R, Hkv * hd)
+                    s = score_rows(k_new, Kc[P:])                          # the test of Eq. 6 on K
+                    res.sim[l][b] = s
+                    S = select_lowest(s, ksel)
+                    Kc[P:] = k_new                                          # whole K_r overwritten
+                else:                                                       # random selection
+                    s = np.asarray(scores[l][b], dtype=np.float32)
+                    res.sim[l][b] = s
+                    S = select_lowest(s, ksel)
                 if forced is not None and l in forced and not refresh_response and ksel > 0:
                     S = np.sort(np.asarray(forced[l])[b].astype(np.int64))
                 res.selected[l][b, :len(S)] = S
