@@ -170,6 +170,23 @@ dllm_status dllm_set_cache(dllm_session* s, int layer, int which, const float* h
  * steps that follow); count = -1 clears.  V-verify still runs and V is still
  * overwritten.  Lets a test tell a legal tie flip from an arithmetic fault. */
 dllm_status dllm_force_selection(dllm_session* s, int layer, const int32_t* h_idx, int count);
+/* The paper's ablations of the adaptive step (Sec. 4.3 selection strategies,
+ * Sec. A.6 metric, Sec. A.5 V update).  Defaults: V-verify, cosine, whole-V
+ * overwrite.
+ *   strategy DLLM_SELECT_K_VERIFY: the test of Eq. 6 on the post-RoPE K; K of all
+ *     response rows is projected and overwritten, V only at the selected rows.
+ *   strategy DLLM_SELECT_RANDOM: no projection over all rows; the k_sel lowest of
+ *     the scores given with dllm_set_scores are taken (same tie rule), V only at
+ *     the selected rows.
+ *   metric DLLM_METRIC_L2: score = -||new - cached||_2 instead of the cosine.
+ *   v_selected_only != 0 (V-verify): only the selected tokens' V is written.
+ * Response-refresh and full steps are unaffected. */
+typedef enum { DLLM_SELECT_V_VERIFY = 0, DLLM_SELECT_K_VERIFY = 1, DLLM_SELECT_RANDOM = 2 } dllm_select_strategy;
+typedef enum { DLLM_METRIC_COSINE = 0, DLLM_METRIC_L2 = 1 } dllm_metric;
+dllm_status dllm_session_set_selection(dllm_session* s, int strategy, int metric, int v_selected_only);
+/* Scores of one layer for DLLM_SELECT_RANDOM: host float [B, R]; they stay in
+ * place until set again (any other strategy overwrites them with its own). */
+dllm_status dllm_set_scores(dllm_session* s, int layer, const float* h_scores, void* stream);
 /* Number of kernel launches the library has enqueued for this session. */
 uint64_t dllm_launch_count(const dllm_session* s);
 /* 1: replay each step kind from a CUDA graph captured on first use (default);

@@ -179,7 +179,9 @@ struct dllm_model {
 struct StepKey {
   int rp, rr, ksel;
   uint64_t forced_sig;
+  int variant = 0;
   bool operator<(const StepKey& o) const {
+    if (variant != o.variant) return variant < o.variant;
     if (rp != o.rp) return rp < o.rp;
     if (rr != o.rr) return rr < o.rr;
     if (ksel != o.ksel) return ksel < o.ksel;
@@ -201,6 +203,7 @@ struct dllm_session {
   bool use_graphs = true;
   bool simt_gemm = false;
   bool use_pdl = true;
+  int sel_strategy = DLLM_SELECT_V_VERIFY, sel_metric = DLLM_METRIC_COSINE, v_selected_only = 0;  // ablation variants
   bool use_mk = false;         // persistent layer kernel for the step kinds it covers (opt-in)
   bool mk_maps_ready = false;  // weight / cache tensor maps uploaded to the workspace
   struct GraphEntry {
@@ -420,6 +423,7 @@ dllm_status enqueue_step_mk(dllm_session* s, int rr, int ksel, cudaStream_t stre
 
 bool step_uses_mk(const dllm_session* s, int rp, int ksel) {
   const dllm_config& c = s->m->cfg;
+  if (s->sel_strategy != DLLM_SELECT_V_VERIFY || s->sel_metric != DLLM_METRIC_COSINE || s->v_selected_only) return false;
   return s->use_mk && !s->profiling && !s->simt_gemm &&
          mk_supported(c.dtype, s->B, s->P, s->R, c.d_model, c.n_heads, c.n_kv_heads, c.head_dim, c.d_ffn, c.n_layers, rp,
                       ksel);
@@ -440,7 +444,6 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
   const int c0 = 0, c1 = BR + (rp ? BP : 0);
   const int a_seq = (rp ? s->P : 0) + ksel;
   const int Ma = s->B * a_seq;
-  const bool project_v = rr || ksel > 0;
   float* x = s->wsp<float>(s->ws.x);
   uint8_t* u = s->wsp<uint8_t>(s->ws.u);
   int32_t* act = s->wsp<int32_t>(s->ws.act);
@@ -458,11 +461,20 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
     int32_t* sel = s->wsp<int32_t>(s->ws.sel) + (size_t)l * BR;
     const int32_t* forced = s->wsp<int32_t>(s->ws.forced) + (size_t)l * BR;
 
-    if (project_v) {
+    const bool adaptive = !rr && ksel > 0;
+    if (rr || (adaptive && s->sel_strategy == DLLM_SELECT_V_VERIFY)) {
       // V for ALL response rows (the 2 r d^2 term of Sec. A.7), V-verify, V overwrite
       if ((st = run_gemm(s, L, u, Wv, BR, dkv, d, &part)) != DLLM_OK) return st;
-      launch_vverify(L, dt, part, s->cache(l, DLLM_CACHE_V), sim, g, dkv);
-    }
+      launch_vverify(L, dt, part, s->cache(l, DLLM_CACHE_V), sim, g, dkv, rr ? 0 : s->sel_metric,
+                     rr || !s->v_selected_only);
+    } else if (adaptive && s->sel_strategy == DLLM_SELECT_K_VERIFY) {
+      // ablation: the same test on K; K of ALL response rows is projected, rotated and overwritten
+      if ((st = run_gemm(s, L, u, Wq + (size_t)dq * d * es, BR, dkv, d, &part)) != DLLM_OK) return st;
+      launch_kverify(L, dt, part, s->cache(l, DLLM_CACHE_K), sim, s->wsp<float>(s->ws.rope), g, Hkv, hd,
+                     s->sel_metric);
+    }  // random selection: the scores were set by dllm_set_scores
+    // V of the active rows is still missing when the verify pass did not write it
+    const bool v_for_active = adaptive && (s->sel_strategy != DLLM_SELECT_V_VERIFY || s->v_selected_only);
     if (rp) {
       if ((st = run_gemm(s, L, u + (size_t)BR * d * es, Wv, BP, dkv, d, &part)) != DLLM_OK) return st;
       launch_scatter_rows(L, dt, part, nullptr, BR, s->cache(l, DLLM_CACHE_V), g, BP, dkv);
@@ -475,6 +487,10 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
       } else {
         launch_select(L, sim, forced, mode, ksel, sel, s->R, act, inv, g, rp);
         launch_gather_rows(L, dt, u, act, ua, Ma, d);
+      }
+      if (v_for_active) {
+        if ((st = run_gemm(s, L, ua, Wv, Ma, dkv, d, &part)) != DLLM_OK) return st;
+        launch_scatter_rows(L, dt, part, act, 0, s->cache(l, DLLM_CACHE_V), g, Ma, dkv);
       }
       // Q and K of the active rows in one GEMM over the stacked [W_q; W_k]
       if ((st = run_gemm(s, L, ua, Wq, Ma, dq + dkv, d, &part)) != DLLM_OK) return st;
@@ -535,7 +551,7 @@ dllm_status run_step(dllm_session* s, int rp, int rr, float rho, dllm_kround kr,
   } else if (!graph_ok) {
     st = enqueue_step(s, rp, rr, ksel, stream);
   } else {
-    StepKey key{rp, rr, ksel, forced_signature(s)};
+    StepKey key{rp, rr, ksel, forced_signature(s), s->sel_strategy * 4 + s->sel_metric * 2 + s->v_selected_only};
     auto it = s->graphs.find(key);
     if (it == s->graphs.end()) {
       cudaGraph_t graph = nullptr;
@@ -943,6 +959,27 @@ dllm_status dllm_session_use_pdl(dllm_session* s, int enable) {
     s->graphs.clear();
   }
   s->use_pdl = enable != 0;
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_set_selection(dllm_session* s, int strategy, int metric, int v_selected_only) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (strategy < DLLM_SELECT_V_VERIFY || strategy > DLLM_SELECT_RANDOM || (metric != DLLM_METRIC_COSINE && metric != DLLM_METRIC_L2))
+    return fail(&s->err, DLLM_INVALID_ARG, "unknown selection strategy or metric");
+  s->sel_strategy = strategy;
+  s->sel_metric = metric;
+  s->v_selected_only = v_selected_only != 0;
+  return DLLM_OK;
+}
+
+dllm_status dllm_set_scores(dllm_session* s, int layer, const float* h_scores, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (!h_scores) return fail(&s->err, DLLM_INVALID_ARG, "h_scores is NULL");
+  if (layer < 0 || layer >= s->m->cfg.n_layers) return fail(&s->err, DLLM_INVALID_ARG, "layer out of range");
+  const size_t BR = (size_t)s->B * s->R;
+  cudaStream_t st = (cudaStream_t)stream;
+  CU_TRY(&s->err, cudaStreamSynchronize(st));
+  CU_TRY(&s->err, h2d(s->d_ws + s->ws.sim + (size_t)layer * BR * 4, h_scores, BR * 4, st));
   return DLLM_OK;
 }
 

@@ -23,6 +23,36 @@ namespace dllm {
     }                                             \
   } while (0)
 
+// ------------------------------------------------------------------ four-wide helpers
+template <typename T>
+__device__ __forceinline__ void store4(T* p, const float (&v)[4]);
+template <>
+__device__ __forceinline__ void store4<float>(float* p, const float (&v)[4]) {
+  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+template <>
+__device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, const float (&v)[4]) {
+  const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
+}
+// Sum of the slabs of four consecutive columns, slab 0 first; up to four loads in flight.
+__device__ __forceinline__ void sum_partials4(const Partials& part, int row, int col, float (&v)[4]) {
+  const int n = part.count(row, col);
+  const float* base = part.p + (size_t)row * part.N + col;
+  v[0] = v[1] = v[2] = v[3] = 0.f;
+  for (int s = 0; s < n; s += 4) {
+    float4 t[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      t[q] = __ldcg(reinterpret_cast<const float4*>(base + (size_t)min(s + q, n - 1) * part.split_stride));
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (s + q < n) {
+        v[0] += t[q].x; v[1] += t[q].y; v[2] += t[q].z; v[3] += t[q].w;
+      }
+  }
+}
+
 // ------------------------------------------------------------------ embed
 template <typename T>
 __global__ void embed_kernel(const T* __restrict__ E, const int32_t* __restrict__ tokens, float* __restrict__ x, Geo g,
@@ -85,8 +115,12 @@ void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gai
 }
 
 // ------------------------------------------------------------------ V-verify (Eq. 6) + V overwrite
+// metric 0: cosine (Eq. 6); 1: negated Euclidean distance (Sec. A.6), so that the
+// least similar rows have the lowest score either way.  write_v 0: the cache is
+// left as it is (the selected-only variant of Sec. A.5 writes the selected rows later).
 template <typename T>
-__global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restrict__ sim, Geo g, int dkv) {
+__global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restrict__ sim, Geo g, int dkv, int metric,
+                               int write_v) {
   pdl_wait();
   pdl_trigger();
   __shared__ float red[32];
@@ -101,21 +135,91 @@ __global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restr
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
       vn[t] = Vec8<T>::round(vn[t]);  // compare what the cache will hold
-      dot += vn[t] * vo[t];
-      na += vn[t] * vn[t];
-      nb += vo[t] * vo[t];
+      if (metric == 0) {
+        dot += vn[t] * vo[t];
+        na += vn[t] * vn[t];
+        nb += vo[t] * vo[t];
+      } else {
+        const float df = vn[t] - vo[t];
+        dot += df * df;
+      }
     }
-    Vec8<T>::store(vrow + i, vn);
+    if (write_v) Vec8<T>::store(vrow + i, vn);
   }
   dot = block_sum(dot, red);
-  na = block_sum(na, red);
-  nb = block_sum(nb, red);
-  if (threadIdx.x == 0) sim[c] = dot / fmaxf(sqrtf(na * nb), 1e-8f);
+  if (metric == 0) {
+    na = block_sum(na, red);
+    nb = block_sum(nb, red);
+  }
+  if (threadIdx.x == 0) sim[c] = metric == 0 ? dot / fmaxf(sqrtf(na * nb), 1e-8f) : -sqrtf(dot);
 }
 
-void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv) {
+void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv, int metric,
+                    int write_v) {
   const int rows = g.B * g.R;
-  DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(256), 0, part, (T*)Vc_layer, sim, g, dkv)));
+  DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(256), 0, part, (T*)Vc_layer, sim, g, dkv,
+                                 metric, write_v)));
+  L.count();
+}
+
+// ------------------------------------------------------------------ K-verify: the same test on the post-RoPE K
+// One block per response row: slab sum of the K projection, RoPE at the row's
+// position, rounding to the cache dtype, score against the cached K row, and
+// the whole-K overwrite (the symmetric reading of the K-verify ablation, Sec. 4.3).
+template <typename T>
+__global__ void kverify_kernel(Partials part, T* __restrict__ Kc, float* __restrict__ sim,
+                               const float* __restrict__ rope_tab, Geo g, int Hkv, int hd, int metric) {
+  pdl_wait();
+  pdl_trigger();
+  __shared__ float red[32];
+  const int c = blockIdx.x;
+  const int b = c / g.R, j = c - b * g.R, pos = g.P + j;
+  const int half = hd >> 1, q4 = half >> 2, dkv = Hkv * hd;
+  T* krow = Kc + ((size_t)b * g.n + pos) * dkv;
+  const float* tab = rope_tab + (size_t)pos * hd;
+  float dot = 0.f, na = 0.f, nb = 0.f;
+  for (int gidx = threadIdx.x; gidx < Hkv * q4; gidx += blockDim.x) {
+    const int head = gidx / q4, i0 = (gidx - head * q4) * 4, col0 = head * hd;
+    float lo[4], hi[4], o_lo[4], o_hi[4], c_lo[4], c_hi[4];
+    sum_partials4(part, c, col0 + i0, lo);
+    sum_partials4(part, c, col0 + i0 + half, hi);
+    const float4 cs = *reinterpret_cast<const float4*>(tab + i0);
+    const float4 sn = *reinterpret_cast<const float4*>(tab + half + i0);
+    const float cc[4] = {cs.x, cs.y, cs.z, cs.w}, ss[4] = {sn.x, sn.y, sn.z, sn.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      o_lo[t] = Vec8<T>::round(lo[t] * cc[t] - hi[t] * ss[t]);
+      o_hi[t] = Vec8<T>::round(hi[t] * cc[t] + lo[t] * ss[t]);
+      c_lo[t] = to_f32<T>(krow[col0 + i0 + t]);
+      c_hi[t] = to_f32<T>(krow[col0 + i0 + half + t]);
+    }
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      if (metric == 0) {
+        dot += o_lo[t] * c_lo[t] + o_hi[t] * c_hi[t];
+        na += o_lo[t] * o_lo[t] + o_hi[t] * o_hi[t];
+        nb += c_lo[t] * c_lo[t] + c_hi[t] * c_hi[t];
+      } else {
+        const float d0 = o_lo[t] - c_lo[t], d1 = o_hi[t] - c_hi[t];
+        dot += d0 * d0 + d1 * d1;
+      }
+    }
+    store4<T>(krow + col0 + i0, o_lo);
+    store4<T>(krow + col0 + i0 + half, o_hi);
+  }
+  dot = block_sum(dot, red);
+  if (metric == 0) {
+    na = block_sum(na, red);
+    nb = block_sum(nb, red);
+  }
+  if (threadIdx.x == 0) sim[c] = metric == 0 ? dot / fmaxf(sqrtf(na * nb), 1e-8f) : -sqrtf(dot);
+}
+
+void launch_kverify(const Launch& L, int dtype, Partials part, void* Kc_layer, float* sim, const float* rope_tab, Geo g,
+                    int Hkv, int hd, int metric) {
+  const int rows = g.B * g.R;
+  DLLM_DISPATCH(dtype, (launch_k(L, kverify_kernel<T>, dim3(rows), dim3(256), 0, part, (T*)Kc_layer, sim, rope_tab, g,
+                                 Hkv, hd, metric)));
   L.count();
 }
 
@@ -200,9 +304,9 @@ __global__ void select_kernel(const float* __restrict__ sim, const int32_t* __re
   }
   for (int j = threadIdx.x; j < R; j += blockDim.x) {
     const float s = sim[(size_t)b * R + j];
-    // s in [-1, 1] up to rounding; NaN (degenerate input) sorts first
-    const float qf = rintf(s * 1048576.0f);
-    const long long q = (s == s) ? (long long)qf + (1ll << 22) : 0ll;
+    // key = round(s * 2^20), offset into 1 .. 2^32 - 1 (scores beyond +-2047 saturate); NaN sorts first
+    const float qf = fminf(fmaxf(rintf(s * 1048576.0f), -2147483520.0f), 2147483520.0f);
+    const long long q = (s == s) ? (long long)qf + (1ll << 31) : 0ll;
     keys[j] = ((unsigned long long)q << 32) | (unsigned)j;
     flag[j] = 0;
   }
@@ -257,35 +361,6 @@ void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32
 // ------------------------------------------------------------------ RoPE + K scatter
 // One thread per (active row, head, four rotation pairs).  Rotate-half pairing:
 // element i with i + hd/2, angle pos * theta^(-2i/hd) from a table built on the host.
-template <typename T>
-__device__ __forceinline__ void store4(T* p, const float (&v)[4]);
-template <>
-__device__ __forceinline__ void store4<float>(float* p, const float (&v)[4]) {
-  *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
-}
-template <>
-__device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, const float (&v)[4]) {
-  const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
-  *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const uint32_t*>(&a), *reinterpret_cast<const uint32_t*>(&b));
-}
-// Sum of the slabs of four consecutive columns, slab 0 first; up to four loads in flight.
-__device__ __forceinline__ void sum_partials4(const Partials& part, int row, int col, float (&v)[4]) {
-  const int n = part.count(row, col);
-  const float* base = part.p + (size_t)row * part.N + col;
-  v[0] = v[1] = v[2] = v[3] = 0.f;
-  for (int s = 0; s < n; s += 4) {
-    float4 t[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-      t[q] = __ldcg(reinterpret_cast<const float4*>(base + (size_t)min(s + q, n - 1) * part.split_stride));
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-      if (s + q < n) {
-        v[0] += t[q].x; v[1] += t[q].y; v[2] += t[q].z; v[3] += t[q].w;
-      }
-  }
-}
-
 template <typename T>
 __global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ rope_tab,
                                T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int Ma, int H, int Hkv, int hd) {
@@ -606,9 +681,9 @@ __global__ void select_gather_kernel(const float* __restrict__ sim, const int32_
     } else {
       for (int j = threadIdx.x; j < R; j += blockDim.x) {
         const float s = sim[(size_t)b * R + j];
-        // s in [-1, 1] up to rounding; NaN (degenerate input) sorts first
-        const float qf = rintf(s * 1048576.0f);
-        const long long q = (s == s) ? (long long)qf + (1ll << 22) : 0ll;
+        // key = round(s * 2^20), offset into 1 .. 2^32 - 1 (scores beyond +-2047 saturate); NaN sorts first
+        const float qf = fminf(fmaxf(rintf(s * 1048576.0f), -2147483520.0f), 2147483520.0f);
+        const long long q = (s == s) ? (long long)qf + (1ll << 31) : 0ll;
         keys[j] = ((unsigned long long)q << 32) | (unsigned)j;
       }
       __syncthreads();

@@ -72,7 +72,12 @@ void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gai
 // V-verify (Eq. 6) fused with the whole-V overwrite: for every response row
 // sums the partials, rounds to the cache dtype, takes the cosine against the
 // cached row, overwrites the cached row, writes sim[row].
-void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv);
+void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv,
+                    int metric = 0, int write_v = 1);
+// The same test on K (ablation of Sec. 4.3): slab sum of the K projection of all
+// response rows, RoPE, score against the cached (post-RoPE) K, whole-K overwrite.
+void launch_kverify(const Launch& L, int dtype, Partials part, void* Kc_layer, float* sim, const float* rope_tab, Geo g,
+                    int Hkv, int hd, int metric);
 // Bottom-k selection per sequence + active-row list.  mode 0: all R rows,
 // 1: bottom-k by (round(sim*2^20), index), 2: forced list.
 // inv (may be null): for every carried row its position in the active list, or -1.

@@ -427,9 +427,9 @@ __device__ void phase_select(const Ctx& c, int l, uint8_t* scratch) {
     } else {
       for (int j = c.tid; j < R; j += MK_WORKERS) {
         const float s = __ldcg(sim + (size_t)b * R + j);
-        // s in [-1, 1] up to rounding; NaN (degenerate input) sorts first
-        const float qf = rintf(s * 1048576.0f);
-        const long long q = (s == s) ? (long long)qf + (1ll << 22) : 0ll;
+        // key = round(s * 2^20), offset into 1 .. 2^32 - 1 (scores beyond +-2047 saturate); NaN sorts first
+        const float qf = fminf(fmaxf(rintf(s * 1048576.0f), -2147483520.0f), 2147483520.0f);
+        const long long q = (s == s) ? (long long)qf + (1ll << 31) : 0ll;
         keys[j] = ((unsigned long long)q << 32) | (unsigned)j;
       }
       wk_sync();

@@ -63,6 +63,8 @@ SIGNATURES = {
     "dllm_get_cache": (_I, [_P, _I, _I, _P, _P]),
     "dllm_set_cache": (_I, [_P, _I, _I, _P, _P]),
     "dllm_force_selection": (_I, [_P, _I, _P, _I]),
+    "dllm_session_set_selection": (_I, [_P, _I, _I, _I]),
+    "dllm_set_scores": (_I, [_P, _I, _P, _P]),
     "dllm_launch_count": (C.c_uint64, [_P]),
     "dllm_session_use_graphs": (_I, [_P, _I]),
     "dllm_session_use_simt_gemm": (_I, [_P, _I]),
@@ -293,6 +295,16 @@ class Session:
             return
         a = np.ascontiguousarray(idx, dtype=np.int32).reshape(self.B, -1)
         _check(lib.dllm_force_selection(self.handle, layer, _np_ptr(a), a.shape[1]))
+
+    def set_selection(self, strategy: str = "v_verify", metric: str = "cosine", v_update: str = "all") -> None:
+        """Ablation variants of the adaptive step (Sec. 4.3, Sec. A.5, Sec. A.6)."""
+        st = {"v_verify": 0, "k_verify": 1, "random": 2}[strategy]
+        me = {"cosine": 0, "l2": 1}[metric]
+        _check(lib.dllm_session_set_selection(self.handle, st, me, int(v_update == "selected")))
+
+    def set_scores(self, layer: int, scores: np.ndarray) -> None:
+        a = np.ascontiguousarray(scores, dtype=np.float32).reshape(self.B, self.R)
+        _check(lib.dllm_set_scores(self.handle, layer, _np_ptr(a), self.sp))
 
     def launch_count(self) -> int:
         return int(lib.dllm_launch_count(self.handle))

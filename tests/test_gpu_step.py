@@ -51,7 +51,7 @@ def unmask(orc, ses, step, count):
     ses.set_response_tokens(resp)
 
 
-def compare_step(orc, ses, r, tol, check_sets=True, what=""):
+def compare_step(orc, ses, r, tol, check_sets=True, what="", sim_atol=None):
     ses.sync()
     hid = ses.hidden()
     err = rel_l2(hid, r.hidden)
@@ -64,7 +64,7 @@ def compare_step(orc, ses, r, tol, check_sets=True, what=""):
                 assert selection_matches(idx[b], r.selected[l][b], None if r.sim[l] is None else r.sim[l][b]), \
                     f"{what}: layer {l} seq {b}: {idx[b].tolist()} vs {r.selected[l][b].tolist()}"
         if r.sim[l] is not None:
-            np.testing.assert_allclose(sim, r.sim[l], atol=5e-3 if tol > 1e-3 else 2e-5)
+            np.testing.assert_allclose(sim, r.sim[l], atol=sim_atol or (5e-3 if tol > 1e-3 else 2e-5))
     return err
 
 
