@@ -125,6 +125,12 @@ dllm_status dllm_step_full(dllm_session* s, void* stream);
  * Returns DLLM_BAD_STATE before the first full step. */
 dllm_status dllm_step_cached(dllm_session* s, int refresh_prompt, int refresh_response, float rho,
                              dllm_kround kround, void* stream);
+/* dllm_step_cached with one update ratio PER LAYER (the cross-layer allocation of
+ * Sec. A.4, Table 11: e.g. 0.375 -> 0.125 front-heavy): h_rho host float
+ * [n_layers], n_layers must equal the model's.  Layer l recomputes
+ * floor(rho_l * R) rows; a layer with 0 rows is fully cached. */
+dllm_status dllm_step_cached_layers(dllm_session* s, int refresh_prompt, int refresh_response, const float* h_rho,
+                                    int n_layers, dllm_kround kround, void* stream);
 /* Applies the schedule at step k of K (counting down): refresh everything at
  * k = K, the prompt when k mod Kp == 0, the response when k mod Kr == 0. */
 dllm_status dllm_step_scheduled(dllm_session* s, int k, int K, int Kp, int Kr, float rho,

@@ -243,11 +243,15 @@ class DLLMOracle:
         if not self.valid and not (refresh_prompt and refresh_response):
             raise RuntimeError("cached step before any full step")
         H, Hkv, hd, d = c.n_heads, c.n_kv_heads, c.head_dim, c.d_model
-        ksel = R if refresh_response else k_selected(rho, R, kround)
+        # rho may be one ratio or one per layer (the cross-layer allocation of Sec. A.4, Table 11)
+        rhos = [float(rho)] * c.n_layers if np.ndim(rho) == 0 else [float(r) for r in rho]
+        if len(rhos) != c.n_layers:
+            raise ValueError("one rho per layer expected")
+        ksels = [R if refresh_response else k_selected(r, R, kround) for r in rhos]
         res = StepResult(hidden=np.zeros((B, R, d), self.dt), logits=None, x0=None, conf=None)
-        res.selected = [np.zeros((B, ksel), np.int32) for _ in range(c.n_layers)]
-        verify = (not refresh_response) and ksel > 0
-        res.sim = [np.zeros((B, R), np.float32) if verify else None for _ in range(c.n_layers)]
+        res.selected = [np.zeros((B, ksels[l]), np.int32) for l in range(c.n_layers)]
+        res.sim = [np.zeros((B, R), np.float32) if (not refresh_response and ksels[l] > 0) else None
+                   for l in range(c.n_layers)]
         logits = np.zeros((B, R, c.vocab), self.dt)
 
         for b in range(B):
@@ -258,6 +262,7 @@ class DLLMOracle:
             x[carried] = E[self.tokens[b, carried]].astype(self.dt)
             for l in range(c.n_layers):
                 p = f"layers.{l}."
+                ksel = ksels[l]
                 Kc, Vc, Ac, Fc = self.Kc[l][b], self.Vc[l][b], self.Ac[l][b], self.Fc[l][b]
                 # a. pre-attention norm of the carried rows
                 u = np.zeros((n, d), self.dt)

@@ -180,8 +180,10 @@ struct StepKey {
   int rp, rr, ksel;
   uint64_t forced_sig;
   int variant = 0;
+  uint64_t ksel_sig = 0;  // per-layer row counts (cross-layer allocation of rho)
   bool operator<(const StepKey& o) const {
     if (variant != o.variant) return variant < o.variant;
+    if (ksel_sig != o.ksel_sig) return ksel_sig < o.ksel_sig;
     if (rp != o.rp) return rp < o.rp;
     if (rr != o.rr) return rr < o.rr;
     if (ksel != o.ksel) return ksel < o.ksel;
@@ -197,7 +199,7 @@ struct dllm_session {
   Workspace ws;
   bool valid = false;      // caches hold a full step
   bool have_pred = false;
-  int last_ksel = 0;
+  std::vector<int> last_ksel;  // per layer
   std::vector<int> forced_count;  // per layer, -1 = none
   uint64_t launches = 0;
   bool use_graphs = true;
@@ -432,7 +434,7 @@ bool step_uses_mk(const dllm_session* s, int rp, int ksel) {
 // Enqueue one denoising step.  Active rows per sequence: the prompt rows on a
 // prompt refresh plus either all R response rows (response refresh) or the
 // ksel rows V-verify picks.
-dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t stream) {
+dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>& ksels, cudaStream_t stream) {
   const dllm_config& c = s->m->cfg;
   const WeightLayout& wl = s->m->lay;
   const Geo g = s->geo();
@@ -442,8 +444,6 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
   Launch L{stream, s->wsp<int>(s->ws.status), &s->launches, s->use_pdl && !s->profiling};
   uint8_t* W = s->m->d_w;
   const int c0 = 0, c1 = BR + (rp ? BP : 0);
-  const int a_seq = (rp ? s->P : 0) + ksel;
-  const int Ma = s->B * a_seq;
   float* x = s->wsp<float>(s->ws.x);
   uint8_t* u = s->wsp<uint8_t>(s->ws.u);
   int32_t* act = s->wsp<int32_t>(s->ws.act);
@@ -461,6 +461,9 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, int ksel, cudaStream_t
     int32_t* sel = s->wsp<int32_t>(s->ws.sel) + (size_t)l * BR;
     const int32_t* forced = s->wsp<int32_t>(s->ws.forced) + (size_t)l * BR;
 
+    const int ksel = ksels[l];  // rows of the response this layer recomputes
+    const int a_seq = (rp ? s->P : 0) + ksel;
+    const int Ma = s->B * a_seq;
     const bool adaptive = !rr && ksel > 0;
     if (rr || (adaptive && s->sel_strategy == DLLM_SELECT_V_VERIFY)) {
       // V for ALL response rows (the 2 r d^2 term of Sec. A.7), V-verify, V overwrite
@@ -530,34 +533,45 @@ uint64_t forced_signature(const dllm_session* s) {
   return h;
 }
 
-dllm_status run_step(dllm_session* s, int rp, int rr, float rho, dllm_kround kr, void* stream_v) {
+dllm_status run_step(dllm_session* s, int rp, int rr, const float* rhos, int n_rho, dllm_kround kr, void* stream_v) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
-  if (!(rho >= 0.f && rho <= 1.f)) return fail(&s->err, DLLM_INVALID_ARG, "rho must lie in [0, 1]");
+  const int T = s->m->cfg.n_layers;
+  if (!rhos || (n_rho != 1 && n_rho != T)) return fail(&s->err, DLLM_INVALID_ARG, "one rho, or one per layer");
+  for (int i = 0; i < n_rho; ++i)
+    if (!(rhos[i] >= 0.f && rhos[i] <= 1.f)) return fail(&s->err, DLLM_INVALID_ARG, "rho must lie in [0, 1]");
   if (kr != DLLM_K_FLOOR && kr != DLLM_K_CEIL) return fail(&s->err, DLLM_INVALID_ARG, "bad kround");
   rp = rp != 0;
   rr = rr != 0;
   if (!s->valid && !(rp && rr)) return fail(&s->err, DLLM_BAD_STATE, "cached step before any full step");
-  const int ksel = rr ? s->R : k_selected(rho, s->R, kr);
+  std::vector<int> ksels(T);
+  bool uniform = true;
+  uint64_t sig = 1469598103934665603ull;
+  for (int l = 0; l < T; ++l) {
+    ksels[l] = rr ? s->R : k_selected(rhos[n_rho == 1 ? 0 : l], s->R, kr);
+    uniform = uniform && ksels[l] == ksels[0];
+    sig = (sig ^ (uint64_t)ksels[l]) * 1099511628211ull;
+  }
   if (!rr)
-    for (int l = 0; l < s->m->cfg.n_layers; ++l)
-      if (s->forced_count[l] >= 0 && s->forced_count[l] != ksel)
+    for (int l = 0; l < T; ++l)
+      if (s->forced_count[l] >= 0 && s->forced_count[l] != ksels[l])
         return fail(&s->err, DLLM_INVALID_ARG, "forced selection of layer %d has %d rows, step selects %d", l,
-                    s->forced_count[l], ksel);
+                    s->forced_count[l], ksels[l]);
   cudaStream_t stream = (cudaStream_t)stream_v;
   dllm_status st = DLLM_OK;
   const bool graph_ok = s->use_graphs && !s->profiling && stream != nullptr && stream != cudaStreamLegacy;
-  if (step_uses_mk(s, rp, ksel)) {
-    st = enqueue_step_mk(s, rr, ksel, stream);  // a handful of launches: no graph needed
+  if (uniform && step_uses_mk(s, rp, ksels[0])) {
+    st = enqueue_step_mk(s, rr, ksels[0], stream);  // a handful of launches: no graph needed
   } else if (!graph_ok) {
-    st = enqueue_step(s, rp, rr, ksel, stream);
+    st = enqueue_step(s, rp, rr, ksels, stream);
   } else {
-    StepKey key{rp, rr, ksel, forced_signature(s), s->sel_strategy * 4 + s->sel_metric * 2 + s->v_selected_only};
+    StepKey key{rp, rr, ksels[0], forced_signature(s), s->sel_strategy * 4 + s->sel_metric * 2 + s->v_selected_only,
+                uniform ? 0 : sig};
     auto it = s->graphs.find(key);
     if (it == s->graphs.end()) {
       cudaGraph_t graph = nullptr;
       CU_TRY(&s->err, cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal));
       const uint64_t before = s->launches;
-      st = enqueue_step(s, rp, rr, ksel, stream);
+      st = enqueue_step(s, rp, rr, ksels, stream);
       cudaError_t e = cudaStreamEndCapture(stream, &graph);
       if (st != DLLM_OK) {
         if (graph) cudaGraphDestroy(graph);
@@ -578,7 +592,7 @@ dllm_status run_step(dllm_session* s, int rp, int rr, float rho, dllm_kround kr,
   if (st != DLLM_OK) return st;
   s->valid = true;
   s->have_pred = true;
-  s->last_ksel = ksel;
+  s->last_ksel = ksels;
   return DLLM_OK;
 }
 
@@ -746,11 +760,21 @@ dllm_status dllm_session_set_prompt(dllm_session* s, const int32_t* h_prompt, vo
   return DLLM_OK;
 }
 
-dllm_status dllm_step_full(dllm_session* s, void* stream) { return run_step(s, 1, 1, 0.f, DLLM_K_FLOOR, stream); }
+dllm_status dllm_step_full(dllm_session* s, void* stream) {
+  const float rho = 0.f;
+  return run_step(s, 1, 1, &rho, 1, DLLM_K_FLOOR, stream);
+}
 
 dllm_status dllm_step_cached(dllm_session* s, int refresh_prompt, int refresh_response, float rho, dllm_kround kround,
                              void* stream) {
-  return run_step(s, refresh_prompt, refresh_response, rho, kround, stream);
+  return run_step(s, refresh_prompt, refresh_response, &rho, 1, kround, stream);
+}
+
+dllm_status dllm_step_cached_layers(dllm_session* s, int refresh_prompt, int refresh_response, const float* h_rho,
+                                    int n_layers, dllm_kround kround, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (n_layers != s->m->cfg.n_layers) return fail(&s->err, DLLM_INVALID_ARG, "one rho per layer expected");
+  return run_step(s, refresh_prompt, refresh_response, h_rho, n_layers, kround, stream);
 }
 
 dllm_status dllm_step_scheduled(dllm_session* s, int k, int K, int Kp, int Kr, float rho, dllm_kround kround,
@@ -759,7 +783,7 @@ dllm_status dllm_step_scheduled(dllm_session* s, int k, int K, int Kp, int Kr, f
   if (K <= 0 || k <= 0 || k > K || Kp <= 0 || Kr <= 0)
     return fail(&s->err, DLLM_INVALID_ARG, "need 1 <= k <= K and positive K_p, K_r");
   const int rp = (k == K) || (k % Kp == 0), rr = (k == K) || (k % Kr == 0);
-  return run_step(s, rp, rr, rho, kround, stream);
+  return run_step(s, rp, rr, &rho, 1, kround, stream);
 }
 
 dllm_status dllm_remask_low_confidence(dllm_session* s, int block_start, int block_len, int n_transfer, void* stream) {
@@ -874,10 +898,11 @@ dllm_status dllm_get_selected(dllm_session* s, int layer, int32_t* h_idx, float*
   if (!s->have_pred) return fail(&s->err, DLLM_BAD_STATE, "no step has run");
   CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
   const size_t BR = (size_t)s->B * s->R;
-  if (k_sel_out) *k_sel_out = s->last_ksel;
-  if (h_idx && s->last_ksel > 0)
-    CU_TRY(&s->err, cudaMemcpy2D(h_idx, (size_t)s->last_ksel * 4, s->d_ws + s->ws.sel + (size_t)layer * BR * 4,
-                                 (size_t)s->R * 4, (size_t)s->last_ksel * 4, s->B, cudaMemcpyDeviceToHost));
+  const int k_l = layer < (int)s->last_ksel.size() ? s->last_ksel[layer] : 0;
+  if (k_sel_out) *k_sel_out = k_l;
+  if (h_idx && k_l > 0)
+    CU_TRY(&s->err, cudaMemcpy2D(h_idx, (size_t)k_l * 4, s->d_ws + s->ws.sel + (size_t)layer * BR * 4,
+                                 (size_t)s->R * 4, (size_t)k_l * 4, s->B, cudaMemcpyDeviceToHost));
   if (h_sim)
     CU_TRY(&s->err, cudaMemcpy(h_sim, s->d_ws + s->ws.sim + (size_t)layer * BR * 4, BR * 4, cudaMemcpyDeviceToHost));
   return DLLM_OK;

@@ -50,6 +50,7 @@ SIGNATURES = {
     "dllm_session_set_prompt": (_I, [_P, _P, _P]),
     "dllm_step_full": (_I, [_P, _P]),
     "dllm_step_cached": (_I, [_P, _I, _I, _F, _I, _P]),
+    "dllm_step_cached_layers": (_I, [_P, _I, _I, _P, _I, _I, _P]),
     "dllm_step_scheduled": (_I, [_P, _I, _I, _I, _I, _F, _I, _P]),
     "dllm_remask_low_confidence": (_I, [_P, _I, _I, _I, _P]),
     "dllm_generate": (_I, [_P, _I, _I, _I, _F, _I, _I, _P]),
@@ -231,6 +232,12 @@ class Session:
 
     def step_cached(self, refresh_prompt: bool, refresh_response: bool, rho: float, kround: int = K_FLOOR) -> None:
         _check(lib.dllm_step_cached(self.handle, int(refresh_prompt), int(refresh_response), rho, kround, self.sp))
+
+    def step_cached_layers(self, refresh_prompt: bool, refresh_response: bool, rhos, kround: int = K_FLOOR) -> None:
+        """step_cached with one update ratio per layer (Sec. A.4, Table 11)."""
+        a = np.ascontiguousarray(rhos, dtype=np.float32)
+        _check(lib.dllm_step_cached_layers(self.handle, int(refresh_prompt), int(refresh_response), _np_ptr(a),
+                                           int(a.size), kround, self.sp))
 
     def step_scheduled(self, k: int, K: int, Kp: int, Kr: int, rho: float, kround: int = K_FLOOR) -> None:
         _check(lib.dllm_step_scheduled(self.handle, k, K, Kp, Kr, rho, kround, self.sp))

@@ -63,3 +63,31 @@ def test_selection_arguments_are_checked(env):
     assert dllm.lib.dllm_session_set_selection(ses.handle, 3, 0, 0) == dllm.INVALID_ARG
     assert dllm.lib.dllm_session_set_selection(ses.handle, 0, 2, 0) == dllm.INVALID_ARG
     assert dllm.lib.dllm_set_scores(ses.handle, 99, None, None) == dllm.INVALID_ARG
+
+
+@pytest.mark.parametrize("mode", ["fp32", "bf16"])
+def test_per_layer_update_ratio_matches_the_oracle(env, mode):
+    """Cross-layer allocation of rho (Sec. A.4, Table 11): front-heavy, back-heavy, a fully cached layer."""
+    torch, dllm = env
+    if mode == "fp32":
+        cfg, B, P, R, tol = synth.TINY, 1, 64, 32, 1e-4
+    else:
+        cfg, B, P, R, tol = synth.small_bf16_model(), 2, 150, 72, 2e-2
+    orc, ses, _ = make_pair(dllm, cfg, B, P, R)
+    r = orc.step(True, True)
+    ses.step_full()
+    compare_step(orc, ses, r, tol, what="full")
+    step = 0
+    for rp, rr, rhos in ((False, False, [0.375, 0.125]), (False, False, [0.125, 0.375]), (True, False, [0.5, 0.0]),
+                         (False, False, [0.0, 0.25]), (False, True, [0.1, 0.9])):
+        step += 1
+        unmask(orc, ses, step, 3)
+        r = orc.step(rp, rr, rhos)
+        ses.step_cached_layers(rp, rr, rhos)
+        ses.sync()
+        for l in range(cfg.n_layers):
+            assert ses.selected(l)[0].shape == r.selected[l].shape
+        compare_step(orc, ses, r, tol, what=f"step {step} ({rp},{rr},{rhos})")
+        compare_caches(dllm, orc, ses, tol, f"step {step}")
+    with pytest.raises(dllm.DllmError):
+        ses.step_cached_layers(False, False, [0.25])

@@ -127,3 +127,41 @@ def test_unknown_variant_is_rejected():
     o.step(True, True)
     with pytest.raises(ValueError):
         o.step(False, False, 0.5, strategy="q_verify")
+
+
+# ---- cross-layer allocation of the update ratio (Sec. A.4, Table 11) ---------------------------
+def test_per_layer_rho_selects_floor_rho_l_R_rows_per_layer_and_uniform_list_equals_scalar():
+    cfg = GQA_TINY
+    a, _ = make(cfg, B=2, scale=3.0)
+    b, _ = make(cfg, B=2, scale=3.0)
+    for o in (a, b):
+        o.step(True, True)
+        unmask_some(o, 1)
+    ra = a.step(False, False, rho=[0.5, 0.5])
+    rb = b.step(False, False, rho=0.5)
+    assert rel_l2(ra.hidden, rb.hidden) == 0.0
+    unmask_some(a, 2)
+    before = [[c[l].copy() for l in range(cfg.n_layers)] for c in (a.Kc, a.Ac, a.Fc)]
+    r = a.step(False, False, rho=[0.375, 0.125])            # the front-heavy allocation of Table 11
+    R, P = a.R, a.P
+    for l, rho_l in enumerate((0.375, 0.125)):
+        k = O.k_selected(rho_l, R)
+        assert r.selected[l].shape == (2, k)
+        for bb in range(2):
+            rest = np.setdiff1d(np.arange(R), r.selected[l][bb])
+            for c, snap in zip((a.Kc, a.Ac, a.Fc), before):
+                assert np.array_equal(c[l][bb, P + rest], snap[l][bb, P + rest])
+    with pytest.raises(ValueError):
+        a.step(False, False, rho=[0.25])
+
+
+def test_per_layer_rho_zero_layer_is_fully_cached():
+    cfg = GQA_TINY
+    o, _ = make(cfg, scale=3.0)
+    o.step(True, True)
+    unmask_some(o, 1)
+    snap = [c[1].copy() for c in (o.Kc, o.Vc, o.Ac, o.Fc)]
+    r = o.step(False, False, rho=[0.5, 0.0])
+    assert r.sim[1] is None and r.selected[1].shape == (1, 0)
+    for c, s0 in zip((o.Kc, o.Vc, o.Ac, o.Fc), snap):
+        assert np.array_equal(c[1], s0)
