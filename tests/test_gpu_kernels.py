@@ -51,6 +51,32 @@ def test_gemm_bf16_tcgen05(env, M, N, K):
         assert rel_l2(sub, want[: M // 2]) < 2e-6
 
 
+@pytest.mark.parametrize("act_tile,splits,stages", [(32, 1, 2), (64, 3, 4), (128, 2, 3), (128, 5, 6), (256, 1, 4),
+                                                    (256, 4, 2), (0, 0, 0), (64, 13, 9)])
+def test_gemm_bf16_explicit_plans(env, act_tile, splits, stages):
+    """Every activation-tile shape, split factor and ring depth gives the same product; with reduce=False the
+    split-K slabs are left in the scratch buffer and add up to it in slab order."""
+    torch, dllm = env
+    M, N, K = 150, 900, 832          # ragged M and N, 13 k-blocks
+    A = synth.round_to_bf16(synth.random_normal((M, K), seed=5))
+    W = synth.round_to_bf16(synth.random_normal((N, K), seed=6, std=0.05))
+    dA = torch.from_numpy(A).cuda().to(torch.bfloat16)
+    dW = torch.from_numpy(W).cuda().to(torch.bfloat16)
+    want = A.astype(np.float64) @ W.astype(np.float64).T
+    got = dllm.gemm_bf16_planned(dA, dW, act_tile, splits, stages).cpu().numpy()
+    assert rel_l2(got, want) < 2e-6
+    sb = dllm.lib.dllm_gemm_bf16_planned_scratch_bytes(M, N, K, act_tile, splits)
+    if sb:
+        scratch = torch.zeros(sb, dtype=torch.uint8, device="cuda")
+        dllm.gemm_bf16_planned(dA, dW, act_tile, splits, stages, scratch=scratch, reduce=False)
+        slabs = scratch.view(torch.float32).cpu().numpy().reshape(-1, M, N)
+        acc = slabs[0].copy()
+        for sl in slabs[1:]:
+            acc += sl
+        assert np.array_equal(acc, got)      # the reduction adds the slabs in index order
+    assert dllm.lib.dllm_gemm_bf16_planned(None, None, None, M, N, K, 48, 0, 0, None, 0, None) == dllm.INVALID_ARG
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_gemm_simt(env, dtype):
     torch, dllm = env
