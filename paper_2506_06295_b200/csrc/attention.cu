@@ -259,6 +259,19 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
   if (B <= 0 || a_seq <= 0) return cudaSuccess;
   if (hd > HD_MAX || (hd & 31) || H % Hkv) return cudaErrorInvalidValue;
   const bool tensor = dtype == 1 && !force_simt && (hd == 64 || hd == 128) && ((Hkv * hd) % 8 == 0);
+  if (tensor && a_seq * (H / Hkv) > AT_ROWS) {
+    // many active rows per KV head: 128-row tiles on tcgen05
+    int S = 1;
+    cudaError_t e = launch_attention_umma(L, q, Kc, Vc, o, B, a_seq, n, H, Hkv, hd, scratch, scratch_floats, &S);
+    if (e != cudaSuccess) return e;
+    if (S > 1) {
+      const size_t total = (size_t)B * a_seq * H;
+      e = launch_k(L, attn_combine_kernel, dim3((unsigned)((total + 7) / 8)), dim3(256), 0, scratch,
+                   scratch + (size_t)S * total * hd, (__nv_bfloat16*)o, total, S, hd);
+      L.count();
+    }
+    return e != cudaSuccess ? e : cudaGetLastError();
+  }
   if (tensor) {
     AttnPlan p = plan_attention(B, a_seq, n, H, Hkv);
     if (p.S > 1 && (!scratch || scratch_floats < p.scratch_floats)) {   // no room for partials: one split

@@ -1,0 +1,407 @@
+// Flash-style attention on the 5th-generation tensor cores (tcgen05) for the
+// steps with many active rows (response refresh, full steps, batched serving):
+// non-causal attention of the active query rows over ALL n cached keys of
+// their sequence (Sec. A.7), grouped KV heads packed along the row dimension.
+//
+// One CTA (128 threads) = 128 "virtual rows" ((query, head-of-group) pairs) of
+// one (sequence, KV head) x one split of the key range, key tiles of 128:
+//   S = Q K^T        tcgen05.mma, M = 128 rows, N = 128 keys, contraction HD;
+//                    Q and K tiles in shared memory (K-major, 128-byte swizzle),
+//                    S in TMEM (128 lanes x 128 fp32 columns)
+//   softmax          TMEM lane = row, so every thread owns one row: it loads its
+//                    128 scores with tcgen05.ld, takes max / exp2 / sum locally
+//                    (no shuffles) and writes P as bf16 into shared memory in
+//                    the layout of an MMA A operand
+//   O += P V         tcgen05.mma, M = 128 rows, N = HD, contraction 128 keys;
+//                    V is used as stored ([key][hd], "MN-major" B operand); O
+//                    accumulates in TMEM and is rescaled (tcgen05.ld / st) only
+//                    when a row's maximum has grown by more than 2^8 since its
+//                    reference was set; the scores of tile t+1 are issued right
+//                    behind O += P V of tile t, so the tensor pipe works while
+//                    the threads are between barriers
+// K and V tiles arrive by TMA into a two-stage ring; tile t+2 is requested when
+// tile t has been consumed.  Key-range splits write unnormalised partials plus
+// (max, sum) exactly like the mma.sync kernel, and the same merge kernel
+// finishes them.  Every mbarrier wait is bounded.
+#include "attention_core.cuh"
+#include "internal.h"
+#include "tma.cuh"
+#include "umma.cuh"
+
+namespace dllm {
+
+namespace {
+
+constexpr int UA_ROWS = 128;  // virtual rows per CTA (UMMA M)
+constexpr int UA_KEYS = 128;  // keys per tile
+
+// MN-major operand ([k][mn] rows of 64 mn-elements = 128 bytes, 128-byte swizzle,
+// panels of 64 mn-elements): lbo = bytes between panels along MN, sbo = bytes
+// between groups of 8 k-rows.
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+// 2^x on the special-function unit (ex2.approx: relative error about 2^-22, far below the bf16 rounding of P)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <int HD>
+struct UaSmem {
+  static constexpr uint32_t Q_BYTES = UA_ROWS * HD * 2;
+  static constexpr uint32_t KV_TILE = UA_KEYS * HD * 2;        // one K or V tile
+  static constexpr uint32_t STAGE = 2 * KV_TILE;               // K then V
+  static constexpr uint32_t P_BYTES = UA_ROWS * UA_KEYS * 2;
+  static constexpr uint32_t TOTAL = Q_BYTES + 2 * STAGE + P_BYTES + 1024;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                        const __grid_constant__ CUtensorMap tmV,
+                                                        const __nv_bfloat16* __restrict__ q,
+                                                        __nv_bfloat16* __restrict__ o, float* __restrict__ o_part,
+                                                        float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv,
+                                                        int S, int keys_per_split, float scale_log2,
+                                                        int* __restrict__ status) {
+  using SM = UaSmem<HD>;
+  constexpr int PANELS = HD / 64;
+  constexpr uint32_t TMEM_COLS = 256;  // S: columns 0..127, O_t: columns 128..128+HD-1
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t kv_full[2];
+  __shared__ __align__(8) uint64_t bar_s, bar_o;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_gen = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_s = base, kv_s = base + SM::Q_BYTES, p_s = kv_s + 2 * SM::STAGE;
+  uint8_t* p_gen = base_gen + SM::Q_BYTES + 2 * SM::STAGE;
+  volatile int* abortp = &abort_flag;
+
+  const int G = H / Hkv;
+  const int kh = blockIdx.y;
+  const int b = blockIdx.z / S, split = blockIdx.z - b * S;
+  const int row0 = blockIdx.x * UA_ROWS;
+  const int n_rows = a_seq * G;
+  const int key_lo = split * keys_per_split;
+  const int key_hi = min(n, key_lo + keys_per_split);
+  const int n_tiles = (key_hi - key_lo + UA_KEYS - 1) / UA_KEYS;  // >= 1 by construction of the plan
+  const int dq = H * HD;
+
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&kv_full[0]), 1);
+    mbar_init(smem_u32(&kv_full[1]), 1);
+    mbar_init(smem_u32(&bar_s), 1);
+    mbar_init(smem_u32(&bar_o), 1);
+    mbar_fence_init();
+    prefetch_tensormap(&tmK);
+    prefetch_tensormap(&tmV);
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = tmem_slot;
+  pdl_wait();  // Q, K and V come from the preceding kernels
+  pdl_trigger();
+
+  // K/V tile t -> stage t & 1: per 64-column panel two boxes of 64 keys
+  auto issue = [&](int t) {
+    const int st = t & 1;
+    const uint32_t fb = smem_u32(&kv_full[st]);
+    mbar_expect_tx(fb, SM::STAGE);
+    const uint32_t dst = kv_s + st * SM::STAGE;
+    const int key0 = key_lo + t * UA_KEYS;
+#pragma unroll
+    for (int p = 0; p < PANELS; ++p)
+#pragma unroll
+      for (int h2 = 0; h2 < 2; ++h2) {
+        const uint32_t off = p * (UA_KEYS * 128) + h2 * (64 * 128);
+        tma_load_3d(dst + off, &tmK, fb, kh * HD + p * 64, key0 + h2 * 64, b);
+        tma_load_3d(dst + SM::KV_TILE + off, &tmV, fb, kh * HD + p * 64, key0 + h2 * 64, b);
+      }
+  };
+  if (tid == 0) {
+    issue(0);
+    if (n_tiles > 1) issue(1);
+  }
+  // Q tile: 16-byte loads into the swizzled panel layout (rows past the end are zero)
+  for (int e = tid; e < UA_ROWS * (HD / 8); e += 128) {
+    const int r = e / (HD / 8), dc = e - r * (HD / 8);
+    const int vr = row0 + r;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (vr < n_rows) {
+      const int qi = vr / G, g = vr - qi * G;
+      v = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
+    }
+    *reinterpret_cast<uint4*>(base_gen + tile_off<UA_ROWS>(r, dc)) = v;
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic stores -> MMA reads of shared memory
+  __syncthreads();
+
+  constexpr uint32_t idesc_s = make_idesc(UA_ROWS, UA_KEYS);
+  constexpr uint32_t idesc_o = make_idesc(UA_ROWS, HD) | (1u << 16);  // B operand (V) is MN-major
+  const uint32_t row_lane = ((uint32_t)(warp * 32)) << 16;           // this warp's TMEM lanes
+  const int row = warp * 32 + lane;                                   // this thread's row of the tile
+  constexpr float RESCALE_STEP = 8.f;  // log2 units a row's maximum may exceed its reference before O is rescaled
+
+  auto issue_s = [&](int t) {  // S(t) = Q K(t)^T; returns false if the K/V tile never arrived
+    const int st = t & 1;
+    if (!mbar_wait(smem_u32(&kv_full[st]), (uint32_t)(t >> 1) & 1u, abortp)) return false;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t k_s = kv_s + st * SM::STAGE;
+#pragma unroll
+    for (int ks = 0; ks < HD / 16; ++ks) {
+      const uint32_t off = (ks >> 2) * (128 * 128) + (ks & 3) * 32;  // panel, then 32 bytes per k-step
+      umma_bf16(tmem, make_smem_desc(q_s + off), make_smem_desc(k_s + off), idesc_s, ks > 0 ? 1u : 0u);
+    }
+    umma_commit(smem_u32(&bar_s));
+    return true;
+  };
+
+  // m_ref: the maximum the exponentials of this row refer to; it follows the
+  // true running maximum lazily (O in TMEM is only rescaled when the maximum has
+  // grown by more than RESCALE_STEP, which keeps every exponential below 2^8)
+  float m_ref = -INFINITY, l_run = 0.f;
+  bool ok = true;
+  if (tid == 0) ok = issue_s(0);
+
+  for (int t = 0; t < n_tiles; ++t) {
+    const int st = t & 1;
+    const uint32_t v_s = kv_s + st * SM::STAGE + SM::KV_TILE;
+    // S(t) is complete; the MMAs are executed in order, so O += P V of tile t-1 is complete too
+    ok = mbar_wait(smem_u32(&bar_s), (uint32_t)t & 1u, abortp);
+    ok = __syncthreads_and(ok);
+    if (!ok) break;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (tid == 0 && t >= 1 && t + 1 < n_tiles) issue(t + 1);  // stage (t-1)&1 is free: tile t+1 goes there
+    // ---- this thread's row of scores
+    const int key_base = key_lo + t * UA_KEYS;
+    float sv[UA_KEYS];
+    float mx = -INFINITY;
+    {
+      uint32_t r0[32], r1[32], r2[32], r3[32];  // all four loads in flight, one wait
+      tmem_ld32(tmem + row_lane + 0u, r0);
+      tmem_ld32(tmem + row_lane + 32u, r1);
+      tmem_ld32(tmem + row_lane + 64u, r2);
+      tmem_ld32(tmem + row_lane + 96u, r3);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        sv[j] = __uint_as_float(r0[j]);
+        sv[32 + j] = __uint_as_float(r1[j]);
+        sv[64 + j] = __uint_as_float(r2[j]);
+        sv[96 + j] = __uint_as_float(r3[j]);
+      }
+      const int valid = key_hi - key_base;  // >= 1
+#pragma unroll
+      for (int j = 0; j < UA_KEYS; ++j) {
+        sv[j] = (j < valid) ? sv[j] * scale_log2 : -INFINITY;
+        mx = fmaxf(mx, sv[j]);
+      }
+    }
+    // ---- lazy rescale of O (warp-uniform branch: the TMEM accesses are warp-collective)
+    const bool grow = mx > m_ref + RESCALE_STEP;
+    if (__any_sync(0xffffffffu, grow)) {
+      const float corr = grow ? exp2f(m_ref - mx) : 1.f;  // first tile: exp2(-inf) = 0, O is not read (t == 0)
+      if (grow) {
+        m_ref = mx;
+        l_run *= corr;
+      }
+      if (t > 0) {
+#pragma unroll
+        for (int c = 0; c < HD; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(tmem + row_lane + 128u + (uint32_t)c, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
+          tmem_st32(tmem + row_lane + 128u + (uint32_t)c, r);
+        }
+      }
+    }
+    // ---- probabilities -> shared memory (bf16, layout of an MMA A operand)
+    float p_sum = 0.f;
+#pragma unroll
+    for (int c8 = 0; c8 < UA_KEYS / 8; ++c8) {
+      float pv[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        pv[j] = fast_exp2(sv[c8 * 8 + j] - m_ref);
+        p_sum += pv[j];
+      }
+      *reinterpret_cast<uint4*>(p_gen + tile_off<UA_ROWS>(row, c8)) =
+          make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
+    }
+    l_run += p_sum;
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    // ---- O += P V, and straight after it the scores of the next tile
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+      for (int ks = 0; ks < UA_KEYS / 16; ++ks) {
+        const uint32_t a_off = (ks >> 2) * (UA_ROWS * 128) + (ks & 3) * 32;  // P: K-major, panels of 64 keys
+        const uint32_t b_off = ks * (16 * 128);                             // V: 16 key rows of 128 bytes
+        umma_bf16(tmem + 128, make_smem_desc(p_s + a_off), make_smem_desc_mn(v_s + b_off, UA_KEYS * 128, 1024), idesc_o,
+                  (t > 0 || ks > 0) ? 1u : 0u);
+      }
+      if (t + 1 < n_tiles)
+        ok = issue_s(t + 1);
+      else
+        umma_commit(smem_u32(&bar_o));  // last tile: O is final when this fires
+    }
+  }
+  if (ok) {
+    ok = mbar_wait(smem_u32(&bar_o), 0u, abortp);
+    ok = __syncthreads_and(ok);
+  }
+
+  if (ok) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int vr = row0 + row;
+    const bool live = vr < n_rows;
+    const int qi = live ? vr / G : 0, g = live ? vr - qi * G : 0;
+    const size_t orow = ((size_t)b * a_seq + qi) * H + (kh * G + g);  // (row, head) index
+    const float inv = 1.f / l_run;
+    const size_t total = (size_t)gridDim.z / S * a_seq * H;
+#pragma unroll
+    for (int c = 0; c < HD; c += 32) {
+      uint32_t r[32];
+      tmem_ld32(tmem + row_lane + 128u + (uint32_t)c, r);  // warp-collective: every lane takes part
+      tmem_ld_wait();
+      if (!live) continue;
+      if (S == 1) {
+        __nv_bfloat16* dst = o + orow * HD + c;
+#pragma unroll
+        for (int i = 0; i < 32; i += 8)
+          *reinterpret_cast<uint4*>(dst + i) = make_uint4(
+              pack_bf16(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv),
+              pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv),
+              pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv),
+              pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv));
+      } else {
+        float* dst = o_part + ((size_t)split * total + orow) * HD + c;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+          *reinterpret_cast<uint4*>(dst + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+      }
+    }
+    if (live && S > 1) {
+      float* ml = ml_part + ((size_t)split * total + orow) * 2;
+      ml[0] = m_ref;
+      ml[1] = l_run;
+    }
+  } else {
+    if (tid == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+    drain_delay();
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+template <int HD>
+cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
+                        float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
+  constexpr int SMEM = (int)UaSmem<HD>::TOTAL;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int G = H / Hkv;
+  const size_t total = (size_t)B * a_seq * H;
+  float* o_part = scratch;
+  float* ml_part = scratch ? scratch + (size_t)S * total * HD : nullptr;
+  dim3 grid((a_seq * G + UA_ROWS - 1) / UA_ROWS, Hkv, B * S);
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+  cudaError_t e = launch_k(L, attn_umma_kernel<HD>, grid, dim3(128), SMEM, tmK, tmV, (const __nv_bfloat16*)q,
+                           (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split, scale_log2,
+                           L.d_status);
+  L.count();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+}  // namespace
+
+// Key-range splits for 128-row tiles: enough CTAs to cover the SMs, whole
+// 128-key tiles per split, no more splits than the scratch holds.
+AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats) {
+  AttnPlan p;
+  const int G = H / Hkv;
+  const long tiles = (long)((a_seq * G + UA_ROWS - 1) / UA_ROWS) * Hkv * B;
+  int S = 1;
+  if (tiles < 148) S = (int)((148 + tiles - 1) / tiles);
+  const int key_tiles = (n + UA_KEYS - 1) / UA_KEYS;
+  if (S > key_tiles) S = key_tiles;
+  const size_t per_split = (size_t)B * a_seq * H * (128 + 2);
+  if (S > 1 && (size_t)S * per_split > scratch_floats) S = (int)(scratch_floats / per_split);
+  if (S < 1) S = 1;
+  const int tiles_per_split = (key_tiles + S - 1) / S;
+  p.keys_per_split = tiles_per_split * UA_KEYS;
+  p.S = (key_tiles + tiles_per_split - 1) / tiles_per_split;
+  p.scratch_floats = p.S > 1 ? (size_t)p.S * per_split : 0;
+  return p;
+}
+
+cudaError_t launch_attention_umma(const Launch& L, const void* q, const void* Kc, const void* Vc, void* o, int B,
+                                  int a_seq, int n, int H, int Hkv, int hd, float* scratch, size_t scratch_floats,
+                                  int* S_out) {
+  const AttnPlan p = plan_attention_umma(B, a_seq, n, H, Hkv, scratch ? scratch_floats : 0);
+  CUtensorMap tmK, tmV;
+  if (!get_tensor_map_3d(Kc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, 64, &tmK) ||
+      !get_tensor_map_3d(Vc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, 64, &tmV))
+    return cudaErrorInvalidValue;
+  if (S_out) *S_out = p.S;
+  return hd == 64 ? launch_umma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
+                  : launch_umma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
+}
+
+}  // namespace dllm

@@ -204,4 +204,11 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
                              int a_seq, int n, int H, int Hkv, int hd, float* scratch, size_t scratch_floats,
                              bool force_simt);
 
+// The same attention with 128-row tiles on tcgen05 (attention_umma.cu), for
+// many active rows per KV head.  *S_out: key-range splits used (> 1: the caller
+// merges the partials in `scratch` with the combine kernel).
+cudaError_t launch_attention_umma(const Launch& L, const void* q, const void* Kc, const void* Vc, void* o, int B,
+                                  int a_seq, int n, int H, int Hkv, int hd, float* scratch, size_t scratch_floats,
+                                  int* S_out);
+
 }  // namespace dllm
