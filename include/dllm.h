@@ -88,6 +88,17 @@ size_t dllm_workspace_bytes(const dllm_config* cfg, int B, int P, int R);
  * everything else has the model dtype. */
 dllm_status dllm_tensor_offset(const dllm_config* cfg, const char* name, size_t* offset_bytes,
                                size_t* n_elements);
+/* Row blocking of a tensor inside the blob.  *block_rows == 0: its n_elements
+ * are contiguous from its offset.  Otherwise its rows are stored in blocks of
+ * *block_rows consecutive rows, block b starting *block_stride_bytes * b after
+ * the tensor's offset.  Only ".wg" and ".wu" of a bf16 model with
+ * d_ffn % 64 == 0 are blocked (64 rows of W_gate, then the same 64 rows of
+ * W_up, and so on), so that the projection that forms both halves of the
+ * SwiGLU FFN (Sec. A.7 counts it as 2 of the 3 d x d_ffn products) can apply
+ * silu(gate) * up to its own output tile.  dllm_model_set_tensor() places the
+ * rows itself; only a caller that writes the blob directly needs this. */
+dllm_status dllm_tensor_blocks(const dllm_config* cfg, const char* name, size_t* block_rows,
+                               size_t* block_stride_bytes);
 
 /* ---- model p_theta --------------------------------------------------------- */
 /* Binds a model handle to a caller-owned device blob of dllm_weights_bytes(). */
@@ -241,6 +252,16 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
 size_t dllm_gemm_bf16_planned_scratch_bytes(int M, int N, int K, int act_tile, int splits);
 dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
                                    int splits, int stages, void* d_partials, size_t partials_bytes, void* stream);
+/* Gate and up projection of the SwiGLU FFN with the activation applied in the
+ * GEMM's epilogue (Sec. A.7's FFN: two of its three d x d_ffn products):
+ * out[M, d_ffn] (bf16, DEVICE) = silu(A Wg^T) * (A Wu^T), A [M, K] bf16,
+ * d_Wgu [2 * d_ffn, K] bf16 holding 64 rows of Wg, the same 64 rows of Wu, the
+ * next 64 of Wg and so on (the blocked layout of dllm_tensor_blocks).  No
+ * split-K, no scratch; products accumulate in fp32 and the result is rounded to
+ * bf16 once.  d_ffn must be a multiple of 64, K of 8.  act_tile / stages as in
+ * dllm_gemm_bf16_planned. */
+dllm_status dllm_ffn_gate_up_bf16(const void* d_A, const void* d_Wgu, void* d_out, int M, int d_ffn, int K,
+                                  int act_tile, int stages, void* stream);
 /* The same product on the plain fp32 ALUs (operands fp32 or bf16): the GEMM of
  * the fp32 mode. */
 dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int dtype,

@@ -54,7 +54,7 @@ WeightLayout make_layout(const dllm_config& c) {
     l.wqkv = take((dq + 2 * dkv) * d * es);  // rows: W_q, then W_k, then W_v
     l.wo = take(d * dq * es);
     l.norm2 = take(d * 4);
-    l.wgu = take(2 * m * d * es);            // rows: W_gate, then W_up
+    l.wgu = take(2 * m * d * es);            // rows: W_gate, then W_up (or blocks of 64 and 64: gu_interleaved)
     l.wd = take(d * m * es);
   }
   w.total = off;
@@ -78,9 +78,16 @@ const char* check_supported(const dllm_config* c) {
   return nullptr;
 }
 
+// bf16 models whose d_ffn is a multiple of 64 store W_gate and W_up row-interleaved in blocks of 64: gate row r
+// is stacked row (r / 64) * 128 + r % 64 and up row r is 64 rows further, so that one 128-row GEMM tile holds
+// both halves of 64 FFN columns and its epilogue can form silu(gate) * up (Sec. A.7's FFN, one pass less).
+bool gu_interleaved(const dllm_config& c) { return c.dtype == DLLM_BF16 && c.d_ffn % 64 == 0; }
+
 struct TensorRef {
   size_t off, n;
   bool f32;
+  size_t block_rows = 0;    // 0: contiguous; else the rows come in blocks of this many ...
+  size_t block_stride = 0;  // ... whose starts are this many bytes apart
 };
 
 bool find_tensor(const dllm_config& c, const WeightLayout& w, const char* name, TensorRef* out) {
@@ -99,8 +106,11 @@ bool find_tensor(const dllm_config& c, const WeightLayout& w, const char* name, 
   if (!strcmp(t, "wk")) return *out = {L.wqkv + dq * d * es, dkv * d, false}, true;
   if (!strcmp(t, "wv")) return *out = {L.wqkv + (dq + dkv) * d * es, dkv * d, false}, true;
   if (!strcmp(t, "wo")) return *out = {L.wo, d * dq, false}, true;
-  if (!strcmp(t, "wg")) return *out = {L.wgu, m * d, false}, true;
-  if (!strcmp(t, "wu")) return *out = {L.wgu + m * d * es, m * d, false}, true;
+  if (!strcmp(t, "wg") || !strcmp(t, "wu")) {
+    const bool up = t[1] == 'u';
+    if (gu_interleaved(c)) return *out = {L.wgu + (up ? 64 * d * es : 0), m * d, false, 64, 128 * d * es}, true;
+    return *out = {L.wgu + (up ? m * d * es : 0), m * d, false}, true;
+  }
   if (!strcmp(t, "wd")) return *out = {L.wd, d * m, false}, true;
   return false;
 }
@@ -303,8 +313,9 @@ int k_selected(float rho, int R, dllm_kround kr) {
 
 // One GEMM of the step: out = A[M,K] * W[N,K]^T as split-K partial slabs.
 dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void* W, int M, int N, int K,
-                     Partials* out) {
+                     Partials* out, void* swiglu_out = nullptr, bool* fused = nullptr) {
   float* part = s->wsp<float>(s->ws.part);
+  if (fused) *fused = false;
   *out = Partials{part, (size_t)M * N, 1, N};
   if (M <= 0) return DLLM_OK;
   // algorithmic traffic of one projection: the weight matrix and the activation
@@ -324,9 +335,12 @@ dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void
   if ((size_t)plan.S_max * M * N > s->ws.part_floats)
     return fail(&s->err, DLLM_UNSUPPORTED, "GEMM %dx%dx%d with %d slabs exceeds the workspace", M, N, K, plan.S_max);
   const char* why = nullptr;
-  cudaError_t e = launch_gemm_bf16(L, A, W, part, M, N, K, plan, &why);
+  // an unsplit gate / up projection of an interleaved weight finishes SwiGLU in its own epilogue
+  const bool fuse = swiglu_out && plan.S_max == 1 && gu_interleaved(s->m->cfg);
+  cudaError_t e = launch_gemm_bf16(L, A, W, part, M, N, K, plan, &why, fuse ? swiglu_out : nullptr, fuse ? N / 2 : 0);
   if (e != cudaSuccess)
     return fail(&s->err, DLLM_CUDA_ERROR, "bf16 GEMM %dx%dx%d: %s", M, N, K, why ? why : cudaGetErrorString(e));
+  if (fused) *fused = fuse;
   *out = make_partials(part, M, N, plan);
   return DLLM_OK;
 }
@@ -344,7 +358,7 @@ dllm_status enqueue_step_mk(dllm_session* s, int rr, int ksel, cudaStream_t stre
   MkParams p;
   memset(&p, 0, sizeof p);
   p.B = s->B; p.P = s->P; p.R = s->R; p.n = s->n; p.d = d; p.H = H; p.Hkv = Hkv; p.hd = hd; p.dq = dq; p.dkv = dkv;
-  p.m = m; p.T = c.n_layers; p.eps = c.rms_eps;
+  p.m = m; p.T = c.n_layers; p.eps = c.rms_eps; p.gu_interleaved = gu_interleaved(c);
   p.rr = rr; p.ksel = ksel; p.a_seq = ksel; p.Ma = s->B * ksel; p.BR = BR;
   for (int l = 0; l < c.n_layers; ++l)
     if (!rr && s->forced_count[l] >= 0) p.forced_mask |= 1ull << l;
@@ -509,8 +523,11 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.obuf), W + lo.wo, Ma, d, dq, &part)) != DLLM_OK) return st;
       launch_oproj_epilogue(L, dt, part, act, x, reinterpret_cast<const float*>(W + lo.norm2),
                             s->cache(l, DLLM_CACHE_ATTN), s->wsp<uint8_t>(s->ws.hn), g, Ma, c.rms_eps);
-      if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.hn), W + lo.wgu, Ma, 2 * m, d, &part)) != DLLM_OK) return st;
-      launch_silu_mul(L, dt, part, s->wsp<uint8_t>(s->ws.ffn), Ma, m);
+      bool fused = false;
+      if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.hn), W + lo.wgu, Ma, 2 * m, d, &part, s->wsp<uint8_t>(s->ws.ffn),
+                         &fused)) != DLLM_OK)
+        return st;
+      if (!fused) launch_silu_mul(L, dt, part, s->wsp<uint8_t>(s->ws.ffn), Ma, m, gu_interleaved(c));
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.ffn), W + lo.wd, Ma, d, m, &part)) != DLLM_OK) return st;
     }
     // FFNOut rows -> cache, residual assembly for all carried rows, next norm
@@ -639,6 +656,17 @@ dllm_status dllm_tensor_offset(const dllm_config* cfg, const char* name, size_t*
   return DLLM_OK;
 }
 
+dllm_status dllm_tensor_blocks(const dllm_config* cfg, const char* name, size_t* block_rows, size_t* block_stride_bytes) {
+  const char* why = check_config(cfg);
+  if (why) return fail(nullptr, DLLM_INVALID_ARG, "%s", why);
+  if (!name) return fail(nullptr, DLLM_INVALID_ARG, "name is NULL");
+  TensorRef t;
+  if (!find_tensor(*cfg, make_layout(*cfg), name, &t)) return fail(nullptr, DLLM_INVALID_ARG, "unknown tensor '%s'", name);
+  if (block_rows) *block_rows = t.block_rows;
+  if (block_stride_bytes) *block_stride_bytes = t.block_stride;
+  return DLLM_OK;
+}
+
 dllm_status dllm_model_create(const dllm_config* cfg, void* d_weights, dllm_model** out) {
   if (!out) return fail(nullptr, DLLM_INVALID_ARG, "out is NULL");
   *out = nullptr;
@@ -674,7 +702,13 @@ dllm_status dllm_model_set_tensor(dllm_model* m, const char* name, const float* 
     return fail(&m->err, DLLM_OUT_OF_MEMORY, "host allocation failed");
   }
   for (size_t i = 0; i < t.n; ++i) tmp[i] = f32_to_bf16_rne(h_src[i]);
-  CU_TRY(&m->err, cudaMemcpy(m->d_w + t.off, tmp.data(), t.n * 2, cudaMemcpyHostToDevice));
+  if (t.block_rows) {
+    const size_t block_bytes = t.block_rows * (size_t)m->cfg.d_model * 2;
+    CU_TRY(&m->err, cudaMemcpy2D(m->d_w + t.off, t.block_stride, tmp.data(), block_bytes, block_bytes,
+                                 t.n * 2 / block_bytes, cudaMemcpyHostToDevice));
+  } else {
+    CU_TRY(&m->err, cudaMemcpy(m->d_w + t.off, tmp.data(), t.n * 2, cudaMemcpyHostToDevice));
+  }
   CU_TRY(&m->err, cudaDeviceSynchronize());
   return DLLM_OK;
 }
@@ -1105,6 +1139,22 @@ dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C,
   cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
   if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "bf16 GEMM: %s", why ? why : cudaGetErrorString(e));
   if (p.S_max > 1 && d_C) launch_reduce_partials(L, make_partials(part, M, N, p), d_C, M);
+  CU_TRY(nullptr, cudaGetLastError());
+  return DLLM_OK;
+}
+
+dllm_status dllm_ffn_gate_up_bf16(const void* d_A, const void* d_Wgu, void* d_out, int M, int d_ffn, int K,
+                                  int act_tile, int stages, void* stream) {
+  if (!d_A || !d_Wgu || !d_out || M <= 0 || d_ffn <= 0 || K <= 0)
+    return fail(nullptr, DLLM_INVALID_ARG, "bad gate / up arguments");
+  if (K % 8 || d_ffn % 64) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8 and d_ffn of 64");
+  if (act_tile < 0 || stages < 0 || (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 256))
+    return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128 or 256");
+  const GemmPlan p = plan_gemm_bf16(M, 2 * d_ffn, K, 1, stages, act_tile);
+  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  const char* why = nullptr;
+  cudaError_t e = launch_gemm_bf16(L, d_A, d_Wgu, nullptr, M, 2 * d_ffn, K, p, &why, d_out, d_ffn);
+  if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "gate / up GEMM: %s", why ? why : cudaGetErrorString(e));
   CU_TRY(nullptr, cudaGetLastError());
   return DLLM_OK;
 }

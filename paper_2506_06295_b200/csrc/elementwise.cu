@@ -488,7 +488,7 @@ void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int3
 
 // ------------------------------------------------------------------ SwiGLU gate
 template <typename T>
-__global__ void silu_mul_kernel(Partials part, T* __restrict__ out, int Ma, int m) {
+__global__ void silu_mul_kernel(Partials part, T* __restrict__ out, int Ma, int m, int interleaved) {
   pdl_wait();
   pdl_trigger();
   const int mv = m >> 3;
@@ -496,19 +496,20 @@ __global__ void silu_mul_kernel(Partials part, T* __restrict__ out, int Ma, int 
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
     const int r = (int)(idx / mv), j = (int)(idx - (size_t)r * mv) * 8;
     float gt[8], up[8];
-    sum_partials8(part.p, part.split_stride, part.count(r, j), (size_t)r * part.N + j, gt);
-    sum_partials8(part.p, part.split_stride, part.count(r, m + j), (size_t)r * part.N + m + j, up);
+    const int cg = interleaved ? (j >> 6) * 128 + (j & 63) : j, cu = interleaved ? cg + 64 : m + j;
+    sum_partials8(part.p, part.split_stride, part.count(r, cg), (size_t)r * part.N + cg, gt);
+    sum_partials8(part.p, part.split_stride, part.count(r, cu), (size_t)r * part.N + cu, up);
 #pragma unroll
     for (int t = 0; t < 8; ++t) gt[t] = gt[t] / (1.f + expf(-gt[t])) * up[t];
     Vec8<T>::store(out + (size_t)r * m + j, gt);
   }
 }
 
-void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int Ma, int m) {
+void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int Ma, int m, int interleaved) {
   if (Ma <= 0) return;
   const size_t total = (size_t)Ma * (m >> 3);
   const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
-  DLLM_DISPATCH(dtype, (launch_k(L, silu_mul_kernel<T>, dim3(blocks), dim3(256), 0, part, (T*)out, Ma, m)));
+  DLLM_DISPATCH(dtype, (launch_k(L, silu_mul_kernel<T>, dim3(blocks), dim3(256), 0, part, (T*)out, Ma, m, interleaved)));
   L.count();
 }
 

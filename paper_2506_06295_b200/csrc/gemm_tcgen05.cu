@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
                                                                 const __grid_constant__ CUtensorMap tmA,
                                                                 float* __restrict__ part, int M, int N, int num_kb,
                                                                 int kb_per_split, size_t split_stride, int STAGES,
+                                                                __nv_bfloat16* __restrict__ act_out, int m_ffn,
                                                                 int* __restrict__ status) {
   using SL = SmemLayout<BN>;
   extern __shared__ uint8_t smem_raw[];
@@ -166,8 +167,48 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   const bool have = mbar_wait(smem_u32(&accum_bar), 0u, abortp);
   if (!have && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_EPI);
   // the whole warp must agree before the warp-collective TMEM loads
-  const bool warp_ok = __all_sync(0xffffffffu, have);
-  if (warp_ok) {
+  bool warp_ok = __all_sync(0xffffffffu, have);
+  if (act_out) warp_ok = __syncthreads_and(warp_ok);  // the SwiGLU epilogue exchanges data between warps
+  if (warp_ok && act_out) {
+    // SwiGLU epilogue (no split-K): the tile's 128 weight rows are 64 gate rows followed by the 64 up rows
+    // of the same FFN columns, so TMEM lanes 0..63 hold gate and 64..127 hold up.  The accumulator goes
+    // through shared memory (the ring is drained: every MMA has completed) 64 activation rows at a time,
+    // transposed to [row][weight row], and comes back as silu(gate) * up in bf16, 8 bytes per thread.
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    constexpr int EXS = 132;   // floats per staged row: 16-byte aligned, rows 4 banks apart
+    constexpr int CH = BN < 64 ? BN : 64;
+    float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // [CH][EXS]
+    const int q = threadIdx.x & 15, rsub = threadIdx.x >> 4;  // 4 FFN columns, 8 rows per pass
+    const int col = blockIdx.y * 64 + 4 * q;
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += CH) {
+      if (m0 + c0 >= M) break;  // uniform across the CTA
+#pragma unroll
+      for (int c = 0; c < CH; c += 16) {
+        uint32_t r[16];
+        tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + c), r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[j]);
+      }
+      __syncthreads();
+#pragma unroll
+      for (int rr = rsub; rr < CH; rr += 8) {
+        const int m = m0 + c0 + rr;
+        const float4 gt = *reinterpret_cast<const float4*>(ex + rr * EXS + 4 * q);
+        const float4 up = *reinterpret_cast<const float4*>(ex + rr * EXS + 64 + 4 * q);
+        if (m < M && col < m_ffn) {
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(gt.x / (1.f + expf(-gt.x)) * up.x, gt.y / (1.f + expf(-gt.y)) * up.y);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(gt.z / (1.f + expf(-gt.z)) * up.z, gt.w / (1.f + expf(-gt.w)) * up.w);
+          uint2 pk;
+          pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(act_out + (size_t)m * m_ffn + col) = pk;
+        }
+      }
+      __syncthreads();
+    }
+  } else if (warp_ok) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const int n = n0 + warp * 32 + lane;
     float* out = part + (size_t)blockIdx.z * split_stride + n;
@@ -265,7 +306,7 @@ constexpr int max_stages(int bn) {
 
 template <int BN>
 cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMap& tmA, float* part, int M, int N,
-                       int num_kb, const GemmPlan& plan) {
+                       int num_kb, const GemmPlan& plan, void* act_out, int m_ffn) {
   using SL = SmemLayout<BN>;
   static bool configured = false;
   if (!configured) {
@@ -277,7 +318,7 @@ cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMa
   const int stages = plan.stages < 2 ? 2 : plan.stages > max_stages(BN) ? max_stages(BN) : plan.stages;
   dim3 grid((M + BN - 1) / BN, (N + TILE_W - 1) / TILE_W, plan.S_max);
   cudaError_t e = launch_k(L, gemm_bf16_tcgen05_kernel<BN>, grid, dim3(128), SL::total(stages), tmW, tmA, part, M, N,
-                           num_kb, plan.upc, (size_t)M * N, stages, L.d_status);
+                           num_kb, plan.upc, (size_t)M * N, stages, (__nv_bfloat16*)act_out, m_ffn, L.d_status);
   L.count();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -336,12 +377,16 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
 }
 
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
-                             const GemmPlan& plan, const char** err) {
+                             const GemmPlan& plan, const char** err, void* act_out, int m_ffn) {
   static const char* e_shape = "bf16 GEMM needs K % 8 == 0 and 16-byte aligned operands";
   static const char* e_map = "cuTensorMapEncodeTiled failed or is unavailable";
   if (M <= 0 || N <= 0) return cudaSuccess;
   if (K <= 0 || (K & 7) || ((uintptr_t)A & 15) || ((uintptr_t)W & 15)) {
     if (err) *err = e_shape;
+    return cudaErrorInvalidValue;
+  }
+  if (act_out && (plan.S_max != 1 || N != 2 * m_ffn || (m_ffn & 63) || ((uintptr_t)act_out & 7))) {
+    if (err) *err = "the SwiGLU epilogue needs an unsplit plan and d_ffn % 64 == 0";
     return cudaErrorInvalidValue;
   }
   CUtensorMap tmW, tmA;
@@ -352,10 +397,10 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
   }
   const int num_kb = (K + TILE_K - 1) / TILE_K;
   switch (plan.BN) {
-    case 32: return launch_one<32>(L, tmW, tmA, part, M, N, num_kb, plan);
-    case 64: return launch_one<64>(L, tmW, tmA, part, M, N, num_kb, plan);
-    case 128: return launch_one<128>(L, tmW, tmA, part, M, N, num_kb, plan);
-    default: return launch_one<256>(L, tmW, tmA, part, M, N, num_kb, plan);
+    case 32: return launch_one<32>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
+    case 64: return launch_one<64>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
+    case 128: return launch_one<128>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
+    default: return launch_one<256>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
   }
 }
 

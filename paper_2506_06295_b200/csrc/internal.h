@@ -108,7 +108,9 @@ void launch_scatter_rows(const Launch& L, int dtype, Partials part, const int32_
 void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int32_t* act, const float* x,
                            const float* gain2, void* Ac_layer, void* hn, Geo g, int Ma, float eps);
 // act[i][j] = silu(gate) * up from partials [Ma, 2m] (gate columns first).
-void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int Ma, int m);
+// interleaved: the columns of `part` are blocks of 64 gate columns followed by the 64 up columns of the same
+// FFN columns (the layout of the stacked weight when d_ffn % 64 == 0 in bf16); else all gate, then all up.
+void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int Ma, int m, int interleaved = 0);
 // x[c] = (x[c] + AttnOut[c]) + FFNOut[c] for carried rows c0 <= c < c1.
 void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer, const void* Fc_layer, Geo g, int c0,
                      int c1);
@@ -142,8 +144,10 @@ struct GemmPlan {
 GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split = 0, int force_stages = 0, int force_bn = 0);  // 0 = auto
 Partials make_partials(const float* p, int M, int N, const GemmPlan& plan);
 // Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
+// act_out != nullptr (unsplit plan, W = gate / up rows interleaved in blocks of 64, N = 2 * m_ffn): instead of
+// fp32 slabs the epilogue writes silu(gate) * up as bf16 [M, m_ffn].
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
-                             const GemmPlan& plan, const char** err);
+                             const GemmPlan& plan, const char** err, void* act_out = nullptr, int m_ffn = 0);
 
 // ---------------- megakernel.cu ----------------
 // One projection inside the persistent layer kernel: units (tile, k-block) in
@@ -158,6 +162,7 @@ struct alignas(64) MkParams {
   float eps;
   int rr, ksel, a_seq, Ma, BR;
   int attn_S, attn_kps;          // key-range splits of the attention phase, keys per split
+  int gu_interleaved;            // gate / up rows of the stacked weight alternate in blocks of 64
   int has_comb;                  // attention partials are merged in a phase of their own
   unsigned long long forced_mask;  // bit l: layer l takes its selection from the forced list
   const uint8_t* W;              // weight blob

@@ -619,8 +619,9 @@ __device__ void phase_silu(const Ctx& c) {
   for (size_t idx = (size_t)c.cta * MK_WORKERS + c.tid; idx < total; idx += (size_t)c.G * MK_WORKERS) {
     const int r = (int)(idx / mv), j = (int)(idx - (size_t)r * mv) * 8;
     float gt[8], up[8];
-    sum_partials8(part.p, part.split_stride, part.count(r, j), (size_t)r * part.N + j, gt);
-    sum_partials8(part.p, part.split_stride, part.count(r, m + j), (size_t)r * part.N + m + j, up);
+    const int cg = p.gu_interleaved ? (j >> 6) * 128 + (j & 63) : j, cu = p.gu_interleaved ? cg + 64 : m + j;
+    sum_partials8(part.p, part.split_stride, part.count(r, cg), (size_t)r * part.N + cg, gt);
+    sum_partials8(part.p, part.split_stride, part.count(r, cu), (size_t)r * part.N + cu, up);
 #pragma unroll
     for (int t = 0; t < 8; ++t) gt[t] = gt[t] / (1.f + expf(-gt[t])) * up[t];
     Vec8<bf16>::store(out + (size_t)r * m + j, gt);

@@ -42,6 +42,7 @@ SIGNATURES = {
     "dllm_cache_bytes": (_SZ, [C.POINTER(Config), _I, _I, _I]),
     "dllm_workspace_bytes": (_SZ, [C.POINTER(Config), _I, _I, _I]),
     "dllm_tensor_offset": (_I, [C.POINTER(Config), C.c_char_p, C.POINTER(_SZ), C.POINTER(_SZ)]),
+    "dllm_tensor_blocks": (_I, [C.POINTER(Config), C.c_char_p, C.POINTER(_SZ), C.POINTER(_SZ)]),
     "dllm_model_create": (_I, [C.POINTER(Config), _P, C.POINTER(_P)]),
     "dllm_model_set_tensor": (_I, [_P, C.c_char_p, _P, _SZ]),
     "dllm_model_destroy": (_I, [_P]),
@@ -78,6 +79,7 @@ SIGNATURES = {
     "dllm_gemm_bf16": (_I, [_P, _P, _P, _I, _I, _I, _P, _P]),
     "dllm_gemm_bf16_planned_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I]),
     "dllm_gemm_bf16_planned": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
+    "dllm_ffn_gate_up_bf16": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _P]),
     "dllm_gemm_simt": (_I, [_P, _P, _P, _I, _I, _I, _I, _P]),
     "dllm_attention_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I, _I, _I]),
     "dllm_attention": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
@@ -129,6 +131,13 @@ def tensor_offset(cfg, name: str) -> tuple[int, int]:
     return off.value, n.value
 
 
+def tensor_blocks(cfg, name: str) -> tuple[int, int]:
+    """(rows per block, bytes between block starts); (0, 0) for a contiguous tensor."""
+    rows, stride = _SZ(), _SZ()
+    _check(lib.dllm_tensor_blocks(C.byref(make_config(cfg)), name.encode(), C.byref(rows), C.byref(stride)))
+    return rows.value, stride.value
+
+
 def _stream_ptr(stream) -> int:
     if stream is None:
         return 0
@@ -165,12 +174,19 @@ class Model:
         return self
 
     def tensor_view(self, name: str):
-        """torch view of one tensor inside the blob (for filling weights on the device)."""
+        """torch view of one tensor inside the blob (for filling weights on the device): flat for a
+        contiguous tensor, [blocks, rows per block, d_model] (strided) for a row-blocked one."""
         import torch
         off, n = tensor_offset(self.cfg, name)
         is_f32 = name.endswith(("norm1", "norm2", "norm_f")) or self.cfg.dtype != "bf16"
         dt, es = (torch.float32, 4) if is_f32 else (torch.bfloat16, 2)
-        return self.blob[off:off + n * es].view(dt)
+        rows, stride = tensor_blocks(self.cfg, name)
+        if rows == 0:
+            return self.blob[off:off + n * es].view(dt)
+        d = self.cfg.d_model
+        nb = n // (rows * d)
+        span = self.blob[off:off + (nb - 1) * stride + rows * d * es].view(dt)
+        return span.as_strided((nb, rows, d), (stride // es, d, 1))
 
     def random_init_on_device(self, seed: int, std: float = 0.02) -> "Model":
         """N(0, std^2) weights and unit norm gains drawn with torch on the device
@@ -184,10 +200,12 @@ class Model:
             if name.endswith(("norm1", "norm2", "norm_f")):
                 v.fill_(1.0)
             else:
-                chunk = 1 << 26
-                for s in range(0, v.numel(), chunk):
-                    e = min(v.numel(), s + chunk)
-                    v[s:e] = (torch.randn(e - s, generator=gen, device=self.device, dtype=torch.float32) * std).to(v.dtype)
+                per = v[0].numel() if v.dim() > 1 else 1      # a blocked tensor is filled block by block
+                chunk = max(1, (1 << 26) // per)
+                for s in range(0, v.shape[0], chunk):
+                    e = min(v.shape[0], s + chunk)
+                    r = torch.randn((e - s) * per, generator=gen, device=self.device, dtype=torch.float32) * std
+                    v[s:e] = r.to(v.dtype).view(v[s:e].shape)
         return self
 
     def close(self):
@@ -379,6 +397,18 @@ def gemm_bf16_planned(A, W, act_tile=0, splits=0, stages=0, out=None, scratch=No
                                       M, N, K, act_tile, splits, stages, C.c_void_p(scratch.data_ptr()),
                                       scratch.numel(), C.c_void_p(sp)))
     return Cm
+
+
+def ffn_gate_up_bf16(A, Wgu, act_tile=0, stages=0, stream=None):
+    """silu(A Wg^T) * (A Wu^T) as bf16 [M, d_ffn]; Wgu [2 d_ffn, K] alternates 64 rows of Wg and 64 of Wu."""
+    import torch
+    M, K = A.shape
+    m = Wgu.shape[0] // 2
+    out = torch.empty((M, m), dtype=torch.bfloat16, device=A.device)
+    sp = _stream_ptr(stream if stream is not None else torch.cuda.current_stream(A.device))
+    _check(lib.dllm_ffn_gate_up_bf16(C.c_void_p(A.data_ptr()), C.c_void_p(Wgu.data_ptr()), C.c_void_p(out.data_ptr()),
+                                     M, m, K, act_tile, stages, C.c_void_p(sp)))
+    return out
 
 
 def gemm_simt(A, W, stream=None):

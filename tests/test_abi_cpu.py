@@ -54,9 +54,16 @@ def test_weight_blob_layout(dllm):
             off, n = dllm.tensor_offset(cfg, name)
             assert n == int(np.prod(shape))
             size = n * (4 if name.endswith(("norm1", "norm2", "norm_f")) else es)
-            assert off % 16 == 0 and off + size <= total
-            spans.append((off, off + size, name))
+            rows, stride = dllm.tensor_blocks(cfg, name)
+            assert off % 16 == 0
+            if rows == 0:
+                spans.append((off, off + size, name))
+            else:   # row-blocked: one span per block
+                blk = rows * cfg.d_model * es
+                assert size % blk == 0 and stride >= blk
+                spans += [(off + b * stride, off + b * stride + blk, name) for b in range(size // blk)]
         spans.sort()
+        assert spans[-1][1] <= total
         for (a0, a1, an), (b0, b1, bn) in zip(spans, spans[1:]):
             assert a1 <= b0, f"{an} overlaps {bn}"
         # W_q, W_k, W_v are stacked contiguously (one GEMM for Q and K), so are W_gate, W_up
@@ -64,9 +71,16 @@ def test_weight_blob_layout(dllm):
         k, nk = dllm.tensor_offset(cfg, "layers.1.wk")
         v, _ = dllm.tensor_offset(cfg, "layers.1.wv")
         assert k == q + nq * es and v == k + nk * es
+        # ... so are W_gate and W_up: one after the other, or (bf16, d_ffn % 64 == 0) alternating in blocks of 64 rows
         g, ng = dllm.tensor_offset(cfg, "layers.0.wg")
         u, _ = dllm.tensor_offset(cfg, "layers.0.wu")
-        assert u == g + ng * es
+        rows, stride = dllm.tensor_blocks(cfg, "layers.0.wg")
+        if cfg.dtype == "bf16" and cfg.d_ffn % 64 == 0:
+            assert (rows, stride) == (64, 128 * cfg.d_model * es) == dllm.tensor_blocks(cfg, "layers.0.wu")
+            assert u == g + 64 * cfg.d_model * es
+        else:
+            assert rows == 0 and u == g + ng * es
+        assert dllm.tensor_blocks(cfg, "layers.1.wq") == (0, 0) == dllm.tensor_blocks(cfg, "lm_head")
 
 
 def test_llada_sizes_fit_one_gpu(dllm):

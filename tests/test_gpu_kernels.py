@@ -77,6 +77,27 @@ def test_gemm_bf16_explicit_plans(env, act_tile, splits, stages):
     assert dllm.lib.dllm_gemm_bf16_planned(None, None, None, M, N, K, 48, 0, 0, None, 0, None) == dllm.INVALID_ARG
 
 
+@pytest.mark.parametrize("M,m,K,act_tile", [(64, 1216, 512, 0), (3, 64, 64, 32), (70, 832, 448, 64), (130, 192, 1088, 128),
+                                            (300, 320, 256, 256), (257, 128, 832, 0)])
+def test_ffn_gate_up_epilogue(env, M, m, K, act_tile):
+    """Gate / up projection with SwiGLU in the GEMM epilogue against silu(A Wg^T) * (A Wu^T) in float64."""
+    torch, dllm = env
+    A = synth.round_to_bf16(synth.random_normal((M, K), seed=M + 3))
+    Wg = synth.round_to_bf16(synth.random_normal((m, K), seed=m + 1, std=0.08))
+    Wu = synth.round_to_bf16(synth.random_normal((m, K), seed=m + 2, std=0.08))
+    Wgu = np.stack([Wg.reshape(m // 64, 64, K), Wu.reshape(m // 64, 64, K)], axis=1).reshape(2 * m, K)
+    dA = torch.from_numpy(A).cuda().to(torch.bfloat16)
+    dW = torch.from_numpy(np.ascontiguousarray(Wgu)).cuda().to(torch.bfloat16)
+    got = dllm.ffn_gate_up_bf16(dA, dW, act_tile).float().cpu().numpy()
+    gate = A.astype(np.float64) @ Wg.astype(np.float64).T
+    want = gate / (1 + np.exp(-gate)) * (A.astype(np.float64) @ Wu.astype(np.float64).T)
+    assert rel_l2(got, want) < 3e-3                                     # one rounding to bf16: 2^-9 per element
+    assert np.abs(got - want).max() <= 2 ** -8 * np.abs(want).max() + 1e-6
+    assert np.array_equal(got, dllm.ffn_gate_up_bf16(dA, dW, act_tile).float().cpu().numpy())
+    assert dllm.lib.dllm_ffn_gate_up_bf16(None, None, None, M, m, K, 0, 0, None) == dllm.INVALID_ARG
+    assert dllm.lib.dllm_ffn_gate_up_bf16(dA.data_ptr(), dW.data_ptr(), dA.data_ptr(), M, 100, K, 0, 0, None) == dllm.INVALID_ARG
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_gemm_simt(env, dtype):
     torch, dllm = env

@@ -170,6 +170,36 @@ def test_small_bf16_step_kinds(env, gqa, path):
         assert err < 2e-2
 
 
+@pytest.mark.parametrize("path", ["tcgen05_gemm", "layer_kernel"])
+def test_bf16_gate_up_layouts(env, path):
+    """W_gate / W_up stored one after the other (d_ffn not a multiple of 64) and row-blocked (a multiple of 64,
+    where an unsplit gate / up GEMM applies SwiGLU itself and a split one leaves it to the next kernel) give the
+    oracle's step; the blocked model also accepts weights written straight into the blob."""
+    import dataclasses
+    torch, dllm = env
+    for d_ffn in (840, 832):
+        cfg = dataclasses.replace(synth.small_bf16_model(), d_ffn=d_ffn)
+        assert (dllm.tensor_blocks(cfg, "layers.0.wg")[0] == 64) == (d_ffn % 64 == 0)
+        B, P, R = 2, 150, 72
+        orc, ses, w = make_pair(dllm, cfg, B, P, R)
+        ses.use_layer_kernel(path == "layer_kernel")
+        if d_ffn % 64 == 0:   # rewrite the gate / up weights through the strided view: same model
+            for l in range(cfg.n_layers):
+                for t in ("wg", "wu"):
+                    v = ses.model.tensor_view(f"layers.{l}.{t}")
+                    v.zero_()
+                    v.copy_(torch.from_numpy(w[f"layers.{l}.{t}"]).cuda().to(torch.bfloat16).view(v.shape))
+        r = orc.step(True, True)
+        ses.step_full()
+        compare_step(orc, ses, r, 2e-2, what=f"full m={d_ffn}")
+        for step, (rp, rr, rho) in enumerate(((False, False, 0.25), (True, False, 0.5), (False, True, 0.0)), 1):
+            unmask(orc, ses, step, 3)
+            r = orc.step(rp, rr, rho)
+            ses.step_cached(rp, rr, rho)
+            compare_step(orc, ses, r, 2e-2, what=f"m={d_ffn} step {step}")
+        compare_caches(dllm, orc, ses, 2e-2, f"m={d_ffn}")
+
+
 def test_small_bf16_forced_selection_and_rho_invariants(env):
     torch, dllm = env
     cfg = synth.small_bf16_model()
