@@ -129,6 +129,31 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return warp_sum(t);
 }
 
+// Three sums over the block at once (one pair of barriers); `red` holds >= 96 floats.
+__device__ __forceinline__ void block_sum3(float& a, float& b, float& c, float* red) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  a = warp_sum(a);
+  b = warp_sum(b);
+  c = warp_sum(c);
+  __syncthreads();
+  if (lane == 0) {
+    red[w] = a;
+    red[32 + w] = b;
+    red[64 + w] = c;
+  }
+  __syncthreads();
+  a = warp_sum(lane < nw ? red[lane] : 0.f);
+  b = warp_sum(lane < nw ? red[32 + lane] : 0.f);
+  c = warp_sum(lane < nw ? red[64 + lane] : 0.f);
+}
+
+// Threads for a kernel that walks one row of `width` elements eight at a time: one trip when the row fits
+// (all loads of a row in flight at once), at most 512.
+inline int row_threads(int width) {
+  const int t = ((width + 7) / 8 + 31) / 32 * 32;
+  return t < 64 ? 64 : t > 512 ? 512 : t;
+}
+
 // Sum of n_slabs partial results for eight consecutive columns, slab 0 first.
 // The loads of up to four slabs are issued together so that their latencies
 // overlap; the adds keep the slab order.

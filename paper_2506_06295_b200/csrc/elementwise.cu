@@ -114,16 +114,92 @@ void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gai
   L.count();
 }
 
+// ------------------------------------------------------------------ selection inside a kernel
+// Bottom-k selection of sequence b by the whole CTA (R <= 1024: R^2 comparisons out of shared memory, 13 R + 16
+// bytes at `keys`).  Fills slot[j] = position of response row j among the selected rows, or -1; with `write` the
+// CTA also writes the index list, the active list (np prompt rows first) and its inverse.
+// mode 0: every row; 1: the ksel lowest scores (Sec. 3.2.2); 2: the forced list.  Ends with a barrier.
+__device__ __forceinline__ int32_t* select_sequence(unsigned long long* keys, const float* __restrict__ sim,
+                                                    const int32_t* __restrict__ forced, int mode, int ksel,
+                                                    int32_t* __restrict__ sel, int32_t* __restrict__ act,
+                                                    int32_t* __restrict__ inv, const Geo& g, int np, int b, bool write) {
+  const int R = g.R;
+  int32_t* slot = reinterpret_cast<int32_t*>(keys + R);
+  uint32_t* words = reinterpret_cast<uint32_t*>(slot + R);  // one ballot word per 32 rows
+  const int a_seq = np + ksel;
+  if (mode == 0) {
+    for (int j = threadIdx.x; j < R; j += blockDim.x) slot[j] = j;
+  } else if (mode == 2) {
+    for (int j = threadIdx.x; j < R; j += blockDim.x) slot[j] = -1;
+    __syncthreads();
+    for (int r = threadIdx.x; r < ksel; r += blockDim.x) slot[forced[(size_t)b * R + r]] = r;
+  } else {
+    for (int j = threadIdx.x; j < R; j += blockDim.x) {
+      const float s = __ldcg(sim + (size_t)b * R + j);
+      // key = round(s * 2^20), offset into 1 .. 2^32 - 1 (scores beyond +-2047 saturate); NaN sorts first
+      const float qf = fminf(fmaxf(rintf(s * 1048576.0f), -2147483520.0f), 2147483520.0f);
+      const long long q = (s == s) ? (long long)qf + (1ll << 31) : 0ll;
+      keys[j] = ((unsigned long long)q << 32) | (unsigned)j;
+    }
+    __syncthreads();
+    // rank of every key (two keys per shared-memory load); a row is selected iff its rank is below ksel
+    const int Rw = (R + 31) & ~31;
+    for (int j = threadIdx.x; j < Rw; j += blockDim.x) {
+      bool f = false;
+      if (j < R) {
+        const unsigned long long kj = keys[j];
+        int rank = 0;
+#pragma unroll 4
+        for (int i = 0; i + 1 < R; i += 2) {
+          const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(keys + i);
+          rank += (kk.x < kj) + (kk.y < kj);
+        }
+        if (R & 1) rank += (keys[R - 1] < kj);
+        f = rank < ksel;
+      }
+      const unsigned bal = __ballot_sync(0xffffffffu, f);
+      if ((threadIdx.x & 31) == 0) words[j >> 5] = bal;
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < R; j += blockDim.x) {
+      const unsigned wj = words[j >> 5];
+      int r = -1;
+      if ((wj >> (j & 31)) & 1u) {
+        r = __popc(wj & ((1u << (j & 31)) - 1u));
+        for (int w = 0; w < (j >> 5); ++w) r += __popc(words[w]);
+      }
+      slot[j] = r;
+    }
+  }
+  __syncthreads();
+  if (write) {
+    for (int j = threadIdx.x; j < R; j += blockDim.x) {
+      const int r = slot[j];
+      inv[(size_t)b * R + j] = r >= 0 ? b * a_seq + np + r : -1;
+      if (r >= 0) {
+        sel[(size_t)b * R + r] = j;
+        act[(size_t)b * a_seq + np + r] = b * R + j;
+      }
+    }
+    for (int i = threadIdx.x; i < np; i += blockDim.x) {
+      act[(size_t)b * a_seq + i] = g.B * R + b * g.P + i;
+      inv[(size_t)g.B * R + (size_t)b * g.P + i] = b * a_seq + i;
+    }
+  }
+  __syncthreads();
+  return slot;
+}
+
 // ------------------------------------------------------------------ V-verify (Eq. 6) + V overwrite
 // metric 0: cosine (Eq. 6); 1: negated Euclidean distance (Sec. A.6), so that the
 // least similar rows have the lowest score either way.  write_v 0: the cache is
 // left as it is (the selected-only variant of Sec. A.5 writes the selected rows later).
 template <typename T>
-__global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restrict__ sim, Geo g, int dkv, int metric,
-                               int write_v) {
+__global__ void __launch_bounds__(512, 2) vverify_kernel(Partials part, T* __restrict__ Vc, float* __restrict__ sim,
+                                                         Geo g, int dkv, int metric, int write_v, SelectArgs sa) {
   pdl_wait();
   pdl_trigger();
-  __shared__ float red[32];
+  __shared__ float red[96];
   const int c = blockIdx.x;  // response row, carried order
   const int b = c / g.R, j = c - b * g.R;
   T* vrow = Vc + ((size_t)b * g.n + g.P + j) * dkv;
@@ -146,19 +222,31 @@ __global__ void vverify_kernel(Partials part, T* __restrict__ Vc, float* __restr
     }
     if (write_v) Vec8<T>::store(vrow + i, vn);
   }
-  dot = block_sum(dot, red);
-  if (metric == 0) {
-    na = block_sum(na, red);
-    nb = block_sum(nb, red);
-  }
+  block_sum3(dot, na, nb, red);
   if (threadIdx.x == 0) sim[c] = metric == 0 ? dot / fmaxf(sqrtf(na * nb), 1e-8f) : -sqrtf(dot);
+  if (sa.counter == nullptr) return;
+  // The CTA that finishes a sequence's last row selects that sequence's rows (Sec. 3.2.2) and writes the
+  // active list, so no launch of its own stands between the scores and the projection of the selected rows.
+  __shared__ int last;
+  if (threadIdx.x == 0) {
+    __threadfence();  // this row's score before the ticket
+    last = atomicAdd(sa.counter + b, 1) == g.R - 1;
+    if (last) sa.counter[b] = 0;  // ready for the next launch; nobody else touches it any more
+  }
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
+  extern __shared__ unsigned long long keys[];
+  select_sequence(keys, sim, sa.forced, sa.mode, sa.ksel, sa.sel, sa.act, sa.inv, g, sa.np, b, true);
 }
 
 void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv, int metric,
-                    int write_v) {
+                    int write_v, const SelectArgs* select) {
   const int rows = g.B * g.R;
-  DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(256), 0, part, (T*)Vc_layer, sim, g, dkv,
-                                 metric, write_v)));
+  const SelectArgs sa = select ? *select : SelectArgs{};
+  const size_t smem = select ? (size_t)g.R * 13 + 16 : 0;
+  DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(row_threads(dkv)), smem, part, (T*)Vc_layer, sim, g,
+                                 dkv, metric, write_v, sa)));
   L.count();
 }
 
@@ -444,14 +532,18 @@ __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__
   extern __shared__ float hrow[];
   __shared__ float red[32];
   const int r = blockIdx.x;
+  const int d = g.d;
+  const bool one_trip = d <= (int)blockDim.x * 8;  // the row fits one pass: it stays in registers
+  const int i0 = threadIdx.x * 8;
+  float hv[8], gv[8];
+  if (one_trip && i0 < d) Vec8<float>::load(gain2 + i0, gv);  // independent of the row: ahead of the dependent loads
   const int c = act[r];
   int b, pos;
   carried_to_pos(c, g, b, pos);
-  const int d = g.d;
   T* arow = Ac + ((size_t)b * g.n + pos) * d;
   const float* xr = x + (size_t)c * d;
   float ss = 0.f;
-  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
+  for (int i = i0; i < d; i += blockDim.x * 8) {
     float a[8], xv[8];
     sum_partials8(part.p, part.split_stride, part.count(r, i), (size_t)r * part.N + i, a);
     Vec8<float>::load(xr + i, xv);
@@ -460,15 +552,24 @@ __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__
       a[t] = Vec8<T>::round(a[t]);
       xv[t] += a[t];
       ss += xv[t] * xv[t];
+      hv[t] = xv[t];
     }
     Vec8<T>::store(arow + i, a);
-    Vec8<float>::store(hrow + i, xv);
+    if (!one_trip) Vec8<float>::store(hrow + i, xv);
   }
   ss = block_sum(ss, red);
   const float rs = rsqrtf(ss / (float)d + eps);
   T* out = hn + (size_t)r * d;
-  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
-    float v[8], gv[8];
+  if (one_trip) {
+    if (i0 < d) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) hv[t] = hv[t] * rs * gv[t];
+      Vec8<T>::store(out + i0, hv);
+    }
+    return;
+  }
+  for (int i = i0; i < d; i += blockDim.x * 8) {
+    float v[8];
     Vec8<float>::load(hrow + i, v);
     Vec8<float>::load(gain2 + i, gv);
 #pragma unroll
@@ -480,8 +581,9 @@ __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__
 void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int32_t* act, const float* x,
                            const float* gain2, void* Ac_layer, void* hn, Geo g, int Ma, float eps) {
   if (Ma <= 0) return;
-  const size_t smem = (size_t)g.d * sizeof(float);
-  DLLM_DISPATCH(dtype, (launch_k(L, oproj_epilogue_kernel<T>, dim3(Ma), dim3(256), smem, part, act, x, gain2, (T*)Ac_layer,
+  const int threads = row_threads(g.d);
+  const size_t smem = g.d <= threads * 8 ? 0 : (size_t)g.d * sizeof(float);  // staging only if a row takes several passes
+  DLLM_DISPATCH(dtype, (launch_k(L, oproj_epilogue_kernel<T>, dim3(Ma), dim3(threads), smem, part, act, x, gain2, (T*)Ac_layer,
                                                                             (T*)hn, g, eps)));
   L.count();
 }
@@ -593,7 +695,7 @@ void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t*
 // (Sec. 3.2 item (3)); u = rmsnorm(x) * gain, the next layer's first norm (the
 // final norm after the last layer).  inv == nullptr: no row is active.
 template <typename T>
-__global__ void tail_kernel(Partials part, const int32_t* __restrict__ inv, float* __restrict__ x,
+__global__ void __launch_bounds__(512, 2) tail_kernel(Partials part, const int32_t* __restrict__ inv, float* __restrict__ x,
                             const T* __restrict__ Ac, T* __restrict__ Fc, const float* __restrict__ gain,
                             T* __restrict__ u, Geo g, int c0, float eps) {
   pdl_wait();
@@ -605,10 +707,14 @@ __global__ void tail_kernel(Partials part, const int32_t* __restrict__ inv, floa
   carried_to_pos(c, g, b, pos);
   const int d = g.d;
   const size_t crow = ((size_t)b * g.n + pos) * d;
+  const bool one_trip = d <= (int)blockDim.x * 8;  // the row fits one pass: it stays in registers
+  const int i0 = threadIdx.x * 8;
+  float hv[8], gv[8];
+  if (one_trip && i0 < d) Vec8<float>::load(gain + i0, gv);
   const int r = inv ? inv[c] : -1;
   float* xr = x + (size_t)c * d;
   float ss = 0.f;
-  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
+  for (int i = i0; i < d; i += blockDim.x * 8) {
     float xv[8], a[8], f[8];
     Vec8<float>::load(xr + i, xv);
     Vec8<T>::load(Ac + crow + i, a);
@@ -624,15 +730,24 @@ __global__ void tail_kernel(Partials part, const int32_t* __restrict__ inv, floa
     for (int t = 0; t < 8; ++t) {
       xv[t] = (xv[t] + a[t]) + f[t];
       ss += xv[t] * xv[t];
+      hv[t] = xv[t];
     }
     Vec8<float>::store(xr + i, xv);
-    Vec8<float>::store(hrow + i, xv);
+    if (!one_trip) Vec8<float>::store(hrow + i, xv);
   }
   ss = block_sum(ss, red);
   const float rs = rsqrtf(ss / (float)d + eps);
   T* orow = u + (size_t)c * d;
-  for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
-    float v[8], gv[8];
+  if (one_trip) {
+    if (i0 < d) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) hv[t] = hv[t] * rs * gv[t];
+      Vec8<T>::store(orow + i0, hv);
+    }
+    return;
+  }
+  for (int i = i0; i < d; i += blockDim.x * 8) {
+    float v[8];
     Vec8<float>::load(hrow + i, v);
     Vec8<float>::load(gain + i, gv);
 #pragma unroll
@@ -644,8 +759,9 @@ __global__ void tail_kernel(Partials part, const int32_t* __restrict__ inv, floa
 void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, const void* Ac_layer,
                  void* Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps) {
   if (c1 <= c0) return;
-  const size_t smem = (size_t)g.d * sizeof(float);
-  DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T>, dim3(c1 - c0), dim3(256), smem, part, inv, x, (const T*)Ac_layer,
+  const int threads = row_threads(g.d);
+  const size_t smem = g.d <= threads * 8 ? 0 : (size_t)g.d * sizeof(float);  // staging only if a row takes several passes
+  DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T>, dim3(c1 - c0), dim3(threads), smem, part, inv, x, (const T*)Ac_layer,
                                  (T*)Fc_layer, gain, (T*)u, g, c0, eps)));
   L.count();
 }
@@ -654,9 +770,9 @@ void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, 
 // grid (a_seq, B): CTA (i, b) produces row i of sequence b's active list and
 // copies that row of u into ua.  Rows below the prompt length (on a prompt
 // refresh) are the prompt rows; the others are the selected response rows, for
-// which every CTA repeats the bottom-k selection of its sequence (R <= 1024,
-// R^2 comparisons out of shared memory) instead of waiting for another launch.
-// CTA (0, b) writes the index list, the active list and its inverse.
+// which every CTA repeats the bottom-k selection of its sequence instead of
+// waiting for another launch.  CTA (0, b) writes the index list, the active
+// list and its inverse.
 template <typename T>
 __global__ void select_gather_kernel(const float* __restrict__ sim, const int32_t* __restrict__ forced, int mode,
                                      int ksel, int32_t* __restrict__ sel, int32_t* __restrict__ act,
@@ -664,65 +780,17 @@ __global__ void select_gather_kernel(const float* __restrict__ sim, const int32_
                                      int refresh_prompt) {
   pdl_wait();
   pdl_trigger();
-  extern __shared__ unsigned long long keys[];  // R keys, R slots (int), R flags (bytes)
+  extern __shared__ unsigned long long keys[];  // R keys, R slots (int), R / 8 bytes of ballot words
   const int R = g.R, b = blockIdx.y, ridx = blockIdx.x;
-  int32_t* slot = reinterpret_cast<int32_t*>(keys + R);
-  unsigned char* flag = reinterpret_cast<unsigned char*>(slot + R);
   __shared__ int my_j;
   const int np = refresh_prompt ? g.P : 0;
   const int a_seq = np + ksel;
   const bool leader = ridx == 0;
   if (ridx >= np || leader) {
-    if (mode == 0) {
-      for (int j = threadIdx.x; j < R; j += blockDim.x) slot[j] = j;
-    } else if (mode == 2) {
-      for (int j = threadIdx.x; j < R; j += blockDim.x) slot[j] = -1;
-      __syncthreads();
-      for (int r = threadIdx.x; r < ksel; r += blockDim.x) slot[forced[(size_t)b * R + r]] = r;
-    } else {
-      for (int j = threadIdx.x; j < R; j += blockDim.x) {
-        const float s = sim[(size_t)b * R + j];
-        // key = round(s * 2^20), offset into 1 .. 2^32 - 1 (scores beyond +-2047 saturate); NaN sorts first
-        const float qf = fminf(fmaxf(rintf(s * 1048576.0f), -2147483520.0f), 2147483520.0f);
-        const long long q = (s == s) ? (long long)qf + (1ll << 31) : 0ll;
-        keys[j] = ((unsigned long long)q << 32) | (unsigned)j;
-      }
-      __syncthreads();
-      for (int j = threadIdx.x; j < R; j += blockDim.x) {
-        const unsigned long long kj = keys[j];
-        int rank = 0;
-        for (int i = 0; i < R; ++i) rank += (keys[i] < kj);
-        flag[j] = (rank < ksel);
-      }
-      __syncthreads();
-      for (int j = threadIdx.x; j < R; j += blockDim.x) {
-        int r = -1;
-        if (flag[j]) {
-          r = 0;
-          for (int i = 0; i < j; ++i) r += flag[i];
-        }
-        slot[j] = r;
-      }
-    }
-    __syncthreads();
-    // slot[j]: position of response row j among the selected rows, or -1
+    const int32_t* slot = select_sequence(keys, sim, forced, mode, ksel, sel, act, inv, g, np, b, leader);
     if (ridx >= np)
       for (int j = threadIdx.x; j < R; j += blockDim.x)
         if (slot[j] == ridx - np) my_j = j;
-    if (leader) {
-      for (int j = threadIdx.x; j < R; j += blockDim.x) {
-        const int r = slot[j];
-        inv[(size_t)b * R + j] = r >= 0 ? b * a_seq + np + r : -1;
-        if (r >= 0) {
-          sel[(size_t)b * R + r] = j;
-          act[(size_t)b * a_seq + np + r] = b * R + j;
-        }
-      }
-      for (int i = threadIdx.x; i < np; i += blockDim.x) {
-        act[(size_t)b * a_seq + i] = g.B * R + b * g.P + i;
-        inv[(size_t)g.B * R + (size_t)b * g.P + i] = b * a_seq + i;
-      }
-    }
     __syncthreads();
   }
   const int c = ridx < np ? g.B * R + b * g.P + ridx : b * R + my_j;
