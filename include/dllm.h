@@ -252,15 +252,6 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
 size_t dllm_gemm_bf16_planned_scratch_bytes(int M, int N, int K, int act_tile, int splits);
 dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
                                    int splits, int stages, void* d_partials, size_t partials_bytes, void* stream);
-/* The projection of a SUBSET of rows, the selected rows of Sec. 3.2.2, without
- * copying them first: C[M,N] = A[rows[i], :] * W^T, where d_src is a bf16
- * matrix [src_rows, K] (DEVICE) and d_rows holds M int32 row numbers (DEVICE,
- * each in 0 .. src_rows-1, repeats allowed; not checked).  The rows are
- * fetched by TMA row gathers.  Scratch as for dllm_gemm_bf16_planned with
- * splits = 0 (dllm_gemm_bf16_planned_scratch_bytes(M, N, K, act_tile, 0)). */
-dllm_status dllm_gemm_bf16_gathered(const void* d_src, int src_rows, const int32_t* d_rows, const void* d_W, float* d_C,
-                                    int M, int N, int K, int act_tile, void* d_partials, size_t partials_bytes,
-                                    void* stream);
 /* Gate and up projection of the SwiGLU FFN with the activation applied in the
  * GEMM's epilogue (Sec. A.7's FFN: two of its three d x d_ffn products):
  * out[M, d_ffn] (bf16, DEVICE) = silu(A Wg^T) * (A Wu^T), A [M, K] bf16,

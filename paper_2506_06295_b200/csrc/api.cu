@@ -125,7 +125,7 @@ uint16_t f32_to_bf16_rne(float f) {
 
 // workspace carve-up
 struct Workspace {
-  size_t status, tokens, x, u, ua, qbuf, obuf, hn, ffn, x0, conf, sim, sel, forced, act, inv, selcnt, mkbar, mkmaps, rope, attn, part,
+  size_t status, tokens, x, u, ua, qbuf, obuf, hn, ffn, x0, conf, sim, sel, forced, act, inv, mkbar, mkmaps, rope, attn, part,
       total;
   size_t part_floats, attn_floats;
 };
@@ -157,7 +157,6 @@ Workspace make_workspace(const dllm_config& c, int B, int P, int R) {
   w.forced = take(T * BR * 4);
   w.act = take(rows * 4);
   w.inv = take(rows * 4);
-  w.selcnt = take((size_t)B * 4);  // tickets of the selection fused into V-verify (zero between launches)
   w.mkbar = take((1 + 13 * T) * 4);  // one grid-barrier counter per phase of the persistent layer kernel
   w.mkmaps = take((size_t)7 * T * sizeof(CUtensorMap));
   w.rope = take(n * c.head_dim * 4);
@@ -314,8 +313,7 @@ int k_selected(float rho, int R, dllm_kround kr) {
 
 // One GEMM of the step: out = A[M,K] * W[N,K]^T as split-K partial slabs.
 dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void* W, int M, int N, int K,
-                     Partials* out, void* swiglu_out = nullptr, bool* fused = nullptr,
-                     const int32_t* gather_idx = nullptr, int src_rows = 0) {
+                     Partials* out, void* swiglu_out = nullptr, bool* fused = nullptr) {
   float* part = s->wsp<float>(s->ws.part);
   if (fused) *fused = false;
   *out = Partials{part, (size_t)M * N, 1, N};
@@ -339,8 +337,7 @@ dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void
   const char* why = nullptr;
   // an unsplit gate / up projection of an interleaved weight finishes SwiGLU in its own epilogue
   const bool fuse = swiglu_out && plan.S_max == 1 && gu_interleaved(s->m->cfg);
-  cudaError_t e = launch_gemm_bf16(L, A, W, part, M, N, K, plan, &why, fuse ? swiglu_out : nullptr, fuse ? N / 2 : 0,
-                                   gather_idx, src_rows);
+  cudaError_t e = launch_gemm_bf16(L, A, W, part, M, N, K, plan, &why, fuse ? swiglu_out : nullptr, fuse ? N / 2 : 0);
   if (e != cudaSuccess)
     return fail(&s->err, DLLM_CUDA_ERROR, "bf16 GEMM %dx%dx%d: %s", M, N, K, why ? why : cudaGetErrorString(e));
   if (fused) *fused = fuse;
@@ -483,21 +480,15 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
     const int Ma = s->B * a_seq;
     const bool adaptive = !rr && ksel > 0;
     const int mode = rr ? 0 : (s->forced_count[l] >= 0 ? 2 : 1);
-    // On the tensor-core path the projections of the active rows fetch them from u by TMA row gathers, and the
-    // V-verify launch selects them itself: no selection or gather launch in between.
-    const bool gathered = dt == DLLM_BF16 && !s->simt_gemm && s->R <= 1024 && Ma > 0;
-    bool selected = false;
+    // A response refresh alone takes every response row in carried order: u itself is the operand of the
+    // projections and V-verify writes the (identity) lists, so no selection or gather launch is needed.
+    const bool identity = rr && !rp && Ma > 0;
     if (rr || (adaptive && s->sel_strategy == DLLM_SELECT_V_VERIFY)) {
       // V for ALL response rows (the 2 r d^2 term of Sec. A.7), V-verify, V overwrite
       if ((st = run_gemm(s, L, u, Wv, BR, dkv, d, &part)) != DLLM_OK) return st;
-      SelectArgs sa;
-      sa.counter = s->wsp<int32_t>(s->ws.selcnt);
-      sa.forced = forced;
-      sa.mode = mode; sa.ksel = ksel; sa.np = rp ? s->P : 0;
-      sa.sel = sel; sa.act = act; sa.inv = inv;
+      const IdentityLists id{sel, act, inv};
       launch_vverify(L, dt, part, s->cache(l, DLLM_CACHE_V), sim, g, dkv, rr ? 0 : s->sel_metric,
-                     rr || !s->v_selected_only, gathered ? &sa : nullptr);
-      selected = gathered;
+                     rr || !s->v_selected_only, identity ? &id : nullptr);
     } else if (adaptive && s->sel_strategy == DLLM_SELECT_K_VERIFY) {
       // ablation: the same test on K; K of ALL response rows is projected, rotated and overwritten
       if ((st = run_gemm(s, L, u, Wq + (size_t)dq * d * es, BR, dkv, d, &part)) != DLLM_OK) return st;
@@ -512,24 +503,20 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
     }
     if (Ma > 0) {
       const uint8_t* ua = s->wsp<uint8_t>(s->ws.ua);
-      const int32_t* gidx = nullptr;
-      if (gathered) {
-        if (!selected) launch_select(L, sim, forced, mode, ksel, sel, s->R, act, inv, g, rp);
+      if (identity) {
         ua = u;
-        gidx = act;
       } else if (s->R <= 1024) {
         launch_select_gather(L, dt, sim, forced, mode, ksel, sel, act, inv, u, s->wsp<uint8_t>(s->ws.ua), g, rp);
       } else {
         launch_select(L, sim, forced, mode, ksel, sel, s->R, act, inv, g, rp);
         launch_gather_rows(L, dt, u, act, s->wsp<uint8_t>(s->ws.ua), Ma, d);
       }
-      const int src_rows = s->B * s->n;
       if (v_for_active) {
-        if ((st = run_gemm(s, L, ua, Wv, Ma, dkv, d, &part, nullptr, nullptr, gidx, src_rows)) != DLLM_OK) return st;
+        if ((st = run_gemm(s, L, ua, Wv, Ma, dkv, d, &part)) != DLLM_OK) return st;
         launch_scatter_rows(L, dt, part, act, 0, s->cache(l, DLLM_CACHE_V), g, Ma, dkv);
       }
       // Q and K of the active rows in one GEMM over the stacked [W_q; W_k]
-      if ((st = run_gemm(s, L, ua, Wq, Ma, dq + dkv, d, &part, nullptr, nullptr, gidx, src_rows)) != DLLM_OK) return st;
+      if ((st = run_gemm(s, L, ua, Wq, Ma, dq + dkv, d, &part)) != DLLM_OK) return st;
       launch_qk_rope(L, dt, part, act, s->wsp<float>(s->ws.rope), s->wsp<uint8_t>(s->ws.qbuf),
                      s->cache(l, DLLM_CACHE_K), g, Ma, H, Hkv, hd);
       // algorithmic traffic: K and V of every sequence once, Q in, O out
@@ -1129,27 +1116,6 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
   float* part = p.S_max > 1 ? static_cast<float*>(d_partials) : d_C;
   const char* why = nullptr;
   cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
-  if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "bf16 GEMM: %s", why ? why : cudaGetErrorString(e));
-  if (p.S_max > 1) launch_reduce_partials(L, make_partials(part, M, N, p), d_C, M);
-  CU_TRY(nullptr, cudaGetLastError());
-  return DLLM_OK;
-}
-
-dllm_status dllm_gemm_bf16_gathered(const void* d_src, int src_rows, const int32_t* d_rows, const void* d_W, float* d_C,
-                                    int M, int N, int K, int act_tile, void* d_partials, size_t partials_bytes,
-                                    void* stream) {
-  if (!d_src || !d_rows || !d_W || !d_C || src_rows <= 0 || M <= 0 || N <= 0 || K <= 0)
-    return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
-  if (K % 8) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8");
-  if (act_tile < 0 || (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 256))
-    return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128 or 256");
-  const GemmPlan p = plan_gemm_bf16(M, N, K, 0, 0, act_tile);
-  if (p.S_max > 1 && (!d_partials || partials_bytes < (size_t)p.S_max * M * N * 4))
-    return fail(nullptr, DLLM_INVALID_ARG, "this plan needs %zu bytes of slab scratch", (size_t)p.S_max * M * N * 4);
-  Launch L{(cudaStream_t)stream, nullptr, nullptr};
-  float* part = p.S_max > 1 ? static_cast<float*>(d_partials) : d_C;
-  const char* why = nullptr;
-  cudaError_t e = launch_gemm_bf16(L, d_src, d_W, part, M, N, K, p, &why, nullptr, 0, d_rows, src_rows);
   if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "bf16 GEMM: %s", why ? why : cudaGetErrorString(e));
   if (p.S_max > 1) launch_reduce_partials(L, make_partials(part, M, N, p), d_C, M);
   CU_TRY(nullptr, cudaGetLastError());

@@ -196,7 +196,7 @@ __device__ __forceinline__ int32_t* select_sequence(unsigned long long* keys, co
 // left as it is (the selected-only variant of Sec. A.5 writes the selected rows later).
 template <typename T>
 __global__ void __launch_bounds__(512, 2) vverify_kernel(Partials part, T* __restrict__ Vc, float* __restrict__ sim,
-                                                         Geo g, int dkv, int metric, int write_v, SelectArgs sa) {
+                                                         Geo g, int dkv, int metric, int write_v, IdentityLists id) {
   pdl_wait();
   pdl_trigger();
   __shared__ float red[96];
@@ -224,29 +224,20 @@ __global__ void __launch_bounds__(512, 2) vverify_kernel(Partials part, T* __res
   }
   block_sum3(dot, na, nb, red);
   if (threadIdx.x == 0) sim[c] = metric == 0 ? dot / fmaxf(sqrtf(na * nb), 1e-8f) : -sqrtf(dot);
-  if (sa.counter == nullptr) return;
-  // The CTA that finishes a sequence's last row selects that sequence's rows (Sec. 3.2.2) and writes the
-  // active list, so no launch of its own stands between the scores and the projection of the selected rows.
-  __shared__ int last;
-  if (threadIdx.x == 0) {
-    __threadfence();  // this row's score before the ticket
-    last = atomicAdd(sa.counter + b, 1) == g.R - 1;
-    if (last) sa.counter[b] = 0;  // ready for the next launch; nobody else touches it any more
+  // a response refresh recomputes every response row, in carried order: the lists are the identity
+  if (id.act && threadIdx.x == 0) {
+    id.sel[c] = j;
+    id.act[c] = c;
+    id.inv[c] = c;
   }
-  __syncthreads();
-  if (!last) return;
-  __threadfence();
-  extern __shared__ unsigned long long keys[];
-  select_sequence(keys, sim, sa.forced, sa.mode, sa.ksel, sa.sel, sa.act, sa.inv, g, sa.np, b, true);
 }
 
 void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv, int metric,
-                    int write_v, const SelectArgs* select) {
+                    int write_v, const IdentityLists* lists) {
   const int rows = g.B * g.R;
-  const SelectArgs sa = select ? *select : SelectArgs{};
-  const size_t smem = select ? (size_t)g.R * 13 + 16 : 0;
-  DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(row_threads(dkv)), smem, part, (T*)Vc_layer, sim, g,
-                                 dkv, metric, write_v, sa)));
+  const IdentityLists id = lists ? *lists : IdentityLists{};
+  DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(row_threads(dkv)), 0, part, (T*)Vc_layer, sim, g, dkv,
+                                 metric, write_v, id)));
   L.count();
 }
 

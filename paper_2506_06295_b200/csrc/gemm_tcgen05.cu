@@ -60,7 +60,6 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
                                                                 float* __restrict__ part, int M, int N, int num_kb,
                                                                 int kb_per_split, size_t split_stride, int STAGES,
                                                                 __nv_bfloat16* __restrict__ act_out, int m_ffn,
-                                                                const int32_t* __restrict__ gather_idx,
                                                                 int* __restrict__ status) {
   using SL = SmemLayout<BN>;
   extern __shared__ uint8_t smem_raw[];
@@ -69,7 +68,6 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   __shared__ __align__(8) uint64_t accum_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag;
-  __shared__ int32_t grow[BN];  // source rows of this activation tile (gathered operand only)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * BN;       // activation rows
@@ -111,10 +109,6 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   volatile int* abortp = &abort_flag;
   pdl_wait();     // the activation rows and the slab buffer belong to the preceding kernels
   pdl_trigger();
-  if (warp == 0 && gather_idx) {  // rows past the end repeat the last one: their outputs are never written
-    for (int i = lane; i < BN; i += 32) grow[i] = __ldcg(gather_idx + min(m0 + i, M - 1));
-    __syncwarp();
-  }
 
   if (warp == 0 && lane == 0) {
     // ---------------- TMA producer ----------------
@@ -132,14 +126,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
         mbar_expect_tx(fb, SL::STAGE_BYTES);
         tma_load_2d(dstW, &tmW, fb, kc, n0);
       }
-      if (gather_idx) {
-#pragma unroll 4
-        for (int q = 0; q < BN / 4; ++q)
-          tma_gather4_2d(dstW + W_STAGE_BYTES + q * 512, &tmA, fb, kc, grow[4 * q], grow[4 * q + 1], grow[4 * q + 2],
-                         grow[4 * q + 3]);
-      } else {
-        tma_load_2d(dstW + W_STAGE_BYTES, &tmA, fb, kc, m0);
-      }
+      tma_load_2d(dstW + W_STAGE_BYTES, &tmA, fb, kc, m0);
       if (++s == STAGES) {
         s = 0;
         ph ^= 1u;
@@ -319,7 +306,7 @@ constexpr int max_stages(int bn) {
 
 template <int BN>
 cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMap& tmA, float* part, int M, int N,
-                       int num_kb, const GemmPlan& plan, void* act_out, int m_ffn, const int32_t* gather_idx) {
+                       int num_kb, const GemmPlan& plan, void* act_out, int m_ffn) {
   using SL = SmemLayout<BN>;
   static bool configured = false;
   if (!configured) {
@@ -331,7 +318,7 @@ cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMa
   const int stages = plan.stages < 2 ? 2 : plan.stages > max_stages(BN) ? max_stages(BN) : plan.stages;
   dim3 grid((M + BN - 1) / BN, (N + TILE_W - 1) / TILE_W, plan.S_max);
   cudaError_t e = launch_k(L, gemm_bf16_tcgen05_kernel<BN>, grid, dim3(128), SL::total(stages), tmW, tmA, part, M, N,
-                           num_kb, plan.upc, (size_t)M * N, stages, (__nv_bfloat16*)act_out, m_ffn, gather_idx, L.d_status);
+                           num_kb, plan.upc, (size_t)M * N, stages, (__nv_bfloat16*)act_out, m_ffn, L.d_status);
   L.count();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -390,8 +377,7 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
 }
 
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
-                             const GemmPlan& plan, const char** err, void* act_out, int m_ffn,
-                             const int32_t* gather_idx, int src_rows) {
+                             const GemmPlan& plan, const char** err, void* act_out, int m_ffn) {
   static const char* e_shape = "bf16 GEMM needs K % 8 == 0 and 16-byte aligned operands";
   static const char* e_map = "cuTensorMapEncodeTiled failed or is unavailable";
   if (M <= 0 || N <= 0) return cudaSuccess;
@@ -405,17 +391,16 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
   }
   CUtensorMap tmW, tmA;
   if (!get_tensor_map_2d(W, (uint64_t)N, (uint64_t)K, TILE_W, &tmW) ||
-      !(gather_idx ? get_tensor_map_2d(A, (uint64_t)src_rows, (uint64_t)K, 1, &tmA)
-                   : get_tensor_map_2d(A, (uint64_t)M, (uint64_t)K, (uint32_t)plan.BN, &tmA))) {
+      !get_tensor_map_2d(A, (uint64_t)M, (uint64_t)K, (uint32_t)plan.BN, &tmA)) {
     if (err) *err = e_map;
     return cudaErrorInvalidValue;
   }
   const int num_kb = (K + TILE_K - 1) / TILE_K;
   switch (plan.BN) {
-    case 32: return launch_one<32>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn, gather_idx);
-    case 64: return launch_one<64>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn, gather_idx);
-    case 128: return launch_one<128>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn, gather_idx);
-    default: return launch_one<256>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn, gather_idx);
+    case 32: return launch_one<32>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
+    case 64: return launch_one<64>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
+    case 128: return launch_one<128>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
+    default: return launch_one<256>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
   }
 }
 

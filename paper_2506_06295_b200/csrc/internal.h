@@ -72,17 +72,13 @@ void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gai
 // V-verify (Eq. 6) fused with the whole-V overwrite: for every response row
 // sums the partials, rounds to the cache dtype, takes the cosine against the
 // cached row, overwrites the cached row, writes sim[row].
-// Selection fused into the V-verify launch: the CTA that completes a sequence's scores (a ticket per sequence in
-// `counter`, B zero-initialised ints that the kernel resets) writes the index list, the active list (np prompt
-// rows first) and its inverse.  R <= 1024.
-struct SelectArgs {
-  int32_t* counter = nullptr;
-  const int32_t* forced = nullptr;
-  int mode = 0, ksel = 0, np = 0;
+// Lists of a response refresh without prompt refresh, where every response row is active in carried order:
+// V-verify writes sel[c] = row within the sequence, act[c] = c, inv[c] = c for its row c.
+struct IdentityLists {
   int32_t *sel = nullptr, *act = nullptr, *inv = nullptr;
 };
 void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv,
-                    int metric = 0, int write_v = 1, const SelectArgs* select = nullptr);
+                    int metric = 0, int write_v = 1, const IdentityLists* lists = nullptr);
 // The same test on K (ablation of Sec. 4.3): slab sum of the K projection of all
 // response rows, RoPE, score against the cached (post-RoPE) K, whole-K overwrite.
 void launch_kverify(const Launch& L, int dtype, Partials part, void* Kc_layer, float* sim, const float* rope_tab, Geo g,
@@ -155,11 +151,8 @@ Partials make_partials(const float* p, int M, int N, const GemmPlan& plan);
 // Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
 // act_out != nullptr (unsplit plan, W = gate / up rows interleaved in blocks of 64, N = 2 * m_ffn): instead of
 // fp32 slabs the epilogue writes silu(gate) * up as bf16 [M, m_ffn].
-// gather_idx != nullptr (device, M entries < src_rows): row i of the activation operand is row gather_idx[i] of
-// A [src_rows, K], fetched by TMA row gathers.
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
-                             const GemmPlan& plan, const char** err, void* act_out = nullptr, int m_ffn = 0,
-                             const int32_t* gather_idx = nullptr, int src_rows = 0);
+                             const GemmPlan& plan, const char** err, void* act_out = nullptr, int m_ffn = 0);
 
 // ---------------- megakernel.cu ----------------
 // One projection inside the persistent layer kernel: units (tile, k-block) in

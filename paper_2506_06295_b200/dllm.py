@@ -79,7 +79,6 @@ SIGNATURES = {
     "dllm_gemm_bf16": (_I, [_P, _P, _P, _I, _I, _I, _P, _P]),
     "dllm_gemm_bf16_planned_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I]),
     "dllm_gemm_bf16_planned": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
-    "dllm_gemm_bf16_gathered": (_I, [_P, _I, _P, _P, _P, _I, _I, _I, _I, _P, _SZ, _P]),
     "dllm_ffn_gate_up_bf16": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _P]),
     "dllm_gemm_simt": (_I, [_P, _P, _P, _I, _I, _I, _I, _P]),
     "dllm_attention_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I, _I, _I]),
@@ -397,21 +396,6 @@ def gemm_bf16_planned(A, W, act_tile=0, splits=0, stages=0, out=None, scratch=No
     _check(lib.dllm_gemm_bf16_planned(C.c_void_p(A.data_ptr()), C.c_void_p(W.data_ptr()), C.c_void_p(cptr),
                                       M, N, K, act_tile, splits, stages, C.c_void_p(scratch.data_ptr()),
                                       scratch.numel(), C.c_void_p(sp)))
-    return Cm
-
-
-def gemm_bf16_gathered(src, rows, W, act_tile=0, stream=None):
-    """C = src[rows] @ W.T: src [src_rows, K] bf16, rows int32 [M] (device), W [N, K] bf16; returns fp32 [M, N]."""
-    import torch
-    M, K = rows.numel(), src.shape[1]
-    N = W.shape[0]
-    Cm = torch.empty((M, N), dtype=torch.float32, device=src.device)
-    sb = lib.dllm_gemm_bf16_planned_scratch_bytes(M, N, K, act_tile, 0)
-    scratch = torch.empty(max(sb, 16), dtype=torch.uint8, device=src.device)
-    sp = _stream_ptr(stream if stream is not None else torch.cuda.current_stream(src.device))
-    _check(lib.dllm_gemm_bf16_gathered(C.c_void_p(src.data_ptr()), src.shape[0], C.c_void_p(rows.data_ptr()),
-                                       C.c_void_p(W.data_ptr()), C.c_void_p(Cm.data_ptr()), M, N, K, act_tile,
-                                       C.c_void_p(scratch.data_ptr()), scratch.numel(), C.c_void_p(sp)))
     return Cm
 
 

@@ -98,29 +98,6 @@ def test_ffn_gate_up_epilogue(env, M, m, K, act_tile):
     assert dllm.lib.dllm_ffn_gate_up_bf16(dA.data_ptr(), dW.data_ptr(), dA.data_ptr(), M, 100, K, 0, 0, None) == dllm.INVALID_ARG
 
 
-@pytest.mark.parametrize("M,N,K,act_tile", [(64, 4096, 4096, 0), (1, 128, 64, 32), (3, 200, 320, 0), (70, 384, 832, 0),
-                                            (150, 256, 448, 128), (300, 128, 192, 256), (45, 640, 1088, 64)])
-def test_gemm_bf16_gathered_rows(env, M, N, K, act_tile):
-    """The projection of selected rows fetched by TMA row gathers equals the product of the copied rows."""
-    torch, dllm = env
-    src_rows = 777
-    src = synth.round_to_bf16(synth.random_normal((src_rows, K), seed=K + 1))
-    W = synth.round_to_bf16(synth.random_normal((N, K), seed=N + 2, std=0.05))
-    rng = np.random.default_rng(M)
-    rows = np.sort(rng.choice(src_rows, size=M, replace=False)).astype(np.int32)
-    if M > 4:
-        rows[1] = rows[0]                   # a repeat, and the last row of the matrix
-        rows[-1] = src_rows - 1
-    d_src = torch.from_numpy(src).cuda().to(torch.bfloat16)
-    dW = torch.from_numpy(W).cuda().to(torch.bfloat16)
-    got = dllm.gemm_bf16_gathered(d_src, torch.from_numpy(rows).cuda(), dW, act_tile).cpu().numpy()
-    want = src[rows].astype(np.float64) @ W.astype(np.float64).T
-    assert rel_l2(got, want) < 2e-6
-    # bit-identical to the same plan run on a contiguous copy of the rows
-    copy = dllm.gemm_bf16_planned(d_src[torch.from_numpy(rows.astype(np.int64)).cuda()].contiguous(), dW, act_tile).cpu().numpy()
-    assert np.array_equal(got, copy)
-
-
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_gemm_simt(env, dtype):
     torch, dllm = env
