@@ -252,6 +252,15 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
 size_t dllm_gemm_bf16_planned_scratch_bytes(int M, int N, int K, int act_tile, int splits);
 dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
                                    int splits, int stages, void* d_partials, size_t partials_bytes, void* stream);
+/* The same product computed by PAIRS of CTAs (tcgen05 cta_group::2): two CTAs
+ * of a cluster share one activation tile of act_tile (128 or 256) rows, each
+ * staging half of it, so the tile crosses the L2 -> SM fabric once per 256
+ * weight rows.  N must be a multiple of 256.  splits / stages / scratch as for
+ * dllm_gemm_bf16_planned; the result is bit-identical to the one-CTA kernel
+ * with the same act_tile and splits. */
+size_t dllm_gemm_bf16_pair_scratch_bytes(int M, int N, int K, int act_tile, int splits);
+dllm_status dllm_gemm_bf16_pair(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
+                                int splits, int stages, void* d_partials, size_t partials_bytes, void* stream);
 /* Gate and up projection of the SwiGLU FFN with the activation applied in the
  * GEMM's epilogue (Sec. A.7's FFN: two of its three d x d_ffn products):
  * out[M, d_ffn] (bf16, DEVICE) = silu(A Wg^T) * (A Wu^T), A [M, K] bf16,

@@ -1165,6 +1165,31 @@ dllm_status dllm_ffn_gate_up_bf16(const void* d_A, const void* d_Wgu, void* d_ou
   return DLLM_OK;
 }
 
+size_t dllm_gemm_bf16_pair_scratch_bytes(int M, int N, int K, int act_tile, int splits) {
+  if (M <= 0 || N <= 0 || K <= 0 || splits < 0 || (act_tile != 128 && act_tile != 256)) return 0;
+  const GemmPlan p = plan_gemm_bf16(M, N, K, splits, 0, act_tile, 1);
+  return p.S_max > 1 ? (size_t)p.S_max * M * N * 4 : 0;
+}
+
+dllm_status dllm_gemm_bf16_pair(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int act_tile,
+                                int splits, int stages, void* d_partials, size_t partials_bytes, void* stream) {
+  if (!d_A || !d_W || !d_C || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
+  if (K % 8 || N % 256) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8 and N of 256");
+  if (splits < 0 || stages < 0 || (act_tile != 128 && act_tile != 256))
+    return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 128 or 256");
+  const GemmPlan p = plan_gemm_bf16(M, N, K, splits, stages, act_tile, 1);
+  if (p.S_max > 1 && (!d_partials || partials_bytes < (size_t)p.S_max * M * N * 4))
+    return fail(nullptr, DLLM_INVALID_ARG, "this plan needs %zu bytes of slab scratch", (size_t)p.S_max * M * N * 4);
+  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  float* part = p.S_max > 1 ? static_cast<float*>(d_partials) : d_C;
+  const char* why = nullptr;
+  cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
+  if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "bf16 GEMM: %s", why ? why : cudaGetErrorString(e));
+  if (p.S_max > 1) launch_reduce_partials(L, make_partials(part, M, N, p), d_C, M);
+  CU_TRY(nullptr, cudaGetLastError());
+  return DLLM_OK;
+}
+
 dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, int N, int K, int dtype,
                            void* stream) {
   if (!d_A || !d_W || !d_C || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");

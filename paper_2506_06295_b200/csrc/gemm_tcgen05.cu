@@ -54,6 +54,73 @@ struct SmemLayout {
   static constexpr uint32_t total(int stages) { return (uint32_t)stages * STAGE_BYTES + 1024; }  // + slack to align the base to 1024
 };
 
+// Epilogue of one CTA (128 threads, all of them): its accumulator, TMEM lanes = 128 weight rows from n0 (tile
+// number tile_y), columns = BN activation rows from m0, goes to the fp32 slab (coalesced: lane = output column)
+// or, with act_out, through the SwiGLU combination.  `ex`: at least min(BN, 64) * 528 bytes of shared memory
+// that nothing else uses any more.
+template <int BN>
+__device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0, int n0, int tile_y, int M, int N,
+                                              float* __restrict__ slab, __nv_bfloat16* __restrict__ act_out, int m_ffn) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (act_out) {
+    // SwiGLU epilogue (no split-K): the tile's 128 weight rows are 64 gate rows followed by the 64 up rows
+    // of the same FFN columns, so TMEM lanes 0..63 hold gate and 64..127 hold up.  The accumulator goes
+    // through shared memory (every MMA has completed) 64 activation rows at a time, transposed to
+    // [row][weight row], and comes back as silu(gate) * up in bf16, 8 bytes per thread.
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    constexpr int EXS = 132;   // floats per staged row: 16-byte aligned, rows 4 banks apart
+    constexpr int CH = BN < 64 ? BN : 64;
+    const int q = threadIdx.x & 15, rsub = threadIdx.x >> 4;  // 4 FFN columns, 8 rows per pass
+    const int col = tile_y * 64 + 4 * q;
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += CH) {
+      if (m0 + c0 >= M) break;  // uniform across the CTA
+#pragma unroll
+      for (int c = 0; c < CH; c += 16) {
+        uint32_t r[16];
+        tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + c), r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[j]);
+      }
+      __syncthreads();
+#pragma unroll
+      for (int rr = rsub; rr < CH; rr += 8) {
+        const int m = m0 + c0 + rr;
+        const float4 gt = *reinterpret_cast<const float4*>(ex + rr * EXS + 4 * q);
+        const float4 up = *reinterpret_cast<const float4*>(ex + rr * EXS + 64 + 4 * q);
+        if (m < M && col < m_ffn) {
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(gt.x / (1.f + expf(-gt.x)) * up.x, gt.y / (1.f + expf(-gt.y)) * up.y);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(gt.z / (1.f + expf(-gt.z)) * up.z, gt.w / (1.f + expf(-gt.w)) * up.w);
+          uint2 pk;
+          pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(act_out + (size_t)m * m_ffn + col) = pk;
+        }
+      }
+      __syncthreads();
+    }
+  } else {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int n = n0 + warp * 32 + lane;
+    float* out = slab + n;
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 16) {
+      if (m0 + c >= M) break;  // uniform across the CTA
+      uint32_t r[16];
+      tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (n < N) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + c + j;
+          if (m < M) out[(size_t)m * N] = __uint_as_float(r[j]);
+        }
+      }
+    }
+  }
+}
+
 template <int BN>
 __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                 const __grid_constant__ CUtensorMap tmA,
@@ -169,63 +236,9 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   // the whole warp must agree before the warp-collective TMEM loads
   bool warp_ok = __all_sync(0xffffffffu, have);
   if (act_out) warp_ok = __syncthreads_and(warp_ok);  // the SwiGLU epilogue exchanges data between warps
-  if (warp_ok && act_out) {
-    // SwiGLU epilogue (no split-K): the tile's 128 weight rows are 64 gate rows followed by the 64 up rows
-    // of the same FFN columns, so TMEM lanes 0..63 hold gate and 64..127 hold up.  The accumulator goes
-    // through shared memory (the ring is drained: every MMA has completed) 64 activation rows at a time,
-    // transposed to [row][weight row], and comes back as silu(gate) * up in bf16, 8 bytes per thread.
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    constexpr int EXS = 132;   // floats per staged row: 16-byte aligned, rows 4 banks apart
-    constexpr int CH = BN < 64 ? BN : 64;
-    float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // [CH][EXS]
-    const int q = threadIdx.x & 15, rsub = threadIdx.x >> 4;  // 4 FFN columns, 8 rows per pass
-    const int col = blockIdx.y * 64 + 4 * q;
-#pragma unroll 1
-    for (int c0 = 0; c0 < BN; c0 += CH) {
-      if (m0 + c0 >= M) break;  // uniform across the CTA
-#pragma unroll
-      for (int c = 0; c < CH; c += 16) {
-        uint32_t r[16];
-        tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + c), r);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-        for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[j]);
-      }
-      __syncthreads();
-#pragma unroll
-      for (int rr = rsub; rr < CH; rr += 8) {
-        const int m = m0 + c0 + rr;
-        const float4 gt = *reinterpret_cast<const float4*>(ex + rr * EXS + 4 * q);
-        const float4 up = *reinterpret_cast<const float4*>(ex + rr * EXS + 64 + 4 * q);
-        if (m < M && col < m_ffn) {
-          const __nv_bfloat162 lo = __floats2bfloat162_rn(gt.x / (1.f + expf(-gt.x)) * up.x, gt.y / (1.f + expf(-gt.y)) * up.y);
-          const __nv_bfloat162 hi = __floats2bfloat162_rn(gt.z / (1.f + expf(-gt.z)) * up.z, gt.w / (1.f + expf(-gt.w)) * up.w);
-          uint2 pk;
-          pk.x = *reinterpret_cast<const uint32_t*>(&lo);
-          pk.y = *reinterpret_cast<const uint32_t*>(&hi);
-          *reinterpret_cast<uint2*>(act_out + (size_t)m * m_ffn + col) = pk;
-        }
-      }
-      __syncthreads();
-    }
-  } else if (warp_ok) {
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const int n = n0 + warp * 32 + lane;
-    float* out = part + (size_t)blockIdx.z * split_stride + n;
-#pragma unroll 1
-    for (int c = 0; c < BN; c += 16) {
-      if (m0 + c >= M) break;  // uniform across the CTA
-      uint32_t r[16];
-      tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      if (n < N) {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int m = m0 + c + j;
-          if (m < M) out[(size_t)m * N] = __uint_as_float(r[j]);
-        }
-      }
-    }
+  if (warp_ok) {
+    float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // the drained ring
+    gemm_epilogue<BN>(tmem_d, ex, m0, n0, (int)blockIdx.y, M, N, part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
   } else {
     drain_delay();  // gave up: let copies in flight land before shared memory is released
   }
@@ -233,6 +246,150 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"((uint32_t)BN) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- CTA-pair kernel
+// The same product with cta_group::2: two CTAs of a cluster (consecutive weight tiles, blockIdx.x = 2p, 2p + 1)
+// work on one 256 x BN tile.  Each stages its own 128 weight rows and HALF of the activation tile, the first CTA
+// of the pair issues MMAs that read both CTAs' shared memory, and each CTA ends with its own 128 x BN
+// accumulator in its own TMEM.  Against the one-CTA kernel the activation tile crosses the L2 -> SM fabric once
+// per 256 weight rows instead of once per 128, which is what bounds the product from about 128 activation rows
+// on.  Loads carry no multicast: every byte is requested by the CTA that stages it.
+template <int BN>
+struct PairLayout {
+  static constexpr uint32_t A_HALF_BYTES = (BN / 2) * TILE_K * 2;
+  static constexpr uint32_t STAGE_BYTES = W_STAGE_BYTES + A_HALF_BYTES;
+  static constexpr uint32_t total(int stages) { return (uint32_t)stages * STAGE_BYTES + 1024; }
+};
+
+template <int BN>
+__global__ void __launch_bounds__(128) gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                             const __grid_constant__ CUtensorMap tmA,
+                                                             float* __restrict__ part, int M, int N, int num_kb,
+                                                             int kb_per_split, size_t split_stride, int STAGES,
+                                                             __nv_bfloat16* __restrict__ act_out, int m_ffn,
+                                                             int* __restrict__ status) {
+  using PL = PairLayout<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];   // used in the pair's first CTA: bytes of both CTAs
+  __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];  // in each CTA: its stage may be refilled
+  __shared__ __align__(8) uint64_t accum_bar;              // in each CTA: the accumulator is complete
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int m0 = blockIdx.y * BN;
+  const int n0 = blockIdx.x * TILE_W;  // the pair: blockIdx.x = 2p, 2p + 1
+  const int kb0 = blockIdx.z * kb_per_split;
+  const int kb1 = min(num_kb, kb0 + kb_per_split);
+  const int nkb = kb1 - kb0;
+  const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    mbar_init(smem_u32(&accum_bar), 1);
+    mbar_fence_init();
+    prefetch_tensormap(&tmW);
+    prefetch_tensormap(&tmA);
+  }
+  if (warp == 1) {  // the same warp of both CTAs: BN fp32 columns x 128 lanes in each CTA's TMEM
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"((uint32_t)BN)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync();  // both CTAs' barriers exist before either signals the other's
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_d = tmem_base_slot;
+  volatile int* abortp = &abort_flag;
+
+  int pre = 0;
+  if (threadIdx.x == 0) {
+    pre = min(STAGES, nkb);  // weights are written by no kernel: stream them ahead of the dependency
+    for (int i = 0; i < pre; ++i) {
+      if (leader) mbar_expect_tx(smem_u32(&full_bar[i]), 2 * PL::STAGE_BYTES);
+      tma_load_2d_pair(tiles + i * PL::STAGE_BYTES, &tmW, cluster_addr(smem_u32(&full_bar[i]), 0), (kb0 + i) * TILE_K, n0);
+    }
+  }
+  pdl_wait();     // the activation rows and the slab buffer belong to the preceding kernels
+  pdl_trigger();
+
+  if (warp == 0 && lane == 0) {
+    // ---------------- TMA producer (both CTAs) ----------------
+    int s = 0;
+    uint32_t ph = 0;
+    for (int i = 0; i < nkb; ++i) {
+      const uint32_t fb = cluster_addr(smem_u32(&full_bar[s]), 0);
+      const uint32_t dstW = tiles + s * PL::STAGE_BYTES;
+      const int kc = (kb0 + i) * TILE_K;
+      if (i >= pre) {
+        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) {
+          if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+          break;
+        }
+        if (leader) mbar_expect_tx(smem_u32(&full_bar[s]), 2 * PL::STAGE_BYTES);
+        tma_load_2d_pair(dstW, &tmW, fb, kc, n0);
+      }
+      tma_load_2d_pair(dstW + W_STAGE_BYTES, &tmA, fb, kc, m0 + (int)rank * (BN / 2));
+      if (++s == STAGES) {
+        s = 0;
+        ph ^= 1u;
+      }
+    }
+  } else if (leader && warp == 1 && lane == 0) {
+    // ---------------- MMA issuer (first CTA of the pair) ----------------
+    constexpr uint32_t idesc = make_idesc(2 * TILE_W, BN);
+    bool ok = true;
+    int s = 0;
+    uint32_t ph = 0;
+    for (int i = 0; i < nkb && ok; ++i) {
+      if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp)) {
+        if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_MMA);
+        ok = false;
+        break;
+      }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t sW = tiles + s * PL::STAGE_BYTES;
+      const uint64_t dW = make_smem_desc(sW);
+      const uint64_t dA = make_smem_desc(sW + W_STAGE_BYTES);
+#pragma unroll
+      for (int k = 0; k < TILE_K / UMMA_K; ++k)
+        umma_bf16_pair(tmem_d, dW + (uint64_t)(2 * k), dA + (uint64_t)(2 * k), idesc, (i > 0 || k > 0) ? 1u : 0u);
+      umma_commit_pair(smem_u32(&empty_bar[s]));  // both CTAs may refill the stage once these MMAs have read it
+      if (++s == STAGES) {
+        s = 0;
+        ph ^= 1u;
+      }
+    }
+    if (ok) umma_commit_pair(smem_u32(&accum_bar));
+  }
+  __syncwarp();
+
+  // ---------------- epilogue: each CTA writes its own 128 output columns ----------------
+  const bool have = mbar_wait(smem_u32(&accum_bar), 0u, abortp);
+  if (!have && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_EPI);
+  bool warp_ok = __all_sync(0xffffffffu, have);
+  if (act_out) warp_ok = __syncthreads_and(warp_ok);
+  if (warp_ok) {
+    float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // the drained ring
+    gemm_epilogue<BN>(tmem_d, ex, m0, n0, (int)blockIdx.x, M, N, part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
+  } else {
+    drain_delay();
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync();  // neither CTA leaves, nor is TMEM freed, while the other may still use this one's memory
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"((uint32_t)BN) : "memory");
   }
 }
 
@@ -323,6 +480,28 @@ cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMa
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
+template <int BN>
+cudaError_t launch_pair(const Launch& L, const CUtensorMap& tmW, const CUtensorMap& tmA, float* part, int M, int N,
+                        int num_kb, const GemmPlan& plan, void* act_out, int m_ffn) {
+  using PL = PairLayout<BN>;
+  constexpr int fit = (227 * 1024 - 1024 - 256) / (int)PL::STAGE_BYTES;
+  constexpr int most = fit < MAX_STAGES ? fit : MAX_STAGES;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)PL::total(most));
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int stages = plan.stages < 2 ? 2 : plan.stages > most ? most : plan.stages;
+  dim3 grid(N / TILE_W, (M + BN - 1) / BN, plan.S_max);  // pairs along x
+  cudaError_t e = launch_k_cluster(L, gemm_bf16_pair_kernel<BN>, grid, dim3(128), PL::total(stages), dim3(2, 1, 1), tmW,
+                                   tmA, part, M, N, num_kb, plan.upc, (size_t)M * N, stages, (__nv_bfloat16*)act_out,
+                                   m_ffn, L.d_status);
+  L.count();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 }  // namespace
 
 bool get_tensor_map_2d(const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
@@ -353,10 +532,11 @@ Partials make_partials(const float* p, int M, int N, const GemmPlan& plan) {
 // Tile shape, ring depth and split-K factor, from sweeps on B200: up to 256
 // activation rows the product is bound by streaming W, so k ranges are split
 // until at least one CTA per SM (two with 128-row tiles) streams weights.
-GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, int force_bn) {
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, int force_bn, int force_pair) {
   GemmPlan p;
   p.BN = M <= 32 ? 32 : M <= 64 ? 64 : M <= 256 ? 128 : 256;
   if (force_bn == 32 || force_bn == 64 || force_bn == 128 || force_bn == 256) p.BN = force_bn;
+  p.pair = force_pair > 0 && (p.BN == 128 || p.BN == 256) && N % (2 * TILE_W) == 0;
   p.stages = force_stages > 0 ? force_stages : (p.BN == 128 ? 3 : 4);
   p.num_kb = (K + TILE_K - 1) / TILE_K;
   p.m_tiles = (M + p.BN - 1) / p.BN;
@@ -391,11 +571,19 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
   }
   CUtensorMap tmW, tmA;
   if (!get_tensor_map_2d(W, (uint64_t)N, (uint64_t)K, TILE_W, &tmW) ||
-      !get_tensor_map_2d(A, (uint64_t)M, (uint64_t)K, (uint32_t)plan.BN, &tmA)) {
+      !get_tensor_map_2d(A, (uint64_t)M, (uint64_t)K, (uint32_t)(plan.pair ? plan.BN / 2 : plan.BN), &tmA)) {
     if (err) *err = e_map;
     return cudaErrorInvalidValue;
   }
   const int num_kb = (K + TILE_K - 1) / TILE_K;
+  if (plan.pair) {
+    if (N % (2 * TILE_W)) {
+      if (err) *err = "CTA pairs need N % 256 == 0";
+      return cudaErrorInvalidValue;
+    }
+    return plan.BN == 128 ? launch_pair<128>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn)
+                          : launch_pair<256>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
+  }
   switch (plan.BN) {
     case 32: return launch_one<32>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
     case 64: return launch_one<64>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);

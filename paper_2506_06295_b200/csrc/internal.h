@@ -40,6 +40,26 @@ inline cudaError_t launch_k(const Launch& L, void (*kernel)(KArgs...), dim3 grid
   cfg.numAttrs = L.pdl ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
+// The same for a kernel whose CTAs form clusters of `cluster` (grid dimensions are multiples of it).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k_cluster(const Launch& L, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                    dim3 cluster, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = L.stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster.x;
+  attr[0].val.clusterDim.y = cluster.y;
+  attr[0].val.clusterDim.z = cluster.z;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = L.pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // Partial sums of one GEMM: slabs of [M, N] fp32, slab stride in floats.  With
 // upc == 0 every element has S slabs; otherwise the tile that holds (row, col)
@@ -145,8 +165,11 @@ struct GemmPlan {
   int upc;          // k-blocks per split
   int ctas;         // grid size
   int S_max;        // split-K factor: slabs per output element
+  int pair = 0;     // 1: CTA pairs (cta_group::2) share the activation tile of BN rows
 };
-GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split = 0, int force_stages = 0, int force_bn = 0);  // 0 = auto
+// 0 = auto.  force_pair: 0 auto, 1 CTA pairs (BN 128 or 256, N a multiple of 256), -1 never.
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split = 0, int force_stages = 0, int force_bn = 0,
+                        int force_pair = 0);
 Partials make_partials(const float* p, int M, int N, const GemmPlan& plan);
 // Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
 // act_out != nullptr (unsplit plan, W = gate / up rows interleaved in blocks of 64, N = 2 * m_ffn): instead of

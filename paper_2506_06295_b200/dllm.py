@@ -79,6 +79,8 @@ SIGNATURES = {
     "dllm_gemm_bf16": (_I, [_P, _P, _P, _I, _I, _I, _P, _P]),
     "dllm_gemm_bf16_planned_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I]),
     "dllm_gemm_bf16_planned": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
+    "dllm_gemm_bf16_pair_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I]),
+    "dllm_gemm_bf16_pair": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
     "dllm_ffn_gate_up_bf16": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _P]),
     "dllm_gemm_simt": (_I, [_P, _P, _P, _I, _I, _I, _I, _P]),
     "dllm_attention_scratch_bytes": (_SZ, [_I, _I, _I, _I, _I, _I, _I]),
@@ -396,6 +398,22 @@ def gemm_bf16_planned(A, W, act_tile=0, splits=0, stages=0, out=None, scratch=No
     _check(lib.dllm_gemm_bf16_planned(C.c_void_p(A.data_ptr()), C.c_void_p(W.data_ptr()), C.c_void_p(cptr),
                                       M, N, K, act_tile, splits, stages, C.c_void_p(scratch.data_ptr()),
                                       scratch.numel(), C.c_void_p(sp)))
+    return Cm
+
+
+def gemm_bf16_pair(A, W, act_tile=256, splits=0, stages=0, out=None, scratch=None, stream=None):
+    """gemm_bf16 by CTA pairs (cta_group::2); N % 256 == 0."""
+    import torch
+    M, K = A.shape
+    N = W.shape[0]
+    Cm = out if out is not None else torch.empty((M, N), dtype=torch.float32, device=A.device)
+    sb = lib.dllm_gemm_bf16_pair_scratch_bytes(M, N, K, act_tile, splits)
+    if scratch is None:
+        scratch = torch.empty(max(sb, 16), dtype=torch.uint8, device=A.device)
+    sp = _stream_ptr(stream if stream is not None else torch.cuda.current_stream(A.device))
+    _check(lib.dllm_gemm_bf16_pair(C.c_void_p(A.data_ptr()), C.c_void_p(W.data_ptr()), C.c_void_p(Cm.data_ptr()),
+                                   M, N, K, act_tile, splits, stages, C.c_void_p(scratch.data_ptr()), scratch.numel(),
+                                   C.c_void_p(sp)))
     return Cm
 
 

@@ -98,6 +98,32 @@ def test_ffn_gate_up_epilogue(env, M, m, K, act_tile):
     assert dllm.lib.dllm_ffn_gate_up_bf16(dA.data_ptr(), dW.data_ptr(), dA.data_ptr(), M, 100, K, 0, 0, None) == dllm.INVALID_ARG
 
 
+@pytest.mark.parametrize("M,N,K,act_tile,splits,stages", [
+    (256, 256, 64, 256, 1, 2),        # one pair, one k-block
+    (130, 512, 448, 128, 1, 3),       # 128-row tiles, ragged second tile
+    (256, 4096, 4096, 256, 4, 3),     # the V projection of a 256-token response
+    (300, 768, 832, 256, 3, 5),       # two activation tiles, 13 k-blocks in 3 splits
+    (768, 1024, 1024, 256, 0, 0),     # default split and ring depth
+    (70, 256, 320, 128, 2, 2),        # fewer rows than a tile
+])
+def test_gemm_bf16_cta_pairs(env, M, N, K, act_tile, splits, stages):
+    """The CTA-pair kernel (cta_group::2) gives the product, bit-identical to the one-CTA kernel with the same
+    tile rows and k ranges (the same sums in the same order)."""
+    torch, dllm = env
+    A = synth.round_to_bf16(synth.random_normal((M, K), seed=M + K + 3))
+    W = synth.round_to_bf16(synth.random_normal((N, K), seed=N + 5 * K, std=0.05))
+    dA = torch.from_numpy(A).cuda().to(torch.bfloat16)
+    dW = torch.from_numpy(W).cuda().to(torch.bfloat16)
+    got = dllm.gemm_bf16_pair(dA, dW, act_tile, splits, stages).cpu().numpy()
+    want = A.astype(np.float64) @ W.astype(np.float64).T
+    assert rel_l2(got, want) < 2e-6
+    assert np.array_equal(got, dllm.gemm_bf16_pair(dA, dW, act_tile, splits, stages).cpu().numpy())
+    if splits:
+        one = dllm.gemm_bf16_planned(dA, dW, act_tile, splits, stages).cpu().numpy()
+        assert np.array_equal(got, one)
+    assert dllm.lib.dllm_gemm_bf16_pair(dA.data_ptr(), dW.data_ptr(), dA.data_ptr(), M, 128, K, 256, 0, 0, None, 0, None) == dllm.INVALID_ARG
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_gemm_simt(env, dtype):
     torch, dllm = env
