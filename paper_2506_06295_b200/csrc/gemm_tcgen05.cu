@@ -534,20 +534,37 @@ Partials make_partials(const float* p, int M, int N, const GemmPlan& plan) {
 // until at least one CTA per SM (two with 128-row tiles) streams weights.
 GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, int force_bn, int force_pair) {
   GemmPlan p;
+  const int sms = sm_count();
+  const long n_tiles = (N + TILE_W - 1) / TILE_W;
   p.BN = M <= 32 ? 32 : M <= 64 ? 64 : M <= 256 ? 128 : 256;
+  p.pair = 0;
+  int pair_stages = 3;
+  if (force_pair == 0 && force_bn == 0 && force_split <= 1 && N % (2 * TILE_W) == 0) {
+    // CTA pairs where they measured faster (B200): products that need no split between 65 and 1024 activation
+    // rows, where the activation tile's trips through the L2 -> SM fabric bound the one-CTA kernel.
+    if (M > 64 && M <= 256 && n_tiles >= sms) {
+      p.pair = 1;
+      p.BN = 256;
+    } else if (M > 256 && M <= 1024) {
+      p.pair = 1;
+      const bool one_wave = n_tiles * ((M + 127) / 128) <= 2L * sms;  // all 128-row pair tiles resident at once
+      p.BN = one_wave ? 128 : 256;
+      pair_stages = one_wave ? 4 : 3;
+    }
+  }
   if (force_bn == 32 || force_bn == 64 || force_bn == 128 || force_bn == 256) p.BN = force_bn;
-  p.pair = force_pair > 0 && (p.BN == 128 || p.BN == 256) && N % (2 * TILE_W) == 0;
-  p.stages = force_stages > 0 ? force_stages : (p.BN == 128 ? 3 : 4);
+  if (force_pair > 0) p.pair = (p.BN == 128 || p.BN == 256) && N % (2 * TILE_W) == 0;
+  p.stages = force_stages > 0 ? force_stages : p.pair ? pair_stages : (p.BN == 128 ? 3 : 4);
   p.num_kb = (K + TILE_K - 1) / TILE_K;
   p.m_tiles = (M + p.BN - 1) / p.BN;
-  const long tiles = (long)p.m_tiles * ((N + TILE_W - 1) / TILE_W);
-  const int sms = sm_count();
+  const long tiles = (long)p.m_tiles * n_tiles;
   // every split adds a slab the consumer has to read: with few activation rows
   // one wave of CTAs is enough, with 128-row tiles two CTAs per SM pay off
   int S = p.BN == 128 ? (int)(2L * sms / tiles) : (int)((sms + tiles - 1) / tiles);  // all CTAs resident at once
   const int max_s = p.num_kb / 4 > 1 ? p.num_kb / 4 : 1;
   if (S > max_s) S = max_s;
   if (S < 1) S = 1;
+  if (p.pair && force_pair == 0) S = 1;
   if (force_split > 0) S = force_split < p.num_kb ? force_split : p.num_kb;
   p.upc = (p.num_kb + S - 1) / S;                 // k-blocks per split
   p.S_max = (p.num_kb + p.upc - 1) / p.upc;       // no empty split

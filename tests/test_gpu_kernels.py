@@ -78,7 +78,10 @@ def test_gemm_bf16_explicit_plans(env, act_tile, splits, stages):
 
 
 @pytest.mark.parametrize("M,m,K,act_tile", [(64, 1216, 512, 0), (3, 64, 64, 32), (70, 832, 448, 64), (130, 192, 1088, 128),
-                                            (300, 320, 256, 256), (257, 128, 832, 0)])
+                                            (300, 320, 256, 256), (257, 128, 832, 0),
+                                            (300, 256, 192, 0),      # default plan: CTA pairs, 128-row tiles
+                                            (200, 9472, 64, 0),      # default plan: CTA pairs, 256-row tiles
+                                            (600, 19200, 64, 0)])    # CTA pairs, 256-row tiles, three row tiles
 def test_ffn_gate_up_epilogue(env, M, m, K, act_tile):
     """Gate / up projection with SwiGLU in the GEMM epilogue against silu(A Wg^T) * (A Wu^T) in float64."""
     torch, dllm = env
