@@ -46,6 +46,7 @@ constexpr int UMMA_K = 16;
 constexpr uint32_t W_STAGE_BYTES = TILE_W * TILE_K * 2;
 
 constexpr int MAX_STAGES = 12;
+constexpr int RASTER = 16;     // activation tiles per group of the launch-order remap
 
 template <int BN>
 struct SmemLayout {
@@ -137,8 +138,19 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * BN;       // activation rows
-  const int n0 = blockIdx.y * TILE_W;   // weight rows = output columns
+  // Tile of this CTA.  With many activation tiles, CTAs that run together (consecutive in x-major launch order)
+  // take RASTER activation tiles times a few weight tiles, so that their operands stay in L2 while the other
+  // dimension is swept; otherwise every sweep over the weight tiles would re-read all activations from HBM.
+  int mt = blockIdx.x, nt = blockIdx.y;
+  if (gridDim.x > RASTER) {
+    const int lin = blockIdx.x + gridDim.x * blockIdx.y, per = RASTER * gridDim.y;
+    const int grp = lin / per, within = lin - grp * per;
+    const int wide = min(RASTER, (int)gridDim.x - grp * RASTER);
+    nt = within / wide;
+    mt = grp * RASTER + within - nt * wide;
+  }
+  const int m0 = mt * BN;       // activation rows
+  const int n0 = nt * TILE_W;   // weight rows = output columns
   const int kb0 = blockIdx.z * kb_per_split;
   const int kb1 = min(num_kb, kb0 + kb_per_split);
   const int nkb = kb1 - kb0;            // >= 1 by construction of the plan
@@ -238,7 +250,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   if (act_out) warp_ok = __syncthreads_and(warp_ok);  // the SwiGLU epilogue exchanges data between warps
   if (warp_ok) {
     float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // the drained ring
-    gemm_epilogue<BN>(tmem_d, ex, m0, n0, (int)blockIdx.y, M, N, part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
+    gemm_epilogue<BN>(tmem_d, ex, m0, n0, nt, M, N, part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
   } else {
     drain_delay();  // gave up: let copies in flight land before shared memory is released
   }
