@@ -505,7 +505,8 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
       const uint8_t* ua = s->wsp<uint8_t>(s->ws.ua);
       if (identity) {
         ua = u;
-      } else if (s->R <= 1024) {
+      } else if (s->R <= 1024 && (long)Ma * s->R <= 64L * 1024) {
+        // few active rows: every CTA of the gather repeats the selection rather than wait for a launch
         launch_select_gather(L, dt, sim, forced, mode, ksel, sel, act, inv, u, s->wsp<uint8_t>(s->ws.ua), g, rp);
       } else {
         launch_select(L, sim, forced, mode, ksel, sel, s->R, act, inv, g, rp);
