@@ -33,7 +33,12 @@ def _newer(target: str, deps: list[str]) -> bool:
     return all(os.path.getmtime(d) <= t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, timeline: bool = False) -> str:
+    """timeline=True builds libdllm_b200_timeline.so instead: the same library with device-timestamp records in
+    every kernel (see timeline.py); the product library is never built with them."""
+    OBJ = os.path.join(HERE, "_build_timeline" if timeline else "_build")
+    LIB = os.path.join(HERE, "libdllm_b200_timeline.so" if timeline else "libdllm_b200.so")
+    flags = NVCC_FLAGS + (["-DDLLM_TIMELINE"] if timeline else [])
     os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(HERE, "..", "include", "dllm.h"))
@@ -46,7 +51,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
         if not force and _newer(obj, [src] + headers):
             return obj
-        cmd = [nvcc, *NVCC_FLAGS, "-c", src, "-o", obj]
+        cmd = [nvcc, *flags, "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         r = subprocess.run(cmd, capture_output=True, text=True)

@@ -386,3 +386,4 @@ extern "C" dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, 
   return DLLM_OK;
 }
 
+DLLM_TIMELINE_HOOKS(attention)

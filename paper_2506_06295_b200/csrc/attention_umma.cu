@@ -405,3 +405,5 @@ cudaError_t launch_attention_umma(const Launch& L, const void* q, const void* Kc
 }
 
 }  // namespace dllm
+
+DLLM_TIMELINE_HOOKS(attention_umma)

@@ -33,7 +33,57 @@ enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_E
 // in the stream has completed and its writes are visible (returns at once for
 // a launch without the attribute).  pdl_trigger(): lets the next grid become
 // resident once every CTA of this grid has called it.
+#ifndef DLLM_TIMELINE
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#define DLLM_TIMELINE_HOOKS(stem)
+#else
+// Timeline build (python -m paper_2506_06295_b200.timeline): thread 0 of every CTA records the global timer
+// before and after the dependency wait, so that a replayed CUDA graph yields, per kernel, when its CTAs became
+// resident and when its predecessor had completed -- the time a kernel really takes inside the step, which
+// neither serialised profiler runs nor event pairs around single launches show.  Records: {grid | block << 48,
+// t_resident, t_released, SM id | CTA << 32}, one array and one cursor per translation unit.
+static __device__ unsigned long long* g_timeline;
+static __device__ unsigned int g_timeline_n;
+constexpr unsigned int TIMELINE_CAP = 1u << 20;
+__device__ __forceinline__ unsigned long long timeline_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void pdl_wait() {
+  const bool rec = threadIdx.x == 0 && g_timeline != nullptr;
+  unsigned long long t0 = 0;
+  if (rec) t0 = timeline_now();
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (rec) {
+    const unsigned long long t1 = timeline_now();
+    const unsigned int i = atomicAdd(&g_timeline_n, 1u);
+    if (i < TIMELINE_CAP) {
+      unsigned int smid;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      g_timeline[4 * i] = (unsigned long long)gridDim.x | ((unsigned long long)gridDim.y << 16) |
+                          ((unsigned long long)gridDim.z << 32) | ((unsigned long long)blockDim.x << 48);
+      g_timeline[4 * i + 1] = t0;
+      g_timeline[4 * i + 2] = t1;
+      g_timeline[4 * i + 3] = smid | ((unsigned long long)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) << 32);
+    }
+  }
+}
+// One pair of host entry points per translation unit: set the record array (device, 32 bytes x 2^20; NULL = off)
+// and clear the cursor; read the cursor.
+#define DLLM_TIMELINE_HOOKS(stem)                                              \
+  extern "C" int dllm_timeline_set_##stem(unsigned long long* d_records) {     \
+    unsigned int zero = 0;                                                     \
+    cudaError_t e = cudaMemcpyToSymbol(dllm::g_timeline, &d_records, sizeof d_records); \
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(dllm::g_timeline_n, &zero, sizeof zero); \
+    return (int)e;                                                             \
+  }                                                                            \
+  extern "C" unsigned int dllm_timeline_count_##stem() {                       \
+    unsigned int n = 0;                                                        \
+    cudaMemcpyFromSymbol(&n, dllm::g_timeline_n, sizeof n);                    \
+    return n < dllm::TIMELINE_CAP ? n : dllm::TIMELINE_CAP;                    \
+  }
+#endif
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <typename T>

@@ -994,3 +994,5 @@ void launch_mask_column(const Launch& L, float* logits, int rows, int vocab, int
 }
 
 }  // namespace dllm
+
+DLLM_TIMELINE_HOOKS(elementwise)

@@ -65,3 +65,5 @@ void launch_gemm_simt(const Launch& L, int dtype, const void* A, const void* W, 
 }
 
 }  // namespace dllm
+
+DLLM_TIMELINE_HOOKS(gemm_simt)

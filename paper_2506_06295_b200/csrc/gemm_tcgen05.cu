@@ -622,3 +622,5 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
 }
 
 }  // namespace dllm
+
+DLLM_TIMELINE_HOOKS(gemm_tcgen05)

@@ -879,3 +879,5 @@ cudaError_t launch_layer_megakernel(const Launch& L, const MkParams& p) {
 }
 
 }  // namespace dllm
+
+DLLM_TIMELINE_HOOKS(megakernel)

@@ -13,7 +13,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdllm_b200.so")
+# DLLM_B200_LIB names another build of the same library (the timeline build of timeline.py)
+LIB_PATH = os.environ.get("DLLM_B200_LIB") or os.path.join(_HERE, "libdllm_b200.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2506_06295_b200.build` "
