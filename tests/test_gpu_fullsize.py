@@ -78,6 +78,26 @@ def test_llada_width_two_layers_against_the_oracle(env):
             for l in range(cfg.n_layers):
                 assert rel_l2(ses.get_cache(l, which), ref[l]) < 2e-2
 
+    # a response refresh (256 rows: CTA pairs in the gate / up projection and the LM head, no selection launch)
+    # and a prompt refresh with adaptive response update (512 + 64 rows)
+    for step, (rp, rr) in ((3, (False, True)), (4, (True, False))):
+        resp = orc.tokens[:, P:].copy()
+        resp[0, 7 * step] = (31 * step) % (cfg.vocab - 1)
+        orc.tokens[:, P:] = resp
+        ses.set_response_tokens(resp)
+        r = orc.step(rp, rr, wl.rho)
+        ses.step_cached(rp, rr, wl.rho)
+        ses.sync()
+        assert rel_l2(ses.hidden(), r.hidden) < 2e-2, f"step {step}"
+        for which, ref in ((dllm.CACHE_K, orc.Kc), (dllm.CACHE_V, orc.Vc), (dllm.CACHE_ATTN, orc.Ac),
+                           (dllm.CACHE_FFN, orc.Fc)):
+            for l in range(cfg.n_layers):
+                assert rel_l2(ses.get_cache(l, which), ref[l]) < 2e-2, f"step {step} cache {which} layer {l}"
+        if not rr:
+            for l in range(cfg.n_layers):
+                idx, _ = ses.selected(l)
+                assert selection_matches(idx[0], r.selected[l][0], r.sim[l][0]), f"step {step} layer {l}"
+
 
 def test_llada_full_depth_properties_and_layer0_samples(env):
     torch, dllm = env
