@@ -350,6 +350,27 @@ def main():
     per_kind = {"full": time_kind(True, True, args.full_steps), "refresh": time_kind(False, True, 6),
                 "mixed": time_kind(True, False, 6), "partial": time_kind(False, False, 12)}
 
+    # ---- the same schedule with the prediction restricted to the block each step works on -------
+    # (reported beside the headline, never as it: the headline step predicts every response row)
+    ses.set_prompt(prompt)
+    for k in (wl.steps, wl.steps - 1, wl.steps - 2):        # graphs of the step kinds with a block head
+        ses.step_scheduled_block(k, wl.steps, wl.Kp, wl.Kr, wl.rho, 0, wl.block_len)
+    ses.set_prompt(prompt)
+    barrier()
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b0.record(stream)
+    for i in range(K):
+        k = wl.steps - (i % wl.steps)
+        if i and k == wl.steps:
+            ses.set_prompt(prompt)
+        bs, nt = block_plan(wl.steps - k, wl.steps, wl.gen_len, wl.block_len)
+        ses.step_scheduled_block(k, wl.steps, wl.Kp, wl.Kr, wl.rho, bs, wl.block_len)
+        ses.remask_low_confidence(bs, wl.block_len, nt)
+    b1.record(stream)
+    barrier()
+    ms_block = b0.elapsed_time(b1)
+    block_tokens = ses.tokens()
+
     # ---- end to end through host buffers ---------------------------------------------------------
     ses.set_prompt(prompt)
     host_tok = torch.empty((wl.batch, wl.gen_len), dtype=torch.int32).pin_memory()
@@ -415,6 +436,10 @@ def main():
         "full_recompute_tokens_per_s": wl.batch * wl.gen_len / wl.steps * world / (per_kind["full"] / 1e3),
         "e2e": {"value": tokens / (ms_e2e / 1e3), "unit": "tokens/s",
                 "h2d_bytes_per_step": wl.batch * wl.gen_len * 4, "d2h_bytes_per_step": wl.batch * (wl.prompt_len + wl.gen_len) * 4},
+        "block_only_prediction": {"value": tokens / (ms_block / 1e3), "unit": "tokens/s", "ms_per_step": ms_block / K,
+                                  "same_tokens_as_headline_run": bool((block_tokens == final_tokens).all()),
+                                  "what": "dllm_step_scheduled_block: logits, estimate and confidence only for the "
+                                          "block the step works on; layers and caches identical"},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"kernel": "gemm_bf16_tcgen05_kernel", "bound": "hbm", "achieved": gemm_gbs,

@@ -146,6 +146,20 @@ dllm_status dllm_step_cached_layers(dllm_session* s, int refresh_prompt, int ref
  * k = K, the prompt when k mod Kp == 0, the response when k mod Kr == 0. */
 dllm_status dllm_step_scheduled(dllm_session* s, int k, int K, int Kp, int Kr, float rho,
                                 dllm_kround kround, void* stream);
+/* The same step with the prediction (Eqs. 3-4: logits, greedy estimate, confidence)
+ * restricted to response positions [block_start, block_start + block_len) of
+ * every sequence: the only positions the transition of a semi-autoregressive
+ * step reads (Eq. 5 over the current block).  The layers, the caches and the
+ * hidden states are exactly those of dllm_step_scheduled; x0 / conf of the
+ * block are bit-identical to it, those of other positions keep the values of
+ * an earlier step (dllm_get_logits recomputes all rows from the hidden states
+ * and is unaffected).  The LM head then streams its weights for block_len rows
+ * instead of R and the estimate reads block_len rows of logits. */
+dllm_status dllm_step_scheduled_block(dllm_session* s, int k, int K, int Kp, int Kr, float rho, dllm_kround kround,
+                                      int block_start, int block_len, void* stream);
+/* enable != 0: dllm_generate uses dllm_step_scheduled_block with the block each
+ * step works on (the generated tokens are the same).  Default off. */
+dllm_status dllm_session_predict_block_only(dllm_session* s, int enable);
 /* Transition S with low-confidence remasking (Eq. 5): among the still masked
  * response positions in [block_start, block_start + block_len) the
  * min(n_transfer, #masked) positions with the highest confidence (ties: lowest

@@ -191,7 +191,10 @@ struct StepKey {
   uint64_t forced_sig;
   int variant = 0;
   uint64_t ksel_sig = 0;  // per-layer row counts (cross-layer allocation of rho)
+  int head_start = 0, head_len = 0;  // prediction restricted to one block of the response (0 rows: all of it)
   bool operator<(const StepKey& o) const {
+    if (head_start != o.head_start) return head_start < o.head_start;
+    if (head_len != o.head_len) return head_len < o.head_len;
     if (variant != o.variant) return variant < o.variant;
     if (ksel_sig != o.ksel_sig) return ksel_sig < o.ksel_sig;
     if (rp != o.rp) return rp < o.rp;
@@ -216,6 +219,7 @@ struct dllm_session {
   bool simt_gemm = false;
   bool use_pdl = true;
   int sel_strategy = DLLM_SELECT_V_VERIFY, sel_metric = DLLM_METRIC_COSINE, v_selected_only = 0;  // ablation variants
+  bool block_head = false;     // dllm_generate predicts only the block each step works on
   bool use_mk = false;         // persistent layer kernel for the step kinds it covers (opt-in)
   bool mk_maps_ready = false;  // weight / cache tensor maps uploaded to the workspace
   struct GraphEntry {
@@ -448,7 +452,8 @@ bool step_uses_mk(const dllm_session* s, int rp, int ksel) {
 // Enqueue one denoising step.  Active rows per sequence: the prompt rows on a
 // prompt refresh plus either all R response rows (response refresh) or the
 // ksel rows V-verify picks.
-dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>& ksels, cudaStream_t stream) {
+dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>& ksels, cudaStream_t stream,
+                         int head_start = 0, int head_len = 0) {
   const dllm_config& c = s->m->cfg;
   const WeightLayout& wl = s->m->lay;
   const Geo g = s->geo();
@@ -542,10 +547,23 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
     launch_tail(L, dt, part, Ma > 0 ? inv : nullptr, x, s->cache(l, DLLM_CACHE_ATTN), s->cache(l, DLLM_CACHE_FFN),
                 gain_next, u, g, c0, c1, c.rms_eps);
   }
-  // prediction at the response rows (Eqs. 3-4); u holds the final norm
-  if ((st = run_gemm(s, L, u, W + wl.lm_head, BR, c.vocab, d, &part)) != DLLM_OK) return st;
+  // prediction at the response rows (Eqs. 3-4); u holds the final norm.  With head_len > 0 only the rows of
+  // one block are predicted: the transition of a semi-autoregressive step reads no others (Eq. 5).
+  const uint8_t* head_in = u;
+  int head_rows = BR;
+  if (head_len > 0) {
+    head_rows = s->B * head_len;
+    if (s->B == 1) {
+      head_in = u + (size_t)head_start * d * es;
+    } else {
+      launch_gather_block_rows(L, dt, u, s->wsp<uint8_t>(s->ws.ua), s->B, s->R, head_start, head_len, d);
+      head_in = s->wsp<uint8_t>(s->ws.ua);
+    }
+  }
+  if ((st = run_gemm(s, L, head_in, W + wl.lm_head, head_rows, c.vocab, d, &part)) != DLLM_OK) return st;
   if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
-  launch_argmax_conf(L, part.p, BR, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf));
+  launch_argmax_conf(L, part.p, head_rows, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf),
+                     s->R, head_start, head_len);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "step launch: %s", cudaGetErrorString(e));
   return DLLM_OK;
@@ -557,7 +575,8 @@ uint64_t forced_signature(const dllm_session* s) {
   return h;
 }
 
-dllm_status run_step(dllm_session* s, int rp, int rr, const float* rhos, int n_rho, dllm_kround kr, void* stream_v) {
+dllm_status run_step(dllm_session* s, int rp, int rr, const float* rhos, int n_rho, dllm_kround kr, void* stream_v,
+                     int head_start = 0, int head_len = 0) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
   const int T = s->m->cfg.n_layers;
   if (!rhos || (n_rho != 1 && n_rho != T)) return fail(&s->err, DLLM_INVALID_ARG, "one rho, or one per layer");
@@ -583,19 +602,22 @@ dllm_status run_step(dllm_session* s, int rp, int rr, const float* rhos, int n_r
   cudaStream_t stream = (cudaStream_t)stream_v;
   dllm_status st = DLLM_OK;
   const bool graph_ok = s->use_graphs && !s->profiling && stream != nullptr && stream != cudaStreamLegacy;
-  if (uniform && step_uses_mk(s, rp, ksels[0])) {
+  if (head_len < 0 || head_start < 0 || head_start + head_len > s->R)
+    return fail(&s->err, DLLM_INVALID_ARG, "block [%d, %d) outside the response", head_start, head_start + head_len);
+  if (head_len == s->R) head_start = head_len = 0;  // the whole response: the ordinary step
+  if (head_len == 0 && uniform && step_uses_mk(s, rp, ksels[0])) {
     st = enqueue_step_mk(s, rr, ksels[0], stream);  // a handful of launches: no graph needed
   } else if (!graph_ok) {
-    st = enqueue_step(s, rp, rr, ksels, stream);
+    st = enqueue_step(s, rp, rr, ksels, stream, head_start, head_len);
   } else {
     StepKey key{rp, rr, ksels[0], forced_signature(s), s->sel_strategy * 4 + s->sel_metric * 2 + s->v_selected_only,
-                uniform ? 0 : sig};
+                uniform ? 0 : sig, head_start, head_len};
     auto it = s->graphs.find(key);
     if (it == s->graphs.end()) {
       cudaGraph_t graph = nullptr;
       CU_TRY(&s->err, cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal));
       const uint64_t before = s->launches;
-      st = enqueue_step(s, rp, rr, ksels, stream);
+      st = enqueue_step(s, rp, rr, ksels, stream, head_start, head_len);
       cudaError_t e = cudaStreamEndCapture(stream, &graph);
       if (st != DLLM_OK) {
         if (graph) cudaGraphDestroy(graph);
@@ -827,6 +849,22 @@ dllm_status dllm_step_scheduled(dllm_session* s, int k, int K, int Kp, int Kr, f
   return run_step(s, rp, rr, &rho, 1, kround, stream);
 }
 
+dllm_status dllm_step_scheduled_block(dllm_session* s, int k, int K, int Kp, int Kr, float rho, dllm_kround kround,
+                                      int block_start, int block_len, void* stream) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (K <= 0 || k <= 0 || k > K || Kp <= 0 || Kr <= 0)
+    return fail(&s->err, DLLM_INVALID_ARG, "need 1 <= k <= K and positive K_p, K_r");
+  if (block_len <= 0) return fail(&s->err, DLLM_INVALID_ARG, "block_len must be positive");
+  const int rp = (k == K) || (k % Kp == 0), rr = (k == K) || (k % Kr == 0);
+  return run_step(s, rp, rr, &rho, 1, kround, stream, block_start, block_len);
+}
+
+dllm_status dllm_session_predict_block_only(dllm_session* s, int enable) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  s->block_head = enable != 0;
+  return DLLM_OK;
+}
+
 dllm_status dllm_remask_low_confidence(dllm_session* s, int block_start, int block_len, int n_transfer, void* stream) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
   if (block_start < 0 || block_len <= 0 || block_start + block_len > s->R || n_transfer < 0)
@@ -850,9 +888,11 @@ dllm_status dllm_generate(dllm_session* s, int K, int Kp, int Kr, float rho, dll
   if (K % blocks) return fail(&s->err, DLLM_INVALID_ARG, "K must be a multiple of the number of blocks");
   const int spb = K / blocks;
   for (int k = K; k >= 1; --k) {
-    dllm_status st = dllm_step_scheduled(s, k, K, Kp, Kr, rho, kround, stream);
-    if (st != DLLM_OK) return st;
     const int t = K - k, blk = std::min(t / spb, blocks - 1), i = t - blk * spb;
+    dllm_status st = s->block_head
+                         ? dllm_step_scheduled_block(s, k, K, Kp, Kr, rho, kround, blk * block_len, block_len, stream)
+                         : dllm_step_scheduled(s, k, K, Kp, Kr, rho, kround, stream);
+    if (st != DLLM_OK) return st;
     const int n_transfer = block_len / spb + (i < block_len % spb ? 1 : 0);
     st = dllm_remask_low_confidence(s, blk * block_len, block_len, n_transfer, stream);
     if (st != DLLM_OK) return st;

@@ -829,8 +829,10 @@ __device__ __forceinline__ void online_add(MaxSum& t, float v, int i) {
   }
 }
 
+// blk_len > 0: logits row r belongs to response row blk_start + r % blk_len of sequence r / blk_len (the rows
+// of one generation block); otherwise logits row r is carried response row r.
 __global__ void argmax_conf_kernel(const float* __restrict__ logits, int vocab, int mask_id, int32_t* __restrict__ x0,
-                                   float* __restrict__ conf) {
+                                   float* __restrict__ conf, int R, int blk_start, int blk_len) {
   pdl_wait();
   pdl_trigger();
   __shared__ MaxSum sh[32];
@@ -881,16 +883,40 @@ __global__ void argmax_conf_kernel(const float* __restrict__ logits, int vocab, 
       t = merge(t, q);
     }
     if (lane == 0) {
-      x0[row] = t.a;
-      conf[row] = 1.f / t.s;
+      const size_t out = blk_len > 0 ? (row / blk_len) * R + blk_start + row % blk_len : row;
+      x0[out] = t.a;
+      conf[out] = 1.f / t.s;
     }
   }
 }
 
 void launch_argmax_conf(const Launch& L, const float* logits, int rows, int vocab, int mask_id, int32_t* x0,
-                        float* conf) {
+                        float* conf, int R, int blk_start, int blk_len) {
   if (rows <= 0) return;
-  launch_k(L, argmax_conf_kernel, dim3(rows), dim3(512), 0, logits, vocab, mask_id, x0, conf);
+  launch_k(L, argmax_conf_kernel, dim3(rows), dim3(512), 0, logits, vocab, mask_id, x0, conf, R, blk_start, blk_len);
+  L.count();
+}
+
+// ------------------------------------------------------------------ rows of one generation block, all sequences
+// dst[b * len + i] = src[b * R + start + i] (rows of d elements): the final-norm rows the LM head needs when only
+// the block a step works on is predicted.
+template <typename T>
+__global__ void gather_block_rows_kernel(const T* __restrict__ src, T* __restrict__ dst, int R, int start, int len,
+                                         int d) {
+  pdl_wait();
+  pdl_trigger();
+  const int r = blockIdx.x, b = r / len, i = r - b * len;
+  const uint4* s4 = reinterpret_cast<const uint4*>(src + ((size_t)b * R + start + i) * d);
+  uint4* o4 = reinterpret_cast<uint4*>(dst + (size_t)r * d);
+  const int nvec = d * (int)sizeof(T) / 16;
+  for (int v = threadIdx.x; v < nvec; v += blockDim.x) o4[v] = s4[v];
+}
+
+void launch_gather_block_rows(const Launch& L, int dtype, const void* src, void* dst, int B, int R, int start, int len,
+                              int d) {
+  if (B * len <= 0) return;
+  DLLM_DISPATCH(dtype, (launch_k(L, gather_block_rows_kernel<T>, dim3(B * len), dim3(128), 0, (const T*)src, (T*)dst, R,
+                                 start, len, d)));
   L.count();
 }
 

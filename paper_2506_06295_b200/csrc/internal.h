@@ -141,7 +141,10 @@ void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer,
                      int c1);
 // (x0, conf) per response row from fp32 logits; the mask id never wins.
 void launch_argmax_conf(const Launch& L, const float* logits, int rows, int vocab, int mask_id, int32_t* x0,
-                        float* conf);
+                        float* conf, int R = 0, int blk_start = 0, int blk_len = 0);
+// dst[b * len + i] = src[b * R + start + i], rows of d elements (d * element size a multiple of 16 bytes)
+void launch_gather_block_rows(const Launch& L, int dtype, const void* src, void* dst, int B, int R, int start, int len,
+                              int d);
 void launch_remask(const Launch& L, int32_t* tokens, const int32_t* x0, const float* conf, Geo g, int mask_id,
                    int block_start, int block_len, int n_transfer);
 void launch_reduce_partials(const Launch& L, Partials part, float* C, int M);

@@ -43,6 +43,8 @@ SIGNATURES = {
     "dllm_cache_bytes": (_SZ, [C.POINTER(Config), _I, _I, _I]),
     "dllm_workspace_bytes": (_SZ, [C.POINTER(Config), _I, _I, _I]),
     "dllm_tensor_offset": (_I, [C.POINTER(Config), C.c_char_p, C.POINTER(_SZ), C.POINTER(_SZ)]),
+    "dllm_step_scheduled_block": (_I, [_P, _I, _I, _I, _I, _F, _I, _I, _I, _P]),
+    "dllm_session_predict_block_only": (_I, [_P, _I]),
     "dllm_tensor_blocks": (_I, [C.POINTER(Config), C.c_char_p, C.POINTER(_SZ), C.POINTER(_SZ)]),
     "dllm_model_create": (_I, [C.POINTER(Config), _P, C.POINTER(_P)]),
     "dllm_model_set_tensor": (_I, [_P, C.c_char_p, _P, _SZ]),
@@ -262,6 +264,15 @@ class Session:
 
     def step_scheduled(self, k: int, K: int, Kp: int, Kr: int, rho: float, kround: int = K_FLOOR) -> None:
         _check(lib.dllm_step_scheduled(self.handle, k, K, Kp, Kr, rho, kround, self.sp))
+
+    def step_scheduled_block(self, k: int, K: int, Kp: int, Kr: int, rho: float, block_start: int, block_len: int,
+                             kround: int = K_FLOOR) -> None:
+        """step_scheduled with logits / estimate / confidence only for one block of the response."""
+        _check(lib.dllm_step_scheduled_block(self.handle, k, K, Kp, Kr, rho, kround, block_start, block_len, self.sp))
+
+    def predict_block_only(self, on: bool) -> None:
+        """generate() predicts only the block each step works on (same tokens, smaller LM head)."""
+        _check(lib.dllm_session_predict_block_only(self.handle, int(on)))
 
     def remask_low_confidence(self, block_start: int, block_len: int, n_transfer: int) -> None:
         _check(lib.dllm_remask_low_confidence(self.handle, block_start, block_len, n_transfer, self.sp))

@@ -117,6 +117,51 @@ def test_tiny_fp32_generation_matches_token_for_token(env):
     assert np.array_equal(got, want)
 
 
+@pytest.mark.parametrize("mode", ["fp32", "bf16"])
+def test_block_only_prediction_gives_the_same_generation(env, mode):
+    """Predicting only the block a step works on (the only rows Eq. 5 reads) leaves hidden states and caches
+    untouched, gives bit-identical estimates and confidences for the block, and generates the same tokens; in
+    fp32 those are the oracle's tokens."""
+    torch, dllm = env
+    if mode == "fp32":
+        wl = synth.WORKLOADS["tiny"]
+        cfg, B, P, R, K, Kp, Kr, rho, bl = wl.model, 2, wl.prompt_len, wl.gen_len, wl.steps, wl.Kp, wl.Kr, wl.rho, 16
+    else:
+        cfg, B, P, R, K, Kp, Kr, rho, bl = synth.small_bf16_model(), 2, 100, 48, 12, 6, 3, 0.25, 16
+    orc, ses_all, _ = make_pair(dllm, cfg, B, P, R)
+    _, ses_blk, _ = make_pair(dllm, cfg, B, P, R)
+    # one step each way on the same state: same hidden states, same (x0, conf) inside the block
+    ses_all.step_full()
+    ses_blk.step_full()
+    for k, bs in ((K - 1, 0), (K - 2, bl)):
+        ses_all.step_scheduled(k, K, Kp, Kr, rho)
+        ses_blk.step_scheduled_block(k, K, Kp, Kr, rho, bs, bl)
+        ses_all.sync(), ses_blk.sync()
+        assert np.array_equal(ses_all.hidden(), ses_blk.hidden())
+        (xa, ca), (xb, cb) = ses_all.pred(), ses_blk.pred()
+        assert np.array_equal(xa[:, bs:bs + bl], xb[:, bs:bs + bl])
+        assert np.array_equal(ca[:, bs:bs + bl], cb[:, bs:bs + bl])
+        for l in range(cfg.n_layers):
+            for w in range(4):
+                assert np.array_equal(ses_all.get_cache(l, w), ses_blk.get_cache(l, w))
+    assert ses_blk.launch_count() > 0
+    # whole generations
+    prompt = synth.make_prompt(cfg, B, P)
+    toks = []
+    for ses, on in ((ses_all, False), (ses_blk, True)):
+        ses.set_prompt(prompt)
+        ses.predict_block_only(on)
+        ses.generate(K, Kp, Kr, rho, bl)
+        ses.sync()
+        toks.append(ses.tokens())
+    assert (toks[1][:, P:] != cfg.mask_id).all()
+    assert np.array_equal(toks[0], toks[1])
+    if mode == "fp32":
+        assert np.array_equal(toks[1], orc.generate(K, Kp, Kr, rho, bl))
+    with pytest.raises(dllm.DllmError):
+        ses_blk.step_scheduled_block(1, K, Kp, Kr, rho, R - 1, bl)      # block leaves the response
+
+
 def test_tiny_fp32_stepwise_generation_with_graphs_off_and_on(env):
     torch, dllm = env
     wl = synth.WORKLOADS["tiny"]
