@@ -317,31 +317,36 @@ int k_selected(float rho, int R, dllm_kround kr) {
 
 // One GEMM of the step: out = A[M,K] * W[N,K]^T as split-K partial slabs.
 dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void* W, int M, int N, int K,
-                     Partials* out, void* swiglu_out = nullptr, bool* fused = nullptr) {
+                     Partials* out, void* swiglu_out = nullptr, bool* fused = nullptr, int estimate_mask_id = -1) {
   float* part = s->wsp<float>(s->ws.part);
   if (fused) *fused = false;
   *out = Partials{part, (size_t)M * N, 1, N};
   if (M <= 0) return DLLM_OK;
-  // algorithmic traffic of one projection: the weight matrix and the activation
-  // rows once in, one fp32 result out (split-K slabs are overhead, not counted)
   const double es = (double)s->es();
-  s->prof_begin(0, ((double)N * K + (double)M * K) * es + (double)M * N * 4.0, 2.0 * M * N * K, L.stream);
+  const bool tensor = !(s->m->cfg.dtype == DLLM_FP32 || s->simt_gemm);
+  const GemmPlan plan = tensor ? plan_gemm_bf16(M, N, K) : GemmPlan{};
+  // an unsplit gate / up projection of an interleaved weight finishes SwiGLU in its own epilogue, and an unsplit
+  // LM head writes per-tile estimate records instead of logits
+  const bool estimate = tensor && !swiglu_out && estimate_mask_id >= 0 && plan.S_max == 1;
+  const bool fuse = estimate || (tensor && swiglu_out && plan.S_max == 1 && gu_interleaved(s->m->cfg));
+  // algorithmic traffic of one projection: the weight matrix and the activation rows once in, one result out
+  // (fp32, or what the fused epilogue writes; split-K slabs are overhead, not counted)
+  const double out_bytes = estimate ? (double)M * ((N + 127) / 128) * 16.0 : fuse ? (double)M * (N / 2) * 2.0 : (double)M * N * 4.0;
+  s->prof_begin(0, ((double)N * K + (double)M * K) * es + out_bytes, 2.0 * M * N * K, L.stream);
   struct End {
     dllm_session* s;
     cudaStream_t st;
     ~End() { s->prof_end(st); }
   } end_guard{s, L.stream};
-  if (s->m->cfg.dtype == DLLM_FP32 || s->simt_gemm) {
+  if (!tensor) {
     launch_gemm_simt(L, s->m->cfg.dtype, A, W, part, M, N, K);
     return DLLM_OK;
   }
-  const GemmPlan plan = plan_gemm_bf16(M, N, K);
   if ((size_t)plan.S_max * M * N > s->ws.part_floats)
     return fail(&s->err, DLLM_UNSUPPORTED, "GEMM %dx%dx%d with %d slabs exceeds the workspace", M, N, K, plan.S_max);
   const char* why = nullptr;
-  // an unsplit gate / up projection of an interleaved weight finishes SwiGLU in its own epilogue
-  const bool fuse = swiglu_out && plan.S_max == 1 && gu_interleaved(s->m->cfg);
-  cudaError_t e = launch_gemm_bf16(L, A, W, part, M, N, K, plan, &why, fuse ? swiglu_out : nullptr, fuse ? N / 2 : 0);
+  cudaError_t e = launch_gemm_bf16(L, A, W, part, M, N, K, plan, &why, fuse && !estimate ? swiglu_out : nullptr,
+                                   estimate ? -1 - estimate_mask_id : fuse ? N / 2 : 0);
   if (e != cudaSuccess)
     return fail(&s->err, DLLM_CUDA_ERROR, "bf16 GEMM %dx%dx%d: %s", M, N, K, why ? why : cudaGetErrorString(e));
   if (fused) *fused = fuse;
@@ -560,10 +565,16 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
       head_in = s->wsp<uint8_t>(s->ws.ua);
     }
   }
-  if ((st = run_gemm(s, L, head_in, W + wl.lm_head, head_rows, c.vocab, d, &part)) != DLLM_OK) return st;
+  bool est = false;
+  if ((st = run_gemm(s, L, head_in, W + wl.lm_head, head_rows, c.vocab, d, &part, nullptr, &est, c.mask_id)) != DLLM_OK)
+    return st;
   if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
-  launch_argmax_conf(L, part.p, head_rows, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf),
-                     s->R, head_start, head_len);
+  if (est)  // the projection left one (max, sum exp, argmax) record per row and weight tile instead of logits
+    launch_estimate_merge(L, part.p, head_rows, (c.vocab + 127) / 128, s->wsp<int32_t>(s->ws.x0),
+                          s->wsp<float>(s->ws.conf), s->R, head_start, head_len);
+  else
+    launch_argmax_conf(L, part.p, head_rows, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf),
+                       s->R, head_start, head_len);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "step launch: %s", cudaGetErrorString(e));
   return DLLM_OK;

@@ -179,6 +179,30 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return warp_sum(t);
 }
 
+// Online (max, argmax, sum exp) for the greedy estimate and its confidence (Eq. 4).  Ties go to the lowest id.
+struct MaxSum {
+  float m, s;
+  int a;
+};
+__device__ __forceinline__ MaxSum merge(MaxSum p, MaxSum q) {
+  if (q.m > p.m || (q.m == p.m && q.a < p.a)) {
+    MaxSum t = p;
+    p = q;
+    q = t;
+  }
+  if (q.m > -INFINITY) p.s += q.s * expf(q.m - p.m);
+  return p;
+}
+__device__ __forceinline__ void online_add(MaxSum& t, float v, int i) {
+  if (v > t.m) {
+    t.s = t.s * expf(t.m - v) + 1.f;
+    t.m = v;
+    t.a = i;
+  } else {
+    t.s += expf(v - t.m);
+  }
+}
+
 // Three sums over the block at once (one pair of barriers); `red` holds >= 96 floats.
 __device__ __forceinline__ void block_sum3(float& a, float& b, float& c, float* red) {
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;

@@ -805,30 +805,6 @@ void launch_select_gather(const Launch& L, int dtype, const float* sim, const in
 // ------------------------------------------------------------------ greedy estimate + confidence (Eq. 4)
 // Online (max, argmax, sum exp) per thread, merged across the block.  Ties go
 // to the lowest id.  The mask id is skipped: the estimate is never [MASK].
-struct MaxSum {
-  float m, s;
-  int a;
-};
-__device__ __forceinline__ MaxSum merge(MaxSum p, MaxSum q) {
-  if (q.m > p.m || (q.m == p.m && q.a < p.a)) {
-    MaxSum t = p;
-    p = q;
-    q = t;
-  }
-  if (q.m > -INFINITY) p.s += q.s * expf(q.m - p.m);
-  return p;
-}
-
-__device__ __forceinline__ void online_add(MaxSum& t, float v, int i) {
-  if (v > t.m) {
-    t.s = t.s * expf(t.m - v) + 1.f;
-    t.m = v;
-    t.a = i;
-  } else {
-    t.s += expf(v - t.m);
-  }
-}
-
 // blk_len > 0: logits row r belongs to response row blk_start + r % blk_len of sequence r / blk_len (the rows
 // of one generation block); otherwise logits row r is carried response row r.
 __global__ void argmax_conf_kernel(const float* __restrict__ logits, int vocab, int mask_id, int32_t* __restrict__ x0,
@@ -894,6 +870,42 @@ void launch_argmax_conf(const Launch& L, const float* logits, int rows, int voca
                         float* conf, int R, int blk_start, int blk_len) {
   if (rows <= 0) return;
   launch_k(L, argmax_conf_kernel, dim3(rows), dim3(512), 0, logits, vocab, mask_id, x0, conf, R, blk_start, blk_len);
+  L.count();
+}
+
+// Merge of the per-tile (max, argmax, sum exp) records the LM-head projection writes from its epilogue
+// (records [rows][n_tiles] of {max, sum, argmax bits, -}): one warp per row, tiles in a fixed order.
+__global__ void estimate_merge_kernel(const float4* __restrict__ rec, int rows, int n_tiles, int32_t* __restrict__ x0,
+                                      float* __restrict__ conf, int R, int blk_start, int blk_len) {
+  pdl_wait();
+  pdl_trigger();
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  MaxSum t{-INFINITY, 0.f, 0x7fffffff};
+  for (int i = lane; i < n_tiles; i += 32) {
+    const float4 q = __ldcg(rec + (size_t)row * n_tiles + i);
+    t = merge(t, MaxSum{q.x, q.y, __float_as_int(q.z)});
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    MaxSum q;
+    q.m = __shfl_xor_sync(0xffffffffu, t.m, o);
+    q.s = __shfl_xor_sync(0xffffffffu, t.s, o);
+    q.a = __shfl_xor_sync(0xffffffffu, t.a, o);
+    t = merge(t, q);
+  }
+  if (lane == 0) {
+    const size_t out = blk_len > 0 ? (size_t)(row / blk_len) * R + blk_start + row % blk_len : (size_t)row;
+    x0[out] = t.a;
+    conf[out] = 1.f / t.s;
+  }
+}
+
+void launch_estimate_merge(const Launch& L, const float* records, int rows, int n_tiles, int32_t* x0, float* conf,
+                           int R, int blk_start, int blk_len) {
+  if (rows <= 0) return;
+  launch_k(L, estimate_merge_kernel, dim3((rows + 7) / 8), dim3(256), 0, reinterpret_cast<const float4*>(records), rows,
+           n_tiles, x0, conf, R, blk_start, blk_len);
   L.count();
 }
 

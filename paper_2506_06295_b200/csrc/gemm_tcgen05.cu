@@ -63,7 +63,74 @@ template <int BN>
 __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0, int n0, int tile_y, int M, int N,
                                               float* __restrict__ slab, __nv_bfloat16* __restrict__ act_out, int m_ffn) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (act_out) {
+  if (m_ffn < 0) {
+    // Estimate epilogue of the LM head (no split-K, act_out == nullptr, m_ffn = -1 - mask id): instead of 128
+    // logits per row the CTA writes one record per activation row, {max, sum exp(v - max), argmax, -} over its
+    // 128 vocabulary columns (Eq. 4; the mask id and columns past N are skipped); a merge over the tiles
+    // follows.  Staged like the SwiGLU epilogue; two threads share a row, 64 columns each.
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    constexpr int EXS = 132;
+    constexpr int CH = BN < 64 ? BN : 64;
+    const int mask_id = -1 - m_ffn, n_tiles = (N + TILE_W - 1) / TILE_W;
+    float4* rec = reinterpret_cast<float4*>(slab);
+    const int rr = threadIdx.x >> 1, half = threadIdx.x & 1;
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += CH) {
+      if (m0 + c0 >= M) break;  // uniform across the CTA
+#pragma unroll
+      for (int c = 0; c < CH; c += 16) {
+        uint32_t r[16];
+        tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + c), r);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[j]);
+      }
+      __syncthreads();
+      MaxSum t{-INFINITY, 0.f, 0x7fffffff};
+      if (rr < CH) {
+        // two passes over the thread's 64 columns: maximum and its first index, then the exponentials as four
+        // independent sums (one serial chain of dependent exponentials would dominate the epilogue)
+        const float* row = ex + rr * EXS + half * 64;
+        const int nb = n0 + half * 64;
+#pragma unroll 4
+        for (int j = 0; j < 64; j += 4) {
+          const float4 v = *reinterpret_cast<const float4*>(row + j);
+          const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int n = nb + j + q;
+            if (n < N && n != mask_id && e[q] > t.m) {
+              t.m = e[q];
+              t.a = n;
+            }
+          }
+        }
+        if (t.m > -INFINITY) {
+          float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+          for (int j = 0; j < 64; j += 4) {
+            const float4 v = *reinterpret_cast<const float4*>(row + j);
+            const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const int n = nb + j + q;
+              s4[q] += (n < N && n != mask_id) ? expf(e[q] - t.m) : 0.f;
+            }
+          }
+          t.s = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+        }
+      }
+      MaxSum o;
+      o.m = __shfl_xor_sync(0xffffffffu, t.m, 1);
+      o.s = __shfl_xor_sync(0xffffffffu, t.s, 1);
+      o.a = __shfl_xor_sync(0xffffffffu, t.a, 1);
+      t = merge(t, o);
+      const int m = m0 + c0 + rr;
+      if (rr < CH && half == 0 && m < M)
+        rec[(size_t)m * n_tiles + tile_y] = make_float4(t.m, t.s, __int_as_float(t.a), 0.f);
+      __syncthreads();
+    }
+  } else if (act_out) {
     // SwiGLU epilogue (no split-K): the tile's 128 weight rows are 64 gate rows followed by the 64 up rows
     // of the same FFN columns, so TMEM lanes 0..63 hold gate and 64..127 hold up.  The accumulator goes
     // through shared memory (every MMA has completed) 64 activation rows at a time, transposed to
@@ -247,7 +314,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   if (!have && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_EPI);
   // the whole warp must agree before the warp-collective TMEM loads
   bool warp_ok = __all_sync(0xffffffffu, have);
-  if (act_out) warp_ok = __syncthreads_and(warp_ok);  // the SwiGLU epilogue exchanges data between warps
+  if (act_out || m_ffn < 0) warp_ok = __syncthreads_and(warp_ok);  // these epilogues exchange data between warps
   if (warp_ok) {
     float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // the drained ring
     gemm_epilogue<BN>(tmem_d, ex, m0, n0, nt, M, N, part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
@@ -390,7 +457,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_pair_kernel(const __grid_consta
   const bool have = mbar_wait(smem_u32(&accum_bar), 0u, abortp);
   if (!have && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_EPI);
   bool warp_ok = __all_sync(0xffffffffu, have);
-  if (act_out) warp_ok = __syncthreads_and(warp_ok);
+  if (act_out || m_ffn < 0) warp_ok = __syncthreads_and(warp_ok);
   if (warp_ok) {
     float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // the drained ring
     gemm_epilogue<BN>(tmem_d, ex, m0, n0, (int)blockIdx.x, M, N, part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
@@ -592,6 +659,10 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
   if (M <= 0 || N <= 0) return cudaSuccess;
   if (K <= 0 || (K & 7) || ((uintptr_t)A & 15) || ((uintptr_t)W & 15)) {
     if (err) *err = e_shape;
+    return cudaErrorInvalidValue;
+  }
+  if (!act_out && m_ffn < 0 && (plan.S_max != 1 || ((uintptr_t)part & 15))) {
+    if (err) *err = "the estimate epilogue needs an unsplit plan";
     return cudaErrorInvalidValue;
   }
   if (act_out && (plan.S_max != 1 || N != 2 * m_ffn || (m_ffn & 63) || ((uintptr_t)act_out & 7))) {

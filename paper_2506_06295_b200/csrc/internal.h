@@ -142,6 +142,9 @@ void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer,
 // (x0, conf) per response row from fp32 logits; the mask id never wins.
 void launch_argmax_conf(const Launch& L, const float* logits, int rows, int vocab, int mask_id, int32_t* x0,
                         float* conf, int R = 0, int blk_start = 0, int blk_len = 0);
+// x0 / conf from the per-tile records of the LM head's estimate epilogue; row mapping as launch_argmax_conf
+void launch_estimate_merge(const Launch& L, const float* records, int rows, int n_tiles, int32_t* x0, float* conf,
+                           int R = 0, int blk_start = 0, int blk_len = 0);
 // dst[b * len + i] = src[b * R + start + i], rows of d elements (d * element size a multiple of 16 bytes)
 void launch_gather_block_rows(const Launch& L, int dtype, const void* src, void* dst, int B, int R, int start, int len,
                               int d);
@@ -177,6 +180,8 @@ Partials make_partials(const float* p, int M, int N, const GemmPlan& plan);
 // Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
 // act_out != nullptr (unsplit plan, W = gate / up rows interleaved in blocks of 64, N = 2 * m_ffn): instead of
 // fp32 slabs the epilogue writes silu(gate) * up as bf16 [M, m_ffn].
+// act_out == nullptr and m_ffn = -1 - mask_id (unsplit plan): instead of logits the epilogue writes, at `part`,
+// one {max, sum exp, argmax, -} record per row and weight tile, [M][ceil(N / 128)] float4 (see launch_estimate_merge).
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
                              const GemmPlan& plan, const char** err, void* act_out = nullptr, int m_ffn = 0);
 
