@@ -169,15 +169,22 @@ __device__ __forceinline__ void combine_row(const float* __restrict__ o_part, co
     if (s < S) L += wgt[s] * ml[s].y;
   }
   const float inv = 1.f / L;
-  for (int d = lane; d < hd; d += 32) {
-    float v[MAXS];
+  // hd <= 128: up to four trips; the partial outputs of all of them are fetched before the first store
+  float v[4][MAXS];
 #pragma unroll
-    for (int s = 0; s < MAXS; ++s) v[s] = o_part[((size_t)min(s, S - 1) * total + rh) * hd + d];
+  for (int t = 0; t < 4; ++t) {
+    const int d = lane + 32 * t;
+#pragma unroll
+    for (int s = 0; s < MAXS; ++s) v[t][s] = d < hd ? o_part[((size_t)min(s, S - 1) * total + rh) * hd + d] : 0.f;
+  }
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    const int d = lane + 32 * t;
     float acc = 0.f;
 #pragma unroll
     for (int s = 0; s < MAXS; ++s)
-      if (s < S) acc += wgt[s] * v[s];
-    o[rh * hd + d] = __float2bfloat16_rn(acc * inv);
+      if (s < S) acc += wgt[s] * v[t][s];
+    if (d < hd) o[rh * hd + d] = __float2bfloat16_rn(acc * inv);
   }
 }
 

@@ -122,17 +122,29 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
   }
   // Q tile: plain 16-byte loads into the swizzled layout (rows of other heads /
   // past the end are zero)
-  for (int e = tid; e < AT_ROWS * (HD / 8); e += 128) {
-    const int r = e / (HD / 8), dc = e - r * (HD / 8);
-    const int vr = row0 + r;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (vr < n_rows) {
-      const int qi = vr / G, g = vr - qi * G;
-      v = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
+  {
+    constexpr int PER = AT_ROWS * (HD / 8) / 128;  // 16-byte chunks per thread: all loads first, then the stores
+    uint4 qv[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int e = tid + i * 128;
+      const int r = e / (HD / 8), dc = e - r * (HD / 8);
+      const int vr = row0 + r;
+      qv[i] = make_uint4(0, 0, 0, 0);
+      if (vr < n_rows) {
+        const int qi = vr / G, g = vr - qi * G;
+        qv[i] = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
+      }
     }
-    *reinterpret_cast<uint4*>(q_gen + tile_off<AT_ROWS>(r, dc)) = v;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int e = tid + i * 128;
+      const int r = e / (HD / 8), dc = e - r * (HD / 8);
+      *reinterpret_cast<uint4*>(q_gen + tile_off<AT_ROWS>(r, dc)) = qv[i];
+    }
   }
   at_sync();
+  if (tid == 0) timeline_mark(1);  // Q staged
   // Q fragments of this warp's 16 rows stay in registers
   uint32_t qf[HD / 16][4];
 #pragma unroll
@@ -152,6 +164,7 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
     ok = mbar_wait(smem_u32(&full_bar[st]), ((it0 + (uint32_t)t) >> 1) & 1u, abort_flag);
     ok = at_sync_and(ok);                     // uniform over the 128 threads: nobody is left behind at a barrier
     if (!ok) break;
+    if (tid == 0) timeline_mark(2 + (t < 5 ? t : 5));  // K/V tile t has landed
     const uint32_t k_s = kv_s + st * STAGE_BYTES, v_s = k_s + TILE_BYTES;
     // ---- S = Q K^T for 16 rows x 64 keys
     float sacc[AT_KEYS / 8][4];
@@ -233,6 +246,7 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
     drain_delay();
     return false;
   }
+  if (tid == 0) timeline_mark(8);  // all tiles done
   // ---- epilogue
 #pragma unroll
   for (int h2 = 0; h2 < 2; ++h2) {

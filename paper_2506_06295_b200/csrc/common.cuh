@@ -36,6 +36,7 @@ enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_E
 #ifndef DLLM_TIMELINE
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #define DLLM_TIMELINE_HOOKS(stem)
+__device__ __forceinline__ void timeline_mark(int) {}
 #else
 // Timeline build (python -m paper_2506_06295_b200.timeline): thread 0 of every CTA records the global timer
 // before and after the dependency wait, so that a replayed CUDA graph yields, per kernel, when its CTAs became
@@ -67,6 +68,21 @@ __device__ __forceinline__ void pdl_wait() {
       g_timeline[4 * i + 2] = t1;
       g_timeline[4 * i + 3] = smid | ((unsigned long long)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) << 32);
     }
+  }
+}
+// A point inside a kernel (called by one thread per CTA): the same record with the mark in the top four bits of
+// the first word and the time in the second and third.
+__device__ __forceinline__ void timeline_mark(int id) {
+  if (g_timeline == nullptr) return;
+  const unsigned long long t = timeline_now();
+  const unsigned int i = atomicAdd(&g_timeline_n, 1u);
+  if (i < TIMELINE_CAP) {
+    g_timeline[4 * i] = (unsigned long long)gridDim.x | ((unsigned long long)gridDim.y << 16) |
+                        ((unsigned long long)gridDim.z << 32) | ((unsigned long long)(blockDim.x & 0xfff) << 48) |
+                        ((unsigned long long)id << 60);
+    g_timeline[4 * i + 1] = t;
+    g_timeline[4 * i + 2] = t;
+    g_timeline[4 * i + 3] = (unsigned long long)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) << 32;
   }
 }
 // One pair of host entry points per translation unit: set the record array (device, 32 bytes x 2^20; NULL = off)
@@ -200,6 +216,20 @@ __device__ __forceinline__ void online_add(MaxSum& t, float v, int i) {
     t.a = i;
   } else {
     t.s += expf(v - t.m);
+  }
+}
+
+// Copy of one row of nvec 16-byte words by the whole block: four loads in flight per thread before the first
+// store (a plain load-store loop waits a memory round trip per trip).
+__device__ __forceinline__ void copy_row16(const uint4* __restrict__ src, uint4* __restrict__ dst, int nvec) {
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x * 4) {
+    uint4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (i + k * (int)blockDim.x < nvec) v[k] = src[i + k * blockDim.x];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (i + k * (int)blockDim.x < nvec) dst[i + k * blockDim.x] = v[k];
   }
 }
 

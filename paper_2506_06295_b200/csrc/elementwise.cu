@@ -110,7 +110,7 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
 void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gain, void* out, int d, float eps, int c0,
                     int c1) {
   if (c1 <= c0) return;
-  DLLM_DISPATCH(dtype, (launch_k(L, rmsnorm_kernel<T>, dim3(c1 - c0), dim3(256), 0, x, gain, (T*)out, d, eps, c0)));
+  DLLM_DISPATCH(dtype, (launch_k(L, rmsnorm_kernel<T>, dim3(c1 - c0), dim3(row_threads(d)), 0, x, gain, (T*)out, d, eps, c0)));
   L.count();
 }
 
@@ -425,10 +425,8 @@ __global__ void gather_rows_kernel(const T* __restrict__ src, const int32_t* __r
   pdl_wait();
   pdl_trigger();
   const size_t r = blockIdx.x;
-  const uint4* s = reinterpret_cast<const uint4*>(src + (size_t)act[r] * d);
-  uint4* o = reinterpret_cast<uint4*>(dst + r * d);
-  const int nvec = d * (int)sizeof(T) / 16;
-  for (int i = threadIdx.x; i < nvec; i += blockDim.x) o[i] = s[i];
+  copy_row16(reinterpret_cast<const uint4*>(src + (size_t)act[r] * d), reinterpret_cast<uint4*>(dst + r * d),
+             d * (int)sizeof(T) / 16);
 }
 
 void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32_t* act, void* dst, int rows, int d) {
@@ -506,7 +504,7 @@ void launch_scatter_rows(const Launch& L, int dtype, Partials part, const int32_
                          Geo g, int rows, int width) {
   if (rows <= 0) return;
   DLLM_DISPATCH(dtype,
-                (launch_k(L, scatter_rows_kernel<T>, dim3(rows), dim3(128), 0, part, act, c_base, (T*)cache_layer, g, width)));
+                (launch_k(L, scatter_rows_kernel<T>, dim3(rows), dim3(row_threads(width)), 0, part, act, c_base, (T*)cache_layer, g, width)));
   L.count();
 }
 
@@ -632,7 +630,7 @@ void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer,
                      int c1) {
   if (c1 <= c0) return;
   DLLM_DISPATCH(dtype,
-                (launch_k(L, residual_kernel<T>, dim3(c1 - c0), dim3(128), 0, x, (const T*)Ac_layer, (const T*)Fc_layer, g, c0)));
+                (launch_k(L, residual_kernel<T>, dim3(c1 - c0), dim3(row_threads(g.d)), 0, x, (const T*)Ac_layer, (const T*)Fc_layer, g, c0)));
   L.count();
 }
 
@@ -674,7 +672,7 @@ __global__ void embed_norm_kernel(const T* __restrict__ E, const int32_t* __rest
 void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, const float* gain,
                        void* u, Geo g, int c0, int c1, float eps) {
   if (c1 <= c0) return;
-  DLLM_DISPATCH(dtype, (launch_k(L, embed_norm_kernel<T>, dim3(c1 - c0), dim3(256), 0, (const T*)E, tokens, x, gain,
+  DLLM_DISPATCH(dtype, (launch_k(L, embed_norm_kernel<T>, dim3(c1 - c0), dim3(row_threads(g.d)), 0, (const T*)E, tokens, x, gain,
                                  (T*)u, g, c0, eps)));
   L.count();
 }
@@ -785,10 +783,8 @@ __global__ void select_gather_kernel(const float* __restrict__ sim, const int32_
     __syncthreads();
   }
   const int c = ridx < np ? g.B * R + b * g.P + ridx : b * R + my_j;
-  const uint4* s4 = reinterpret_cast<const uint4*>(u + (size_t)c * g.d);
-  uint4* o4 = reinterpret_cast<uint4*>(ua + ((size_t)b * a_seq + ridx) * g.d);
-  const int nvec = g.d * (int)sizeof(T) / 16;
-  for (int i = threadIdx.x; i < nvec; i += blockDim.x) o4[i] = s4[i];
+  copy_row16(reinterpret_cast<const uint4*>(u + (size_t)c * g.d),
+             reinterpret_cast<uint4*>(ua + ((size_t)b * a_seq + ridx) * g.d), g.d * (int)sizeof(T) / 16);
 }
 
 void launch_select_gather(const Launch& L, int dtype, const float* sim, const int32_t* forced, int mode, int ksel,
@@ -918,10 +914,8 @@ __global__ void gather_block_rows_kernel(const T* __restrict__ src, T* __restric
   pdl_wait();
   pdl_trigger();
   const int r = blockIdx.x, b = r / len, i = r - b * len;
-  const uint4* s4 = reinterpret_cast<const uint4*>(src + ((size_t)b * R + start + i) * d);
-  uint4* o4 = reinterpret_cast<uint4*>(dst + (size_t)r * d);
-  const int nvec = d * (int)sizeof(T) / 16;
-  for (int v = threadIdx.x; v < nvec; v += blockDim.x) o4[v] = s4[v];
+  copy_row16(reinterpret_cast<const uint4*>(src + ((size_t)b * R + start + i) * d),
+             reinterpret_cast<uint4*>(dst + (size_t)r * d), d * (int)sizeof(T) / 16);
 }
 
 void launch_gather_block_rows(const Launch& L, int dtype, const void* src, void* dst, int B, int R, int start, int len,

@@ -64,6 +64,8 @@ def collect(workload: str, kind: str):
         a = bufs[st].cpu().numpy().reshape(-1, 4)[:n]
         recs += [(int(t1), int(t0), int(tag), st) for tag, t0, t1, _ in a]
         getattr(dllm.lib, "dllm_timeline_set_" + st)(None)
+    marks = [r for r in recs if (r[2] >> 60)]
+    recs = [r for r in recs if not (r[2] >> 60)]
     recs.sort()
     # CTAs of one launch share (file, grid, block) and are released together; later waves of a large grid are
     # released as earlier CTAs exit, so a gap is allowed inside a launch as long as the signature stays
@@ -85,6 +87,15 @@ def collect(workload: str, kind: str):
                     "ctas": L["n"], "start_us": (L["t1"] - base) / 1e3,
                     "resident_before_us": (L["t1"] - L["t0min"]) / 1e3, "last_cta_us": (L["t0max"] - L["t1"]) / 1e3,
                     "dur_us": (nxt - L["t1"]) / 1e3 if nxt is not None else 0.0})
+    # marks inside kernels: time after the release of the launch they belong to (same signature, latest release before)
+    sig = lambda tag: tag & ((1 << 60) - 1)
+    for t1, _t0, tag, st in marks:
+        cands = [L for L in launches if L["key"][0] == st and (L["key"][1] & ((1 << 60) - 1)) == sig(tag) and L["t1"] <= t1]
+        if cands:
+            cands[-1].setdefault("marks", {}).setdefault(tag >> 60, []).append((t1 - cands[-1]["t1"]) / 1e3)
+    for o, L in zip(out, launches):
+        if "marks" in L:
+            o["marks"] = {int(k): [min(v), sum(v) / len(v), max(v)] for k, v in sorted(L["marks"].items())}
     return out, cfg.n_layers, truncated
 
 
@@ -111,6 +122,8 @@ def main(argv=None) -> int:
             print(f"  {o['file']:15s} grid {str(tuple(o['grid'])):16s} x {o['block']:4d}  ctas {o['ctas']:5d}  "
                   f"dur {o['dur_us']:8.2f} us  resident {o['resident_before_us']:7.2f} us before release, "
                   f"last CTA in {o['last_cta_us']:+.2f} us")
+            for k, (lo_, av, hi) in o.get("marks", {}).items():
+                print(f"      mark {k}: min {lo_:6.2f}  mean {av:6.2f}  max {hi:6.2f} us after the release")
     agg = collections.OrderedDict()
     for o in out:
         a = agg.setdefault((o["file"], tuple(o["grid"]), o["block"]), [0, 0.0])
