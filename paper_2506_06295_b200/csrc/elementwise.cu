@@ -775,7 +775,54 @@ __global__ void select_gather_kernel(const float* __restrict__ sim, const int32_
   const int np = refresh_prompt ? g.P : 0;
   const int a_seq = np + ksel;
   const bool leader = ridx == 0;
-  if (ridx >= np || leader) {
+  if (mode == 1 && R <= (int)blockDim.x && (ridx >= np || leader)) {
+    // One key per thread (the usual case, R <= 256): key -> shared memory, rank against all keys, one ballot
+    // word per warp, position among the selected rows from the ballot words: three barriers in all.
+    uint32_t* words = reinterpret_cast<uint32_t*>(keys + R);
+    const int j = threadIdx.x;
+    unsigned long long kj = ~0ull;
+    if (j < R) {
+      const float s = __ldcg(sim + (size_t)b * R + j);
+      const float qf = fminf(fmaxf(rintf(s * 1048576.0f), -2147483520.0f), 2147483520.0f);
+      const long long q = (s == s) ? (long long)qf + (1ll << 31) : 0ll;
+      kj = ((unsigned long long)q << 32) | (unsigned)j;
+      keys[j] = kj;
+    }
+    __syncthreads();
+    int rank = 0;
+    if (j < R) {
+#pragma unroll 8
+      for (int i = 0; i + 1 < R; i += 2) {
+        const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(keys + i);
+        rank += (kk.x < kj) + (kk.y < kj);
+      }
+      if (R & 1) rank += (keys[R - 1] < kj);
+    }
+    const bool f = j < R && rank < ksel;
+    const unsigned bal = __ballot_sync(0xffffffffu, f);
+    if ((j & 31) == 0) words[j >> 5] = bal;
+    __syncthreads();
+    int r = -1;
+    if (f) {
+      r = __popc(bal & ((1u << (j & 31)) - 1u));
+      for (int w = 0; w < (j >> 5); ++w) r += __popc(words[w]);
+      if (r == ridx - np) my_j = j;
+    }
+    if (leader) {
+      if (j < R) {
+        inv[(size_t)b * R + j] = r >= 0 ? b * a_seq + np + r : -1;
+        if (r >= 0) {
+          sel[(size_t)b * R + r] = j;
+          act[(size_t)b * a_seq + np + r] = b * R + j;
+        }
+      }
+      for (int i = threadIdx.x; i < np; i += blockDim.x) {
+        act[(size_t)b * a_seq + i] = g.B * R + b * g.P + i;
+        inv[(size_t)g.B * R + (size_t)b * g.P + i] = b * a_seq + i;
+      }
+    }
+    __syncthreads();
+  } else if (ridx >= np || leader) {
     const int32_t* slot = select_sequence(keys, sim, forced, mode, ksel, sel, act, inv, g, np, b, leader);
     if (ridx >= np)
       for (int j = threadIdx.x; j < R; j += blockDim.x)
