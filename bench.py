@@ -233,6 +233,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llada8b", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-timeline", action="store_true", help="skip the in-graph GEMM figure (a second process)")
     ap.add_argument("--full-steps", type=int, default=6, help="timed full-recompute steps for the speedup figure")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (small case for ncu "
                     "captures: same widths, a few GB of weights); the bench line then names the reduced depth")
@@ -397,17 +398,45 @@ def main():
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
-    # ---- per-kernel times: same K steps, launched kernel by kernel with event pairs --------------
+    # ---- per-kernel times: the same K steps with an event pair around every GEMM and attention launch.
+    # The pairs are event-record nodes of each step's graph (no host latency inside a pair, no overlap between
+    # launches); each step ends with a synchronisation that reads them back, so the replay's own time is the
+    # sum of per-step event pairs, not a span that would include those host gaps.
     ses.set_prompt(prompt)
     ses.profile(True)
-    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    p0.record(stream)
-    run_steps(K)
-    p1.record(stream)
+    for k in (wl.steps, wl.steps - 1, wl.steps - 2):        # instantiate the profiling graphs outside the replay
+        ses.step_scheduled(k, wl.steps, wl.Kp, wl.Kr, wl.rho)
+    ses.profile(False)
+    ses.set_prompt(prompt)
+    ses.profile(True)
+    step_ev = []
+
+    def open_step(i):
+        a = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        step_ev.append([a, None])
+    for i in range(K):
+        k = wl.steps - (i % wl.steps)
+        if i and k == wl.steps:
+            ses.set_prompt(prompt)
+        open_step(i)
+        ses.step_scheduled(k, wl.steps, wl.Kp, wl.Kr, wl.rho)
+        bs, nt = block_plan(wl.steps - k, wl.steps, wl.gen_len, wl.block_len)
+        ses.remask_low_confidence(bs, wl.block_len, nt)
+        b = torch.cuda.Event(enable_timing=True)
+        b.record(stream)
+        step_ev[-1][1] = b
     ses.sync()
-    ms_replay = p0.elapsed_time(p1)
+    ms_replay = sum(a.elapsed_time(b) for a, b in step_ev)
     g = ses.profile_read(0)
     at = ses.profile_read(1)
+    ses.profile(False)
+
+    # algorithmic GEMM bytes of ONE adaptive partial step (the library's own count), for the in-graph figure
+    ses.profile(True)
+    ses.step_cached(False, False, wl.rho)
+    ses.sync()
+    partial_gemm_bytes = ses.profile_read(0)["bytes"]
     ses.profile(False)
 
     # max over ranks
@@ -451,10 +480,13 @@ def main():
                      "attention": {"ms_total": at["ms"], "launches": at["launches"],
                                    "gbs": at["bytes"] / (at["ms"] / 1e3) / 1e9 if at["ms"] > 0 else 0.0,
                                    "tflops": at["flops"] / (at["ms"] / 1e3) / 1e12 if at["ms"] > 0 else 0.0},
-                     "how": "CUDA-event pairs around every GEMM launch in a kernel-by-kernel replay of the same K steps; "
-                            "share = GEMM event time / event time of that replay"},
+                     "how": "CUDA-event pairs around every GEMM launch (event-record nodes in the step graphs, launches "
+                            "serialised, no programmatic overlap) in a replay of the same K steps; share = GEMM event "
+                            "time / summed per-step event time of that replay"},
         "unmasked_tokens": int((final_tokens[:, wl.prompt_len:] != cfg.mask_id).sum()),
     }
+    if world == 1 and not args.no_timeline:
+        line["roofline"]["in_graph"] = in_graph_gemm(args.workload, partial_gemm_bytes, peaks)
     if not args.no_cpu_baseline:
         t = time_oracle(wl, budget_s=25.0, steps=K)
         line["cpu_baseline"] = {"value": t["tokens_per_s"], "unit": "tokens/s", "cores": t["cores"], "kind": "oracle",
@@ -462,6 +494,32 @@ def main():
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def in_graph_gemm(workload, gemm_bytes, peaks):
+    """GEMM time INSIDE the replayed graph of one adaptive partial step (programmatic dependent launch, warm L2),
+    from the device timestamps of the timeline build, in a process of its own after this one has freed nothing it
+    needs: achieved = the step's algorithmic GEMM bytes / the summed in-graph durations of its GEMM launches.
+    Reported beside the event-pair figure, which serialises the launches.  None if the run fails."""
+    try:
+        with tempfile.TemporaryDirectory() as td:
+            out = os.path.join(td, "tl.json")
+            r = subprocess.run([sys.executable, "-m", "paper_2506_06295_b200.timeline", "--workload", workload,
+                                "--kind", "partial", "--json", out], cwd=ROOT, capture_output=True, text=True, timeout=600)
+            if r.returncode != 0:
+                return None
+            launches = json.load(open(out))
+        gemm = [o for o in launches if o["file"].startswith("gemm")]
+        us = sum(o["dur_us"] for o in gemm)
+        total = launches[-1]["start_us"]
+        gbs = gemm_bytes / (us * 1e-6) / 1e9
+        return {"achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "gemm_us": us, "gemm_launches": len(gemm),
+                "step_us": total, "gemm_share_of_step": us / max(total, 1e-9),
+                "how": "one adaptive partial step replayed as a CUDA graph in the timeline build of the library: "
+                       "per launch, device time from its predecessor's completion to its own (globaltimer at "
+                       "griddepcontrol.wait of every CTA)"}
+    except Exception:
+        return None
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch from the ncu capture summarised under

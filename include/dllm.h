@@ -235,9 +235,12 @@ dllm_status dllm_session_use_pdl(dllm_session* s, int enable);
  * by kernel like the other step kinds, which measured faster on B200. */
 dllm_status dllm_session_use_layer_kernel(dllm_session* s, int enable);
 
-/* Per-kernel timing.  While enabled, steps are launched kernel by kernel (no
- * graph replay) and every projection GEMM (class 0) and attention launch
- * (class 1) is bracketed by CUDA events on the caller's stream.  _profile_read
+/* Per-kernel timing.  While enabled, every projection GEMM (class 0) and
+ * attention launch (class 1) is bracketed by CUDA events on the caller's stream
+ * and no launch overlaps its predecessor (no programmatic dependent launch).
+ * With CUDA graphs on, the event records are nodes of the step's graph, so no
+ * host latency falls between a pair and its kernel; every step then ends with
+ * a stream synchronisation that reads the pairs back.  _profile_read
  * synchronises the device and returns, for one class, the summed event time,
  * the number of launches, and the algorithmic bytes and FLOPs of those launches
  * (GEMM: W and A once in, one fp32 result out; attention: K, V, Q in, O out).

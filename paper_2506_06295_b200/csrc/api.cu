@@ -192,7 +192,9 @@ struct StepKey {
   int variant = 0;
   uint64_t ksel_sig = 0;  // per-layer row counts (cross-layer allocation of rho)
   int head_start = 0, head_len = 0;  // prediction restricted to one block of the response (0 rows: all of it)
+  int prof = 0;                      // graph with event-record nodes around the GEMM and attention launches
   bool operator<(const StepKey& o) const {
+    if (prof != o.prof) return prof < o.prof;
     if (head_start != o.head_start) return head_start < o.head_start;
     if (head_len != o.head_len) return head_len < o.head_len;
     if (variant != o.variant) return variant < o.variant;
@@ -225,17 +227,26 @@ struct dllm_session {
   struct GraphEntry {
     cudaGraphExec_t exec;
     uint64_t kernels;
+    size_t rec0 = 0, rec1 = 0;  // profiling graphs: their event pairs are graph_prof[rec0 .. rec1)
   };
   std::map<StepKey, GraphEntry> graphs;
   std::string err;
-  // profiling: event pairs around GEMM (class 0) and attention (class 1) launches
+  // profiling: event pairs around GEMM (class 0) and attention (class 1) launches.  Launched kernel by kernel the
+  // pairs are recorded by the host; inside a captured step they become event-record nodes of the graph (no host
+  // latency between a pair and its kernel), are re-recorded at every replay and read back after it.
   struct ProfRec {
     int cls;
     cudaEvent_t a, b;
     double bytes, flops;
   };
+  struct ProfSum {
+    double ms = 0, bytes = 0, flops = 0;
+    uint64_t launches = 0;
+  };
   bool profiling = false;
-  std::vector<ProfRec> prof;
+  std::vector<ProfRec> prof;        // recorded by the host, one pair per launch
+  std::vector<ProfRec> graph_prof;  // owned by profiling graphs
+  ProfSum prof_sum[2];              // read back from graph replays
   std::vector<cudaEvent_t> event_pool;
   cudaEvent_t take_event() {
     if (!event_pool.empty()) {
@@ -247,15 +258,34 @@ struct dllm_session {
     cudaEventCreate(&e);
     return e;
   }
+  // inside a stream capture the record becomes an event-record node of the graph (a plain cudaEventRecord would
+  // only express a dependency of the capture)
+  static void record(cudaEvent_t e, cudaStream_t st) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) == cudaSuccess && cs == cudaStreamCaptureStatusActive)
+      cudaEventRecordWithFlags(e, st, cudaEventRecordExternal);
+    else
+      cudaEventRecord(e, st);
+  }
   void prof_begin(int cls, double bytes, double flops, cudaStream_t st) {
     if (!profiling) return;
     ProfRec r{cls, take_event(), take_event(), bytes, flops};
-    cudaEventRecord(r.a, st);
+    record(r.a, st);
     prof.push_back(r);
   }
   void prof_end(cudaStream_t st) {
     if (!profiling) return;
-    cudaEventRecord(prof.back().b, st);
+    record(prof.back().b, st);
+  }
+
+  void drop_graphs() {
+    for (auto& kv : graphs) cudaGraphExecDestroy(kv.second.exec);
+    graphs.clear();
+    for (auto& r : graph_prof) {
+      event_pool.push_back(r.a);
+      event_pool.push_back(r.b);
+    }
+    graph_prof.clear();
   }
 
   size_t es() const { return esize(m->cfg); }
@@ -612,7 +642,7 @@ dllm_status run_step(dllm_session* s, int rp, int rr, const float* rhos, int n_r
                     s->forced_count[l], ksels[l]);
   cudaStream_t stream = (cudaStream_t)stream_v;
   dllm_status st = DLLM_OK;
-  const bool graph_ok = s->use_graphs && !s->profiling && stream != nullptr && stream != cudaStreamLegacy;
+  const bool graph_ok = s->use_graphs && stream != nullptr && stream != cudaStreamLegacy;
   if (head_len < 0 || head_start < 0 || head_start + head_len > s->R)
     return fail(&s->err, DLLM_INVALID_ARG, "block [%d, %d) outside the response", head_start, head_start + head_len);
   if (head_len == s->R) head_start = head_len = 0;  // the whole response: the ordinary step
@@ -622,14 +652,19 @@ dllm_status run_step(dllm_session* s, int rp, int rr, const float* rhos, int n_r
     st = enqueue_step(s, rp, rr, ksels, stream, head_start, head_len);
   } else {
     StepKey key{rp, rr, ksels[0], forced_signature(s), s->sel_strategy * 4 + s->sel_metric * 2 + s->v_selected_only,
-                uniform ? 0 : sig, head_start, head_len};
+                uniform ? 0 : sig, head_start, head_len, s->profiling ? 1 : 0};
     auto it = s->graphs.find(key);
     if (it == s->graphs.end()) {
       cudaGraph_t graph = nullptr;
       CU_TRY(&s->err, cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal));
       const uint64_t before = s->launches;
+      const size_t host_recs = s->prof.size();
       st = enqueue_step(s, rp, rr, ksels, stream, head_start, head_len);
       cudaError_t e = cudaStreamEndCapture(stream, &graph);
+      // event pairs recorded during the capture belong to the graph
+      const size_t rec0 = s->graph_prof.size();
+      s->graph_prof.insert(s->graph_prof.end(), s->prof.begin() + host_recs, s->prof.end());
+      s->prof.resize(host_recs);
       if (st != DLLM_OK) {
         if (graph) cudaGraphDestroy(graph);
         return st;
@@ -641,10 +676,23 @@ dllm_status run_step(dllm_session* s, int rp, int rr, const float* rhos, int n_r
       if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "graph instantiate: %s", cudaGetErrorString(e));
       const uint64_t kernels = s->launches - before;
       s->launches = before;  // counted at every replay instead
-      it = s->graphs.emplace(key, dllm_session::GraphEntry{exec, kernels}).first;
+      it = s->graphs.emplace(key, dllm_session::GraphEntry{exec, kernels, rec0, s->graph_prof.size()}).first;
     }
     CU_TRY(&s->err, cudaGraphLaunch(it->second.exec, stream));
     s->launches += it->second.kernels;
+    if (s->profiling && it->second.rec1 > it->second.rec0) {
+      CU_TRY(&s->err, cudaStreamSynchronize(stream));
+      for (size_t i = it->second.rec0; i < it->second.rec1; ++i) {
+        const dllm_session::ProfRec& r = s->graph_prof[i];
+        float t = 0.f;
+        CU_TRY(&s->err, cudaEventElapsedTime(&t, r.a, r.b));
+        dllm_session::ProfSum& acc = s->prof_sum[r.cls];
+        acc.ms += t;
+        acc.bytes += r.bytes;
+        acc.flops += r.flops;
+        ++acc.launches;
+      }
+    }
   }
   if (st != DLLM_OK) return st;
   s->valid = true;
@@ -1072,8 +1120,7 @@ dllm_status dllm_session_use_graphs(dllm_session* s, int enable) {
 dllm_status dllm_session_use_pdl(dllm_session* s, int enable) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
   if ((enable != 0) != s->use_pdl) {
-    for (auto& kv : s->graphs) cudaGraphExecDestroy(kv.second.exec);
-    s->graphs.clear();
+    s->drop_graphs();
   }
   s->use_pdl = enable != 0;
   return DLLM_OK;
@@ -1109,8 +1156,7 @@ dllm_status dllm_session_use_layer_kernel(dllm_session* s, int enable) {
 dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
   if ((enable != 0) != s->simt_gemm) {
-    for (auto& kv : s->graphs) cudaGraphExecDestroy(kv.second.exec);
-    s->graphs.clear();
+    s->drop_graphs();
   }
   s->simt_gemm = enable != 0;
   return DLLM_OK;
@@ -1124,6 +1170,7 @@ dllm_status dllm_session_profile(dllm_session* s, int enable) {
     s->event_pool.push_back(r.b);
   }
   s->prof.clear();
+  s->prof_sum[0] = s->prof_sum[1] = dllm_session::ProfSum{};
   s->profiling = enable != 0;
   return DLLM_OK;
 }
@@ -1133,8 +1180,8 @@ dllm_status dllm_session_profile_read(dllm_session* s, int cls, double* total_ms
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
   if (cls < 0 || cls > 1) return fail(&s->err, DLLM_INVALID_ARG, "class must be 0 (GEMM) or 1 (attention)");
   CU_TRY(&s->err, cudaDeviceSynchronize());
-  double ms = 0, by = 0, fl = 0;
-  uint64_t cnt = 0;
+  double ms = s->prof_sum[cls].ms, by = s->prof_sum[cls].bytes, fl = s->prof_sum[cls].flops;
+  uint64_t cnt = s->prof_sum[cls].launches;
   for (auto& r : s->prof) {
     if (r.cls != cls) continue;
     float t = 0.f;
