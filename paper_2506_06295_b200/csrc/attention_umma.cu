@@ -93,6 +93,7 @@ struct UaSmem {
 template <int HD>
 __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
                                                         const __grid_constant__ CUtensorMap tmV,
+                                                        const __grid_constant__ CUtensorMap tmQ, int q_by_tma,
                                                         const __nv_bfloat16* __restrict__ q,
                                                         __nv_bfloat16* __restrict__ o, float* __restrict__ o_part,
                                                         float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv,
@@ -103,7 +104,7 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
   constexpr uint32_t TMEM_COLS = 256;  // S: columns 0..127, O_t: columns 128..128+HD-1
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t kv_full[2];
-  __shared__ __align__(8) uint64_t bar_s, bar_o;
+  __shared__ __align__(8) uint64_t bar_s, bar_o, bar_q;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
@@ -130,6 +131,7 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
     mbar_init(smem_u32(&kv_full[1]), 1);
     mbar_init(smem_u32(&bar_s), 1);
     mbar_init(smem_u32(&bar_o), 1);
+    mbar_init(smem_u32(&bar_q), 1);
     mbar_fence_init();
     prefetch_tensormap(&tmK);
     prefetch_tensormap(&tmV);
@@ -164,22 +166,46 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
       }
   };
   if (tid == 0) {
+    if (q_by_tma) {
+      // one query head per KV head: the tile's rows are consecutive rows of q, one box per 64-column panel
+      // (rows past this sequence's end belong to no live row: whatever lands there is never written back)
+      const uint32_t qb = smem_u32(&bar_q);
+      mbar_expect_tx(qb, SM::Q_BYTES);
+#pragma unroll
+      for (int p = 0; p < PANELS; ++p) tma_load_2d(q_s + p * (UA_ROWS * 128), &tmQ, qb, kh * HD + p * 64, b * a_seq + row0);
+    }
     issue(0);
     if (n_tiles > 1) issue(1);
   }
+  if (!q_by_tma) {
   // Q tile: 16-byte loads into the swizzled panel layout (rows past the end are zero)
-  for (int e = tid; e < UA_ROWS * (HD / 8); e += 128) {
-    const int r = e / (HD / 8), dc = e - r * (HD / 8);
-    const int vr = row0 + r;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (vr < n_rows) {
-      const int qi = vr / G, g = vr - qi * G;
-      v = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
+  // (eight loads in flight per thread before the first store: a load-store loop would wait one round trip per trip)
+  constexpr int Q_CHUNKS = UA_ROWS * (HD / 8) / 128;  // 16-byte chunks per thread
+#pragma unroll 1
+  for (int i0 = 0; i0 < Q_CHUNKS; i0 += 8) {
+    uint4 qv[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int e = tid + (i0 + i) * 128;
+      const int r = e / (HD / 8), dc = e - r * (HD / 8);
+      const int vr = row0 + r;
+      qv[i] = make_uint4(0, 0, 0, 0);
+      if (vr < n_rows) {
+        const int qi = vr / G, g = vr - qi * G;
+        qv[i] = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
+      }
     }
-    *reinterpret_cast<uint4*>(base_gen + tile_off<UA_ROWS>(r, dc)) = v;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int e = tid + (i0 + i) * 128;
+      const int r = e / (HD / 8), dc = e - r * (HD / 8);
+      *reinterpret_cast<uint4*>(base_gen + tile_off<UA_ROWS>(r, dc)) = qv[i];
+    }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic stores -> MMA reads of shared memory
+  }
   __syncthreads();
+  if (tid == 0) timeline_mark(1);  // Q staged (or requested)
 
   constexpr uint32_t idesc_s = make_idesc(UA_ROWS, UA_KEYS);
   constexpr uint32_t idesc_o = make_idesc(UA_ROWS, HD) | (1u << 16);  // B operand (V) is MN-major
@@ -206,7 +232,10 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
   // grown by more than RESCALE_STEP, which keeps every exponential below 2^8)
   float m_ref = -INFINITY, l_run = 0.f;
   bool ok = true;
-  if (tid == 0) ok = issue_s(0);
+  if (tid == 0) {
+    if (q_by_tma) ok = mbar_wait(smem_u32(&bar_q), 0u, abortp);
+    if (ok) ok = issue_s(0);
+  }
 
   for (int t = 0; t < n_tiles; ++t) {
     const int st = t & 1;
@@ -216,6 +245,7 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
     ok = __syncthreads_and(ok);
     if (!ok) break;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (tid == 0) timeline_mark(2 + (t < 5 ? t : 5));  // scores of tile t complete
     if (tid == 0 && t >= 1 && t + 1 < n_tiles) issue(t + 1);  // stage (t-1)&1 is free: tile t+1 goes there
     // ---- this thread's row of scores
     const int key_base = key_lo + t * UA_KEYS;
@@ -236,11 +266,13 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
         sv[96 + j] = __uint_as_float(r3[j]);
       }
       const int valid = key_hi - key_base;  // >= 1
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one of 128 steps
 #pragma unroll
       for (int j = 0; j < UA_KEYS; ++j) {
         sv[j] = (j < valid) ? sv[j] * scale_log2 : -INFINITY;
-        mx = fmaxf(mx, sv[j]);
+        mx4[j & 3] = fmaxf(mx4[j & 3], sv[j]);
       }
+      mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
     }
     // ---- lazy rescale of O (warp-uniform branch: the TMEM accesses are warp-collective)
     const bool grow = mx > m_ref + RESCALE_STEP;
@@ -263,22 +295,23 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
       }
     }
     // ---- probabilities -> shared memory (bf16, layout of an MMA A operand)
-    float p_sum = 0.f;
+    float p_sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int c8 = 0; c8 < UA_KEYS / 8; ++c8) {
       float pv[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         pv[j] = fast_exp2(sv[c8 * 8 + j] - m_ref);
-        p_sum += pv[j];
+        p_sum4[j & 3] += pv[j];
       }
       *reinterpret_cast<uint4*>(p_gen + tile_off<UA_ROWS>(row, c8)) =
           make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
     }
-    l_run += p_sum;
+    l_run += (p_sum4[0] + p_sum4[1]) + (p_sum4[2] + p_sum4[3]);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
+
     // ---- O += P V, and straight after it the scores of the next tile
     if (tid == 0) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -302,6 +335,7 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
 
   if (ok) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (tid == 0) timeline_mark(8);  // O complete
     const int vr = row0 + row;
     const bool live = vr < n_rows;
     const int qi = live ? vr / G : 0, g = live ? vr - qi * G : 0;
@@ -347,7 +381,8 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
 }
 
 template <int HD>
-cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
+cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
+                        int q_by_tma, const void* q, void* o,
                         float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
   constexpr int SMEM = (int)UaSmem<HD>::TOTAL;
   static bool configured = false;
@@ -362,7 +397,7 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
   float* ml_part = scratch ? scratch + (size_t)S * total * HD : nullptr;
   dim3 grid((a_seq * G + UA_ROWS - 1) / UA_ROWS, Hkv, B * S);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
-  cudaError_t e = launch_k(L, attn_umma_kernel<HD>, grid, dim3(128), SMEM, tmK, tmV, (const __nv_bfloat16*)q,
+  cudaError_t e = launch_k(L, attn_umma_kernel<HD>, grid, dim3(128), SMEM, tmK, tmV, tmQ, q_by_tma, (const __nv_bfloat16*)q,
                            (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split, scale_log2,
                            L.d_status);
   L.count();
@@ -400,8 +435,12 @@ cudaError_t launch_attention_umma(const Launch& L, const void* q, const void* Kc
       !get_tensor_map_3d(Vc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, 64, &tmV))
     return cudaErrorInvalidValue;
   if (S_out) *S_out = p.S;
-  return hd == 64 ? launch_umma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
-                  : launch_umma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
+  // with one query head per KV head a row tile is 128 consecutive rows of q: fetched by TMA
+  CUtensorMap tmQ = tmK;
+  const int q_by_tma = H == Hkv && ((uintptr_t)q & 15) == 0 &&
+                       get_tensor_map_2d(q, (uint64_t)B * a_seq, (uint64_t)H * hd, UA_ROWS, &tmQ);
+  return hd == 64 ? launch_umma<64>(L, tmK, tmV, tmQ, q_by_tma, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
+                  : launch_umma<128>(L, tmK, tmV, tmQ, q_by_tma, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
 }
 
 }  // namespace dllm
