@@ -925,9 +925,14 @@ __global__ void estimate_merge_kernel(const float4* __restrict__ rec, int rows, 
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (row >= rows) return;
   MaxSum t{-INFINITY, 0.f, 0x7fffffff};
-  for (int i = lane; i < n_tiles; i += 32) {
-    const float4 q = __ldcg(rec + (size_t)row * n_tiles + i);
-    t = merge(t, MaxSum{q.x, q.y, __float_as_int(q.z)});
+  for (int i0 = lane; i0 < n_tiles; i0 += 32 * 8) {  // eight records in flight per lane
+    float4 q[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (i0 + 32 * k < n_tiles) q[k] = __ldcg(rec + (size_t)row * n_tiles + i0 + 32 * k);
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (i0 + 32 * k < n_tiles) t = merge(t, MaxSum{q[k].x, q[k].y, __float_as_int(q[k].z)});
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
