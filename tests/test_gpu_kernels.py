@@ -22,6 +22,7 @@ def env():
 
 
 GEMM_SHAPES = [
+    (4400, 384, 128),    # 18 activation tiles: the launch-order remap with a narrow last group (16 + 2)
     (3, 200, 320),       # tiny M (long-prompt regime), ragged N
     (64, 4096, 4096),    # selected rows x a square projection: split-K
     (70, 1536, 832),     # ragged M, K = 13 blocks

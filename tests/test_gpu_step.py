@@ -162,6 +162,39 @@ def test_block_only_prediction_gives_the_same_generation(env, mode):
         ses_blk.step_scheduled_block(1, K, Kp, Kr, rho, R - 1, bl)      # block leaves the response
 
 
+@pytest.mark.parametrize("graphs", [False, True], ids=["host_events", "graph_event_nodes"])
+def test_profiling_counts_every_projection_and_changes_no_result(env, graphs):
+    """Per-kernel timing brackets every projection (class 0) and attention launch (class 1) with an event pair,
+    recorded by the host or as nodes of the step's graph; the step's results are those of an unprofiled step."""
+    torch, dllm = env
+    cfg = synth.small_bf16_model()
+    B, P, R = 2, 150, 72
+    _, ses, _ = make_pair(dllm, cfg, B, P, R)
+    _, ref, _ = make_pair(dllm, cfg, B, P, R)
+    ses.use_graphs(graphs)
+    for s_ in (ses, ref):
+        s_.step_full()
+    ses.profile(True)
+    steps = ((False, False, 0.25), (False, True, 0.0), (False, False, 0.25), (True, False, 0.5))
+    for rp, rr, rho in steps:
+        ses.step_cached(rp, rr, rho)
+        ref.step_cached(rp, rr, rho)
+    ses.sync(), ref.sync()
+    g, a = ses.profile_read(0), ses.profile_read(1)
+    # per layer: V (all response rows), Q/K, O, gate/up, down (+ V of the prompt rows on a prompt refresh); LM head
+    expect = sum(cfg.n_layers * (5 + (1 if rp else 0)) + 1 for rp, _, _ in steps)
+    assert g["launches"] == expect and a["launches"] == len(steps) * cfg.n_layers
+    assert g["ms"] > 0 and a["ms"] > 0 and g["bytes"] > 0 and g["flops"] > 0 and a["flops"] > 0
+    assert np.array_equal(ses.hidden(), ref.hidden())
+    assert np.array_equal(ses.tokens(), ref.tokens())
+    ses.profile(False)
+    assert ses.profile_read(0)["launches"] == 0
+    ses.step_cached(False, False, 0.25)       # unprofiled steps still run (and replay their own graphs)
+    ref.step_cached(False, False, 0.25)
+    ses.sync(), ref.sync()
+    assert np.array_equal(ses.hidden(), ref.hidden())
+
+
 def test_tiny_fp32_stepwise_generation_with_graphs_off_and_on(env):
     torch, dllm = env
     wl = synth.WORKLOADS["tiny"]
