@@ -113,10 +113,11 @@ def main(argv=None) -> int:
     total = out[-1]["start_us"]
     print(f"{args.workload}, {args.kind} step: {len(out)} launches, {total:.1f} us from the first release to the last"
           + (" (record arrays overflowed: totals are low)" if truncated else ""))
-    # launches of one layer: the step starts with one launch (embedding), then n_layers equal groups
-    per = (len(out) - 1) // n_layers
+    # launches of one layer: the step starts with one launch (embedding), then n_layers equal groups, then the
+    # LM head and the estimate
+    per = max(1, (len(out) - 3) // n_layers)
     lo = 1 + args.layer * per
-    if not truncated and 0 <= args.layer < n_layers:
+    if not truncated and 0 <= args.layer < n_layers and lo + per < len(out):
         print(f"layer {args.layer} ({per} launches, {out[lo + per]['start_us'] - out[lo]['start_us']:.1f} us):")
         for o in out[lo:lo + per]:
             print(f"  {o['file']:15s} grid {str(tuple(o['grid'])):16s} x {o['block']:4d}  ctas {o['ctas']:5d}  "

@@ -116,6 +116,20 @@ def test_invalid_arguments_are_rejected_without_a_gpu(dllm):
     assert dllm.lib.dllm_gemm_bf16_scratch_bytes(256, 126464, 4096) == 0      # enough tiles: no split
 
 
+def test_timeline_build_exports_its_hooks_and_the_product_library_has_none(dllm):
+    """The timeline variant is a separate library with the same ABI plus one pair of hooks per kernel file; the
+    product library carries no instrumentation."""
+    path = build_mod.build(timeline=True)
+    assert path.endswith("libdllm_b200_timeline.so") and os.path.exists(path)
+    tl = C.CDLL(path)
+    from paper_2506_06295_b200 import timeline
+    for stem in timeline.STEMS:
+        assert hasattr(tl, "dllm_timeline_set_" + stem) and hasattr(tl, "dllm_timeline_count_" + stem)
+        assert not hasattr(dllm.lib, "dllm_timeline_set_" + stem)
+    for name in declared_functions():
+        assert hasattr(tl, name)
+
+
 def test_binding_has_no_fallback():
     src = open(os.path.join(ROOT, "paper_2506_06295_b200", "dllm.py")).read()
     assert "oracle" not in src.replace("no CPU or PyTorch fallback", "")

@@ -7,6 +7,8 @@ Tolerances (relative L2 of the response hidden states): 1e-4 in fp32 mode,
 within 1e-3 of the k-th similarity; to tell a legal tie flip from an arithmetic
 fault the bf16 runs are repeated with the oracle's sets forced into the GPU
 path."""
+import os
+
 import numpy as np
 import pytest
 
@@ -193,6 +195,30 @@ def test_profiling_counts_every_projection_and_changes_no_result(env, graphs):
     ref.step_cached(False, False, 0.25)
     ses.sync(), ref.sync()
     assert np.array_equal(ses.hidden(), ref.hidden())
+
+
+def test_timeline_of_a_step_lists_every_launch_once():
+    """The in-graph timeline (separate library build, own process) sees each kernel launch of a step exactly
+    once, in order, with non-negative durations."""
+    import json
+    import subprocess
+    import sys
+    import tempfile
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with tempfile.TemporaryDirectory() as td:
+        out = os.path.join(td, "tl.json")
+        r = subprocess.run([sys.executable, "-m", "paper_2506_06295_b200.timeline", "--workload", "tiny", "--kind",
+                            "partial", "--layer", "1", "--json", out], cwd=root, capture_output=True, text=True, timeout=600)
+        assert r.returncode == 0, r.stderr[-2000:]
+        launches = json.load(open(out))
+    cfg = synth.WORKLOADS["tiny"].model
+    # fp32 model, partial step: embedding, 12 launches per layer (V, V-verify, selection + gather, Q/K, RoPE,
+    # attention, O, its epilogue, gate/up, SwiGLU, down, tail), LM head, estimate
+    assert len(launches) == 1 + 12 * cfg.n_layers + 2, [(o["file"], o["grid"]) for o in launches]
+    starts = [o["start_us"] for o in launches]
+    assert starts == sorted(starts) and all(o["dur_us"] >= 0 for o in launches)
+    assert all(o["ctas"] == o["grid"][0] * o["grid"][1] * o["grid"][2] for o in launches)
+    assert "layer 1 (12 launches" in r.stdout
 
 
 def test_tiny_fp32_stepwise_generation_with_graphs_off_and_on(env):
