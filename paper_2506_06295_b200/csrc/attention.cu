@@ -188,6 +188,9 @@ __device__ __forceinline__ void combine_row(const float* __restrict__ o_part, co
   }
 }
 
+// MAXS: 4, 8 or 16 splits held in registers (one instantiation each, so that few splits cost few registers and
+// every CTA of a large merge is resident at once); 0: any number of splits, one at a time.
+template <int MAXS>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restrict__ o_part,
                                                            const float* __restrict__ ml_part,
                                                            __nv_bfloat16* __restrict__ o, size_t total, int S, int hd) {
@@ -196,22 +199,35 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restri
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const size_t rh = (size_t)blockIdx.x * 8 + warp;
   if (rh >= total) return;
-  if (S <= 4) return combine_row<4>(o_part, ml_part, o, total, rh, S, hd, lane);
-  if (S <= 8) return combine_row<8>(o_part, ml_part, o, total, rh, S, hd, lane);
-  if (S <= 16) return combine_row<16>(o_part, ml_part, o, total, rh, S, hd, lane);
-  float M = -INFINITY, L = 0.f;
-  for (int s = 0; s < S; ++s) M = fmaxf(M, ml_part[((size_t)s * total + rh) * 2]);
-  for (int s = 0; s < S; ++s) {
-    const float* ml = ml_part + ((size_t)s * total + rh) * 2;
-    L += exp2f(ml[0] - M) * ml[1];
+  if constexpr (MAXS > 0) {
+    combine_row<MAXS>(o_part, ml_part, o, total, rh, S, hd, lane);
+  } else {
+    float M = -INFINITY, L = 0.f;
+    for (int s = 0; s < S; ++s) M = fmaxf(M, ml_part[((size_t)s * total + rh) * 2]);
+    for (int s = 0; s < S; ++s) {
+      const float* ml = ml_part + ((size_t)s * total + rh) * 2;
+      L += exp2f(ml[0] - M) * ml[1];
+    }
+    const float inv = 1.f / L;
+    for (int d = lane; d < hd; d += 32) {
+      float acc = 0.f;
+      for (int s = 0; s < S; ++s)
+        acc += exp2f(ml_part[((size_t)s * total + rh) * 2] - M) * o_part[((size_t)s * total + rh) * hd + d];
+      o[rh * hd + d] = __float2bfloat16_rn(acc * inv);
+    }
   }
-  const float inv = 1.f / L;
-  for (int d = lane; d < hd; d += 32) {
-    float acc = 0.f;
-    for (int s = 0; s < S; ++s)
-      acc += exp2f(ml_part[((size_t)s * total + rh) * 2] - M) * o_part[((size_t)s * total + rh) * hd + d];
-    o[rh * hd + d] = __float2bfloat16_rn(acc * inv);
-  }
+}
+
+cudaError_t launch_combine(const Launch& L, const float* o_part, const float* ml_part, __nv_bfloat16* o, size_t total,
+                           int S, int hd) {
+  const dim3 grid((unsigned)((total + 7) / 8)), block(256);
+  cudaError_t e;
+  if (S <= 4) e = launch_k(L, attn_combine_kernel<4>, grid, block, 0, o_part, ml_part, o, total, S, hd);
+  else if (S <= 8) e = launch_k(L, attn_combine_kernel<8>, grid, block, 0, o_part, ml_part, o, total, S, hd);
+  else if (S <= 16) e = launch_k(L, attn_combine_kernel<16>, grid, block, 0, o_part, ml_part, o, total, S, hd);
+  else e = launch_k(L, attn_combine_kernel<0>, grid, block, 0, o_part, ml_part, o, total, S, hd);
+  L.count();
+  return e;
 }
 
 template <int HD>
@@ -235,8 +251,7 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
                                                      L.d_status);
   L.count();
   if (S > 1) {
-    launch_k(L, attn_combine_kernel, dim3((unsigned)((total + 7) / 8)), dim3(256), 0, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
-    L.count();
+    launch_combine(L, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
   }
   return cudaGetLastError();
 }
@@ -273,9 +288,7 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
     if (e != cudaSuccess) return e;
     if (S > 1) {
       const size_t total = (size_t)B * a_seq * H;
-      e = launch_k(L, attn_combine_kernel, dim3((unsigned)((total + 7) / 8)), dim3(256), 0, scratch,
-                   scratch + (size_t)S * total * hd, (__nv_bfloat16*)o, total, S, hd);
-      L.count();
+      e = launch_combine(L, scratch, scratch + (size_t)S * total * hd, (__nv_bfloat16*)o, total, S, hd);
     }
     return e != cudaSuccess ? e : cudaGetLastError();
   }
