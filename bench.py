@@ -523,9 +523,9 @@ def in_graph_gemm(workload, gemm_bytes, peaks):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch from the ncu capture summarised under
-# profiles/ncu_gemm_bf16_tcgen05_partial_step_2layers.md: 454 MB per layer of an adaptive partial step over 5
-# launches, plus the LM head's 1,166 MB once per step (32 layers: 15.69 GB / 161 launches).
-TRAFFIC_PER_LAUNCH = {"llada8b": 97.5e6}
+# profiles/ncu_gemm_bf16_tcgen05_partial_step_2layers.md: 451 MB per layer of an adaptive partial step over 5
+# launches, plus the LM head's 1,051 MB once per step (32 layers: 15.48 GB / 161 launches).
+TRAFFIC_PER_LAUNCH = {"llada8b": 96.2e6}
 
 if __name__ == "__main__":
     main()

@@ -952,7 +952,8 @@ __global__ void estimate_merge_kernel(const float4* __restrict__ rec, int rows, 
 void launch_estimate_merge(const Launch& L, const float* records, int rows, int n_tiles, int32_t* x0, float* conf,
                            int R, int blk_start, int blk_len) {
   if (rows <= 0) return;
-  launch_k(L, estimate_merge_kernel, dim3((rows + 7) / 8), dim3(256), 0, reinterpret_cast<const float4*>(records), rows,
+  // two rows per CTA: 256 rows spread over 128 SMs (each warp walks its row's records in a few round trips)
+  launch_k(L, estimate_merge_kernel, dim3((rows + 1) / 2), dim3(64), 0, reinterpret_cast<const float4*>(records), rows,
            n_tiles, x0, conf, R, blk_start, blk_len);
   L.count();
 }
