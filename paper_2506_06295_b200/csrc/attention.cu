@@ -122,6 +122,7 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(const T* __restrict__ q,
 template <int HD>
 __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ CUtensorMap tmK,
                                                        const __grid_constant__ CUtensorMap tmV,
+                                                       const __grid_constant__ CUtensorMap tmQ, int q_by_tma,
                                                        const __nv_bfloat16* __restrict__ q,
                                                        __nv_bfloat16* __restrict__ o, float* __restrict__ o_part,
                                                        float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv,
@@ -136,6 +137,9 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ C
     mbar_init(smem_u32(&full_bar[0]), 1);
     mbar_init(smem_u32(&full_bar[1]), 1);
     mbar_fence_init();
+    prefetch_tensormap(&tmK);  // the descriptors are fetched while the predecessor still runs
+    prefetch_tensormap(&tmV);
+    if (q_by_tma) prefetch_tensormap(&tmQ);
   }
   __syncthreads();
   pdl_wait();  // K, V and Q come from the preceding kernels
@@ -143,7 +147,8 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ C
   uint32_t kv_iter = 0;
   const bool ok = attn_tile<HD>((int)threadIdx.x, smem_raw + (base - smem_u32(smem_raw)), base, full_bar, kv_iter,
                                 &abort_flag, &tmK, &tmV, q, o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split,
-                                scale_log2, (int)gridDim.z / S, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z);
+                                scale_log2, (int)gridDim.z / S, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z,
+                                q_by_tma ? &tmQ : nullptr);
   if (!ok && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
 }
 
@@ -246,7 +251,11 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
   float* ml_part = scratch ? scratch + (size_t)S * total * HD : nullptr;
   dim3 grid((a_seq * G + AT_ROWS - 1) / AT_ROWS, Hkv, B * S);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
-  launch_k(L, attn_mma_kernel<HD>, dim3(grid), dim3(128), SMEM, tmK, tmV, (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part,
+  // with one query head per KV head a row tile is 64 consecutive rows of q: fetched by TMA
+  CUtensorMap tmQ = tmK;
+  const int q_by_tma = H == Hkv && ((uintptr_t)q & 15) == 0 &&
+                       get_tensor_map_2d(q, (uint64_t)B * a_seq, (uint64_t)H * HD, AT_ROWS, &tmQ);
+  launch_k(L, attn_mma_kernel<HD>, dim3(grid), dim3(128), SMEM, tmK, tmV, tmQ, q_by_tma, (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part,
                                                      ml_part, a_seq, n, H, Hkv, S, keys_per_split, scale_log2,
                                                      L.d_status);
   L.count();

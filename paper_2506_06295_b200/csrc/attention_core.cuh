@@ -80,7 +80,8 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
                                           const CUtensorMap* tmV, const __nv_bfloat16* __restrict__ q,
                                           __nv_bfloat16* __restrict__ o, float* __restrict__ o_part,
                                           float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv, int S,
-                                          int keys_per_split, float scale_log2, int B, int bx, int by, int bz) {
+                                          int keys_per_split, float scale_log2, int B, int bx, int by, int bz,
+                                          const CUtensorMap* tmQ = nullptr) {
 
   constexpr int PANELS = HD / 64;
   constexpr uint32_t TILE_BYTES = AT_KEYS * HD * 2;   // one K or V tile
@@ -104,10 +105,17 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
   const uint32_t it0 = kv_iter;
   kv_iter += (uint32_t)n_tiles;
   at_sync();  // the previous tile's readers are done with the Q and K/V regions
+  // tmQ (one query head per KV head, so a row tile is AT_ROWS consecutive rows of q): the Q tile arrives by TMA
+  // together with the first K/V tile, on that tile's barrier; rows past the sequence's end belong to no live row
+  const bool q_tma = tmQ != nullptr;
   auto issue = [&](int t) {
     const int st = (int)((it0 + (uint32_t)t) & 1u);
     const uint32_t fb = smem_u32(&full_bar[st]);
-    mbar_expect_tx(fb, STAGE_BYTES);
+    mbar_expect_tx(fb, STAGE_BYTES + ((q_tma && t == 0) ? AT_ROWS * HD * 2 : 0));
+    if (q_tma && t == 0) {
+#pragma unroll
+      for (int p = 0; p < PANELS; ++p) tma_load_2d(q_s + p * (AT_ROWS * 128), tmQ, fb, kh * HD + p * 64, b * a_seq + row0);
+    }
     const uint32_t dst = kv_s + st * STAGE_BYTES;
     const int key0 = key_lo + t * AT_KEYS;
 #pragma unroll
@@ -122,7 +130,9 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
   }
   // Q tile: plain 16-byte loads into the swizzled layout (rows of other heads /
   // past the end are zero)
-  {
+  if (q_tma) {
+    mbar_wait(smem_u32(&full_bar[(int)(it0 & 1u)]), (it0 >> 1) & 1u, abort_flag);  // the loop checks the outcome again
+  } else {
     constexpr int PER = AT_ROWS * (HD / 8) / 128;  // 16-byte chunks per thread: all loads first, then the stores
     uint4 qv[PER];
 #pragma unroll
