@@ -181,10 +181,17 @@ class StepResult:
 class DLLMOracle:
     """Model p_theta with Prompt Cache C_p and Response Cache C_r (Sec. 3.2):
     per layer K, V [B, n, dkv] and AttnOut, FFNOut [B, n, d]; rows [0, P) are
-    C_p, rows [P, n) are C_r."""
+    C_p, rows [P, n) are C_r.
+
+    compact_prompt_outs=True is the storage variant that the memory limitation of
+    Sec. A.10 item (1) invites: AttnOut and FFNOut are kept for the response rows
+    only, [B, R, d].  The prompt's AttnOut / FFNOut are never read between prompt
+    refreshes (the prompt's residual stream is not carried on those steps) and on
+    a prompt refresh they are recomputed before they are used, so within a step
+    they live in a temporary and are dropped at the end of the layer."""
 
     def __init__(self, cfg, weights: dict, batch: int, prompt_len: int, gen_len: int,
-                 dtype=np.float64):
+                 dtype=np.float64, compact_prompt_outs: bool = False):
         self.cfg = cfg
         self.dt = np.dtype(dtype)
         self.B, self.P, self.R = batch, prompt_len, gen_len
@@ -195,8 +202,10 @@ class DLLMOracle:
         dkv, d = c.n_kv_heads * c.head_dim, c.d_model
         self.Kc = [np.zeros((batch, n, dkv), self.dt) for _ in range(T)]
         self.Vc = [np.zeros((batch, n, dkv), self.dt) for _ in range(T)]
-        self.Ac = [np.zeros((batch, n, d), self.dt) for _ in range(T)]
-        self.Fc = [np.zeros((batch, n, d), self.dt) for _ in range(T)]
+        self.compact = bool(compact_prompt_outs)
+        rows_out = gen_len if self.compact else n
+        self.Ac = [np.zeros((batch, rows_out, d), self.dt) for _ in range(T)]
+        self.Fc = [np.zeros((batch, rows_out, d), self.dt) for _ in range(T)]
         self.tokens = np.full((batch, n), c.mask_id, dtype=np.int64)
         self.valid = False
         self.macs = {"proj": 0, "attn": 0, "ffn": 0, "lm_head": 0}
@@ -264,6 +273,12 @@ class DLLMOracle:
                 p = f"layers.{l}."
                 ksel = ksels[l]
                 Kc, Vc, Ac, Fc = self.Kc[l][b], self.Vc[l][b], self.Ac[l][b], self.Fc[l][b]
+                if self.compact:
+                    # the layer works on full-height temporaries whose response rows are the stored ones; the
+                    # prompt rows hold nothing until (and unless) this step recomputes them
+                    Ac_resp, Fc_resp = Ac, Fc
+                    Ac, Fc = np.zeros((n, d), self.dt), np.zeros((n, d), self.dt)
+                    Ac[P:], Fc[P:] = Ac_resp, Fc_resp
                 # a. pre-attention norm of the carried rows
                 u = np.zeros((n, d), self.dt)
                 u[carried] = rmsnorm(x[carried], self.w[p + "norm1"].astype(self.dt), c.rms_eps)
@@ -322,6 +337,8 @@ class DLLMOracle:
                     Fc[act] = self._lin(silu(g) * up, p + "wd", "ffn")
                 # g. every carried row continues with the available feature version
                 x[carried] = (x[carried] + Ac[carried]) + Fc[carried]
+                if self.compact:
+                    Ac_resp[...], Fc_resp[...] = Ac[P:], Fc[P:]      # the prompt rows are dropped
             # 3. prediction at the response rows (Eqs. 3-4)
             res.hidden[b] = x[P:]
             z = rmsnorm(x[P:], self.w["norm_f"].astype(self.dt), c.rms_eps)
