@@ -237,7 +237,6 @@ def main():
     ap.add_argument("--full-steps", type=int, default=6, help="timed full-recompute steps for the speedup figure")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (small case for ncu "
                     "captures: same widths, a few GB of weights); the bench line then names the reduced depth")
-    ap.add_argument("--no-layer-kernel", action="store_true", help="launch every step kind kernel by kernel")
     ap.add_argument("--no-pdl", action="store_true", help="plain launches instead of programmatic dependent launch")
     ap.add_argument("--ncu-kinds", default="", help="comma list of step kinds (full,refresh,mixed,partial): after "
                     "warm-up run one step of each between cudaProfilerStart/Stop and exit (for "
@@ -276,8 +275,6 @@ def main():
     ses.set_prompt(prompt)
     if args.no_pdl:
         ses.use_pdl(False)
-    if args.no_layer_kernel:
-        ses.use_layer_kernel(False)
     stream = ses.stream
 
     def barrier():

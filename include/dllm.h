@@ -11,7 +11,11 @@
  * Conventions
  *   - Every call returns a dllm_status; nothing throws, aborts or traps.
  *     dllm_last_error(handle) returns a readable message for the last failure
- *     on that handle (handle may be NULL for failures of a *_create call).
+ *     recorded on that live model or session handle; with NULL (or a pointer
+ *     that is no live handle) it returns the last failure of any call on the
+ *     calling thread, which is how failures of *_create calls, size queries
+ *     and the kernel-level entry points are read.  The string stays valid
+ *     until the same thread calls dllm_last_error again.
  *   - The caller owns all device memory: the weight blob, the cache blob and
  *     the workspace blob are device pointers the caller allocated (256-byte
  *     aligned) with at least the byte counts the size queries return, and must
@@ -65,6 +69,16 @@ typedef enum { DLLM_K_FLOOR = 0, DLLM_K_CEIL = 1 } dllm_kround;
 
 enum { DLLM_CACHE_K = 0, DLLM_CACHE_V = 1, DLLM_CACHE_ATTN = 2, DLLM_CACHE_FFN = 3 };
 
+/* Session flags.  DLLM_SESSION_COMPACT_CACHE: the AttnOut and FFNOut caches keep the
+ * response rows only ([B, R, d_model] per layer instead of [B, n, d_model]).
+ * Between prompt refreshes no step reads the prompt's AttnOut / FFNOut (the
+ * prompt's residual stream is not carried then) and a prompt refresh recomputes
+ * them before it uses them, so every output of every step is bit-identical to
+ * the four-tensor layout; the cache shrinks by 2 * P * d_model elements per
+ * layer and sequence (the memory overhead for long sequences that Sec. A.10
+ * item (1) names; Sec. A.9 counts the four full tensors). */
+enum { DLLM_SESSION_DEFAULT = 0, DLLM_SESSION_COMPACT_CACHE = 1 };
+
 typedef struct dllm_model dllm_model;
 typedef struct dllm_session dllm_session;
 
@@ -78,8 +92,16 @@ size_t dllm_weights_bytes(const dllm_config* cfg);
  * model dtype -- exactly the four tensors per layer of Sec. A.9. */
 size_t dllm_cache_bytes(const dllm_config* cfg, int B, int P, int R);
 /* Bytes of scratch the step needs (residual stream, staging buffers, GEMM
- * partial sums, logits, selection state). */
+ * partial sums, logits, selection state).  The GEMM part follows the launch
+ * plans of the device that is current when the query is made: ask with the
+ * session's device current. */
 size_t dllm_workspace_bytes(const dllm_config* cfg, int B, int P, int R);
+/* The same two sizes for a session created with `flags` (DLLM_SESSION_*; 0 for
+ * an unknown flag).  With DLLM_SESSION_COMPACT_CACHE the cache holds, per layer,
+ * K, V [B, n, Hkv*hd] and AttnOut, FFNOut [B, R, d_model]: Sec. A.9's count
+ * minus 2 * P * d_model elements per layer and sequence. */
+size_t dllm_cache_bytes_ex(const dllm_config* cfg, int B, int P, int R, int flags);
+size_t dllm_workspace_bytes_ex(const dllm_config* cfg, int B, int P, int R, int flags);
 /* Byte offset and element count of one named tensor inside the weight blob, so
  * a caller may fill the blob on the device.  Names: "embed", "lm_head" [vocab,
  * d_model]; "norm_f" [d_model]; "layers.<l>.{norm1,norm2}" [d_model];
@@ -113,6 +135,10 @@ dllm_status dllm_model_destroy(dllm_model* m);
  * zeroed asynchronously on `stream`. */
 dllm_status dllm_session_create(dllm_model* m, int B, int P, int R, void* d_cache, void* d_workspace,
                                 void* stream, dllm_session** out);
+/* The same with session flags; d_cache / d_workspace sized by the _ex queries
+ * with the same flags. */
+dllm_status dllm_session_create_ex(dllm_model* m, int B, int P, int R, int flags, void* d_cache,
+                                   void* d_workspace, void* stream, dllm_session** out);
 dllm_status dllm_session_destroy(dllm_session* s);
 /* tokens <- [prompt ; MASK x R] for every sequence (Eq. 2); caches become
  * invalid until the next full step.  h_prompt: int32 [B, P], ids in [0, vocab). */
@@ -193,7 +219,8 @@ dllm_status dllm_get_logits(dllm_session* s, float* h_out /* [B, R, vocab] */, v
 dllm_status dllm_get_selected(dllm_session* s, int layer, int32_t* h_idx, float* h_sim, int* k_sel_out,
                               void* stream);
 /* One cache tensor of one layer as float32 [B, n, width] (width = Hkv*hd for K
- * and V, d_model for AttnOut and FFNOut). */
+ * and V, d_model for AttnOut and FFNOut).  In a DLLM_SESSION_COMPACT_CACHE
+ * session AttnOut and FFNOut are [B, R, d_model]: the response rows only. */
 dllm_status dllm_get_cache(dllm_session* s, int layer, int which, float* h_out, void* stream);
 dllm_status dllm_set_cache(dllm_session* s, int layer, int which, const float* h_in, void* stream);
 /* Replaces the V-verify choice of `layer` on adaptive steps by the given
@@ -229,12 +256,6 @@ dllm_status dllm_session_use_graphs(dllm_session* s, int enable);
  * projections) overlaps the tail of the kernel before it; 0: plain launches. */
 dllm_status dllm_session_use_pdl(dllm_session* s, int enable);
 
-/* 1: steps without prompt refresh (response refresh, adaptive partial) in bf16
- * run all layers in ONE persistent cooperative kernel (one CTA per SM, weight
- * stream that never stops, grid barriers between phases); 0 (default): kernel
- * by kernel like the other step kinds, which measured faster on B200. */
-dllm_status dllm_session_use_layer_kernel(dllm_session* s, int enable);
-
 /* Per-kernel timing.  While enabled, every projection GEMM (class 0) and
  * attention launch (class 1) is bracketed by CUDA events on the caller's stream
  * and no launch overlaps its predecessor (no programmatic dependent launch).
@@ -253,6 +274,25 @@ dllm_status dllm_session_profile_read(dllm_session* s, int cls, double* total_ms
 dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable);
 
 /* ---- kernel-level entry points (parity tests and micro-benchmarks) --------- */
+/* The kernel-level calls below have no session, so the bounded waits of their
+ * kernels (the same TMA / tcgen05 pipelines the step uses) report into one
+ * status word inside the library image, per GPU (nothing is allocated for it).
+ * dllm_kernel_status synchronises `stream`, reads the word of the current
+ * device and clears it: DLLM_OK, or DLLM_TIMEOUT when a wait of any
+ * kernel-level call since the last read gave up (its output is then
+ * unspecified), as dllm_sync does for a session. */
+dllm_status dllm_kernel_status(void* stream);
+/* Test hooks for the DLLM_TIMEOUT path; they fault nothing and hang nothing.
+ * dllm_debug_set_wait_limit_ns: the time after which a device-side wait of the
+ * TMA / tcgen05 pipelines gives up (0 restores the default of 2 s), on the
+ * current device, for every kernel launched afterwards.
+ * dllm_debug_skip_one_load(1): from now on the first CTA of every launch of
+ * the one-CTA bf16 GEMM kernel leaves out one activation-tile copy, so one of
+ * its pipeline stages never completes, its waits run into the limit, the CTA
+ * records the status code, skips its epilogue, frees its tensor memory and
+ * returns normally; (0) switches that off.  Both calls synchronise the device. */
+dllm_status dllm_debug_set_wait_limit_ns(uint64_t ns);
+dllm_status dllm_debug_skip_one_load(int enable);
 /* C[M,N] (fp32, row-major, DEVICE) = A[M,K] * W[N,K]^T with bf16 operands on
  * the tensor cores (tcgen05 + TMA).  d_partials is scratch of
  * dllm_gemm_bf16_scratch_bytes(M,N,K); partial sums over k ranges are reduced
@@ -295,9 +335,12 @@ dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, 
 /* Non-causal attention of `a` query rows per sequence over n cached keys
  * (Sec. A.7, the 4 r n d term).  d_q [B*a, H*hd], d_k / d_v [B, n, Hkv*hd], d_o
  * [B*a, H*hd]; dtype as above.  bf16 with head_dim 64 or 128 runs on the tensor
- * cores and, when few rows are active, splits the key range over CTAs; the
- * partial results of the splits go to d_scratch (device,
- * dllm_attention_scratch_bytes(); with less the key range is not split). */
+ * cores -- up to 64 (query, head-of-group) rows per KV head on a 64-row
+ * mma.sync kernel, more on a 128-row tcgen05 kernel -- and, when few rows are
+ * active, splits the key range over CTAs; the partial results of the splits go
+ * to d_scratch (device).  dllm_attention_scratch_bytes() is what the plan of
+ * the kernel that shape runs on would like; with less the 64-row kernel does
+ * not split and the 128-row kernel splits as far as the buffer allows. */
 size_t dllm_attention_scratch_bytes(int B, int a, int n, int H, int Hkv, int hd, int dtype);
 dllm_status dllm_attention(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B, int a, int n,
                            int H, int Hkv, int hd, int dtype, void* d_scratch, size_t scratch_bytes, void* stream);
@@ -313,9 +356,10 @@ dllm_status dllm_attention(const void* d_q, const void* d_k, const void* d_v, vo
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress) with that device current; make that first call
  *     before any stream capture.
- *   - Shapes whose split plan needs more than the 8 MiB return
- *     DLLM_UNSUPPORTED with a message; use dllm_attention with your own
- *     scratch for those.
+ *   - It runs exactly what dllm_attention runs when given
+ *     dllm_attention_scratch_bytes() of scratch.  Shapes for which that is
+ *     more than the 8 MiB return DLLM_UNSUPPORTED with a message; use
+ *     dllm_attention with your own scratch for those.
  *   - All calls share the one array and it keeps the previous call's contents
  *     (nothing needs clearing: every value read is written first by the same
  *     call).  Two calls that overlap on the GPU -- different streams, or the

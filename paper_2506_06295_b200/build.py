@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdllm_b200.so")
-SOURCES = ["api.cu", "elementwise.cu", "gemm_simt.cu", "gemm_tcgen05.cu", "attention.cu", "attention_umma.cu", "megakernel.cu"]
+SOURCES = ["api.cu", "elementwise.cu", "gemm_simt.cu", "gemm_tcgen05.cu", "attention.cu", "attention_umma.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-DNDEBUG"]
 

@@ -9,8 +9,10 @@
 
 #include <algorithm>
 #include <map>
+#include <mutex>
 #include <new>
 #include <string>
+#include <unordered_map>
 #include <vector>
 
 #include "../../include/dllm.h"
@@ -21,7 +23,20 @@ using namespace dllm;
 
 namespace {
 
-thread_local std::string g_err;
+thread_local std::string g_err;  // last failure on this thread (what dllm_last_error(NULL) returns)
+
+// Live handles and where each keeps its last message, so that dllm_last_error(handle) can tell a model from a
+// session (and both from a stale pointer) without trusting the caller.
+std::mutex g_handles_mu;
+std::unordered_map<const void*, const std::string*> g_handles;
+void register_handle(const void* h, const std::string* slot) {
+  std::lock_guard<std::mutex> lock(g_handles_mu);
+  g_handles[h] = slot;
+}
+void unregister_handle(const void* h) {
+  std::lock_guard<std::mutex> lock(g_handles_mu);
+  g_handles.erase(h);
+}
 
 size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
@@ -125,12 +140,12 @@ uint16_t f32_to_bf16_rne(float f) {
 
 // workspace carve-up
 struct Workspace {
-  size_t status, tokens, x, u, ua, qbuf, obuf, hn, ffn, x0, conf, sim, sel, forced, act, inv, mkbar, mkmaps, rope, attn, part,
-      total;
+  size_t status, tokens, x, u, ua, qbuf, obuf, hn, ffn, x0, conf, sim, sel, forced, act, inv, rope, pouts, attn,
+      part, total;
   size_t part_floats, attn_floats;
 };
 
-Workspace make_workspace(const dllm_config& c, int B, int P, int R) {
+Workspace make_workspace(const dllm_config& c, int B, int P, int R, int flags) {
   Workspace w;
   const size_t es = esize(c), d = c.d_model, dq = (size_t)c.n_heads * c.head_dim,
                dkv = (size_t)c.n_kv_heads * c.head_dim, m = c.d_ffn, V = c.vocab;
@@ -157,21 +172,38 @@ Workspace make_workspace(const dllm_config& c, int B, int P, int R) {
   w.forced = take(T * BR * 4);
   w.act = take(rows * 4);
   w.inv = take(rows * 4);
-  w.mkbar = take((1 + 13 * T) * 4);  // one grid-barrier counter per phase of the persistent layer kernel
-  w.mkmaps = take((size_t)7 * T * sizeof(CUtensorMap));
   w.rope = take(n * c.head_dim * 4);
-  // partial outputs of split key ranges: splits happen only while fewer than
-  // 148 CTAs of 64 (row, head) pairs exist, so S * pairs < 2 * 148 * 64
-  w.attn_floats = (size_t)2 * 148 * 64 * (128 + 2);
+  // compact caches: AttnOut and FFNOut of the prompt rows live here for the length of one layer of a
+  // prompt-refresh step ([B, P, d] each, carried order)
+  w.pouts = take((flags & DLLM_SESSION_COMPACT_CACHE) ? 2 * (size_t)B * P * d * es : 0);
+  // partial outputs of split key ranges: the 64-row kernel splits only while fewer CTAs than SMs exist, so
+  // splits * (row, head) pairs < 2 * SMs * 64; the 128-row kernel lowers its split count to what this holds
+  w.attn_floats = (size_t)2 * sm_count() * 64 * (128 + 2);
   w.attn = take(w.attn_floats * 4);
-  // largest [M, N] any GEMM writes, or the slabs of a GEMM whose tiles are
-  // split: splitting happens only below 8 tiles per SM (M*N <= 8 G tiles of
-  // 256 x 128) and a tile has at most G/tiles + 2 slabs, so slabs * M * N <=
-  // (1 + 2 * 8) * G * 256 * 128 floats with G = 160 >= the SM count
-  size_t mn = rows * std::max(std::max(dq + dkv, d), 2 * m);
-  mn = std::max(mn, BR * V);
-  mn = std::max(mn, rows * std::max(d, dkv));
-  w.part_floats = std::max(mn, (size_t)17 * 160 * 256 * 128) + 4096;
+  // the GEMM slab buffer: the largest S * M * N over every projection a step of this session can launch (V and
+  // the LM head over the B * R response rows, V over the prompt rows, and Q/K, O, gate/up, down and V over any
+  // number of active rows), and the fp32 staging of the inspection hooks (a cache tensor, the logits)
+  size_t mn = std::max(BR * V, rows * std::max(d, dkv));
+  if (c.dtype == DLLM_BF16) {
+    auto slabs = [&](size_t M, size_t N, size_t K) {
+      if (M == 0) return;
+      const GemmPlan p = plan_gemm_bf16((int)M, (int)N, (int)K);
+      mn = std::max(mn, (size_t)p.S_max * M * N);
+    };
+    slabs(BR, dkv, d);
+    slabs(BR, V, d);
+    slabs((size_t)B * P, dkv, d);
+    for (size_t Ma = 1; Ma <= rows; ++Ma) {
+      slabs(Ma, dq + dkv, d);
+      slabs(Ma, dkv, d);
+      slabs(Ma, d, dq);
+      slabs(Ma, 2 * m, d);
+      slabs(Ma, d, m);
+    }
+  } else {
+    mn = std::max(mn, rows * std::max(std::max(dq + dkv, d), 2 * m));
+  }
+  w.part_floats = mn + 4096;
   w.part = take(w.part_floats * 4);
   w.total = off;
   return w;
@@ -212,6 +244,7 @@ struct dllm_session {
   uint8_t* d_cache;
   uint8_t* d_ws;
   Workspace ws;
+  bool compact = false;    // AttnOut / FFNOut caches hold the response rows only
   bool valid = false;      // caches hold a full step
   bool have_pred = false;
   std::vector<int> last_ksel;  // per layer
@@ -222,8 +255,6 @@ struct dllm_session {
   bool use_pdl = true;
   int sel_strategy = DLLM_SELECT_V_VERIFY, sel_metric = DLLM_METRIC_COSINE, v_selected_only = 0;  // ablation variants
   bool block_head = false;     // dllm_generate predicts only the block each step works on
-  bool use_mk = false;         // persistent layer kernel for the step kinds it covers (opt-in)
-  bool mk_maps_ready = false;  // weight / cache tensor maps uploaded to the workspace
   struct GraphEntry {
     cudaGraphExec_t exec;
     uint64_t kernels;
@@ -291,15 +322,22 @@ struct dllm_session {
   size_t es() const { return esize(m->cfg); }
   size_t dkv() const { return (size_t)m->cfg.n_kv_heads * m->cfg.head_dim; }
   size_t dq() const { return (size_t)m->cfg.n_heads * m->cfg.head_dim; }
-  size_t layer_bytes() const { return (size_t)B * n * (2 * dkv() + 2 * (size_t)m->cfg.d_model) * es(); }
+  size_t out_rows() const { return (size_t)B * (compact ? R : n); }  // rows of an AttnOut / FFNOut tensor
+  size_t layer_bytes() const {
+    return ((size_t)B * n * 2 * dkv() + out_rows() * 2 * (size_t)m->cfg.d_model) * es();
+  }
   uint8_t* cache(int layer, int which) const {
-    const size_t rows = (size_t)B * n;
     size_t off = (size_t)layer * layer_bytes();
-    const size_t kv = rows * dkv() * es(), ad = rows * (size_t)m->cfg.d_model * es();
+    const size_t kv = (size_t)B * n * dkv() * es(), ad = out_rows() * (size_t)m->cfg.d_model * es();
     if (which >= 1) off += kv;
     if (which >= 2) off += kv;
     if (which >= 3) off += ad;
     return d_cache + off;
+  }
+  // AttnOut (which = DLLM_CACHE_ATTN) or FFNOut rows of a layer as the row-wise kernels address them
+  OutRows outs(int layer, int which) const {
+    uint8_t* prompt = d_ws + ws.pouts + (which == DLLM_CACHE_FFN ? (size_t)B * P * m->cfg.d_model * es() : 0);
+    return OutRows{cache(layer, which), compact ? prompt : nullptr, compact ? 1 : 0};
   }
   template <typename T>
   T* wsp(size_t off) const {
@@ -384,106 +422,6 @@ dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void
   return DLLM_OK;
 }
 
-// The layers of a step without prompt refresh as one persistent kernel, then
-// the LM head and the greedy estimate.
-dllm_status enqueue_step_mk(dllm_session* s, int rr, int ksel, cudaStream_t stream) {
-  const dllm_config& c = s->m->cfg;
-  const WeightLayout& wl = s->m->lay;
-  const int d = c.d_model, H = c.n_heads, Hkv = c.n_kv_heads, hd = c.head_dim, m = c.d_ffn;
-  const int dq = H * hd, dkv = Hkv * hd, BR = s->B * s->R;
-  const size_t es = 2, rows = (size_t)s->B * s->n;
-  Launch L{stream, s->wsp<int>(s->ws.status), &s->launches, s->use_pdl};
-  uint8_t* W = s->m->d_w;
-  MkParams p;
-  memset(&p, 0, sizeof p);
-  p.B = s->B; p.P = s->P; p.R = s->R; p.n = s->n; p.d = d; p.H = H; p.Hkv = Hkv; p.hd = hd; p.dq = dq; p.dkv = dkv;
-  p.m = m; p.T = c.n_layers; p.eps = c.rms_eps; p.gu_interleaved = gu_interleaved(c);
-  p.rr = rr; p.ksel = ksel; p.a_seq = ksel; p.Ma = s->B * ksel; p.BR = BR;
-  for (int l = 0; l < c.n_layers; ++l)
-    if (!rr && s->forced_count[l] >= 0) p.forced_mask |= 1ull << l;
-  p.W = W;
-  const LayerOff& l0 = wl.layers[0];
-  p.o_embed = wl.embed; p.o_norm1 = l0.norm1; p.o_wqkv = l0.wqkv; p.o_wo = l0.wo; p.o_norm2 = l0.norm2;
-  p.o_wgu = l0.wgu; p.o_wd = l0.wd; p.o_norm_f = wl.norm_f;
-  p.layer_stride = c.n_layers > 1 ? wl.layers[1].norm1 - l0.norm1 : 0;
-  p.cache = s->d_cache;
-  p.cache_layer_bytes = s->layer_bytes();
-  p.c_v = rows * dkv * es;
-  p.c_a = 2 * p.c_v;
-  p.c_f = p.c_a + rows * d * es;
-  p.tokens = s->wsp<int32_t>(s->ws.tokens);
-  p.x = s->wsp<float>(s->ws.x);
-  p.u = s->wsp<uint8_t>(s->ws.u);
-  p.ua = rr ? p.u : (void*)s->wsp<uint8_t>(s->ws.ua);  // response refresh: the active rows are all rows, in place
-  p.qbuf = s->wsp<uint8_t>(s->ws.qbuf);
-  p.obuf = s->wsp<uint8_t>(s->ws.obuf);
-  p.hn = s->wsp<uint8_t>(s->ws.hn);
-  p.ffn = s->wsp<uint8_t>(s->ws.ffn);
-  p.sim = s->wsp<float>(s->ws.sim);
-  p.sel = s->wsp<int32_t>(s->ws.sel);
-  p.forced = s->wsp<int32_t>(s->ws.forced);
-  p.act = s->wsp<int32_t>(s->ws.act);
-  p.inv = s->wsp<int32_t>(s->ws.inv);
-  p.rope = s->wsp<float>(s->ws.rope);
-  p.attn_scratch = s->wsp<float>(s->ws.attn);
-  p.part = s->wsp<float>(s->ws.part);
-  p.status = s->wsp<int>(s->ws.status);
-  p.bar = s->wsp<unsigned int>(s->ws.mkbar);
-  p.maps_fixed = s->wsp<CUtensorMap>(s->ws.mkmaps);
-  mk_plan(p);
-  if (p.attn_S > 1 && plan_attention(p.B, p.a_seq, p.n, H, Hkv).scratch_floats > s->ws.attn_floats) {
-    p.attn_S = 1;  // no room for the partials of split key ranges
-    p.attn_kps = (p.n + 63) / 64 * 64;
-    p.has_comb = 0;
-  }
-  if (mk_part_floats(p) > s->ws.part_floats)
-    return fail(&s->err, DLLM_UNSUPPORTED, "the slabs of the persistent layer kernel exceed the workspace");
-  if (!s->mk_maps_ready) {
-    std::vector<CUtensorMap> maps((size_t)7 * c.n_layers);
-    bool ok = true;
-    for (int l = 0; l < c.n_layers && ok; ++l) {
-      const LayerOff& lo = wl.layers[l];
-      uint8_t* Wq = W + lo.wqkv;
-      ok = ok && get_tensor_map_2d(Wq + (size_t)(dq + dkv) * d * es, dkv, d, 128, &maps[l * 5 + MK_V]);
-      ok = ok && get_tensor_map_2d(Wq, dq + dkv, d, 128, &maps[l * 5 + MK_QK]);
-      ok = ok && get_tensor_map_2d(W + lo.wo, d, dq, 128, &maps[l * 5 + MK_O]);
-      ok = ok && get_tensor_map_2d(W + lo.wgu, 2 * (uint64_t)m, d, 128, &maps[l * 5 + MK_GU]);
-      ok = ok && get_tensor_map_2d(W + lo.wd, d, m, 128, &maps[l * 5 + MK_D]);
-      ok = ok && get_tensor_map_3d(s->cache(l, DLLM_CACHE_K), s->B, s->n, dkv, 64, &maps[5 * c.n_layers + 2 * l]);
-      ok = ok && get_tensor_map_3d(s->cache(l, DLLM_CACHE_V), s->B, s->n, dkv, 64, &maps[5 * c.n_layers + 2 * l + 1]);
-    }
-    if (!ok) return fail(&s->err, DLLM_CUDA_ERROR, "cuTensorMapEncodeTiled failed or is unavailable");
-    CU_TRY(&s->err, cudaStreamSynchronize(stream));
-    CU_TRY(&s->err, h2d(s->d_ws + s->ws.mkmaps, maps.data(), maps.size() * sizeof(CUtensorMap), stream));
-    s->mk_maps_ready = true;
-  }
-  const void* a_ptr[5] = {p.u, p.ua, p.obuf, p.hn, p.ffn};
-  const int a_cols[5] = {d, d, dq, d, m};
-  for (int g = 0; g < 5; ++g)
-    if (!get_tensor_map_2d(a_ptr[g], (uint64_t)p.g[g].M, (uint64_t)a_cols[g], (uint32_t)p.g[g].BN, &p.amap[g]))
-      return fail(&s->err, DLLM_CUDA_ERROR, "cuTensorMapEncodeTiled failed or is unavailable");
-  CU_TRY(&s->err, cudaMemsetAsync(p.bar, 0, (size_t)(1 + 13 * c.n_layers) * 4, stream));
-  cudaError_t e = launch_layer_megakernel(L, p);
-  if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "persistent layer kernel: %s", cudaGetErrorString(e));
-  // prediction at the response rows (Eqs. 3-4); u already holds the final norm
-  Partials part{nullptr, 0, 1, 0};
-  dllm_status st = run_gemm(s, L, p.u, W + wl.lm_head, BR, c.vocab, d, &part);
-  if (st != DLLM_OK) return st;
-  if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
-  launch_argmax_conf(L, part.p, BR, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf));
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "step launch: %s", cudaGetErrorString(e));
-  return DLLM_OK;
-}
-
-bool step_uses_mk(const dllm_session* s, int rp, int ksel) {
-  const dllm_config& c = s->m->cfg;
-  if (s->sel_strategy != DLLM_SELECT_V_VERIFY || s->sel_metric != DLLM_METRIC_COSINE || s->v_selected_only) return false;
-  return s->use_mk && !s->profiling && !s->simt_gemm &&
-         mk_supported(c.dtype, s->B, s->P, s->R, c.d_model, c.n_heads, c.n_kv_heads, c.head_dim, c.d_ffn, c.n_layers, rp,
-                      ksel);
-}
-
 // Enqueue one denoising step.  Active rows per sequence: the prompt rows on a
 // prompt refresh plus either all R response rows (response refresh) or the
 // ksel rows V-verify picks.
@@ -549,7 +487,8 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
         // few active rows: every CTA of the gather repeats the selection rather than wait for a launch
         launch_select_gather(L, dt, sim, forced, mode, ksel, sel, act, inv, u, s->wsp<uint8_t>(s->ws.ua), g, rp);
       } else {
-        launch_select(L, sim, forced, mode, ksel, sel, s->R, act, inv, g, rp);
+        cudaError_t se = launch_select(L, sim, forced, mode, ksel, sel, s->R, act, inv, g, rp);
+        if (se != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "selection: %s", cudaGetErrorString(se));
         launch_gather_rows(L, dt, u, act, s->wsp<uint8_t>(s->ws.ua), Ma, d);
       }
       if (v_for_active) {
@@ -569,7 +508,7 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
       if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.obuf), W + lo.wo, Ma, d, dq, &part)) != DLLM_OK) return st;
       launch_oproj_epilogue(L, dt, part, act, x, reinterpret_cast<const float*>(W + lo.norm2),
-                            s->cache(l, DLLM_CACHE_ATTN), s->wsp<uint8_t>(s->ws.hn), g, Ma, c.rms_eps);
+                            s->outs(l, DLLM_CACHE_ATTN), s->wsp<uint8_t>(s->ws.hn), g, Ma, c.rms_eps);
       bool fused = false;
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.hn), W + lo.wgu, Ma, 2 * m, d, &part, s->wsp<uint8_t>(s->ws.ffn),
                          &fused)) != DLLM_OK)
@@ -579,7 +518,7 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
     }
     // FFNOut rows -> cache, residual assembly for all carried rows, next norm
     const float* gain_next = reinterpret_cast<const float*>(l + 1 < c.n_layers ? W + wl.layers[l + 1].norm1 : W + wl.norm_f);
-    launch_tail(L, dt, part, Ma > 0 ? inv : nullptr, x, s->cache(l, DLLM_CACHE_ATTN), s->cache(l, DLLM_CACHE_FFN),
+    launch_tail(L, dt, part, Ma > 0 ? inv : nullptr, x, s->outs(l, DLLM_CACHE_ATTN), s->outs(l, DLLM_CACHE_FFN),
                 gain_next, u, g, c0, c1, c.rms_eps);
   }
   // prediction at the response rows (Eqs. 3-4); u holds the final norm.  With head_len > 0 only the rows of
@@ -646,9 +585,7 @@ dllm_status run_step(dllm_session* s, int rp, int rr, const float* rhos, int n_r
   if (head_len < 0 || head_start < 0 || head_start + head_len > s->R)
     return fail(&s->err, DLLM_INVALID_ARG, "block [%d, %d) outside the response", head_start, head_start + head_len);
   if (head_len == s->R) head_start = head_len = 0;  // the whole response: the ordinary step
-  if (head_len == 0 && uniform && step_uses_mk(s, rp, ksels[0])) {
-    st = enqueue_step_mk(s, rr, ksels[0], stream);  // a handful of launches: no graph needed
-  } else if (!graph_ok) {
+  if (!graph_ok) {
     st = enqueue_step(s, rp, rr, ksels, stream, head_start, head_len);
   } else {
     StepKey key{rp, rr, ksels[0], forced_signature(s), s->sel_strategy * 4 + s->sel_metric * 2 + s->v_selected_only,
@@ -705,6 +642,24 @@ dllm_status run_step(dllm_session* s, int rp, int rr, const float* rhos, int n_r
 
 namespace dllm {
 void set_last_error(const char* msg) { g_err = msg ? msg : ""; }
+
+// Status word of the kernel-level entry points (they have no session whose workspace could hold one): a
+// file-scope device variable, one per GPU that loads the library, addressed through cudaGetSymbolAddress
+// once per device -- nothing is allocated.
+static __device__ int g_kernel_status = 0;
+int* kernel_status_word() {
+  static std::mutex mu;
+  static int* per_device[64] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!per_device[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_kernel_status) != cudaSuccess) return nullptr;
+    per_device[dev] = static_cast<int*>(p);
+  }
+  return per_device[dev];
+}
 }  // namespace dllm
 
 // =============================================================================
@@ -713,8 +668,17 @@ void set_last_error(const char* msg) { g_err = msg ? msg : ""; }
 extern "C" {
 
 const char* dllm_last_error(const void* handle) {
-  (void)handle;  // the message of the last failing call on this thread
-  return g_err.c_str();
+  if (handle) {
+    std::lock_guard<std::mutex> lock(g_handles_mu);
+    auto it = g_handles.find(handle);
+    if (it != g_handles.end()) {
+      // copied to a per-thread buffer: the handle's own string may change under another thread's call
+      thread_local std::string copy;
+      copy = *it->second;
+      return copy.c_str();
+    }
+  }
+  return g_err.c_str();  // NULL or unknown handle: the last failing call on this thread
 }
 
 size_t dllm_weights_bytes(const dllm_config* cfg) {
@@ -722,15 +686,20 @@ size_t dllm_weights_bytes(const dllm_config* cfg) {
   return make_layout(*cfg).total;
 }
 
-size_t dllm_cache_bytes(const dllm_config* cfg, int B, int P, int R) {
-  if (check_config(cfg) || B <= 0 || P <= 0 || R <= 0) return 0;
-  const size_t dkv = (size_t)cfg->n_kv_heads * cfg->head_dim;
-  return (size_t)cfg->n_layers * B * ((size_t)P + R) * (2 * dkv + 2 * (size_t)cfg->d_model) * esize(*cfg);
+size_t dllm_cache_bytes_ex(const dllm_config* cfg, int B, int P, int R, int flags) {
+  if (check_config(cfg) || B <= 0 || P <= 0 || R <= 0 || (flags & ~DLLM_SESSION_COMPACT_CACHE)) return 0;
+  const size_t dkv = (size_t)cfg->n_kv_heads * cfg->head_dim, n = (size_t)P + R;
+  const size_t out_rows = (flags & DLLM_SESSION_COMPACT_CACHE) ? (size_t)R : n;
+  return (size_t)cfg->n_layers * B * (n * 2 * dkv + out_rows * 2 * (size_t)cfg->d_model) * esize(*cfg);
 }
+size_t dllm_cache_bytes(const dllm_config* cfg, int B, int P, int R) { return dllm_cache_bytes_ex(cfg, B, P, R, 0); }
 
+size_t dllm_workspace_bytes_ex(const dllm_config* cfg, int B, int P, int R, int flags) {
+  if (check_config(cfg) || B <= 0 || P <= 0 || R <= 0 || (flags & ~DLLM_SESSION_COMPACT_CACHE)) return 0;
+  return make_workspace(*cfg, B, P, R, flags).total;
+}
 size_t dllm_workspace_bytes(const dllm_config* cfg, int B, int P, int R) {
-  if (check_config(cfg) || B <= 0 || P <= 0 || R <= 0) return 0;
-  return make_workspace(*cfg, B, P, R).total;
+  return dllm_workspace_bytes_ex(cfg, B, P, R, 0);
 }
 
 dllm_status dllm_tensor_offset(const dllm_config* cfg, const char* name, size_t* offset_bytes, size_t* n_elements) {
@@ -767,6 +736,7 @@ dllm_status dllm_model_create(const dllm_config* cfg, void* d_weights, dllm_mode
   m->cfg = *cfg;
   m->lay = make_layout(*cfg);
   m->d_w = static_cast<uint8_t*>(d_weights);
+  register_handle(m, &m->err);
   *out = m;
   return DLLM_OK;
 }
@@ -802,15 +772,22 @@ dllm_status dllm_model_set_tensor(dllm_model* m, const char* name, const float* 
 }
 
 dllm_status dllm_model_destroy(dllm_model* m) {
+  if (m) unregister_handle(m);
   delete m;
   return DLLM_OK;
 }
 
 dllm_status dllm_session_create(dllm_model* m, int B, int P, int R, void* d_cache, void* d_workspace, void* stream,
                                 dllm_session** out) {
+  return dllm_session_create_ex(m, B, P, R, 0, d_cache, d_workspace, stream, out);
+}
+
+dllm_status dllm_session_create_ex(dllm_model* m, int B, int P, int R, int flags, void* d_cache, void* d_workspace,
+                                   void* stream, dllm_session** out) {
   if (!out) return fail(nullptr, DLLM_INVALID_ARG, "out is NULL");
   *out = nullptr;
   if (!m) return fail(nullptr, DLLM_INVALID_ARG, "model is NULL");
+  if (flags & ~DLLM_SESSION_COMPACT_CACHE) return fail(&m->err, DLLM_INVALID_ARG, "unknown session flag");
   if (B <= 0 || P <= 0 || R <= 0) return fail(&m->err, DLLM_INVALID_ARG, "B, P and R must be positive");
   if (R > 8192) return fail(&m->err, DLLM_UNSUPPORTED, "R > 8192 is not supported by the selection kernel");
   if (!d_cache || !d_workspace || ((uintptr_t)d_cache & 255) || ((uintptr_t)d_workspace & 255))
@@ -824,7 +801,8 @@ dllm_status dllm_session_create(dllm_model* m, int B, int P, int R, void* d_cach
   s->n = P + R;
   s->d_cache = static_cast<uint8_t*>(d_cache);
   s->d_ws = static_cast<uint8_t*>(d_workspace);
-  s->ws = make_workspace(m->cfg, B, P, R);
+  s->compact = (flags & DLLM_SESSION_COMPACT_CACHE) != 0;
+  s->ws = make_workspace(m->cfg, B, P, R, flags);
   s->forced_count.assign(m->cfg.n_layers, -1);
   cudaStream_t st = (cudaStream_t)stream;
   // rotary table: [pos][cos(hd/2) | sin(hd/2)], angle = pos * theta^(-2i/hd), evaluated in double
@@ -836,7 +814,7 @@ dllm_status dllm_session_create(dllm_model* m, int B, int P, int R, void* d_cach
       tab[(size_t)pos * hd + i] = (float)cos(ang);
       tab[(size_t)pos * hd + half + i] = (float)sin(ang);
     }
-  cudaError_t e = cudaMemsetAsync(d_cache, 0, dllm_cache_bytes(&m->cfg, B, P, R), st);
+  cudaError_t e = cudaMemsetAsync(d_cache, 0, dllm_cache_bytes_ex(&m->cfg, B, P, R, flags), st);
   // everything but the (large) GEMM slab is cleared; the slab is always written before it is read
   if (e == cudaSuccess) e = cudaMemsetAsync(d_workspace, 0, s->ws.part, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -845,12 +823,14 @@ dllm_status dllm_session_create(dllm_model* m, int B, int P, int R, void* d_cach
     delete s;
     return fail(&m->err, DLLM_CUDA_ERROR, "session setup: %s", cudaGetErrorString(e));
   }
+  register_handle(s, &s->err);
   *out = s;
   return DLLM_OK;
 }
 
 dllm_status dllm_session_destroy(dllm_session* s) {
   if (!s) return DLLM_OK;
+  unregister_handle(s);
   for (auto& kv : s->graphs) cudaGraphExecDestroy(kv.second.exec);
   for (auto& r : s->prof) {
     cudaEventDestroy(r.a);
@@ -959,16 +939,43 @@ dllm_status dllm_generate(dllm_session* s, int K, int Kp, int Kr, float rho, dll
   return DLLM_OK;
 }
 
+// Reads and clears a device status word after the stream has drained.
+static dllm_status read_status_word(std::string* slot, int* d_word, cudaStream_t stream) {
+  CU_TRY(slot, cudaStreamSynchronize(stream));
+  int code = 0;
+  CU_TRY(slot, cudaMemcpy(&code, d_word, 4, cudaMemcpyDeviceToHost));
+  if (code == 0) return DLLM_OK;
+  cudaMemsetAsync(d_word, 0, 4, stream);
+  cudaStreamSynchronize(stream);
+  if (code >= 100 && code < 200) return fail(slot, DLLM_TIMEOUT, "a device-side wait gave up (code %d)", code);
+  return fail(slot, DLLM_CUDA_ERROR, "device status %d", code);
+}
+
 dllm_status dllm_sync(dllm_session* s, void* stream) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
-  CU_TRY(&s->err, cudaStreamSynchronize((cudaStream_t)stream));
-  int code = 0;
-  CU_TRY(&s->err, cudaMemcpy(&code, s->d_ws + s->ws.status, 4, cudaMemcpyDeviceToHost));
-  if (code == 0) return DLLM_OK;
-  cudaMemsetAsync(s->d_ws + s->ws.status, 0, 4, (cudaStream_t)stream);
-  cudaStreamSynchronize((cudaStream_t)stream);
-  if (code >= 100 && code < 200) return fail(&s->err, DLLM_TIMEOUT, "a device-side wait gave up (code %d)", code);
-  return fail(&s->err, DLLM_CUDA_ERROR, "device status %d", code);
+  return read_status_word(&s->err, s->wsp<int>(s->ws.status), (cudaStream_t)stream);
+}
+
+dllm_status dllm_kernel_status(void* stream) {
+  int* w = kernel_status_word();
+  if (!w) return fail(nullptr, DLLM_CUDA_ERROR, "no status word on this device");
+  return read_status_word(nullptr, w, (cudaStream_t)stream);
+}
+
+dllm_status dllm_debug_set_wait_limit_ns(uint64_t ns) {
+  CU_TRY(nullptr, cudaDeviceSynchronize());
+  CU_TRY(nullptr, set_wait_limit_gemm_tcgen05(ns));
+  CU_TRY(nullptr, set_wait_limit_attention(ns));
+  CU_TRY(nullptr, set_wait_limit_attention_umma(ns));
+  CU_TRY(nullptr, cudaDeviceSynchronize());
+  return DLLM_OK;
+}
+
+dllm_status dllm_debug_skip_one_load(int enable) {
+  CU_TRY(nullptr, cudaDeviceSynchronize());
+  CU_TRY(nullptr, set_debug_skip_act_load(enable));
+  CU_TRY(nullptr, cudaDeviceSynchronize());
+  return DLLM_OK;
 }
 
 dllm_status dllm_get_tokens(dllm_session* s, int32_t* h_out, void* stream) {
@@ -1053,8 +1060,7 @@ static dllm_status cache_args(dllm_session* s, int layer, int which, const void*
   if (!p) return fail(&s->err, DLLM_INVALID_ARG, "host buffer is NULL");
   if (layer < 0 || layer >= s->m->cfg.n_layers) return fail(&s->err, DLLM_INVALID_ARG, "layer out of range");
   if (which < DLLM_CACHE_K || which > DLLM_CACHE_FFN) return fail(&s->err, DLLM_INVALID_ARG, "bad cache id");
-  const size_t width = which <= DLLM_CACHE_V ? s->dkv() : (size_t)s->m->cfg.d_model;
-  *n_elems = (size_t)s->B * s->n * width;
+  *n_elems = which <= DLLM_CACHE_V ? (size_t)s->B * s->n * s->dkv() : s->out_rows() * (size_t)s->m->cfg.d_model;
   return DLLM_OK;
 }
 
@@ -1147,12 +1153,6 @@ dllm_status dllm_set_scores(dllm_session* s, int layer, const float* h_scores, v
   return DLLM_OK;
 }
 
-dllm_status dllm_session_use_layer_kernel(dllm_session* s, int enable) {
-  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
-  s->use_mk = enable != 0;
-  return DLLM_OK;
-}
-
 dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
   if ((enable != 0) != s->simt_gemm) {
@@ -1211,7 +1211,7 @@ dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, 
   if (K % 8) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8");
   const GemmPlan p = plan_gemm_bf16(M, N, K);
   if (p.S_max > 1 && !d_partials) return fail(nullptr, DLLM_INVALID_ARG, "this shape needs slab scratch");
-  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  Launch L{(cudaStream_t)stream, kernel_status_word(), nullptr};
   float* part = p.S_max > 1 ? static_cast<float*>(d_partials) : d_C;
   const char* why = nullptr;
   cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
@@ -1237,7 +1237,7 @@ dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C,
   const GemmPlan p = plan_gemm_bf16(M, N, K, splits, stages, act_tile);
   if (p.S_max > 1 && (!d_partials || partials_bytes < (size_t)p.S_max * M * N * 4))
     return fail(nullptr, DLLM_INVALID_ARG, "this plan needs %zu bytes of slab scratch", (size_t)p.S_max * M * N * 4);
-  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  Launch L{(cudaStream_t)stream, kernel_status_word(), nullptr};
   if (!d_C && (p.S_max == 1 || !d_partials)) return fail(nullptr, DLLM_INVALID_ARG, "d_C is NULL");
   float* part = p.S_max > 1 ? static_cast<float*>(d_partials) : d_C;
   const char* why = nullptr;
@@ -1256,7 +1256,7 @@ dllm_status dllm_ffn_gate_up_bf16(const void* d_A, const void* d_Wgu, void* d_ou
   if (act_tile < 0 || stages < 0 || (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 256))
     return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128 or 256");
   const GemmPlan p = plan_gemm_bf16(M, 2 * d_ffn, K, 1, stages, act_tile);
-  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  Launch L{(cudaStream_t)stream, kernel_status_word(), nullptr};
   const char* why = nullptr;
   cudaError_t e = launch_gemm_bf16(L, d_A, d_Wgu, nullptr, M, 2 * d_ffn, K, p, &why, d_out, d_ffn);
   if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "gate / up GEMM: %s", why ? why : cudaGetErrorString(e));
@@ -1279,7 +1279,7 @@ dllm_status dllm_gemm_bf16_pair(const void* d_A, const void* d_W, float* d_C, in
   const GemmPlan p = plan_gemm_bf16(M, N, K, splits, stages, act_tile, 1);
   if (p.S_max > 1 && (!d_partials || partials_bytes < (size_t)p.S_max * M * N * 4))
     return fail(nullptr, DLLM_INVALID_ARG, "this plan needs %zu bytes of slab scratch", (size_t)p.S_max * M * N * 4);
-  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  Launch L{(cudaStream_t)stream, kernel_status_word(), nullptr};
   float* part = p.S_max > 1 ? static_cast<float*>(d_partials) : d_C;
   const char* why = nullptr;
   cudaError_t e = launch_gemm_bf16(L, d_A, d_W, part, M, N, K, p, &why);
@@ -1293,7 +1293,7 @@ dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, 
                            void* stream) {
   if (!d_A || !d_W || !d_C || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
   if (dtype != DLLM_FP32 && dtype != DLLM_BF16) return fail(nullptr, DLLM_INVALID_ARG, "bad dtype");
-  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  Launch L{(cudaStream_t)stream, kernel_status_word(), nullptr};
   launch_gemm_simt(L, dtype, d_A, d_W, d_C, M, N, K);
   CU_TRY(nullptr, cudaGetLastError());
   return DLLM_OK;
@@ -1302,7 +1302,7 @@ dllm_status dllm_gemm_simt(const void* d_A, const void* d_W, float* d_C, int M, 
 size_t dllm_attention_scratch_bytes(int B, int a, int n, int H, int Hkv, int hd, int dtype) {
   if (B <= 0 || a <= 0 || n <= 0 || H <= 0 || Hkv <= 0 || H % Hkv || dtype != DLLM_BF16 || (hd != 64 && hd != 128))
     return 0;
-  return plan_attention(B, a, n, H, Hkv).scratch_floats * 4;
+  return choose_attention(B, a, n, H, Hkv, SIZE_MAX).plan.scratch_floats * 4;
 }
 
 dllm_status dllm_attention(const void* d_q, const void* d_k, const void* d_v, void* d_o, int B, int a, int n, int H,
@@ -1311,7 +1311,7 @@ dllm_status dllm_attention(const void* d_q, const void* d_k, const void* d_v, vo
     return fail(nullptr, DLLM_INVALID_ARG, "bad attention arguments");
   if (dtype != DLLM_FP32 && dtype != DLLM_BF16) return fail(nullptr, DLLM_INVALID_ARG, "bad dtype");
   if (hd % 32 || hd > 128) return fail(nullptr, DLLM_UNSUPPORTED, "head_dim must be 32, 64, 96 or 128");
-  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  Launch L{(cudaStream_t)stream, kernel_status_word(), nullptr};
   cudaError_t e = launch_attention(L, dtype, d_q, d_k, d_v, d_o, B, a, n, H, Hkv, hd, static_cast<float*>(d_scratch),
                                    scratch_bytes / 4, false);
   if (e != cudaSuccess) return fail(nullptr, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
@@ -1324,9 +1324,9 @@ dllm_status dllm_vverify_select(const void* d_vnew, void* d_vcache, float* d_sim
     return fail(nullptr, DLLM_INVALID_ARG, "bad V-verify arguments");
   if (dtype != DLLM_FP32 && dtype != DLLM_BF16) return fail(nullptr, DLLM_INVALID_ARG, "bad dtype");
   if (width % 8 || R > 8192) return fail(nullptr, DLLM_UNSUPPORTED, "width must be a multiple of 8 and R <= 8192");
-  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  Launch L{(cudaStream_t)stream, kernel_status_word(), nullptr};
   launch_vverify_rows(L, dtype, d_vnew, d_vcache, d_sim, B * R, width);
-  if (k > 0) launch_select(L, d_sim, nullptr, 1, k, d_idx, k, nullptr, nullptr, Geo{B, 0, R, R, width}, 0);
+  if (k > 0) CU_TRY(nullptr, launch_select(L, d_sim, nullptr, 1, k, d_idx, k, nullptr, nullptr, Geo{B, 0, R, R, width}, 0));
   CU_TRY(nullptr, cudaGetLastError());
   return DLLM_OK;
 }

@@ -239,12 +239,10 @@ template <int HD>
 cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
                        float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
   constexpr int SMEM = AT_ROWS * HD * 2 + 2 * 2 * AT_KEYS * HD * 2 + 1024;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static DeviceOnce once;
+  cudaError_t e0 = once.run(
+      [] { return cudaFuncSetAttribute(attn_mma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM); });
+  if (e0 != cudaSuccess) return e0;
   const int G = H / Hkv;
   const size_t total = (size_t)B * a_seq * H;
   float* o_part = scratch;
@@ -255,14 +253,12 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
   CUtensorMap tmQ = tmK;
   const int q_by_tma = H == Hkv && ((uintptr_t)q & 15) == 0 &&
                        get_tensor_map_2d(q, (uint64_t)B * a_seq, (uint64_t)H * HD, AT_ROWS, &tmQ);
-  launch_k(L, attn_mma_kernel<HD>, dim3(grid), dim3(128), SMEM, tmK, tmV, tmQ, q_by_tma, (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part,
-                                                     ml_part, a_seq, n, H, Hkv, S, keys_per_split, scale_log2,
-                                                     L.d_status);
+  cudaError_t e = launch_k(L, attn_mma_kernel<HD>, dim3(grid), dim3(128), SMEM, tmK, tmV, tmQ, q_by_tma,
+                           (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S,
+                           keys_per_split, scale_log2, L.d_status);
   L.count();
-  if (S > 1) {
-    launch_combine(L, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
-  }
-  return cudaGetLastError();
+  if (e == cudaSuccess && S > 1) e = launch_combine(L, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
@@ -271,10 +267,10 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
 // when few rows are active, whole 64-key tiles per split.
 AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv) {
   AttnPlan p;
-  const int G = H / Hkv;
+  const int G = H / Hkv, sms = sm_count();
   const long tiles = (long)((a_seq * G + AT_ROWS - 1) / AT_ROWS) * Hkv * B;
   int S = 1;
-  if (tiles < 148) S = (int)((148 + tiles - 1) / tiles);
+  if (tiles < sms) S = (int)((sms + tiles - 1) / tiles);
   const int key_tiles = (n + AT_KEYS - 1) / AT_KEYS;
   if (S > key_tiles) S = key_tiles;
   const int tiles_per_split = (key_tiles + S - 1) / S;
@@ -284,13 +280,33 @@ AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv) {
   return p;
 }
 
+// Which tensor-core kernel a bf16 shape takes, and its plan when the caller offers `scratch_floats` floats of
+// scratch (SIZE_MAX: as much as the plan would like).  The 64-row mma.sync kernel never shrinks its plan: without
+// room for the partials it runs one split.  The 128-row tcgen05 kernel lowers its split count to what fits.
+AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats) {
+  AttnChoice c;
+  c.umma = a_seq * (H / Hkv) > AT_ROWS;
+  if (c.umma) {
+    c.plan = plan_attention_umma(B, a_seq, n, H, Hkv, scratch_floats);
+  } else {
+    c.plan = plan_attention(B, a_seq, n, H, Hkv);
+    if (c.plan.S > 1 && scratch_floats < c.plan.scratch_floats) {
+      c.plan.S = 1;
+      c.plan.keys_per_split = ((n + AT_KEYS - 1) / AT_KEYS) * AT_KEYS;
+      c.plan.scratch_floats = 0;
+    }
+  }
+  return c;
+}
+
 cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const void* Kc, const void* Vc, void* o, int B,
                              int a_seq, int n, int H, int Hkv, int hd, float* scratch, size_t scratch_floats,
                              bool force_simt) {
   if (B <= 0 || a_seq <= 0) return cudaSuccess;
   if (hd > HD_MAX || (hd & 31) || H % Hkv) return cudaErrorInvalidValue;
   const bool tensor = dtype == 1 && !force_simt && (hd == 64 || hd == 128) && ((Hkv * hd) % 8 == 0);
-  if (tensor && a_seq * (H / Hkv) > AT_ROWS) {
+  const AttnChoice ch = tensor ? choose_attention(B, a_seq, n, H, Hkv, scratch ? scratch_floats : 0) : AttnChoice{};
+  if (tensor && ch.umma) {
     // many active rows per KV head: 128-row tiles on tcgen05
     int S = 1;
     cudaError_t e = launch_attention_umma(L, q, Kc, Vc, o, B, a_seq, n, H, Hkv, hd, scratch, scratch_floats, &S);
@@ -302,11 +318,7 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
     return e != cudaSuccess ? e : cudaGetLastError();
   }
   if (tensor) {
-    AttnPlan p = plan_attention(B, a_seq, n, H, Hkv);
-    if (p.S > 1 && (!scratch || scratch_floats < p.scratch_floats)) {   // no room for partials: one split
-      p.S = 1;
-      p.keys_per_split = ((n + AT_KEYS - 1) / AT_KEYS) * AT_KEYS;
-    }
+    const AttnPlan p = ch.plan;
     CUtensorMap tmK, tmV;
     if (!get_tensor_map_3d(Kc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, AT_KEYS, &tmK) ||
         !get_tensor_map_3d(Vc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, AT_KEYS, &tmV))
@@ -388,13 +400,15 @@ extern "C" dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, 
     set_last_error("dllm_attention_noalloc: bf16 tensor-core path only, head_dim must be 64 or 128");
     return DLLM_UNSUPPORTED;
   }
-  const AttnPlan plan = plan_attention(B, a, n, H, Hkv);
-  if (plan.scratch_floats > NOALLOC_SCRATCH_FLOATS) {
+  // the plan the kernels would take with unlimited scratch: the call must run exactly what dllm_attention runs
+  // with a buffer of dllm_attention_scratch_bytes(), so a plan that does not fit the array is refused, not shrunk
+  const AttnChoice want = choose_attention(B, a, n, H, Hkv, SIZE_MAX);
+  if (want.plan.scratch_floats > NOALLOC_SCRATCH_FLOATS) {
     char msg[256];
     snprintf(msg, sizeof msg,
-             "dllm_attention_noalloc: this shape splits the key range %d ways and needs %zu bytes of scratch, the "
-             "built-in array holds %zu; use dllm_attention with a caller-owned scratch buffer",
-             plan.S, plan.scratch_floats * sizeof(float), NOALLOC_SCRATCH_BYTES);
+             "dllm_attention_noalloc: this shape splits the key range %d ways (%d-row tiles) and needs %zu bytes of "
+             "scratch, the built-in array holds %zu; use dllm_attention with a caller-owned scratch buffer",
+             want.plan.S, want.umma ? 128 : 64, want.plan.scratch_floats * sizeof(float), NOALLOC_SCRATCH_BYTES);
     set_last_error(msg);
     return DLLM_UNSUPPORTED;
   }
@@ -405,8 +419,8 @@ extern "C" dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, 
     return DLLM_CUDA_ERROR;
   }
   // Nothing in the scratch has to start at zero: every partial (output, max,
-  // sum) that attn_combine_kernel reads is written by this call's attn_mma_kernel first.
-  Launch L{(cudaStream_t)stream, nullptr, nullptr};
+  // sum) that attn_combine_kernel reads is written by this call's attention kernel first.
+  Launch L{(cudaStream_t)stream, kernel_status_word(), nullptr};
   e = launch_attention(L, DLLM_BF16, d_q, d_k, d_v, d_o, B, a, n, H, Hkv, hd, scratch, NOALLOC_SCRATCH_FLOATS, false);
   if (e != cudaSuccess) {
     set_last_error(cudaGetErrorString(e));
@@ -416,3 +430,4 @@ extern "C" dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, 
 }
 
 DLLM_TIMELINE_HOOKS(attention)
+DLLM_WAIT_LIMIT_HOOK(attention)

@@ -385,12 +385,10 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
                         int q_by_tma, const void* q, void* o,
                         float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
   constexpr int SMEM = (int)UaSmem<HD>::TOTAL;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static DeviceOnce once;
+  cudaError_t e0 = once.run(
+      [] { return cudaFuncSetAttribute(attn_umma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM); });
+  if (e0 != cudaSuccess) return e0;
   const int G = H / Hkv;
   const size_t total = (size_t)B * a_seq * H;
   float* o_part = scratch;
@@ -410,10 +408,10 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
 // 128-key tiles per split, no more splits than the scratch holds.
 AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats) {
   AttnPlan p;
-  const int G = H / Hkv;
+  const int G = H / Hkv, sms = sm_count();
   const long tiles = (long)((a_seq * G + UA_ROWS - 1) / UA_ROWS) * Hkv * B;
   int S = 1;
-  if (tiles < 148) S = (int)((148 + tiles - 1) / tiles);
+  if (tiles < sms) S = (int)((sms + tiles - 1) / tiles);
   const int key_tiles = (n + UA_KEYS - 1) / UA_KEYS;
   if (S > key_tiles) S = key_tiles;
   const size_t per_split = (size_t)B * a_seq * H * (128 + 2);
@@ -446,3 +444,4 @@ cudaError_t launch_attention_umma(const Launch& L, const void* q, const void* Kc
 }  // namespace dllm
 
 DLLM_TIMELINE_HOOKS(attention_umma)
+DLLM_WAIT_LIMIT_HOOK(attention_umma)

@@ -26,6 +26,26 @@ __host__ __device__ inline void carried_to_pos(int c, const Geo& g, int& b, int&
   }
 }
 
+// Where the AttnOut / FFNOut row of a carried row lives.  Four-tensor layout (compact == 0): `base` is the
+// layer's [B, n, d] tensor and the row of carried row c sits at its (sequence, position).  Compact layout
+// (compact == 1): `base` is the layer's response-only tensor [B, R, d], which is carried order itself, and
+// the prompt rows (alive only inside a prompt-refresh step) sit in `prompt`, [B, P, d] in carried order.
+struct OutRows {
+  void* base;
+  void* prompt;
+  int compact;
+  template <typename T>
+  __device__ __forceinline__ T* row(int c, const Geo& g) const {
+    if (compact) {
+      const int BR = g.B * g.R;
+      return c < BR ? static_cast<T*>(base) + (size_t)c * g.d : static_cast<T*>(prompt) + (size_t)(c - BR) * g.d;
+    }
+    int b, pos;
+    carried_to_pos(c, g, b, pos);
+    return static_cast<T*>(base) + ((size_t)b * g.n + pos) * g.d;
+  }
+};
+
 // device status word codes
 enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103, ST_TIMEOUT_GRID = 104, ST_RANGE = 201 };
 

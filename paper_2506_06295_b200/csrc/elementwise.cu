@@ -53,31 +53,6 @@ __device__ __forceinline__ void sum_partials4(const Partials& part, int row, int
   }
 }
 
-// ------------------------------------------------------------------ embed
-template <typename T>
-__global__ void embed_kernel(const T* __restrict__ E, const int32_t* __restrict__ tokens, float* __restrict__ x, Geo g,
-                             int c0) {
-  pdl_wait();
-  pdl_trigger();
-  const int c = c0 + blockIdx.x;
-  int b, pos;
-  carried_to_pos(c, g, b, pos);
-  const int tok = tokens[(size_t)b * g.n + pos];
-  const T* src = E + (size_t)tok * g.d;
-  float* dst = x + (size_t)c * g.d;
-  for (int i = threadIdx.x * 8; i < g.d; i += blockDim.x * 8) {
-    float v[8];
-    Vec8<T>::load(src + i, v);
-    Vec8<float>::store(dst + i, v);
-  }
-}
-
-void launch_embed(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, Geo g, int c0, int c1) {
-  if (c1 <= c0) return;
-  DLLM_DISPATCH(dtype, (launch_k(L, embed_kernel<T>, dim3(c1 - c0), dim3(128), 0, (const T*)E, tokens, x, g, c0)));
-  L.count();
-}
-
 // ------------------------------------------------------------------ rmsnorm
 template <typename T>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain, T* __restrict__ out, int d,
@@ -410,12 +385,21 @@ __global__ void select_kernel(const float* __restrict__ sim, const int32_t* __re
   }
 }
 
-void launch_select(const Launch& L, const float* sim, const int32_t* forced, int mode, int ksel, int32_t* sel,
-                   int sel_stride, int32_t* act, int32_t* inv, Geo g, int refresh_prompt) {
+cudaError_t launch_select(const Launch& L, const float* sim, const int32_t* forced, int mode, int ksel, int32_t* sel,
+                          int sel_stride, int32_t* act, int32_t* inv, Geo g, int refresh_prompt) {
+  // 9 bytes per response row: beyond 48 KB (R > 5459) the kernel needs the opt-in for large dynamic shared memory
+  constexpr int MAX_R = 8192;
+  if (g.R > MAX_R) return cudaErrorInvalidValue;
+  static DeviceOnce once;
+  cudaError_t e = once.run([] {
+    return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_R * 9 + 16);
+  });
+  if (e != cudaSuccess) return e;
   const size_t smem = (size_t)g.R * 9 + 16;
-  launch_k(L, select_kernel, dim3(g.B), dim3(256), smem, sim, forced, mode, ksel, sel, sel_stride, act, inv, g,
-           refresh_prompt);
+  e = launch_k(L, select_kernel, dim3(g.B), dim3(256), smem, sim, forced, mode, ksel, sel, sel_stride, act, inv, g,
+               refresh_prompt);
   L.count();
+  return e;
 }
 
 // ------------------------------------------------------------------ gather
@@ -514,7 +498,7 @@ void launch_scatter_rows(const Launch& L, int dtype, Partials part, const int32_
 // hn = rmsnorm(h) * gain2.
 template <typename T>
 __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ x,
-                                      const float* __restrict__ gain2, T* __restrict__ Ac, T* __restrict__ hn, Geo g,
+                                      const float* __restrict__ gain2, OutRows Ac, T* __restrict__ hn, Geo g,
                                       float eps) {
   pdl_wait();
   pdl_trigger();
@@ -527,9 +511,7 @@ __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__
   float hv[8], gv[8];
   if (one_trip && i0 < d) Vec8<float>::load(gain2 + i0, gv);  // independent of the row: ahead of the dependent loads
   const int c = act[r];
-  int b, pos;
-  carried_to_pos(c, g, b, pos);
-  T* arow = Ac + ((size_t)b * g.n + pos) * d;
+  T* arow = Ac.row<T>(c, g);
   const float* xr = x + (size_t)c * d;
   float ss = 0.f;
   for (int i = i0; i < d; i += blockDim.x * 8) {
@@ -568,12 +550,12 @@ __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__
 }
 
 void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int32_t* act, const float* x,
-                           const float* gain2, void* Ac_layer, void* hn, Geo g, int Ma, float eps) {
+                           const float* gain2, OutRows Ac_layer, void* hn, Geo g, int Ma, float eps) {
   if (Ma <= 0) return;
   const int threads = row_threads(g.d);
   const size_t smem = g.d <= threads * 8 ? 0 : (size_t)g.d * sizeof(float);  // staging only if a row takes several passes
-  DLLM_DISPATCH(dtype, (launch_k(L, oproj_epilogue_kernel<T>, dim3(Ma), dim3(threads), smem, part, act, x, gain2, (T*)Ac_layer,
-                                                                            (T*)hn, g, eps)));
+  DLLM_DISPATCH(dtype, (launch_k(L, oproj_epilogue_kernel<T>, dim3(Ma), dim3(threads), smem, part, act, x, gain2, Ac_layer,
+                                 (T*)hn, g, eps)));
   L.count();
 }
 
@@ -601,36 +583,6 @@ void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int M
   const size_t total = (size_t)Ma * (m >> 3);
   const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
   DLLM_DISPATCH(dtype, (launch_k(L, silu_mul_kernel<T>, dim3(blocks), dim3(256), 0, part, (T*)out, Ma, m, interleaved)));
-  L.count();
-}
-
-// ------------------------------------------------------------------ residual assembly
-template <typename T>
-__global__ void residual_kernel(float* __restrict__ x, const T* __restrict__ Ac, const T* __restrict__ Fc, Geo g,
-                                int c0) {
-  pdl_wait();
-  pdl_trigger();
-  const int c = c0 + blockIdx.x;
-  int b, pos;
-  carried_to_pos(c, g, b, pos);
-  const size_t crow = ((size_t)b * g.n + pos) * g.d;
-  float* xr = x + (size_t)c * g.d;
-  for (int i = threadIdx.x * 8; i < g.d; i += blockDim.x * 8) {
-    float xv[8], a[8], f[8];
-    Vec8<float>::load(xr + i, xv);
-    Vec8<T>::load(Ac + crow + i, a);
-    Vec8<T>::load(Fc + crow + i, f);
-#pragma unroll
-    for (int t = 0; t < 8; ++t) xv[t] = (xv[t] + a[t]) + f[t];
-    Vec8<float>::store(xr + i, xv);
-  }
-}
-
-void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer, const void* Fc_layer, Geo g, int c0,
-                     int c1) {
-  if (c1 <= c0) return;
-  DLLM_DISPATCH(dtype,
-                (launch_k(L, residual_kernel<T>, dim3(c1 - c0), dim3(row_threads(g.d)), 0, x, (const T*)Ac_layer, (const T*)Fc_layer, g, c0)));
   L.count();
 }
 
@@ -685,17 +637,16 @@ void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t*
 // final norm after the last layer).  inv == nullptr: no row is active.
 template <typename T>
 __global__ void __launch_bounds__(512, 2) tail_kernel(Partials part, const int32_t* __restrict__ inv, float* __restrict__ x,
-                            const T* __restrict__ Ac, T* __restrict__ Fc, const float* __restrict__ gain,
+                            OutRows Ac, OutRows Fc, const float* __restrict__ gain,
                             T* __restrict__ u, Geo g, int c0, float eps) {
   pdl_wait();
   pdl_trigger();
   extern __shared__ float hrow[];
   __shared__ float red[32];
   const int c = c0 + blockIdx.x;
-  int b, pos;
-  carried_to_pos(c, g, b, pos);
   const int d = g.d;
-  const size_t crow = ((size_t)b * g.n + pos) * d;
+  const T* arow = Ac.row<T>(c, g);
+  T* frow = Fc.row<T>(c, g);
   const bool one_trip = d <= (int)blockDim.x * 8;  // the row fits one pass: it stays in registers
   const int i0 = threadIdx.x * 8;
   float hv[8], gv[8];
@@ -706,14 +657,14 @@ __global__ void __launch_bounds__(512, 2) tail_kernel(Partials part, const int32
   for (int i = i0; i < d; i += blockDim.x * 8) {
     float xv[8], a[8], f[8];
     Vec8<float>::load(xr + i, xv);
-    Vec8<T>::load(Ac + crow + i, a);
+    Vec8<T>::load(arow + i, a);
     if (r >= 0) {
       sum_partials8(part.p, part.split_stride, part.count(r, i), (size_t)r * part.N + i, f);
-      Vec8<T>::store(Fc + crow + i, f);
+      Vec8<T>::store(frow + i, f);
 #pragma unroll
       for (int t = 0; t < 8; ++t) f[t] = Vec8<T>::round(f[t]);
     } else {
-      Vec8<T>::load(Fc + crow + i, f);
+      Vec8<T>::load(frow + i, f);
     }
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
@@ -745,13 +696,13 @@ __global__ void __launch_bounds__(512, 2) tail_kernel(Partials part, const int32
   }
 }
 
-void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, const void* Ac_layer,
-                 void* Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps) {
+void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, OutRows Ac_layer,
+                 OutRows Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps) {
   if (c1 <= c0) return;
   const int threads = row_threads(g.d);
   const size_t smem = g.d <= threads * 8 ? 0 : (size_t)g.d * sizeof(float);  // staging only if a row takes several passes
-  DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T>, dim3(c1 - c0), dim3(threads), smem, part, inv, x, (const T*)Ac_layer,
-                                 (T*)Fc_layer, gain, (T*)u, g, c0, eps)));
+  DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T>, dim3(c1 - c0), dim3(threads), smem, part, inv, x, Ac_layer,
+                                 Fc_layer, gain, (T*)u, g, c0, eps)));
   L.count();
 }
 

@@ -45,6 +45,11 @@ constexpr int TILE_K = 64;   // k per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr uint32_t W_STAGE_BYTES = TILE_W * TILE_K * 2;
 
+// Test hook for the bounded waits: while non-zero, the TMA producer of CTA (0, 0, 0) of every launch of the
+// one-CTA kernel leaves out the activation tile of its first k-block, so that stage's barrier never completes
+// and the CTA's waits run into their limit (it then records a status code and returns; nothing faults).
+static __device__ int g_debug_skip_act_load = 0;
+
 constexpr int MAX_STAGES = 12;
 constexpr int RASTER = 16;     // activation tiles per group of the launch-order remap
 
@@ -272,7 +277,8 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
         mbar_expect_tx(fb, SL::STAGE_BYTES);
         tma_load_2d(dstW, &tmW, fb, kc, n0);
       }
-      tma_load_2d(dstW + W_STAGE_BYTES, &tmA, fb, kc, m0);
+      const bool skip = i == 0 && g_debug_skip_act_load != 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
+      if (!skip) tma_load_2d(dstW + W_STAGE_BYTES, &tmA, fb, kc, m0);
       if (++s == STAGES) {
         s = 0;
         ph ^= 1u;
@@ -494,8 +500,10 @@ struct MapKey {
   const void* base;
   uint64_t batch, rows, cols;
   uint32_t box_rows;
+  int device;  // a map is encoded in the context of the device that was current
   bool operator==(const MapKey& o) const {
-    return base == o.base && batch == o.batch && rows == o.rows && cols == o.cols && box_rows == o.box_rows;
+    return base == o.base && batch == o.batch && rows == o.rows && cols == o.cols && box_rows == o.box_rows &&
+           device == o.device;
   }
 };
 struct MapKeyHash {
@@ -503,7 +511,7 @@ struct MapKeyHash {
     size_t h = std::hash<const void*>()(k.base);
     h ^= std::hash<uint64_t>()(k.rows * 1315423911ull + k.cols + k.batch * 2654435761ull) + 0x9e3779b97f4a7c15ull +
          (h << 6) + (h >> 2);
-    return h ^ (k.box_rows * 2654435761u);
+    return h ^ (k.box_rows * 2654435761u) ^ ((size_t)k.device << 56);
   }
 };
 
@@ -544,13 +552,12 @@ template <int BN>
 cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMap& tmA, float* part, int M, int N,
                        int num_kb, const GemmPlan& plan, void* act_out, int m_ffn) {
   using SL = SmemLayout<BN>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)SL::total(max_stages(BN)));
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static DeviceOnce once;
+  cudaError_t e0 = once.run([] {
+    return cudaFuncSetAttribute(gemm_bf16_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)SL::total(max_stages(BN)));
+  });
+  if (e0 != cudaSuccess) return e0;
   const int stages = plan.stages < 2 ? 2 : plan.stages > max_stages(BN) ? max_stages(BN) : plan.stages;
   dim3 grid((M + BN - 1) / BN, (N + TILE_W - 1) / TILE_W, plan.S_max);
   cudaError_t e = launch_k(L, gemm_bf16_tcgen05_kernel<BN>, grid, dim3(128), SL::total(stages), tmW, tmA, part, M, N,
@@ -565,13 +572,12 @@ cudaError_t launch_pair(const Launch& L, const CUtensorMap& tmW, const CUtensorM
   using PL = PairLayout<BN>;
   constexpr int fit = (227 * 1024 - 1024 - 256) / (int)PL::STAGE_BYTES;
   constexpr int most = fit < MAX_STAGES ? fit : MAX_STAGES;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_bf16_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)PL::total(most));
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static DeviceOnce once;
+  cudaError_t e0 = once.run([] {
+    return cudaFuncSetAttribute(gemm_bf16_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)PL::total(most));
+  });
+  if (e0 != cudaSuccess) return e0;
   const int stages = plan.stages < 2 ? 2 : plan.stages > most ? most : plan.stages;
   dim3 grid(N / TILE_W, (M + BN - 1) / BN, plan.S_max);  // pairs along x
   cudaError_t e = launch_k_cluster(L, gemm_bf16_pair_kernel<BN>, grid, dim3(128), PL::total(stages), dim3(2, 1, 1), tmW,
@@ -583,25 +589,27 @@ cudaError_t launch_pair(const Launch& L, const CUtensorMap& tmW, const CUtensorM
 
 }  // namespace
 
+static int current_device() {
+  int dev = 0;
+  return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
 bool get_tensor_map_2d(const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
-  return get_map(MapKey{base, 0, rows, cols, box_rows}, out);
+  return get_map(MapKey{base, 0, rows, cols, box_rows, current_device()}, out);
 }
 bool get_tensor_map_3d(const void* base, uint64_t batch, uint64_t rows, uint64_t cols, uint32_t box_rows,
                        CUtensorMap* out) {
-  return get_map(MapKey{base, batch, rows, cols, box_rows}, out);
+  return get_map(MapKey{base, batch, rows, cols, box_rows, current_device()}, out);
 }
 
 int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-      n = v;
-    else
-      return 148;  // no device visible (host-only size queries): a B200's count
-  }
-  return n;
+  static std::atomic<int> per_device[64];  // zero-initialised: not yet asked
+  int dev = 0, v = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;  // no device visible (host-only size queries): a B200's count
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && (v = per_device[dev].load(std::memory_order_relaxed)) > 0) return v;
+  if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+  if (tracked) per_device[dev].store(v, std::memory_order_relaxed);
+  return v;
 }
 
 Partials make_partials(const float* p, int M, int N, const GemmPlan& plan) {
@@ -694,4 +702,12 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
 
 }  // namespace dllm
 
+namespace dllm {
+cudaError_t set_debug_skip_act_load(int enable) {
+  const int v = enable != 0;
+  return cudaMemcpyToSymbol(g_debug_skip_act_load, &v, sizeof v);
+}
+}  // namespace dllm
+
 DLLM_TIMELINE_HOOKS(gemm_tcgen05)
+DLLM_WAIT_LIMIT_HOOK(gemm_tcgen05)

@@ -5,9 +5,32 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace dllm {
+
+// One-time set-up per DEVICE of a process (cudaFuncSetAttribute and the like are per device): run(fn) calls
+// fn() the first time it is reached with a given device current and again after a failure.  Devices beyond
+// the 64 tracked ones are set up at every call.
+struct DeviceOnce {
+  std::atomic<uint64_t> done{0};
+  template <class F>
+  cudaError_t run(F&& fn) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool tracked = dev >= 0 && dev < 64;
+    if (tracked && ((done.load(std::memory_order_acquire) >> dev) & 1ull)) return cudaSuccess;
+    e = fn();
+    if (e == cudaSuccess && tracked) done.fetch_or(1ull << dev, std::memory_order_release);
+    return e;
+  }
+};
+// Multiprocessors of the current device (148 on a B200; that value too when no device is visible, for the
+// host-only size queries).
+int sm_count();
 
 struct Launch {
   cudaStream_t stream;
@@ -82,10 +105,11 @@ struct Partials {
 // ---------------- api.cu ----------------
 // Message that dllm_last_error() returns on this thread.
 void set_last_error(const char* msg);
+// Device address, on the current device, of the status word the kernel-level entry points hand to their
+// kernels (read and cleared by dllm_kernel_status); nullptr if it cannot be resolved.
+int* kernel_status_word();
 
 // ---------------- elementwise.cu ----------------
-// x[c] = E[token(c)] for carried rows c0 <= c < c1.
-void launch_embed(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, Geo g, int c0, int c1);
 // out[c] = rmsnorm(x[c]) * gain for carried rows c0 <= c < c1 (out has the model dtype).
 void launch_rmsnorm(const Launch& L, int dtype, const float* x, const float* gain, void* out, int d, float eps,
                     int c0, int c1);
@@ -106,8 +130,8 @@ void launch_kverify(const Launch& L, int dtype, Partials part, void* Kc_layer, f
 // Bottom-k selection per sequence + active-row list.  mode 0: all R rows,
 // 1: bottom-k by (round(sim*2^20), index), 2: forced list.
 // inv (may be null): for every carried row its position in the active list, or -1.
-void launch_select(const Launch& L, const float* sim, const int32_t* forced, int mode, int ksel, int32_t* sel,
-                   int sel_stride, int32_t* act, int32_t* inv, Geo g, int refresh_prompt);
+cudaError_t launch_select(const Launch& L, const float* sim, const int32_t* forced, int mode, int ksel, int32_t* sel,
+                          int sel_stride, int32_t* act, int32_t* inv, Geo g, int refresh_prompt);
 // Selection, active list, inverse list and the gather of the active rows of u
 // into ua in one launch (R <= 1024; sel rows have stride R).
 void launch_select_gather(const Launch& L, int dtype, const float* sim, const int32_t* forced, int mode, int ksel,
@@ -119,8 +143,8 @@ void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t*
 // End of a layer for carried rows c0 <= c < c1: FFNOut rows of the active set
 // (slabs in `part`, row = inv[c]) -> cache; x <- (x + AttnOut) + FFNOut from the
 // caches; u = rmsnorm(x) * gain.  inv == nullptr: no active row.
-void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, const void* Ac_layer,
-                 void* Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps);
+void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, OutRows Ac_layer,
+                 OutRows Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps);
 void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32_t* act, void* dst, int rows, int d);
 // RoPE on Q and K of the active rows; Q -> qbuf [Ma, dq]; K -> K cache rows.
 void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* act, const float* rope_tab, void* qbuf,
@@ -131,14 +155,11 @@ void launch_scatter_rows(const Launch& L, int dtype, Partials part, const int32_
                          Geo g, int rows, int width);
 // AttnOut rows -> cache; h = x + AttnOut; hn = rmsnorm(h) * gain2 (model dtype).
 void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int32_t* act, const float* x,
-                           const float* gain2, void* Ac_layer, void* hn, Geo g, int Ma, float eps);
+                           const float* gain2, OutRows Ac_layer, void* hn, Geo g, int Ma, float eps);
 // act[i][j] = silu(gate) * up from partials [Ma, 2m] (gate columns first).
 // interleaved: the columns of `part` are blocks of 64 gate columns followed by the 64 up columns of the same
 // FFN columns (the layout of the stacked weight when d_ffn % 64 == 0 in bf16); else all gate, then all up.
 void launch_silu_mul(const Launch& L, int dtype, Partials part, void* out, int Ma, int m, int interleaved = 0);
-// x[c] = (x[c] + AttnOut[c]) + FFNOut[c] for carried rows c0 <= c < c1.
-void launch_residual(const Launch& L, int dtype, float* x, const void* Ac_layer, const void* Fc_layer, Geo g, int c0,
-                     int c1);
 // (x0, conf) per response row from fp32 logits; the mask id never wins.
 void launch_argmax_conf(const Launch& L, const float* logits, int rows, int vocab, int mask_id, int32_t* x0,
                         float* conf, int R = 0, int blk_start = 0, int blk_len = 0);
@@ -185,51 +206,12 @@ Partials make_partials(const float* p, int M, int N, const GemmPlan& plan);
 cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, float* part, int M, int N, int K,
                              const GemmPlan& plan, const char** err, void* act_out = nullptr, int m_ffn = 0);
 
-// ---------------- megakernel.cu ----------------
-// One projection inside the persistent layer kernel: units (tile, k-block) in
-// tile-major order, tile = nt * m_tiles + mt, CTA i owns units [i*upc, (i+1)*upc).
-struct MkGemm {
-  int M, N, K, BN, m_tiles, num_kb, total, upc;
-};
-enum { MK_V = 0, MK_QK = 1, MK_O = 2, MK_GU = 3, MK_D = 4 };
-struct alignas(64) MkParams {
-  CUtensorMap amap[5];           // activation operands of V, QK, O, GU, D (rows = the operand's row count)
-  int B, P, R, n, d, H, Hkv, hd, dq, dkv, m, T;
-  float eps;
-  int rr, ksel, a_seq, Ma, BR;
-  int attn_S, attn_kps;          // key-range splits of the attention phase, keys per split
-  int gu_interleaved;            // gate / up rows of the stacked weight alternate in blocks of 64
-  int has_comb;                  // attention partials are merged in a phase of their own
-  unsigned long long forced_mask;  // bit l: layer l takes its selection from the forced list
-  const uint8_t* W;              // weight blob
-  size_t o_embed, o_norm1, o_wqkv, o_wo, o_norm2, o_wgu, o_wd, o_norm_f, layer_stride;
-  uint8_t* cache;                // cache blob: per layer K, V, AttnOut, FFNOut
-  size_t cache_layer_bytes, c_v, c_a, c_f;
-  const int32_t* tokens;
-  float* x;
-  void *u, *ua, *qbuf, *obuf, *hn, *ffn;
-  float* sim;                    // [T][BR]
-  int32_t* sel;                  // [T][BR]
-  const int32_t* forced;         // [T][BR]
-  int32_t* act;                  // [Ma]
-  int32_t* inv;                  // [BR]: position in the active list or -1
-  const float* rope;
-  float* attn_scratch;
-  float* part;
-  int* status;
-  unsigned int* bar;             // grid barrier counters, one per phase (1 + 13 T), zero at launch
-  const CUtensorMap* maps_fixed; // device: [T][5] weights (V, QK, O, GU, D), then [T][2] K and V caches
-  MkGemm g[5];
-};
-// True if the persistent layer kernel covers this step shape (bf16, no prompt
-// refresh, at least one active row, bounded sizes).
-bool mk_supported(int dtype, int B, int P, int R, int d, int H, int Hkv, int hd, int m, int T, int rp, int ksel);
-// Fills p.g[], attn_S, attn_kps, has_comb from the shapes already in p.
-void mk_plan(MkParams& p);
-size_t mk_part_floats(const MkParams& p);
-// Activation tile rows the kernel uses for an M-row operand.
-int mk_act_tile(int M);
-cudaError_t launch_layer_megakernel(const Launch& L, const MkParams& p);
+// Test hooks of the bounded device-side waits (see dllm_debug_* in the C ABI): the wait limit of each
+// translation unit that waits on mbarriers (0 = the 2 s default), and the dropped activation load.
+cudaError_t set_wait_limit_gemm_tcgen05(unsigned long long ns);
+cudaError_t set_wait_limit_attention(unsigned long long ns);
+cudaError_t set_wait_limit_attention_umma(unsigned long long ns);
+cudaError_t set_debug_skip_act_load(int enable);
 
 // ---------------- attention.cu ----------------
 struct AttnPlan {
@@ -238,6 +220,16 @@ struct AttnPlan {
   size_t scratch_floats;
 };
 AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv);
+// Plan of the 128-row tcgen05 kernel (attention_umma.cu) with at most scratch_floats floats for split partials.
+AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats);
+// Which of the two tensor-core kernels a bf16 shape runs on (more than 64 (query, head-of-group) rows per KV
+// head: tcgen05), with the plan it takes given that much scratch.  launch_attention, the scratch-size query
+// and the entry point with built-in scratch all decide through this one function.
+struct AttnChoice {
+  bool umma = false;
+  AttnPlan plan{1, 0, 0};
+};
+AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats);
 // bf16 with head_dim 64 / 128 runs on the tensor cores (scratch holds the
 // partials of split key ranges; without it one split is used); everything else
 // on the plain-ALU kernel.

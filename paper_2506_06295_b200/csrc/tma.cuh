@@ -6,7 +6,18 @@
 
 namespace dllm {
 
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;  // every device-side wait gives up after 2 s
+// Every device-side wait gives up after this many nanoseconds of %globaltimer (2 s unless a test shortens it).
+// One copy per translation unit; DLLM_WAIT_LIMIT_HOOK(stem) defines the host function that sets it on the
+// current device.
+constexpr unsigned long long WAIT_LIMIT_DEFAULT_NS = 2000000000ull;
+static __device__ unsigned long long g_wait_limit_ns = WAIT_LIMIT_DEFAULT_NS;
+#define DLLM_WAIT_LIMIT_HOOK(stem)                                                                      \
+  namespace dllm {                                                                                      \
+  cudaError_t set_wait_limit_##stem(unsigned long long ns) {                                            \
+    const unsigned long long v = ns ? ns : WAIT_LIMIT_DEFAULT_NS;                                       \
+    return cudaMemcpyToSymbol(g_wait_limit_ns, &v, sizeof v);                                           \
+  }                                                                                                     \
+  }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ uint64_t gtime() {
@@ -44,7 +55,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   while (!mbar_try_wait(bar, parity)) {
     if ((++it & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (gtime() - t0 > WAIT_LIMIT_NS) {
+      if (gtime() - t0 > g_wait_limit_ns) {
         *abort_flag = 1;
         return false;
       }

@@ -26,6 +26,7 @@ STATUS_NAMES = ["OK", "INVALID_ARG", "BAD_STATE", "UNSUPPORTED", "OUT_OF_MEMORY"
 FP32, BF16 = 0, 1
 K_FLOOR, K_CEIL = 0, 1
 CACHE_K, CACHE_V, CACHE_ATTN, CACHE_FFN = range(4)
+SESSION_DEFAULT, SESSION_COMPACT_CACHE = 0, 1
 
 
 class Config(C.Structure):
@@ -42,6 +43,9 @@ SIGNATURES = {
     "dllm_weights_bytes": (_SZ, [C.POINTER(Config)]),
     "dllm_cache_bytes": (_SZ, [C.POINTER(Config), _I, _I, _I]),
     "dllm_workspace_bytes": (_SZ, [C.POINTER(Config), _I, _I, _I]),
+    "dllm_cache_bytes_ex": (_SZ, [C.POINTER(Config), _I, _I, _I, _I]),
+    "dllm_workspace_bytes_ex": (_SZ, [C.POINTER(Config), _I, _I, _I, _I]),
+    "dllm_session_create_ex": (_I, [_P, _I, _I, _I, _I, _P, _P, _P, C.POINTER(_P)]),
     "dllm_tensor_offset": (_I, [C.POINTER(Config), C.c_char_p, C.POINTER(_SZ), C.POINTER(_SZ)]),
     "dllm_step_scheduled_block": (_I, [_P, _I, _I, _I, _I, _F, _I, _I, _I, _P]),
     "dllm_session_predict_block_only": (_I, [_P, _I]),
@@ -74,7 +78,6 @@ SIGNATURES = {
     "dllm_session_use_graphs": (_I, [_P, _I]),
     "dllm_session_use_simt_gemm": (_I, [_P, _I]),
     "dllm_session_use_pdl": (_I, [_P, _I]),
-    "dllm_session_use_layer_kernel": (_I, [_P, _I]),
     "dllm_session_profile": (_I, [_P, _I]),
     "dllm_session_profile_read": (_I, [_P, _I, C.POINTER(C.c_double), C.POINTER(C.c_uint64),
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]),
@@ -90,6 +93,9 @@ SIGNATURES = {
     "dllm_attention": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _SZ, _P]),
     "dllm_vverify_select": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _P]),
     "dllm_attention_noalloc": (_I, [_P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _P]),
+    "dllm_kernel_status": (_I, [_P]),
+    "dllm_debug_set_wait_limit_ns": (_I, [C.c_uint64]),
+    "dllm_debug_skip_one_load": (_I, [_I]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
     _fn = getattr(lib, _name)
@@ -122,12 +128,12 @@ def weights_bytes(cfg) -> int:
     return lib.dllm_weights_bytes(C.byref(make_config(cfg)))
 
 
-def cache_bytes(cfg, B, P, R) -> int:
-    return lib.dllm_cache_bytes(C.byref(make_config(cfg)), B, P, R)
+def cache_bytes(cfg, B, P, R, flags: int = 0) -> int:
+    return lib.dllm_cache_bytes_ex(C.byref(make_config(cfg)), B, P, R, flags)
 
 
-def workspace_bytes(cfg, B, P, R) -> int:
-    return lib.dllm_workspace_bytes(C.byref(make_config(cfg)), B, P, R)
+def workspace_bytes(cfg, B, P, R, flags: int = 0) -> int:
+    return lib.dllm_workspace_bytes_ex(C.byref(make_config(cfg)), B, P, R, flags)
 
 
 def tensor_offset(cfg, name: str) -> tuple[int, int]:
@@ -228,21 +234,25 @@ class Model:
 class Session:
     """Tokens (c, y^(k)) plus the per-layer caches C_p, C_r for B sequences."""
 
-    def __init__(self, model: Model, B: int, P: int, R: int, stream=None):
+    def __init__(self, model: Model, B: int, P: int, R: int, stream=None, compact_cache: bool = False):
+        """compact_cache: AttnOut / FFNOut caches for the response rows only (same results, smaller cache)."""
         import torch
         self.model, self.B, self.P, self.R, self.n = model, B, P, R, P + R
         self.cfg = model.cfg
-        self.stream = stream if stream is not None else torch.cuda.Stream(device=model.device)
+        self.compact = bool(compact_cache)
+        flags = SESSION_COMPACT_CACHE if self.compact else SESSION_DEFAULT
+        with torch.cuda.device(model.device):
+            self.stream = stream if stream is not None else torch.cuda.Stream(device=model.device)
+            cb, wb = cache_bytes(self.cfg, B, P, R, flags), workspace_bytes(self.cfg, B, P, R, flags)
         self.sp = C.c_void_p(_stream_ptr(self.stream))
-        cb, wb = cache_bytes(self.cfg, B, P, R), workspace_bytes(self.cfg, B, P, R)
         if cb == 0 or wb == 0:
             raise DllmError(INVALID_ARG, "B, P and R must be positive")
         self.cache = torch.empty(cb, dtype=torch.uint8, device=model.device)
         self.workspace = torch.empty(wb, dtype=torch.uint8, device=model.device)
         torch.cuda.synchronize(model.device)
         h = _P()
-        _check(lib.dllm_session_create(model.handle, B, P, R, C.c_void_p(self.cache.data_ptr()),
-                                       C.c_void_p(self.workspace.data_ptr()), self.sp, C.byref(h)))
+        _check(lib.dllm_session_create_ex(model.handle, B, P, R, flags, C.c_void_p(self.cache.data_ptr()),
+                                          C.c_void_p(self.workspace.data_ptr()), self.sp, C.byref(h)))
         self.handle = h
 
     # -- the calls of the method ------------------------------------------
@@ -320,7 +330,8 @@ class Session:
 
     def get_cache(self, layer: int, which: int) -> np.ndarray:
         width = self.cfg.dkv if which in (CACHE_K, CACHE_V) else self.cfg.d_model
-        out = np.empty((self.B, self.n, width), np.float32)
+        rows = self.R if (self.compact and which in (CACHE_ATTN, CACHE_FFN)) else self.n
+        out = np.empty((self.B, rows, width), np.float32)
         _check(lib.dllm_get_cache(self.handle, layer, which, _np_ptr(out), self.sp))
         return out
 
@@ -353,9 +364,6 @@ class Session:
 
     def use_pdl(self, enable: bool) -> None:
         _check(lib.dllm_session_use_pdl(self.handle, int(enable)))
-
-    def use_layer_kernel(self, enable: bool) -> None:
-        _check(lib.dllm_session_use_layer_kernel(self.handle, int(enable)))
 
     def use_simt_gemm(self, enable: bool) -> None:
         _check(lib.dllm_session_use_simt_gemm(self.handle, int(enable)))
@@ -493,3 +501,20 @@ def vverify_select(vnew, vcache, k, stream=None):
                                    C.c_void_p(sim.data_ptr()), C.c_void_p(idx.data_ptr()), B, R, width, k, dt,
                                    C.c_void_p(sp)))
     return sim, idx[:, :k]
+
+
+def kernel_status(stream=None) -> None:
+    """Raises DllmError(TIMEOUT) if a bounded wait of a kernel-level call gave up since the last read."""
+    import torch
+    sp = _stream_ptr(stream if stream is not None else torch.cuda.current_stream())
+    _check(lib.dllm_kernel_status(C.c_void_p(sp)))
+
+
+def debug_set_wait_limit_ns(ns: int) -> None:
+    """Test hook: limit of the device-side waits (0 restores the 2 s default)."""
+    _check(lib.dllm_debug_set_wait_limit_ns(int(ns)))
+
+
+def debug_skip_one_load(enable: bool) -> None:
+    """Test hook: the first CTA of every one-CTA bf16 GEMM launch leaves out one tile copy (its waits run out)."""
+    _check(lib.dllm_debug_skip_one_load(int(enable)))

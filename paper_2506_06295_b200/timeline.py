@@ -23,7 +23,7 @@ import json
 import os
 import sys
 
-STEMS = ["elementwise", "gemm_simt", "gemm_tcgen05", "attention", "attention_umma", "megakernel"]
+STEMS = ["elementwise", "gemm_simt", "gemm_tcgen05", "attention", "attention_umma"]
 KINDS = {"full": (True, True), "refresh": (False, True), "mixed": (True, False), "partial": (False, False)}
 RECORD_CAP = 1 << 20
 

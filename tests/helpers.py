@@ -8,6 +8,16 @@ def rel_l2(a, b):
     return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
 
 
+def row_rel_max(a, b):
+    """Largest per-row relative L2 error over the last axis: one bad row among hundreds moves the global
+    figure by little, this one by its full error."""
+    a = np.asarray(a, np.float64).reshape(-1, np.shape(a)[-1])
+    b = np.asarray(b, np.float64).reshape(-1, np.shape(b)[-1])
+    num = np.linalg.norm(a - b, axis=-1)
+    den = np.maximum(np.linalg.norm(b, axis=-1), 1e-300)
+    return float((num / den).max())
+
+
 def bf16_round_torch(t):
     import torch
     return t.to(torch.bfloat16).to(torch.float32)

@@ -9,13 +9,19 @@ Two legs:
   * the full 32-layer model with weights drawn on the device: properties that
     hold at any size, plus layer-0 quantities the oracle can compute row by row
     from downloaded weights (layer 0 sees only embeddings).
+
+The other benchmark configurations get the first kind of leg each, at their own
+widths and row counts, so that every kernel path their steps take (grouped KV
+heads on the tcgen05 attention with split key ranges, three selected rows
+against 4128 keys, selection and gather as two launches, the launch-order remap
+of many-tile projections) runs inside a step that is compared with the oracle.
 """
 import numpy as np
 import pytest
 
 from oracle import dllm_oracle as O
 from paper_2506_06295_b200 import synth
-from tests.helpers import rel_l2, selection_matches
+from tests.helpers import rel_l2, row_rel_max, selection_matches
 
 pytestmark = pytest.mark.gpu
 
@@ -190,3 +196,108 @@ def test_llada_full_depth_properties_and_layer0_samples(env):
     cand = [j for j in range(32, 64) if tok_before[j] == cfg.mask_id]
     want = sorted(sorted(cand, key=lambda j: (-float(conf[0, j]), j))[:3])
     assert diff.tolist() == want and np.array_equal(tok_after[diff], x0[0, diff])
+
+
+# ---------------------------------------------------------------- the other configurations, two layers each
+def _weights(cfg):
+    from concurrent.futures import ThreadPoolExecutor
+    names = synth.tensor_names(cfg)
+    with ThreadPoolExecutor(max_workers=8) as ex:
+        return dict(zip([n for n, _ in names], ex.map(lambda ns: synth.make_tensor(cfg, ns[0], ns[1]), names)))
+
+
+def _check_step(dllm, orc, ses, r, what, kround="floor", adaptive=False, tol=2e-2, row_tol=6e-2):
+    """Hidden states (global relative L2 within the stated bf16 bound, and no single row far outside it), the
+    four caches of every layer, and for an adaptive step the similarities and the selected index sets."""
+    cfg, B = orc.cfg, orc.B
+    h = ses.hidden()
+    assert rel_l2(h, r.hidden) < tol, what
+    assert row_rel_max(h, r.hidden) < row_tol, what
+    for which, ref in ((dllm.CACHE_K, orc.Kc), (dllm.CACHE_V, orc.Vc), (dllm.CACHE_ATTN, orc.Ac),
+                       (dllm.CACHE_FFN, orc.Fc)):
+        for l in range(cfg.n_layers):
+            got = ses.get_cache(l, which)
+            assert rel_l2(got, ref[l]) < tol, f"{what}: cache {which} layer {l}"
+            assert row_rel_max(got[:, orc.P:], ref[l][:, orc.P:]) < row_tol, f"{what}: cache {which} layer {l} (row)"
+    if adaptive:
+        for l in range(cfg.n_layers):
+            idx, sim = ses.selected(l)
+            assert idx.shape == r.selected[l].shape, f"{what}: layer {l}"
+            np.testing.assert_allclose(sim, r.sim[l], atol=5e-3, err_msg=f"{what}: layer {l}")
+            for b in range(B):
+                assert selection_matches(idx[b], r.selected[l][b], r.sim[l][b]), f"{what}: layer {l} sequence {b}"
+
+
+def _unmask(orc, ses, step, per_seq):
+    """The same few response tokens revealed on both sides (what the transition would do between steps)."""
+    P, R, V = orc.P, orc.R, orc.cfg.vocab
+    resp = orc.tokens[:, P:].copy()
+    for b in range(orc.B):
+        for i in range(per_seq):
+            j = (37 * step + 101 * i + 13 * b) % R
+            resp[b, j] = (977 * j + 31 * step + b) % (V - 1)
+    orc.tokens[:, P:] = resp
+    ses.set_response_tokens(resp)
+
+
+def _run_config(dllm, cfg, B, P, R, plan):
+    """plan: (refresh_prompt, refresh_response, rho, kround) per cached step after the initial full step."""
+    w = _weights(cfg)
+    prompt = synth.make_prompt(cfg, B, P)
+    orc = O.DLLMOracle(cfg, w, B, P, R, dtype=np.float32)
+    orc.set_prompt(prompt)
+    ses = dllm.Session(dllm.Model(cfg).load(w), B, P, R)
+    ses.set_prompt(prompt)
+    r = orc.step(True, True)
+    ses.step_full()
+    ses.sync()
+    _check_step(dllm, orc, ses, r, "full")
+    for step, (rp, rr, rho, kround) in enumerate(plan, 1):
+        _unmask(orc, ses, step, 3)
+        r = orc.step(rp, rr, rho, kround)
+        ses.step_cached(rp, rr, rho, dllm.K_CEIL if kround == "ceil" else dllm.K_FLOOR)
+        ses.sync()
+        _check_step(dllm, orc, ses, r, f"step {step} ({rp}, {rr}, {rho}, {kround})", adaptive=not rr and rho > 0)
+    return orc, ses
+
+
+def test_dream_width_two_layers_against_the_oracle(env):
+    """Dream-7B widths: d = 3584, 28 query heads on 4 KV heads, FFN 18944, vocab 152064; P = R = 256, rho = 0.5.
+    128 selected rows x 7 heads of a group = 896 rows per KV head: the tcgen05 attention with split key ranges."""
+    torch, dllm = env
+    wl = synth.WORKLOADS["dream7b"]
+    cfg = wl.model.with_layers(2)
+    orc, ses = _run_config(dllm, cfg, 1, wl.prompt_len, wl.gen_len,
+                           [(False, False, wl.rho, "floor"), (False, False, wl.rho, "floor"),
+                            (False, True, 0.0, "floor"), (True, False, wl.rho, "floor")])
+    idx, _ = ses.selected(0)
+    assert idx.shape == (1, 128)
+
+
+def test_long_prompt_two_layers_against_the_oracle(env):
+    """Long-prompt regime on LLaDA widths: P = 4096, R = 32, rho = 0.1: three selected rows (four with the
+    ceiling) against 4128 keys, the key range split over many CTAs; a full step over 4128 rows."""
+    torch, dllm = env
+    wl = synth.WORKLOADS["long"]
+    cfg = wl.model.with_layers(2)
+    orc, ses = _run_config(dllm, cfg, 1, wl.prompt_len, wl.gen_len,
+                           [(False, False, wl.rho, "floor"), (False, False, wl.rho, "ceil"),
+                            (False, True, 0.0, "floor"), (False, False, wl.rho, "floor"),
+                            (True, False, wl.rho, "floor")])
+    assert O.k_selected(wl.rho, wl.gen_len, "floor") == 3 and O.k_selected(wl.rho, wl.gen_len, "ceil") == 4
+    assert ses.selected(1)[0].shape == (1, 3)
+
+
+def test_batched_two_layers_against_the_oracle(env):
+    """Batched serving on LLaDA widths (P = 1024, R = 512 per sequence) with B = 3 so that the float32 oracle
+    finishes in a minute or two: the update ratios of the sweep, selection and gather as two launches (more than
+    128 active rows), 18 activation tiles in the full step's projections (launch-order remap), 1536 rows in
+    V-verify and the layer tail, the tcgen05 attention with and without split key ranges."""
+    torch, dllm = env
+    wl = synth.WORKLOADS["batch16"]
+    cfg = wl.model.with_layers(2)
+    B = 3
+    orc, ses = _run_config(dllm, cfg, B, wl.prompt_len, wl.gen_len,
+                           [(False, False, 0.1, "floor"), (False, False, 0.25, "floor"), (False, True, 0.0, "floor"),
+                            (False, False, 0.5, "floor")])
+    assert ses.selected(0)[0].shape == (B, 256)

@@ -184,7 +184,10 @@ def test_attention(env, case, dtype):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-@pytest.mark.parametrize("B,R,width,k", [(1, 32, 256, 8), (3, 256, 4096, 64), (2, 100, 512, 50), (1, 512, 4096, 51)])
+@pytest.mark.parametrize("B,R,width,k", [(1, 32, 256, 8), (3, 256, 4096, 64), (2, 100, 512, 50), (1, 512, 4096, 51),
+                                         # the longest response the selection kernel admits (keys and flags of one
+                                         # sequence in more than 48 KB of shared memory) and one just past that mark
+                                         (1, 8192, 64, 819), (2, 6000, 64, 1500)])
 def test_vverify_select(env, dtype, B, R, width, k):
     torch, dllm = env
     cache = synth.random_normal((B, R, width), seed=5)

@@ -241,17 +241,15 @@ def test_tiny_fp32_stepwise_generation_with_graphs_off_and_on(env):
 
 # ---------------------------------------------------------------- bf16, several tiles and ragged tails
 @pytest.mark.parametrize("gqa", [False, True], ids=["mha", "gqa"])
-@pytest.mark.parametrize("path", ["simt_gemm", "tcgen05_gemm", "layer_kernel"])
+@pytest.mark.parametrize("path", ["simt_gemm", "tcgen05_gemm"])
 def test_small_bf16_step_kinds(env, gqa, path):
-    """Every step kind against the oracle, on the plain-ALU kernels, on the
-    tensor-core kernels launched one by one, and with the persistent layer
-    kernel (which takes the steps without prompt refresh)."""
+    """Every step kind against the oracle, on the plain-ALU kernels and on the
+    tensor-core kernels."""
     torch, dllm = env
     cfg = synth.small_bf16_model(gqa=gqa)
     B, P, R = 2, 150, 72
     orc, ses, _ = make_pair(dllm, cfg, B, P, R)
     ses.use_simt_gemm(path == "simt_gemm")
-    ses.use_layer_kernel(path == "layer_kernel")
     r = orc.step(True, True)
     ses.step_full()
     compare_step(orc, ses, r, 2e-2, what="full")
@@ -274,8 +272,7 @@ def test_small_bf16_step_kinds(env, gqa, path):
         assert err < 2e-2
 
 
-@pytest.mark.parametrize("path", ["tcgen05_gemm", "layer_kernel"])
-def test_bf16_gate_up_layouts(env, path):
+def test_bf16_gate_up_layouts(env):
     """W_gate / W_up stored one after the other (d_ffn not a multiple of 64) and row-blocked (a multiple of 64,
     where an unsplit gate / up GEMM applies SwiGLU itself and a split one leaves it to the next kernel) give the
     oracle's step; the blocked model also accepts weights written straight into the blob."""
@@ -286,7 +283,6 @@ def test_bf16_gate_up_layouts(env, path):
         assert (dllm.tensor_blocks(cfg, "layers.0.wg")[0] == 64) == (d_ffn % 64 == 0)
         B, P, R = 2, 150, 72
         orc, ses, w = make_pair(dllm, cfg, B, P, R)
-        ses.use_layer_kernel(path == "layer_kernel")
         if d_ffn % 64 == 0:   # rewrite the gate / up weights through the strided view: same model
             for l in range(cfg.n_layers):
                 for t in ("wg", "wu"):

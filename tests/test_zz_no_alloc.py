@@ -32,9 +32,10 @@ def _inputs(torch, B, a, n, H, Hkv, hd, seed):
 
 def test_noalloc_matches_the_allocating_entry_point_on_two_calls_in_a_row(env):
     torch, dllm = env
-    # both shapes split the key range (few active rows), so both use the built-in scratch;
-    # the second is smaller, so stale partials of the first call lie right behind its own
-    for i, shape in enumerate([(1, 64, 768, 8, 8, 128), (2, 19, 333, 4, 2, 64)]):
+    # every shape splits the key range (few row tiles), so every call uses the built-in scratch: the first two
+    # on the 64-row kernel, the third on the 128-row tcgen05 kernel (128 rows per KV head); each is smaller than
+    # or differently laid out from the one before, so stale partials of the previous call lie in and behind its own
+    for i, shape in enumerate([(1, 64, 768, 8, 8, 128), (2, 19, 333, 4, 2, 64), (1, 128, 1024, 8, 8, 128)]):
         B, a, n, H, Hkv, hd = shape
         assert dllm.lib.dllm_attention_scratch_bytes(B, a, n, H, Hkv, hd, dllm.BF16) > 0
         q, k, v = _inputs(torch, *shape, seed=100 + 10 * i)
@@ -52,7 +53,8 @@ def test_noalloc_matches_the_allocating_entry_point_on_two_calls_in_a_row(env):
 
 def test_noalloc_rejects_what_does_not_fit_its_scratch(env):
     torch, dllm = env
-    B, a, n, H, Hkv, hd = 1, 448, 256, 21, 21, 128               # 147 row tiles -> 2 key splits -> 9.8 MB of partials
+    # 64 rows per KV head (the 64-row kernel): 147 row tiles -> 2 key splits -> 9.8 MB of partials
+    B, a, n, H, Hkv, hd = 1, 64, 256, 147, 147, 128
     assert dllm.lib.dllm_attention_scratch_bytes(B, a, n, H, Hkv, hd, dllm.BF16) > 8 * 1024 * 1024
     q, k, v = _inputs(torch, B, a, n, H, Hkv, hd, seed=7)
     out = torch.zeros_like(q)
