@@ -256,6 +256,16 @@ dllm_status dllm_session_use_graphs(dllm_session* s, int enable);
  * projections) overlaps the tail of the kernel before it; 0: plain launches. */
 dllm_status dllm_session_use_pdl(dllm_session* s, int enable);
 
+/* L2 prefetch of the coming projections' weights by the row-wise kernels of a
+ * weight-bound step (at most 512 active rows): between two projections HBM is
+ * nearly idle, so the kernels there may ask for the head of the next weight
+ * matrix.  h_kb: up to five sizes in KB (missing ones are 0 = off): V-verify ->
+ * W_q/W_k; selection + gather -> W_q/W_k continued; RoPE -> W_o, running on
+ * into W_gate/W_up; O-projection epilogue -> W_gate/W_up continued; layer tail
+ * -> the next layer's W_v.  Results are unaffected; a tuning hook (default: all
+ * off until set). */
+dllm_status dllm_session_set_prefetch(dllm_session* s, const int* h_kb, int n);
+
 /* Per-kernel timing.  While enabled, every projection GEMM (class 0) and
  * attention launch (class 1) is bracketed by CUDA events on the caller's stream
  * and no launch overlaps its predecessor (no programmatic dependent launch).
@@ -292,6 +302,11 @@ dllm_status dllm_kernel_status(void* stream);
  * records the status code, skips its epilogue, frees its tensor memory and
  * returns normally; (0) switches that off.  Both calls synchronise the device. */
 dllm_status dllm_debug_set_wait_limit_ns(uint64_t ns);
+/* Tuning hook: overrides the launch plan of the 64-row attention kernel for
+ * every later call in this process: `splits` key-range splits over CTAs and up
+ * to `groups` (1..3) groups of 128 threads per CTA; 0 = automatic.  Results
+ * stay within the attention tolerance; merge orders change with the plan. */
+dllm_status dllm_debug_attention_plan(int splits, int groups);
 dllm_status dllm_debug_skip_one_load(int enable);
 /* C[M,N] (fp32, row-major, DEVICE) = A[M,K] * W[N,K]^T with bf16 operands on
  * the tensor cores (tcgen05 + TMA).  d_partials is scratch of

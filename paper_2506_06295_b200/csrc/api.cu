@@ -255,6 +255,10 @@ struct dllm_session {
   bool use_pdl = true;
   int sel_strategy = DLLM_SELECT_V_VERIFY, sel_metric = DLLM_METRIC_COSINE, v_selected_only = 0;  // ablation variants
   bool block_head = false;     // dllm_generate predicts only the block each step works on
+  // L2 prefetch of the coming projection's weights from the row-wise kernels (KB per slot, 0 = off):
+  // [0] V-verify -> W_q/W_k, [1] selection + gather -> W_q/W_k continued, [2] RoPE -> W_o (running on into
+  // W_gate/W_up), [3] O epilogue -> W_gate/W_up continued, [4] layer tail -> the next layer's W_v
+  size_t pf_kb[5] = {0, 0, 0, 0, 0};
   struct GraphEntry {
     cudaGraphExec_t exec;
     uint64_t kernels;
@@ -456,6 +460,26 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
     const int ksel = ksels[l];  // rows of the response this layer recomputes
     const int a_seq = (rp ? s->P : 0) + ksel;
     const int Ma = s->B * a_seq;
+    // prefetch spans (weight-bound steps only: with many active rows the projections are not waiting for HBM)
+    Prefetch pf_qk0, pf_qk1, pf_o, pf_gu, pf_v;
+    if (dt == DLLM_BF16 && Ma > 0 && Ma <= 512) {
+      auto span = [](const uint8_t* p, size_t lo, size_t want, size_t cap) {
+        Prefetch f;
+        if (lo < cap && want > 0) {
+          f.p = p + lo;
+          f.bytes = std::min(want, cap - lo);
+        }
+        return f;
+      };
+      const size_t KB = 1024, qk_bytes = (size_t)(dq + dkv) * d * es, gu_end = lo.wgu + (size_t)2 * m * d * es;
+      pf_qk0 = span(Wq, 0, s->pf_kb[0] * KB, qk_bytes);
+      pf_qk1 = span(Wq, s->pf_kb[0] * KB, s->pf_kb[1] * KB, qk_bytes);
+      pf_o = span(W + lo.wo, 0, s->pf_kb[2] * KB, gu_end - lo.wo);
+      const size_t into_gu = lo.wo + s->pf_kb[2] * KB > lo.wgu ? lo.wo + s->pf_kb[2] * KB - lo.wgu : 0;
+      pf_gu = span(W + lo.wgu, into_gu, s->pf_kb[3] * KB, (size_t)2 * m * d * es);
+      if (l + 1 < c.n_layers)
+        pf_v = span(W + wl.layers[l + 1].wqkv + (size_t)(dq + dkv) * d * es, 0, s->pf_kb[4] * KB, (size_t)dkv * d * es);
+    }
     const bool adaptive = !rr && ksel > 0;
     const int mode = rr ? 0 : (s->forced_count[l] >= 0 ? 2 : 1);
     // A response refresh alone takes every response row in carried order: u itself is the operand of the
@@ -466,7 +490,7 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
       if ((st = run_gemm(s, L, u, Wv, BR, dkv, d, &part)) != DLLM_OK) return st;
       const IdentityLists id{sel, act, inv};
       launch_vverify(L, dt, part, s->cache(l, DLLM_CACHE_V), sim, g, dkv, rr ? 0 : s->sel_metric,
-                     rr || !s->v_selected_only, identity ? &id : nullptr);
+                     rr || !s->v_selected_only, identity ? &id : nullptr, pf_qk0);
     } else if (adaptive && s->sel_strategy == DLLM_SELECT_K_VERIFY) {
       // ablation: the same test on K; K of ALL response rows is projected, rotated and overwritten
       if ((st = run_gemm(s, L, u, Wq + (size_t)dq * d * es, BR, dkv, d, &part)) != DLLM_OK) return st;
@@ -485,7 +509,8 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
         ua = u;
       } else if (s->R <= 1024 && (long)Ma * s->R <= 64L * 1024) {
         // few active rows: every CTA of the gather repeats the selection rather than wait for a launch
-        launch_select_gather(L, dt, sim, forced, mode, ksel, sel, act, inv, u, s->wsp<uint8_t>(s->ws.ua), g, rp);
+        launch_select_gather(L, dt, sim, forced, mode, ksel, sel, act, inv, u, s->wsp<uint8_t>(s->ws.ua), g, rp,
+                             pf_qk1);
       } else {
         cudaError_t se = launch_select(L, sim, forced, mode, ksel, sel, s->R, act, inv, g, rp);
         if (se != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "selection: %s", cudaGetErrorString(se));
@@ -498,7 +523,7 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
       // Q and K of the active rows in one GEMM over the stacked [W_q; W_k]
       if ((st = run_gemm(s, L, ua, Wq, Ma, dq + dkv, d, &part)) != DLLM_OK) return st;
       launch_qk_rope(L, dt, part, act, s->wsp<float>(s->ws.rope), s->wsp<uint8_t>(s->ws.qbuf),
-                     s->cache(l, DLLM_CACHE_K), g, Ma, H, Hkv, hd);
+                     s->cache(l, DLLM_CACHE_K), g, Ma, H, Hkv, hd, pf_o);
       // algorithmic traffic: K and V of every sequence once, Q in, O out
       s->prof_begin(1, (2.0 * s->B * s->n * dkv + 2.0 * Ma * dq) * (double)es, 4.0 * Ma * (double)s->n * dq, stream);
       cudaError_t e = launch_attention(L, dt, s->wsp<uint8_t>(s->ws.qbuf), s->cache(l, DLLM_CACHE_K),
@@ -508,7 +533,7 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
       if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.obuf), W + lo.wo, Ma, d, dq, &part)) != DLLM_OK) return st;
       launch_oproj_epilogue(L, dt, part, act, x, reinterpret_cast<const float*>(W + lo.norm2),
-                            s->outs(l, DLLM_CACHE_ATTN), s->wsp<uint8_t>(s->ws.hn), g, Ma, c.rms_eps);
+                            s->outs(l, DLLM_CACHE_ATTN), s->wsp<uint8_t>(s->ws.hn), g, Ma, c.rms_eps, pf_gu);
       bool fused = false;
       if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.hn), W + lo.wgu, Ma, 2 * m, d, &part, s->wsp<uint8_t>(s->ws.ffn),
                          &fused)) != DLLM_OK)
@@ -519,7 +544,7 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
     // FFNOut rows -> cache, residual assembly for all carried rows, next norm
     const float* gain_next = reinterpret_cast<const float*>(l + 1 < c.n_layers ? W + wl.layers[l + 1].norm1 : W + wl.norm_f);
     launch_tail(L, dt, part, Ma > 0 ? inv : nullptr, x, s->outs(l, DLLM_CACHE_ATTN), s->outs(l, DLLM_CACHE_FFN),
-                gain_next, u, g, c0, c1, c.rms_eps);
+                gain_next, u, g, c0, c1, c.rms_eps, pf_v);
   }
   // prediction at the response rows (Eqs. 3-4); u holds the final norm.  With head_len > 0 only the rows of
   // one block are predicted: the transition of a semi-autoregressive step reads no others (Eq. 5).
@@ -1150,6 +1175,16 @@ dllm_status dllm_set_scores(dllm_session* s, int layer, const float* h_scores, v
   cudaStream_t st = (cudaStream_t)stream;
   CU_TRY(&s->err, cudaStreamSynchronize(st));
   CU_TRY(&s->err, h2d(s->d_ws + s->ws.sim + (size_t)layer * BR * 4, h_scores, BR * 4, st));
+  return DLLM_OK;
+}
+
+dllm_status dllm_session_set_prefetch(dllm_session* s, const int* h_kb, int n) {
+  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
+  if (n < 0 || n > 5 || (n > 0 && !h_kb)) return fail(&s->err, DLLM_INVALID_ARG, "at most five prefetch sizes");
+  for (int i = 0; i < n; ++i)
+    if (h_kb[i] < 0) return fail(&s->err, DLLM_INVALID_ARG, "negative prefetch size");
+  for (int i = 0; i < 5; ++i) s->pf_kb[i] = i < n ? (size_t)h_kb[i] : 0;
+  s->drop_graphs();
   return DLLM_OK;
 }
 
