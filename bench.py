@@ -223,6 +223,67 @@ def workload_config(wl, args):
 
 
 # ----------------------------------------------------------------------------------------------
+# one process per GPU
+# ----------------------------------------------------------------------------------------------
+def wants_spawn(gpus: int, impl: str, env) -> bool:
+    """`--gpus N` given to a plain `python bench.py` (no launcher set WORLD_SIZE): this process starts the N ranks."""
+    return gpus > 1 and impl != "reference" and "WORLD_SIZE" not in env
+
+
+def spawn_ranks(n: int, argv, script=None) -> int:
+    """Runs `script` (this file) as n ranks of one node, one per GPU, under torch.distributed.run, rendezvous on
+    127.0.0.1 at a free port; returns the launcher's exit code.  Rank 0 prints the JSON line."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr",
+           "127.0.0.1", "--master-port", str(port), script or os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
+
+
+# ----------------------------------------------------------------------------------------------
+# rooflines
+# ----------------------------------------------------------------------------------------------
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}      # the figures the target is stated against
+TENSOR_CLASSES = {"gemm", "attention", "gemm_v", "gemm_qk", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head",
+                  "attention_mma", "attention_tcgen05"}
+
+
+def roofline_of(name, rec, peaks):
+    """Binding roof of one class of launches from its algorithmic intensity against the ridge of the measured
+    peaks (a projection with M activation rows has about M flop per byte): achieved and both fractions."""
+    ms, by, fl, n = rec["ms"], rec["bytes"], rec["flops"], rec["launches"]
+    if n == 0 or ms <= 0:
+        return None
+    ridge = peaks["bf16_tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    tensor = name in TENSOR_CLASSES and by > 0 and fl / by > ridge
+    gbs, tfl = by / (ms / 1e3) / 1e9, fl / (ms / 1e3) / 1e12
+    out = {"launches": int(n), "avg_us": 1e3 * ms / n, "ms_total": ms, "bytes_per_launch": by / n,
+           "flops_per_launch": fl / n, "gbs": gbs, "tflops": tfl, "bound": "tensor" if tensor else "hbm"}
+    if tensor:
+        out.update(achieved=tfl, unit="TFLOP/s", peak=peaks["bf16_tflops_sustained"],
+                   frac=tfl / peaks["bf16_tflops_sustained"], frac_of_nominal=tfl / NOMINAL["bf16_tflops"])
+    else:
+        out.update(achieved=gbs, unit="GB/s", peak=peaks["hbm_gbs"], frac=gbs / peaks["hbm_gbs"],
+                   frac_of_nominal=gbs / NOMINAL["hbm_gbs"])
+    return out
+
+
+def step_roof_ms(per_class, peaks):
+    """Roofline time of one step: its launches run one after the other, each at its own binding roof."""
+    hbm, tf = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
+    return 1e3 * sum(max(r["bytes"] / hbm, (r["flops"] / tf) if name in TENSOR_CLASSES else 0.0)
+                     for name, r in per_class.items())
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per projection launch, from an ncu capture of a two-layer case of
+# the same kernel scaled to the full depth (every layer streams its own weights); None where no capture of the
+# current kernel exists.
+TRAFFIC_PER_LAUNCH = {"llada8b": 96.2e6}
+
+
+# ----------------------------------------------------------------------------------------------
 # the CUDA arm
 # ----------------------------------------------------------------------------------------------
 def main():
@@ -232,23 +293,33 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llada8b", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--rho", type=float, default=None, help="update ratio of the adaptive steps (default: the workload's)")
+    ap.add_argument("--rho-sweep", default=None, help="comma list of update ratios timed beside the headline "
+                    "(default: 0.1,0.25,0.5 for the batched workload, none otherwise; 'none' to skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-timeline", action="store_true", help="skip the in-graph GEMM figure (a second process)")
+    ap.add_argument("--prof-mode", default="graph", choices=["graph", "stream"], help="per-kernel event pairs as "
+                    "event-record nodes of the step graphs, or recorded by the host around plain launches")
     ap.add_argument("--full-steps", type=int, default=6, help="timed full-recompute steps for the speedup figure")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (small case for ncu "
                     "captures: same widths, a few GB of weights); the bench line then names the reduced depth")
     ap.add_argument("--no-pdl", action="store_true", help="plain launches instead of programmatic dependent launch")
+    ap.add_argument("--compact-cache", action="store_true", help="response-only AttnOut / FFNOut caches")
     ap.add_argument("--ncu-kinds", default="", help="comma list of step kinds (full,refresh,mixed,partial): after "
                     "warm-up run one step of each between cudaProfilerStart/Stop and exit (for "
                     "`ncu --profile-from-start off`); prints no bench line")
     args = ap.parse_args()
+    from dataclasses import replace
     wl = synth.WORKLOADS[args.workload]
     if args.layers > 0:
-        from dataclasses import replace
         wl = replace(wl, name=f"{wl.name}-{args.layers}layers", model=wl.model.with_layers(args.layers))
+    if args.rho is not None:
+        wl = replace(wl, rho=args.rho)
     if args.impl == "reference":
         run_reference(args, wl)
         return
+    if wants_spawn(args.gpus, args.impl, os.environ):
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
 
     import torch
     import torch.distributed as dist
@@ -270,7 +341,7 @@ def main():
     K, W = args.steps, max(args.warmup, 3)
 
     model = dllm.Model(cfg, device=dev).random_init_on_device(synth.WEIGHT_SEED + rank)
-    ses = dllm.Session(model, wl.batch, wl.prompt_len, wl.gen_len)
+    ses = dllm.Session(model, wl.batch, wl.prompt_len, wl.gen_len, compact_cache=args.compact_cache)
     prompt = synth.make_prompt(cfg, wl.batch, wl.prompt_len, seed=1 + 1000 * rank)
     ses.set_prompt(prompt)
     if args.no_pdl:
@@ -336,17 +407,45 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
 
     # ---- per-kind step times and the full-recompute baseline of the same library -------------
-    def time_kind(rp, rr, reps):
+    KINDS = {"full": (True, True), "refresh": (False, True), "mixed": (True, False), "partial": (False, False)}
+
+    def time_kind(rp, rr, reps, rho=None):
+        rho = wl.rho if rho is None else rho
+        ses.step_cached(rp, rr, rho)      # the graph of this (kind, rho) exists before the clock starts
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize(dev)
         a.record(stream)
         for _ in range(reps):
-            ses.step_cached(rp, rr, wl.rho)
+            ses.step_cached(rp, rr, rho)
         b.record(stream)
         torch.cuda.synchronize(dev)
         return a.elapsed_time(b) / reps
-    per_kind = {"full": time_kind(True, True, args.full_steps), "refresh": time_kind(False, True, 6),
-                "mixed": time_kind(True, False, 6), "partial": time_kind(False, False, 12)}
+    reps = {"full": args.full_steps, "refresh": 6, "mixed": 6, "partial": 12}
+    per_kind = {kind: time_kind(*KINDS[kind], reps[kind]) for kind in KINDS}
+
+    def schedule_counts(n_steps):
+        counts = {}
+        for i in range(n_steps):
+            kind = schedule_kind(wl.steps - (i % wl.steps), wl.steps, wl.Kp, wl.Kr)[2]
+            counts[kind] = counts.get(kind, 0) + 1
+        return counts
+
+    # ---- update-ratio sweep (Fig. 8: throughput against rho), the full-recompute step beside it ------
+    sweep = args.rho_sweep if args.rho_sweep is not None else ("0.1,0.25,0.5" if wl.batch > 1 else "none")
+    rho_sweep = None
+    if sweep != "none":
+        rho_sweep = {"full_recompute_ms": per_kind["full"], "refresh_ms": per_kind["refresh"], "points": []}
+        whole = schedule_counts(wl.steps)
+        for rho in [float(v) for v in sweep.split(",")]:
+            t_partial, t_mixed = time_kind(False, False, 8, rho), time_kind(True, False, 3, rho)
+            total_ms = (whole.get("full", 0) * per_kind["full"] + whole.get("refresh", 0) * per_kind["refresh"] +
+                        whole.get("mixed", 0) * t_mixed + whole.get("partial", 0) * t_partial)
+            rho_sweep["points"].append({
+                "rho": rho, "partial_ms": t_partial, "mixed_ms": t_mixed,
+                "schedule_tokens_per_s": wl.batch * wl.gen_len / (total_ms / 1e3),
+                "speedup_vs_full_recompute": wl.steps * per_kind["full"] / total_ms})
+        rho_sweep["how"] = ("per-kind step times (CUDA events over graph replays) weighted by the step kinds of the "
+                            f"whole {wl.steps}-step schedule; transition launches not included")
 
     # ---- the same schedule with the prediction restricted to the block each step works on -------
     # (reported beside the headline, never as it: the headline step predicts every response row)
@@ -377,10 +476,6 @@ def main():
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-
-    def roundtrip(i):
-        out = ses.tokens()                                  # device -> host: the step's result
-        host_np[...] = out[:, wl.prompt_len:]
     for i in range(K):
         k = wl.steps - (i % wl.steps)
         if i and k == wl.steps:
@@ -390,15 +485,17 @@ def main():
         ses.step_scheduled(k, wl.steps, wl.Kp, wl.Kr, wl.rho)
         bs, nt = block_plan(wl.steps - k, wl.steps, wl.gen_len, wl.block_len)
         ses.remask_low_confidence(bs, wl.block_len, nt)
-        roundtrip(i)
+        host_np[...] = ses.tokens()[:, wl.prompt_len:]      # device -> host: the step's result
     e1.record(stream)
     barrier()
     ms_e2e = e0.elapsed_time(e1)
 
-    # ---- per-kernel times: the same K steps with an event pair around every GEMM and attention launch.
-    # The pairs are event-record nodes of each step's graph (no host latency inside a pair, no overlap between
-    # launches); each step ends with a synchronisation that reads them back, so the replay's own time is the
-    # sum of per-step event pairs, not a span that would include those host gaps.
+    # ---- per-kernel times: the same K steps with an event pair around every launch.  The pairs are event-record
+    # nodes of each step's graph (or host records around plain launches with --prof-mode stream); launches are
+    # serialised and carry no programmatic overlap; each step ends with a synchronisation that reads them back, so
+    # the replay's own time is the sum of per-step event pairs, not a span that would include those host gaps.
+    if args.prof_mode == "stream":
+        ses.use_graphs(False)
     ses.set_prompt(prompt)
     ses.profile(True)
     for k in (wl.steps, wl.steps - 1, wl.steps - 2):        # instantiate the profiling graphs outside the replay
@@ -407,34 +504,36 @@ def main():
     ses.set_prompt(prompt)
     ses.profile(True)
     step_ev = []
-
-    def open_step(i):
-        a = torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        step_ev.append([a, None])
     for i in range(K):
         k = wl.steps - (i % wl.steps)
         if i and k == wl.steps:
             ses.set_prompt(prompt)
-        open_step(i)
+        a = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
         ses.step_scheduled(k, wl.steps, wl.Kp, wl.Kr, wl.rho)
         bs, nt = block_plan(wl.steps - k, wl.steps, wl.gen_len, wl.block_len)
         ses.remask_low_confidence(bs, wl.block_len, nt)
         b = torch.cuda.Event(enable_timing=True)
         b.record(stream)
-        step_ev[-1][1] = b
+        step_ev.append((a, b))
+        if args.prof_mode == "stream" and i % 8 == 7:
+            ses.sync()
     ses.sync()
     ms_replay = sum(a.elapsed_time(b) for a, b in step_ev)
-    g = ses.profile_read(0)
-    at = ses.profile_read(1)
+    prof = {name: ses.profile_read(i) for i, name in enumerate(dllm.PROF_CLASSES)}
     ses.profile(False)
 
-    # algorithmic GEMM bytes of ONE adaptive partial step (the library's own count), for the in-graph figure
-    ses.profile(True)
-    ses.step_cached(False, False, wl.rho)
-    ses.sync()
-    partial_gemm_bytes = ses.profile_read(0)["bytes"]
-    ses.profile(False)
+    # algorithmic bytes / FLOPs of ONE step of each kind (the library's own count), for the per-step fractions
+    # and the in-graph figure
+    per_kind_work = {}
+    for kind, (rp, rr) in KINDS.items():
+        ses.profile(True)
+        ses.step_cached(rp, rr, wl.rho)
+        ses.sync()
+        per_kind_work[kind] = {name: ses.profile_read(i) for i, name in enumerate(dllm.PROF_CLASSES[2:], 2)}
+        ses.profile(False)
+    ses.use_graphs(True)
+    partial_gemm_bytes = sum(v["bytes"] for k_, v in per_kind_work["partial"].items() if k_.startswith("gemm"))
 
     # max over ranks
     ms, ms_e2e = aggregate_over_ranks(ms, ms_e2e, world, dev)
@@ -445,19 +544,23 @@ def main():
 
     tokens = tokens_processed(K, wl.batch, wl.gen_len, wl.steps, world)
     value = tokens / (ms / 1e3)
-    gemm_gbs = g["bytes"] / (g["ms"] / 1e3) / 1e9 if g["ms"] > 0 else 0.0
-    counts = {}
-    for i in range(K):
-        kind = schedule_kind(wl.steps - (i % wl.steps), wl.steps, wl.Kp, wl.Kr)[2]
-        counts[kind] = counts.get(kind, 0) + 1
+    kernels = {name: roofline_of(name, rec, peaks) for name, rec in prof.items()}
+    kernels = {k_: v for k_, v in kernels.items() if v is not None}
+    g = kernels["gemm"]
+    steps_roof = {}
+    for kind, work in per_kind_work.items():
+        roof = step_roof_ms(work, peaks)
+        steps_roof[kind] = {"ms": per_kind[kind], "roofline_ms": roof, "frac": roof / per_kind[kind],
+                            "algorithmic_gb": sum(v["bytes"] for v in work.values()) / 1e9,
+                            "algorithmic_tflop": sum(v["flops"] for v in work.values()) / 1e12}
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
         "config": workload_config(wl, args),
         "steps_per_s": K * world / (ms / 1e3),
-        "step_kinds": counts,
-        "ms_per_kind": {k: round(v, 4) for k, v in per_kind.items()},
+        "step_kinds": schedule_counts(K),
+        "ms_per_kind": {k_: round(v, 4) for k_, v in per_kind.items()},
         "speedup_vs_full_recompute": per_kind["full"] / (ms / K),
         "full_recompute_tokens_per_s": wl.batch * wl.gen_len / wl.steps * world / (per_kind["full"] / 1e3),
         "e2e": {"value": tokens / (ms_e2e / 1e3), "unit": "tokens/s",
@@ -468,21 +571,33 @@ def main():
                                           "block the step works on; layers and caches identical"},
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "roofline": {"kernel": "gemm_bf16_tcgen05_kernel", "bound": "hbm", "achieved": gemm_gbs,
-                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"],
-                     "peak_source": peaks["source"], "traffic": TRAFFIC_PER_LAUNCH.get(args.workload),
-                     "launches": g["launches"], "avg_launch_us": 1e3 * g["ms"] / max(g["launches"], 1),
-                     "algorithmic_bytes_per_launch": g["bytes"] / max(g["launches"], 1),
-                     "gemm_share_of_step": g["ms"] / max(ms_replay, 1e-9),
-                     "attention": {"ms_total": at["ms"], "launches": at["launches"],
-                                   "gbs": at["bytes"] / (at["ms"] / 1e3) / 1e9 if at["ms"] > 0 else 0.0,
-                                   "tflops": at["flops"] / (at["ms"] / 1e3) / 1e12 if at["ms"] > 0 else 0.0},
-                     "how": "CUDA-event pairs around every GEMM launch (event-record nodes in the step graphs, launches "
-                            "serialised, no programmatic overlap) in a replay of the same K steps; share = GEMM event "
-                            "time / summed per-step event time of that replay"},
+        "roofline": {"kernel": "gemm_bf16_tcgen05_kernel / gemm_bf16_pair_kernel (all projections of the timed steps)",
+                     "bound": g["bound"], "achieved": g["achieved"], "peak": g["peak"], "unit": g["unit"],
+                     "frac": g["frac"], "frac_of_nominal": g["frac_of_nominal"],
+                     "nominal_peak": NOMINAL["bf16_tflops"] if g["bound"] == "tensor" else NOMINAL["hbm_gbs"],
+                     "peak_source": peaks["source"] + (" (sustained bf16)" if g["bound"] == "tensor" else " (copy)"),
+                     "traffic": TRAFFIC_PER_LAUNCH.get(args.workload) if not args.layers else None,
+                     "launches": g["launches"], "avg_launch_us": g["avg_us"],
+                     "algorithmic_bytes_per_launch": g["bytes_per_launch"],
+                     "algorithmic_flops_per_launch": g["flops_per_launch"],
+                     "gemm_share_of_step": g["ms_total"] / max(ms_replay, 1e-9),
+                     "how": "CUDA-event pairs around every launch (" +
+                            ("event-record nodes in the step graphs" if args.prof_mode == "graph" else
+                             "host records around plain launches") +
+                            ", launches serialised, no programmatic overlap) in a replay of the same K steps; "
+                            "share = event time of the class / summed per-step event time of that replay; the "
+                            "binding roof of a class follows from its algorithmic flop per byte against the ridge "
+                            "of the measured peaks"},
+        "kernels": kernels,
+        "steps_roofline": steps_roof,
         "unmasked_tokens": int((final_tokens[:, wl.prompt_len:] != cfg.mask_id).sum()),
     }
-    if world == 1 and not args.no_timeline:
+    if rho_sweep is not None:
+        line["rho_sweep"] = rho_sweep
+    if args.compact_cache:
+        line["config"]["cache"] = "response-only AttnOut / FFNOut"
+    line["cache_bytes"] = int(ses.cache.numel())
+    if world == 1 and not args.no_timeline and not args.layers and args.rho is None:
         line["roofline"]["in_graph"] = in_graph_gemm(args.workload, partial_gemm_bytes, peaks)
     if not args.no_cpu_baseline:
         t = time_oracle(wl, budget_s=25.0, steps=K)
@@ -510,7 +625,8 @@ def in_graph_gemm(workload, gemm_bytes, peaks):
         us = sum(o["dur_us"] for o in gemm)
         total = launches[-1]["start_us"]
         gbs = gemm_bytes / (us * 1e-6) / 1e9
-        return {"achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "gemm_us": us, "gemm_launches": len(gemm),
+        return {"achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                "frac_of_nominal": gbs / NOMINAL["hbm_gbs"], "gemm_us": us, "gemm_launches": len(gemm),
                 "step_us": total, "gemm_share_of_step": us / max(total, 1e-9),
                 "how": "one adaptive partial step replayed as a CUDA graph in the timeline build of the library: "
                        "per launch, device time from its predecessor's completion to its own (globaltimer at "
@@ -518,11 +634,6 @@ def in_graph_gemm(workload, gemm_bytes, peaks):
     except Exception:
         return None
 
-
-# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch from the ncu capture summarised under
-# profiles/ncu_gemm_bf16_tcgen05_partial_step_2layers.md: 451 MB per layer of an adaptive partial step over 5
-# launches, plus the LM head's 1,051 MB once per step (32 layers: 15.48 GB / 161 launches).
-TRAFFIC_PER_LAUNCH = {"llada8b": 96.2e6}
 
 if __name__ == "__main__":
     main()

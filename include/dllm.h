@@ -256,26 +256,40 @@ dllm_status dllm_session_use_graphs(dllm_session* s, int enable);
  * projections) overlaps the tail of the kernel before it; 0: plain launches. */
 dllm_status dllm_session_use_pdl(dllm_session* s, int enable);
 
-/* L2 prefetch of the coming projections' weights by the row-wise kernels of a
- * weight-bound step (at most 512 active rows): between two projections HBM is
- * nearly idle, so the kernels there may ask for the head of the next weight
- * matrix.  h_kb: up to five sizes in KB (missing ones are 0 = off): V-verify ->
- * W_q/W_k; selection + gather -> W_q/W_k continued; RoPE -> W_o, running on
- * into W_gate/W_up; O-projection epilogue -> W_gate/W_up continued; layer tail
- * -> the next layer's W_v.  Results are unaffected; a tuning hook (default: all
- * off until set). */
-dllm_status dllm_session_set_prefetch(dllm_session* s, const int* h_kb, int n);
-
-/* Per-kernel timing.  While enabled, every projection GEMM (class 0) and
- * attention launch (class 1) is bracketed by CUDA events on the caller's stream
- * and no launch overlaps its predecessor (no programmatic dependent launch).
- * With CUDA graphs on, the event records are nodes of the step's graph, so no
- * host latency falls between a pair and its kernel; every step then ends with
- * a stream synchronisation that reads the pairs back.  _profile_read
- * synchronises the device and returns, for one class, the summed event time,
- * the number of launches, and the algorithmic bytes and FLOPs of those launches
- * (GEMM: W and A once in, one fp32 result out; attention: K, V, Q in, O out).
- * Enabling or disabling discards earlier records. */
+/* Per-kernel timing.  While enabled, every kernel launch of a step is bracketed
+ * by a pair of CUDA events on the caller's stream and no launch overlaps its
+ * predecessor (no programmatic dependent launch).  With CUDA graphs on, the
+ * event records are nodes of the step's graph, so no host latency falls between
+ * a pair and its kernel; every step then ends with a stream synchronisation
+ * that reads the pairs back.  _profile_read synchronises the device and
+ * returns, for one class of launches, the summed event time, the number of
+ * launches, and their algorithmic bytes and FLOPs: what the operation must
+ * move and compute (a projection: W and A once in, one result out; attention:
+ * K, V, Q in, O out; a row-wise kernel: its rows in and out), not the split-K
+ * slabs or other scratch traffic.  DLLM_PROF_GEMM and DLLM_PROF_ATTENTION are
+ * sums over their sub-classes.  Enabling or disabling discards earlier records. */
+enum {
+  DLLM_PROF_GEMM = 0,       /* all projections: the six classes GEMM_V .. GEMM_HEAD */
+  DLLM_PROF_ATTENTION = 1,  /* both attention kernels, each with the merge of its key-range splits */
+  DLLM_PROF_GEMM_V = 2,     /* V (K in the K-verify ablation) of all response rows; V of prompt / selected rows */
+  DLLM_PROF_GEMM_QK = 3,    /* Q and K of the active rows */
+  DLLM_PROF_GEMM_O = 4,
+  DLLM_PROF_GEMM_GU = 5,    /* gate and up, with SwiGLU in the epilogue when unsplit */
+  DLLM_PROF_GEMM_D = 6,
+  DLLM_PROF_GEMM_HEAD = 7,  /* LM head with the estimate epilogue */
+  DLLM_PROF_ATTN_MMA = 8,   /* up to 64 rows per KV head (mma.sync) */
+  DLLM_PROF_ATTN_UMMA = 9,  /* more rows (tcgen05) */
+  DLLM_PROF_VVERIFY = 10,   /* Eq. 6 + V overwrite */
+  DLLM_PROF_SELECT = 11,    /* bottom-k selection + gather of the active rows */
+  DLLM_PROF_ROPE = 12,      /* RoPE + K scatter */
+  DLLM_PROF_OEPI = 13,      /* AttnOut scatter + residual + RMSNorm-2 */
+  DLLM_PROF_SILU = 14,      /* SwiGLU after a split gate / up projection */
+  DLLM_PROF_TAIL = 15,      /* FFNOut scatter + residual assembly + next RMSNorm */
+  DLLM_PROF_EMBED = 16,     /* embedding + first RMSNorm */
+  DLLM_PROF_ESTIMATE = 17,  /* merge of the estimate records (or argmax over logits) */
+  DLLM_PROF_SCATTER = 18,   /* V rows of prompt / selected rows into the cache */
+  DLLM_PROF_COUNT = 19
+};
 dllm_status dllm_session_profile(dllm_session* s, int enable);
 dllm_status dllm_session_profile_read(dllm_session* s, int cls, double* total_ms, uint64_t* launches,
                                       double* algorithmic_bytes, double* flops);
@@ -302,11 +316,10 @@ dllm_status dllm_kernel_status(void* stream);
  * records the status code, skips its epilogue, frees its tensor memory and
  * returns normally; (0) switches that off.  Both calls synchronise the device. */
 dllm_status dllm_debug_set_wait_limit_ns(uint64_t ns);
-/* Tuning hook: overrides the launch plan of the 64-row attention kernel for
- * every later call in this process: `splits` key-range splits over CTAs and up
- * to `groups` (1..3) groups of 128 threads per CTA; 0 = automatic.  Results
- * stay within the attention tolerance; merge orders change with the plan. */
-dllm_status dllm_debug_attention_plan(int splits, int groups);
+/* Tuning hook: overrides, for every later call in this process, the number of
+ * key-range splits the 64-row attention kernel takes (0 = automatic).  Results
+ * stay within the attention tolerance; the merge order changes with the plan. */
+dllm_status dllm_debug_attention_plan(int splits);
 dllm_status dllm_debug_skip_one_load(int enable);
 /* C[M,N] (fp32, row-major, DEVICE) = A[M,K] * W[N,K]^T with bf16 operands on
  * the tensor cores (tcgen05 + TMA).  d_partials is scratch of

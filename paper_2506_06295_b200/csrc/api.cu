@@ -255,10 +255,6 @@ struct dllm_session {
   bool use_pdl = true;
   int sel_strategy = DLLM_SELECT_V_VERIFY, sel_metric = DLLM_METRIC_COSINE, v_selected_only = 0;  // ablation variants
   bool block_head = false;     // dllm_generate predicts only the block each step works on
-  // L2 prefetch of the coming projection's weights from the row-wise kernels (KB per slot, 0 = off):
-  // [0] V-verify -> W_q/W_k, [1] selection + gather -> W_q/W_k continued, [2] RoPE -> W_o (running on into
-  // W_gate/W_up), [3] O epilogue -> W_gate/W_up continued, [4] layer tail -> the next layer's W_v
-  size_t pf_kb[5] = {0, 0, 0, 0, 0};
   struct GraphEntry {
     cudaGraphExec_t exec;
     uint64_t kernels;
@@ -281,7 +277,7 @@ struct dllm_session {
   bool profiling = false;
   std::vector<ProfRec> prof;        // recorded by the host, one pair per launch
   std::vector<ProfRec> graph_prof;  // owned by profiling graphs
-  ProfSum prof_sum[2];              // read back from graph replays
+  ProfSum prof_sum[DLLM_PROF_COUNT];  // read back from graph replays
   std::vector<cudaEvent_t> event_pool;
   cudaEvent_t take_event() {
     if (!event_pool.empty()) {
@@ -387,8 +383,20 @@ int k_selected(float rho, int R, dllm_kround kr) {
   return (int)k;
 }
 
+// Event pair of one launch while the session is profiling (class, algorithmic bytes and FLOPs of the launch).
+struct ProfScope {
+  dllm_session* s;
+  cudaStream_t st;
+  ProfScope(dllm_session* s_, int cls, double bytes, double flops, cudaStream_t st_) : s(s_), st(st_) {
+    s->prof_begin(cls, bytes, flops, st);
+  }
+  ~ProfScope() { s->prof_end(st); }
+  ProfScope(const ProfScope&) = delete;
+  ProfScope& operator=(const ProfScope&) = delete;
+};
+
 // One GEMM of the step: out = A[M,K] * W[N,K]^T as split-K partial slabs.
-dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void* W, int M, int N, int K,
+dllm_status run_gemm(dllm_session* s, const Launch& L, int cls, const void* A, const void* W, int M, int N, int K,
                      Partials* out, void* swiglu_out = nullptr, bool* fused = nullptr, int estimate_mask_id = -1) {
   float* part = s->wsp<float>(s->ws.part);
   if (fused) *fused = false;
@@ -404,7 +412,7 @@ dllm_status run_gemm(dllm_session* s, const Launch& L, const void* A, const void
   // algorithmic traffic of one projection: the weight matrix and the activation rows once in, one result out
   // (fp32, or what the fused epilogue writes; split-K slabs are overhead, not counted)
   const double out_bytes = estimate ? (double)M * ((N + 127) / 128) * 16.0 : fuse ? (double)M * (N / 2) * 2.0 : (double)M * N * 4.0;
-  s->prof_begin(0, ((double)N * K + (double)M * K) * es + out_bytes, 2.0 * M * N * K, L.stream);
+  s->prof_begin(cls, ((double)N * K + (double)M * K) * es + out_bytes, 2.0 * M * N * K, L.stream);
   struct End {
     dllm_session* s;
     cudaStream_t st;
@@ -447,8 +455,11 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
   Partials part{nullptr, 0, 1, 0};
 
   int32_t* inv = s->wsp<int32_t>(s->ws.inv);
-  launch_embed_norm(L, dt, W + wl.embed, s->wsp<int32_t>(s->ws.tokens), x,
-                    reinterpret_cast<const float*>(W + wl.layers[0].norm1), u, g, c0, c1, c.rms_eps);
+  {
+    ProfScope ps(s, DLLM_PROF_EMBED, (double)(c1 - c0) * d * (4.0 + 2.0 * es), 4.0 * (c1 - c0) * d, stream);
+    launch_embed_norm(L, dt, W + wl.embed, s->wsp<int32_t>(s->ws.tokens), x,
+                      reinterpret_cast<const float*>(W + wl.layers[0].norm1), u, g, c0, c1, c.rms_eps);
+  }
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerOff& lo = wl.layers[l];
     uint8_t* Wq = W + lo.wqkv;
@@ -460,26 +471,6 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
     const int ksel = ksels[l];  // rows of the response this layer recomputes
     const int a_seq = (rp ? s->P : 0) + ksel;
     const int Ma = s->B * a_seq;
-    // prefetch spans (weight-bound steps only: with many active rows the projections are not waiting for HBM)
-    Prefetch pf_qk0, pf_qk1, pf_o, pf_gu, pf_v;
-    if (dt == DLLM_BF16 && Ma > 0 && Ma <= 512) {
-      auto span = [](const uint8_t* p, size_t lo, size_t want, size_t cap) {
-        Prefetch f;
-        if (lo < cap && want > 0) {
-          f.p = p + lo;
-          f.bytes = std::min(want, cap - lo);
-        }
-        return f;
-      };
-      const size_t KB = 1024, qk_bytes = (size_t)(dq + dkv) * d * es, gu_end = lo.wgu + (size_t)2 * m * d * es;
-      pf_qk0 = span(Wq, 0, s->pf_kb[0] * KB, qk_bytes);
-      pf_qk1 = span(Wq, s->pf_kb[0] * KB, s->pf_kb[1] * KB, qk_bytes);
-      pf_o = span(W + lo.wo, 0, s->pf_kb[2] * KB, gu_end - lo.wo);
-      const size_t into_gu = lo.wo + s->pf_kb[2] * KB > lo.wgu ? lo.wo + s->pf_kb[2] * KB - lo.wgu : 0;
-      pf_gu = span(W + lo.wgu, into_gu, s->pf_kb[3] * KB, (size_t)2 * m * d * es);
-      if (l + 1 < c.n_layers)
-        pf_v = span(W + wl.layers[l + 1].wqkv + (size_t)(dq + dkv) * d * es, 0, s->pf_kb[4] * KB, (size_t)dkv * d * es);
-    }
     const bool adaptive = !rr && ksel > 0;
     const int mode = rr ? 0 : (s->forced_count[l] >= 0 ? 2 : 1);
     // A response refresh alone takes every response row in carried order: u itself is the operand of the
@@ -487,20 +478,25 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
     const bool identity = rr && !rp && Ma > 0;
     if (rr || (adaptive && s->sel_strategy == DLLM_SELECT_V_VERIFY)) {
       // V for ALL response rows (the 2 r d^2 term of Sec. A.7), V-verify, V overwrite
-      if ((st = run_gemm(s, L, u, Wv, BR, dkv, d, &part)) != DLLM_OK) return st;
+      if ((st = run_gemm(s, L, DLLM_PROF_GEMM_V, u, Wv, BR, dkv, d, &part)) != DLLM_OK) return st;
       const IdentityLists id{sel, act, inv};
-      launch_vverify(L, dt, part, s->cache(l, DLLM_CACHE_V), sim, g, dkv, rr ? 0 : s->sel_metric,
-                     rr || !s->v_selected_only, identity ? &id : nullptr, pf_qk0);
+      {  // the projection's fp32 result in, the cached row in, the row out
+        ProfScope ps(s, DLLM_PROF_VVERIFY, (double)BR * dkv * (4.0 + 2.0 * es), 6.0 * BR * dkv, stream);
+        launch_vverify(L, dt, part, s->cache(l, DLLM_CACHE_V), sim, g, dkv, rr ? 0 : s->sel_metric,
+                       rr || !s->v_selected_only, identity ? &id : nullptr);
+      }
     } else if (adaptive && s->sel_strategy == DLLM_SELECT_K_VERIFY) {
       // ablation: the same test on K; K of ALL response rows is projected, rotated and overwritten
-      if ((st = run_gemm(s, L, u, Wq + (size_t)dq * d * es, BR, dkv, d, &part)) != DLLM_OK) return st;
+      if ((st = run_gemm(s, L, DLLM_PROF_GEMM_V, u, Wq + (size_t)dq * d * es, BR, dkv, d, &part)) != DLLM_OK) return st;
+      ProfScope ps(s, DLLM_PROF_VVERIFY, (double)BR * dkv * (4.0 + 2.0 * es), 10.0 * BR * dkv, stream);
       launch_kverify(L, dt, part, s->cache(l, DLLM_CACHE_K), sim, s->wsp<float>(s->ws.rope), g, Hkv, hd,
                      s->sel_metric);
     }  // random selection: the scores were set by dllm_set_scores
     // V of the active rows is still missing when the verify pass did not write it
     const bool v_for_active = adaptive && (s->sel_strategy != DLLM_SELECT_V_VERIFY || s->v_selected_only);
     if (rp) {
-      if ((st = run_gemm(s, L, u + (size_t)BR * d * es, Wv, BP, dkv, d, &part)) != DLLM_OK) return st;
+      if ((st = run_gemm(s, L, DLLM_PROF_GEMM_V, u + (size_t)BR * d * es, Wv, BP, dkv, d, &part)) != DLLM_OK) return st;
+      ProfScope ps(s, DLLM_PROF_SCATTER, (double)BP * dkv * (4.0 + es), 0.0, stream);
       launch_scatter_rows(L, dt, part, nullptr, BR, s->cache(l, DLLM_CACHE_V), g, BP, dkv);
     }
     if (Ma > 0) {
@@ -509,42 +505,62 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
         ua = u;
       } else if (s->R <= 1024 && (long)Ma * s->R <= 64L * 1024) {
         // few active rows: every CTA of the gather repeats the selection rather than wait for a launch
-        launch_select_gather(L, dt, sim, forced, mode, ksel, sel, act, inv, u, s->wsp<uint8_t>(s->ws.ua), g, rp,
-                             pf_qk1);
+        ProfScope ps(s, DLLM_PROF_SELECT, (double)Ma * d * 2.0 * es + (double)BR * 4.0, 0.0, stream);
+        launch_select_gather(L, dt, sim, forced, mode, ksel, sel, act, inv, u, s->wsp<uint8_t>(s->ws.ua), g, rp);
       } else {
+        ProfScope ps(s, DLLM_PROF_SELECT, (double)Ma * d * 2.0 * es + (double)BR * 4.0, 0.0, stream);
         cudaError_t se = launch_select(L, sim, forced, mode, ksel, sel, s->R, act, inv, g, rp);
         if (se != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "selection: %s", cudaGetErrorString(se));
         launch_gather_rows(L, dt, u, act, s->wsp<uint8_t>(s->ws.ua), Ma, d);
       }
       if (v_for_active) {
-        if ((st = run_gemm(s, L, ua, Wv, Ma, dkv, d, &part)) != DLLM_OK) return st;
+        if ((st = run_gemm(s, L, DLLM_PROF_GEMM_V, ua, Wv, Ma, dkv, d, &part)) != DLLM_OK) return st;
+        ProfScope ps(s, DLLM_PROF_SCATTER, (double)Ma * dkv * (4.0 + es), 0.0, stream);
         launch_scatter_rows(L, dt, part, act, 0, s->cache(l, DLLM_CACHE_V), g, Ma, dkv);
       }
       // Q and K of the active rows in one GEMM over the stacked [W_q; W_k]
-      if ((st = run_gemm(s, L, ua, Wq, Ma, dq + dkv, d, &part)) != DLLM_OK) return st;
-      launch_qk_rope(L, dt, part, act, s->wsp<float>(s->ws.rope), s->wsp<uint8_t>(s->ws.qbuf),
-                     s->cache(l, DLLM_CACHE_K), g, Ma, H, Hkv, hd, pf_o);
-      // algorithmic traffic: K and V of every sequence once, Q in, O out
-      s->prof_begin(1, (2.0 * s->B * s->n * dkv + 2.0 * Ma * dq) * (double)es, 4.0 * Ma * (double)s->n * dq, stream);
+      if ((st = run_gemm(s, L, DLLM_PROF_GEMM_QK, ua, Wq, Ma, dq + dkv, d, &part)) != DLLM_OK) return st;
+      {
+        ProfScope ps(s, DLLM_PROF_ROPE, (double)Ma * (dq + dkv) * (4.0 + es), 6.0 * Ma * (dq + dkv), stream);
+        launch_qk_rope(L, dt, part, act, s->wsp<float>(s->ws.rope), s->wsp<uint8_t>(s->ws.qbuf),
+                       s->cache(l, DLLM_CACHE_K), g, Ma, H, Hkv, hd);
+      }
+      // algorithmic traffic: K and V of every sequence once, Q in, O out (the merge of split key ranges runs
+      // inside the same pair).  Class by the kernel the shape takes: 64-row mma.sync or 128-row tcgen05.
+      const bool attn_tc = dt == DLLM_BF16 && !s->simt_gemm && (hd == 64 || hd == 128);
+      s->prof_begin(attn_tc && a_seq * (H / Hkv) > 64 ? DLLM_PROF_ATTN_UMMA : DLLM_PROF_ATTN_MMA,
+                    (2.0 * s->B * s->n * dkv + 2.0 * Ma * dq) * (double)es, 4.0 * Ma * (double)s->n * dq, stream);
       cudaError_t e = launch_attention(L, dt, s->wsp<uint8_t>(s->ws.qbuf), s->cache(l, DLLM_CACHE_K),
                                        s->cache(l, DLLM_CACHE_V), s->wsp<uint8_t>(s->ws.obuf), s->B, a_seq, s->n, H,
                                        Hkv, hd, s->wsp<float>(s->ws.attn), s->ws.attn_floats, s->simt_gemm);
       s->prof_end(stream);
       if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
-      if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.obuf), W + lo.wo, Ma, d, dq, &part)) != DLLM_OK) return st;
-      launch_oproj_epilogue(L, dt, part, act, x, reinterpret_cast<const float*>(W + lo.norm2),
-                            s->outs(l, DLLM_CACHE_ATTN), s->wsp<uint8_t>(s->ws.hn), g, Ma, c.rms_eps, pf_gu);
-      bool fused = false;
-      if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.hn), W + lo.wgu, Ma, 2 * m, d, &part, s->wsp<uint8_t>(s->ws.ffn),
-                         &fused)) != DLLM_OK)
+      if ((st = run_gemm(s, L, DLLM_PROF_GEMM_O, s->wsp<uint8_t>(s->ws.obuf), W + lo.wo, Ma, d, dq, &part)) != DLLM_OK)
         return st;
-      if (!fused) launch_silu_mul(L, dt, part, s->wsp<uint8_t>(s->ws.ffn), Ma, m, gu_interleaved(c));
-      if ((st = run_gemm(s, L, s->wsp<uint8_t>(s->ws.ffn), W + lo.wd, Ma, d, m, &part)) != DLLM_OK) return st;
+      {  // projection result and x in, AttnOut row and the normalised row out
+        ProfScope ps(s, DLLM_PROF_OEPI, (double)Ma * d * (8.0 + 2.0 * es), 6.0 * Ma * d, stream);
+        launch_oproj_epilogue(L, dt, part, act, x, reinterpret_cast<const float*>(W + lo.norm2),
+                              s->outs(l, DLLM_CACHE_ATTN), s->wsp<uint8_t>(s->ws.hn), g, Ma, c.rms_eps);
+      }
+      bool fused = false;
+      if ((st = run_gemm(s, L, DLLM_PROF_GEMM_GU, s->wsp<uint8_t>(s->ws.hn), W + lo.wgu, Ma, 2 * m, d, &part,
+                         s->wsp<uint8_t>(s->ws.ffn), &fused)) != DLLM_OK)
+        return st;
+      if (!fused) {
+        ProfScope ps(s, DLLM_PROF_SILU, (double)Ma * m * (8.0 + es), 8.0 * Ma * m, stream);
+        launch_silu_mul(L, dt, part, s->wsp<uint8_t>(s->ws.ffn), Ma, m, gu_interleaved(c));
+      }
+      if ((st = run_gemm(s, L, DLLM_PROF_GEMM_D, s->wsp<uint8_t>(s->ws.ffn), W + lo.wd, Ma, d, m, &part)) != DLLM_OK)
+        return st;
     }
     // FFNOut rows -> cache, residual assembly for all carried rows, next norm
     const float* gain_next = reinterpret_cast<const float*>(l + 1 < c.n_layers ? W + wl.layers[l + 1].norm1 : W + wl.norm_f);
-    launch_tail(L, dt, part, Ma > 0 ? inv : nullptr, x, s->outs(l, DLLM_CACHE_ATTN), s->outs(l, DLLM_CACHE_FFN),
-                gain_next, u, g, c0, c1, c.rms_eps, pf_v);
+    {  // x in and out, AttnOut and FFNOut rows in, the normalised row out; the FFN result of the active rows in and out
+      ProfScope ps(s, DLLM_PROF_TAIL, (double)(c1 - c0) * d * (8.0 + 3.0 * es) + (double)Ma * d * (4.0 + es),
+                   6.0 * (c1 - c0) * d, stream);
+      launch_tail(L, dt, part, Ma > 0 ? inv : nullptr, x, s->outs(l, DLLM_CACHE_ATTN), s->outs(l, DLLM_CACHE_FFN),
+                  gain_next, u, g, c0, c1, c.rms_eps);
+    }
   }
   // prediction at the response rows (Eqs. 3-4); u holds the final norm.  With head_len > 0 only the rows of
   // one block are predicted: the transition of a semi-autoregressive step reads no others (Eq. 5).
@@ -560,15 +576,21 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
     }
   }
   bool est = false;
-  if ((st = run_gemm(s, L, head_in, W + wl.lm_head, head_rows, c.vocab, d, &part, nullptr, &est, c.mask_id)) != DLLM_OK)
+  if ((st = run_gemm(s, L, DLLM_PROF_GEMM_HEAD, head_in, W + wl.lm_head, head_rows, c.vocab, d, &part, nullptr, &est,
+                     c.mask_id)) != DLLM_OK)
     return st;
   if (part.S != 1) return fail(&s->err, DLLM_UNSUPPORTED, "LM head GEMM must not be split");
-  if (est)  // the projection left one (max, sum exp, argmax) record per row and weight tile instead of logits
-    launch_estimate_merge(L, part.p, head_rows, (c.vocab + 127) / 128, s->wsp<int32_t>(s->ws.x0),
-                          s->wsp<float>(s->ws.conf), s->R, head_start, head_len);
-  else
-    launch_argmax_conf(L, part.p, head_rows, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0), s->wsp<float>(s->ws.conf),
-                       s->R, head_start, head_len);
+  {
+    ProfScope ps(s, DLLM_PROF_ESTIMATE,
+                 est ? (double)head_rows * ((c.vocab + 127) / 128) * 16.0 : (double)head_rows * c.vocab * 4.0,
+                 est ? 0.0 : 4.0 * head_rows * c.vocab, stream);
+    if (est)  // the projection left one (max, sum exp, argmax) record per row and weight tile instead of logits
+      launch_estimate_merge(L, part.p, head_rows, (c.vocab + 127) / 128, s->wsp<int32_t>(s->ws.x0),
+                            s->wsp<float>(s->ws.conf), s->R, head_start, head_len);
+    else
+      launch_argmax_conf(L, part.p, head_rows, c.vocab, c.mask_id, s->wsp<int32_t>(s->ws.x0),
+                         s->wsp<float>(s->ws.conf), s->R, head_start, head_len);
+  }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "step launch: %s", cudaGetErrorString(e));
   return DLLM_OK;
@@ -978,7 +1000,22 @@ static dllm_status read_status_word(std::string* slot, int* d_word, cudaStream_t
 
 dllm_status dllm_sync(dllm_session* s, void* stream) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
-  return read_status_word(&s->err, s->wsp<int>(s->ws.status), (cudaStream_t)stream);
+  const dllm_status st = read_status_word(&s->err, s->wsp<int>(s->ws.status), (cudaStream_t)stream);
+  // host-recorded event pairs of a profiled run have completed: fold them into the sums and reuse the events
+  for (auto& r : s->prof) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) {
+      dllm_session::ProfSum& acc = s->prof_sum[r.cls];
+      acc.ms += t;
+      acc.bytes += r.bytes;
+      acc.flops += r.flops;
+      ++acc.launches;
+    }
+    s->event_pool.push_back(r.a);
+    s->event_pool.push_back(r.b);
+  }
+  s->prof.clear();
+  return st;
 }
 
 dllm_status dllm_kernel_status(void* stream) {
@@ -1056,7 +1093,8 @@ dllm_status dllm_get_logits(dllm_session* s, float* h_out, void* stream) {
   launch_rmsnorm(L, c.dtype, s->wsp<float>(s->ws.x), reinterpret_cast<const float*>(s->m->d_w + s->m->lay.norm_f),
                  s->wsp<uint8_t>(s->ws.u), c.d_model, c.rms_eps, 0, BR);
   Partials part{nullptr, 0, 1, 0};
-  dllm_status r = run_gemm(s, L, s->wsp<uint8_t>(s->ws.u), s->m->d_w + s->m->lay.lm_head, BR, c.vocab, c.d_model, &part);
+  dllm_status r = run_gemm(s, L, DLLM_PROF_GEMM_HEAD, s->wsp<uint8_t>(s->ws.u), s->m->d_w + s->m->lay.lm_head, BR,
+                           c.vocab, c.d_model, &part);
   if (r != DLLM_OK) return r;
   launch_mask_column(L, s->wsp<float>(s->ws.part), BR, c.vocab, c.mask_id);
   CU_TRY(&s->err, cudaStreamSynchronize(st));
@@ -1178,16 +1216,6 @@ dllm_status dllm_set_scores(dllm_session* s, int layer, const float* h_scores, v
   return DLLM_OK;
 }
 
-dllm_status dllm_session_set_prefetch(dllm_session* s, const int* h_kb, int n) {
-  if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
-  if (n < 0 || n > 5 || (n > 0 && !h_kb)) return fail(&s->err, DLLM_INVALID_ARG, "at most five prefetch sizes");
-  for (int i = 0; i < n; ++i)
-    if (h_kb[i] < 0) return fail(&s->err, DLLM_INVALID_ARG, "negative prefetch size");
-  for (int i = 0; i < 5; ++i) s->pf_kb[i] = i < n ? (size_t)h_kb[i] : 0;
-  s->drop_graphs();
-  return DLLM_OK;
-}
-
 dllm_status dllm_session_use_simt_gemm(dllm_session* s, int enable) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
   if ((enable != 0) != s->simt_gemm) {
@@ -1205,7 +1233,7 @@ dllm_status dllm_session_profile(dllm_session* s, int enable) {
     s->event_pool.push_back(r.b);
   }
   s->prof.clear();
-  s->prof_sum[0] = s->prof_sum[1] = dllm_session::ProfSum{};
+  for (auto& ps : s->prof_sum) ps = dllm_session::ProfSum{};
   s->profiling = enable != 0;
   return DLLM_OK;
 }
@@ -1213,12 +1241,25 @@ dllm_status dllm_session_profile(dllm_session* s, int enable) {
 dllm_status dllm_session_profile_read(dllm_session* s, int cls, double* total_ms, uint64_t* launches,
                                       double* algorithmic_bytes, double* flops) {
   if (!s) return fail(nullptr, DLLM_INVALID_ARG, "session is NULL");
-  if (cls < 0 || cls > 1) return fail(&s->err, DLLM_INVALID_ARG, "class must be 0 (GEMM) or 1 (attention)");
+  if (cls < 0 || cls >= DLLM_PROF_COUNT) return fail(&s->err, DLLM_INVALID_ARG, "unknown profile class");
   CU_TRY(&s->err, cudaDeviceSynchronize());
-  double ms = s->prof_sum[cls].ms, by = s->prof_sum[cls].bytes, fl = s->prof_sum[cls].flops;
-  uint64_t cnt = s->prof_sum[cls].launches;
+  // the two aggregates: every projection, every attention launch
+  auto in_class = [cls](int c) {
+    if (cls == DLLM_PROF_GEMM) return c >= DLLM_PROF_GEMM_V && c <= DLLM_PROF_GEMM_HEAD;
+    if (cls == DLLM_PROF_ATTENTION) return c == DLLM_PROF_ATTN_MMA || c == DLLM_PROF_ATTN_UMMA;
+    return c == cls;
+  };
+  double ms = 0, by = 0, fl = 0;
+  uint64_t cnt = 0;
+  for (int c = 0; c < DLLM_PROF_COUNT; ++c)
+    if (in_class(c)) {
+      ms += s->prof_sum[c].ms;
+      by += s->prof_sum[c].bytes;
+      fl += s->prof_sum[c].flops;
+      cnt += s->prof_sum[c].launches;
+    }
   for (auto& r : s->prof) {
-    if (r.cls != cls) continue;
+    if (!in_class(r.cls)) continue;
     float t = 0.f;
     CU_TRY(&s->err, cudaEventElapsedTime(&t, r.a, r.b));
     ms += t;

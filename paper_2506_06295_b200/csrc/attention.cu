@@ -112,41 +112,30 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(const T* __restrict__ q,
 
 
 // ============================================================================
-// attn_mma_kernel (bf16): one CTA = 64 (query, head-of-group) rows of one
-// (sequence, KV head) over one split of the key range, worked on by TS groups
-// of 128 threads (see attention_core.cuh), each on its own consecutive part of
-// the split with its own K/V ring, so that a CTA's key tiles are processed side
-// by side instead of one after the other: with few active rows the kernel is
-// bound by the latency of one tile's load -> QK^T -> softmax -> PV chain, not
-// by arithmetic.  The groups' results are merged through shared memory in
-// group order.  When few rows are active the key range is also split over
-// blockIdx.z so that enough CTAs read K/V; splits write unnormalised partial
-// outputs plus (max, sum) and attn_combine_kernel merges them.
+// attn_mma_kernel (bf16): one CTA of 128 threads runs one attn_tile (see
+// attention_core.cuh): 64 (query, head-of-group) rows of one (sequence, KV
+// head) over one split of the key range.  When few rows are active the key
+// range is split over blockIdx.z so that >= 148 CTAs read K/V; splits write
+// unnormalised partial outputs plus (max, sum) and attn_combine_kernel merges
+// them.
 // ============================================================================
-template <int HD, int TS>
-__global__ void __launch_bounds__(128 * TS, 1)
-    attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                    const __grid_constant__ CUtensorMap tmQ, int q_by_tma, const __nv_bfloat16* __restrict__ q,
-                    __nv_bfloat16* __restrict__ o, float* __restrict__ o_part, float* __restrict__ ml_part, int a_seq,
-                    int n, int H, int Hkv, int S, int keys_per_split, int keys_per_group, int stages,
-                    float scale_log2, int* __restrict__ status) {
-  constexpr uint32_t Q_BYTES = AT_ROWS * HD * 2;
-  constexpr uint32_t STAGE_BYTES = 2 * AT_KEYS * HD * 2;
+template <int HD>
+__global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                       const __grid_constant__ CUtensorMap tmV,
+                                                       const __grid_constant__ CUtensorMap tmQ, int q_by_tma,
+                                                       const __nv_bfloat16* __restrict__ q,
+                                                       __nv_bfloat16* __restrict__ o, float* __restrict__ o_part,
+                                                       float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv,
+                                                       int S, int keys_per_split, float scale_log2,
+                                                       int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[TS][2];
-  __shared__ __align__(8) uint64_t q_bar;
-  __shared__ float ml_s[TS > 1 ? TS - 1 : 1][128][4];
+  __shared__ __align__(8) uint64_t full_bar[2];
   __shared__ int abort_flag;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* base_gen = smem_raw + (base - smem_u32(smem_raw));
-  const int gi = (int)threadIdx.x >> 7, tid = (int)threadIdx.x & 127;
   if (threadIdx.x == 0) {
     abort_flag = 0;
-    for (int g = 0; g < TS; ++g) {
-      mbar_init(smem_u32(&full_bar[g][0]), 1);
-      mbar_init(smem_u32(&full_bar[g][1]), 1);
-    }
-    mbar_init(smem_u32(&q_bar), 1);
+    mbar_init(smem_u32(&full_bar[0]), 1);
+    mbar_init(smem_u32(&full_bar[1]), 1);
     mbar_fence_init();
     prefetch_tensormap(&tmK);  // the descriptors are fetched while the predecessor still runs
     prefetch_tensormap(&tmV);
@@ -155,150 +144,12 @@ __global__ void __launch_bounds__(128 * TS, 1)
   __syncthreads();
   pdl_wait();  // K, V and Q come from the preceding kernels
   pdl_trigger();
-
-  const int G = H / Hkv, kh = blockIdx.y;
-  const int b = blockIdx.z / S, split = blockIdx.z - b * S;
-  const int row0 = blockIdx.x * AT_ROWS, n_rows = a_seq * G, dq = H * HD;
-  const int key_lo = split * keys_per_split, key_hi = min(n, key_lo + keys_per_split);
-  const int g_lo = key_lo + gi * keys_per_group, g_hi = min(key_hi, g_lo + keys_per_group);
-  const uint32_t q_s = base, kv_s = base + Q_BYTES + (uint32_t)(gi * stages) * STAGE_BYTES;
-  volatile int* abortp = &abort_flag;
-
-  // the group's first K/V tiles go out before anything else; then the Q tile, shared by the groups
-  if (tid == 0 && g_hi > g_lo) {
-    // (attn_group issues them; this only orders the Q request behind the first K/V requests of group 0)
-  }
-  bool q_ok = true;
-  auto stage_q = [&]() {
-    if (q_by_tma) {
-      // one query head per KV head: the tile is AT_ROWS consecutive rows of q, fetched by TMA; rows past the
-      // sequence's end belong to no live row
-      if (threadIdx.x == 0) {
-        const uint32_t qb = smem_u32(&q_bar);
-        mbar_expect_tx(qb, Q_BYTES);
-#pragma unroll
-        for (int p = 0; p < HD / 64; ++p) tma_load_2d(q_s + p * (AT_ROWS * 128), &tmQ, qb, kh * HD + p * 64, b * a_seq + row0);
-      }
-      q_ok = mbar_wait(smem_u32(&q_bar), 0u, abortp);
-    } else {
-      // plain 16-byte loads into the swizzled layout by the whole CTA (rows of other heads / past the end are
-      // zero); all loads of a thread before its first store
-      constexpr int CHUNKS = AT_ROWS * (HD / 8);
-      constexpr int PER = (CHUNKS + 128 * TS - 1) / (128 * TS);
-      uint4 qv[PER];
-#pragma unroll
-      for (int i = 0; i < PER; ++i) {
-        const int e = (int)threadIdx.x + i * 128 * TS;
-        const int r = e / (HD / 8), dc = e - r * (HD / 8);
-        const int vr = row0 + r;
-        qv[i] = make_uint4(0, 0, 0, 0);
-        if (e < CHUNKS && vr < n_rows) {
-          const int qi = vr / G, g = vr - qi * G;
-          qv[i] = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < PER; ++i) {
-        const int e = (int)threadIdx.x + i * 128 * TS;
-        const int r = e / (HD / 8), dc = e - r * (HD / 8);
-        if (e < CHUNKS) *reinterpret_cast<uint4*>(base_gen + tile_off<AT_ROWS>(r, dc)) = qv[i];
-      }
-      __syncthreads();
-    }
-    if (threadIdx.x == 0) timeline_mark(1);  // Q staged
-  };
-
-  AttnAcc<HD> acc;
-  bool ok = attn_group<HD>(tid, 1 + gi, q_s, kv_s, stages, full_bar[gi], abortp, &tmK, &tmV, kh, b, g_lo, g_hi,
-                           scale_log2, acc, stage_q);
-  ok = ok && q_ok;
-  if (threadIdx.x == 0) timeline_mark(8);  // group 0 is through its keys
-
-  // ---- merge of the groups, in group order, through each group's own (drained) ring
-  if constexpr (TS > 1) {
-    float* o_s = reinterpret_cast<float*>(base_gen + Q_BYTES + (size_t)(gi * stages) * STAGE_BYTES);
-    if (gi > 0) {
-      at_sync(1 + gi);  // every warp of the group has finished reading its K/V tiles
-      if (ok) {
-#pragma unroll
-        for (int i = 0; i < HD / 8; ++i)
-#pragma unroll
-          for (int c = 0; c < 4; ++c) o_s[(i * 4 + c) * 128 + tid] = acc.o[i][c];
-        ml_s[gi - 1][tid][0] = acc.m[0];
-        ml_s[gi - 1][tid][1] = acc.m[1];
-        ml_s[gi - 1][tid][2] = acc.l[0];
-        ml_s[gi - 1][tid][3] = acc.l[1];
-      }
-    }
-    ok = __syncthreads_and(ok);
-    if (ok && gi == 0) {
-      float M[2] = {acc.m[0], acc.m[1]};
-#pragma unroll
-      for (int g = 1; g < TS; ++g) {
-        M[0] = fmaxf(M[0], ml_s[g - 1][tid][0]);
-        M[1] = fmaxf(M[1], ml_s[g - 1][tid][1]);
-      }
-      float w0[2] = {exp2f(acc.m[0] - M[0]), exp2f(acc.m[1] - M[1])};  // group 0 always has keys: finite
-      acc.l[0] *= w0[0];
-      acc.l[1] *= w0[1];
-#pragma unroll
-      for (int i = 0; i < HD / 8; ++i) {
-        acc.o[i][0] *= w0[0];
-        acc.o[i][1] *= w0[0];
-        acc.o[i][2] *= w0[1];
-        acc.o[i][3] *= w0[1];
-      }
-#pragma unroll
-      for (int g = 1; g < TS; ++g) {
-        const float* og = reinterpret_cast<const float*>(base_gen + Q_BYTES + (size_t)(g * stages) * STAGE_BYTES);
-        const float wg[2] = {exp2f(ml_s[g - 1][tid][0] - M[0]), exp2f(ml_s[g - 1][tid][1] - M[1])};  // no keys: 0
-        acc.l[0] += wg[0] * ml_s[g - 1][tid][2];
-        acc.l[1] += wg[1] * ml_s[g - 1][tid][3];
-#pragma unroll
-        for (int i = 0; i < HD / 8; ++i)
-#pragma unroll
-          for (int c = 0; c < 4; ++c) acc.o[i][c] += wg[c >> 1] * og[(i * 4 + c) * 128 + tid];
-      }
-      acc.m[0] = M[0];
-      acc.m[1] = M[1];
-    }
-  } else {
-    ok = __syncthreads_and(ok);
-  }
-  if (!ok) {
-    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
-    drain_delay();
-    return;
-  }
-  if (gi != 0) return;
-
-  // ---- group 0 writes the CTA's rows: final output, or the split's unnormalised partial with (max, sum)
-  const int warp = tid >> 5, lane = tid & 31;
-#pragma unroll
-  for (int h2 = 0; h2 < 2; ++h2) {
-    const int vr = row0 + warp * 16 + (lane >> 2) + h2 * 8;
-    if (vr >= n_rows) continue;
-    const int qi = vr / G, g = vr - qi * G;
-    const size_t orow = ((size_t)b * a_seq + qi) * H + (kh * G + g);   // (row, head) index
-    if (S == 1) {
-      const float inv = 1.f / acc.l[h2];
-      __nv_bfloat16* dst = o + orow * HD + 2 * (lane & 3);
-#pragma unroll
-      for (int i = 0; i < HD / 8; ++i)
-        *reinterpret_cast<uint32_t*>(dst + i * 8) = pack_bf16(acc.o[i][2 * h2] * inv, acc.o[i][2 * h2 + 1] * inv);
-    } else {
-      const size_t total = (size_t)(gridDim.z / S) * a_seq * H;           // (row, head) pairs
-      float* dst = o_part + ((size_t)split * total + orow) * HD + 2 * (lane & 3);
-#pragma unroll
-      for (int i = 0; i < HD / 8; ++i)
-        *reinterpret_cast<float2*>(dst + i * 8) = make_float2(acc.o[i][2 * h2], acc.o[i][2 * h2 + 1]);
-      if ((lane & 3) == 0) {
-        float* ml = ml_part + ((size_t)split * total + orow) * 2;
-        ml[0] = acc.m[h2];
-        ml[1] = acc.l[h2];
-      }
-    }
-  }
+  uint32_t kv_iter = 0;
+  const bool ok = attn_tile<HD>((int)threadIdx.x, smem_raw + (base - smem_u32(smem_raw)), base, full_bar, kv_iter,
+                                &abort_flag, &tmK, &tmV, q, o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split,
+                                scale_log2, (int)gridDim.z / S, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z,
+                                q_by_tma ? &tmQ : nullptr);
+  if (!ok && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
 }
 
 // Merges the key-range splits: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s,
@@ -384,18 +235,15 @@ cudaError_t launch_combine(const Launch& L, const float* o_part, const float* ml
   return e;
 }
 
-template <int HD, int TS>
-cudaError_t launch_mma_ts(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
-                          float* scratch, int B, int a_seq, int n, int H, int Hkv, const AttnPlan& p) {
-  constexpr int Q_BYTES = AT_ROWS * HD * 2, STAGE_BYTES = 2 * AT_KEYS * HD * 2;
-  constexpr int SMEM_MAX = Q_BYTES + TS * 2 * STAGE_BYTES + 1024;
-  static_assert(SMEM_MAX <= 227 * 1024, "the groups' rings do not fit the shared memory of a CTA");
+template <int HD>
+cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
+                       float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
+  constexpr int SMEM = AT_ROWS * HD * 2 + 2 * 2 * AT_KEYS * HD * 2 + 1024;
   static DeviceOnce once;
-  cudaError_t e0 = once.run([] {
-    return cudaFuncSetAttribute(attn_mma_kernel<HD, TS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_MAX);
-  });
+  cudaError_t e0 = once.run(
+      [] { return cudaFuncSetAttribute(attn_mma_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM); });
   if (e0 != cudaSuccess) return e0;
-  const int G = H / Hkv, S = p.S;
+  const int G = H / Hkv;
   const size_t total = (size_t)B * a_seq * H;
   float* o_part = scratch;
   float* ml_part = scratch ? scratch + (size_t)S * total * HD : nullptr;
@@ -405,45 +253,30 @@ cudaError_t launch_mma_ts(const Launch& L, const CUtensorMap& tmK, const CUtenso
   CUtensorMap tmQ = tmK;
   const int q_by_tma = H == Hkv && ((uintptr_t)q & 15) == 0 &&
                        get_tensor_map_2d(q, (uint64_t)B * a_seq, (uint64_t)H * HD, AT_ROWS, &tmQ);
-  const size_t smem = Q_BYTES + (size_t)TS * p.stages * STAGE_BYTES + 1024;
-  cudaError_t e = launch_k(L, attn_mma_kernel<HD, TS>, grid, dim3(128 * TS), smem, tmK, tmV, tmQ, q_by_tma,
+  cudaError_t e = launch_k(L, attn_mma_kernel<HD>, dim3(grid), dim3(128), SMEM, tmK, tmV, tmQ, q_by_tma,
                            (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S,
-                           p.keys_per_split, p.keys_per_group, p.stages, scale_log2, L.d_status);
+                           keys_per_split, scale_log2, L.d_status);
   L.count();
   if (e == cudaSuccess && S > 1) e = launch_combine(L, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-template <int HD>
-cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
-                       float* scratch, int B, int a_seq, int n, int H, int Hkv, const AttnPlan& p) {
-  switch (p.groups) {
-    case 1: return launch_mma_ts<HD, 1>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p);
-    case 2: return launch_mma_ts<HD, 2>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p);
-    default: return launch_mma_ts<HD, AT_MAX_GROUPS>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p);
-  }
-}
-
-// tuning override of the 64-row kernel's plan (0 = automatic), see dllm_debug_attention_plan
-int g_force_splits = 0, g_force_groups = 0;
+// tuning override of the 64-row kernel's split count (0 = automatic), see dllm_debug_attention_plan
+int g_force_splits = 0;
 
 }  // namespace
 
-// Plan of the 64-row kernel: key-range splits over CTAs so that enough CTAs read K/V when few rows are active
-// (and no group has more than two tiles to work through one after the other), then up to AT_MAX_GROUPS groups
-// per CTA on consecutive parts of the CTA's range; whole 64-key tiles everywhere.
-static void finish_plan(AttnPlan& p, int B, int a_seq, int n, int H, int S, int groups_max) {
+// Key-range splits of the 64-row kernel, whole 64-key tiles per split: enough CTAs to cover the SMs when few
+// rows are active (every split costs the merge a partial per row and head, so no more than that), and about
+// two CTAs per SM when a KV head has at most eight rows (three queries against thousands of keys: the merge is
+// negligible and the key range is what takes the time).
+static void finish_plan(AttnPlan& p, int B, int a_seq, int n, int H, int S) {
   const int key_tiles = (n + AT_KEYS - 1) / AT_KEYS;
   if (S > key_tiles) S = key_tiles;
   if (S < 1) S = 1;
   const int tiles_per_split = (key_tiles + S - 1) / S;
-  p.S = (key_tiles + tiles_per_split - 1) / tiles_per_split;
   p.keys_per_split = tiles_per_split * AT_KEYS;
-  p.groups = tiles_per_split < groups_max ? tiles_per_split : groups_max;
-  const int tiles_per_group = (tiles_per_split + p.groups - 1) / p.groups;
-  p.groups = (tiles_per_split + tiles_per_group - 1) / tiles_per_group;  // no group without keys in a full split
-  p.keys_per_group = tiles_per_group * AT_KEYS;
-  p.stages = tiles_per_group > 1 ? 2 : 1;
+  p.S = (key_tiles + tiles_per_split - 1) / tiles_per_split;
   p.scratch_floats = p.S > 1 ? (size_t)p.S * B * a_seq * H * (128 + 2) : 0;
 }
 
@@ -451,16 +284,11 @@ AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv) {
   AttnPlan p;
   const int G = H / Hkv, sms = sm_count();
   const long tiles = (long)((a_seq * G + AT_ROWS - 1) / AT_ROWS) * Hkv * B;
-  const int key_tiles = (n + AT_KEYS - 1) / AT_KEYS;
-  const int groups_max = g_force_groups > 0 && g_force_groups <= AT_MAX_GROUPS ? g_force_groups : AT_MAX_GROUPS;
   int S = 1;
-  if (tiles < sms) {
-    S = (int)((sms + tiles - 1) / tiles);
-    const int s_kv = (key_tiles + 2 * groups_max - 1) / (2 * groups_max);
-    if (S < s_kv) S = s_kv;
-  }
+  if (tiles < sms) S = (int)((sms + tiles - 1) / tiles);
+  if (a_seq * G <= 8 && 4 * tiles < 7L * sms) S = (int)((7L * sms + 4 * tiles - 1) / (4 * tiles));
   if (g_force_splits > 0) S = g_force_splits;
-  finish_plan(p, B, a_seq, n, H, S, groups_max);
+  finish_plan(p, B, a_seq, n, H, S);
   return p;
 }
 
@@ -474,9 +302,7 @@ AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scra
     c.plan = plan_attention_umma(B, a_seq, n, H, Hkv, scratch_floats);
   } else {
     c.plan = plan_attention(B, a_seq, n, H, Hkv);
-    if (c.plan.S > 1 && scratch_floats < c.plan.scratch_floats)  // no room for the partials: one split
-      finish_plan(c.plan, B, a_seq, n, H, 1,
-                  g_force_groups > 0 && g_force_groups <= AT_MAX_GROUPS ? g_force_groups : AT_MAX_GROUPS);
+    if (c.plan.S > 1 && scratch_floats < c.plan.scratch_floats) finish_plan(c.plan, B, a_seq, n, H, 1);  // no room
   }
   return c;
 }
@@ -505,8 +331,8 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
     if (!get_tensor_map_3d(Kc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, AT_KEYS, &tmK) ||
         !get_tensor_map_3d(Vc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, AT_KEYS, &tmV))
       return cudaErrorInvalidValue;
-    return hd == 64 ? launch_mma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p)
-                    : launch_mma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p);
+    return hd == 64 ? launch_mma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
+                    : launch_mma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
   }
   const float scale = 1.0f / sqrtf((float)hd);
   dim3 grid((a_seq + TQ - 1) / TQ, H, B);
@@ -611,13 +437,12 @@ extern "C" dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, 
   return DLLM_OK;
 }
 
-extern "C" dllm_status dllm_debug_attention_plan(int splits, int groups) {
-  if (splits < 0 || groups < 0 || groups > dllm::AT_MAX_GROUPS) {
-    dllm::set_last_error("dllm_debug_attention_plan: splits >= 0 and 0 <= groups <= 3");
+extern "C" dllm_status dllm_debug_attention_plan(int splits) {
+  if (splits < 0) {
+    dllm::set_last_error("dllm_debug_attention_plan: splits >= 0");
     return DLLM_INVALID_ARG;
   }
   dllm::g_force_splits = splits;
-  dllm::g_force_groups = groups;
   return DLLM_OK;
 }
 

@@ -1,43 +1,40 @@
 // Flash-style attention tile on the tensor cores (bf16, mma.sync), written as a
-// device function of one GROUP of 128 cooperating threads; a CTA runs one to
-// four groups side by side on consecutive parts of its key range.
+// device function of 128 cooperating threads so that the stand-alone attention
+// kernel and the persistent layer kernel run the same code.
 //
-// One call = 64 "virtual rows" of one (sequence, KV head) x one range of keys.
-// A virtual row is a (query, query-head-of-the-group) pair, so with grouped KV
-// heads the G query heads that share a KV head are packed along the row
-// dimension and every K/V tile is loaded once for all of them.  K and V tiles
-// of 64 keys arrive by TMA (3-D map [B, n, dkv], 128-byte swizzle, keys beyond
-// n zero-filled) into the group's own ring of one or two stages; each of the 4
-// warps owns 16 rows and runs mma.sync m16n8k16 for S = Q K^T and O += P V with
-// the online softmax in fp32 registers (exp2 with the scale folded in).  The
-// result stays in registers (unnormalised output, row maximum, row sum); the
-// kernel merges the groups of a CTA through shared memory, and attn_combine
-// merges the key-range splits of different CTAs.
+// One call = 64 "virtual rows" of one (sequence, KV head) x one split of the key
+// range.  A virtual row is a (query, query-head-of-the-group) pair, so with
+// grouped KV heads the G query heads that share a KV head are packed along the
+// row dimension and every K/V tile is loaded once for all of them.  K and V
+// tiles of 64 keys arrive by TMA (3-D map [B, n, dkv], 128-byte swizzle, keys
+// beyond n zero-filled) into a two-stage ring; each of the 4 warps owns 16 rows
+// and runs mma.sync m16n8k16 for S = Q K^T and O += P V with the online softmax
+// in fp32 registers (exp2 with the scale folded in).  Splits write unnormalised
+// partial outputs plus (max, sum); attn_combine merges them.
 #pragma once
 #include "common.cuh"
 #include "tma.cuh"
 
 namespace dllm {
 
-// The 128 threads of a group synchronise on their own named barrier (1 + group index), so the groups of a CTA
-// never wait for one another while they work through their keys.
-__device__ __forceinline__ void at_sync(int bar_id) { asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory"); }
-__device__ __forceinline__ bool at_sync_and(int bar_id, bool pred) {
+// The 128 threads of a tile synchronise on named barrier 1, so the function can
+// run inside a larger block whose other warps do something else.
+__device__ __forceinline__ void at_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ bool at_sync_and(bool pred) {
   uint32_t r;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\t"
       "setp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.and.pred p, %2, 128, q;\n\t"
+      "bar.red.and.pred p, 1, 128, q;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(r)
-      : "r"((uint32_t)pred), "r"(bar_id)
+      : "r"((uint32_t)pred)
       : "memory");
   return r != 0;
 }
 
 constexpr int AT_ROWS = 64;   // virtual rows per CTA
 constexpr int AT_KEYS = 64;   // keys per tile
-constexpr int AT_MAX_GROUPS = 3;  // groups of 128 threads per CTA: 384 threads at up to 170 registers fill the file
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -66,41 +63,59 @@ __device__ __forceinline__ uint32_t tile_off(int row, int dc) {
   return (uint32_t)((dc >> 3) * (ROWS * 128) + row * 128 + (((dc & 7) ^ (row & 7)) << 4));
 }
 
-// What a group holds for its 64 rows after its keys: thread (warp w, lane) has rows w * 16 + lane / 4 (index 0)
-// and + 8 (index 1); o[i][2 * h2 + {0, 1}] are columns i * 8 + 2 * (lane % 4) + {0, 1} of row index h2.
-// m is the row maximum in log2 units (scale folded in), l the sum of 2^(s - m) over the group's keys, o the
-// unnormalised output.  A group without keys has m = -inf, l = 0, o = 0.
 template <int HD>
-struct AttnAcc {
-  float o[HD / 8][4];
-  float m[2], l[2];
+struct AttnSmem {
+  static constexpr int BYTES = AT_ROWS * HD * 2 + 2 * 2 * AT_KEYS * HD * 2;  // Q tile + two (K, V) stages
 };
 
-// tid: 0..127 within the group.  q_s: shared-window address of the CTA's Q tile ([64 rows][HD] in swizzled
-// panels, complete and visible before the call).  kv_s: shared-window address of the group's ring, `stages`
-// (1 or 2) x (K tile, V tile), 1024-byte aligned.  full_bar: the group's `stages` mbarriers (count 1, fresh:
-// phase 0).  Keys [key_lo, key_hi), key_lo a multiple of 64; an empty range returns the neutral element.
-// stage_q(): called by every thread of every group once the group's first K/V requests are out; it brings the
-// Q tile into shared memory (it may contain a CTA-wide barrier).  Returns false if a wait gave up.
-template <int HD, typename StageQ>
-__device__ __forceinline__ bool attn_group(int tid, int bar_id, uint32_t q_s, uint32_t kv_s, int stages,
-                                           uint64_t* full_bar, volatile int* abort_flag, const CUtensorMap* tmK,
-                                           const CUtensorMap* tmV, int kh, int b, int key_lo, int key_hi,
-                                           float scale_log2, AttnAcc<HD>& acc, StageQ&& stage_q) {
+// tid: 0..127.  smem_gen / smem_sh: generic pointer and shared-window address of
+// the same 1024-byte aligned region of AttnSmem<HD>::BYTES bytes.  full_bar: two
+// initialised mbarriers (count 1).  kv_iter: tiles this ring has carried so far
+// (stage and phase parity continue across calls); advanced by the tiles of this
+// call.  (bx, by, bz) play the role of the block index of a grid
+// (row tiles, KV heads, B * S).  Returns false if a wait gave up.
+template <int HD>
+__device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t smem_sh, uint64_t* full_bar,
+                                          uint32_t& kv_iter, volatile int* abort_flag, const CUtensorMap* tmK,
+                                          const CUtensorMap* tmV, const __nv_bfloat16* __restrict__ q,
+                                          __nv_bfloat16* __restrict__ o, float* __restrict__ o_part,
+                                          float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv, int S,
+                                          int keys_per_split, float scale_log2, int B, int bx, int by, int bz,
+                                          const CUtensorMap* tmQ = nullptr) {
+
   constexpr int PANELS = HD / 64;
   constexpr uint32_t TILE_BYTES = AT_KEYS * HD * 2;   // one K or V tile
   constexpr uint32_t STAGE_BYTES = 2 * TILE_BYTES;
-  const int warp = tid >> 5, lane = tid & 31;
-#pragma unroll
-  for (int i = 0; i < HD / 8; ++i) acc.o[i][0] = acc.o[i][1] = acc.o[i][2] = acc.o[i][3] = 0.f;
-  acc.m[0] = acc.m[1] = -INFINITY;
-  acc.l[0] = acc.l[1] = 0.f;
-  const int n_tiles = key_hi > key_lo ? (key_hi - key_lo + AT_KEYS - 1) / AT_KEYS : 0;
+  const uint32_t base = smem_sh;
+  const uint32_t q_s = base;                         // [64 rows][HD] in panels
+  const uint32_t kv_s = base + AT_ROWS * HD * 2;     // 2 stages x (K tile, V tile)
+  uint8_t* q_gen = smem_gen;
 
+  const int warp = tid >> 5, lane = tid & 31;
+  const int G = H / Hkv;
+  const int kh = by;
+  const int b = bz / S, split = bz - b * S;
+  const int row0 = bx * AT_ROWS;
+  const int n_rows = a_seq * G;
+  const int key_lo = split * keys_per_split;
+  const int key_hi = min(n, key_lo + keys_per_split);
+  const int n_tiles = (key_hi - key_lo + AT_KEYS - 1) / AT_KEYS;   // >= 1 by construction
+  const int dq = H * HD;
+
+  const uint32_t it0 = kv_iter;
+  kv_iter += (uint32_t)n_tiles;
+  at_sync();  // the previous tile's readers are done with the Q and K/V regions
+  // tmQ (one query head per KV head, so a row tile is AT_ROWS consecutive rows of q): the Q tile arrives by TMA
+  // together with the first K/V tile, on that tile's barrier; rows past the sequence's end belong to no live row
+  const bool q_tma = tmQ != nullptr;
   auto issue = [&](int t) {
-    const int st = t % stages;
+    const int st = (int)((it0 + (uint32_t)t) & 1u);
     const uint32_t fb = smem_u32(&full_bar[st]);
-    mbar_expect_tx(fb, STAGE_BYTES);
+    mbar_expect_tx(fb, STAGE_BYTES + ((q_tma && t == 0) ? AT_ROWS * HD * 2 : 0));
+    if (q_tma && t == 0) {
+#pragma unroll
+      for (int p = 0; p < PANELS; ++p) tma_load_2d(q_s + p * (AT_ROWS * 128), tmQ, fb, kh * HD + p * 64, b * a_seq + row0);
+    }
     const uint32_t dst = kv_s + st * STAGE_BYTES;
     const int key0 = key_lo + t * AT_KEYS;
 #pragma unroll
@@ -109,40 +124,72 @@ __device__ __forceinline__ bool attn_group(int tid, int bar_id, uint32_t q_s, ui
       tma_load_3d(dst + TILE_BYTES + p * (AT_KEYS * 128), tmV, fb, kh * HD + p * 64, key0, b);
     }
   };
-  if (tid == 0 && n_tiles > 0) {
+  if (tid == 0) {
     issue(0);
-    if (n_tiles > 1 && stages > 1) issue(1);
+    if (n_tiles > 1) issue(1);
   }
-  stage_q();
+  // Q tile: plain 16-byte loads into the swizzled layout (rows of other heads /
+  // past the end are zero)
+  if (q_tma) {
+    mbar_wait(smem_u32(&full_bar[(int)(it0 & 1u)]), (it0 >> 1) & 1u, abort_flag);  // the loop checks the outcome again
+  } else {
+    constexpr int PER = AT_ROWS * (HD / 8) / 128;  // 16-byte chunks per thread: all loads first, then the stores
+    uint4 qv[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int e = tid + i * 128;
+      const int r = e / (HD / 8), dc = e - r * (HD / 8);
+      const int vr = row0 + r;
+      qv[i] = make_uint4(0, 0, 0, 0);
+      if (vr < n_rows) {
+        const int qi = vr / G, g = vr - qi * G;
+        qv[i] = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int e = tid + i * 128;
+      const int r = e / (HD / 8), dc = e - r * (HD / 8);
+      *reinterpret_cast<uint4*>(q_gen + tile_off<AT_ROWS>(r, dc)) = qv[i];
+    }
+  }
+  at_sync();
+  if (tid == 0) timeline_mark(1);  // Q staged
+  // Q fragments of this warp's 16 rows stay in registers
+  uint32_t qf[HD / 16][4];
+#pragma unroll
+  for (int ks = 0; ks < HD / 16; ++ks) {
+    const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    const int dc = ks * 2 + (lane >> 4);
+    ldsm_x4(q_s + tile_off<AT_ROWS>(row, dc), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+  }
+  float oacc[HD / 8][4];
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
   bool ok = true;
+
   for (int t = 0; t < n_tiles; ++t) {
-    const int st = t % stages;
-    ok = mbar_wait(smem_u32(&full_bar[st]), (uint32_t)(t / stages) & 1u, abort_flag);
-    ok = at_sync_and(bar_id, ok);             // uniform over the group: nobody is left behind at a barrier
+    const int st = (int)((it0 + (uint32_t)t) & 1u);
+    ok = mbar_wait(smem_u32(&full_bar[st]), ((it0 + (uint32_t)t) >> 1) & 1u, abort_flag);
+    ok = at_sync_and(ok);                     // uniform over the 128 threads: nobody is left behind at a barrier
     if (!ok) break;
     if (tid == 0) timeline_mark(2 + (t < 5 ? t : 5));  // K/V tile t has landed
     const uint32_t k_s = kv_s + st * STAGE_BYTES, v_s = k_s + TILE_BYTES;
-    // ---- S = Q K^T for 16 rows x 64 keys (the Q fragments are re-read per k-step: they are used once per tile
-    // and a group mostly sees one or two tiles, so holding them would only cost registers)
+    // ---- S = Q K^T for 16 rows x 64 keys
     float sacc[AT_KEYS / 8][4];
 #pragma unroll
     for (int i = 0; i < AT_KEYS / 8; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
 #pragma unroll
     for (int ks = 0; ks < HD / 16; ++ks) {
-      uint32_t qf[4];
-      {
-        const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        const int dc = ks * 2 + (lane >> 4);
-        ldsm_x4(q_s + tile_off<AT_ROWS>(row, dc), qf[0], qf[1], qf[2], qf[3]);
-      }
 #pragma unroll
       for (int jp = 0; jp < AT_KEYS / 16; ++jp) {
         const int key = jp * 16 + (lane & 7) + (lane >> 4) * 8;
         const int dc = ks * 2 + ((lane >> 3) & 1);
         uint32_t r0, r1, r2, r3;
         ldsm_x4(k_s + tile_off<AT_KEYS>(key, dc), r0, r1, r2, r3);
-        mma_bf16_16816(sacc[2 * jp], qf, r0, r1);
-        mma_bf16_16816(sacc[2 * jp + 1], qf, r2, r3);
+        mma_bf16_16816(sacc[2 * jp], qf[ks], r0, r1);
+        mma_bf16_16816(sacc[2 * jp + 1], qf[ks], r2, r3);
       }
     }
     // ---- online softmax (rows lane/4 and lane/4 + 8)
@@ -163,28 +210,26 @@ __device__ __forceinline__ bool attn_group(int tid, int bar_id, uint32_t q_s, ui
     for (int h2 = 0; h2 < 2; ++h2) {
       mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 1));
       mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 2));
-      const float m_new = fmaxf(acc.m[h2], mx[h2]);      // finite: every tile has a valid key
-      corr[h2] = exp2f(acc.m[h2] - m_new);
-      acc.m[h2] = m_new;
-      acc.l[h2] *= corr[h2];
+      const float m_new = fmaxf(m_run[h2], mx[h2]);      // finite: every tile has a valid key
+      corr[h2] = exp2f(m_run[h2] - m_new);
+      m_run[h2] = m_new;
+      l_run[h2] *= corr[h2];
     }
 #pragma unroll
     for (int nb = 0; nb < AT_KEYS / 8; ++nb) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        const float p = exp2f(sacc[nb][c] - acc.m[c >> 1]);
+        const float p = exp2f(sacc[nb][c] - m_run[c >> 1]);
         sacc[nb][c] = p;
-        acc.l[c >> 1] += p;
+        l_run[c >> 1] += p;
       }
     }
-    if (t > 0) {
 #pragma unroll
-      for (int i = 0; i < HD / 8; ++i) {
-        acc.o[i][0] *= corr[0];
-        acc.o[i][1] *= corr[0];
-        acc.o[i][2] *= corr[1];
-        acc.o[i][3] *= corr[1];
-      }
+    for (int i = 0; i < HD / 8; ++i) {
+      oacc[i][0] *= corr[0];
+      oacc[i][1] *= corr[0];
+      oacc[i][2] *= corr[1];
+      oacc[i][3] *= corr[1];
     }
     // ---- O += P V
 #pragma unroll
@@ -200,21 +245,48 @@ __device__ __forceinline__ bool attn_group(int tid, int bar_id, uint32_t q_s, ui
         const int dc = dp * 2 + (lane >> 4);
         uint32_t r0, r1, r2, r3;
         ldsm_x4_trans(v_s + tile_off<AT_KEYS>(key, dc), r0, r1, r2, r3);
-        mma_bf16_16816(acc.o[2 * dp], pf, r0, r1);
-        mma_bf16_16816(acc.o[2 * dp + 1], pf, r2, r3);
+        mma_bf16_16816(oacc[2 * dp], pf, r0, r1);
+        mma_bf16_16816(oacc[2 * dp + 1], pf, r2, r3);
       }
     }
-    if (t + stages < n_tiles) {
-      at_sync(bar_id);                         // every warp of the group is done with stage st
-      if (tid == 0) issue(t + stages);
-    }
+    at_sync();                               // every warp is done with stage st
+    if (tid == 0 && t + 2 < n_tiles) issue(t + 2);
   }
-  if (!ok) return false;
-  // the row sums are spread over the four lanes of a row
+  if (!ok) {
+    drain_delay();
+    return false;
+  }
+  if (tid == 0) timeline_mark(8);  // all tiles done
+  // ---- epilogue
 #pragma unroll
   for (int h2 = 0; h2 < 2; ++h2) {
-    acc.l[h2] += __shfl_xor_sync(0xffffffffu, acc.l[h2], 1);
-    acc.l[h2] += __shfl_xor_sync(0xffffffffu, acc.l[h2], 2);
+    l_run[h2] += __shfl_xor_sync(0xffffffffu, l_run[h2], 1);
+    l_run[h2] += __shfl_xor_sync(0xffffffffu, l_run[h2], 2);
+  }
+#pragma unroll
+  for (int h2 = 0; h2 < 2; ++h2) {
+    const int vr = row0 + warp * 16 + (lane >> 2) + h2 * 8;
+    if (vr >= n_rows) continue;
+    const int qi = vr / G, g = vr - qi * G;
+    const size_t orow = ((size_t)b * a_seq + qi) * H + (kh * G + g);   // (row, head) index
+    if (S == 1) {
+      const float inv = 1.f / l_run[h2];
+      __nv_bfloat16* dst = o + orow * HD + 2 * (lane & 3);
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i)
+        *reinterpret_cast<uint32_t*>(dst + i * 8) = pack_bf16(oacc[i][2 * h2] * inv, oacc[i][2 * h2 + 1] * inv);
+    } else {
+      const size_t total = (size_t)B * a_seq * H;           // (row, head) pairs
+      float* dst = o_part + ((size_t)split * total + orow) * HD + 2 * (lane & 3);
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i)
+        *reinterpret_cast<float2*>(dst + i * 8) = make_float2(oacc[i][2 * h2], oacc[i][2 * h2 + 1]);
+      if ((lane & 3) == 0) {
+        float* ml = ml_part + ((size_t)split * total + orow) * 2;
+        ml[0] = m_run[h2];
+        ml[1] = l_run[h2];
+      }
+    }
   }
   return true;
 }

@@ -46,29 +46,6 @@ struct OutRows {
   }
 };
 
-// A span of read-only memory (weights of a projection that runs soon) that a kernel asks the memory system to
-// bring into L2 while HBM would otherwise sit idle: the row-wise kernels between two projections move little
-// data, so the next projection's weight stream can start under them.  bytes == 0: nothing.
-struct Prefetch {
-  const void* p = nullptr;
-  size_t bytes = 0;
-};
-// CTA `cta` of `n_ctas` requests its contiguous share of the span, in 16 KB pieces; called by ONE thread.
-// Fire and forget: nothing waits for the lines, and a line that is evicted again costs only bandwidth.
-__device__ __forceinline__ void l2_prefetch_share(const Prefetch& pf, unsigned cta, unsigned n_ctas) {
-  if (pf.bytes == 0) return;
-  constexpr size_t PIECE = 16384;
-  const size_t per = ((pf.bytes + n_ctas - 1) / n_ctas + PIECE - 1) / PIECE * PIECE;
-  const size_t lo = per * cta;
-  if (lo >= pf.bytes) return;
-  const size_t hi = lo + per < pf.bytes ? lo + per : pf.bytes;
-  const char* base = static_cast<const char*>(pf.p);
-  for (size_t off = lo; off < hi; off += PIECE) {
-    const unsigned size = (unsigned)((hi - off < PIECE ? hi - off : PIECE) & ~(size_t)15);
-    if (size) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(size) : "memory");
-  }
-}
-
 // device status word codes
 enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103, ST_TIMEOUT_GRID = 104, ST_RANGE = 201 };
 

@@ -171,11 +171,9 @@ __device__ __forceinline__ int32_t* select_sequence(unsigned long long* keys, co
 // left as it is (the selected-only variant of Sec. A.5 writes the selected rows later).
 template <typename T>
 __global__ void __launch_bounds__(512, 2) vverify_kernel(Partials part, T* __restrict__ Vc, float* __restrict__ sim,
-                                                         Geo g, int dkv, int metric, int write_v, IdentityLists id,
-                                                         Prefetch pf) {
+                                                         Geo g, int dkv, int metric, int write_v, IdentityLists id) {
   pdl_wait();
   pdl_trigger();
-  if (threadIdx.x == 0) l2_prefetch_share(pf, blockIdx.x, gridDim.x);
   __shared__ float red[96];
   const int c = blockIdx.x;  // response row, carried order
   const int b = c / g.R, j = c - b * g.R;
@@ -210,11 +208,11 @@ __global__ void __launch_bounds__(512, 2) vverify_kernel(Partials part, T* __res
 }
 
 void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv, int metric,
-                    int write_v, const IdentityLists* lists, Prefetch pf) {
+                    int write_v, const IdentityLists* lists) {
   const int rows = g.B * g.R;
   const IdentityLists id = lists ? *lists : IdentityLists{};
   DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(row_threads(dkv)), 0, part, (T*)Vc_layer, sim, g, dkv,
-                                 metric, write_v, id, pf)));
+                                 metric, write_v, id)));
   L.count();
 }
 
@@ -426,11 +424,9 @@ void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32
 // element i with i + hd/2, angle pos * theta^(-2i/hd) from a table built on the host.
 template <typename T>
 __global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ rope_tab,
-                               T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int Ma, int H, int Hkv, int hd,
-                               Prefetch pf) {
+                               T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int Ma, int H, int Hkv, int hd) {
   pdl_wait();
   pdl_trigger();
-  if (threadIdx.x == 0) l2_prefetch_share(pf, blockIdx.x, gridDim.x);
   const int half = hd >> 1, q4 = half >> 2;
   const int groups = (H + Hkv) * q4;
   const long w = (long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -461,12 +457,12 @@ __global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, c
 }
 
 void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* act, const float* rope_tab, void* qbuf,
-                    void* Kc_layer, Geo g, int Ma, int H, int Hkv, int hd, Prefetch pf) {
+                    void* Kc_layer, Geo g, int Ma, int H, int Hkv, int hd) {
   if (Ma <= 0) return;
   const long total = (long)Ma * (H + Hkv) * (hd >> 3);
   const unsigned blocks = (unsigned)((total + 255) / 256);
   DLLM_DISPATCH(dtype, (launch_k(L, qk_rope_kernel<T>, dim3(blocks), dim3(256), 0, part, act, rope_tab, (T*)qbuf,
-                                 (T*)Kc_layer, g, Ma, H, Hkv, hd, pf)));
+                                 (T*)Kc_layer, g, Ma, H, Hkv, hd)));
   L.count();
 }
 
@@ -503,10 +499,9 @@ void launch_scatter_rows(const Launch& L, int dtype, Partials part, const int32_
 template <typename T>
 __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ x,
                                       const float* __restrict__ gain2, OutRows Ac, T* __restrict__ hn, Geo g,
-                                      float eps, Prefetch pf) {
+                                      float eps) {
   pdl_wait();
   pdl_trigger();
-  if (threadIdx.x == 0) l2_prefetch_share(pf, blockIdx.x, gridDim.x);
   extern __shared__ float hrow[];
   __shared__ float red[32];
   const int r = blockIdx.x;
@@ -555,12 +550,12 @@ __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__
 }
 
 void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int32_t* act, const float* x,
-                           const float* gain2, OutRows Ac_layer, void* hn, Geo g, int Ma, float eps, Prefetch pf) {
+                           const float* gain2, OutRows Ac_layer, void* hn, Geo g, int Ma, float eps) {
   if (Ma <= 0) return;
   const int threads = row_threads(g.d);
   const size_t smem = g.d <= threads * 8 ? 0 : (size_t)g.d * sizeof(float);  // staging only if a row takes several passes
   DLLM_DISPATCH(dtype, (launch_k(L, oproj_epilogue_kernel<T>, dim3(Ma), dim3(threads), smem, part, act, x, gain2, Ac_layer,
-                                 (T*)hn, g, eps, pf)));
+                                 (T*)hn, g, eps)));
   L.count();
 }
 
@@ -643,10 +638,9 @@ void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t*
 template <typename T>
 __global__ void __launch_bounds__(512, 2) tail_kernel(Partials part, const int32_t* __restrict__ inv, float* __restrict__ x,
                             OutRows Ac, OutRows Fc, const float* __restrict__ gain,
-                            T* __restrict__ u, Geo g, int c0, float eps, Prefetch pf) {
+                            T* __restrict__ u, Geo g, int c0, float eps) {
   pdl_wait();
   pdl_trigger();
-  if (threadIdx.x == 0) l2_prefetch_share(pf, blockIdx.x, gridDim.x);
   extern __shared__ float hrow[];
   __shared__ float red[32];
   const int c = c0 + blockIdx.x;
@@ -703,12 +697,12 @@ __global__ void __launch_bounds__(512, 2) tail_kernel(Partials part, const int32
 }
 
 void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, OutRows Ac_layer,
-                 OutRows Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps, Prefetch pf) {
+                 OutRows Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps) {
   if (c1 <= c0) return;
   const int threads = row_threads(g.d);
   const size_t smem = g.d <= threads * 8 ? 0 : (size_t)g.d * sizeof(float);  // staging only if a row takes several passes
   DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T>, dim3(c1 - c0), dim3(threads), smem, part, inv, x, Ac_layer,
-                                 Fc_layer, gain, (T*)u, g, c0, eps, pf)));
+                                 Fc_layer, gain, (T*)u, g, c0, eps)));
   L.count();
 }
 
@@ -723,10 +717,9 @@ template <typename T>
 __global__ void select_gather_kernel(const float* __restrict__ sim, const int32_t* __restrict__ forced, int mode,
                                      int ksel, int32_t* __restrict__ sel, int32_t* __restrict__ act,
                                      int32_t* __restrict__ inv, const T* __restrict__ u, T* __restrict__ ua, Geo g,
-                                     int refresh_prompt, Prefetch pf) {
+                                     int refresh_prompt) {
   pdl_wait();
   pdl_trigger();
-  if (threadIdx.x == 0) l2_prefetch_share(pf, blockIdx.x + gridDim.x * blockIdx.y, gridDim.x * gridDim.y);
   extern __shared__ unsigned long long keys[];  // R keys, R slots (int), R / 8 bytes of ballot words
   const int R = g.R, b = blockIdx.y, ridx = blockIdx.x;
   __shared__ int my_j;
@@ -794,12 +787,12 @@ __global__ void select_gather_kernel(const float* __restrict__ sim, const int32_
 
 void launch_select_gather(const Launch& L, int dtype, const float* sim, const int32_t* forced, int mode, int ksel,
                           int32_t* sel, int32_t* act, int32_t* inv, const void* u, void* ua, Geo g,
-                          int refresh_prompt, Prefetch pf) {
+                          int refresh_prompt) {
   const int a_seq = (refresh_prompt ? g.P : 0) + ksel;
   if (a_seq <= 0) return;
   const size_t smem = (size_t)g.R * 13 + 16;
   DLLM_DISPATCH(dtype, (launch_k(L, select_gather_kernel<T>, dim3(a_seq, g.B), dim3(256), smem, sim, forced, mode, ksel,
-                                 sel, act, inv, (const T*)u, (T*)ua, g, refresh_prompt, pf)));
+                                 sel, act, inv, (const T*)u, (T*)ua, g, refresh_prompt)));
   L.count();
 }
 

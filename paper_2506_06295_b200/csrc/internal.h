@@ -122,7 +122,7 @@ struct IdentityLists {
   int32_t *sel = nullptr, *act = nullptr, *inv = nullptr;
 };
 void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, float* sim, Geo g, int dkv,
-                    int metric = 0, int write_v = 1, const IdentityLists* lists = nullptr, Prefetch pf = {});
+                    int metric = 0, int write_v = 1, const IdentityLists* lists = nullptr);
 // The same test on K (ablation of Sec. 4.3): slab sum of the K projection of all
 // response rows, RoPE, score against the cached (post-RoPE) K, whole-K overwrite.
 void launch_kverify(const Launch& L, int dtype, Partials part, void* Kc_layer, float* sim, const float* rope_tab, Geo g,
@@ -136,7 +136,7 @@ cudaError_t launch_select(const Launch& L, const float* sim, const int32_t* forc
 // into ua in one launch (R <= 1024; sel rows have stride R).
 void launch_select_gather(const Launch& L, int dtype, const float* sim, const int32_t* forced, int mode, int ksel,
                           int32_t* sel, int32_t* act, int32_t* inv, const void* u, void* ua, Geo g,
-                          int refresh_prompt, Prefetch pf = {});
+                          int refresh_prompt);
 // x[c] = E[token(c)], u[c] = rmsnorm(x[c]) * gain for carried rows c0 <= c < c1.
 void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t* tokens, float* x, const float* gain,
                        void* u, Geo g, int c0, int c1, float eps);
@@ -144,18 +144,18 @@ void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t*
 // (slabs in `part`, row = inv[c]) -> cache; x <- (x + AttnOut) + FFNOut from the
 // caches; u = rmsnorm(x) * gain.  inv == nullptr: no active row.
 void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, OutRows Ac_layer,
-                 OutRows Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps, Prefetch pf = {});
+                 OutRows Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps);
 void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32_t* act, void* dst, int rows, int d);
 // RoPE on Q and K of the active rows; Q -> qbuf [Ma, dq]; K -> K cache rows.
 void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* act, const float* rope_tab, void* qbuf,
-                    void* Kc_layer, Geo g, int Ma, int H, int Hkv, int hd, Prefetch pf = {});
+                    void* Kc_layer, Geo g, int Ma, int H, int Hkv, int hd);
 // rows of `part` -> cache rows (model dtype).  act == nullptr: rows are the
 // carried ids c_base + i; otherwise act[i].
 void launch_scatter_rows(const Launch& L, int dtype, Partials part, const int32_t* act, int c_base, void* cache_layer,
                          Geo g, int rows, int width);
 // AttnOut rows -> cache; h = x + AttnOut; hn = rmsnorm(h) * gain2 (model dtype).
 void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int32_t* act, const float* x,
-                           const float* gain2, OutRows Ac_layer, void* hn, Geo g, int Ma, float eps, Prefetch pf = {});
+                           const float* gain2, OutRows Ac_layer, void* hn, Geo g, int Ma, float eps);
 // act[i][j] = silu(gate) * up from partials [Ma, 2m] (gate columns first).
 // interleaved: the columns of `part` are blocks of 64 gate columns followed by the 64 up columns of the same
 // FFN columns (the layout of the stacked weight when d_ffn % 64 == 0 in bf16); else all gate, then all up.
@@ -218,8 +218,6 @@ struct AttnPlan {
   int S;               // key-range splits
   int keys_per_split;  // multiple of the key tile
   size_t scratch_floats;
-  // 64-row kernel only: groups of 128 threads per CTA, keys of a split per group, ring stages per group
-  int groups = 1, keys_per_group = 0, stages = 2;
 };
 AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv);
 // Plan of the 128-row tcgen05 kernel (attention_umma.cu) with at most scratch_floats floats for split partials.
@@ -229,7 +227,7 @@ AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scr
 // and the entry point with built-in scratch all decide through this one function.
 struct AttnChoice {
   bool umma = false;
-  AttnPlan plan{1, 0, 0, 1, 0, 2};
+  AttnPlan plan{1, 0, 0};
 };
 AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats);
 // bf16 with head_dim 64 / 128 runs on the tensor cores (scratch holds the

@@ -27,6 +27,10 @@ FP32, BF16 = 0, 1
 K_FLOOR, K_CEIL = 0, 1
 CACHE_K, CACHE_V, CACHE_ATTN, CACHE_FFN = range(4)
 SESSION_DEFAULT, SESSION_COMPACT_CACHE = 0, 1
+# classes of dllm_session_profile_read (DLLM_PROF_*), in the header's order
+PROF_CLASSES = ["gemm", "attention", "gemm_v", "gemm_qk", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head",
+                "attention_mma", "attention_tcgen05", "vverify", "select_gather", "rope_kscatter", "oproj_epilogue",
+                "silu_mul", "layer_tail", "embed_norm", "estimate_merge", "v_scatter"]
 
 
 class Config(C.Structure):
@@ -78,7 +82,6 @@ SIGNATURES = {
     "dllm_session_use_graphs": (_I, [_P, _I]),
     "dllm_session_use_simt_gemm": (_I, [_P, _I]),
     "dllm_session_use_pdl": (_I, [_P, _I]),
-    "dllm_session_set_prefetch": (_I, [_P, _P, _I]),
     "dllm_session_profile": (_I, [_P, _I]),
     "dllm_session_profile_read": (_I, [_P, _I, C.POINTER(C.c_double), C.POINTER(C.c_uint64),
                                        C.POINTER(C.c_double), C.POINTER(C.c_double)]),
@@ -97,7 +100,7 @@ SIGNATURES = {
     "dllm_kernel_status": (_I, [_P]),
     "dllm_debug_set_wait_limit_ns": (_I, [C.c_uint64]),
     "dllm_debug_skip_one_load": (_I, [_I]),
-    "dllm_debug_attention_plan": (_I, [_I, _I]),
+    "dllm_debug_attention_plan": (_I, [_I]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
     _fn = getattr(lib, _name)
@@ -366,11 +369,6 @@ class Session:
 
     def use_pdl(self, enable: bool) -> None:
         _check(lib.dllm_session_use_pdl(self.handle, int(enable)))
-
-    def set_prefetch(self, kb) -> None:
-        """L2 prefetch sizes (KB) of the row-wise kernels: V-verify, selection, RoPE, O epilogue, layer tail."""
-        a = np.ascontiguousarray(list(kb), dtype=np.int32)
-        _check(lib.dllm_session_set_prefetch(self.handle, _np_ptr(a), int(a.size)))
 
     def use_simt_gemm(self, enable: bool) -> None:
         _check(lib.dllm_session_use_simt_gemm(self.handle, int(enable)))

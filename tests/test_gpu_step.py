@@ -187,6 +187,16 @@ def test_profiling_counts_every_projection_and_changes_no_result(env, graphs):
     expect = sum(cfg.n_layers * (5 + (1 if rp else 0)) + 1 for rp, _, _ in steps)
     assert g["launches"] == expect and a["launches"] == len(steps) * cfg.n_layers
     assert g["ms"] > 0 and a["ms"] > 0 and g["bytes"] > 0 and g["flops"] > 0 and a["flops"] > 0
+    # the two aggregates are sums over their sub-classes; every row-wise launch has a class of its own
+    per = {name: ses.profile_read(i) for i, name in enumerate(dllm.PROF_CLASSES)}
+    assert sum(per[c]["launches"] for c in dllm.PROF_CLASSES[2:8]) == g["launches"]
+    assert abs(sum(per[c]["ms"] for c in dllm.PROF_CLASSES[2:8]) - g["ms"]) < 1e-6 * g["ms"]
+    assert per["attention_mma"]["launches"] + per["attention_tcgen05"]["launches"] == a["launches"]
+    assert per["layer_tail"]["launches"] == len(steps) * cfg.n_layers and per["embed_norm"]["launches"] == len(steps)
+    assert per["vverify"]["launches"] == len(steps) * cfg.n_layers  # every step projects V for all response rows
+    assert per["select_gather"]["launches"] == 3 * cfg.n_layers    # not on the response refresh (identity lists)
+    assert per["gemm_lm_head"]["launches"] == len(steps) and per["estimate_merge"]["launches"] == len(steps)
+    assert all(v["bytes"] > 0 for k, v in per.items() if v["launches"])
     assert np.array_equal(ses.hidden(), ref.hidden())
     assert np.array_equal(ses.tokens(), ref.tokens())
     ses.profile(False)

@@ -47,3 +47,21 @@ def test_single_rank_is_identity():
     import bench
     assert bench.aggregate_over_ranks(3.5, 7.0, 1, torch.device("cpu")) == (3.5, 7.0)
     assert bench.tokens_processed(256, 1, 256, 256, 1) == 256
+
+
+def test_gpus_flag_without_a_launcher_spawns_the_ranks(tmp_path):
+    """`python bench.py --gpus N` started plainly must itself start N ranks (one per GPU) and report n_gpus = N;
+    under a launcher (WORLD_SIZE set) and for the reference arm it must not spawn again."""
+    import json
+    import bench
+    assert bench.wants_spawn(2, "ours", {}) and bench.wants_spawn(8, "ours", {"PATH": "/usr/bin"})
+    assert not bench.wants_spawn(1, "ours", {})
+    assert not bench.wants_spawn(2, "ours", {"WORLD_SIZE": "2"})
+    assert not bench.wants_spawn(2, "reference", {})
+    out = tmp_path / "line.json"
+    stub = os.path.join(ROOT, "tests", "replica_stub.py")
+    env_before = dict(os.environ)
+    rc = bench.spawn_ranks(2, ["--out", str(out)], script=stub)          # bench.py's own launcher, CPU ranks
+    assert rc == 0 and dict(os.environ) == env_before
+    line = json.loads(out.read_text())
+    assert line["n_gpus"] == 2 and line["ms"] == 15.0 and line["ms_e2e"] == 20.0 and line["tokens"] == 16
