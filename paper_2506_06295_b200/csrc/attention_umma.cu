@@ -3,26 +3,30 @@
 // non-causal attention of the active query rows over ALL n cached keys of
 // their sequence (Sec. A.7), grouped KV heads packed along the row dimension.
 //
-// One CTA (128 threads) = 128 "virtual rows" ((query, head-of-group) pairs) of
-// one (sequence, KV head) x one split of the key range, key tiles of 128:
-//   S = Q K^T        tcgen05.mma, M = 128 rows, N = 128 keys, contraction HD;
-//                    Q and K tiles in shared memory (K-major, 128-byte swizzle),
-//                    S in TMEM (128 lanes x 128 fp32 columns)
-//   softmax          TMEM lane = row, so every thread owns one row: it loads its
-//                    128 scores with tcgen05.ld, takes max / exp2 / sum locally
-//                    (no shuffles) and writes P as bf16 into shared memory in
-//                    the layout of an MMA A operand
-//   O += P V         tcgen05.mma, M = 128 rows, N = HD, contraction 128 keys;
-//                    V is used as stored ([key][hd], "MN-major" B operand); O
-//                    accumulates in TMEM and is rescaled (tcgen05.ld / st) only
-//                    when a row's maximum has grown by more than 2^8 since its
-//                    reference was set; the scores of tile t+1 are issued right
-//                    behind O += P V of tile t, so the tensor pipe works while
-//                    the threads are between barriers
-// K and V tiles arrive by TMA into a two-stage ring; tile t+2 is requested when
-// tile t has been consumed.  Key-range splits write unnormalised partials plus
-// (max, sum) exactly like the mma.sync kernel, and the same merge kernel
-// finishes them.  Every mbarrier wait is bounded.
+// One CTA = TWO tiles of 128 "virtual rows" ((query, head-of-group) pairs) of
+// one (sequence, KV head) x one split of the key range, key tiles of 64, ten
+// warps with fixed roles:
+//   warp 9           TMA: the Q tiles, then K/V tiles into a three-stage ring
+//   warp 8           issues every tcgen05.mma of the CTA
+//   warps 0-3, 4-7   the softmax group of row tile 0 resp. 1 (one row per thread)
+// Per key tile t and row tile i:
+//   S_i = Q_i K^T     tcgen05.mma, M = 128 rows, N = 64 keys, contraction HD; Q and
+//                     K in shared memory (K-major, 128-byte swizzle), S_i in TMEM
+//   softmax           TMEM lane = row, so every thread of group i owns one row: it
+//                     loads its 64 scores with tcgen05.ld, takes max / exp2 / sum
+//                     locally (no shuffles) and writes P_i as bf16 into shared
+//                     memory in the layout of an MMA A operand
+//   O_i += P_i V      tcgen05.mma, M = 128 rows, N = HD, contraction 64 keys; V is
+//                     used as stored ([key][hd], "MN-major" B operand); O_i
+//                     accumulates in TMEM and is rescaled (tcgen05.ld / st) only
+//                     when a row's maximum has grown by more than 2^8 since its
+//                     reference was set
+// The MMA warp issues O_i += P_i V of tile t and, right behind it, S_i of tile
+// t+1, alternating between the row tiles: while one group is in its softmax the
+// tensor pipe works for the other, and both row tiles read every K/V tile that
+// arrives once.  Key-range splits write unnormalised partials plus (max, sum)
+// exactly like the mma.sync kernel, and the same merge kernel finishes them.
+// Every mbarrier wait is bounded.
 #include "attention_core.cuh"
 #include "internal.h"
 #include "tma.cuh"
@@ -32,8 +36,11 @@ namespace dllm {
 
 namespace {
 
-constexpr int UA_ROWS = 128;  // virtual rows per CTA (UMMA M)
-constexpr int UA_KEYS = 128;  // keys per tile
+constexpr int UA_ROWS = 128;   // virtual rows per row tile (UMMA M); a CTA works on two row tiles
+constexpr int UA_TILES = 2;
+constexpr int UA_KEYS = 64;    // keys per tile
+constexpr int UA_STAGES = 3;   // K/V ring
+constexpr int UA_THREADS = 320;  // two softmax groups of 128, one MMA warp, one TMA warp
 
 // MN-major operand ([k][mn] rows of 64 mn-elements = 128 bytes, 128-byte swizzle,
 // panels of 64 mn-elements): lbo = bytes between panels along MN, sbo = bytes
@@ -83,43 +90,40 @@ __device__ __forceinline__ float fast_exp2(float x) {
 
 template <int HD>
 struct UaSmem {
-  static constexpr uint32_t Q_BYTES = UA_ROWS * HD * 2;
-  static constexpr uint32_t KV_TILE = UA_KEYS * HD * 2;        // one K or V tile
-  static constexpr uint32_t STAGE = 2 * KV_TILE;               // K then V
-  static constexpr uint32_t P_BYTES = UA_ROWS * UA_KEYS * 2;
-  static constexpr uint32_t TOTAL = Q_BYTES + 2 * STAGE + P_BYTES + 1024;
+  static constexpr uint32_t Q_TILE = UA_ROWS * HD * 2;           // one row tile of Q
+  static constexpr uint32_t KV_TILE = UA_KEYS * HD * 2;          // one K or V tile
+  static constexpr uint32_t STAGE = 2 * KV_TILE;                 // K then V
+  static constexpr uint32_t P_TILE = UA_ROWS * UA_KEYS * 2;      // probabilities of one row tile
+  static constexpr uint32_t TOTAL = UA_TILES * Q_TILE + UA_STAGES * STAGE + UA_TILES * P_TILE + 1024;
+  static constexpr uint32_t TMEM_COLS = (UA_TILES * (UA_KEYS + HD)) <= 256 ? 256 : 512;  // S_0, S_1, O_0, O_1
 };
 
 template <int HD>
-__global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ CUtensorMap tmK,
-                                                        const __grid_constant__ CUtensorMap tmV,
-                                                        const __grid_constant__ CUtensorMap tmQ, int q_by_tma,
-                                                        const __nv_bfloat16* __restrict__ q,
-                                                        __nv_bfloat16* __restrict__ o, float* __restrict__ o_part,
-                                                        float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv,
-                                                        int S, int keys_per_split, float scale_log2,
-                                                        int* __restrict__ status) {
+__global__ void __launch_bounds__(UA_THREADS, 1)
+    attn_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                     const __grid_constant__ CUtensorMap tmQ, int q_by_tma, const __nv_bfloat16* __restrict__ q,
+                     __nv_bfloat16* __restrict__ o, float* __restrict__ o_part, float* __restrict__ ml_part, int a_seq,
+                     int n, int H, int Hkv, int S, int keys_per_split, float scale_log2, int* __restrict__ status) {
   using SM = UaSmem<HD>;
   constexpr int PANELS = HD / 64;
-  constexpr uint32_t TMEM_COLS = 256;  // S: columns 0..127, O_t: columns 128..128+HD-1
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t kv_full[2];
-  __shared__ __align__(8) uint64_t bar_s, bar_o, bar_q;
+  __shared__ __align__(8) uint64_t kv_full[UA_STAGES], kv_empty[UA_STAGES];
+  __shared__ __align__(8) uint64_t s_full[UA_TILES], p_full[UA_TILES], o_full[UA_TILES], q_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_s = base, kv_s = base + SM::Q_BYTES, p_s = kv_s + 2 * SM::STAGE;
-  uint8_t* p_gen = base_gen + SM::Q_BYTES + 2 * SM::STAGE;
+  const uint32_t q_s = base, kv_s = q_s + UA_TILES * SM::Q_TILE, p_s = kv_s + UA_STAGES * SM::STAGE;
   volatile int* abortp = &abort_flag;
 
   const int G = H / Hkv;
   const int kh = blockIdx.y;
   const int b = blockIdx.z / S, split = blockIdx.z - b * S;
-  const int row0 = blockIdx.x * UA_ROWS;
+  const int row0 = blockIdx.x * (UA_TILES * UA_ROWS);
   const int n_rows = a_seq * G;
+  const int live = row0 + UA_ROWS < n_rows ? 2 : 1;              // row tiles of this CTA that hold rows
   const int key_lo = split * keys_per_split;
   const int key_hi = min(n, key_lo + keys_per_split);
   const int n_tiles = (key_hi - key_lo + UA_KEYS - 1) / UA_KEYS;  // >= 1 by construction of the plan
@@ -127,18 +131,24 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
 
   if (tid == 0) {
     abort_flag = 0;
-    mbar_init(smem_u32(&kv_full[0]), 1);
-    mbar_init(smem_u32(&kv_full[1]), 1);
-    mbar_init(smem_u32(&bar_s), 1);
-    mbar_init(smem_u32(&bar_o), 1);
-    mbar_init(smem_u32(&bar_q), 1);
+    for (int i = 0; i < UA_STAGES; ++i) {
+      mbar_init(smem_u32(&kv_full[i]), 1);
+      mbar_init(smem_u32(&kv_empty[i]), 1);
+    }
+    for (int i = 0; i < UA_TILES; ++i) {
+      mbar_init(smem_u32(&s_full[i]), 1);
+      mbar_init(smem_u32(&p_full[i]), UA_ROWS);      // every thread of the tile's softmax group arrives
+      mbar_init(smem_u32(&o_full[i]), 1);
+    }
+    mbar_init(smem_u32(&q_bar), q_by_tma ? 1 : UA_TILES * UA_ROWS);
     mbar_fence_init();
     prefetch_tensormap(&tmK);
     prefetch_tensormap(&tmV);
+    if (q_by_tma) prefetch_tensormap(&tmQ);
   }
-  if (warp == 0) {
+  if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
-                 "r"(TMEM_COLS)
+                 "r"(SM::TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -148,235 +158,248 @@ __global__ void __launch_bounds__(128) attn_umma_kernel(const __grid_constant__ 
   const uint32_t tmem = tmem_slot;
   pdl_wait();  // Q, K and V come from the preceding kernels
   pdl_trigger();
-
-  // K/V tile t -> stage t & 1: per 64-column panel two boxes of 64 keys
-  auto issue = [&](int t) {
-    const int st = t & 1;
-    const uint32_t fb = smem_u32(&kv_full[st]);
-    mbar_expect_tx(fb, SM::STAGE);
-    const uint32_t dst = kv_s + st * SM::STAGE;
-    const int key0 = key_lo + t * UA_KEYS;
-#pragma unroll
-    for (int p = 0; p < PANELS; ++p)
-#pragma unroll
-      for (int h2 = 0; h2 < 2; ++h2) {
-        const uint32_t off = p * (UA_KEYS * 128) + h2 * (64 * 128);
-        tma_load_3d(dst + off, &tmK, fb, kh * HD + p * 64, key0 + h2 * 64, b);
-        tma_load_3d(dst + SM::KV_TILE + off, &tmV, fb, kh * HD + p * 64, key0 + h2 * 64, b);
-      }
-  };
-  if (tid == 0) {
-    if (q_by_tma) {
-      // one query head per KV head: the tile's rows are consecutive rows of q, one box per 64-column panel
-      // (rows past this sequence's end belong to no live row: whatever lands there is never written back)
-      const uint32_t qb = smem_u32(&bar_q);
-      mbar_expect_tx(qb, SM::Q_BYTES);
-#pragma unroll
-      for (int p = 0; p < PANELS; ++p) tma_load_2d(q_s + p * (UA_ROWS * 128), &tmQ, qb, kh * HD + p * 64, b * a_seq + row0);
-    }
-    issue(0);
-    if (n_tiles > 1) issue(1);
-  }
-  if (!q_by_tma) {
-  // Q tile: 16-byte loads into the swizzled panel layout (rows past the end are zero)
-  // (eight loads in flight per thread before the first store: a load-store loop would wait one round trip per trip)
-  constexpr int Q_CHUNKS = UA_ROWS * (HD / 8) / 128;  // 16-byte chunks per thread
-#pragma unroll 1
-  for (int i0 = 0; i0 < Q_CHUNKS; i0 += 8) {
-    uint4 qv[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int e = tid + (i0 + i) * 128;
-      const int r = e / (HD / 8), dc = e - r * (HD / 8);
-      const int vr = row0 + r;
-      qv[i] = make_uint4(0, 0, 0, 0);
-      if (vr < n_rows) {
-        const int qi = vr / G, g = vr - qi * G;
-        qv[i] = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int e = tid + (i0 + i) * 128;
-      const int r = e / (HD / 8), dc = e - r * (HD / 8);
-      *reinterpret_cast<uint4*>(base_gen + tile_off<UA_ROWS>(r, dc)) = qv[i];
-    }
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic stores -> MMA reads of shared memory
-  }
-  __syncthreads();
-  if (tid == 0) timeline_mark(1);  // Q staged (or requested)
-
-  constexpr uint32_t idesc_s = make_idesc(UA_ROWS, UA_KEYS);
-  constexpr uint32_t idesc_o = make_idesc(UA_ROWS, HD) | (1u << 16);  // B operand (V) is MN-major
-  const uint32_t row_lane = ((uint32_t)(warp * 32)) << 16;           // this warp's TMEM lanes
-  const int row = warp * 32 + lane;                                   // this thread's row of the tile
-  constexpr float RESCALE_STEP = 8.f;  // log2 units a row's maximum may exceed its reference before O is rescaled
-
-  auto issue_s = [&](int t) {  // S(t) = Q K(t)^T; returns false if the K/V tile never arrived
-    const int st = t & 1;
-    if (!mbar_wait(smem_u32(&kv_full[st]), (uint32_t)(t >> 1) & 1u, abortp)) return false;
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t k_s = kv_s + st * SM::STAGE;
-#pragma unroll
-    for (int ks = 0; ks < HD / 16; ++ks) {
-      const uint32_t off = (ks >> 2) * (128 * 128) + (ks & 3) * 32;  // panel, then 32 bytes per k-step
-      umma_bf16(tmem, make_smem_desc(q_s + off), make_smem_desc(k_s + off), idesc_s, ks > 0 ? 1u : 0u);
-    }
-    umma_commit(smem_u32(&bar_s));
-    return true;
-  };
-
-  // m_ref: the maximum the exponentials of this row refer to; it follows the
-  // true running maximum lazily (O in TMEM is only rescaled when the maximum has
-  // grown by more than RESCALE_STEP, which keeps every exponential below 2^8)
-  float m_ref = -INFINITY, l_run = 0.f;
   bool ok = true;
-  if (tid == 0) {
-    if (q_by_tma) ok = mbar_wait(smem_u32(&bar_q), 0u, abortp);
-    if (ok) ok = issue_s(0);
-  }
 
-  for (int t = 0; t < n_tiles; ++t) {
-    const int st = t & 1;
-    const uint32_t v_s = kv_s + st * SM::STAGE + SM::KV_TILE;
-    // S(t) is complete; the MMAs are executed in order, so O += P V of tile t-1 is complete too
-    ok = mbar_wait(smem_u32(&bar_s), (uint32_t)t & 1u, abortp);
-    ok = __syncthreads_and(ok);
-    if (!ok) break;
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (tid == 0) timeline_mark(2 + (t < 5 ? t : 5));  // scores of tile t complete
-    if (tid == 0 && t >= 1 && t + 1 < n_tiles) issue(t + 1);  // stage (t-1)&1 is free: tile t+1 goes there
-    // ---- this thread's row of scores
-    const int key_base = key_lo + t * UA_KEYS;
-    float sv[UA_KEYS];
-    float mx = -INFINITY;
-    {
-      uint32_t r0[32], r1[32], r2[32], r3[32];  // all four loads in flight, one wait
-      tmem_ld32(tmem + row_lane + 0u, r0);
-      tmem_ld32(tmem + row_lane + 32u, r1);
-      tmem_ld32(tmem + row_lane + 64u, r2);
-      tmem_ld32(tmem + row_lane + 96u, r3);
-      tmem_ld_wait();
+  if (warp == 9) {
+    // ---------------- TMA producer: the Q tiles, then the K/V tiles of the key range ----------------
+    if (lane == 0) {
+      if (q_by_tma) {
+        // one query head per KV head: the rows of a tile are consecutive rows of q, one box per 64-column panel
+        // (rows past this sequence's end belong to no live row: whatever lands there is never written back)
+        const uint32_t qb = smem_u32(&q_bar);
+        mbar_expect_tx(qb, (uint32_t)live * SM::Q_TILE);
+        for (int i = 0; i < live; ++i)
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        sv[j] = __uint_as_float(r0[j]);
-        sv[32 + j] = __uint_as_float(r1[j]);
-        sv[64 + j] = __uint_as_float(r2[j]);
-        sv[96 + j] = __uint_as_float(r3[j]);
+          for (int p = 0; p < PANELS; ++p)
+            tma_load_2d(q_s + i * SM::Q_TILE + p * (UA_ROWS * 128), &tmQ, qb, kh * HD + p * 64,
+                        b * a_seq + row0 + i * UA_ROWS);
       }
-      const int valid = key_hi - key_base;  // >= 1
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one of 128 steps
+      for (int t = 0; t < n_tiles; ++t) {
+        const int st = t % UA_STAGES;
+        if (t >= UA_STAGES && !mbar_wait(smem_u32(&kv_empty[st]), (uint32_t)(t / UA_STAGES - 1) & 1u, abortp)) {
+          ok = false;
+          break;
+        }
+        const uint32_t fb = smem_u32(&kv_full[st]);
+        mbar_expect_tx(fb, SM::STAGE);
+        const uint32_t dst = kv_s + st * SM::STAGE;
+        const int key0 = key_lo + t * UA_KEYS;
 #pragma unroll
-      for (int j = 0; j < UA_KEYS; ++j) {
-        sv[j] = (j < valid) ? sv[j] * scale_log2 : -INFINITY;
-        mx4[j & 3] = fmaxf(mx4[j & 3], sv[j]);
-      }
-      mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-    }
-    // ---- lazy rescale of O (warp-uniform branch: the TMEM accesses are warp-collective)
-    const bool grow = mx > m_ref + RESCALE_STEP;
-    if (__any_sync(0xffffffffu, grow)) {
-      const float corr = grow ? exp2f(m_ref - mx) : 1.f;  // first tile: exp2(-inf) = 0, O is not read (t == 0)
-      if (grow) {
-        m_ref = mx;
-        l_run *= corr;
-      }
-      if (t > 0) {
-#pragma unroll
-        for (int c = 0; c < HD; c += 32) {
-          uint32_t r[32];
-          tmem_ld32(tmem + row_lane + 128u + (uint32_t)c, r);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
-          tmem_st32(tmem + row_lane + 128u + (uint32_t)c, r);
+        for (int p = 0; p < PANELS; ++p) {
+          tma_load_3d(dst + p * (UA_KEYS * 128), &tmK, fb, kh * HD + p * 64, key0, b);
+          tma_load_3d(dst + SM::KV_TILE + p * (UA_KEYS * 128), &tmV, fb, kh * HD + p * 64, key0, b);
         }
       }
     }
-    // ---- probabilities -> shared memory (bf16, layout of an MMA A operand)
-    float p_sum4[4] = {0.f, 0.f, 0.f, 0.f};
+  } else if (warp == 8) {
+    // ---------------- MMA issuer ----------------
+    // Per key tile t and row tile i:  S_i(t) = Q_i K(t)^T  ->  [softmax group i]  ->  O_i += P_i(t) V(t), and right
+    // behind it S_i(t+1), so that the tensor pipe works on one row tile while the other is in its softmax.  A
+    // commit covers every MMA issued before it, so when s_full[i] flips for tile t+1 the product O_i += P_i V of
+    // tile t has completed too: the group may then rescale O_i and overwrite P_i.
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc(UA_ROWS, UA_KEYS);
+      constexpr uint32_t idesc_o = make_idesc(UA_ROWS, HD) | (1u << 16);  // B operand (V) is MN-major
+      auto issue_s = [&](int i, int st) {
+        const uint32_t qi_s = q_s + i * SM::Q_TILE, k_s = kv_s + st * SM::STAGE;
 #pragma unroll
-    for (int c8 = 0; c8 < UA_KEYS / 8; ++c8) {
-      float pv[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        pv[j] = fast_exp2(sv[c8 * 8 + j] - m_ref);
-        p_sum4[j & 3] += pv[j];
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint32_t qoff = (ks >> 2) * (UA_ROWS * 128) + (ks & 3) * 32;  // panel, then 32 bytes per k-step
+          const uint32_t koff = (ks >> 2) * (UA_KEYS * 128) + (ks & 3) * 32;
+          umma_bf16(tmem + (uint32_t)(i * UA_KEYS), make_smem_desc(qi_s + qoff), make_smem_desc(k_s + koff), idesc_s,
+                    ks > 0 ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&s_full[i]));
+      };
+      ok = mbar_wait(smem_u32(&q_bar), 0u, abortp) && mbar_wait(smem_u32(&kv_full[0]), 0u, abortp);
+      if (ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        for (int i = 0; i < live; ++i) issue_s(i, 0);
       }
-      *reinterpret_cast<uint4*>(p_gen + tile_off<UA_ROWS>(row, c8)) =
-          make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
-    }
-    l_run += (p_sum4[0] + p_sum4[1]) + (p_sum4[2] + p_sum4[3]);
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncthreads();
-
-    // ---- O += P V, and straight after it the scores of the next tile
-    if (tid == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int st = t % UA_STAGES, st_next = (t + 1) % UA_STAGES;
+        const uint32_t v_s = kv_s + st * SM::STAGE + SM::KV_TILE;
+        bool next_ready = t + 1 >= n_tiles;
+        for (int i = 0; i < live && ok; ++i) {
+          ok = mbar_wait(smem_u32(&p_full[i]), (uint32_t)t & 1u, abortp);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-      for (int ks = 0; ks < UA_KEYS / 16; ++ks) {
-        const uint32_t a_off = (ks >> 2) * (UA_ROWS * 128) + (ks & 3) * 32;  // P: K-major, panels of 64 keys
-        const uint32_t b_off = ks * (16 * 128);                             // V: 16 key rows of 128 bytes
-        umma_bf16(tmem + 128, make_smem_desc(p_s + a_off), make_smem_desc_mn(v_s + b_off, UA_KEYS * 128, 1024), idesc_o,
-                  (t > 0 || ks > 0) ? 1u : 0u);
+          for (int ks = 0; ks < UA_KEYS / 16; ++ks)   // P_i: K-major, one panel of 64 keys; V: 16 key rows of 128 bytes
+            umma_bf16(tmem + (uint32_t)(UA_TILES * UA_KEYS + i * HD), make_smem_desc(p_s + i * SM::P_TILE + ks * 32),
+                      make_smem_desc_mn(v_s + ks * (16 * 128), UA_KEYS * 128, 1024), idesc_o, (t > 0 || ks > 0) ? 1u : 0u);
+          if (t + 1 < n_tiles) {
+            if (!next_ready) {
+              ok = mbar_wait(smem_u32(&kv_full[st_next]), (uint32_t)((t + 1) / UA_STAGES) & 1u, abortp);
+              if (!ok) break;
+              asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+              next_ready = true;
+            }
+            issue_s(i, st_next);
+          } else {
+            umma_commit(smem_u32(&o_full[i]));  // last tile: O_i is final when this fires
+          }
+        }
+        if (ok) umma_commit(smem_u32(&kv_empty[st]));  // the stage may be refilled once these MMAs have read it
       }
-      if (t + 1 < n_tiles)
-        ok = issue_s(t + 1);
-      else
-        umma_commit(smem_u32(&bar_o));  // last tile: O is final when this fires
-    }
-  }
-  if (ok) {
-    ok = mbar_wait(smem_u32(&bar_o), 0u, abortp);
-    ok = __syncthreads_and(ok);
-  }
-
-  if (ok) {
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (tid == 0) timeline_mark(8);  // O complete
-    const int vr = row0 + row;
-    const bool live = vr < n_rows;
-    const int qi = live ? vr / G : 0, g = live ? vr - qi * G : 0;
-    const size_t orow = ((size_t)b * a_seq + qi) * H + (kh * G + g);  // (row, head) index
-    const float inv = 1.f / l_run;
-    const size_t total = (size_t)gridDim.z / S * a_seq * H;
-#pragma unroll
-    for (int c = 0; c < HD; c += 32) {
-      uint32_t r[32];
-      tmem_ld32(tmem + row_lane + 128u + (uint32_t)c, r);  // warp-collective: every lane takes part
-      tmem_ld_wait();
-      if (!live) continue;
-      if (S == 1) {
-        __nv_bfloat16* dst = o + orow * HD + c;
-#pragma unroll
-        for (int i = 0; i < 32; i += 8)
-          *reinterpret_cast<uint4*>(dst + i) = make_uint4(
-              pack_bf16(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv),
-              pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv),
-              pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv),
-              pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv));
-      } else {
-        float* dst = o_part + ((size_t)split * total + orow) * HD + c;
-#pragma unroll
-        for (int i = 0; i < 32; i += 4)
-          *reinterpret_cast<uint4*>(dst + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
-      }
-    }
-    if (live && S > 1) {
-      float* ml = ml_part + ((size_t)split * total + orow) * 2;
-      ml[0] = m_ref;
-      ml[1] = l_run;
     }
   } else {
+    // ---------------- softmax groups: warps 0-3 own row tile 0, warps 4-7 row tile 1 ----------------
+    const int i = warp >> 2;                                  // row tile
+    const int row = (warp & 3) * 32 + lane;                   // row of the tile = TMEM lane
+    const uint32_t row_lane = ((uint32_t)((warp & 3) * 32)) << 16;
+    const uint32_t s_col = (uint32_t)(i * UA_KEYS), o_col = (uint32_t)(UA_TILES * UA_KEYS + i * HD);
+    const int gtid = tid & 127;
+    if (!q_by_tma) {
+      // Q tiles: 16-byte loads into the swizzled panel layout by the 256 softmax threads (rows past the end are
+      // zero); eight loads in flight per thread before the first store
+      constexpr int Q_CHUNKS = HD / 8;  // 16-byte chunks per thread: 256 rows x HD / 8 chunks over 256 threads
+#pragma unroll 1
+      for (int i0 = 0; i0 < Q_CHUNKS; i0 += 8) {
+        uint4 qv[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int e = (tid & 255) + (i0 + k) * 256;
+          const int r = e / (HD / 8), dc = e - r * (HD / 8);   // r: row of the CTA's 256
+          const int vr = row0 + r;
+          qv[k] = make_uint4(0, 0, 0, 0);
+          if (vr < n_rows) {
+            const int qi = vr / G, g = vr - qi * G;
+            qv[k] = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int e = (tid & 255) + (i0 + k) * 256;
+          const int r = e / (HD / 8), dc = e - r * (HD / 8);
+          *reinterpret_cast<uint4*>(base_gen + (r >> 7) * SM::Q_TILE + tile_off<UA_ROWS>(r & 127, dc)) = qv[k];
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic stores -> MMA reads of shared memory
+      mbar_arrive(smem_u32(&q_bar));
+    }
+    if (gtid == 0 && i == 0) timeline_mark(1);  // Q staged (or requested)
+
+    constexpr float RESCALE_STEP = 8.f;  // log2 units a row's maximum may exceed its reference before O is rescaled
+    // m_ref: the maximum the exponentials of this row refer to; it follows the true running maximum lazily (O in
+    // TMEM is only rescaled when the maximum has grown by more than RESCALE_STEP, which keeps every exponential
+    // below 2^8)
+    float m_ref = -INFINITY, l_run = 0.f;
+    uint8_t* p_gen = base_gen + UA_TILES * SM::Q_TILE + UA_STAGES * SM::STAGE + i * SM::P_TILE;
+    if (i < live) {
+      for (int t = 0; t < n_tiles; ++t) {
+        ok = mbar_wait(smem_u32(&s_full[i]), (uint32_t)t & 1u, abortp);
+        ok = __all_sync(0xffffffffu, ok);  // the TMEM accesses below are warp-collective: the warp stays together
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (gtid == 0 && i == 0) timeline_mark(2 + (t < 5 ? t : 5));  // scores of tile t complete
+        // ---- this thread's row of scores
+        const int valid = key_hi - (key_lo + t * UA_KEYS);  // >= 1
+        float sv[UA_KEYS];
+        float mx;
+        {
+          uint32_t r0[32], r1[32];  // both loads in flight, one wait
+          tmem_ld32(tmem + row_lane + s_col, r0);
+          tmem_ld32(tmem + row_lane + s_col + 32u, r1);
+          tmem_ld_wait();
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one of 64 steps
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            sv[j] = (j < valid) ? __uint_as_float(r0[j]) * scale_log2 : -INFINITY;
+            sv[32 + j] = (32 + j < valid) ? __uint_as_float(r1[j]) * scale_log2 : -INFINITY;
+            mx4[j & 3] = fmaxf(mx4[j & 3], fmaxf(sv[j], sv[32 + j]));
+          }
+          mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        }
+        // ---- lazy rescale of O (warp-uniform branch: the TMEM accesses are warp-collective)
+        const bool grow = mx > m_ref + RESCALE_STEP;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float corr = grow ? exp2f(m_ref - mx) : 1.f;  // first tile: exp2(-inf) = 0, O is not read (t == 0)
+          if (grow) {
+            m_ref = mx;
+            l_run *= corr;
+          }
+          if (t > 0) {
+#pragma unroll
+            for (int c = 0; c < HD; c += 32) {
+              uint32_t r[32];
+              tmem_ld32(tmem + row_lane + o_col + (uint32_t)c, r);
+              tmem_ld_wait();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
+              tmem_st32(tmem + row_lane + o_col + (uint32_t)c, r);
+            }
+          }
+        }
+        // ---- probabilities -> shared memory (bf16, layout of an MMA A operand: one 128-byte row per tile row)
+        float p_sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c8 = 0; c8 < UA_KEYS / 8; ++c8) {
+          float pv[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            pv[j] = fast_exp2(sv[c8 * 8 + j] - m_ref);
+            p_sum4[j & 3] += pv[j];
+          }
+          *reinterpret_cast<uint4*>(p_gen + tile_off<UA_ROWS>(row, c8)) =
+              make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
+        }
+        l_run += (p_sum4[0] + p_sum4[1]) + (p_sum4[2] + p_sum4[3]);
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(smem_u32(&p_full[i]));
+      }
+      if (ok) ok = mbar_wait(smem_u32(&o_full[i]), 0u, abortp);
+      ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below are warp-collective
+      if (ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (gtid == 0 && i == 0) timeline_mark(8);  // O complete
+        const int vr = row0 + i * UA_ROWS + row;
+        const bool is_live = vr < n_rows;
+        const int qi = is_live ? vr / G : 0, g = is_live ? vr - qi * G : 0;
+        const size_t orow = ((size_t)b * a_seq + qi) * H + (kh * G + g);  // (row, head) index
+        const float inv = 1.f / l_run;
+        const size_t total = (size_t)gridDim.z / S * a_seq * H;
+#pragma unroll
+        for (int c = 0; c < HD; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(tmem + row_lane + o_col + (uint32_t)c, r);  // warp-collective: every lane takes part
+          tmem_ld_wait();
+          if (!is_live) continue;
+          if (S == 1) {
+            __nv_bfloat16* dst = o + orow * HD + c;
+#pragma unroll
+            for (int k = 0; k < 32; k += 8)
+              *reinterpret_cast<uint4*>(dst + k) = make_uint4(
+                  pack_bf16(__uint_as_float(r[k]) * inv, __uint_as_float(r[k + 1]) * inv),
+                  pack_bf16(__uint_as_float(r[k + 2]) * inv, __uint_as_float(r[k + 3]) * inv),
+                  pack_bf16(__uint_as_float(r[k + 4]) * inv, __uint_as_float(r[k + 5]) * inv),
+                  pack_bf16(__uint_as_float(r[k + 6]) * inv, __uint_as_float(r[k + 7]) * inv));
+          } else {
+            float* dst = o_part + ((size_t)split * total + orow) * HD + c;
+#pragma unroll
+            for (int k = 0; k < 32; k += 4)
+              *reinterpret_cast<uint4*>(dst + k) = make_uint4(r[k], r[k + 1], r[k + 2], r[k + 3]);
+          }
+        }
+        if (is_live && S > 1) {
+          float* ml = ml_part + ((size_t)split * total + orow) * 2;
+          ml[0] = m_ref;
+          ml[1] = l_run;
+        }
+      }
+    }
+  }
+  // a wait that gave up anywhere in the CTA: record it once, let copies in flight land
+  ok = __syncthreads_and(ok);
+  if (!ok) {
     if (tid == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
     drain_delay();
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  if (warp == 9) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(SM::TMEM_COLS) : "memory");
   }
 }
 
@@ -393,9 +416,9 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
   const size_t total = (size_t)B * a_seq * H;
   float* o_part = scratch;
   float* ml_part = scratch ? scratch + (size_t)S * total * HD : nullptr;
-  dim3 grid((a_seq * G + UA_ROWS - 1) / UA_ROWS, Hkv, B * S);
+  dim3 grid((a_seq * G + UA_TILES * UA_ROWS - 1) / (UA_TILES * UA_ROWS), Hkv, B * S);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
-  cudaError_t e = launch_k(L, attn_umma_kernel<HD>, grid, dim3(128), SMEM, tmK, tmV, tmQ, q_by_tma, (const __nv_bfloat16*)q,
+  cudaError_t e = launch_k(L, attn_umma_kernel<HD>, grid, dim3(UA_THREADS), SMEM, tmK, tmV, tmQ, q_by_tma, (const __nv_bfloat16*)q,
                            (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split, scale_log2,
                            L.d_status);
   L.count();
@@ -404,12 +427,12 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
 
 }  // namespace
 
-// Key-range splits for 128-row tiles: enough CTAs to cover the SMs, whole
-// 128-key tiles per split, no more splits than the scratch holds.
+// Key-range splits for CTAs of two 128-row tiles: enough CTAs to cover the SMs,
+// whole 64-key tiles per split, no more splits than the scratch holds.
 AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats) {
   AttnPlan p;
   const int G = H / Hkv, sms = sm_count();
-  const long tiles = (long)((a_seq * G + UA_ROWS - 1) / UA_ROWS) * Hkv * B;
+  const long tiles = (long)((a_seq * G + UA_TILES * UA_ROWS - 1) / (UA_TILES * UA_ROWS)) * Hkv * B;
   int S = 1;
   if (tiles < sms) S = (int)((sms + tiles - 1) / tiles);
   const int key_tiles = (n + UA_KEYS - 1) / UA_KEYS;

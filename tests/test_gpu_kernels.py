@@ -152,11 +152,15 @@ ATT_CASES = [
     (1, 128, 512, 28, 4, 128), # Dream-7B partial-step shape
     (1, 3, 4128, 2, 2, 128),   # long-prompt regime: 3 queries, 65 key tiles, ragged last tile
     (2, 200, 333, 4, 2, 64),   # several row tiles, G = 2, ragged keys
-    # more than 64 (query, head-of-group) rows per KV head: the tcgen05 kernel (128-row tiles, 128-key tiles)
+    # more than 64 (query, head-of-group) rows per KV head: the tcgen05 kernel (two 128-row tiles per CTA, 64-key tiles)
     (1, 256, 768, 8, 8, 128),  # LLaDA-8B response-refresh shape, 8 of the 32 heads
-    (1, 130, 1000, 2, 2, 128), # ragged row tile (2 rows in the second), 8 key tiles with a ragged last one
-    (1, 65, 64, 1, 1, 128),    # smallest case of that kernel: one key tile, half of it masked off
+    (1, 130, 1000, 2, 2, 128), # ragged second row tile (2 rows), 16 key tiles with a ragged last one
+    (1, 65, 64, 1, 1, 128),    # smallest case of that kernel: one row tile, one key tile
     (3, 90, 260, 6, 2, 64),    # head_dim 64, G = 3, three sequences
+    (1, 300, 520, 4, 4, 128),  # two CTAs per head, the second with one live row tile; 9 key tiles: the ring is reused
+    (2, 512, 1536, 2, 2, 128), # batched-serving refresh shape: 24 key tiles, two full CTAs per (sequence, head)
+    (1, 40, 200, 28, 4, 128),  # grouped heads: 280 rows per KV head gathered from 7 query heads (no TMA for Q)
+    (1, 200, 3000, 1, 1, 64),  # head_dim 64, one CTA's worth of rows against 47 key tiles: many key-range splits
 ]
 
 
