@@ -317,7 +317,7 @@ dllm_status dllm_kernel_status(void* stream);
  * returns normally; (0) switches that off.  Both calls synchronise the device. */
 dllm_status dllm_debug_set_wait_limit_ns(uint64_t ns);
 /* Tuning hook: overrides, for every later call in this process, the number of
- * key-range splits the 64-row attention kernel takes (0 = automatic).  Results
+ * key-range splits the tensor-core attention kernels take (0 = automatic).  Results
  * stay within the attention tolerance; the merge order changes with the plan. */
 dllm_status dllm_debug_attention_plan(int splits);
 dllm_status dllm_debug_skip_one_load(int enable);

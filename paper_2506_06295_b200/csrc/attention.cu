@@ -261,10 +261,12 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-// tuning override of the 64-row kernel's split count (0 = automatic), see dllm_debug_attention_plan
-int g_force_splits = 0;
 
 }  // namespace
+
+// tuning override of the key-range split count of both tensor-core kernels (0 = automatic), see
+// dllm_debug_attention_plan
+int g_attn_force_splits = 0;
 
 // Key-range splits of the 64-row kernel, whole 64-key tiles per split: enough CTAs to cover the SMs when few
 // rows are active (every split costs the merge a partial per row and head, so no more than that), and about
@@ -287,7 +289,7 @@ AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv) {
   int S = 1;
   if (tiles < sms) S = (int)((sms + tiles - 1) / tiles);
   if (a_seq * G <= 8 && 4 * tiles < 7L * sms) S = (int)((7L * sms + 4 * tiles - 1) / (4 * tiles));
-  if (g_force_splits > 0) S = g_force_splits;
+  if (g_attn_force_splits > 0) S = g_attn_force_splits;
   finish_plan(p, B, a_seq, n, H, S);
   return p;
 }
@@ -442,7 +444,7 @@ extern "C" dllm_status dllm_debug_attention_plan(int splits) {
     dllm::set_last_error("dllm_debug_attention_plan: splits >= 0");
     return DLLM_INVALID_ARG;
   }
-  dllm::g_force_splits = splits;
+  dllm::g_attn_force_splits = splits;
   return DLLM_OK;
 }
 

@@ -436,6 +436,7 @@ AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scr
   int S = 1;
   if (tiles < sms) S = (int)((sms + tiles - 1) / tiles);
   const int key_tiles = (n + UA_KEYS - 1) / UA_KEYS;
+  if (g_attn_force_splits > 0) S = g_attn_force_splits;
   if (S > key_tiles) S = key_tiles;
   const size_t per_split = (size_t)B * a_seq * H * (128 + 2);
   if (S > 1 && (size_t)S * per_split > scratch_floats) S = (int)(scratch_floats / per_split);

@@ -230,7 +230,9 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
 
   int pre = 0;  // stages whose weight tile was requested before the dependency wait
+  int dbg_skip = 0;
   if (threadIdx.x == 0) {
+    dbg_skip = g_debug_skip_act_load;  // read here, long before it is used: not on the path behind the dependency wait
     abort_flag = 0;
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
@@ -277,7 +279,7 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
         mbar_expect_tx(fb, SL::STAGE_BYTES);
         tma_load_2d(dstW, &tmW, fb, kc, n0);
       }
-      const bool skip = i == 0 && g_debug_skip_act_load != 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
+      const bool skip = i == 0 && dbg_skip != 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0;
       if (!skip) tma_load_2d(dstW + W_STAGE_BYTES, &tmA, fb, kc, m0);
       if (++s == STAGES) {
         s = 0;
@@ -296,6 +298,8 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
         ok = false;
         break;
       }
+      if (i == 0) timeline_mark(1);                    // first stage complete: activations have arrived
+      else if (i == STAGES) timeline_mark(2);          // first stage whose weights were not requested ahead of the wait
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t sW = tiles + s * SL::STAGE_BYTES;
       const uint64_t dW = make_smem_desc(sW);
@@ -318,12 +322,14 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   // ---------------- epilogue: TMEM -> registers -> global (all four warps) ----------------
   const bool have = mbar_wait(smem_u32(&accum_bar), 0u, abortp);
   if (!have && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_EPI);
+  if (threadIdx.x == 0) timeline_mark(3);              // accumulator complete
   // the whole warp must agree before the warp-collective TMEM loads
   bool warp_ok = __all_sync(0xffffffffu, have);
   if (act_out || m_ffn < 0) warp_ok = __syncthreads_and(warp_ok);  // these epilogues exchange data between warps
   if (warp_ok) {
     float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // the drained ring
     gemm_epilogue<BN>(tmem_d, ex, m0, n0, nt, M, N, part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
+    if (threadIdx.x == 0) timeline_mark(4);            // this thread's part of the epilogue written
   } else {
     drain_delay();  // gave up: let copies in flight land before shared memory is released
   }

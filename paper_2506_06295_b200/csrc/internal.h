@@ -230,6 +230,7 @@ struct AttnChoice {
   AttnPlan plan{1, 0, 0};
 };
 AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats);
+extern int g_attn_force_splits;  // tuning override of both plans' split count (0 = automatic)
 // bf16 with head_dim 64 / 128 runs on the tensor cores (scratch holds the
 // partials of split key ranges; without it one split is used); everything else
 // on the plain-ALU kernel.
