@@ -269,9 +269,10 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
 int g_attn_force_splits = 0;
 
 // Key-range splits of the 64-row kernel, whole 64-key tiles per split: enough CTAs to cover the SMs when few
-// rows are active (every split costs the merge a partial per row and head, so no more than that), and about
-// two CTAs per SM when a KV head has at most eight rows (three queries against thousands of keys: the merge is
-// negligible and the key range is what takes the time).
+// rows are active (every split costs the merge a partial per row and head, so no more than that), and two CTAs
+// per SM (what the shared memory of an SM holds) when a split would otherwise be left with more than eight key
+// tiles to work through one after the other (a few queries against thousands of keys).  From sweeps on B200:
+// 64 rows x 768 keys x 32 heads is fastest with 4 splits, 3 or 36 rows x 4128 keys x 32 heads with 9 or 10.
 static void finish_plan(AttnPlan& p, int B, int a_seq, int n, int H, int S) {
   const int key_tiles = (n + AT_KEYS - 1) / AT_KEYS;
   if (S > key_tiles) S = key_tiles;
@@ -287,8 +288,11 @@ AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv) {
   const int G = H / Hkv, sms = sm_count();
   const long tiles = (long)((a_seq * G + AT_ROWS - 1) / AT_ROWS) * Hkv * B;
   int S = 1;
-  if (tiles < sms) S = (int)((sms + tiles - 1) / tiles);
-  if (a_seq * G <= 8 && 4 * tiles < 7L * sms) S = (int)((7L * sms + 4 * tiles - 1) / (4 * tiles));
+  if (tiles < sms) {
+    S = (int)((sms + tiles - 1) / tiles);
+    const int key_tiles = (n + AT_KEYS - 1) / AT_KEYS;
+    if ((key_tiles + S - 1) / S > 8) S = (int)((2L * sms + tiles - 1) / tiles);
+  }
   if (g_attn_force_splits > 0) S = g_attn_force_splits;
   finish_plan(p, B, a_seq, n, H, S);
   return p;

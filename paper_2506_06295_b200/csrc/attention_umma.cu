@@ -39,7 +39,7 @@ namespace {
 constexpr int UA_ROWS = 128;   // virtual rows per row tile (UMMA M); a CTA works on two row tiles
 constexpr int UA_TILES = 2;
 constexpr int UA_KEYS = 64;    // keys per tile
-constexpr int UA_STAGES = 3;   // K/V ring
+constexpr int UA_STAGES = 4;   // K/V ring
 constexpr int UA_THREADS = 320;  // two softmax groups of 128, one MMA warp, one TMA warp
 
 // MN-major operand ([k][mn] rows of 64 mn-elements = 128 bytes, 128-byte swizzle,
@@ -95,7 +95,11 @@ struct UaSmem {
   static constexpr uint32_t STAGE = 2 * KV_TILE;                 // K then V
   static constexpr uint32_t P_TILE = UA_ROWS * UA_KEYS * 2;      // probabilities of one row tile
   static constexpr uint32_t TOTAL = UA_TILES * Q_TILE + UA_STAGES * STAGE + UA_TILES * P_TILE + 1024;
-  static constexpr uint32_t TMEM_COLS = (UA_TILES * (UA_KEYS + HD)) <= 256 ? 256 : 512;  // S_0, S_1, O_0, O_1
+  // TMEM columns: two score buffers per row tile (S_i of tile t+1 is computed while the group still works on tile
+  // t), then O_0, O_1
+  static constexpr uint32_t O_COL = UA_TILES * 2 * UA_KEYS;
+  static constexpr uint32_t TMEM_COLS = 512;
+  static_assert(O_COL + UA_TILES * HD <= TMEM_COLS, "tensor memory holds 512 columns");
 };
 
 template <int HD>
@@ -108,7 +112,7 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
   constexpr int PANELS = HD / 64;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t kv_full[UA_STAGES], kv_empty[UA_STAGES];
-  __shared__ __align__(8) uint64_t s_full[UA_TILES], p_full[UA_TILES], o_full[UA_TILES], q_bar;
+  __shared__ __align__(8) uint64_t s_full[UA_TILES][2], p_full[UA_TILES], pv_done[UA_TILES], o_full[UA_TILES], q_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
@@ -136,8 +140,10 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
       mbar_init(smem_u32(&kv_empty[i]), 1);
     }
     for (int i = 0; i < UA_TILES; ++i) {
-      mbar_init(smem_u32(&s_full[i]), 1);
+      mbar_init(smem_u32(&s_full[i][0]), 1);
+      mbar_init(smem_u32(&s_full[i][1]), 1);
       mbar_init(smem_u32(&p_full[i]), UA_ROWS);      // every thread of the tile's softmax group arrives
+      mbar_init(smem_u32(&pv_done[i]), 1);
       mbar_init(smem_u32(&o_full[i]), 1);
     }
     mbar_init(smem_u32(&q_bar), q_by_tma ? 1 : UA_TILES * UA_ROWS);
@@ -193,51 +199,54 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
     }
   } else if (warp == 8) {
     // ---------------- MMA issuer ----------------
-    // Per key tile t and row tile i:  S_i(t) = Q_i K(t)^T  ->  [softmax group i]  ->  O_i += P_i(t) V(t), and right
-    // behind it S_i(t+1), so that the tensor pipe works on one row tile while the other is in its softmax.  A
-    // commit covers every MMA issued before it, so when s_full[i] flips for tile t+1 the product O_i += P_i V of
-    // tile t has completed too: the group may then rescale O_i and overwrite P_i.
+    // Per key tile t and row tile i:  S_i(t) = Q_i K(t)^T  ->  [softmax group i]  ->  O_i += P_i(t) V(t).  The scores
+    // of tile t+2 are issued right behind O_i += P_i V of tile t, into the score buffer the group has just read,
+    // so a group always finds its next scores waiting and the tensor pipe works on one row tile while the other
+    // is in its softmax.  pv_done[i] (a commit behind every O_i += P_i V) tells group i that P_i may be overwritten
+    // and O_i rescaled.
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(UA_ROWS, UA_KEYS);
       constexpr uint32_t idesc_o = make_idesc(UA_ROWS, HD) | (1u << 16);  // B operand (V) is MN-major
-      auto issue_s = [&](int i, int st) {
-        const uint32_t qi_s = q_s + i * SM::Q_TILE, k_s = kv_s + st * SM::STAGE;
+      auto issue_s = [&](int i, int t) {
+        const uint32_t qi_s = q_s + i * SM::Q_TILE, k_s = kv_s + (t % UA_STAGES) * SM::STAGE;
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
           const uint32_t qoff = (ks >> 2) * (UA_ROWS * 128) + (ks & 3) * 32;  // panel, then 32 bytes per k-step
           const uint32_t koff = (ks >> 2) * (UA_KEYS * 128) + (ks & 3) * 32;
-          umma_bf16(tmem + (uint32_t)(i * UA_KEYS), make_smem_desc(qi_s + qoff), make_smem_desc(k_s + koff), idesc_s,
-                    ks > 0 ? 1u : 0u);
+          umma_bf16(tmem + (uint32_t)((i * 2 + (t & 1)) * UA_KEYS), make_smem_desc(qi_s + qoff),
+                    make_smem_desc(k_s + koff), idesc_s, ks > 0 ? 1u : 0u);
         }
-        umma_commit(smem_u32(&s_full[i]));
+        umma_commit(smem_u32(&s_full[i][t & 1]));
       };
-      ok = mbar_wait(smem_u32(&q_bar), 0u, abortp) && mbar_wait(smem_u32(&kv_full[0]), 0u, abortp);
-      if (ok) {
+      ok = mbar_wait(smem_u32(&q_bar), 0u, abortp);
+      for (int t = 0; t < 2 && t < n_tiles && ok; ++t) {
+        ok = mbar_wait(smem_u32(&kv_full[t]), 0u, abortp);
+        if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        for (int i = 0; i < live; ++i) issue_s(i, 0);
+        for (int i = 0; i < live; ++i) issue_s(i, t);
       }
       for (int t = 0; t < n_tiles && ok; ++t) {
-        const int st = t % UA_STAGES, st_next = (t + 1) % UA_STAGES;
+        const int st = t % UA_STAGES;
         const uint32_t v_s = kv_s + st * SM::STAGE + SM::KV_TILE;
-        bool next_ready = t + 1 >= n_tiles;
+        bool ahead_ready = t + 2 >= n_tiles;
         for (int i = 0; i < live && ok; ++i) {
           ok = mbar_wait(smem_u32(&p_full[i]), (uint32_t)t & 1u, abortp);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
           for (int ks = 0; ks < UA_KEYS / 16; ++ks)   // P_i: K-major, one panel of 64 keys; V: 16 key rows of 128 bytes
-            umma_bf16(tmem + (uint32_t)(UA_TILES * UA_KEYS + i * HD), make_smem_desc(p_s + i * SM::P_TILE + ks * 32),
+            umma_bf16(tmem + SM::O_COL + (uint32_t)(i * HD), make_smem_desc(p_s + i * SM::P_TILE + ks * 32),
                       make_smem_desc_mn(v_s + ks * (16 * 128), UA_KEYS * 128, 1024), idesc_o, (t > 0 || ks > 0) ? 1u : 0u);
-          if (t + 1 < n_tiles) {
-            if (!next_ready) {
-              ok = mbar_wait(smem_u32(&kv_full[st_next]), (uint32_t)((t + 1) / UA_STAGES) & 1u, abortp);
+          umma_commit(smem_u32(&pv_done[i]));
+          if (t + 1 == n_tiles) umma_commit(smem_u32(&o_full[i]));  // last tile: O_i is final when this fires
+          if (t + 2 < n_tiles) {
+            if (!ahead_ready) {
+              ok = mbar_wait(smem_u32(&kv_full[(t + 2) % UA_STAGES]), (uint32_t)((t + 2) / UA_STAGES) & 1u, abortp);
               if (!ok) break;
               asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-              next_ready = true;
+              ahead_ready = true;
             }
-            issue_s(i, st_next);
-          } else {
-            umma_commit(smem_u32(&o_full[i]));  // last tile: O_i is final when this fires
+            issue_s(i, t + 2);  // into the buffer whose scores (tile t) group i has read before it signalled P_i
           }
         }
         if (ok) umma_commit(smem_u32(&kv_empty[st]));  // the stage may be refilled once these MMAs have read it
@@ -248,7 +257,7 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
     const int i = warp >> 2;                                  // row tile
     const int row = (warp & 3) * 32 + lane;                   // row of the tile = TMEM lane
     const uint32_t row_lane = ((uint32_t)((warp & 3) * 32)) << 16;
-    const uint32_t s_col = (uint32_t)(i * UA_KEYS), o_col = (uint32_t)(UA_TILES * UA_KEYS + i * HD);
+    const uint32_t o_col = SM::O_COL + (uint32_t)(i * HD);
     const int gtid = tid & 127;
     if (!q_by_tma) {
       // Q tiles: 16-byte loads into the swizzled panel layout by the 256 softmax threads (rows past the end are
@@ -288,31 +297,39 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
     uint8_t* p_gen = base_gen + UA_TILES * SM::Q_TILE + UA_STAGES * SM::STAGE + i * SM::P_TILE;
     if (i < live) {
       for (int t = 0; t < n_tiles; ++t) {
-        ok = mbar_wait(smem_u32(&s_full[i]), (uint32_t)t & 1u, abortp);
+        ok = mbar_wait(smem_u32(&s_full[i][t & 1]), (uint32_t)(t >> 1) & 1u, abortp);
         ok = __all_sync(0xffffffffu, ok);  // the TMEM accesses below are warp-collective: the warp stays together
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (gtid == 0 && i == 0) timeline_mark(2 + (t < 5 ? t : 5));  // scores of tile t complete
-        // ---- this thread's row of scores
+        // ---- this thread's row of scores (raw: the scale is folded into the exponent's multiply-add)
         const int valid = key_hi - (key_lo + t * UA_KEYS);  // >= 1
         float sv[UA_KEYS];
         float mx;
         {
           uint32_t r0[32], r1[32];  // both loads in flight, one wait
+          const uint32_t s_col = (uint32_t)((i * 2 + (t & 1)) * UA_KEYS);
           tmem_ld32(tmem + row_lane + s_col, r0);
           tmem_ld32(tmem + row_lane + s_col + 32u, r1);
           tmem_ld_wait();
-          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one of 64 steps
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            sv[j] = (j < valid) ? __uint_as_float(r0[j]) * scale_log2 : -INFINITY;
-            sv[32 + j] = (32 + j < valid) ? __uint_as_float(r1[j]) * scale_log2 : -INFINITY;
-            mx4[j & 3] = fmaxf(mx4[j & 3], fmaxf(sv[j], sv[32 + j]));
+            sv[j] = __uint_as_float(r0[j]);
+            sv[32 + j] = __uint_as_float(r1[j]);
           }
-          mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+          if (valid < UA_KEYS) {  // the ragged last tile of the sequence: keys past the end count for nothing
+#pragma unroll
+            for (int j = 0; j < UA_KEYS; ++j)
+              if (j >= valid) sv[j] = -INFINITY;
+          }
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one of 64 steps
+#pragma unroll
+          for (int j = 0; j < UA_KEYS; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sv[j]);
+          mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;  // scale_log2 > 0
         }
         // ---- lazy rescale of O (warp-uniform branch: the TMEM accesses are warp-collective)
         const bool grow = mx > m_ref + RESCALE_STEP;
+        bool pv_waited = t == 0;  // O_i += P_i V of tile t-1 known to be complete (nothing to wait for at tile 0)
         if (__any_sync(0xffffffffu, grow)) {
           const float corr = grow ? exp2f(m_ref - mx) : 1.f;  // first tile: exp2(-inf) = 0, O is not read (t == 0)
           if (grow) {
@@ -320,6 +337,11 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
             l_run *= corr;
           }
           if (t > 0) {
+            ok = mbar_wait(smem_u32(&pv_done[i]), (uint32_t)(t - 1) & 1u, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            pv_waited = true;
 #pragma unroll
             for (int c = 0; c < HD; c += 32) {
               uint32_t r[32];
@@ -331,20 +353,29 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
             }
           }
         }
-        // ---- probabilities -> shared memory (bf16, layout of an MMA A operand: one 128-byte row per tile row)
+        // ---- probabilities (bf16, packed) ...
         float p_sum4[4] = {0.f, 0.f, 0.f, 0.f};
+        uint4 pk[UA_KEYS / 8];
 #pragma unroll
         for (int c8 = 0; c8 < UA_KEYS / 8; ++c8) {
           float pv[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
-            pv[j] = fast_exp2(sv[c8 * 8 + j] - m_ref);
+            pv[j] = fast_exp2(fmaf(sv[c8 * 8 + j], scale_log2, -m_ref));
             p_sum4[j & 3] += pv[j];
           }
-          *reinterpret_cast<uint4*>(p_gen + tile_off<UA_ROWS>(row, c8)) =
-              make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
+          pk[c8] = make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
         }
         l_run += (p_sum4[0] + p_sum4[1]) + (p_sum4[2] + p_sum4[3]);
+        // ... -> shared memory in the layout of an MMA A operand (one 128-byte row per tile row), once the
+        // product that read the previous tile's probabilities has completed
+        if (!pv_waited) {
+          ok = mbar_wait(smem_u32(&pv_done[i]), (uint32_t)(t - 1) & 1u, abortp);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        }
+#pragma unroll
+        for (int c8 = 0; c8 < UA_KEYS / 8; ++c8) *reinterpret_cast<uint4*>(p_gen + tile_off<UA_ROWS>(row, c8)) = pk[c8];
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive(smem_u32(&p_full[i]));
@@ -427,18 +458,33 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
 
 }  // namespace
 
-// Key-range splits for CTAs of two 128-row tiles: enough CTAs to cover the SMs,
-// whole 64-key tiles per split, no more splits than the scratch holds.
+// Key-range splits for CTAs of two 128-row tiles, whole 64-key tiles per split, no more splits than the scratch
+// holds.  A split shortens the key range a CTA walks through but adds a partial result per (row, head) pair that
+// the merge has to write and read, so the count is the one a small cost model likes best (microseconds, fitted
+// to sweeps on B200: about 1.5 us per key tile of a CTA at head_dim 128, one CTA per SM at a time, 4 us of
+// fixed cost, and for a merge 2.5 us plus 1040 bytes per pair and split at 5 TB/s).
 AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats) {
   AttnPlan p;
   const int G = H / Hkv, sms = sm_count();
   const long tiles = (long)((a_seq * G + UA_TILES * UA_ROWS - 1) / (UA_TILES * UA_ROWS)) * Hkv * B;
-  int S = 1;
-  if (tiles < sms) S = (int)((sms + tiles - 1) / tiles);
   const int key_tiles = (n + UA_KEYS - 1) / UA_KEYS;
-  if (g_attn_force_splits > 0) S = g_attn_force_splits;
-  if (S > key_tiles) S = key_tiles;
   const size_t per_split = (size_t)B * a_seq * H * (128 + 2);
+  const double pairs = (double)B * a_seq * H;
+  int best = 1;
+  double best_us = 0.0;
+  for (int S = 1; S <= key_tiles && S <= 16; ++S) {
+    if (S > 1 && (size_t)S * per_split > scratch_floats) break;
+    const int tps = (key_tiles + S - 1) / S;
+    if (S > 1 && (key_tiles + tps - 1) / tps != S) continue;  // the same tiles per split as a smaller count
+    const double waves = (double)((tiles * S + sms - 1) / sms);
+    const double us = 4.0 + waves * tps * 1.5 + (S > 1 ? 2.5 + S * pairs * 1040.0 / 5.0e6 : 0.0);
+    if (S == 1 || us < best_us) {
+      best = S;
+      best_us = us;
+    }
+  }
+  int S = g_attn_force_splits > 0 ? g_attn_force_splits : best;
+  if (S > key_tiles) S = key_tiles;
   if (S > 1 && (size_t)S * per_split > scratch_floats) S = (int)(scratch_floats / per_split);
   if (S < 1) S = 1;
   const int tiles_per_split = (key_tiles + S - 1) / S;

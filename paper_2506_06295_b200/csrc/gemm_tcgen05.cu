@@ -82,13 +82,15 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += CH) {
       if (m0 + c0 >= M) break;  // uniform across the CTA
+      {  // all TMEM loads of the chunk in flight, one wait (a load-wait-store loop pays the TMEM latency per trip)
+        uint32_t r[CH / 16][16];
 #pragma unroll
-      for (int c = 0; c < CH; c += 16) {
-        uint32_t r[16];
-        tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + c), r);
+        for (int c = 0; c < CH; c += 16) tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + c), r[c / 16]);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-        for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[j]);
+        for (int c = 0; c < CH; c += 16)
+#pragma unroll
+          for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[c / 16][j]);
       }
       __syncthreads();
       MaxSum t{-INFINITY, 0.f, 0x7fffffff};
@@ -148,13 +150,15 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += CH) {
       if (m0 + c0 >= M) break;  // uniform across the CTA
+      {  // all TMEM loads of the chunk in flight, one wait (a load-wait-store loop pays the TMEM latency per trip)
+        uint32_t r[CH / 16][16];
 #pragma unroll
-      for (int c = 0; c < CH; c += 16) {
-        uint32_t r[16];
-        tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + c), r);
+        for (int c = 0; c < CH; c += 16) tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + c), r[c / 16]);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-        for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[j]);
+        for (int c = 0; c < CH; c += 16)
+#pragma unroll
+          for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[c / 16][j]);
       }
       __syncthreads();
 #pragma unroll
@@ -177,18 +181,22 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const int n = n0 + warp * 32 + lane;
     float* out = slab + n;
+    constexpr int CH = BN < 64 ? BN : 64;  // columns (activation rows) per trip: their TMEM loads are in flight together
 #pragma unroll 1
-    for (int c = 0; c < BN; c += 16) {
-      if (m0 + c >= M) break;  // uniform across the CTA
-      uint32_t r[16];
-      tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
+    for (int c0 = 0; c0 < BN; c0 += CH) {
+      if (m0 + c0 >= M) break;  // uniform across the CTA
+      uint32_t r[CH / 16][16];
+#pragma unroll
+      for (int c = 0; c < CH; c += 16) tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + c), r[c / 16]);
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
       if (n < N) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int m = m0 + c + j;
-          if (m < M) out[(size_t)m * N] = __uint_as_float(r[j]);
-        }
+        for (int c = 0; c < CH; c += 16)
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + c + j;
+            if (m < M) out[(size_t)m * N] = __uint_as_float(r[c / 16][j]);
+          }
       }
     }
   }
