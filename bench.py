@@ -396,7 +396,9 @@ def main():
     l0 = ses.launch_count()
     torch.cuda.profiler.start()       # no-op unless a profiler waits for it (`ncu --profile-from-start off`)
     ev0.record(stream)
+    t_host = time.perf_counter()
     run_steps(K)
+    host_enqueue_ms = 1e3 * (time.perf_counter() - t_host)    # the host only enqueues: it runs ahead of the device
     ev1.record(stream)
     barrier()
     torch.cuda.profiler.stop()
@@ -570,6 +572,7 @@ def main():
                                   "what": "dllm_step_scheduled_block: logits, estimate and confidence only for the "
                                           "block the step works on; layers and caches identical"},
         "gpu_launches": int(launches),
+        "host_enqueue_ms_per_step": host_enqueue_ms / K,
         "clocks": clocks,
         "roofline": {"kernel": "gemm_bf16_tcgen05_kernel / gemm_bf16_pair_kernel (all projections of the timed steps)",
                      "bound": g["bound"], "achieved": g["achieved"], "peak": g["peak"], "unit": g["unit"],

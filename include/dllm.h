@@ -316,10 +316,19 @@ dllm_status dllm_kernel_status(void* stream);
  * records the status code, skips its epilogue, frees its tensor memory and
  * returns normally; (0) switches that off.  Both calls synchronise the device. */
 dllm_status dllm_debug_set_wait_limit_ns(uint64_t ns);
+/* Tuning / test hook: kernel choice of the bf16 projections whose plan has no
+ * split and 256-row activation tiles, for every later call in this process:
+ * 0 automatic (the persistent kernel when there are more tiles than SMs), 1
+ * always the persistent kernel, -1 always the one-tile-per-CTA kernel.  The two
+ * kernels give bit-identical results. */
+dllm_status dllm_debug_gemm_plan(int persistent);
 /* Tuning hook: overrides, for every later call in this process, the number of
- * key-range splits the tensor-core attention kernels take (0 = automatic).  Results
- * stay within the attention tolerance; the merge order changes with the plan. */
-dllm_status dllm_debug_attention_plan(int splits);
+ * key-range splits the tensor-core attention kernels take (0 = automatic) and,
+ * if tcgen05_min_rows > 0, the number of (query, head-of-group) rows per KV head
+ * from which the 128-row tcgen05 kernel is taken instead of the 64-row mma.sync
+ * kernel.  Results stay within the attention tolerance; the merge order changes
+ * with the plan. */
+dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows);
 dllm_status dllm_debug_skip_one_load(int enable);
 /* C[M,N] (fp32, row-major, DEVICE) = A[M,K] * W[N,K]^T with bf16 operands on
  * the tensor cores (tcgen05 + TMA).  d_partials is scratch of

@@ -267,6 +267,8 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
 // tuning override of the key-range split count of both tensor-core kernels (0 = automatic), see
 // dllm_debug_attention_plan
 int g_attn_force_splits = 0;
+// (query, head-of-group) rows per KV head from which a bf16 shape takes the 128-row tcgen05 kernel
+int g_attn_umma_min_rows = AT_ROWS + 1;
 
 // Key-range splits of the 64-row kernel, whole 64-key tiles per split: enough CTAs to cover the SMs when few
 // rows are active (every split costs the merge a partial per row and head, so no more than that), and two CTAs
@@ -303,7 +305,7 @@ AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv) {
 // room for the partials it runs one split.  The 128-row tcgen05 kernel lowers its split count to what fits.
 AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats) {
   AttnChoice c;
-  c.umma = a_seq * (H / Hkv) > AT_ROWS;
+  c.umma = a_seq * (H / Hkv) >= g_attn_umma_min_rows;
   if (c.umma) {
     c.plan = plan_attention_umma(B, a_seq, n, H, Hkv, scratch_floats);
   } else {
@@ -443,12 +445,13 @@ extern "C" dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, 
   return DLLM_OK;
 }
 
-extern "C" dllm_status dllm_debug_attention_plan(int splits) {
-  if (splits < 0) {
-    dllm::set_last_error("dllm_debug_attention_plan: splits >= 0");
+extern "C" dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows) {
+  if (splits < 0 || tcgen05_min_rows < 0) {
+    dllm::set_last_error("dllm_debug_attention_plan: arguments must not be negative");
     return DLLM_INVALID_ARG;
   }
   dllm::g_attn_force_splits = splits;
+  if (tcgen05_min_rows > 0) dllm::g_attn_umma_min_rows = tcgen05_min_rows;
   return DLLM_OK;
 }
 

@@ -39,7 +39,7 @@ namespace {
 constexpr int UA_ROWS = 128;   // virtual rows per row tile (UMMA M); a CTA works on two row tiles
 constexpr int UA_TILES = 2;
 constexpr int UA_KEYS = 64;    // keys per tile
-constexpr int UA_STAGES = 4;   // K/V ring
+constexpr int UA_STAGES = 6;   // K/V ring
 constexpr int UA_THREADS = 320;  // two softmax groups of 128, one MMA warp, one TMA warp
 
 // MN-major operand ([k][mn] rows of 64 mn-elements = 128 bytes, 128-byte swizzle,
@@ -90,14 +90,12 @@ __device__ __forceinline__ float fast_exp2(float x) {
 
 template <int HD>
 struct UaSmem {
-  static constexpr uint32_t Q_TILE = UA_ROWS * HD * 2;           // one row tile of Q
   static constexpr uint32_t KV_TILE = UA_KEYS * HD * 2;          // one K or V tile
   static constexpr uint32_t STAGE = 2 * KV_TILE;                 // K then V
-  static constexpr uint32_t P_TILE = UA_ROWS * UA_KEYS * 2;      // probabilities of one row tile
-  static constexpr uint32_t TOTAL = UA_TILES * Q_TILE + UA_STAGES * STAGE + UA_TILES * P_TILE + 1024;
-  // TMEM columns: two score buffers per row tile (S_i of tile t+1 is computed while the group still works on tile
-  // t), then O_0, O_1
-  static constexpr uint32_t O_COL = UA_TILES * 2 * UA_KEYS;
+  static constexpr uint32_t TOTAL = UA_STAGES * STAGE + 1024;    // shared memory holds nothing but the K/V ring
+  // Tensor memory, 128 lanes = the rows of a tile: Q_i as bf16 pairs (HD / 2 columns each), the scores S_i (64
+  // fp32 columns each; the probabilities P_i overwrite the first 32 of them as bf16 pairs), the outputs O_i.
+  static constexpr uint32_t Q_COL = 0, S_COL = UA_TILES * (HD / 2), O_COL = S_COL + UA_TILES * UA_KEYS;
   static constexpr uint32_t TMEM_COLS = 512;
   static_assert(O_COL + UA_TILES * HD <= TMEM_COLS, "tensor memory holds 512 columns");
 };
@@ -105,21 +103,20 @@ struct UaSmem {
 template <int HD>
 __global__ void __launch_bounds__(UA_THREADS, 1)
     attn_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                     const __grid_constant__ CUtensorMap tmQ, int q_by_tma, const __nv_bfloat16* __restrict__ q,
+                     const __nv_bfloat16* __restrict__ q,
                      __nv_bfloat16* __restrict__ o, float* __restrict__ o_part, float* __restrict__ ml_part, int a_seq,
                      int n, int H, int Hkv, int S, int keys_per_split, float scale_log2, int* __restrict__ status) {
   using SM = UaSmem<HD>;
   constexpr int PANELS = HD / 64;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t kv_full[UA_STAGES], kv_empty[UA_STAGES];
-  __shared__ __align__(8) uint64_t s_full[UA_TILES][2], p_full[UA_TILES], pv_done[UA_TILES], o_full[UA_TILES], q_bar;
+  __shared__ __align__(8) uint64_t s_full[UA_TILES], p_full[UA_TILES], o_full[UA_TILES], q_bar;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* base_gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_s = base, kv_s = q_s + UA_TILES * SM::Q_TILE, p_s = kv_s + UA_STAGES * SM::STAGE;
+  const uint32_t kv_s = base;
   volatile int* abortp = &abort_flag;
 
   const int G = H / Hkv;
@@ -140,17 +137,14 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
       mbar_init(smem_u32(&kv_empty[i]), 1);
     }
     for (int i = 0; i < UA_TILES; ++i) {
-      mbar_init(smem_u32(&s_full[i][0]), 1);
-      mbar_init(smem_u32(&s_full[i][1]), 1);
-      mbar_init(smem_u32(&p_full[i]), UA_ROWS);      // every thread of the tile's softmax group arrives
-      mbar_init(smem_u32(&pv_done[i]), 1);
+      mbar_init(smem_u32(&s_full[i]), 1);
+      mbar_init(smem_u32(&p_full[i]), UA_ROWS / 32);  // one arrival per warp of the tile's softmax group
       mbar_init(smem_u32(&o_full[i]), 1);
     }
-    mbar_init(smem_u32(&q_bar), q_by_tma ? 1 : UA_TILES * UA_ROWS);
+    mbar_init(smem_u32(&q_bar), UA_TILES * UA_ROWS / 32);  // one arrival per softmax warp
     mbar_fence_init();
     prefetch_tensormap(&tmK);
     prefetch_tensormap(&tmV);
-    if (q_by_tma) prefetch_tensormap(&tmQ);
   }
   if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
@@ -167,19 +161,8 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
   bool ok = true;
 
   if (warp == 9) {
-    // ---------------- TMA producer: the Q tiles, then the K/V tiles of the key range ----------------
+    // ---------------- TMA producer: the K/V tiles of the key range ----------------
     if (lane == 0) {
-      if (q_by_tma) {
-        // one query head per KV head: the rows of a tile are consecutive rows of q, one box per 64-column panel
-        // (rows past this sequence's end belong to no live row: whatever lands there is never written back)
-        const uint32_t qb = smem_u32(&q_bar);
-        mbar_expect_tx(qb, (uint32_t)live * SM::Q_TILE);
-        for (int i = 0; i < live; ++i)
-#pragma unroll
-          for (int p = 0; p < PANELS; ++p)
-            tma_load_2d(q_s + i * SM::Q_TILE + p * (UA_ROWS * 128), &tmQ, qb, kh * HD + p * 64,
-                        b * a_seq + row0 + i * UA_ROWS);
-      }
       for (int t = 0; t < n_tiles; ++t) {
         const int st = t % UA_STAGES;
         if (t >= UA_STAGES && !mbar_wait(smem_u32(&kv_empty[st]), (uint32_t)(t / UA_STAGES - 1) & 1u, abortp)) {
@@ -199,54 +182,53 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
     }
   } else if (warp == 8) {
     // ---------------- MMA issuer ----------------
-    // Per key tile t and row tile i:  S_i(t) = Q_i K(t)^T  ->  [softmax group i]  ->  O_i += P_i(t) V(t).  The scores
-    // of tile t+2 are issued right behind O_i += P_i V of tile t, into the score buffer the group has just read,
-    // so a group always finds its next scores waiting and the tensor pipe works on one row tile while the other
-    // is in its softmax.  pv_done[i] (a commit behind every O_i += P_i V) tells group i that P_i may be overwritten
-    // and O_i rescaled.
+    // Per key tile t and row tile i:  S_i(t) = Q_i K(t)^T  ->  [softmax group i]  ->  O_i += P_i(t) V(t), and right
+    // behind it S_i(t+1), so that the tensor pipe works on one row tile while the other is in its softmax.  Q_i
+    // and P_i are A operands in tensor memory (P_i in the columns its scores came from), so shared memory is
+    // read for K and V only.  A commit covers every MMA issued before it, so when s_full[i] flips for tile t+1
+    // the product O_i += P_i V of tile t has completed too: the group may then rescale O_i.
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(UA_ROWS, UA_KEYS);
       constexpr uint32_t idesc_o = make_idesc(UA_ROWS, HD) | (1u << 16);  // B operand (V) is MN-major
-      auto issue_s = [&](int i, int t) {
-        const uint32_t qi_s = q_s + i * SM::Q_TILE, k_s = kv_s + (t % UA_STAGES) * SM::STAGE;
+      auto issue_s = [&](int i, int st) {
+        const uint32_t k_s = kv_s + st * SM::STAGE;
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ++ks) {
-          const uint32_t qoff = (ks >> 2) * (UA_ROWS * 128) + (ks & 3) * 32;  // panel, then 32 bytes per k-step
-          const uint32_t koff = (ks >> 2) * (UA_KEYS * 128) + (ks & 3) * 32;
-          umma_bf16(tmem + (uint32_t)((i * 2 + (t & 1)) * UA_KEYS), make_smem_desc(qi_s + qoff),
-                    make_smem_desc(k_s + koff), idesc_s, ks > 0 ? 1u : 0u);
+          const uint32_t koff = (ks >> 2) * (UA_KEYS * 128) + (ks & 3) * 32;  // panel, then 32 bytes per k-step
+          // A = 16 dimensions of Q_i from tensor memory (8 columns of bf16 pairs per k-step)
+          umma_bf16_ta(tmem + SM::S_COL + (uint32_t)(i * UA_KEYS), tmem + SM::Q_COL + (uint32_t)(i * (HD / 2) + ks * 8),
+                       make_smem_desc(k_s + koff), idesc_s, ks > 0 ? 1u : 0u);
         }
-        umma_commit(smem_u32(&s_full[i][t & 1]));
+        umma_commit(smem_u32(&s_full[i]));
       };
-      ok = mbar_wait(smem_u32(&q_bar), 0u, abortp);
-      for (int t = 0; t < 2 && t < n_tiles && ok; ++t) {
-        ok = mbar_wait(smem_u32(&kv_full[t]), 0u, abortp);
-        if (!ok) break;
+      ok = mbar_wait(smem_u32(&q_bar), 0u, abortp) && mbar_wait(smem_u32(&kv_full[0]), 0u, abortp);
+      if (ok) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        for (int i = 0; i < live; ++i) issue_s(i, t);
+        for (int i = 0; i < live; ++i) issue_s(i, 0);
       }
       for (int t = 0; t < n_tiles && ok; ++t) {
-        const int st = t % UA_STAGES;
+        const int st = t % UA_STAGES, st_next = (t + 1) % UA_STAGES;
         const uint32_t v_s = kv_s + st * SM::STAGE + SM::KV_TILE;
-        bool ahead_ready = t + 2 >= n_tiles;
+        bool next_ready = t + 1 >= n_tiles;
         for (int i = 0; i < live && ok; ++i) {
           ok = mbar_wait(smem_u32(&p_full[i]), (uint32_t)t & 1u, abortp);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-          for (int ks = 0; ks < UA_KEYS / 16; ++ks)   // P_i: K-major, one panel of 64 keys; V: 16 key rows of 128 bytes
-            umma_bf16(tmem + SM::O_COL + (uint32_t)(i * HD), make_smem_desc(p_s + i * SM::P_TILE + ks * 32),
-                      make_smem_desc_mn(v_s + ks * (16 * 128), UA_KEYS * 128, 1024), idesc_o, (t > 0 || ks > 0) ? 1u : 0u);
-          umma_commit(smem_u32(&pv_done[i]));
-          if (t + 1 == n_tiles) umma_commit(smem_u32(&o_full[i]));  // last tile: O_i is final when this fires
-          if (t + 2 < n_tiles) {
-            if (!ahead_ready) {
-              ok = mbar_wait(smem_u32(&kv_full[(t + 2) % UA_STAGES]), (uint32_t)((t + 2) / UA_STAGES) & 1u, abortp);
+          for (int ks = 0; ks < UA_KEYS / 16; ++ks)   // A = 16 keys of P_i from tensor memory; V: 16 key rows of 128 bytes
+            umma_bf16_ta(tmem + SM::O_COL + (uint32_t)(i * HD), tmem + SM::S_COL + (uint32_t)(i * UA_KEYS + ks * 8),
+                         make_smem_desc_mn(v_s + ks * (16 * 128), UA_KEYS * 128, 1024), idesc_o,
+                         (t > 0 || ks > 0) ? 1u : 0u);
+          if (t + 1 < n_tiles) {
+            if (!next_ready) {
+              ok = mbar_wait(smem_u32(&kv_full[st_next]), (uint32_t)((t + 1) / UA_STAGES) & 1u, abortp);
               if (!ok) break;
               asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-              ahead_ready = true;
+              next_ready = true;
             }
-            issue_s(i, t + 2);  // into the buffer whose scores (tile t) group i has read before it signalled P_i
+            issue_s(i, st_next);
+          } else {
+            umma_commit(smem_u32(&o_full[i]));  // last tile: O_i is final when this fires
           }
         }
         if (ok) umma_commit(smem_u32(&kv_empty[st]));  // the stage may be refilled once these MMAs have read it
@@ -257,48 +239,47 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
     const int i = warp >> 2;                                  // row tile
     const int row = (warp & 3) * 32 + lane;                   // row of the tile = TMEM lane
     const uint32_t row_lane = ((uint32_t)((warp & 3) * 32)) << 16;
-    const uint32_t o_col = SM::O_COL + (uint32_t)(i * HD);
+    const uint32_t s_col = SM::S_COL + (uint32_t)(i * UA_KEYS), o_col = SM::O_COL + (uint32_t)(i * HD);
     const int gtid = tid & 127;
-    if (!q_by_tma) {
-      // Q tiles: 16-byte loads into the swizzled panel layout by the 256 softmax threads (rows past the end are
-      // zero); eight loads in flight per thread before the first store
-      constexpr int Q_CHUNKS = HD / 8;  // 16-byte chunks per thread: 256 rows x HD / 8 chunks over 256 threads
-#pragma unroll 1
-      for (int i0 = 0; i0 < Q_CHUNKS; i0 += 8) {
-        uint4 qv[8];
+    {
+      // Q_i: every thread fetches its own row (HD bf16 = HD / 8 16-byte words, zero past the last row) and
+      // writes it to its TMEM lane as bf16 pairs; all loads of a thread are in flight before the first use
+      const int vr = row0 + i * UA_ROWS + row;
+      uint4 qv[HD / 8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const int e = (tid & 255) + (i0 + k) * 256;
-          const int r = e / (HD / 8), dc = e - r * (HD / 8);   // r: row of the CTA's 256
-          const int vr = row0 + r;
-          qv[k] = make_uint4(0, 0, 0, 0);
-          if (vr < n_rows) {
-            const int qi = vr / G, g = vr - qi * G;
-            qv[k] = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
-          }
-        }
+      for (int w = 0; w < HD / 8; ++w) qv[w] = make_uint4(0, 0, 0, 0);
+      if (vr < n_rows) {
+        const int qi = vr / G, g = vr - qi * G;
+        const uint4* src = reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const int e = (tid & 255) + (i0 + k) * 256;
-          const int r = e / (HD / 8), dc = e - r * (HD / 8);
-          *reinterpret_cast<uint4*>(base_gen + (r >> 7) * SM::Q_TILE + tile_off<UA_ROWS>(r & 127, dc)) = qv[k];
-        }
+        for (int w = 0; w < HD / 8; ++w) qv[w] = __ldcg(src + w);
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic stores -> MMA reads of shared memory
-      mbar_arrive(smem_u32(&q_bar));
+#pragma unroll
+      for (int c = 0; c < HD / 2; c += 32) {
+        uint32_t r[32];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+          r[4 * w] = qv[c / 4 + w].x;
+          r[4 * w + 1] = qv[c / 4 + w].y;
+          r[4 * w + 2] = qv[c / 4 + w].z;
+          r[4 * w + 3] = qv[c / 4 + w].w;
+        }
+        tmem_st32(tmem + row_lane + SM::Q_COL + (uint32_t)(i * (HD / 2) + c), r);  // waits for the store
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&q_bar));
     }
-    if (gtid == 0 && i == 0) timeline_mark(1);  // Q staged (or requested)
+    if (gtid == 0 && i == 0) timeline_mark(1);  // Q in tensor memory
 
     constexpr float RESCALE_STEP = 8.f;  // log2 units a row's maximum may exceed its reference before O is rescaled
     // m_ref: the maximum the exponentials of this row refer to; it follows the true running maximum lazily (O in
     // TMEM is only rescaled when the maximum has grown by more than RESCALE_STEP, which keeps every exponential
     // below 2^8)
     float m_ref = -INFINITY, l_run = 0.f;
-    uint8_t* p_gen = base_gen + UA_TILES * SM::Q_TILE + UA_STAGES * SM::STAGE + i * SM::P_TILE;
     if (i < live) {
       for (int t = 0; t < n_tiles; ++t) {
-        ok = mbar_wait(smem_u32(&s_full[i][t & 1]), (uint32_t)(t >> 1) & 1u, abortp);
-        ok = __all_sync(0xffffffffu, ok);  // the TMEM accesses below are warp-collective: the warp stays together
+        ok = mbar_wait(smem_u32(&s_full[i]), (uint32_t)t & 1u, abortp);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (gtid == 0 && i == 0) timeline_mark(2 + (t < 5 ? t : 5));  // scores of tile t complete
@@ -308,7 +289,6 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
         float mx;
         {
           uint32_t r0[32], r1[32];  // both loads in flight, one wait
-          const uint32_t s_col = (uint32_t)((i * 2 + (t & 1)) * UA_KEYS);
           tmem_ld32(tmem + row_lane + s_col, r0);
           tmem_ld32(tmem + row_lane + s_col + 32u, r1);
           tmem_ld_wait();
@@ -329,7 +309,6 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
         }
         // ---- lazy rescale of O (warp-uniform branch: the TMEM accesses are warp-collective)
         const bool grow = mx > m_ref + RESCALE_STEP;
-        bool pv_waited = t == 0;  // O_i += P_i V of tile t-1 known to be complete (nothing to wait for at tile 0)
         if (__any_sync(0xffffffffu, grow)) {
           const float corr = grow ? exp2f(m_ref - mx) : 1.f;  // first tile: exp2(-inf) = 0, O is not read (t == 0)
           if (grow) {
@@ -337,11 +316,6 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
             l_run *= corr;
           }
           if (t > 0) {
-            ok = mbar_wait(smem_u32(&pv_done[i]), (uint32_t)(t - 1) & 1u, abortp);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            pv_waited = true;
 #pragma unroll
             for (int c = 0; c < HD; c += 32) {
               uint32_t r[32];
@@ -353,32 +327,23 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
             }
           }
         }
-        // ---- probabilities (bf16, packed) ...
+        // ---- probabilities -> tensor memory as bf16 pairs (the A operand of O_i += P_i V), over the first 32 of
+        // the columns this thread has just read its scores from
         float p_sum4[4] = {0.f, 0.f, 0.f, 0.f};
-        uint4 pk[UA_KEYS / 8];
+        uint32_t pk[UA_KEYS / 2];
 #pragma unroll
-        for (int c8 = 0; c8 < UA_KEYS / 8; ++c8) {
-          float pv[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            pv[j] = fast_exp2(fmaf(sv[c8 * 8 + j], scale_log2, -m_ref));
-            p_sum4[j & 3] += pv[j];
-          }
-          pk[c8] = make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
+        for (int c2 = 0; c2 < UA_KEYS / 2; ++c2) {
+          const float p0 = fast_exp2(fmaf(sv[2 * c2], scale_log2, -m_ref));
+          const float p1 = fast_exp2(fmaf(sv[2 * c2 + 1], scale_log2, -m_ref));
+          p_sum4[c2 & 1] += p0;
+          p_sum4[2 + (c2 & 1)] += p1;
+          pk[c2] = pack_bf16(p0, p1);
         }
         l_run += (p_sum4[0] + p_sum4[1]) + (p_sum4[2] + p_sum4[3]);
-        // ... -> shared memory in the layout of an MMA A operand (one 128-byte row per tile row), once the
-        // product that read the previous tile's probabilities has completed
-        if (!pv_waited) {
-          ok = mbar_wait(smem_u32(&pv_done[i]), (uint32_t)(t - 1) & 1u, abortp);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-        }
-#pragma unroll
-        for (int c8 = 0; c8 < UA_KEYS / 8; ++c8) *reinterpret_cast<uint4*>(p_gen + tile_off<UA_ROWS>(row, c8)) = pk[c8];
+        tmem_st32(tmem + row_lane + s_col, pk);  // waits for the store
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(smem_u32(&p_full[i]));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&p_full[i]));
       }
       if (ok) ok = mbar_wait(smem_u32(&o_full[i]), 0u, abortp);
       ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below are warp-collective
@@ -435,8 +400,7 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
 }
 
 template <int HD>
-cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const CUtensorMap& tmQ,
-                        int q_by_tma, const void* q, void* o,
+cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
                         float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
   constexpr int SMEM = (int)UaSmem<HD>::TOTAL;
   static DeviceOnce once;
@@ -449,7 +413,7 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
   float* ml_part = scratch ? scratch + (size_t)S * total * HD : nullptr;
   dim3 grid((a_seq * G + UA_TILES * UA_ROWS - 1) / (UA_TILES * UA_ROWS), Hkv, B * S);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
-  cudaError_t e = launch_k(L, attn_umma_kernel<HD>, grid, dim3(UA_THREADS), SMEM, tmK, tmV, tmQ, q_by_tma, (const __nv_bfloat16*)q,
+  cudaError_t e = launch_k(L, attn_umma_kernel<HD>, grid, dim3(UA_THREADS), SMEM, tmK, tmV, (const __nv_bfloat16*)q,
                            (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split, scale_log2,
                            L.d_status);
   L.count();
@@ -503,12 +467,8 @@ cudaError_t launch_attention_umma(const Launch& L, const void* q, const void* Kc
       !get_tensor_map_3d(Vc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, 64, &tmV))
     return cudaErrorInvalidValue;
   if (S_out) *S_out = p.S;
-  // with one query head per KV head a row tile is 128 consecutive rows of q: fetched by TMA
-  CUtensorMap tmQ = tmK;
-  const int q_by_tma = H == Hkv && ((uintptr_t)q & 15) == 0 &&
-                       get_tensor_map_2d(q, (uint64_t)B * a_seq, (uint64_t)H * hd, UA_ROWS, &tmQ);
-  return hd == 64 ? launch_umma<64>(L, tmK, tmV, tmQ, q_by_tma, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
-                  : launch_umma<128>(L, tmK, tmV, tmQ, q_by_tma, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
+  return hd == 64 ? launch_umma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
+                  : launch_umma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
 }
 
 }  // namespace dllm

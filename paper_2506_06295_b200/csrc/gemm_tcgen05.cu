@@ -29,9 +29,11 @@
 // Every wait on an mbarrier is bounded (2 s of %globaltimer); on expiry the
 // CTA records a code in the status word, skips its epilogue, lets copies in
 // flight land, frees its TMEM and returns.
+#include <algorithm>
 #include <mutex>
 #include <unordered_map>
 
+#include "../../include/dllm.h"
 #include "internal.h"
 #include "tma.cuh"
 #include "umma.cuh"
@@ -60,14 +62,24 @@ struct SmemLayout {
   static constexpr uint32_t total(int stages) { return (uint32_t)stages * STAGE_BYTES + 1024; }  // + slack to align the base to 1024
 };
 
-// Epilogue of one CTA (128 threads, all of them): its accumulator, TMEM lanes = 128 weight rows from n0 (tile
-// number tile_y), columns = BN activation rows from m0, goes to the fp32 slab (coalesced: lane = output column)
-// or, with act_out, through the SwiGLU combination.  `ex`: at least min(BN, 64) * 528 bytes of shared memory
-// that nothing else uses any more.
-template <int BN>
-__device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0, int n0, int tile_y, int M, int N,
-                                              float* __restrict__ slab, __nv_bfloat16* __restrict__ act_out, int m_ffn) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+// Epilogue of one tile by 128 threads: the accumulator, TMEM lanes = 128 weight rows from n0 (tile number
+// tile_y), columns = BN activation rows from m0, goes to the fp32 slab (coalesced: lane = output column) or,
+// with act_out, through the SwiGLU combination.  `ex`: at least min(BN, 64) * 528 bytes of shared memory that
+// nothing else uses meanwhile.  tl = 0..127 identifies the thread: it works on TMEM lane tl, so its warp must be
+// the one allowed to touch lanes 32 * (tl / 32) .. + 31 (warp index % 4 == tl / 32).  NAMED_BAR == 0: the 128
+// threads are the whole CTA (__syncthreads); otherwise they meet on that named barrier.
+template <int NAMED_BAR>
+__device__ __forceinline__ void epilogue_sync() {
+  if constexpr (NAMED_BAR == 0)
+    epilogue_sync<NAMED_BAR>();
+  else
+    asm volatile("bar.sync %0, 128;" ::"n"(NAMED_BAR) : "memory");
+}
+template <int BN, int NAMED_BAR = 0>
+__device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int tl, int m0, int n0, int tile_y, int M,
+                                              int N, float* __restrict__ slab, __nv_bfloat16* __restrict__ act_out,
+                                              int m_ffn) {
+  const int warp = tl >> 5, lane = tl & 31;
   if (m_ffn < 0) {
     // Estimate epilogue of the LM head (no split-K, act_out == nullptr, m_ffn = -1 - mask id): instead of 128
     // logits per row the CTA writes one record per activation row, {max, sum exp(v - max), argmax, -} over its
@@ -78,7 +90,7 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0
     constexpr int CH = BN < 64 ? BN : 64;
     const int mask_id = -1 - m_ffn, n_tiles = (N + TILE_W - 1) / TILE_W;
     float4* rec = reinterpret_cast<float4*>(slab);
-    const int rr = threadIdx.x >> 1, half = threadIdx.x & 1;
+    const int rr = tl >> 1, half = tl & 1;
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += CH) {
       if (m0 + c0 >= M) break;  // uniform across the CTA
@@ -90,9 +102,9 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0
 #pragma unroll
         for (int c = 0; c < CH; c += 16)
 #pragma unroll
-          for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[c / 16][j]);
+          for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + tl] = __uint_as_float(r[c / 16][j]);
       }
-      __syncthreads();
+      epilogue_sync<NAMED_BAR>();
       MaxSum t{-INFINITY, 0.f, 0x7fffffff};
       if (rr < CH) {
         // two passes over the thread's 64 columns: maximum and its first index, then the exponentials as four
@@ -135,7 +147,7 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0
       const int m = m0 + c0 + rr;
       if (rr < CH && half == 0 && m < M)
         rec[(size_t)m * n_tiles + tile_y] = make_float4(t.m, t.s, __int_as_float(t.a), 0.f);
-      __syncthreads();
+      epilogue_sync<NAMED_BAR>();
     }
   } else if (act_out) {
     // SwiGLU epilogue (no split-K): the tile's 128 weight rows are 64 gate rows followed by the 64 up rows
@@ -145,7 +157,7 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     constexpr int EXS = 132;   // floats per staged row: 16-byte aligned, rows 4 banks apart
     constexpr int CH = BN < 64 ? BN : 64;
-    const int q = threadIdx.x & 15, rsub = threadIdx.x >> 4;  // 4 FFN columns, 8 rows per pass
+    const int q = tl & 15, rsub = tl >> 4;  // 4 FFN columns, 8 rows per pass
     const int col = tile_y * 64 + 4 * q;
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += CH) {
@@ -158,9 +170,9 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0
 #pragma unroll
         for (int c = 0; c < CH; c += 16)
 #pragma unroll
-          for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + threadIdx.x] = __uint_as_float(r[c / 16][j]);
+          for (int j = 0; j < 16; ++j) ex[(c + j) * EXS + tl] = __uint_as_float(r[c / 16][j]);
       }
-      __syncthreads();
+      epilogue_sync<NAMED_BAR>();
 #pragma unroll
       for (int rr = rsub; rr < CH; rr += 8) {
         const int m = m0 + c0 + rr;
@@ -175,7 +187,7 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int m0
           *reinterpret_cast<uint2*>(act_out + (size_t)m * m_ffn + col) = pk;
         }
       }
-      __syncthreads();
+      epilogue_sync<NAMED_BAR>();
     }
   } else {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -336,7 +348,8 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   if (act_out || m_ffn < 0) warp_ok = __syncthreads_and(warp_ok);  // these epilogues exchange data between warps
   if (warp_ok) {
     float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // the drained ring
-    gemm_epilogue<BN>(tmem_d, ex, m0, n0, nt, M, N, part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
+    gemm_epilogue<BN>(tmem_d, ex, (int)threadIdx.x, m0, n0, nt, M, N, part + (size_t)blockIdx.z * split_stride, act_out,
+                      m_ffn);
     if (threadIdx.x == 0) timeline_mark(4);            // this thread's part of the epilogue written
   } else {
     drain_delay();  // gave up: let copies in flight land before shared memory is released
@@ -345,6 +358,185 @@ __global__ void __launch_bounds__(128) gemm_bf16_tcgen05_kernel(const __grid_con
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"((uint32_t)BN) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- persistent kernel (many tiles, no split-K)
+// The same product for shapes with more tiles than SMs (many active rows: batched serving, full steps): one
+// CTA per SM walks through tiles blockIdx.x, blockIdx.x + gridDim.x, ... with fixed roles -- warp 0 requests
+// the operand tiles of one tile after the other without a gap, warp 1 issues the MMAs into one of TWO
+// accumulators in tensor memory, warps 2-5 run the epilogue of the accumulator that has just been completed --
+// so the epilogue of a tile (TMEM -> registers -> global, or the SwiGLU / estimate forms) runs under the main
+// loop of the next one and the operand stream never drains between tiles.  Tile order is the launch order of
+// the one-tile kernel including its remap, so CTAs that run together share operands in L2.  The k loop of a
+// tile is the same as in the one-tile kernel: results are bit-identical to it.
+constexpr int PERSIST_THREADS = 192;
+template <int BN>
+struct PersistLayout {
+  static constexpr uint32_t STAGE_BYTES = W_STAGE_BYTES + BN * TILE_K * 2;
+  static constexpr uint32_t EX_BYTES = 64 * 132 * 4;  // staging of the SwiGLU / estimate epilogues
+  static constexpr uint32_t total(int stages, bool staged) {
+    return (uint32_t)stages * STAGE_BYTES + (staged ? EX_BYTES : 0) + 1024;
+  }
+};
+
+template <int BN>
+__global__ void __launch_bounds__(PERSIST_THREADS, 1)
+    gemm_bf16_persistent_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmA,
+                                float* __restrict__ part, int M, int N, int num_kb, int m_tiles, int n_tiles,
+                                int STAGES, __nv_bfloat16* __restrict__ act_out, int m_ffn, int* __restrict__ status) {
+  using PL = PersistLayout<BN>;
+  static_assert(2 * BN <= 512, "two accumulators must fit the 512 columns of tensor memory");
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
+  __shared__ __align__(8) uint64_t acc_full[2], acc_empty[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tiles_s = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  float* ex = reinterpret_cast<float*>(smem_raw + (tiles_s - smem_u32(smem_raw)) + (size_t)STAGES * PL::STAGE_BYTES);
+  const int total_tiles = m_tiles * n_tiles;
+  // tile L of the walk -> (activation tile, weight tile): groups of RASTER activation tiles, weight tiles inside
+  auto tile_of = [&](int L, int& mt, int& nt) {
+    const int per = RASTER * n_tiles, grp = L / per, within = L - grp * per;
+    const int wide = min(RASTER, m_tiles - grp * RASTER);
+    nt = within / wide;
+    mt = grp * RASTER + within - nt * wide;
+  };
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&acc_full[a]), 1);
+      mbar_init(smem_u32(&acc_empty[a]), 128);  // every epilogue thread arrives once it has read its part
+    }
+    mbar_fence_init();
+    prefetch_tensormap(&tmW);
+    prefetch_tensormap(&tmA);
+  }
+  if (warp == 1) {  // TMEM: two accumulators of BN fp32 columns x 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"((uint32_t)(2 * BN))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_d = tmem_base_slot;
+  volatile int* abortp = &abort_flag;
+  pdl_wait();     // the activation rows and the output buffer belong to the preceding kernels
+  pdl_trigger();
+  bool ok = true;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      for (int L = blockIdx.x; L < total_tiles && ok; L += gridDim.x) {
+        int mt, nt;
+        tile_of(L, mt, nt);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abortp)) {
+            if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+            ok = false;
+            break;
+          }
+          const uint32_t fb = smem_u32(&full_bar[s]);
+          const uint32_t dst = tiles_s + s * PL::STAGE_BYTES;
+          mbar_expect_tx(fb, PL::STAGE_BYTES);
+          tma_load_2d(dst, &tmW, fb, kb * TILE_K, nt * TILE_W);
+          tma_load_2d(dst + W_STAGE_BYTES, &tmA, fb, kb * TILE_K, mt * BN);
+          if (++s == STAGES) {
+            s = 0;
+            ph ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(TILE_W, BN);
+      int s = 0, j = 0;
+      uint32_t ph = 0;
+      for (int L = blockIdx.x; L < total_tiles && ok; L += gridDim.x, ++j) {
+        const int a = j & 1;
+        // the epilogue of the tile that used this accumulator two tiles ago has read it
+        if (!mbar_wait(smem_u32(&acc_empty[a]), ((uint32_t)(j >> 1) & 1u) ^ 1u, abortp)) {
+          if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_MMA);
+          ok = false;
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp)) {
+            if (status) atomicCAS(status, ST_OK, ST_TIMEOUT_MMA);
+            ok = false;
+            break;
+          }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t sW = tiles_s + s * PL::STAGE_BYTES;
+          const uint64_t dW = make_smem_desc(sW);
+          const uint64_t dA = make_smem_desc(sW + W_STAGE_BYTES);
+#pragma unroll
+          for (int k = 0; k < TILE_K / UMMA_K; ++k)
+            umma_bf16(tmem_d + (uint32_t)(a * BN), dW + (uint64_t)(2 * k), dA + (uint64_t)(2 * k), idesc,
+                      (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&empty_bar[s]));  // stage reusable once these MMAs have read it
+          if (++s == STAGES) {
+            s = 0;
+            ph ^= 1u;
+          }
+        }
+        if (ok) umma_commit(smem_u32(&acc_full[a]));
+      }
+    }
+  } else {
+    // ---------------- epilogue warps 2..5: TMEM lanes 32 * (warp % 4) .. + 31 ----------------
+    const int tl = (warp & 3) * 32 + lane;
+    int j = 0;
+    for (int L = blockIdx.x; L < total_tiles; L += gridDim.x, ++j) {
+      const int a = j & 1;
+      int mt, nt;
+      tile_of(L, mt, nt);
+      bool have = mbar_wait(smem_u32(&acc_full[a]), (uint32_t)(j >> 1) & 1u, abortp);
+      // the 128 epilogue threads agree (the TMEM loads are warp-collective and the staged forms exchange data)
+      {
+        uint32_t r;
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.ne.u32 q, %1, 0;\n\t"
+            "bar.red.and.pred p, 1, 128, q;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(r)
+            : "r"((uint32_t)have)
+            : "memory");
+        have = r != 0;
+      }
+      if (!have) {
+        if (tl == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_EPI);
+        ok = false;
+        break;
+      }
+      gemm_epilogue<BN, 1>(tmem_d + (uint32_t)(a * BN), ex, tl, mt * BN, nt * TILE_W, nt, M, N, part, act_out, m_ffn);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      mbar_arrive(smem_u32(&acc_empty[a]));
+    }
+  }
+  ok = __syncthreads_and(ok);
+  if (!ok) drain_delay();  // gave up: let copies in flight land before shared memory is released
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"((uint32_t)(2 * BN)) : "memory");
   }
 }
 
@@ -480,7 +672,8 @@ __global__ void __launch_bounds__(128) gemm_bf16_pair_kernel(const __grid_consta
   if (act_out || m_ffn < 0) warp_ok = __syncthreads_and(warp_ok);
   if (warp_ok) {
     float* ex = reinterpret_cast<float*>(smem_raw + (tiles - smem_u32(smem_raw)));  // the drained ring
-    gemm_epilogue<BN>(tmem_d, ex, m0, n0, (int)blockIdx.x, M, N, part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
+    gemm_epilogue<BN>(tmem_d, ex, (int)threadIdx.x, m0, n0, (int)blockIdx.x, M, N,
+                      part + (size_t)blockIdx.z * split_stride, act_out, m_ffn);
   } else {
     drain_delay();
   }
@@ -581,6 +774,28 @@ cudaError_t launch_one(const Launch& L, const CUtensorMap& tmW, const CUtensorMa
 }
 
 template <int BN>
+cudaError_t launch_persistent(const Launch& L, const CUtensorMap& tmW, const CUtensorMap& tmA, float* part, int M,
+                              int N, int num_kb, const GemmPlan& plan, void* act_out, int m_ffn) {
+  using PL = PersistLayout<BN>;
+  const bool staged = act_out != nullptr || m_ffn < 0;
+  const int fit = (227 * 1024 - 1024 - 512 - (staged ? (int)PL::EX_BYTES : 0)) / (int)PL::STAGE_BYTES;
+  const int stages = fit < MAX_STAGES ? fit : MAX_STAGES;
+  static DeviceOnce once;
+  cudaError_t e0 = once.run([] {
+    return cudaFuncSetAttribute(gemm_bf16_persistent_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                227 * 1024 - 512);
+  });
+  if (e0 != cudaSuccess) return e0;
+  const int n_tiles = (N + TILE_W - 1) / TILE_W, m_tiles = (M + BN - 1) / BN;
+  const int ctas = std::min(m_tiles * n_tiles, sm_count());
+  cudaError_t e = launch_k(L, gemm_bf16_persistent_kernel<BN>, dim3(ctas), dim3(PERSIST_THREADS),
+                           PL::total(stages, staged), tmW, tmA, part, M, N, num_kb, m_tiles, n_tiles, stages,
+                           (__nv_bfloat16*)act_out, m_ffn, L.d_status);
+  L.count();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+template <int BN>
 cudaError_t launch_pair(const Launch& L, const CUtensorMap& tmW, const CUtensorMap& tmA, float* part, int M, int N,
                         int num_kb, const GemmPlan& plan, void* act_out, int m_ffn) {
   using PL = PairLayout<BN>;
@@ -626,6 +841,10 @@ int sm_count() {
   return v;
 }
 
+// tuning / test override of the kernel choice for unsplit plans with 256-row tiles: 0 automatic, 1 always the
+// persistent kernel, -1 never (see dllm_debug_gemm_plan)
+int g_gemm_force_persistent = 0;
+
 Partials make_partials(const float* p, int M, int N, const GemmPlan& plan) {
   return Partials{p, (size_t)M * N, plan.S_max, N};  // every element has S_max slabs
 }
@@ -633,7 +852,8 @@ Partials make_partials(const float* p, int M, int N, const GemmPlan& plan) {
 // Tile shape, ring depth and split-K factor, from sweeps on B200: up to 256
 // activation rows the product is bound by streaming W, so k ranges are split
 // until at least one CTA per SM (two with 128-row tiles) streams weights.
-GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, int force_bn, int force_pair) {
+GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, int force_bn, int force_pair,
+                        int force_persistent) {
   GemmPlan p;
   const int sms = sm_count();
   const long n_tiles = (N + TILE_W - 1) / TILE_W;
@@ -667,6 +887,10 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
   if (S < 1) S = 1;
   if (p.pair && force_pair == 0) S = 1;
   if (force_split > 0) S = force_split < p.num_kb ? force_split : p.num_kb;
+  // more tiles than SMs, no split, one-CTA 256-row tiles: the persistent kernel (epilogue under the next main loop)
+  if (force_persistent == 0) force_persistent = g_gemm_force_persistent;
+  p.persistent = (force_persistent >= 0) && !p.pair && p.BN == 256 && S == 1 &&
+                 (force_persistent > 0 || tiles > sms);
   p.upc = (p.num_kb + S - 1) / S;                 // k-blocks per split
   p.S_max = (p.num_kb + p.upc - 1) / p.upc;       // no empty split
   p.ctas = (int)tiles * p.S_max;
@@ -706,6 +930,7 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
     return plan.BN == 128 ? launch_pair<128>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn)
                           : launch_pair<256>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
   }
+  if (plan.persistent) return launch_persistent<256>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
   switch (plan.BN) {
     case 32: return launch_one<32>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
     case 64: return launch_one<64>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
@@ -722,6 +947,15 @@ cudaError_t set_debug_skip_act_load(int enable) {
   return cudaMemcpyToSymbol(g_debug_skip_act_load, &v, sizeof v);
 }
 }  // namespace dllm
+
+extern "C" dllm_status dllm_debug_gemm_plan(int persistent) {
+  if (persistent < -1 || persistent > 1) {
+    dllm::set_last_error("dllm_debug_gemm_plan: -1, 0 or 1");
+    return DLLM_INVALID_ARG;
+  }
+  dllm::g_gemm_force_persistent = persistent;
+  return DLLM_OK;
+}
 
 DLLM_TIMELINE_HOOKS(gemm_tcgen05)
 DLLM_WAIT_LIMIT_HOOK(gemm_tcgen05)

@@ -193,10 +193,12 @@ struct GemmPlan {
   int ctas;         // grid size
   int S_max;        // split-K factor: slabs per output element
   int pair = 0;     // 1: CTA pairs (cta_group::2) share the activation tile of BN rows
+  int persistent = 0;  // 1: one CTA per SM walks through the tiles, epilogue under the next tile's main loop
 };
 // 0 = auto.  force_pair: 0 auto, 1 CTA pairs (BN 128 or 256, N a multiple of 256), -1 never.
+// force_persistent: 0 auto, 1 the persistent kernel (unsplit plans with 256-row tiles only), -1 never.
 GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split = 0, int force_stages = 0, int force_bn = 0,
-                        int force_pair = 0);
+                        int force_pair = 0, int force_persistent = 0);
 Partials make_partials(const float* p, int M, int N, const GemmPlan& plan);
 // Returns cudaSuccess or the failing error.  part must hold S*M*N floats.
 // act_out != nullptr (unsplit plan, W = gate / up rows interleaved in blocks of 64, N = 2 * m_ffn): instead of
@@ -230,7 +232,8 @@ struct AttnChoice {
   AttnPlan plan{1, 0, 0};
 };
 AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats);
-extern int g_attn_force_splits;  // tuning override of both plans' split count (0 = automatic)
+extern int g_attn_force_splits;   // tuning override of both plans' split count (0 = automatic)
+extern int g_attn_umma_min_rows;  // rows per KV head from which the tcgen05 kernel is taken
 // bf16 with head_dim 64 / 128 runs on the tensor cores (scratch holds the
 // partials of split key ranges; without it one split is used); everything else
 // on the plain-ALU kernel.

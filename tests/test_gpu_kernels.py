@@ -187,6 +187,32 @@ def test_attention(env, case, dtype):
         assert rel_l2(got[b * a:(b + 1) * a], want) < tol
 
 
+@pytest.mark.parametrize("M,N,K", [(520, 7680, 320), (4400, 1280, 200), (300, 20000, 64)])
+def test_gemm_persistent_kernel_is_bit_identical_to_the_one_tile_kernel(env, M, N, K):
+    """Unsplit products with more tiles than SMs run on the persistent kernel (one CTA per SM walks through the
+    tiles, two accumulators, epilogue under the next main loop).  Same k loop per tile: the same bits as the
+    one-tile-per-CTA kernel, for the plain epilogue and for the SwiGLU epilogue; ragged activation tiles, a ragged
+    k block, more than 16 activation tiles (the launch-order remap), fewer tiles than SMs."""
+    torch, dllm = env
+    A = torch.from_numpy(synth.round_to_bf16(synth.random_normal((M, K), seed=21))).cuda().to(torch.bfloat16)
+    W = torch.from_numpy(synth.round_to_bf16(synth.random_normal((N, K), seed=22, std=0.05))).cuda().to(torch.bfloat16)
+    out = {}
+    try:
+        for mode in (-1, 1):
+            dllm._check(dllm.lib.dllm_debug_gemm_plan(mode))
+            c = dllm.gemm_bf16_planned(A, W, act_tile=256, splits=1)
+            g = dllm.ffn_gate_up_bf16(A, W[:N // 128 * 128], act_tile=256) if K % 8 == 0 else None
+            torch.cuda.synchronize()
+            out[mode] = (c.cpu().numpy(), g.float().cpu().numpy())
+    finally:
+        dllm._check(dllm.lib.dllm_debug_gemm_plan(0))
+    dllm.kernel_status()
+    want = A.double().cpu().numpy() @ W.double().cpu().numpy().T
+    assert rel_l2(out[1][0], want) < 1e-5
+    assert np.array_equal(out[-1][0], out[1][0])
+    assert np.array_equal(out[-1][1], out[1][1])
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("B,R,width,k", [(1, 32, 256, 8), (3, 256, 4096, 64), (2, 100, 512, 50), (1, 512, 4096, 51),
                                          # the longest response the selection kernel admits (keys and flags of one
