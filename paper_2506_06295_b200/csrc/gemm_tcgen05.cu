@@ -71,7 +71,7 @@ struct SmemLayout {
 template <int NAMED_BAR>
 __device__ __forceinline__ void epilogue_sync() {
   if constexpr (NAMED_BAR == 0)
-    epilogue_sync<NAMED_BAR>();
+    __syncthreads();
   else
     asm volatile("bar.sync %0, 128;" ::"n"(NAMED_BAR) : "memory");
 }
