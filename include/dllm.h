@@ -323,12 +323,14 @@ dllm_status dllm_debug_set_wait_limit_ns(uint64_t ns);
  * kernels give bit-identical results. */
 dllm_status dllm_debug_gemm_plan(int persistent);
 /* Tuning hook: overrides, for every later call in this process, the number of
- * key-range splits the tensor-core attention kernels take (0 = automatic) and,
- * if tcgen05_min_rows > 0, the number of (query, head-of-group) rows per KV head
+ * key-range splits the tensor-core attention kernels take (0 = automatic); if
+ * tcgen05_min_rows > 0, the number of (query, head-of-group) rows per KV head
  * from which the 128-row tcgen05 kernel is taken instead of the 64-row mma.sync
- * kernel.  Results stay within the attention tolerance; the merge order changes
- * with the plan. */
-dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows);
+ * kernel; and whether shapes with at most 32 rows per KV head and at least 1024
+ * keys take the few-rows kernel (warps share the rows and split the key tiles;
+ * 1, the default) or stay on the 64-row kernel (0).  Results stay within the
+ * attention tolerance; the merge order changes with the plan. */
+dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows, int few_rows_kernel);
 dllm_status dllm_debug_skip_one_load(int enable);
 /* C[M,N] (fp32, row-major, DEVICE) = A[M,K] * W[N,K]^T with bf16 operands on
  * the tensor cores (tcgen05 + TMA).  d_partials is scratch of

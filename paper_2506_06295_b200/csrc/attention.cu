@@ -152,6 +152,195 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ C
   if (!ok && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
 }
 
+// ============================================================================
+// attn_mma_few_kernel (bf16): the same attention when a KV head has at most 16 * RG (query, head-of-group) rows
+// (RG = 1 or 2: a few selected rows against a long prompt).  A CTA holds RG * KW warps: warp (rg, kw) works on
+// rows 16 rg .. 16 rg + 15 and on the key tiles kw, kw + KW, ... of the CTA's split, so KW tiles are in the
+// load -> QK^T -> softmax -> PV chain at once instead of one; every way kw has its own one-stage K/V buffer and
+// barrier, refilled by its first warp.  The ways are merged through shared memory in way order.  Splits over
+// CTAs, partials and the merge kernel as in attn_mma_kernel.
+// ============================================================================
+template <int HD, int RG, int KW>
+__global__ void __launch_bounds__(32 * RG * KW, RG == 2 ? 2 : 1)
+    attn_mma_few_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                        const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ o,
+                        float* __restrict__ o_part, float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv,
+                        int S, int keys_per_split, float scale_log2, int* __restrict__ status) {
+  constexpr uint32_t Q_BYTES = AT_ROWS * HD * 2;          // the tile layout of the 64-row kernel; RG * 16 rows used
+  constexpr uint32_t TILE_BYTES = AT_KEYS * HD * 2, STAGE_BYTES = 2 * TILE_BYTES;
+  constexpr int ROWS = 16 * RG, NT = 32 * RG * KW, PANELS = HD / 64;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[KW];
+  __shared__ float ml_s[KW > 1 ? KW - 1 : 1][RG][32][4];
+  __shared__ int abort_flag;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_gen = smem_raw + (base - smem_u32(smem_raw));
+  const int warp = (int)threadIdx.x >> 5, lane = (int)threadIdx.x & 31;
+  const int rg = warp % RG, kw = warp / RG;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int w = 0; w < KW; ++w) mbar_init(smem_u32(&full_bar[w]), 1);
+    mbar_fence_init();
+    prefetch_tensormap(&tmK);
+    prefetch_tensormap(&tmV);
+  }
+  __syncthreads();
+  pdl_wait();  // K, V and Q come from the preceding kernels
+  pdl_trigger();
+
+  const int G = H / Hkv, kh = blockIdx.y;
+  const int b = blockIdx.z / S, split = blockIdx.z - b * S;
+  const int row0 = blockIdx.x * ROWS, n_rows = a_seq * G, dq = H * HD;
+  const int key_lo = split * keys_per_split, key_hi = min(n, key_lo + keys_per_split);
+  const int n_tiles = (key_hi - key_lo + AT_KEYS - 1) / AT_KEYS;   // >= 1 by construction of the plan
+  const uint32_t q_s = base, kv_s = base + Q_BYTES + (uint32_t)kw * STAGE_BYTES;
+  volatile int* abortp = &abort_flag;
+
+  auto issue = [&](int t) {  // key tile t of the split into this way's buffer
+    const uint32_t fb = smem_u32(&full_bar[kw]);
+    mbar_expect_tx(fb, STAGE_BYTES);
+    const int key0 = key_lo + t * AT_KEYS;
+#pragma unroll
+    for (int p = 0; p < PANELS; ++p) {
+      tma_load_3d(kv_s + p * (AT_KEYS * 128), &tmK, fb, kh * HD + p * 64, key0, b);
+      tma_load_3d(kv_s + TILE_BYTES + p * (AT_KEYS * 128), &tmV, fb, kh * HD + p * 64, key0, b);
+    }
+  };
+  if (rg == 0 && lane == 0 && kw < n_tiles) issue(kw);
+  // Q rows of the tile: 16-byte loads into the swizzled layout (rows past the end are zero)
+  {
+    constexpr int CHUNKS = ROWS * (HD / 8);
+    constexpr int PER = (CHUNKS + NT - 1) / NT;
+    uint4 qv[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int e = (int)threadIdx.x + i * NT;
+      const int r = e / (HD / 8), dc = e - r * (HD / 8);
+      const int vr = row0 + r;
+      qv[i] = make_uint4(0, 0, 0, 0);
+      if (e < CHUNKS && vr < n_rows) {
+        const int qi = vr / G, g = vr - qi * G;
+        qv[i] = __ldcg(reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD + dc * 8));
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int e = (int)threadIdx.x + i * NT;
+      const int r = e / (HD / 8), dc = e - r * (HD / 8);
+      if (e < CHUNKS) *reinterpret_cast<uint4*>(base_gen + tile_off<AT_ROWS>(r, dc)) = qv[i];
+    }
+  }
+  __syncthreads();
+
+  AttnAcc<HD> acc;
+  attn_acc_clear(acc);
+  bool ok = true;
+  int it = 0;
+  for (int t = kw; t < n_tiles; t += KW, ++it) {
+    ok = mbar_wait(smem_u32(&full_bar[kw]), (uint32_t)it & 1u, abortp);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) break;
+    attn_warp_tile<HD>(lane, rg, q_s, kv_s, kv_s + TILE_BYTES, key_lo + t * AT_KEYS, key_hi, scale_log2, acc);
+    if (t + KW < n_tiles) {
+      // every warp of the way has read the buffer before its first warp asks for the next tile
+      if constexpr (RG > 1)
+        asm volatile("bar.sync %0, %1;" ::"r"(1 + kw), "n"(32 * RG) : "memory");
+      else
+        __syncwarp();
+      if (rg == 0 && lane == 0) issue(t + KW);
+    }
+  }
+  attn_warp_finish(acc);
+
+  // ---- merge of the ways, in way order, through each way's own (drained) buffer
+  if constexpr (KW > 1) {
+    float* o_s = reinterpret_cast<float*>(base_gen + Q_BYTES + (size_t)kw * STAGE_BYTES) + rg * (HD / 2) * 32;
+    if (kw > 0) {
+      if constexpr (RG > 1)
+        asm volatile("bar.sync %0, %1;" ::"r"(1 + kw), "n"(32 * RG) : "memory");  // the way is done with its tiles
+      else
+        __syncwarp();
+      if (ok) {
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) o_s[(i * 4 + c) * 32 + lane] = acc.o[i][c];
+        ml_s[kw - 1][rg][lane][0] = acc.m[0];
+        ml_s[kw - 1][rg][lane][1] = acc.m[1];
+        ml_s[kw - 1][rg][lane][2] = acc.l[0];
+        ml_s[kw - 1][rg][lane][3] = acc.l[1];
+      }
+    }
+    ok = __syncthreads_and(ok);
+    if (ok && kw == 0) {
+      float M[2] = {acc.m[0], acc.m[1]};
+#pragma unroll
+      for (int w = 1; w < KW; ++w) {
+        M[0] = fmaxf(M[0], ml_s[w - 1][rg][lane][0]);
+        M[1] = fmaxf(M[1], ml_s[w - 1][rg][lane][1]);
+      }
+      const float w0[2] = {exp2f(acc.m[0] - M[0]), exp2f(acc.m[1] - M[1])};  // way 0 always has a tile: finite
+      acc.l[0] *= w0[0];
+      acc.l[1] *= w0[1];
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i) {
+        acc.o[i][0] *= w0[0];
+        acc.o[i][1] *= w0[0];
+        acc.o[i][2] *= w0[1];
+        acc.o[i][3] *= w0[1];
+      }
+#pragma unroll
+      for (int w = 1; w < KW; ++w) {
+        const float* ow = reinterpret_cast<const float*>(base_gen + Q_BYTES + (size_t)w * STAGE_BYTES) + rg * (HD / 2) * 32;
+        const float ww[2] = {exp2f(ml_s[w - 1][rg][lane][0] - M[0]), exp2f(ml_s[w - 1][rg][lane][1] - M[1])};  // no tile: 0
+        acc.l[0] += ww[0] * ml_s[w - 1][rg][lane][2];
+        acc.l[1] += ww[1] * ml_s[w - 1][rg][lane][3];
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) acc.o[i][c] += ww[c >> 1] * ow[(i * 4 + c) * 32 + lane];
+      }
+      acc.m[0] = M[0];
+      acc.m[1] = M[1];
+    }
+  } else {
+    ok = __syncthreads_and(ok);
+  }
+  if (!ok) {
+    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+    drain_delay();
+    return;
+  }
+  if (kw != 0) return;
+
+  // ---- way 0 writes the CTA's rows: final output, or the split's unnormalised partial with (max, sum)
+#pragma unroll
+  for (int h2 = 0; h2 < 2; ++h2) {
+    const int vr = row0 + rg * 16 + (lane >> 2) + h2 * 8;
+    if (vr >= n_rows) continue;
+    const int qi = vr / G, g = vr - qi * G;
+    const size_t orow = ((size_t)b * a_seq + qi) * H + (kh * G + g);   // (row, head) index
+    if (S == 1) {
+      const float inv = 1.f / acc.l[h2];
+      __nv_bfloat16* dst = o + orow * HD + 2 * (lane & 3);
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i)
+        *reinterpret_cast<uint32_t*>(dst + i * 8) = pack_bf16(acc.o[i][2 * h2] * inv, acc.o[i][2 * h2 + 1] * inv);
+    } else {
+      const size_t total = (size_t)(gridDim.z / S) * a_seq * H;           // (row, head) pairs
+      float* dst = o_part + ((size_t)split * total + orow) * HD + 2 * (lane & 3);
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i)
+        *reinterpret_cast<float2*>(dst + i * 8) = make_float2(acc.o[i][2 * h2], acc.o[i][2 * h2 + 1]);
+      if ((lane & 3) == 0) {
+        float* ml = ml_part + ((size_t)split * total + orow) * 2;
+        ml[0] = acc.m[h2];
+        ml[1] = acc.l[h2];
+      }
+    }
+  }
+}
+
 // Merges the key-range splits: out = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s,
 // splits in index order.  One warp per (row, head); the (max, sum) pairs of all
 // splits are fetched together, then the partial outputs.
@@ -264,11 +453,40 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
 
 }  // namespace
 
+namespace {
+template <int HD, int RG, int KW>
+cudaError_t launch_few(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
+                       float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
+  constexpr int SMEM = AT_ROWS * HD * 2 + KW * 2 * AT_KEYS * HD * 2 + 1024;
+  static_assert(SMEM <= 227 * 1024, "the ways' buffers do not fit the shared memory of a CTA");
+  static_assert(RG * 32 * (HD / 2) * 4 <= 2 * AT_KEYS * HD * 2, "a way's buffer must hold its warps' outputs");
+  static DeviceOnce once;
+  cudaError_t e0 = once.run([] {
+    return cudaFuncSetAttribute(attn_mma_few_kernel<HD, RG, KW>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+  });
+  if (e0 != cudaSuccess) return e0;
+  const int G = H / Hkv;
+  const size_t total = (size_t)B * a_seq * H;
+  float* o_part = scratch;
+  float* ml_part = scratch ? scratch + (size_t)S * total * HD : nullptr;
+  dim3 grid((a_seq * G + 16 * RG - 1) / (16 * RG), Hkv, B * S);
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+  cudaError_t e = launch_k(L, attn_mma_few_kernel<HD, RG, KW>, grid, dim3(32 * RG * KW), SMEM, tmK, tmV,
+                           (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S,
+                           keys_per_split, scale_log2, L.d_status);
+  L.count();
+  if (e == cudaSuccess && S > 1) e = launch_combine(L, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+}  // namespace
+
 // tuning override of the key-range split count of both tensor-core kernels (0 = automatic), see
 // dllm_debug_attention_plan
 int g_attn_force_splits = 0;
 // (query, head-of-group) rows per KV head from which a bf16 shape takes the 128-row tcgen05 kernel
 int g_attn_umma_min_rows = AT_ROWS + 1;
+// 0: shapes with very few rows per KV head stay on the 64-row kernel (tuning / test switch)
+int g_attn_few_rows = 1;
 
 // Key-range splits of the 64-row kernel, whole 64-key tiles per split: enough CTAs to cover the SMs when few
 // rows are active (every split costs the merge a partial per row and head, so no more than that), and two CTAs
@@ -288,6 +506,20 @@ static void finish_plan(AttnPlan& p, int B, int a_seq, int n, int H, int S) {
 AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv) {
   AttnPlan p;
   const int G = H / Hkv, sms = sm_count();
+  // At most 32 rows per KV head against at least 16 key tiles: the kernel whose warps share the rows and take
+  // different key tiles (6 ways of one 16-row warp, one CTA per SM; or 3 ways of two, two CTAs per SM); a
+  // split keeps at least two tiles per way.
+  if (a_seq * G <= 32 && (n + AT_KEYS - 1) / AT_KEYS >= 16 && g_attn_few_rows) {
+    const int key_tiles = (n + AT_KEYS - 1) / AT_KEYS;
+    p.few_rg = a_seq * G <= 16 ? 1 : 2;
+    const int ways = p.few_rg == 1 ? 6 : 3, per_sm = p.few_rg == 1 ? 1 : 2;
+    const long ctas = (long)Hkv * B;
+    int S = (int)(((long)per_sm * sms + ctas - 1) / ctas);
+    if (S > key_tiles / (2 * ways)) S = key_tiles / (2 * ways);
+    if (g_attn_force_splits > 0) S = g_attn_force_splits;
+    finish_plan(p, B, a_seq, n, H, S);
+    return p;
+  }
   const long tiles = (long)((a_seq * G + AT_ROWS - 1) / AT_ROWS) * Hkv * B;
   int S = 1;
   if (tiles < sms) {
@@ -311,6 +543,7 @@ AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scra
   } else {
     c.plan = plan_attention(B, a_seq, n, H, Hkv);
     if (c.plan.S > 1 && scratch_floats < c.plan.scratch_floats) finish_plan(c.plan, B, a_seq, n, H, 1);  // no room
+    // (finish_plan keeps the kernel choice p.few_rg)
   }
   return c;
 }
@@ -339,6 +572,12 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
     if (!get_tensor_map_3d(Kc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, AT_KEYS, &tmK) ||
         !get_tensor_map_3d(Vc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, AT_KEYS, &tmV))
       return cudaErrorInvalidValue;
+    if (p.few_rg == 1)
+      return hd == 64 ? launch_few<64, 1, 6>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
+                      : launch_few<128, 1, 6>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
+    if (p.few_rg == 2)
+      return hd == 64 ? launch_few<64, 2, 3>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
+                      : launch_few<128, 2, 3>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
     return hd == 64 ? launch_mma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
                     : launch_mma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
   }
@@ -445,13 +684,14 @@ extern "C" dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, 
   return DLLM_OK;
 }
 
-extern "C" dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows) {
+extern "C" dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows, int few_rows_kernel) {
   if (splits < 0 || tcgen05_min_rows < 0) {
     dllm::set_last_error("dllm_debug_attention_plan: arguments must not be negative");
     return DLLM_INVALID_ARG;
   }
   dllm::g_attn_force_splits = splits;
   if (tcgen05_min_rows > 0) dllm::g_attn_umma_min_rows = tcgen05_min_rows;
+  dllm::g_attn_few_rows = few_rows_kernel != 0;
   return DLLM_OK;
 }
 

@@ -291,4 +291,116 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
   return true;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// The same arithmetic for ONE warp and ONE 64-key tile, used by the kernel for very few query rows, where the
+// warps of a CTA share their 16 rows and take different key tiles (the chain load -> QK^T -> softmax -> PV of
+// a tile takes a warp about as long whether its row tile is full or nearly empty, so with 3 or 30 rows it pays
+// to work on several tiles at once).  q_s: the CTA's Q tile (swizzled panels of AT_ROWS rows); rg: which 16
+// rows of it; k_s / v_s: the tile; keys [key0, key_hi) of it count.  acc carries (o, m, l) across the warp's
+// tiles; l holds per-lane partial sums until attn_warp_finish.
+template <int HD>
+struct AttnAcc {
+  float o[HD / 8][4];
+  float m[2], l[2];
+};
+template <int HD>
+__device__ __forceinline__ void attn_acc_clear(AttnAcc<HD>& acc) {
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) acc.o[i][0] = acc.o[i][1] = acc.o[i][2] = acc.o[i][3] = 0.f;
+  acc.m[0] = acc.m[1] = -INFINITY;
+  acc.l[0] = acc.l[1] = 0.f;
+}
+template <int HD>
+__device__ __forceinline__ void attn_warp_tile(int lane, int rg, uint32_t q_s, uint32_t k_s, uint32_t v_s, int key0,
+                                               int key_hi, float scale_log2, AttnAcc<HD>& acc) {
+  // ---- S = Q K^T for 16 rows x 64 keys
+  float sacc[AT_KEYS / 8][4];
+#pragma unroll
+  for (int i = 0; i < AT_KEYS / 8; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
+#pragma unroll
+  for (int ks = 0; ks < HD / 16; ++ks) {
+    uint32_t qf[4];
+    {
+      const int row = rg * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+      const int dc = ks * 2 + (lane >> 4);
+      ldsm_x4(q_s + tile_off<AT_ROWS>(row, dc), qf[0], qf[1], qf[2], qf[3]);
+    }
+#pragma unroll
+    for (int jp = 0; jp < AT_KEYS / 16; ++jp) {
+      const int key = jp * 16 + (lane & 7) + (lane >> 4) * 8;
+      const int dc = ks * 2 + ((lane >> 3) & 1);
+      uint32_t r0, r1, r2, r3;
+      ldsm_x4(k_s + tile_off<AT_KEYS>(key, dc), r0, r1, r2, r3);
+      mma_bf16_16816(sacc[2 * jp], qf, r0, r1);
+      mma_bf16_16816(sacc[2 * jp + 1], qf, r2, r3);
+    }
+  }
+  // ---- online softmax (rows lane/4 and lane/4 + 8)
+  const int key_base = key0 + 2 * (lane & 3);
+  float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+  for (int nb = 0; nb < AT_KEYS / 8; ++nb) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int key = key_base + nb * 8 + (c & 1);
+      const float v = (key < key_hi) ? sacc[nb][c] * scale_log2 : -INFINITY;
+      sacc[nb][c] = v;
+      mx[c >> 1] = fmaxf(mx[c >> 1], v);
+    }
+  }
+  float corr[2];
+#pragma unroll
+  for (int h2 = 0; h2 < 2; ++h2) {
+    mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 1));
+    mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 2));
+    const float m_new = fmaxf(acc.m[h2], mx[h2]);      // finite: every tile has a valid key
+    corr[h2] = exp2f(acc.m[h2] - m_new);                 // first tile: exp2(-inf) = 0
+    acc.m[h2] = m_new;
+    acc.l[h2] *= corr[h2];
+  }
+#pragma unroll
+  for (int nb = 0; nb < AT_KEYS / 8; ++nb) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float p = exp2f(sacc[nb][c] - acc.m[c >> 1]);
+      sacc[nb][c] = p;
+      acc.l[c >> 1] += p;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) {
+    acc.o[i][0] *= corr[0];
+    acc.o[i][1] *= corr[0];
+    acc.o[i][2] *= corr[1];
+    acc.o[i][3] *= corr[1];
+  }
+  // ---- O += P V
+#pragma unroll
+  for (int kk = 0; kk < AT_KEYS / 16; ++kk) {
+    uint32_t pf[4];
+    pf[0] = pack_bf16(sacc[2 * kk][0], sacc[2 * kk][1]);
+    pf[1] = pack_bf16(sacc[2 * kk][2], sacc[2 * kk][3]);
+    pf[2] = pack_bf16(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1]);
+    pf[3] = pack_bf16(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3]);
+#pragma unroll
+    for (int dp = 0; dp < HD / 16; ++dp) {
+      const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+      const int dc = dp * 2 + (lane >> 4);
+      uint32_t r0, r1, r2, r3;
+      ldsm_x4_trans(v_s + tile_off<AT_KEYS>(key, dc), r0, r1, r2, r3);
+      mma_bf16_16816(acc.o[2 * dp], pf, r0, r1);
+      mma_bf16_16816(acc.o[2 * dp + 1], pf, r2, r3);
+    }
+  }
+}
+// the row sums are spread over the four lanes of a row
+template <int HD>
+__device__ __forceinline__ void attn_warp_finish(AttnAcc<HD>& acc) {
+#pragma unroll
+  for (int h2 = 0; h2 < 2; ++h2) {
+    acc.l[h2] += __shfl_xor_sync(0xffffffffu, acc.l[h2], 1);
+    acc.l[h2] += __shfl_xor_sync(0xffffffffu, acc.l[h2], 2);
+  }
+}
+
 }  // namespace dllm

@@ -220,6 +220,7 @@ struct AttnPlan {
   int S;               // key-range splits
   int keys_per_split;  // multiple of the key tile
   size_t scratch_floats;
+  int few_rg = 0;      // 64-row kernel family: 0 = the 64-row kernel, 1 / 2 = the few-rows kernel with 16 / 32 rows per CTA
 };
 AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv);
 // Plan of the 128-row tcgen05 kernel (attention_umma.cu) with at most scratch_floats floats for split partials.
@@ -229,11 +230,12 @@ AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scr
 // and the entry point with built-in scratch all decide through this one function.
 struct AttnChoice {
   bool umma = false;
-  AttnPlan plan{1, 0, 0};
+  AttnPlan plan{1, 0, 0, 0};
 };
 AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats);
 extern int g_attn_force_splits;   // tuning override of both plans' split count (0 = automatic)
 extern int g_attn_umma_min_rows;  // rows per KV head from which the tcgen05 kernel is taken
+extern int g_attn_few_rows;       // 0: never the few-rows kernel
 // bf16 with head_dim 64 / 128 runs on the tensor cores (scratch holds the
 // partials of split key ranges; without it one split is used); everything else
 // on the plain-ALU kernel.

@@ -150,7 +150,10 @@ ATT_CASES = [
     (2, 33, 130, 7, 1, 64),    # GQA, 7 query heads per KV head
     (1, 64, 768, 8, 8, 128),   # LLaDA-8B partial-step shape, 8 of the 32 heads
     (1, 128, 512, 28, 4, 128), # Dream-7B partial-step shape
-    (1, 3, 4128, 2, 2, 128),   # long-prompt regime: 3 queries, 65 key tiles, ragged last tile
+    (1, 3, 4128, 2, 2, 128),   # long-prompt regime: 3 queries, 65 key tiles, ragged last tile (few-rows kernel, 6 ways)
+    (2, 30, 1100, 3, 3, 64),   # few-rows kernel with two row groups and 3 ways, 18 key tiles, head_dim 64
+    (1, 5, 2000, 8, 2, 128),   # grouped heads: 20 rows per KV head, few-rows kernel, ragged last tile
+    (3, 16, 1024, 2, 2, 128),  # exactly 16 rows and 16 key tiles: the smallest shape of the few-rows kernel
     (2, 200, 333, 4, 2, 64),   # several row tiles, G = 2, ragged keys
     # more than 64 (query, head-of-group) rows per KV head: the tcgen05 kernel (two 128-row tiles per CTA, 64-key tiles)
     (1, 256, 768, 8, 8, 128),  # LLaDA-8B response-refresh shape, 8 of the 32 heads
