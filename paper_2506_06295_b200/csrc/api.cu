@@ -177,8 +177,9 @@ Workspace make_workspace(const dllm_config& c, int B, int P, int R, int flags) {
   // prompt-refresh step ([B, P, d] each, carried order)
   w.pouts = take((flags & DLLM_SESSION_COMPACT_CACHE) ? 2 * (size_t)B * P * d * es : 0);
   // partial outputs of split key ranges: the 64-row kernel splits only while fewer CTAs than SMs exist, so
-  // splits * (row, head) pairs < 2 * SMs * 64; the 128-row kernel lowers its split count to what this holds
-  w.attn_floats = (size_t)2 * sm_count() * 64 * (128 + 2);
+  // splits * (row, head) pairs < 2 * SMs * 64 (the few-rows kernel: 32 rows); the tcgen05 kernel, whose CTAs
+  // hold up to 256 rows, lowers its split count to what this holds
+  w.attn_floats = (size_t)2 * sm_count() * 256 * (128 + 2);
   w.attn = take(w.attn_floats * 4);
   // the GEMM slab buffer: the largest S * M * N over every projection a step of this session can launch (V and
   // the LM head over the B * R response rows, V over the prompt rows, and Q/K, O, gate/up, down and V over any

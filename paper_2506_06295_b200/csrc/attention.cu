@@ -491,8 +491,9 @@ int g_attn_few_rows = 1;
 // Key-range splits of the 64-row kernel, whole 64-key tiles per split: enough CTAs to cover the SMs when few
 // rows are active (every split costs the merge a partial per row and head, so no more than that), and two CTAs
 // per SM (what the shared memory of an SM holds) when a split would otherwise be left with more than eight key
-// tiles to work through one after the other (a few queries against thousands of keys).  From sweeps on B200:
-// 64 rows x 768 keys x 32 heads is fastest with 4 splits, 3 or 36 rows x 4128 keys x 32 heads with 9 or 10.
+// tiles to work through one after the other (a few queries against thousands of keys), but never fewer than
+// three key tiles per split.  From sweeps on B200: 64 rows x 768 keys x 32 heads is fastest with 4 splits, 36
+// rows x 4128 keys x 32 heads with 9 or 10, 56 rows x 2048 keys x 4 KV heads with 8 to 10 (11.8 us; 32: 36 us).
 static void finish_plan(AttnPlan& p, int B, int a_seq, int n, int H, int S) {
   const int key_tiles = (n + AT_KEYS - 1) / AT_KEYS;
   if (S > key_tiles) S = key_tiles;
@@ -507,14 +508,15 @@ AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv) {
   AttnPlan p;
   const int G = H / Hkv, sms = sm_count();
   // At most 32 rows per KV head against at least 16 key tiles: the kernel whose warps share the rows and take
-  // different key tiles (6 ways of one 16-row warp, one CTA per SM; or 3 ways of two, two CTAs per SM); a
-  // split keeps at least two tiles per way.
+  // different key tiles (6 ways of one 16-row warp, or 3 ways of two).  One wave of CTAs: as many splits as
+  // keep the CTA count within the SM count (sweeps: 3 x 4128 x 32 heads 18.6 us with 4 splits against 25.0 on the
+  // 64-row kernel, 25.6 with 5; 32 rows 23.7 against 26.2; four sequences 46 against 73), two tiles per way at least.
   if (a_seq * G <= 32 && (n + AT_KEYS - 1) / AT_KEYS >= 16 && g_attn_few_rows) {
     const int key_tiles = (n + AT_KEYS - 1) / AT_KEYS;
     p.few_rg = a_seq * G <= 16 ? 1 : 2;
-    const int ways = p.few_rg == 1 ? 6 : 3, per_sm = p.few_rg == 1 ? 1 : 2;
+    const int ways = p.few_rg == 1 ? 6 : 3;
     const long ctas = (long)Hkv * B;
-    int S = (int)(((long)per_sm * sms + ctas - 1) / ctas);
+    int S = (int)(sms / ctas);
     if (S > key_tiles / (2 * ways)) S = key_tiles / (2 * ways);
     if (g_attn_force_splits > 0) S = g_attn_force_splits;
     finish_plan(p, B, a_seq, n, H, S);
@@ -526,6 +528,7 @@ AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv) {
     S = (int)((sms + tiles - 1) / tiles);
     const int key_tiles = (n + AT_KEYS - 1) / AT_KEYS;
     if ((key_tiles + S - 1) / S > 8) S = (int)((2L * sms + tiles - 1) / tiles);
+    if (S > key_tiles / 3) S = key_tiles / 3 > 1 ? key_tiles / 3 : 1;  // three key tiles per split at least
   }
   if (g_attn_force_splits > 0) S = g_attn_force_splits;
   finish_plan(p, B, a_seq, n, H, S);

@@ -105,7 +105,8 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
     attn_umma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                      const __nv_bfloat16* __restrict__ q,
                      __nv_bfloat16* __restrict__ o, float* __restrict__ o_part, float* __restrict__ ml_part, int a_seq,
-                     int n, int H, int Hkv, int S, int keys_per_split, float scale_log2, int* __restrict__ status) {
+                     int n, int H, int Hkv, int S, int keys_per_split, int row_tiles_per_cta, float scale_log2,
+                     int* __restrict__ status) {
   using SM = UaSmem<HD>;
   constexpr int PANELS = HD / 64;
   extern __shared__ uint8_t smem_raw[];
@@ -122,9 +123,11 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
   const int G = H / Hkv;
   const int kh = blockIdx.y;
   const int b = blockIdx.z / S, split = blockIdx.z - b * S;
-  const int row0 = blockIdx.x * (UA_TILES * UA_ROWS);
+  // row_tiles_per_cta = 1: every CTA takes one 128-row tile only (its second softmax group idles); the plan
+  // asks for that when two-tile CTAs would be too few to fill the GPU
+  const int row0 = blockIdx.x * (row_tiles_per_cta * UA_ROWS);
   const int n_rows = a_seq * G;
-  const int live = row0 + UA_ROWS < n_rows ? 2 : 1;              // row tiles of this CTA that hold rows
+  const int live = (row_tiles_per_cta > 1 && row0 + UA_ROWS < n_rows) ? 2 : 1;  // row tiles of this CTA that hold rows
   const int key_lo = split * keys_per_split;
   const int key_hi = min(n, key_lo + keys_per_split);
   const int n_tiles = (key_hi - key_lo + UA_KEYS - 1) / UA_KEYS;  // >= 1 by construction of the plan
@@ -248,7 +251,7 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
       uint4 qv[HD / 8];
 #pragma unroll
       for (int w = 0; w < HD / 8; ++w) qv[w] = make_uint4(0, 0, 0, 0);
-      if (vr < n_rows) {
+      if (vr < n_rows && i < live) {
         const int qi = vr / G, g = vr - qi * G;
         const uint4* src = reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD);
 #pragma unroll
@@ -401,7 +404,8 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
 
 template <int HD>
 cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
-                        float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
+                        float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split,
+                        int row_tiles_per_cta) {
   constexpr int SMEM = (int)UaSmem<HD>::TOTAL;
   static DeviceOnce once;
   cudaError_t e0 = once.run(
@@ -411,11 +415,12 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
   const size_t total = (size_t)B * a_seq * H;
   float* o_part = scratch;
   float* ml_part = scratch ? scratch + (size_t)S * total * HD : nullptr;
-  dim3 grid((a_seq * G + UA_TILES * UA_ROWS - 1) / (UA_TILES * UA_ROWS), Hkv, B * S);
+  const int rows_per_cta = row_tiles_per_cta * UA_ROWS;
+  dim3 grid((a_seq * G + rows_per_cta - 1) / rows_per_cta, Hkv, B * S);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   cudaError_t e = launch_k(L, attn_umma_kernel<HD>, grid, dim3(UA_THREADS), SMEM, tmK, tmV, (const __nv_bfloat16*)q,
-                           (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split, scale_log2,
-                           L.d_status);
+                           (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split, row_tiles_per_cta,
+                           scale_log2, L.d_status);
   L.count();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -424,30 +429,35 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
 
 // Key-range splits for CTAs of two 128-row tiles, whole 64-key tiles per split, no more splits than the scratch
 // holds.  A split shortens the key range a CTA walks through but adds a partial result per (row, head) pair that
-// the merge has to write and read, so the count is the one a small cost model likes best (microseconds, fitted
-// to sweeps on B200: about 1.5 us per key tile of a CTA at head_dim 128, one CTA per SM at a time, 4 us of
-// fixed cost, and for a merge 2.5 us plus 1040 bytes per pair and split at 5 TB/s).
+// the merge has to write and read, and a CTA with one row tile instead of two doubles the CTAs but loses the
+// overlap of the two softmax groups, so both are what a small cost model likes best (microseconds, fitted to
+// sweeps on B200: per key tile of a CTA 1.76 us with two row tiles and 1.36 us with one, one CTA per SM at a
+// time, 4 us of fixed cost, and for a merge 2.5 us plus 1040 bytes per pair and split at 5 TB/s).
 AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats) {
   AttnPlan p;
   const int G = H / Hkv, sms = sm_count();
-  const long tiles = (long)((a_seq * G + UA_TILES * UA_ROWS - 1) / (UA_TILES * UA_ROWS)) * Hkv * B;
   const int key_tiles = (n + UA_KEYS - 1) / UA_KEYS;
   const size_t per_split = (size_t)B * a_seq * H * (128 + 2);
   const double pairs = (double)B * a_seq * H;
-  int best = 1;
-  double best_us = 0.0;
-  for (int S = 1; S <= key_tiles && S <= 16; ++S) {
-    if (S > 1 && (size_t)S * per_split > scratch_floats) break;
-    const int tps = (key_tiles + S - 1) / S;
-    if (S > 1 && (key_tiles + tps - 1) / tps != S) continue;  // the same tiles per split as a smaller count
-    const double waves = (double)((tiles * S + sms - 1) / sms);
-    const double us = 4.0 + waves * tps * 1.5 + (S > 1 ? 2.5 + S * pairs * 1040.0 / 5.0e6 : 0.0);
-    if (S == 1 || us < best_us) {
-      best = S;
-      best_us = us;
+  int best_s = 1, best_rt = UA_TILES;
+  double best_us = -1.0;
+  for (int rt = UA_TILES; rt >= 1; --rt) {   // row tiles per CTA: two (the groups overlap), or one (twice the CTAs)
+    const long ctas = (long)((a_seq * G + rt * UA_ROWS - 1) / (rt * UA_ROWS)) * Hkv * B;
+    const double tile_us = rt == 2 ? 1.76 : 1.36;  // a key tile of a CTA, from 16 x 512 x 1536 and 16 x 128 x 1536
+    for (int S = 1; S <= key_tiles && S <= 16; ++S) {
+      if (S > 1 && (size_t)S * per_split > scratch_floats) break;
+      const int tps = (key_tiles + S - 1) / S;
+      if (S > 1 && (key_tiles + tps - 1) / tps != S) continue;  // the same tiles per split as a smaller count
+      const double waves = (double)((ctas * S + sms - 1) / sms);
+      const double us = 4.0 + waves * tps * tile_us + (S > 1 ? 2.5 + S * pairs * 1040.0 / 5.0e6 : 0.0);
+      if (best_us < 0.0 || us < best_us) {
+        best_s = S;
+        best_rt = rt;
+        best_us = us;
+      }
     }
   }
-  int S = g_attn_force_splits > 0 ? g_attn_force_splits : best;
+  int S = g_attn_force_splits > 0 ? g_attn_force_splits : best_s;
   if (S > key_tiles) S = key_tiles;
   if (S > 1 && (size_t)S * per_split > scratch_floats) S = (int)(scratch_floats / per_split);
   if (S < 1) S = 1;
@@ -455,6 +465,7 @@ AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scr
   p.keys_per_split = tiles_per_split * UA_KEYS;
   p.S = (key_tiles + tiles_per_split - 1) / tiles_per_split;
   p.scratch_floats = p.S > 1 ? (size_t)p.S * per_split : 0;
+  p.row_tiles = a_seq * G <= UA_ROWS ? 1 : best_rt;
   return p;
 }
 
@@ -467,8 +478,9 @@ cudaError_t launch_attention_umma(const Launch& L, const void* q, const void* Kc
       !get_tensor_map_3d(Vc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, 64, &tmV))
     return cudaErrorInvalidValue;
   if (S_out) *S_out = p.S;
-  return hd == 64 ? launch_umma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
-                  : launch_umma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
+  return hd == 64
+             ? launch_umma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split, p.row_tiles)
+             : launch_umma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split, p.row_tiles);
 }
 
 }  // namespace dllm

@@ -8,7 +8,10 @@
 // preceding GEMM are reduced here, in slab order, so the GEMM never needs
 // atomics and every row's value is independent of which other rows were in the
 // same launch.
+#include <algorithm>
+
 #include "internal.h"
+#include "tma.cuh"
 
 namespace dllm {
 
@@ -51,6 +54,230 @@ __device__ __forceinline__ void sum_partials4(const Partials& part, int row, int
         v[0] += t[q].x; v[1] += t[q].y; v[2] += t[q].z; v[3] += t[q].w;
       }
   }
+}
+
+// ------------------------------------------------------------------ streaming forms for many rows
+// With thousands of carried rows (batched serving) the one-row-per-CTA kernels above leave HBM idle while a CTA
+// reduces and stores: two rows per SM in flight, nothing requested meanwhile.  The streaming forms run one CTA
+// per SM for the whole launch: a producer thread fetches the rows of the CTA (blockIdx.x, + gridDim.x, ...) by
+// untiled bulk copies into a ring of shared-memory stages, ahead of four consumer warps that each take a whole
+// row (no block barrier: lane-local sums and one warp reduction per row) and write its results straight to
+// global memory.  Split-K slabs are not supported here (S = 1: with this many rows no projection is split).
+constexpr int STREAM_CONSUMERS = 4;                 // warps 1..4; warp 0 produces
+constexpr int STREAM_THREADS = 32 * (1 + STREAM_CONSUMERS);
+constexpr int STREAM_MAX_STAGES = 12;
+
+// End of a layer, streaming: see tail_kernel.  Stage = [x row fp32 | AttnOut row | FFN row (fp32 projection
+// result of an active row, or the cached row)].
+template <typename T>
+__global__ void __launch_bounds__(STREAM_THREADS, 1)
+    tail_stream_kernel(const float* __restrict__ part, const int32_t* __restrict__ inv, float* __restrict__ x,
+                       OutRows Ac, OutRows Fc, const float* __restrict__ gain, T* __restrict__ u, Geo g, int c0, int c1,
+                       float eps, int stages, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STREAM_MAX_STAGES], empty_bar[STREAM_MAX_STAGES];
+  __shared__ int meta[STREAM_MAX_STAGES];
+  __shared__ int abort_flag;
+  const int d = g.d, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t xb = (uint32_t)d * 4, ab = (uint32_t)d * sizeof(T), fb = (uint32_t)d * 4;
+  const uint32_t stage_bytes = xb + ab + fb;
+  const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
+  uint8_t* base_gen = smem_raw + (base - smem_u32(smem_raw));
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_wait();
+  pdl_trigger();
+  volatile int* abortp = &abort_flag;
+  const int n_rows = c1 - c0;
+  const int my_rows = (int)blockIdx.x < n_rows ? (n_rows - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  bool ok = true;
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int i = 0; i < my_rows; ++i) {
+        const int s = i % stages, c = c0 + blockIdx.x + i * gridDim.x;
+        if (i >= stages && !mbar_wait(smem_u32(&empty_bar[s]), (uint32_t)(i / stages - 1) & 1u, abortp)) {
+          ok = false;
+          break;
+        }
+        const int r = inv ? inv[c] : -1;
+        meta[s] = r;
+        const uint32_t dst = base + s * stage_bytes, bar = smem_u32(&full_bar[s]);
+        mbar_expect_tx(bar, xb + ab + (r >= 0 ? fb : ab));
+        bulk_load_1d(dst, x + (size_t)c * d, xb, bar);
+        bulk_load_1d(dst + xb, Ac.row<T>(c, g), ab, bar);
+        if (r >= 0)
+          bulk_load_1d(dst + xb + ab, part + (size_t)r * d, fb, bar);
+        else
+          bulk_load_1d(dst + xb + ab, Fc.row<T>(c, g), ab, bar);
+      }
+    }
+  } else {
+    const int w = warp - 1;
+    for (int i = w; i < my_rows; i += STREAM_CONSUMERS) {
+      const int s = i % stages, c = c0 + blockIdx.x + i * gridDim.x;
+      ok = mbar_wait(smem_u32(&full_bar[s]), (uint32_t)(i / stages) & 1u, abortp);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const int r = meta[s];
+      float* xs = reinterpret_cast<float*>(base_gen + (size_t)s * stage_bytes);
+      const T* as = reinterpret_cast<const T*>(base_gen + (size_t)s * stage_bytes + xb);
+      const uint8_t* fs = base_gen + (size_t)s * stage_bytes + xb + ab;
+      float* xr = x + (size_t)c * d;
+      T* frow = Fc.row<T>(c, g);
+      float ss = 0.f;
+      for (int j = lane * 8; j < d; j += 256) {
+        float xv[8], a[8], f[8];
+        Vec8<float>::load(xs + j, xv);
+        Vec8<T>::load(as + j, a);
+        if (r >= 0) {
+          Vec8<float>::load(reinterpret_cast<const float*>(fs) + j, f);
+          Vec8<T>::store(frow + j, f);
+#pragma unroll
+          for (int t = 0; t < 8; ++t) f[t] = Vec8<T>::round(f[t]);
+        } else {
+          Vec8<T>::load(reinterpret_cast<const T*>(fs) + j, f);
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          xv[t] = (xv[t] + a[t]) + f[t];
+          ss += xv[t] * xv[t];
+        }
+        Vec8<float>::store(xr + j, xv);
+        Vec8<float>::store(xs + j, xv);   // kept for the second pass
+      }
+      ss = warp_sum(ss);
+      const float rs = rsqrtf(ss / (float)d + eps);
+      T* orow = u + (size_t)c * d;
+      for (int j = lane * 8; j < d; j += 256) {
+        float v[8], gv[8];
+        Vec8<float>::load(xs + j, v);
+        Vec8<float>::load(gain + j, gv);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) v[t] = v[t] * rs * gv[t];
+        Vec8<T>::store(orow + j, v);
+      }
+      // the stage was written by this warp through the generic proxy; the next bulk copy goes through the async one
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));
+    }
+  }
+  ok = __syncthreads_and(ok);
+  if (!ok) {
+    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+    drain_delay();
+  }
+}
+
+// V-verify (Eq. 6) + V overwrite, streaming: see vverify_kernel.  Stage = [projected row fp32 | cached row].
+template <typename T>
+__global__ void __launch_bounds__(STREAM_THREADS, 1)
+    vverify_stream_kernel(const float* __restrict__ part, T* __restrict__ Vc, float* __restrict__ sim, Geo g, int dkv,
+                          int metric, int write_v, IdentityLists id, int stages, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STREAM_MAX_STAGES], empty_bar[STREAM_MAX_STAGES];
+  __shared__ int abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t nb_ = (uint32_t)dkv * 4, cb = (uint32_t)dkv * sizeof(T), stage_bytes = nb_ + cb;
+  const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
+  uint8_t* base_gen = smem_raw + (base - smem_u32(smem_raw));
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_wait();
+  pdl_trigger();
+  volatile int* abortp = &abort_flag;
+  const int n_rows = g.B * g.R;
+  const int my_rows = (int)blockIdx.x < n_rows ? (n_rows - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  auto cache_row = [&](int c) {
+    const int b = c / g.R, j = c - b * g.R;
+    return Vc + ((size_t)b * g.n + g.P + j) * dkv;
+  };
+  bool ok = true;
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int i = 0; i < my_rows; ++i) {
+        const int s = i % stages, c = blockIdx.x + i * gridDim.x;
+        if (i >= stages && !mbar_wait(smem_u32(&empty_bar[s]), (uint32_t)(i / stages - 1) & 1u, abortp)) {
+          ok = false;
+          break;
+        }
+        const uint32_t dst = base + s * stage_bytes, bar = smem_u32(&full_bar[s]);
+        mbar_expect_tx(bar, stage_bytes);
+        bulk_load_1d(dst, part + (size_t)c * dkv, nb_, bar);
+        bulk_load_1d(dst + nb_, cache_row(c), cb, bar);
+      }
+    }
+  } else {
+    const int w = warp - 1;
+    for (int i = w; i < my_rows; i += STREAM_CONSUMERS) {
+      const int s = i % stages, c = blockIdx.x + i * gridDim.x;
+      ok = mbar_wait(smem_u32(&full_bar[s]), (uint32_t)(i / stages) & 1u, abortp);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const float* ns = reinterpret_cast<const float*>(base_gen + (size_t)s * stage_bytes);
+      const T* cs = reinterpret_cast<const T*>(base_gen + (size_t)s * stage_bytes + nb_);
+      T* vrow = cache_row(c);
+      float dot = 0.f, na = 0.f, nb = 0.f;
+      for (int j = lane * 8; j < dkv; j += 256) {
+        float vn[8], vo[8];
+        Vec8<float>::load(ns + j, vn);
+        Vec8<T>::load(cs + j, vo);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          vn[t] = Vec8<T>::round(vn[t]);  // compare what the cache will hold
+          if (metric == 0) {
+            dot += vn[t] * vo[t];
+            na += vn[t] * vn[t];
+            nb += vo[t] * vo[t];
+          } else {
+            const float df = vn[t] - vo[t];
+            dot += df * df;
+          }
+        }
+        if (write_v) Vec8<T>::store(vrow + j, vn);
+      }
+      dot = warp_sum(dot);
+      na = warp_sum(na);
+      nb = warp_sum(nb);
+      if (lane == 0) {
+        sim[c] = metric == 0 ? dot / fmaxf(sqrtf(na * nb), 1e-8f) : -sqrtf(dot);
+        if (id.act) {  // a response refresh recomputes every response row, in carried order: identity lists
+          id.sel[c] = c % g.R;
+          id.act[c] = c;
+          id.inv[c] = c;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));
+    }
+  }
+  ok = __syncthreads_and(ok);
+  if (!ok) {
+    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+    drain_delay();
+  }
+}
+
+// Rows from which the streaming forms are taken (a property of the session's response rows, so that every
+// step kind of a session reduces a row in the same order).
+constexpr int STREAM_MIN_ROWS = 1024;
+static int stream_stages(size_t stage_bytes) {
+  const size_t fit = (227 * 1024 - 2048) / stage_bytes;
+  return (int)(fit < (size_t)STREAM_MAX_STAGES ? fit : (size_t)STREAM_MAX_STAGES);
 }
 
 // ------------------------------------------------------------------ rmsnorm
@@ -211,6 +438,23 @@ void launch_vverify(const Launch& L, int dtype, Partials part, void* Vc_layer, f
                     int write_v, const IdentityLists* lists) {
   const int rows = g.B * g.R;
   const IdentityLists id = lists ? *lists : IdentityLists{};
+  const size_t es = dtype == 0 ? 4 : 2, stage = (size_t)dkv * (4 + es);
+  if (rows >= STREAM_MIN_ROWS && part.S == 1 && part.upc == 0 && stream_stages(stage) >= STREAM_CONSUMERS + 1) {
+    const int stages = stream_stages(stage);
+    const size_t smem = (size_t)stages * stage + 128;
+    const int ctas = std::min(rows, sm_count());
+    DLLM_DISPATCH(dtype, {
+      static DeviceOnce once;
+      cudaError_t e0 = once.run([] {
+        return cudaFuncSetAttribute(vverify_stream_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
+      });
+      if (e0 == cudaSuccess)
+        launch_k(L, vverify_stream_kernel<T>, dim3(ctas), dim3(STREAM_THREADS), smem, part.p, (T*)Vc_layer, sim, g, dkv,
+                 metric, write_v, id, stages, L.d_status);
+    });
+    L.count();
+    return;
+  }
   DLLM_DISPATCH(dtype, (launch_k(L, vverify_kernel<T>, dim3(rows), dim3(row_threads(dkv)), 0, part, (T*)Vc_layer, sim, g, dkv,
                                  metric, write_v, id)));
   L.count();
@@ -699,6 +943,25 @@ __global__ void __launch_bounds__(512, 2) tail_kernel(Partials part, const int32
 void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, float* x, OutRows Ac_layer,
                  OutRows Fc_layer, const float* gain, void* u, Geo g, int c0, int c1, float eps) {
   if (c1 <= c0) return;
+  {
+    const size_t es = dtype == 0 ? 4 : 2, stage = (size_t)g.d * (8 + es);
+    if (g.B * g.R >= STREAM_MIN_ROWS && part.S == 1 && part.upc == 0 && stream_stages(stage) >= STREAM_CONSUMERS + 1) {
+      const int stages = stream_stages(stage);
+      const size_t smem_s = (size_t)stages * stage + 128;
+      const int ctas = std::min(c1 - c0, sm_count());
+      DLLM_DISPATCH(dtype, {
+        static DeviceOnce once;
+        cudaError_t e0 = once.run([] {
+          return cudaFuncSetAttribute(tail_stream_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
+        });
+        if (e0 == cudaSuccess)
+          launch_k(L, tail_stream_kernel<T>, dim3(ctas), dim3(STREAM_THREADS), smem_s, part.p, inv, x, Ac_layer, Fc_layer,
+                   gain, (T*)u, g, c0, c1, eps, stages, L.d_status);
+      });
+      L.count();
+      return;
+    }
+  }
   const int threads = row_threads(g.d);
   const size_t smem = g.d <= threads * 8 ? 0 : (size_t)g.d * sizeof(float);  // staging only if a row takes several passes
   DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T>, dim3(c1 - c0), dim3(threads), smem, part, inv, x, Ac_layer,

@@ -221,6 +221,7 @@ struct AttnPlan {
   int keys_per_split;  // multiple of the key tile
   size_t scratch_floats;
   int few_rg = 0;      // 64-row kernel family: 0 = the 64-row kernel, 1 / 2 = the few-rows kernel with 16 / 32 rows per CTA
+  int row_tiles = 2;   // tcgen05 kernel: 128-row tiles per CTA (2, or 1 when two-tile CTAs would be too few)
 };
 AttnPlan plan_attention(int B, int a_seq, int n, int H, int Hkv);
 // Plan of the 128-row tcgen05 kernel (attention_umma.cu) with at most scratch_floats floats for split partials.
@@ -230,7 +231,7 @@ AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scr
 // and the entry point with built-in scratch all decide through this one function.
 struct AttnChoice {
   bool umma = false;
-  AttnPlan plan{1, 0, 0, 0};
+  AttnPlan plan{1, 0, 0, 0, 2};
 };
 AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats);
 extern int g_attn_force_splits;   // tuning override of both plans' split count (0 = automatic)

@@ -24,11 +24,13 @@ def env():
     return torch, dllm
 
 
-@pytest.mark.parametrize("which", ["tiny_fp32", "bf16_mha", "bf16_gqa"])
+@pytest.mark.parametrize("which", ["tiny_fp32", "bf16_mha", "bf16_gqa", "bf16_many_rows", "fp32_many_rows"])
 def test_compact_session_matches_the_four_tensor_session_and_the_compact_oracle(env, which):
     torch, dllm = env
-    cfg = synth.TINY if which == "tiny_fp32" else synth.small_bf16_model(gqa=which == "bf16_gqa")
+    cfg = synth.TINY if which in ("tiny_fp32", "fp32_many_rows") else synth.small_bf16_model(gqa=which == "bf16_gqa")
     B, P, R = (2, 64, 32) if which == "tiny_fp32" else (2, 150, 72)
+    if which.endswith("many_rows"):     # 1088 response rows: V-verify and the layer tail take their streaming forms
+        B, P, R = 8, 40, 136
     tol = 1e-4 if cfg.dtype == "fp32" else 2e-2
     w = synth.make_weights(cfg)
     prompt = synth.make_prompt(cfg, B, P)
