@@ -53,8 +53,8 @@ def test_noalloc_matches_the_allocating_entry_point_on_two_calls_in_a_row(env):
 
 def test_noalloc_rejects_what_does_not_fit_its_scratch(env):
     torch, dllm = env
-    # 64 rows per KV head (the 64-row kernel): 147 row tiles -> 2 key splits -> 9.8 MB of partials
-    B, a, n, H, Hkv, hd = 1, 64, 256, 147, 147, 128
+    # 64 rows per KV head (the 64-row kernel): 128 row tiles, 12 key tiles -> 2 key splits -> 8.5 MB of partials
+    B, a, n, H, Hkv, hd = 1, 64, 768, 128, 128, 128
     assert dllm.lib.dllm_attention_scratch_bytes(B, a, n, H, Hkv, hd, dllm.BF16) > 8 * 1024 * 1024
     q, k, v = _inputs(torch, B, a, n, H, Hkv, hd, seed=7)
     out = torch.zeros_like(q)
