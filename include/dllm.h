@@ -340,8 +340,9 @@ size_t dllm_gemm_bf16_scratch_bytes(int M, int N, int K);
 dllm_status dllm_gemm_bf16(const void* d_A, const void* d_W, float* d_C, int M, int N, int K,
                            void* d_partials, void* stream);
 /* The same product with an explicit launch plan, for tuning: act_tile = rows of
- * A per CTA (32, 64, 128 or 256), splits = split-K factor, stages = depth of the
- * TMA ring (clamped to what fits shared memory); 0 picks the default of each.
+ * A per CTA (32, 64, 128 or 256; 192 with splits = 1 only: the persistent kernel),
+ * splits = split-K factor, stages = depth of the TMA ring (clamped to what fits
+ * shared memory); 0 picks the default of each.
  * d_partials (device, partials_bytes >= dllm_gemm_bf16_planned_scratch_bytes)
  * holds the split-K slabs; with splits > 1 and d_C NULL the slabs are left
  * unreduced there (what the step's fused consumers read). */

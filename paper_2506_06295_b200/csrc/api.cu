@@ -1309,8 +1309,10 @@ dllm_status dllm_gemm_bf16_planned(const void* d_A, const void* d_W, float* d_C,
   if (!d_A || !d_W || M <= 0 || N <= 0 || K <= 0) return fail(nullptr, DLLM_INVALID_ARG, "bad GEMM arguments");
   if (K % 8) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8");
   if (act_tile < 0 || splits < 0 || stages < 0) return fail(nullptr, DLLM_INVALID_ARG, "negative plan parameter");
-  if (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 256)
-    return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128 or 256");
+  if (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 192 && act_tile != 256)
+    return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128, 192 or 256");
+  if (act_tile == 192 && splits != 1)
+    return fail(nullptr, DLLM_INVALID_ARG, "192-row tiles exist in the unsplit persistent kernel only: splits must be 1");
   const GemmPlan p = plan_gemm_bf16(M, N, K, splits, stages, act_tile);
   if (p.S_max > 1 && (!d_partials || partials_bytes < (size_t)p.S_max * M * N * 4))
     return fail(nullptr, DLLM_INVALID_ARG, "this plan needs %zu bytes of slab scratch", (size_t)p.S_max * M * N * 4);
@@ -1330,8 +1332,9 @@ dllm_status dllm_ffn_gate_up_bf16(const void* d_A, const void* d_Wgu, void* d_ou
   if (!d_A || !d_Wgu || !d_out || M <= 0 || d_ffn <= 0 || K <= 0)
     return fail(nullptr, DLLM_INVALID_ARG, "bad gate / up arguments");
   if (K % 8 || d_ffn % 64) return fail(nullptr, DLLM_INVALID_ARG, "K must be a multiple of 8 and d_ffn of 64");
-  if (act_tile < 0 || stages < 0 || (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 256))
-    return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128 or 256");
+  if (act_tile < 0 || stages < 0 ||
+      (act_tile && act_tile != 32 && act_tile != 64 && act_tile != 128 && act_tile != 192 && act_tile != 256))
+    return fail(nullptr, DLLM_INVALID_ARG, "act_tile must be 0, 32, 64, 128, 192 or 256");
   const GemmPlan p = plan_gemm_bf16(M, 2 * d_ffn, K, 1, stages, act_tile);
   Launch L{(cudaStream_t)stream, kernel_status_word(), nullptr};
   const char* why = nullptr;

@@ -387,6 +387,8 @@ __global__ void __launch_bounds__(PERSIST_THREADS, 1)
                                 int STAGES, __nv_bfloat16* __restrict__ act_out, int m_ffn, int* __restrict__ status) {
   using PL = PersistLayout<BN>;
   static_assert(2 * BN <= 512, "two accumulators must fit the 512 columns of tensor memory");
+  // column distance of the two accumulators: an allocation is a power of two, so 192-row tiles sit 256 apart
+  constexpr uint32_t ACC = BN > 128 ? 256 : BN > 64 ? 128 : BN > 32 ? 64 : 32;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
@@ -422,7 +424,7 @@ __global__ void __launch_bounds__(PERSIST_THREADS, 1)
   }
   if (warp == 1) {  // TMEM: two accumulators of BN fp32 columns x 128 lanes
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                 "r"((uint32_t)(2 * BN))
+                 "r"(2u * ACC)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -488,7 +490,7 @@ __global__ void __launch_bounds__(PERSIST_THREADS, 1)
           const uint64_t dA = make_smem_desc(sW + W_STAGE_BYTES);
 #pragma unroll
           for (int k = 0; k < TILE_K / UMMA_K; ++k)
-            umma_bf16(tmem_d + (uint32_t)(a * BN), dW + (uint64_t)(2 * k), dA + (uint64_t)(2 * k), idesc,
+            umma_bf16(tmem_d + (uint32_t)a * ACC, dW + (uint64_t)(2 * k), dA + (uint64_t)(2 * k), idesc,
                       (kb > 0 || k > 0) ? 1u : 0u);
           umma_commit(smem_u32(&empty_bar[s]));  // stage reusable once these MMAs have read it
           if (++s == STAGES) {
@@ -526,7 +528,7 @@ __global__ void __launch_bounds__(PERSIST_THREADS, 1)
         ok = false;
         break;
       }
-      gemm_epilogue<BN, 1>(tmem_d + (uint32_t)(a * BN), ex, tl, mt * BN, nt * TILE_W, nt, M, N, part, act_out, m_ffn);
+      gemm_epilogue<BN, 1>(tmem_d + (uint32_t)a * ACC, ex, tl, mt * BN, nt * TILE_W, nt, M, N, part, act_out, m_ffn);
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       mbar_arrive(smem_u32(&acc_empty[a]));
     }
@@ -536,7 +538,7 @@ __global__ void __launch_bounds__(PERSIST_THREADS, 1)
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"((uint32_t)(2 * BN)) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(2u * ACC) : "memory");
   }
 }
 
@@ -875,7 +877,13 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
       pair_stages = one_wave ? 4 : 3;
     }
   }
-  if (force_bn == 32 || force_bn == 64 || force_bn == 128 || force_bn == 256) p.BN = force_bn;
+  // 192-row tiles (persistent kernel only) where they leave at least 15 % fewer padded activation rows than
+  // 256-row tiles: the 576 rows of a mixed step (prompt refresh + adaptive response update) are 3 x 192, not 3 x 256
+  if (!p.pair && p.BN == 256 && force_split <= 1 && force_persistent >= 0 && g_gemm_force_persistent >= 0) {
+    const long pad192 = (M + 191) / 192 * 192L, pad256 = (M + 255) / 256 * 256L;
+    if (pad192 * 115 <= pad256 * 100 && n_tiles * (pad192 / 192) > sms) p.BN = 192;
+  }
+  if (force_bn == 32 || force_bn == 64 || force_bn == 128 || force_bn == 192 || force_bn == 256) p.BN = force_bn;
   if (force_pair > 0) p.pair = (p.BN == 128 || p.BN == 256) && N % (2 * TILE_W) == 0;
   p.stages = force_stages > 0 ? force_stages : p.pair ? pair_stages : (p.BN == 128 ? 3 : 4);
   p.num_kb = (K + TILE_K - 1) / TILE_K;
@@ -891,8 +899,8 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
   if (force_split > 0) S = force_split < p.num_kb ? force_split : p.num_kb;
   // more tiles than SMs, no split, one-CTA 256-row tiles: the persistent kernel (epilogue under the next main loop)
   if (force_persistent == 0) force_persistent = g_gemm_force_persistent;
-  p.persistent = (force_persistent >= 0) && !p.pair && p.BN == 256 && S == 1 &&
-                 (force_persistent > 0 || tiles > sms);
+  p.persistent = (force_persistent >= 0) && !p.pair && (p.BN == 256 || p.BN == 192) && S == 1 &&
+                 (force_persistent > 0 || tiles > sms || p.BN == 192);
   p.upc = (p.num_kb + S - 1) / S;                 // k-blocks per split
   p.S_max = (p.num_kb + p.upc - 1) / p.upc;       // no empty split
   p.ctas = (int)tiles * p.S_max;
@@ -932,7 +940,13 @@ cudaError_t launch_gemm_bf16(const Launch& L, const void* A, const void* W, floa
     return plan.BN == 128 ? launch_pair<128>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn)
                           : launch_pair<256>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
   }
-  if (plan.persistent) return launch_persistent<256>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
+  if (plan.persistent)
+    return plan.BN == 192 ? launch_persistent<192>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn)
+                          : launch_persistent<256>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
+  if (plan.BN == 192) {
+    if (err) *err = "192-row tiles exist in the persistent kernel only";
+    return cudaErrorInvalidValue;
+  }
   switch (plan.BN) {
     case 32: return launch_one<32>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);
     case 64: return launch_one<64>(L, tmW, tmA, part, M, N, num_kb, plan, act_out, m_ffn);

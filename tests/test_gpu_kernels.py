@@ -216,6 +216,27 @@ def test_gemm_persistent_kernel_is_bit_identical_to_the_one_tile_kernel(env, M, 
     assert np.array_equal(out[-1][1], out[1][1])
 
 
+@pytest.mark.parametrize("M,N,K,forced", [(576, 20000, 320, 0), (530, 1280, 200, 192), (192, 384, 64, 192)])
+def test_gemm_192_row_tiles(env, M, N, K, forced):
+    """Activation tiles of 192 rows in the persistent kernel (the 576 rows of a mixed step are 3 x 192, not
+    3 x 256): the default plan takes them for 576 rows against many weight tiles; ragged last tile, a ragged k
+    block, a single tile.  The k loop per output element is the same: the same bits as with 256-row tiles, for
+    the plain and for the SwiGLU epilogue."""
+    torch, dllm = env
+    A = torch.from_numpy(synth.round_to_bf16(synth.random_normal((M, K), seed=31))).cuda().to(torch.bfloat16)
+    W = torch.from_numpy(synth.round_to_bf16(synth.random_normal((N, K), seed=32, std=0.05))).cuda().to(torch.bfloat16)
+    Wg = W[:N // 128 * 128]
+    c = dllm.gemm_bf16_planned(A, W, act_tile=forced, splits=1).cpu().numpy()
+    g = dllm.ffn_gate_up_bf16(A, Wg, act_tile=forced).float().cpu().numpy()
+    c256 = dllm.gemm_bf16_planned(A, W, act_tile=256, splits=1).cpu().numpy()
+    g256 = dllm.ffn_gate_up_bf16(A, Wg, act_tile=256).float().cpu().numpy()
+    dllm.kernel_status()
+    want = A.double().cpu().numpy() @ W.double().cpu().numpy().T
+    assert rel_l2(c, want) < 1e-5
+    assert np.array_equal(c, c256) and np.array_equal(g, g256)
+    assert dllm.lib.dllm_gemm_bf16_planned(A.data_ptr(), W.data_ptr(), A.data_ptr(), M, N, K, 192, 2, 0, None, 0, None) == dllm.INVALID_ARG
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("B,R,width,k", [(1, 32, 256, 8), (3, 256, 4096, 64), (2, 100, 512, 50), (1, 512, 4096, 51),
                                          # the longest response the selection kernel admits (keys and flags of one

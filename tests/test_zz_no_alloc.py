@@ -32,10 +32,11 @@ def _inputs(torch, B, a, n, H, Hkv, hd, seed):
 
 def test_noalloc_matches_the_allocating_entry_point_on_two_calls_in_a_row(env):
     torch, dllm = env
-    # every shape splits the key range (few row tiles), so every call uses the built-in scratch: the first two
-    # on the 64-row kernel, the third on the 128-row tcgen05 kernel (128 rows per KV head); each is smaller than
-    # or differently laid out from the one before, so stale partials of the previous call lie in and behind its own
-    for i, shape in enumerate([(1, 64, 768, 8, 8, 128), (2, 19, 333, 4, 2, 64), (1, 128, 512, 8, 8, 128)]):
+    # every shape splits the key range into partials in scratch, so every call uses the built-in scratch: the
+    # first two on the 64-row kernel with more splits than a cluster merges (21 and 10), the third on the 128-row
+    # tcgen05 kernel (128 rows per KV head); each is differently laid out from the one before, so stale partials of
+    # the previous call lie in and behind its own
+    for i, shape in enumerate([(1, 36, 4128, 2, 2, 128), (2, 40, 2000, 2, 1, 64), (1, 128, 512, 8, 8, 128)]):
         B, a, n, H, Hkv, hd = shape
         assert dllm.lib.dllm_attention_scratch_bytes(B, a, n, H, Hkv, hd, dllm.BF16) > 0
         q, k, v = _inputs(torch, *shape, seed=100 + 10 * i)
@@ -53,8 +54,8 @@ def test_noalloc_matches_the_allocating_entry_point_on_two_calls_in_a_row(env):
 
 def test_noalloc_rejects_what_does_not_fit_its_scratch(env):
     torch, dllm = env
-    # 64 rows per KV head (the 64-row kernel): 128 row tiles, 12 key tiles -> 2 key splits -> 8.5 MB of partials
-    B, a, n, H, Hkv, hd = 1, 64, 768, 128, 128, 128
+    # 256 rows per KV head (the tcgen05 kernel), 16 heads, 2048 keys: key splits with 16 MB of partials
+    B, a, n, H, Hkv, hd = 1, 256, 2048, 16, 16, 128
     assert dllm.lib.dllm_attention_scratch_bytes(B, a, n, H, Hkv, hd, dllm.BF16) > 8 * 1024 * 1024
     q, k, v = _inputs(torch, B, a, n, H, Hkv, hd, seed=7)
     out = torch.zeros_like(q)
