@@ -280,7 +280,7 @@ def step_roof_ms(per_class, peaks):
 # dram__bytes_read.sum + dram__bytes_write.sum per projection launch, from an ncu capture of a two-layer case of
 # the same kernel scaled to the full depth (every layer streams its own weights); None where no capture of the
 # current kernel exists.
-TRAFFIC_PER_LAUNCH = {"llada8b": 96.2e6}
+TRAFFIC_PER_LAUNCH = {"llada8b": 96.4e6}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -353,14 +353,18 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
+    host_s = [0.0]   # host time spent in the step and transition calls (they only enqueue)
+
     def run_steps(n, per_step=None):
         for i in range(n):
             k = wl.steps - (i % wl.steps)
             if i and k == wl.steps:
-                ses.set_prompt(prompt)          # a new generation starts
+                ses.set_prompt(prompt)          # a new generation starts (a blocking copy from pageable memory)
+            t0 = time.perf_counter()
             ses.step_scheduled(k, wl.steps, wl.Kp, wl.Kr, wl.rho)
             bs, nt = block_plan(wl.steps - k, wl.steps, wl.gen_len, wl.block_len)
             ses.remask_low_confidence(bs, wl.block_len, nt)
+            host_s[0] += time.perf_counter() - t0
             if per_step:
                 per_step(i)
 
@@ -396,9 +400,9 @@ def main():
     l0 = ses.launch_count()
     torch.cuda.profiler.start()       # no-op unless a profiler waits for it (`ncu --profile-from-start off`)
     ev0.record(stream)
-    t_host = time.perf_counter()
+    host_s[0] = 0.0
     run_steps(K)
-    host_enqueue_ms = 1e3 * (time.perf_counter() - t_host)    # the host only enqueues: it runs ahead of the device
+    host_enqueue_ms = 1e3 * host_s[0]    # the host only enqueues: it runs ahead of the device
     ev1.record(stream)
     barrier()
     torch.cuda.profiler.stop()
@@ -536,6 +540,7 @@ def main():
         ses.profile(False)
     ses.use_graphs(True)
     partial_gemm_bytes = sum(v["bytes"] for k_, v in per_kind_work["partial"].items() if k_.startswith("gemm"))
+    partial_gemm_flops = sum(v["flops"] for k_, v in per_kind_work["partial"].items() if k_.startswith("gemm"))
 
     # max over ranks
     ms, ms_e2e = aggregate_over_ranks(ms, ms_e2e, world, dev)
@@ -548,6 +553,11 @@ def main():
     value = tokens / (ms / 1e3)
     kernels = {name: roofline_of(name, rec, peaks) for name, rec in prof.items()}
     kernels = {k_: v for k_, v in kernels.items() if v is not None}
+    # share of the summed event time of all launches ("gemm" and "attention" are sums of classes listed beside
+    # them): the figure to hold against the share column of a profiler's launch list of the same command
+    kernel_ms = sum(v["ms_total"] for k_, v in kernels.items() if k_ not in ("gemm", "attention"))
+    for v in kernels.values():
+        v["share_of_kernel_time"] = v["ms_total"] / max(kernel_ms, 1e-9)
     g = kernels["gemm"]
     steps_roof = {}
     for kind, work in per_kind_work.items():
@@ -584,6 +594,7 @@ def main():
                      "algorithmic_bytes_per_launch": g["bytes_per_launch"],
                      "algorithmic_flops_per_launch": g["flops_per_launch"],
                      "gemm_share_of_step": g["ms_total"] / max(ms_replay, 1e-9),
+                     "gemm_share_of_kernel_time": g["share_of_kernel_time"],
                      "how": "CUDA-event pairs around every launch (" +
                             ("event-record nodes in the step graphs" if args.prof_mode == "graph" else
                              "host records around plain launches") +
@@ -601,7 +612,8 @@ def main():
         line["config"]["cache"] = "response-only AttnOut / FFNOut"
     line["cache_bytes"] = int(ses.cache.numel())
     if world == 1 and not args.no_timeline and not args.layers and args.rho is None:
-        line["roofline"]["in_graph"] = in_graph_gemm(args.workload, partial_gemm_bytes, peaks)
+        line["roofline"]["in_graph"] = in_graph_gemm(args.workload, partial_gemm_bytes, partial_gemm_flops,
+                                                     line["roofline"]["bound"], peaks)
     if not args.no_cpu_baseline:
         t = time_oracle(wl, budget_s=25.0, steps=K)
         line["cpu_baseline"] = {"value": t["tokens_per_s"], "unit": "tokens/s", "cores": t["cores"], "kind": "oracle",
@@ -611,11 +623,12 @@ def main():
         dist.destroy_process_group()
 
 
-def in_graph_gemm(workload, gemm_bytes, peaks):
+def in_graph_gemm(workload, gemm_bytes, gemm_flops, bound, peaks):
     """GEMM time INSIDE the replayed graph of one adaptive partial step (programmatic dependent launch, warm L2),
     from the device timestamps of the timeline build, in a process of its own after this one has freed nothing it
-    needs: achieved = the step's algorithmic GEMM bytes / the summed in-graph durations of its GEMM launches.
-    Reported beside the event-pair figure, which serialises the launches.  None if the run fails."""
+    needs: achieved = the step's algorithmic GEMM bytes (flops where the class is tensor bound) / the summed
+    in-graph durations of its GEMM launches.  Reported beside the event-pair figure, which serialises the
+    launches.  None if the run fails."""
     try:
         with tempfile.TemporaryDirectory() as td:
             out = os.path.join(td, "tl.json")
@@ -627,9 +640,12 @@ def in_graph_gemm(workload, gemm_bytes, peaks):
         gemm = [o for o in launches if o["file"].startswith("gemm")]
         us = sum(o["dur_us"] for o in gemm)
         total = launches[-1]["start_us"]
-        gbs = gemm_bytes / (us * 1e-6) / 1e9
-        return {"achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                "frac_of_nominal": gbs / NOMINAL["hbm_gbs"], "gemm_us": us, "gemm_launches": len(gemm),
+        if bound == "tensor":
+            ach, unit, peak, nominal = gemm_flops / (us * 1e-6) / 1e12, "TFLOP/s", peaks["bf16_tflops_sustained"], NOMINAL["bf16_tflops"]
+        else:
+            ach, unit, peak, nominal = gemm_bytes / (us * 1e-6) / 1e9, "GB/s", peaks["hbm_gbs"], NOMINAL["hbm_gbs"]
+        return {"achieved": ach, "unit": unit, "frac": ach / peak,
+                "frac_of_nominal": ach / nominal, "gemm_us": us, "gemm_launches": len(gemm),
                 "step_us": total, "gemm_share_of_step": us / max(total, 1e-9),
                 "how": "one adaptive partial step replayed as a CUDA graph in the timeline build of the library: "
                        "per launch, device time from its predecessor's completion to its own (globaltimer at "
