@@ -328,9 +328,11 @@ dllm_status dllm_debug_gemm_plan(int persistent);
  * from which the 128-row tcgen05 kernel is taken instead of the 64-row mma.sync
  * kernel; and whether shapes with at most 32 rows per KV head and at least 1024
  * keys take the few-rows kernel (warps share the rows and split the key tiles;
- * 1, the default) or stay on the 64-row kernel (0).  Results stay within the
- * attention tolerance; the merge order changes with the plan. */
-dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows, int few_rows_kernel);
+ * 1, the default) or stay on the 64-row kernel (0); and whether a CTA of the
+ * tcgen05 kernel takes one or two 128-row tiles (tcgen05_row_tiles 1 or 2;
+ * 0 = the plan's choice).  Results stay within the attention tolerance; the
+ * merge order changes with the plan. */
+dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows, int few_rows_kernel, int tcgen05_row_tiles);
 dllm_status dllm_debug_skip_one_load(int enable);
 /* C[M,N] (fp32, row-major, DEVICE) = A[M,K] * W[N,K]^T with bf16 operands on
  * the tensor cores (tcgen05 + TMA).  d_partials is scratch of

@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ C
                                 &abort_flag, &tmK, &tmV, q, o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split,
                                 scale_log2, (int)gridDim.z / S, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z,
                                 q_by_tma ? &tmQ : nullptr);
-  if (!ok && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+  if (!ok && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_ATTN);
 }
 
 // ============================================================================
@@ -307,7 +307,7 @@ __global__ void __launch_bounds__(32 * RG * KW, RG == 2 ? 2 : 1)
     ok = __syncthreads_and(ok);
   }
   if (!ok) {
-    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_ATTN_FEW);
     drain_delay();
     return;
   }
@@ -487,6 +487,8 @@ int g_attn_force_splits = 0;
 int g_attn_umma_min_rows = AT_ROWS + 1;
 // 0: shapes with very few rows per KV head stay on the 64-row kernel (tuning / test switch)
 int g_attn_few_rows = 1;
+// 128-row tiles per CTA of the tcgen05 kernel: 0 = the plan's choice, 1 or 2 forced (tuning / test switch)
+int g_attn_umma_row_tiles = 0;
 
 // Key-range splits of the 64-row kernel, whole 64-key tiles per split: enough CTAs to cover the SMs when few
 // rows are active (every split costs the merge a partial per row and head, so no more than that), and two CTAs
@@ -687,14 +689,16 @@ extern "C" dllm_status dllm_attention_noalloc(const void* d_q, const void* d_k, 
   return DLLM_OK;
 }
 
-extern "C" dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows, int few_rows_kernel) {
-  if (splits < 0 || tcgen05_min_rows < 0) {
-    dllm::set_last_error("dllm_debug_attention_plan: arguments must not be negative");
+extern "C" dllm_status dllm_debug_attention_plan(int splits, int tcgen05_min_rows, int few_rows_kernel,
+                                                 int tcgen05_row_tiles) {
+  if (splits < 0 || tcgen05_min_rows < 0 || tcgen05_row_tiles < 0 || tcgen05_row_tiles > 2) {
+    dllm::set_last_error("dllm_debug_attention_plan: arguments must not be negative, row tiles 0, 1 or 2");
     return DLLM_INVALID_ARG;
   }
   dllm::g_attn_force_splits = splits;
   if (tcgen05_min_rows > 0) dllm::g_attn_umma_min_rows = tcgen05_min_rows;
   dllm::g_attn_few_rows = few_rows_kernel != 0;
+  dllm::g_attn_umma_row_tiles = tcgen05_row_tiles;
   return DLLM_OK;
 }
 

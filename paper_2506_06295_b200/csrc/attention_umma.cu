@@ -6,16 +6,17 @@
 // One CTA = TWO tiles of 128 "virtual rows" ((query, head-of-group) pairs) of
 // one (sequence, KV head) x one split of the key range, key tiles of 64, ten
 // warps with fixed roles:
-//   warp 9           TMA: the Q tiles, then K/V tiles into a three-stage ring
+//   warp 9           TMA: K/V tiles into a six-stage ring (all that shared memory holds)
 //   warp 8           issues every tcgen05.mma of the CTA
 //   warps 0-3, 4-7   the softmax group of row tile 0 resp. 1 (one row per thread)
 // Per key tile t and row tile i:
-//   S_i = Q_i K^T     tcgen05.mma, M = 128 rows, N = 64 keys, contraction HD; Q and
-//                     K in shared memory (K-major, 128-byte swizzle), S_i in TMEM
+//   S_i = Q_i K^T     tcgen05.mma, M = 128 rows, N = 64 keys, contraction HD; Q_i is
+//                     the A operand in tensor memory (written there once by its
+//                     group), K in shared memory (K-major, 128-byte swizzle)
 //   softmax           TMEM lane = row, so every thread of group i owns one row: it
 //                     loads its 64 scores with tcgen05.ld, takes max / exp2 / sum
-//                     locally (no shuffles) and writes P_i as bf16 into shared
-//                     memory in the layout of an MMA A operand
+//                     locally (no shuffles) and writes P_i as bf16 pairs over the
+//                     first 32 score columns: the A operand of the next product
 //   O_i += P_i V      tcgen05.mma, M = 128 rows, N = HD, contraction 64 keys; V is
 //                     used as stored ([key][hd], "MN-major" B operand); O_i
 //                     accumulates in TMEM and is rescaled (tcgen05.ld / st) only
@@ -24,9 +25,14 @@
 // The MMA warp issues O_i += P_i V of tile t and, right behind it, S_i of tile
 // t+1, alternating between the row tiles: while one group is in its softmax the
 // tensor pipe works for the other, and both row tiles read every K/V tile that
-// arrives once.  Key-range splits write unnormalised partials plus (max, sum)
-// exactly like the mma.sync kernel, and the same merge kernel finishes them.
-// Every mbarrier wait is bounded.
+// arrives once.  A CTA with ONE live row tile (at most 128 rows per KV head, the
+// odd last tile, or a plan of one-tile CTAs) gives both groups that tile's rows:
+// group 0 takes the even key tiles of the CTA's range and group 1 the odd ones,
+// each with its own scores, running maximum, sum and output accumulator, and the
+// two halves are merged through shared memory at the end (group 1's first).
+// Key-range splits write unnormalised partials plus (max, sum) exactly like the
+// mma.sync kernel, and the same merge kernel finishes them.  Every mbarrier wait
+// is bounded.
 #include "attention_core.cuh"
 #include "internal.h"
 #include "tma.cuh"
@@ -41,6 +47,10 @@ constexpr int UA_TILES = 2;
 constexpr int UA_KEYS = 64;    // keys per tile
 constexpr int UA_STAGES = 6;   // K/V ring
 constexpr int UA_THREADS = 320;  // two softmax groups of 128, one MMA warp, one TMA warp
+// key tiles from which a CTA with one live row tile shares them between its two softmax groups: the exchange and
+// merge of the two halves at the end cost about as much as the overlap saves on eight tiles (B200: 24 tiles per CTA
+// 135 -> 114 us at 16 x 128 rows x 1536 keys; 3-4 tiles per CTA 13.8 -> 15.0 us at 128 rows x 768 keys)
+constexpr int UA_KPAR_MIN_TILES = 8;
 
 // MN-major operand ([k][mn] rows of 64 mn-elements = 128 bytes, 128-byte swizzle,
 // panels of 64 mn-elements): lbo = bytes between panels along MN, sbo = bytes
@@ -132,6 +142,9 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
   const int key_hi = min(n, key_lo + keys_per_split);
   const int n_tiles = (key_hi - key_lo + UA_KEYS - 1) / UA_KEYS;  // >= 1 by construction of the plan
   const int dq = H * HD;
+  // one live row tile and enough key tiles: both softmax groups work on that tile's rows, group i on the key
+  // tiles t with t % 2 == i
+  const bool kpar = live == 1 && n_tiles >= UA_KPAR_MIN_TILES;
 
   if (tid == 0) {
     abort_flag = 0;
@@ -205,11 +218,44 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
         umma_commit(smem_u32(&s_full[i]));
       };
       ok = mbar_wait(smem_u32(&q_bar), 0u, abortp) && mbar_wait(smem_u32(&kv_full[0]), 0u, abortp);
-      if (ok) {
+      if (ok && kpar) {
+        // group i owns key tiles i, i + 2, ...: S_0(0), S_1(1); then per tile t (group i = t % 2):
+        // O_i += P_i(t) V(t) and right behind it S_i(t + 2)
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        issue_s(0, 0);
+        ok = mbar_wait(smem_u32(&kv_full[1]), 0u, abortp);
+        if (ok) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          issue_s(1, 1);
+        }
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          const int i = t & 1, u = t >> 1;
+          const int st = t % UA_STAGES;
+          const uint32_t v_s = kv_s + st * SM::STAGE + SM::KV_TILE;
+          ok = mbar_wait(smem_u32(&p_full[i]), (uint32_t)u & 1u, abortp);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+          for (int ks = 0; ks < UA_KEYS / 16; ++ks)
+            umma_bf16_ta(tmem + SM::O_COL + (uint32_t)(i * HD), tmem + SM::S_COL + (uint32_t)(i * UA_KEYS + ks * 8),
+                         make_smem_desc_mn(v_s + ks * (16 * 128), UA_KEYS * 128, 1024), idesc_o,
+                         (u > 0 || ks > 0) ? 1u : 0u);
+          if (t + 2 < n_tiles) {
+            const int st2 = (t + 2) % UA_STAGES;
+            ok = mbar_wait(smem_u32(&kv_full[st2]), (uint32_t)((t + 2) / UA_STAGES) & 1u, abortp);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            issue_s(i, st2);
+          } else {
+            umma_commit(smem_u32(&o_full[i]));  // the group's last tile: O_i is final when this fires
+          }
+          umma_commit(smem_u32(&kv_empty[st]));  // only group i reads tile t
+        }
+      } else if (ok) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         for (int i = 0; i < live; ++i) issue_s(i, 0);
       }
-      for (int t = 0; t < n_tiles && ok; ++t) {
+      for (int t = 0; t < n_tiles && ok && !kpar; ++t) {
         const int st = t % UA_STAGES, st_next = (t + 1) % UA_STAGES;
         const uint32_t v_s = kv_s + st * SM::STAGE + SM::KV_TILE;
         bool next_ready = t + 1 >= n_tiles;
@@ -247,11 +293,11 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
     {
       // Q_i: every thread fetches its own row (HD bf16 = HD / 8 16-byte words, zero past the last row) and
       // writes it to its TMEM lane as bf16 pairs; all loads of a thread are in flight before the first use
-      const int vr = row0 + i * UA_ROWS + row;
+      const int vr = row0 + (kpar ? 0 : i * UA_ROWS) + row;
       uint4 qv[HD / 8];
 #pragma unroll
       for (int w = 0; w < HD / 8; ++w) qv[w] = make_uint4(0, 0, 0, 0);
-      if (vr < n_rows && i < live) {
+      if (vr < n_rows && (i < live || kpar)) {
         const int qi = vr / G, g = vr - qi * G;
         const uint4* src = reinterpret_cast<const uint4*>(q + ((size_t)b * a_seq + qi) * dq + (kh * G + g) * HD);
 #pragma unroll
@@ -280,12 +326,14 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
     // TMEM is only rescaled when the maximum has grown by more than RESCALE_STEP, which keeps every exponential
     // below 2^8)
     float m_ref = -INFINITY, l_run = 0.f;
-    if (i < live) {
-      for (int t = 0; t < n_tiles; ++t) {
-        ok = mbar_wait(smem_u32(&s_full[i]), (uint32_t)t & 1u, abortp);
+    if (i < live || kpar) {
+      // u counts this group's tiles; with kpar they are the key tiles i, i + 2, ...
+      const int t_step = kpar ? 2 : 1;
+      for (int t = kpar ? i : 0, u = 0; t < n_tiles; t += t_step, ++u) {
+        ok = mbar_wait(smem_u32(&s_full[i]), (uint32_t)u & 1u, abortp);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (gtid == 0 && i == 0) timeline_mark(2 + (t < 5 ? t : 5));  // scores of tile t complete
+        if (gtid == 0 && i == 0) timeline_mark(2 + (u < 5 ? u : 5));  // scores of this group's tile u complete
         // ---- this thread's row of scores (raw: the scale is folded into the exponent's multiply-add)
         const int valid = key_hi - (key_lo + t * UA_KEYS);  // >= 1
         float sv[UA_KEYS];
@@ -313,12 +361,12 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
         // ---- lazy rescale of O (warp-uniform branch: the TMEM accesses are warp-collective)
         const bool grow = mx > m_ref + RESCALE_STEP;
         if (__any_sync(0xffffffffu, grow)) {
-          const float corr = grow ? exp2f(m_ref - mx) : 1.f;  // first tile: exp2(-inf) = 0, O is not read (t == 0)
+          const float corr = grow ? exp2f(m_ref - mx) : 1.f;  // first tile: exp2(-inf) = 0, O is not read (u == 0)
           if (grow) {
             m_ref = mx;
             l_run *= corr;
           }
-          if (t > 0) {
+          if (u > 0) {
 #pragma unroll
             for (int c = 0; c < HD; c += 32) {
               uint32_t r[32];
@@ -350,10 +398,54 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
       }
       if (ok) ok = mbar_wait(smem_u32(&o_full[i]), 0u, abortp);
       ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below are warp-collective
-      if (ok) {
+      // ---- one live row tile shared by the groups: group 1 hands its half (max, sum, unnormalised output) to
+      // group 0 through the K/V ring, which nothing reads any more once both groups' last products are complete
+      constexpr int XS = HD + 4;  // floats per exchanged row: 16-byte aligned, rows 4 banks apart
+      float* xo = reinterpret_cast<float*>(smem_raw + (base - smem_u32(smem_raw)));
+      float* xml = xo + UA_ROWS * XS;
+      float w_self = 1.f, w_peer = 0.f;  // weights of this group's and the other group's half in the merged row
+      bool peer = false, write_out = ok;
+      if (kpar) {
+        static_assert((UA_ROWS * XS + 2 * UA_ROWS) * 4 <= UA_STAGES * SM::STAGE, "the exchange area must fit the ring");
+        {  // both groups are past their last product (or gave up): all 256 threads agree
+          uint32_t r;
+          asm volatile(
+              "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, 2, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+              : "=r"(r)
+              : "r"((uint32_t)ok)
+              : "memory");
+          ok = r != 0;
+        }
+        if (ok && i == 1) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+          for (int c = 0; c < HD; c += 32) {
+            uint32_t r[32];
+            tmem_ld32(tmem + row_lane + o_col + (uint32_t)c, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int k = 0; k < 32; k += 4)
+              *reinterpret_cast<uint4*>(xo + row * XS + c + k) = make_uint4(r[k], r[k + 1], r[k + 2], r[k + 3]);
+          }
+          xml[2 * row] = m_ref;
+          xml[2 * row + 1] = l_run;
+        }
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        write_out = ok && i == 0;  // group 0 writes the merged rows
+        if (write_out) {
+          const float m1 = xml[2 * row], l1 = xml[2 * row + 1];
+          const float M = fmaxf(m_ref, m1);
+          w_self = exp2f(m_ref - M);
+          w_peer = exp2f(m1 - M);
+          l_run = w_self * l_run + w_peer * l1;
+          m_ref = M;
+          peer = true;
+        }
+      }
+      if (write_out) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (gtid == 0 && i == 0) timeline_mark(8);  // O complete
-        const int vr = row0 + i * UA_ROWS + row;
+        const int vr = row0 + (kpar ? 0 : i * UA_ROWS) + row;
         const bool is_live = vr < n_rows;
         const int qi = is_live ? vr / G : 0, g = is_live ? vr - qi * G : 0;
         const size_t orow = ((size_t)b * a_seq + qi) * H + (kh * G + g);  // (row, head) index
@@ -365,6 +457,16 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
           tmem_ld32(tmem + row_lane + o_col + (uint32_t)c, r);  // warp-collective: every lane takes part
           tmem_ld_wait();
           if (!is_live) continue;
+          if (peer) {
+#pragma unroll
+            for (int k = 0; k < 32; k += 4) {
+              const float4 x = *reinterpret_cast<const float4*>(xo + row * XS + c + k);
+              r[k] = __float_as_uint(w_self * __uint_as_float(r[k]) + w_peer * x.x);
+              r[k + 1] = __float_as_uint(w_self * __uint_as_float(r[k + 1]) + w_peer * x.y);
+              r[k + 2] = __float_as_uint(w_self * __uint_as_float(r[k + 2]) + w_peer * x.z);
+              r[k + 3] = __float_as_uint(w_self * __uint_as_float(r[k + 3]) + w_peer * x.w);
+            }
+          }
           if (S == 1) {
             __nv_bfloat16* dst = o + orow * HD + c;
 #pragma unroll
@@ -392,7 +494,7 @@ __global__ void __launch_bounds__(UA_THREADS, 1)
   // a wait that gave up anywhere in the CTA: record it once, let copies in flight land
   ok = __syncthreads_and(ok);
   if (!ok) {
-    if (tid == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+    if (tid == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_ATTN_UMMA);
     drain_delay();
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -431,8 +533,9 @@ cudaError_t launch_umma(const Launch& L, const CUtensorMap& tmK, const CUtensorM
 // holds.  A split shortens the key range a CTA walks through but adds a partial result per (row, head) pair that
 // the merge has to write and read, and a CTA with one row tile instead of two doubles the CTAs but loses the
 // overlap of the two softmax groups, so both are what a small cost model likes best (microseconds, fitted to
-// sweeps on B200: per key tile of a CTA 1.76 us with two row tiles and 1.36 us with one, one CTA per SM at a
-// time, 4 us of fixed cost, and for a merge 2.5 us plus 1040 bytes per pair and split at 5 TB/s).
+// sweeps on B200: per key tile of a CTA 1.76 us with two row tiles, 1.36 us with one and 1.15 us with one whose
+// groups share the key tiles, one CTA per SM at a time, 4 us of fixed cost, and for a merge 2.5 us plus 1040 bytes
+// per pair and split at 5 TB/s).
 AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scratch_floats) {
   AttnPlan p;
   const int G = H / Hkv, sms = sm_count();
@@ -442,11 +545,14 @@ AttnPlan plan_attention_umma(int B, int a_seq, int n, int H, int Hkv, size_t scr
   int best_s = 1, best_rt = UA_TILES;
   double best_us = -1.0;
   for (int rt = UA_TILES; rt >= 1; --rt) {   // row tiles per CTA: two (the groups overlap), or one (twice the CTAs)
+    if (g_attn_umma_row_tiles && rt != g_attn_umma_row_tiles) continue;
     const long ctas = (long)((a_seq * G + rt * UA_ROWS - 1) / (rt * UA_ROWS)) * Hkv * B;
-    const double tile_us = rt == 2 ? 1.76 : 1.36;  // a key tile of a CTA, from 16 x 512 x 1536 and 16 x 128 x 1536
     for (int S = 1; S <= key_tiles && S <= 16; ++S) {
       if (S > 1 && (size_t)S * per_split > scratch_floats) break;
       const int tps = (key_tiles + S - 1) / S;
+      // a key tile of a CTA, from 16 x 512 x 1536 and 16 x 128 x 1536 (the latter with and without the two groups
+      // sharing the key tiles)
+      const double tile_us = rt == 2 ? 1.76 : tps >= UA_KPAR_MIN_TILES ? 1.15 : 1.36;
       if (S > 1 && (key_tiles + tps - 1) / tps != S) continue;  // the same tiles per split as a smaller count
       const double waves = (double)((ctas * S + sms - 1) / sms);
       const double us = 4.0 + waves * tps * tile_us + (S > 1 ? 2.5 + S * pairs * 1040.0 / 5.0e6 : 0.0);

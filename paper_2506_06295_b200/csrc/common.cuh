@@ -47,7 +47,14 @@ struct OutRows {
 };
 
 // device status word codes
-enum : int { ST_OK = 0, ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103, ST_TIMEOUT_GRID = 104, ST_RANGE = 201 };
+enum : int {
+  ST_OK = 0,
+  ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103,  // GEMM: operand copies, MMA issuer, epilogue
+  ST_TIMEOUT_GRID = 104,
+  ST_TIMEOUT_ATTN = 111, ST_TIMEOUT_ATTN_FEW = 112, ST_TIMEOUT_ATTN_UMMA = 113,  // attention: 64-row, few-rows, tcgen05
+  ST_TIMEOUT_ROWS_TAIL = 121, ST_TIMEOUT_ROWS_VVERIFY = 122,                   // streaming row kernels
+  ST_RANGE = 201
+};
 
 // Programmatic dependent launch.  pdl_wait(): blocks until the preceding grid
 // in the stream has completed and its writes are visible (returns at once for

@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1)
   }
   ok = __syncthreads_and(ok);
   if (!ok) {
-    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_ROWS_TAIL);
     drain_delay();
   }
 }
@@ -267,7 +267,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1)
   }
   ok = __syncthreads_and(ok);
   if (!ok) {
-    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_TMA);
+    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_ROWS_VVERIFY);
     drain_delay();
   }
 }

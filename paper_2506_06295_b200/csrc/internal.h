@@ -237,6 +237,7 @@ AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scra
 extern int g_attn_force_splits;   // tuning override of both plans' split count (0 = automatic)
 extern int g_attn_umma_min_rows;  // rows per KV head from which the tcgen05 kernel is taken
 extern int g_attn_few_rows;       // 0: never the few-rows kernel
+extern int g_attn_umma_row_tiles; // tcgen05 kernel: 0 = the plan chooses one or two 128-row tiles per CTA, 1 / 2 forced
 // bf16 with head_dim 64 / 128 runs on the tensor cores (scratch holds the
 // partials of split key ranges; without it one split is used); everything else
 // on the plain-ALU kernel.

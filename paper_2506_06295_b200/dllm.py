@@ -100,7 +100,7 @@ SIGNATURES = {
     "dllm_kernel_status": (_I, [_P]),
     "dllm_debug_set_wait_limit_ns": (_I, [C.c_uint64]),
     "dllm_debug_skip_one_load": (_I, [_I]),
-    "dllm_debug_attention_plan": (_I, [_I, _I, _I]),
+    "dllm_debug_attention_plan": (_I, [_I, _I, _I, _I]),
     "dllm_debug_gemm_plan": (_I, [_I]),
 }
 for _name, (_res, _args) in SIGNATURES.items():

@@ -164,6 +164,12 @@ ATT_CASES = [
     (2, 512, 1536, 2, 2, 128), # batched-serving refresh shape: 24 key tiles, two full CTAs per (sequence, head)
     (1, 40, 200, 28, 4, 128),  # grouped heads: 280 rows per KV head gathered from 7 query heads (no TMA for Q)
     (1, 200, 3000, 1, 1, 64),  # head_dim 64, one CTA's worth of rows against 47 key tiles: many key-range splits
+    # one live 128-row tile per CTA: its two softmax groups take the even and the odd key tiles and merge at the end
+    (1, 100, 1000, 4, 4, 128), # ragged rows, 16 key tiles with a ragged last one
+    (2, 128, 520, 2, 2, 64),   # nine key tiles: five for group 0, four for group 1 (the last with 8 keys)
+    (1, 128, 512, 2, 2, 128),  # eight key tiles, the fewest that are shared
+    (1, 128, 448, 2, 2, 128),  # seven key tiles: not shared, the second group idles
+    (4, 128, 1536, 4, 4, 128), # batched adaptive step shape: 24 key tiles per CTA
 ]
 
 
