@@ -633,7 +633,8 @@ def in_graph_gemm(workload, gemm_bytes, gemm_flops, bound, peaks):
         with tempfile.TemporaryDirectory() as td:
             out = os.path.join(td, "tl.json")
             r = subprocess.run([sys.executable, "-m", "paper_2506_06295_b200.timeline", "--workload", workload,
-                                "--kind", "partial", "--json", out], cwd=ROOT, capture_output=True, text=True, timeout=600)
+                                "--kind", "partial", "--no-marks", "--json", out], cwd=ROOT, capture_output=True,
+                               text=True, timeout=600)
             if r.returncode != 0:
                 return None
             launches = json.load(open(out))

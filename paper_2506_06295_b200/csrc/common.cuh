@@ -72,6 +72,7 @@ __device__ __forceinline__ void timeline_mark(int) {}
 // t_resident, t_released, SM id | CTA << 32}, one array and one cursor per translation unit.
 static __device__ unsigned long long* g_timeline;
 static __device__ unsigned int g_timeline_n;
+static __device__ int g_timeline_marks = 1;  // 0: only the launches are recorded, the marks inside kernels are not
 constexpr unsigned int TIMELINE_CAP = 1u << 20;
 __device__ __forceinline__ unsigned long long timeline_now() {
   unsigned long long t;
@@ -100,7 +101,7 @@ __device__ __forceinline__ void pdl_wait() {
 // A point inside a kernel (called by one thread per CTA): the same record with the mark in the top four bits of
 // the first word and the time in the second and third.
 __device__ __forceinline__ void timeline_mark(int id) {
-  if (g_timeline == nullptr) return;
+  if (g_timeline == nullptr || !g_timeline_marks) return;
   const unsigned long long t = timeline_now();
   const unsigned int i = atomicAdd(&g_timeline_n, 1u);
   if (i < TIMELINE_CAP) {
@@ -112,9 +113,13 @@ __device__ __forceinline__ void timeline_mark(int id) {
     g_timeline[4 * i + 3] = (unsigned long long)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) << 32;
   }
 }
-// One pair of host entry points per translation unit: set the record array (device, 32 bytes x 2^20; NULL = off)
-// and clear the cursor; read the cursor.
+// Host entry points per translation unit: set the record array (device, 32 bytes x 2^20; NULL = off) and clear
+// the cursor; read the cursor; switch the marks inside kernels on or off (each costs an atomic and four stores,
+// which a figure of what the launches cost should not contain).
 #define DLLM_TIMELINE_HOOKS(stem)                                              \
+  extern "C" int dllm_timeline_marks_##stem(int on) {                          \
+    return (int)cudaMemcpyToSymbol(dllm::g_timeline_marks, &on, sizeof on);    \
+  }                                                                            \
   extern "C" int dllm_timeline_set_##stem(unsigned long long* d_records) {     \
     unsigned int zero = 0;                                                     \
     cudaError_t e = cudaMemcpyToSymbol(dllm::g_timeline, &d_records, sizeof d_records); \

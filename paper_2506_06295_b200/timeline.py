@@ -28,9 +28,10 @@ KINDS = {"full": (True, True), "refresh": (False, True), "mixed": (True, False),
 RECORD_CAP = 1 << 20
 
 
-def collect(workload: str, kind: str):
+def collect(workload: str, kind: str, marks: bool = True):
     """Runs one step and returns the launches in completion order: dicts with file, grid, block, ctas,
-    start_us (predecessor complete), resident_before_us, last_cta_us, dur_us."""
+    start_us (predecessor complete), resident_before_us, last_cta_us, dur_us.  marks=False: the marks inside
+    the kernels are not recorded (they slow the projections down by several percent)."""
     from . import build as build_mod
     os.environ["DLLM_B200_LIB"] = build_mod.build(timeline=True)
     import torch
@@ -53,6 +54,8 @@ def collect(workload: str, kind: str):
         bufs[st] = torch.zeros(RECORD_CAP * 4, dtype=torch.int64, device=model.device)
         if setter(C.c_void_p(bufs[st].data_ptr())) != 0:
             raise RuntimeError("could not arm the timeline of " + st)
+        if getattr(dllm.lib, "dllm_timeline_marks_" + st)(1 if marks else 0) != 0:
+            raise RuntimeError("could not switch the marks of " + st)
     torch.cuda.synchronize()
     ses.step_cached(rp, rr, wl.rho)
     ses.sync()
@@ -105,8 +108,9 @@ def main(argv=None) -> int:
     ap.add_argument("--kind", default="partial", choices=sorted(KINDS))
     ap.add_argument("--layer", type=int, default=5, help="layer whose launches are listed one by one")
     ap.add_argument("--json", default=None, help="write every launch to this file")
+    ap.add_argument("--no-marks", action="store_true", help="record the launches only, not the marks inside kernels")
     args = ap.parse_args(argv)
-    out, n_layers, truncated = collect(args.workload, args.kind)
+    out, n_layers, truncated = collect(args.workload, args.kind, marks=not args.no_marks)
     if args.json:
         with open(args.json, "w") as f:
             json.dump(out, f)
