@@ -272,6 +272,100 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1)
   }
 }
 
+// After the O projection, streaming: see oproj_epilogue_kernel.  Stage = [projected row fp32 | x row fp32] of
+// active row r (carried row act[r]).
+template <typename T>
+__global__ void __launch_bounds__(STREAM_THREADS, 1)
+    oproj_stream_kernel(const float* __restrict__ part, const int32_t* __restrict__ act, const float* __restrict__ x,
+                        const float* __restrict__ gain2, OutRows Ac, T* __restrict__ hn, Geo g, int Ma, float eps,
+                        int stages, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STREAM_MAX_STAGES], empty_bar[STREAM_MAX_STAGES];
+  __shared__ int meta[STREAM_MAX_STAGES];
+  __shared__ int abort_flag;
+  const int d = g.d, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rb = (uint32_t)d * 4, stage_bytes = 2 * rb;
+  const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
+  uint8_t* base_gen = smem_raw + (base - smem_u32(smem_raw));
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_wait();
+  pdl_trigger();
+  volatile int* abortp = &abort_flag;
+  const int my_rows = (int)blockIdx.x < Ma ? (Ma - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  bool ok = true;
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int i = 0; i < my_rows; ++i) {
+        const int s = i % stages, r = blockIdx.x + i * gridDim.x;
+        if (i >= stages && !mbar_wait(smem_u32(&empty_bar[s]), (uint32_t)(i / stages - 1) & 1u, abortp)) {
+          ok = false;
+          break;
+        }
+        const int c = act[r];
+        meta[s] = c;
+        const uint32_t dst = base + s * stage_bytes, bar = smem_u32(&full_bar[s]);
+        mbar_expect_tx(bar, stage_bytes);
+        bulk_load_1d(dst, part + (size_t)r * d, rb, bar);
+        bulk_load_1d(dst + rb, x + (size_t)c * d, rb, bar);
+      }
+    }
+  } else {
+    const int w = warp - 1;
+    for (int i = w; i < my_rows; i += STREAM_CONSUMERS) {
+      const int s = i % stages, r = blockIdx.x + i * gridDim.x;
+      ok = mbar_wait(smem_u32(&full_bar[s]), (uint32_t)(i / stages) & 1u, abortp);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const int c = meta[s];
+      const float* ps = reinterpret_cast<const float*>(base_gen + (size_t)s * stage_bytes);
+      float* xs = reinterpret_cast<float*>(base_gen + (size_t)s * stage_bytes + rb);
+      T* arow = Ac.row<T>(c, g);
+      float ss = 0.f;
+      for (int j = lane * 8; j < d; j += 256) {
+        float a[8], xv[8];
+        Vec8<float>::load(ps + j, a);
+        Vec8<float>::load(xs + j, xv);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          a[t] = Vec8<T>::round(a[t]);
+          xv[t] += a[t];
+          ss += xv[t] * xv[t];
+        }
+        Vec8<T>::store(arow + j, a);
+        Vec8<float>::store(xs + j, xv);   // kept for the second pass
+      }
+      ss = warp_sum(ss);
+      const float rs = rsqrtf(ss / (float)d + eps);
+      T* out = hn + (size_t)r * d;
+      for (int j = lane * 8; j < d; j += 256) {
+        float v[8], gv[8];
+        Vec8<float>::load(xs + j, v);
+        Vec8<float>::load(gain2 + j, gv);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) v[t] = v[t] * rs * gv[t];
+        Vec8<T>::store(out + j, v);
+      }
+      // the stage was written by this warp through the generic proxy; the next bulk copy goes through the async one
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));
+    }
+  }
+  ok = __syncthreads_and(ok);
+  if (!ok) {
+    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_ROWS_OEPI);
+    drain_delay();
+  }
+}
+
 // Rows from which the streaming forms are taken (a property of the session's response rows, so that every
 // step kind of a session reduces a row in the same order).
 constexpr int STREAM_MIN_ROWS = 1024;
@@ -796,6 +890,24 @@ __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__
 void launch_oproj_epilogue(const Launch& L, int dtype, Partials part, const int32_t* act, const float* x,
                            const float* gain2, OutRows Ac_layer, void* hn, Geo g, int Ma, float eps) {
   if (Ma <= 0) return;
+  const size_t stage = (size_t)g.d * 8;
+  if (g.B * g.R >= STREAM_MIN_ROWS && part.S == 1 && part.upc == 0 && (g.d & 7) == 0 &&
+      stream_stages(stage) >= STREAM_CONSUMERS + 1) {
+    const int stages = stream_stages(stage);
+    const size_t smem = (size_t)stages * stage + 128;
+    const int ctas = std::min(Ma, sm_count());
+    DLLM_DISPATCH(dtype, {
+      static DeviceOnce once;
+      cudaError_t e0 = once.run([] {
+        return cudaFuncSetAttribute(oproj_stream_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
+      });
+      if (e0 == cudaSuccess)
+        launch_k(L, oproj_stream_kernel<T>, dim3(ctas), dim3(STREAM_THREADS), smem, part.p, act, x, gain2, Ac_layer,
+                 (T*)hn, g, Ma, eps, stages, L.d_status);
+    });
+    L.count();
+    return;
+  }
   const int threads = row_threads(g.d);
   const size_t smem = g.d <= threads * 8 ? 0 : (size_t)g.d * sizeof(float);  // staging only if a row takes several passes
   DLLM_DISPATCH(dtype, (launch_k(L, oproj_epilogue_kernel<T>, dim3(Ma), dim3(threads), smem, part, act, x, gain2, Ac_layer,
