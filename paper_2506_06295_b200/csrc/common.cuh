@@ -52,7 +52,8 @@ enum : int {
   ST_TIMEOUT_TMA = 101, ST_TIMEOUT_MMA = 102, ST_TIMEOUT_EPI = 103,  // GEMM: operand copies, MMA issuer, epilogue
   ST_TIMEOUT_GRID = 104,
   ST_TIMEOUT_ATTN = 111, ST_TIMEOUT_ATTN_FEW = 112, ST_TIMEOUT_ATTN_UMMA = 113,  // attention: 64-row, few-rows, tcgen05
-  ST_TIMEOUT_ROWS_TAIL = 121, ST_TIMEOUT_ROWS_VVERIFY = 122, ST_TIMEOUT_ROWS_OEPI = 123,  // streaming row kernels
+  ST_TIMEOUT_ROWS_TAIL = 121, ST_TIMEOUT_ROWS_VVERIFY = 122, ST_TIMEOUT_ROWS_OEPI = 123,
+  ST_TIMEOUT_ROWS_ROPE = 124,  // streaming row kernels
   ST_RANGE = 201
 };
 

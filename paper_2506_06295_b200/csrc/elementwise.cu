@@ -366,6 +366,97 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1)
   }
 }
 
+// RoPE + K scatter, streaming: see qk_rope_kernel.  Stage = the projected [Q | K] row (fp32) of active row r.  A
+// consumer warp rotates a whole row: hd / 8 lanes cover the hd / 2 pairs of a head four at a time (element i with
+// i + hd / 2), so a warp takes 256 / hd heads per trip; the row's cos / sin values are read once.
+template <typename T>
+__global__ void __launch_bounds__(STREAM_THREADS, 1)
+    qk_rope_stream_kernel(const float* __restrict__ part, const int32_t* __restrict__ act,
+                          const float* __restrict__ rope_tab, T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int Ma,
+                          int H, int Hkv, int hd, int stages, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STREAM_MAX_STAGES], empty_bar[STREAM_MAX_STAGES];
+  __shared__ int meta[STREAM_MAX_STAGES];
+  __shared__ int abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int dq = H * hd, dkv = Hkv * hd, width = dq + dkv, half = hd >> 1;
+  const uint32_t stage_bytes = (uint32_t)width * 4;
+  const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
+  uint8_t* base_gen = smem_raw + (base - smem_u32(smem_raw));
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    mbar_fence_init();
+  }
+  __syncthreads();
+  pdl_wait();
+  pdl_trigger();
+  volatile int* abortp = &abort_flag;
+  const int my_rows = (int)blockIdx.x < Ma ? (Ma - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  bool ok = true;
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int i = 0; i < my_rows; ++i) {
+        const int s = i % stages, r = blockIdx.x + i * gridDim.x;
+        if (i >= stages && !mbar_wait(smem_u32(&empty_bar[s]), (uint32_t)(i / stages - 1) & 1u, abortp)) {
+          ok = false;
+          break;
+        }
+        meta[s] = act[r];
+        const uint32_t bar = smem_u32(&full_bar[s]);
+        mbar_expect_tx(bar, stage_bytes);
+        bulk_load_1d(base + s * stage_bytes, part + (size_t)r * width, stage_bytes, bar);
+      }
+    }
+  } else {
+    const int w = warp - 1;
+    const int lph = hd >> 3;                 // lanes per head: four pairs each
+    const int hpt = 32 / lph;                // heads per trip of a warp
+    const int hl = lane / lph, i0 = (lane - hl * lph) * 4;
+    for (int i = w; i < my_rows; i += STREAM_CONSUMERS) {
+      const int s = i % stages, r = blockIdx.x + i * gridDim.x;
+      ok = mbar_wait(smem_u32(&full_bar[s]), (uint32_t)(i / stages) & 1u, abortp);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      int b, pos;
+      carried_to_pos(meta[s], g, b, pos);
+      const float* row = reinterpret_cast<const float*>(base_gen + (size_t)s * stage_bytes);
+      const float* tab = rope_tab + (size_t)pos * hd;  // [cos(half) | sin(half)]
+      const float4 cs = *reinterpret_cast<const float4*>(tab + i0);
+      const float4 sn = *reinterpret_cast<const float4*>(tab + half + i0);
+      const float cc[4] = {cs.x, cs.y, cs.z, cs.w}, ss[4] = {sn.x, sn.y, sn.z, sn.w};
+      T* qrow = qbuf + (size_t)r * dq;
+      T* krow = Kc + ((size_t)b * g.n + pos) * dkv;
+      for (int h0 = 0; h0 < H + Hkv; h0 += hpt) {
+        const int head = h0 + hl;
+        if (head >= H + Hkv) break;          // the last trip may be partly empty
+        const float4 lo4 = *reinterpret_cast<const float4*>(row + head * hd + i0);
+        const float4 hi4 = *reinterpret_cast<const float4*>(row + head * hd + half + i0);
+        const float lo[4] = {lo4.x, lo4.y, lo4.z, lo4.w}, hi[4] = {hi4.x, hi4.y, hi4.z, hi4.w};
+        float o_lo[4], o_hi[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          o_lo[t] = lo[t] * cc[t] - hi[t] * ss[t];
+          o_hi[t] = hi[t] * cc[t] + lo[t] * ss[t];
+        }
+        T* dst = head < H ? qrow + head * hd : krow + (head - H) * hd;
+        store4<T>(dst + i0, o_lo);
+        store4<T>(dst + i0 + half, o_hi);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));
+    }
+  }
+  ok = __syncthreads_and(ok);
+  if (!ok) {
+    if (threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_ROWS_ROPE);
+    drain_delay();
+  }
+}
+
 // Rows from which the streaming forms are taken (a property of the session's response rows, so that every
 // step kind of a session reduces a row in the same order).
 constexpr int STREAM_MIN_ROWS = 1024;
@@ -797,6 +888,25 @@ __global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, c
 void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* act, const float* rope_tab, void* qbuf,
                     void* Kc_layer, Geo g, int Ma, int H, int Hkv, int hd) {
   if (Ma <= 0) return;
+  const size_t stage = (size_t)(H + Hkv) * hd * 4;
+  // streaming form: unsplit slabs, a head size whose pairs a group of lanes covers exactly (a power of two, 32..256)
+  if (g.B * g.R >= STREAM_MIN_ROWS && part.S == 1 && part.upc == 0 && hd >= 32 && hd <= 256 && (hd & (hd - 1)) == 0 &&
+      stream_stages(stage) >= STREAM_CONSUMERS + 1) {
+    const int stages = stream_stages(stage);
+    const size_t smem = (size_t)stages * stage + 128;
+    const int ctas = std::min(Ma, sm_count());
+    DLLM_DISPATCH(dtype, {
+      static DeviceOnce once;
+      cudaError_t e0 = once.run([] {
+        return cudaFuncSetAttribute(qk_rope_stream_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024);
+      });
+      if (e0 == cudaSuccess)
+        launch_k(L, qk_rope_stream_kernel<T>, dim3(ctas), dim3(STREAM_THREADS), smem, part.p, act, rope_tab, (T*)qbuf,
+                 (T*)Kc_layer, g, Ma, H, Hkv, hd, stages, L.d_status);
+    });
+    L.count();
+    return;
+  }
   const long total = (long)Ma * (H + Hkv) * (hd >> 3);
   const unsigned blocks = (unsigned)((total + 255) / 256);
   DLLM_DISPATCH(dtype, (launch_k(L, qk_rope_kernel<T>, dim3(blocks), dim3(256), 0, part, act, rope_tab, (T*)qbuf,
