@@ -825,7 +825,9 @@ cudaError_t launch_select(const Launch& L, const float* sim, const int32_t* forc
   });
   if (e != cudaSuccess) return e;
   const size_t smem = (size_t)g.R * 9 + 16;
-  e = launch_k(L, select_kernel, dim3(g.B), dim3(256), smem, sim, forced, mode, ksel, sel, sel_stride, act, inv, g,
+  // one key per thread up to 1024 response rows (the rank of a key costs R comparisons of its thread)
+  const int threads = g.R <= 256 ? 256 : g.R >= 1024 ? 1024 : (g.R + 31) / 32 * 32;
+  e = launch_k(L, select_kernel, dim3(g.B), dim3(threads), smem, sim, forced, mode, ksel, sel, sel_stride, act, inv, g,
                refresh_prompt);
   L.count();
   return e;
