@@ -863,9 +863,9 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
   p.pair = 0;
   int pair_stages = 3;
   if (force_pair == 0 && force_bn == 0 && force_split <= 1 && N % (2 * TILE_W) == 0) {
-    // CTA pairs where they measured faster (B200): products that need no split between 65 and 1024 activation
+    // CTA pairs where they measured faster (B200): products that need no split between 129 and 1024 activation
     // rows, where the activation tile's trips through the L2 -> SM fabric bound the one-CTA kernel.
-    if (M > 64 && M <= 256 && n_tiles >= sms) {
+    if (M > 128 && M <= 256 && n_tiles >= sms) {   // (65..128 rows: one-CTA 128-row tiles measured 10 % faster)
       p.pair = 1;
       p.BN = 256;
     } else if (M > 256 && M <= 1024 && n_tiles * ((M + 255) / 256) <= sms) {
