@@ -862,19 +862,35 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
   p.BN = M <= 32 ? 32 : M <= 64 ? 64 : M <= 256 ? 128 : 256;
   p.pair = 0;
   int pair_stages = 3;
-  if (force_pair == 0 && force_bn == 0 && force_split <= 1 && N % (2 * TILE_W) == 0) {
+  const bool automatic = force_pair == 0 && force_bn == 0 && force_split == 0;
+  const long tiles64 = n_tiles * ((M + 63) / 64), tiles128 = n_tiles * ((M + 127) / 128);
+  const long tiles256 = n_tiles * ((M + 255) / 256);
+  if (automatic && M > 64 && M <= 128 && tiles64 <= sms) {
+    // 65..128 rows against few weight tiles (the product will be split): two 64-row tiles per weight tile put
+    // twice the CTAs on the weight stream (128 x 4096 x 4096: 14.9 against 17.8 us, 128 x 4096 x 3584: 10.0
+    // against 11.8 us; with many weight tiles the 128-row tile stays: every weight tile crosses the fabric once)
+    p.BN = 64;
+  } else if (automatic && M > 256 && M <= 1024 && 2L * sms / tiles128 >= 2) {
+    // so few 128-row tiles that they fill the SMs only when the k range is split: 320 x 4096 x 12288 43.8 against
+    // 66.4 us without a split, 384 x 3584 x 18944 53.8 against 96.0 us, 512 x 4096 x 3584 20.0 against 24.4 us
+    p.BN = 128;
+  } else if (force_pair == 0 && force_bn == 0 && force_split <= 1 && N % (2 * TILE_W) == 0) {
     // CTA pairs where they measured faster (B200): products that need no split between 129 and 1024 activation
     // rows, where the activation tile's trips through the L2 -> SM fabric bound the one-CTA kernel.
     if (M > 128 && M <= 256 && n_tiles >= sms) {   // (65..128 rows: one-CTA 128-row tiles measured 10 % faster)
       p.pair = 1;
       p.BN = 256;
-    } else if (M > 256 && M <= 1024 && n_tiles * ((M + 255) / 256) <= sms) {
-      // (with more 256-row tiles than SMs the persistent kernel below measured faster: gate / up at 512, 768 and
+    } else if (M > 256 && M <= 1024 && 4 * tiles128 <= 11L * sms) {
+      // pairs on 128-row tiles up to 2.75 tiles per SM: 768 x 8192 x 4096 44.4 us against 48.3 on 256-row pair
+      // tiles and 52.7 on the persistent kernel (192 tiles of 256 rows are 1.3 waves of its CTAs)
+      p.pair = 1;
+      p.BN = 128;
+      pair_stages = tiles128 <= 2L * sms ? 4 : 3;  // all 128-row pair tiles resident at once: a deeper ring
+    } else if (M > 256 && M <= 1024 && tiles256 <= 2L * sms) {
+      // (with more 256-row tiles than that the persistent kernel below measured faster: gate / up at 512, 768 and
       // 1024 rows 114 -> 91, 136 -> 127, 181 -> 162 us)
       p.pair = 1;
-      const bool one_wave = n_tiles * ((M + 127) / 128) <= 2L * sms;  // all 128-row pair tiles resident at once
-      p.BN = one_wave ? 128 : 256;
-      pair_stages = one_wave ? 4 : 3;
+      p.BN = 256;
     }
   }
   // 192-row tiles (persistent kernel only) where they leave at least 15 % fewer padded activation rows than
@@ -891,7 +907,9 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
   const long tiles = (long)p.m_tiles * n_tiles;
   // every split adds a slab the consumer has to read: with few activation rows
   // one wave of CTAs is enough, with 128-row tiles two CTAs per SM pay off
-  int S = p.BN == 128 ? (int)(2L * sms / tiles) : (int)((sms + tiles - 1) / tiles);  // all CTAs resident at once
+  // (two CTAs per SM also for 64-row tiles when there are two or more of them per weight tile)
+  const bool two_per_sm = p.BN == 128 || (p.BN == 64 && p.m_tiles > 1);
+  int S = two_per_sm ? (int)(2L * sms / tiles) : (int)((sms + tiles - 1) / tiles);  // all CTAs resident at once
   const int max_s = p.num_kb / 4 > 1 ? p.num_kb / 4 : 1;
   if (S > max_s) S = max_s;
   if (S < 1) S = 1;
