@@ -426,7 +426,7 @@ def main():
         b.record(stream)
         torch.cuda.synchronize(dev)
         return a.elapsed_time(b) / reps
-    reps = {"full": args.full_steps, "refresh": 6, "mixed": 6, "partial": 12}
+    reps = {"full": args.full_steps, "refresh": 16, "mixed": 6, "partial": 16}
     per_kind = {kind: time_kind(*KINDS[kind], reps[kind]) for kind in KINDS}
 
     def schedule_counts(n_steps):
