@@ -1103,12 +1103,15 @@ void launch_embed_norm(const Launch& L, int dtype, const void* E, const int32_t*
 // rounded to the cache dtype; x <- (x + AttnOut) + FFNOut from the caches
 // (Sec. 3.2 item (3)); u = rmsnorm(x) * gain, the next layer's first norm (the
 // final norm after the last layer).  inv == nullptr: no row is active.
-template <typename T>
+// With active rows (inv != nullptr) the launch before this one is the down projection, which writes nothing but
+// `part`; everything else a row needs (its place in the active list, x, AttnOut, a cached FFNOut row, the gain) was
+// written by launches that had completed before that projection passed its own dependency wait.  A one-pass row
+// therefore fetches all of it BEFORE the wait, while the projection still runs, and only the projection result
+// (active rows) after it.
+template <typename T, bool EARLY>
 __global__ void __launch_bounds__(512, 2) tail_kernel(Partials part, const int32_t* __restrict__ inv, float* __restrict__ x,
                             OutRows Ac, OutRows Fc, const float* __restrict__ gain,
                             T* __restrict__ u, Geo g, int c0, float eps) {
-  pdl_wait();
-  pdl_trigger();
   extern __shared__ float hrow[];
   __shared__ float red[32];
   const int c = c0 + blockIdx.x;
@@ -1117,10 +1120,48 @@ __global__ void __launch_bounds__(512, 2) tail_kernel(Partials part, const int32
   T* frow = Fc.row<T>(c, g);
   const bool one_trip = d <= (int)blockDim.x * 8;  // the row fits one pass: it stays in registers
   const int i0 = threadIdx.x * 8;
-  float hv[8], gv[8];
-  if (one_trip && i0 < d) Vec8<float>::load(gain + i0, gv);
-  const int r = inv ? inv[c] : -1;
   float* xr = x + (size_t)c * d;
+  float hv[8], gv[8];
+  int r = -1;
+  if constexpr (EARLY) {   // the host passes EARLY only with inv != nullptr and a one-pass row
+    float ae[8], fe[8];
+    r = __ldcg(inv + c);
+    if (i0 < d) {
+      Vec8<float>::load(gain + i0, gv);
+      Vec8<float>::load_cg(xr + i0, hv);
+      Vec8<T>::load_cg(arow + i0, ae);
+      if (r < 0) Vec8<T>::load_cg(frow + i0, fe);
+    }
+    pdl_wait();
+    pdl_trigger();
+    float ss = 0.f;
+    if (i0 < d) {
+      if (r >= 0) {
+        sum_partials8(part.p, part.split_stride, part.count(r, i0), (size_t)r * part.N + i0, fe);
+        Vec8<T>::store(frow + i0, fe);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) fe[t] = Vec8<T>::round(fe[t]);
+      }
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        hv[t] = (hv[t] + ae[t]) + fe[t];
+        ss += hv[t] * hv[t];
+      }
+      Vec8<float>::store(xr + i0, hv);
+    }
+    ss = block_sum(ss, red);
+    const float rs = rsqrtf(ss / (float)d + eps);
+    if (i0 < d) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) hv[t] = hv[t] * rs * gv[t];
+      Vec8<T>::store(u + (size_t)c * d + i0, hv);
+    }
+    return;
+  }
+  pdl_wait();
+  pdl_trigger();
+  if (one_trip && i0 < d) Vec8<float>::load(gain + i0, gv);
+  r = inv ? inv[c] : -1;
   float ss = 0.f;
   for (int i = i0; i < d; i += blockDim.x * 8) {
     float xv[8], a[8], f[8];
@@ -1188,8 +1229,12 @@ void launch_tail(const Launch& L, int dtype, Partials part, const int32_t* inv, 
   }
   const int threads = row_threads(g.d);
   const size_t smem = g.d <= threads * 8 ? 0 : (size_t)g.d * sizeof(float);  // staging only if a row takes several passes
-  DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T>, dim3(c1 - c0), dim3(threads), smem, part, inv, x, Ac_layer,
-                                 Fc_layer, gain, (T*)u, g, c0, eps)));
+  if (inv != nullptr && smem == 0)
+    DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T, true>, dim3(c1 - c0), dim3(threads), smem, part, inv, x, Ac_layer,
+                                   Fc_layer, gain, (T*)u, g, c0, eps)));
+  else
+    DLLM_DISPATCH(dtype, (launch_k(L, tail_kernel<T, false>, dim3(c1 - c0), dim3(threads), smem, part, inv, x, Ac_layer,
+                                   Fc_layer, gain, (T*)u, g, c0, eps)));
   L.count();
 }
 
