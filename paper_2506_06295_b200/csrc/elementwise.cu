@@ -581,20 +581,30 @@ __device__ __forceinline__ int32_t* select_sequence(unsigned long long* keys, co
 // metric 0: cosine (Eq. 6); 1: negated Euclidean distance (Sec. A.6), so that the
 // least similar rows have the lowest score either way.  write_v 0: the cache is
 // left as it is (the selected-only variant of Sec. A.5 writes the selected rows later).
+// The launch before this one is the V projection, which writes nothing but `part`: a row that fits one pass
+// fetches its cached V row before the dependency wait, while the projection still runs.
 template <typename T>
 __global__ void __launch_bounds__(512, 2) vverify_kernel(Partials part, T* __restrict__ Vc, float* __restrict__ sim,
                                                          Geo g, int dkv, int metric, int write_v, IdentityLists id) {
-  pdl_wait();
-  pdl_trigger();
   __shared__ float red[96];
   const int c = blockIdx.x;  // response row, carried order
   const int b = c / g.R, j = c - b * g.R;
   T* vrow = Vc + ((size_t)b * g.n + g.P + j) * dkv;
+  const bool one_trip = dkv <= (int)blockDim.x * 8;
+  float vo0[8];
+  if (one_trip && (int)threadIdx.x * 8 < dkv) Vec8<T>::load_cg(vrow + threadIdx.x * 8, vo0);
+  pdl_wait();
+  pdl_trigger();
   float dot = 0.f, na = 0.f, nb = 0.f;
   for (int i = threadIdx.x * 8; i < dkv; i += blockDim.x * 8) {
     float vn[8], vo[8];
     sum_partials8(part.p, part.split_stride, part.count(c, i), (size_t)c * part.N + i, vn);
-    Vec8<T>::load(vrow + i, vo);
+    if (one_trip) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) vo[t] = vo0[t];
+    } else {
+      Vec8<T>::load(vrow + i, vo);
+    }
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
       vn[t] = Vec8<T>::round(vn[t]);  // compare what the cache will hold
@@ -856,26 +866,29 @@ void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32
 template <typename T>
 __global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ rope_tab,
                                T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int Ma, int H, int Hkv, int hd) {
-  pdl_wait();
-  pdl_trigger();
+  // The launch before this one is the Q / K projection, which writes nothing but `part`: the row's position and
+  // its cos / sin values are fetched before the dependency wait, while the projection still runs.
   const int half = hd >> 1, q4 = half >> 2;
   const int groups = (H + Hkv) * q4;
   const long w = (long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (w >= (long)Ma * groups) return;
-  const int r = (int)(w / groups), gidx = (int)(w - (long)r * groups);
+  const bool live = w < (long)Ma * groups;
+  const int r = live ? (int)(w / groups) : 0, gidx = live ? (int)(w - (long)r * groups) : 0;
   const int head = gidx / q4, i0 = (gidx - head * q4) * 4;
   int b, pos;
-  carried_to_pos(act[r], g, b, pos);
+  carried_to_pos(__ldcg(act + r), g, b, pos);
   const int dq = H * hd, dkv = Hkv * hd;
   const bool is_q = head < H;
   const int col0 = is_q ? head * hd : dq + (head - H) * hd;
   T* dst = is_q ? qbuf + (size_t)r * dq + head * hd : Kc + ((size_t)b * g.n + pos) * dkv + (head - H) * hd;
   const float* tab = rope_tab + (size_t)pos * hd;  // [cos(half) | sin(half)]
+  const float4 cs = *reinterpret_cast<const float4*>(tab + i0);
+  const float4 sn = *reinterpret_cast<const float4*>(tab + half + i0);
+  pdl_wait();
+  pdl_trigger();
+  if (!live) return;
   float lo[4], hi[4];
   sum_partials4(part, r, col0 + i0, lo);
   sum_partials4(part, r, col0 + i0 + half, hi);
-  const float4 cs = *reinterpret_cast<const float4*>(tab + i0);
-  const float4 sn = *reinterpret_cast<const float4*>(tab + half + i0);
   const float cc[4] = {cs.x, cs.y, cs.z, cs.w}, ss[4] = {sn.x, sn.y, sn.z, sn.w};
   float o_lo[4], o_hi[4];
 #pragma unroll
@@ -950,24 +963,34 @@ template <typename T>
 __global__ void oproj_epilogue_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ x,
                                       const float* __restrict__ gain2, OutRows Ac, T* __restrict__ hn, Geo g,
                                       float eps) {
-  pdl_wait();
-  pdl_trigger();
+  // The launch before this one is the O projection, which writes nothing but `part`: the row's place (act), its x
+  // row and the gain are fetched before the dependency wait, while the projection still runs.
   extern __shared__ float hrow[];
   __shared__ float red[32];
   const int r = blockIdx.x;
   const int d = g.d;
   const bool one_trip = d <= (int)blockDim.x * 8;  // the row fits one pass: it stays in registers
   const int i0 = threadIdx.x * 8;
-  float hv[8], gv[8];
-  if (one_trip && i0 < d) Vec8<float>::load(gain2 + i0, gv);  // independent of the row: ahead of the dependent loads
-  const int c = act[r];
+  float hv[8], gv[8], x0[8];
+  const int c = __ldcg(act + r);
   T* arow = Ac.row<T>(c, g);
   const float* xr = x + (size_t)c * d;
+  if (one_trip && i0 < d) {
+    Vec8<float>::load(gain2 + i0, gv);
+    Vec8<float>::load_cg(xr + i0, x0);
+  }
+  pdl_wait();
+  pdl_trigger();
   float ss = 0.f;
   for (int i = i0; i < d; i += blockDim.x * 8) {
     float a[8], xv[8];
     sum_partials8(part.p, part.split_stride, part.count(r, i), (size_t)r * part.N + i, a);
-    Vec8<float>::load(xr + i, xv);
+    if (one_trip) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) xv[t] = x0[t];
+    } else {
+      Vec8<float>::load(xr + i, xv);
+    }
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
       a[t] = Vec8<T>::round(a[t]);
