@@ -301,3 +301,18 @@ def test_batched_two_layers_against_the_oracle(env):
                            [(False, False, 0.1, "floor"), (False, False, 0.25, "floor"), (False, True, 0.0, "floor"),
                             (False, False, 0.5, "floor")])
     assert ses.selected(0)[0].shape == (B, 256)
+
+
+def test_dream_width_batched_two_layers_against_the_oracle(env):
+    """Dream-7B widths with B = 4 sequences of P = 64, R = 256: 1024 response rows, from which the row-wise kernels
+    take their streaming forms (V-verify on 512-wide V rows, RoPE over 28 + 4 heads, the O epilogue and the layer
+    tail on 3584-wide rows: other ring depths than at the LLaDA widths), grouped heads on the tcgen05 attention;
+    full, partial, refresh and mixed steps, every cache and the hidden states compared per layer."""
+    torch, dllm = env
+    wl = synth.WORKLOADS["dream7b"]
+    cfg = wl.model.with_layers(2)
+    B = 4
+    orc, ses = _run_config(dllm, cfg, B, 64, wl.gen_len,
+                           [(False, False, 0.5, "floor"), (False, True, 0.0, "floor"), (False, False, 0.25, "floor"),
+                            (True, False, 0.25, "floor")])
+    assert ses.selected(0)[0].shape == (B, 64)
