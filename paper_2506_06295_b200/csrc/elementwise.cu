@@ -861,43 +861,55 @@ void launch_gather_rows(const Launch& L, int dtype, const void* src, const int32
 }
 
 // ------------------------------------------------------------------ RoPE + K scatter
-// One thread per (active row, head, four rotation pairs).  Rotate-half pairing:
-// element i with i + hd/2, angle pos * theta^(-2i/hd) from a table built on the host.
-template <typename T>
+// One thread per (active row, HP consecutive heads, four rotation pairs).  Rotate-half pairing:
+// element i with i + hd/2, angle pos * theta^(-2i/hd) from a table built on the host.  HP = 2 (the heads of a
+// thread share the row's position and rotation values) halves the CTAs when there are several per SM slot, so
+// that all of them are resident, and have fetched those values, before the projection ahead of them ends.
+template <typename T, int HP>
 __global__ void qk_rope_kernel(Partials part, const int32_t* __restrict__ act, const float* __restrict__ rope_tab,
                                T* __restrict__ qbuf, T* __restrict__ Kc, Geo g, int Ma, int H, int Hkv, int hd) {
   // The launch before this one is the Q / K projection, which writes nothing but `part`: the row's position and
   // its cos / sin values are fetched before the dependency wait, while the projection still runs.
   const int half = hd >> 1, q4 = half >> 2;
-  const int groups = (H + Hkv) * q4;
+  const int heads = H + Hkv, hgroups = (heads + HP - 1) / HP;
+  const int groups = hgroups * q4;
   const long w = (long)blockIdx.x * blockDim.x + threadIdx.x;
   const bool live = w < (long)Ma * groups;
   const int r = live ? (int)(w / groups) : 0, gidx = live ? (int)(w - (long)r * groups) : 0;
-  const int head = gidx / q4, i0 = (gidx - head * q4) * 4;
+  const int hg = gidx / q4, i0 = (gidx - hg * q4) * 4;
   int b, pos;
   carried_to_pos(__ldcg(act + r), g, b, pos);
   const int dq = H * hd, dkv = Hkv * hd;
-  const bool is_q = head < H;
-  const int col0 = is_q ? head * hd : dq + (head - H) * hd;
-  T* dst = is_q ? qbuf + (size_t)r * dq + head * hd : Kc + ((size_t)b * g.n + pos) * dkv + (head - H) * hd;
   const float* tab = rope_tab + (size_t)pos * hd;  // [cos(half) | sin(half)]
   const float4 cs = *reinterpret_cast<const float4*>(tab + i0);
   const float4 sn = *reinterpret_cast<const float4*>(tab + half + i0);
   pdl_wait();
   pdl_trigger();
   if (!live) return;
-  float lo[4], hi[4];
-  sum_partials4(part, r, col0 + i0, lo);
-  sum_partials4(part, r, col0 + i0 + half, hi);
   const float cc[4] = {cs.x, cs.y, cs.z, cs.w}, ss[4] = {sn.x, sn.y, sn.z, sn.w};
-  float o_lo[4], o_hi[4];
+  float lo[HP][4], hi[HP][4];
 #pragma unroll
-  for (int t = 0; t < 4; ++t) {
-    o_lo[t] = lo[t] * cc[t] - hi[t] * ss[t];
-    o_hi[t] = hi[t] * cc[t] + lo[t] * ss[t];
+  for (int u = 0; u < HP; ++u) {
+    const int head = hg * HP + u;
+    if (head >= heads) break;
+    const int col0 = head < H ? head * hd : dq + (head - H) * hd;
+    sum_partials4(part, r, col0 + i0, lo[u]);
+    sum_partials4(part, r, col0 + i0 + half, hi[u]);
   }
-  store4<T>(dst + i0, o_lo);
-  store4<T>(dst + i0 + half, o_hi);
+#pragma unroll
+  for (int u = 0; u < HP; ++u) {
+    const int head = hg * HP + u;
+    if (head >= heads) break;
+    T* dst = head < H ? qbuf + (size_t)r * dq + head * hd : Kc + ((size_t)b * g.n + pos) * dkv + (head - H) * hd;
+    float o_lo[4], o_hi[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      o_lo[t] = lo[u][t] * cc[t] - hi[u][t] * ss[t];
+      o_hi[t] = hi[u][t] * cc[t] + lo[u][t] * ss[t];
+    }
+    store4<T>(dst + i0, o_lo);
+    store4<T>(dst + i0 + half, o_hi);
+  }
 }
 
 void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* act, const float* rope_tab, void* qbuf,
@@ -923,9 +935,15 @@ void launch_qk_rope(const Launch& L, int dtype, Partials part, const int32_t* ac
     return;
   }
   const long total = (long)Ma * (H + Hkv) * (hd >> 3);
-  const unsigned blocks = (unsigned)((total + 255) / 256);
-  DLLM_DISPATCH(dtype, (launch_k(L, qk_rope_kernel<T>, dim3(blocks), dim3(256), 0, part, act, rope_tab, (T*)qbuf,
-                                 (T*)Kc_layer, g, Ma, H, Hkv, hd)));
+  const long blocks1 = (total + 255) / 256;
+  if (blocks1 > 2L * sm_count()) {   // two heads per thread: half the CTAs
+    const long total2 = (long)Ma * ((H + Hkv + 1) / 2) * (hd >> 3);
+    DLLM_DISPATCH(dtype, (launch_k(L, qk_rope_kernel<T, 2>, dim3((unsigned)((total2 + 255) / 256)), dim3(256), 0, part, act,
+                                   rope_tab, (T*)qbuf, (T*)Kc_layer, g, Ma, H, Hkv, hd)));
+  } else {
+    DLLM_DISPATCH(dtype, (launch_k(L, qk_rope_kernel<T, 1>, dim3((unsigned)blocks1), dim3(256), 0, part, act, rope_tab,
+                                   (T*)qbuf, (T*)Kc_layer, g, Ma, H, Hkv, hd)));
+  }
   L.count();
 }
 
