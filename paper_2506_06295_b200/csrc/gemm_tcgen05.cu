@@ -870,6 +870,13 @@ GemmPlan plan_gemm_bf16(int M, int N, int K, int force_split, int force_stages, 
     // twice the CTAs on the weight stream (128 x 4096 x 4096: 14.9 against 17.8 us, 128 x 4096 x 3584: 10.0
     // against 11.8 us; with many weight tiles the 128-row tile stays: every weight tile crosses the fabric once)
     p.BN = 64;
+  } else if (automatic && M > 128 && M <= 256 && tiles64 <= sms && (K + TILE_K - 1) / TILE_K <= 64) {
+    // 129..256 rows against few weight tiles and a short k range (256 x 4096 x 4096, the V projection of every
+    // cached step): four 64-row tiles per weight tile with two splits take as long as two 128-row tiles with four
+    // (15.3 against 15.6 us) and leave the consumer half the slabs to sum (19.4 against 20.9 us with the
+    // reduction); with a long k range the doubled weight traffic through the L2 -> SM fabric costs more (256 x
+    // 4096 x 12288: 36.8 against 32.6 us)
+    p.BN = 64;
   } else if (automatic && M > 256 && M <= 1024 && 2L * sms / tiles128 >= 2) {
     // so few 128-row tiles that they fill the SMs only when the k range is split: 320 x 4096 x 12288 43.8 against
     // 66.4 us without a split, 384 x 3584 x 18944 53.8 against 96.0 us, 512 x 4096 x 3584 20.0 against 24.4 us
