@@ -280,7 +280,7 @@ def step_roof_ms(per_class, peaks):
 # dram__bytes_read.sum + dram__bytes_write.sum per projection launch, from an ncu capture of a two-layer case of
 # the same kernel scaled to the full depth (every layer streams its own weights); None where no capture of the
 # current kernel exists.
-TRAFFIC_PER_LAUNCH = {"llada8b": 96.3e6}
+TRAFFIC_PER_LAUNCH = {"llada8b": 96.2e6}
 
 
 # ----------------------------------------------------------------------------------------------

@@ -1082,7 +1082,7 @@ __global__ void silu_mul_kernel(Partials part, T* __restrict__ out, int Ma, int 
     sum_partials8(part.p, part.split_stride, part.count(r, cg), (size_t)r * part.N + cg, gt);
     sum_partials8(part.p, part.split_stride, part.count(r, cu), (size_t)r * part.N + cu, up);
 #pragma unroll
-    for (int t = 0; t < 8; ++t) gt[t] = gt[t] / (1.f + expf(-gt[t])) * up[t];
+    for (int t = 0; t < 8; ++t) gt[t] = __fdividef(gt[t], 1.f + __expf(-gt[t])) * up[t];  // as in the GEMM epilogue
     Vec8<T>::store(out + (size_t)r * m + j, gt);
   }
 }

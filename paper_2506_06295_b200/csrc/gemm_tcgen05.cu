@@ -179,8 +179,12 @@ __device__ __forceinline__ void gemm_epilogue(uint32_t tmem_d, float* ex, int tl
         const float4 gt = *reinterpret_cast<const float4*>(ex + rr * EXS + 4 * q);
         const float4 up = *reinterpret_cast<const float4*>(ex + rr * EXS + 64 + 4 * q);
         if (m < M && col < m_ffn) {
-          const __nv_bfloat162 lo = __floats2bfloat162_rn(gt.x / (1.f + expf(-gt.x)) * up.x, gt.y / (1.f + expf(-gt.y)) * up.y);
-          const __nv_bfloat162 hi = __floats2bfloat162_rn(gt.z / (1.f + expf(-gt.z)) * up.z, gt.w / (1.f + expf(-gt.w)) * up.w);
+          // silu(g) * u with the fast exponential and division (relative error ~1e-6, far below the bf16 rounding
+          // of the result)
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(__fdividef(gt.x, 1.f + __expf(-gt.x)) * up.x,
+                                                          __fdividef(gt.y, 1.f + __expf(-gt.y)) * up.y);
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(__fdividef(gt.z, 1.f + __expf(-gt.z)) * up.z,
+                                                          __fdividef(gt.w, 1.f + __expf(-gt.w)) * up.w);
           uint2 pk;
           pk.x = *reinterpret_cast<const uint32_t*>(&lo);
           pk.y = *reinterpret_cast<const uint32_t*>(&hi);
