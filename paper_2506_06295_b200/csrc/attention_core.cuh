@@ -56,6 +56,51 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
 }
+// 2^x on the special-function unit (ex2.approx: relative error about 2^-22, far below the bf16 rounding of P;
+// 2^-inf = 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Online-softmax update of one warp's 16 x 64 score fragment (rows lane / 4 and lane / 4 + 8; raw scores in,
+// probabilities out): new running maxima m (in log2 units of the scaled scores), the factors `corr` by which the
+// sums and outputs so far shrink, and the row sums l advanced by this tile's (per-lane partial) sums.  The scale
+// is folded into the exponent's multiply-add; keys at or past key_hi count for nothing (only a sequence's last
+// tile has any: a warp-uniform test).  key_base: the first of this lane's keys.
+__device__ __forceinline__ void softmax_tile(float (&sacc)[8][4], int key_base, int key_hi, int lane, float scale_log2,
+                                             float (&m)[2], float (&l)[2], float (&corr)[2]) {
+  if (key_base - 2 * (lane & 3) + 64 > key_hi) {
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        if (key_base + nb * 8 + (c & 1) >= key_hi) sacc[nb][c] = -INFINITY;
+  }
+  float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+  for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) mx[c >> 1] = fmaxf(mx[c >> 1], sacc[nb][c]);
+#pragma unroll
+  for (int h2 = 0; h2 < 2; ++h2) {
+    mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 1));
+    mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 2));
+    const float m_new = fmaxf(m[h2], mx[h2] * scale_log2);  // finite: every tile has a valid key; scale_log2 > 0
+    corr[h2] = fast_exp2(m[h2] - m_new);                      // first tile: 2^-inf = 0
+    m[h2] = m_new;
+    l[h2] *= corr[h2];
+  }
+#pragma unroll
+  for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float p = fast_exp2(fmaf(sacc[nb][c], scale_log2, -m[c >> 1]));
+      sacc[nb][c] = p;
+      l[c >> 1] += p;
+    }
+}
+
 // Byte offset of the 16-byte chunk `dc` (8 bf16) of row `row` in a tile stored
 // as panels of 64 columns: panel = [rows][128 bytes], chunk index XOR (row % 8).
 template <int ROWS>
@@ -193,37 +238,8 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
       }
     }
     // ---- online softmax (rows lane/4 and lane/4 + 8)
-    const int key_base = key_lo + t * AT_KEYS + 2 * (lane & 3);
-    float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-    for (int nb = 0; nb < AT_KEYS / 8; ++nb) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int key = key_base + nb * 8 + (c & 1);
-        const float v = (key < key_hi) ? sacc[nb][c] * scale_log2 : -INFINITY;
-        sacc[nb][c] = v;
-        mx[c >> 1] = fmaxf(mx[c >> 1], v);
-      }
-    }
     float corr[2];
-#pragma unroll
-    for (int h2 = 0; h2 < 2; ++h2) {
-      mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 1));
-      mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 2));
-      const float m_new = fmaxf(m_run[h2], mx[h2]);      // finite: every tile has a valid key
-      corr[h2] = exp2f(m_run[h2] - m_new);
-      m_run[h2] = m_new;
-      l_run[h2] *= corr[h2];
-    }
-#pragma unroll
-    for (int nb = 0; nb < AT_KEYS / 8; ++nb) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const float p = exp2f(sacc[nb][c] - m_run[c >> 1]);
-        sacc[nb][c] = p;
-        l_run[c >> 1] += p;
-      }
-    }
+    softmax_tile(sacc, key_lo + t * AT_KEYS + 2 * (lane & 3), key_hi, lane, scale_log2, m_run, l_run, corr);
 #pragma unroll
     for (int i = 0; i < HD / 8; ++i) {
       oacc[i][0] *= corr[0];
@@ -336,37 +352,8 @@ __device__ __forceinline__ void attn_warp_tile(int lane, int rg, uint32_t q_s, u
     }
   }
   // ---- online softmax (rows lane/4 and lane/4 + 8)
-  const int key_base = key0 + 2 * (lane & 3);
-  float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-  for (int nb = 0; nb < AT_KEYS / 8; ++nb) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const int key = key_base + nb * 8 + (c & 1);
-      const float v = (key < key_hi) ? sacc[nb][c] * scale_log2 : -INFINITY;
-      sacc[nb][c] = v;
-      mx[c >> 1] = fmaxf(mx[c >> 1], v);
-    }
-  }
   float corr[2];
-#pragma unroll
-  for (int h2 = 0; h2 < 2; ++h2) {
-    mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 1));
-    mx[h2] = fmaxf(mx[h2], __shfl_xor_sync(0xffffffffu, mx[h2], 2));
-    const float m_new = fmaxf(acc.m[h2], mx[h2]);      // finite: every tile has a valid key
-    corr[h2] = exp2f(acc.m[h2] - m_new);                 // first tile: exp2(-inf) = 0
-    acc.m[h2] = m_new;
-    acc.l[h2] *= corr[h2];
-  }
-#pragma unroll
-  for (int nb = 0; nb < AT_KEYS / 8; ++nb) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const float p = exp2f(sacc[nb][c] - acc.m[c >> 1]);
-      sacc[nb][c] = p;
-      acc.l[c >> 1] += p;
-    }
-  }
+  softmax_tile(sacc, key0 + 2 * (lane & 3), key_hi, lane, scale_log2, acc.m, acc.l, corr);
 #pragma unroll
   for (int i = 0; i < HD / 8; ++i) {
     acc.o[i][0] *= corr[0];
