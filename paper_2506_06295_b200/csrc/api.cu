@@ -533,7 +533,11 @@ dllm_status enqueue_step(dllm_session* s, int rp, int rr, const std::vector<int>
                     (2.0 * s->B * s->n * dkv + 2.0 * Ma * dq) * (double)es, 4.0 * Ma * (double)s->n * dq, stream);
       cudaError_t e = launch_attention(L, dt, s->wsp<uint8_t>(s->ws.qbuf), s->cache(l, DLLM_CACHE_K),
                                        s->cache(l, DLLM_CACHE_V), s->wsp<uint8_t>(s->ws.obuf), s->B, a_seq, s->n, H,
-                                       Hkv, hd, s->wsp<float>(s->ws.attn), s->ws.attn_floats, s->simt_gemm);
+                                       Hkv, hd, s->wsp<float>(s->ws.attn), s->ws.attn_floats, s->simt_gemm,
+                                       // the launch before attention is RoPE + K scatter (after the Q / K projection):
+                                       // every V row of the layer and, unless the prompt is refreshed, the prompt's K
+                                       // rows were written at least two launches earlier
+                                       rp ? 0 : s->P, s->n);
       s->prof_end(stream);
       if (e != cudaSuccess) return fail(&s->err, DLLM_CUDA_ERROR, "attention: %s", cudaGetErrorString(e));
       if ((st = run_gemm(s, L, DLLM_PROF_GEMM_O, s->wsp<uint8_t>(s->ws.obuf), W + lo.wo, Ma, d, dq, &part)) != DLLM_OK)

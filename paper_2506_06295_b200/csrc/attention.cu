@@ -126,8 +126,8 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ C
                                                        const __nv_bfloat16* __restrict__ q,
                                                        __nv_bfloat16* __restrict__ o, float* __restrict__ o_part,
                                                        float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv,
-                                                       int S, int keys_per_split, float scale_log2,
-                                                       int* __restrict__ status) {
+                                                       int S, int keys_per_split, float scale_log2, int k_static,
+                                                       int v_static, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[2];
   __shared__ int abort_flag;
@@ -142,13 +142,11 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const __grid_constant__ C
     if (q_by_tma) prefetch_tensormap(&tmQ);
   }
   __syncthreads();
-  pdl_wait();  // K, V and Q come from the preceding kernels
-  pdl_trigger();
-  uint32_t kv_iter = 0;
+  uint32_t kv_iter = 0;   // (attn_tile waits for the launch before this one and releases the dependents)
   const bool ok = attn_tile<HD>((int)threadIdx.x, smem_raw + (base - smem_u32(smem_raw)), base, full_bar, kv_iter,
                                 &abort_flag, &tmK, &tmV, q, o, o_part, ml_part, a_seq, n, H, Hkv, S, keys_per_split,
                                 scale_log2, (int)gridDim.z / S, (int)blockIdx.x, (int)blockIdx.y, (int)blockIdx.z,
-                                q_by_tma ? &tmQ : nullptr);
+                                q_by_tma ? &tmQ : nullptr, k_static, v_static);
   if (!ok && threadIdx.x == 0 && status) atomicCAS(status, ST_OK, ST_TIMEOUT_ATTN);
 }
 
@@ -426,7 +424,8 @@ cudaError_t launch_combine(const Launch& L, const float* o_part, const float* ml
 
 template <int HD>
 cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
-                       float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
+                       float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split, int k_static,
+                       int v_static) {
   constexpr int SMEM = AT_ROWS * HD * 2 + 2 * 2 * AT_KEYS * HD * 2 + 1024;
   static DeviceOnce once;
   cudaError_t e0 = once.run(
@@ -444,7 +443,7 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
                        get_tensor_map_2d(q, (uint64_t)B * a_seq, (uint64_t)H * HD, AT_ROWS, &tmQ);
   cudaError_t e = launch_k(L, attn_mma_kernel<HD>, dim3(grid), dim3(128), SMEM, tmK, tmV, tmQ, q_by_tma,
                            (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S,
-                           keys_per_split, scale_log2, L.d_status);
+                           keys_per_split, scale_log2, k_static, v_static, L.d_status);
   L.count();
   if (e == cudaSuccess && S > 1) e = launch_combine(L, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
   return e != cudaSuccess ? e : cudaGetLastError();
@@ -555,7 +554,7 @@ AttnChoice choose_attention(int B, int a_seq, int n, int H, int Hkv, size_t scra
 
 cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const void* Kc, const void* Vc, void* o, int B,
                              int a_seq, int n, int H, int Hkv, int hd, float* scratch, size_t scratch_floats,
-                             bool force_simt) {
+                             bool force_simt, int k_static, int v_static) {
   if (B <= 0 || a_seq <= 0) return cudaSuccess;
   if (hd > HD_MAX || (hd & 31) || H % Hkv) return cudaErrorInvalidValue;
   const bool tensor = dtype == 1 && !force_simt && (hd == 64 || hd == 128) && ((Hkv * hd) % 8 == 0);
@@ -583,8 +582,8 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
     if (p.few_rg == 2)
       return hd == 64 ? launch_few<64, 2, 3>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
                       : launch_few<128, 2, 3>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
-    return hd == 64 ? launch_mma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
-                    : launch_mma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
+    return hd == 64 ? launch_mma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split, k_static, v_static)
+                    : launch_mma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split, k_static, v_static);
   }
   const float scale = 1.0f / sqrtf((float)hd);
   dim3 grid((a_seq + TQ - 1) / TQ, H, B);

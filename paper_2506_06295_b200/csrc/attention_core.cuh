@@ -119,6 +119,10 @@ struct AttnSmem {
 // (stage and phase parity continue across calls); advanced by the tiles of this
 // call.  (bx, by, bz) play the role of the block index of a grid
 // (row tiles, KV heads, B * S).  Returns false if a wait gave up.
+// The function itself waits for the launch before this one (griddepcontrol.wait) and releases the dependents.
+// k_static / v_static: the first so many keys of every sequence hold K / V rows that no launch since the one
+// BEFORE the previous launch has written (0: none); tiles made of such rows only are requested ahead of the wait,
+// while the previous launch (which writes Q and the newest K rows) still runs.
 template <int HD>
 __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t smem_sh, uint64_t* full_bar,
                                           uint32_t& kv_iter, volatile int* abort_flag, const CUtensorMap* tmK,
@@ -126,7 +130,7 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
                                           __nv_bfloat16* __restrict__ o, float* __restrict__ o_part,
                                           float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv, int S,
                                           int keys_per_split, float scale_log2, int B, int bx, int by, int bz,
-                                          const CUtensorMap* tmQ = nullptr) {
+                                          const CUtensorMap* tmQ, int k_static, int v_static) {
 
   constexpr int PANELS = HD / 64;
   constexpr uint32_t TILE_BYTES = AT_KEYS * HD * 2;   // one K or V tile
@@ -153,11 +157,13 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
   // tmQ (one query head per KV head, so a row tile is AT_ROWS consecutive rows of q): the Q tile arrives by TMA
   // together with the first K/V tile, on that tile's barrier; rows past the sequence's end belong to no live row
   const bool q_tma = tmQ != nullptr;
-  auto issue = [&](int t) {
+  // what: 1 = the K tile, 2 = the V tile, 4 = arm the stage's barrier with everything that will arrive on it
+  // (K, V and, for the first tile, the Q tile by TMA), 8 = the Q tile
+  auto issue = [&](int t, int what) {
     const int st = (int)((it0 + (uint32_t)t) & 1u);
     const uint32_t fb = smem_u32(&full_bar[st]);
-    mbar_expect_tx(fb, STAGE_BYTES + ((q_tma && t == 0) ? AT_ROWS * HD * 2 : 0));
-    if (q_tma && t == 0) {
+    if (what & 4) mbar_expect_tx(fb, STAGE_BYTES + ((q_tma && t == 0) ? AT_ROWS * HD * 2 : 0));
+    if ((what & 8) && q_tma && t == 0) {
 #pragma unroll
       for (int p = 0; p < PANELS; ++p) tma_load_2d(q_s + p * (AT_ROWS * 128), tmQ, fb, kh * HD + p * 64, b * a_seq + row0);
     }
@@ -165,13 +171,22 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
     const int key0 = key_lo + t * AT_KEYS;
 #pragma unroll
     for (int p = 0; p < PANELS; ++p) {
-      tma_load_3d(dst + p * (AT_KEYS * 128), tmK, fb, kh * HD + p * 64, key0, b);
-      tma_load_3d(dst + TILE_BYTES + p * (AT_KEYS * 128), tmV, fb, kh * HD + p * 64, key0, b);
+      if (what & 1) tma_load_3d(dst + p * (AT_KEYS * 128), tmK, fb, kh * HD + p * 64, key0, b);
+      if (what & 2) tma_load_3d(dst + TILE_BYTES + p * (AT_KEYS * 128), tmV, fb, kh * HD + p * 64, key0, b);
     }
   };
+  int early[2] = {0, 0};  // what of the first two tiles was requested ahead of the dependency wait
   if (tid == 0) {
-    issue(0);
-    if (n_tiles > 1) issue(1);
+    for (int t = 0; t < 2 && t < n_tiles; ++t) {
+      const int hi = min(key_lo + (t + 1) * AT_KEYS, n);  // one past the tile's last existing key
+      early[t] = (hi <= k_static ? 1 : 0) | (hi <= v_static ? 2 : 0);
+      if (early[t]) issue(t, early[t] | 4);
+    }
+  }
+  pdl_wait();  // Q and the newest K rows come from the launch before this one
+  pdl_trigger();
+  if (tid == 0) {
+    for (int t = 0; t < 2 && t < n_tiles; ++t) issue(t, (3 & ~early[t]) | (early[t] ? 0 : 4) | 8);
   }
   // Q tile: plain 16-byte loads into the swizzled layout (rows of other heads /
   // past the end are zero)
@@ -266,7 +281,7 @@ __device__ __forceinline__ bool attn_tile(int tid, uint8_t* smem_gen, uint32_t s
       }
     }
     at_sync();                               // every warp is done with stage st
-    if (tid == 0 && t + 2 < n_tiles) issue(t + 2);
+    if (tid == 0 && t + 2 < n_tiles) issue(t + 2, 1 | 2 | 4);
   }
   if (!ok) {
     drain_delay();

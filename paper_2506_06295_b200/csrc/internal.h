@@ -240,10 +240,12 @@ extern int g_attn_few_rows;       // 0: never the few-rows kernel
 extern int g_attn_umma_row_tiles; // tcgen05 kernel: 0 = the plan chooses one or two 128-row tiles per CTA, 1 / 2 forced
 // bf16 with head_dim 64 / 128 runs on the tensor cores (scratch holds the
 // partials of split key ranges; without it one split is used); everything else
-// on the plain-ALU kernel.
+// on the plain-ALU kernel.  k_static / v_static: the first so many keys of every sequence hold K / V rows that
+// no launch since the one BEFORE the launch preceding this attention has written (0 when unknown): the 64-row
+// kernel requests tiles made of such rows ahead of its dependency wait.
 cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const void* Kc, const void* Vc, void* o, int B,
                              int a_seq, int n, int H, int Hkv, int hd, float* scratch, size_t scratch_floats,
-                             bool force_simt);
+                             bool force_simt, int k_static = 0, int v_static = 0);
 
 // The same attention with 128-row tiles on tcgen05 (attention_umma.cu), for
 // many active rows per KV head.  *S_out: key-range splits used (> 1: the caller

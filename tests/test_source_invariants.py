@@ -23,7 +23,7 @@ def test_every_kernel_releases_its_dependents_only_after_its_own_dependency_wait
     launches earlier.  That is only sound while every kernel calls griddepcontrol.launch_dependents after its own
     griddepcontrol.wait: then a launch can become resident only once the launch before it has passed its wait, i.e.
     once everything older has completed."""
-    files = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
+    files = sorted(glob.glob(os.path.join(CSRC, "*.cu")) + glob.glob(os.path.join(CSRC, "*.cuh")))
     assert files
     triggers = 0
     for f in files:
