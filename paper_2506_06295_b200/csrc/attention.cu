@@ -163,7 +163,8 @@ __global__ void __launch_bounds__(32 * RG * KW, RG == 2 ? 2 : 1)
     attn_mma_few_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                         const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ o,
                         float* __restrict__ o_part, float* __restrict__ ml_part, int a_seq, int n, int H, int Hkv,
-                        int S, int keys_per_split, float scale_log2, int* __restrict__ status) {
+                        int S, int keys_per_split, float scale_log2, int k_static, int v_static,
+                        int* __restrict__ status) {
   constexpr uint32_t Q_BYTES = AT_ROWS * HD * 2;          // the tile layout of the 64-row kernel; RG * 16 rows used
   constexpr uint32_t TILE_BYTES = AT_KEYS * HD * 2, STAGE_BYTES = 2 * TILE_BYTES;
   constexpr int ROWS = 16 * RG, NT = 32 * RG * KW, PANELS = HD / 64;
@@ -183,8 +184,6 @@ __global__ void __launch_bounds__(32 * RG * KW, RG == 2 ? 2 : 1)
     prefetch_tensormap(&tmV);
   }
   __syncthreads();
-  pdl_wait();  // K, V and Q come from the preceding kernels
-  pdl_trigger();
 
   const int G = H / Hkv, kh = blockIdx.y;
   const int b = blockIdx.z / S, split = blockIdx.z - b * S;
@@ -194,17 +193,29 @@ __global__ void __launch_bounds__(32 * RG * KW, RG == 2 ? 2 : 1)
   const uint32_t q_s = base, kv_s = base + Q_BYTES + (uint32_t)kw * STAGE_BYTES;
   volatile int* abortp = &abort_flag;
 
-  auto issue = [&](int t) {  // key tile t of the split into this way's buffer
+  // key tile t of the split into this way's buffer; what: 1 = the K tile, 2 = the V tile, 4 = arm the barrier
+  auto issue = [&](int t, int what) {
     const uint32_t fb = smem_u32(&full_bar[kw]);
-    mbar_expect_tx(fb, STAGE_BYTES);
+    if (what & 4) mbar_expect_tx(fb, STAGE_BYTES);
     const int key0 = key_lo + t * AT_KEYS;
 #pragma unroll
     for (int p = 0; p < PANELS; ++p) {
-      tma_load_3d(kv_s + p * (AT_KEYS * 128), &tmK, fb, kh * HD + p * 64, key0, b);
-      tma_load_3d(kv_s + TILE_BYTES + p * (AT_KEYS * 128), &tmV, fb, kh * HD + p * 64, key0, b);
+      if (what & 1) tma_load_3d(kv_s + p * (AT_KEYS * 128), &tmK, fb, kh * HD + p * 64, key0, b);
+      if (what & 2) tma_load_3d(kv_s + TILE_BYTES + p * (AT_KEYS * 128), &tmV, fb, kh * HD + p * 64, key0, b);
     }
   };
-  if (rg == 0 && lane == 0 && kw < n_tiles) issue(kw);
+  // The way's first tile: what only holds rows older than the launch before this one (see launch_attention) is
+  // requested ahead of the dependency wait, the rest after it.
+  const bool issuer = rg == 0 && lane == 0 && kw < n_tiles;
+  int early = 0;
+  if (issuer) {
+    const int hi = min(key_lo + (kw + 1) * AT_KEYS, n);
+    early = (hi <= k_static ? 1 : 0) | (hi <= v_static ? 2 : 0);
+    if (early) issue(kw, early | 4);
+  }
+  pdl_wait();  // Q and the newest K rows come from the launch before this one
+  pdl_trigger();
+  if (issuer && early != 3) issue(kw, (3 & ~early) | (early ? 0 : 4));
   // Q rows of the tile: 16-byte loads into the swizzled layout (rows past the end are zero)
   {
     constexpr int CHUNKS = ROWS * (HD / 8);
@@ -245,7 +256,7 @@ __global__ void __launch_bounds__(32 * RG * KW, RG == 2 ? 2 : 1)
         asm volatile("bar.sync %0, %1;" ::"r"(1 + kw), "n"(32 * RG) : "memory");
       else
         __syncwarp();
-      if (rg == 0 && lane == 0) issue(t + KW);
+      if (rg == 0 && lane == 0) issue(t + KW, 1 | 2 | 4);
     }
   }
   attn_warp_finish(acc);
@@ -455,7 +466,8 @@ cudaError_t launch_mma(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
 namespace {
 template <int HD, int RG, int KW>
 cudaError_t launch_few(const Launch& L, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q, void* o,
-                       float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split) {
+                       float* scratch, int B, int a_seq, int n, int H, int Hkv, int S, int keys_per_split, int k_static,
+                       int v_static) {
   constexpr int SMEM = AT_ROWS * HD * 2 + KW * 2 * AT_KEYS * HD * 2 + 1024;
   static_assert(SMEM <= 227 * 1024, "the ways' buffers do not fit the shared memory of a CTA");
   static_assert(RG * 32 * (HD / 2) * 4 <= 2 * AT_KEYS * HD * 2, "a way's buffer must hold its warps' outputs");
@@ -472,7 +484,7 @@ cudaError_t launch_few(const Launch& L, const CUtensorMap& tmK, const CUtensorMa
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   cudaError_t e = launch_k(L, attn_mma_few_kernel<HD, RG, KW>, grid, dim3(32 * RG * KW), SMEM, tmK, tmV,
                            (const __nv_bfloat16*)q, (__nv_bfloat16*)o, o_part, ml_part, a_seq, n, H, Hkv, S,
-                           keys_per_split, scale_log2, L.d_status);
+                           keys_per_split, scale_log2, k_static, v_static, L.d_status);
   L.count();
   if (e == cudaSuccess && S > 1) e = launch_combine(L, o_part, ml_part, (__nv_bfloat16*)o, total, S, HD);
   return e != cudaSuccess ? e : cudaGetLastError();
@@ -576,14 +588,15 @@ cudaError_t launch_attention(const Launch& L, int dtype, const void* q, const vo
     if (!get_tensor_map_3d(Kc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, AT_KEYS, &tmK) ||
         !get_tensor_map_3d(Vc, (uint64_t)B, (uint64_t)n, (uint64_t)Hkv * hd, AT_KEYS, &tmV))
       return cudaErrorInvalidValue;
+    const int S = p.S, kps = p.keys_per_split, ks = k_static, vs = v_static;
     if (p.few_rg == 1)
-      return hd == 64 ? launch_few<64, 1, 6>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
-                      : launch_few<128, 1, 6>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
+      return hd == 64 ? launch_few<64, 1, 6>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, S, kps, ks, vs)
+                      : launch_few<128, 1, 6>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, S, kps, ks, vs);
     if (p.few_rg == 2)
-      return hd == 64 ? launch_few<64, 2, 3>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split)
-                      : launch_few<128, 2, 3>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split);
-    return hd == 64 ? launch_mma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split, k_static, v_static)
-                    : launch_mma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, p.S, p.keys_per_split, k_static, v_static);
+      return hd == 64 ? launch_few<64, 2, 3>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, S, kps, ks, vs)
+                      : launch_few<128, 2, 3>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, S, kps, ks, vs);
+    return hd == 64 ? launch_mma<64>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, S, kps, ks, vs)
+                    : launch_mma<128>(L, tmK, tmV, q, o, scratch, B, a_seq, n, H, Hkv, S, kps, ks, vs);
   }
   const float scale = 1.0f / sqrtf((float)hd);
   dim3 grid((a_seq + TQ - 1) / TQ, H, B);
