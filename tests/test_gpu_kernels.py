@@ -196,6 +196,36 @@ def test_attention(env, case, dtype):
         assert rel_l2(got[b * a:(b + 1) * a], want) < tol
 
 
+@pytest.mark.parametrize("case", [
+    (1, 256, 768, 2, 2, 128),   # tcgen05 kernel, two row tiles per CTA, 12 key tiles
+    (2, 128, 1024, 2, 2, 128),  # tcgen05 kernel, one row tile shared by the two softmax groups, 16 key tiles
+    (1, 200, 640, 3, 1, 64),    # tcgen05 kernel, head_dim 64, grouped heads
+    (1, 64, 768, 2, 2, 128),    # 64-row mma.sync kernel
+    (1, 3, 2048, 2, 2, 128),    # few-rows kernel
+])
+@pytest.mark.parametrize("split", [True, False])
+def test_attention_with_row_maxima_that_keep_growing(env, case, split):
+    """Keys whose norm grows with their index: every later key tile raises the running maxima of the online
+    softmax by many powers of two, so the accumulated output and sum are rescaled again and again (the lazy
+    rescale of the tcgen05 kernel only acts beyond 2^8).  Eq. for attention as in Sec. A.7; the oracle is exact."""
+    torch, dllm = env
+    B, a, n, H, Hkv, hd = case
+    q = synth.random_normal((B * a, H * hd), seed=21, std=8.0)
+    ramp = np.linspace(0.15, 1.0, n, dtype=np.float32)[None, :, None]
+    k = synth.random_normal((B, n, Hkv * hd), seed=22, std=1.3) * ramp
+    v = synth.random_normal((B, n, Hkv * hd), seed=23)
+    q, k, v = (synth.round_to_bf16(t) for t in (q, k, v))
+    got = dllm.attention(*(torch.from_numpy(t).cuda().to(torch.bfloat16) for t in (q, k, v)), B, a, n, H, Hkv, hd,
+                         split=split)
+    got = got.to(torch.float32).cpu().numpy()
+    assert np.isfinite(got).all()
+    for b in range(B):
+        want = O.attention(q[b * a:(b + 1) * a].astype(np.float64).reshape(a, H, hd),
+                           k[b].astype(np.float64).reshape(n, Hkv, hd),
+                           v[b].astype(np.float64).reshape(n, Hkv, hd), Hkv)
+        assert rel_l2(got[b * a:(b + 1) * a], want) < 8e-3
+
+
 @pytest.mark.parametrize("M,N,K", [(520, 7680, 320), (4400, 1280, 200), (300, 20000, 64)])
 def test_gemm_persistent_kernel_is_bit_identical_to_the_one_tile_kernel(env, M, N, K):
     """Unsplit products with more tiles than SMs run on the persistent kernel (one CTA per SM walks through the
